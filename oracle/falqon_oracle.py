@@ -1,0 +1,222 @@
+"""ctypes/numpy front end of the CPU oracle (oracle/falqon_oracle.cpp).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, the smoke check and the
+benchmark's CPU-baseline leg; the product path never touches it.  Argument
+marshalling only -- every arithmetic step is in the C++ file.
+"""
+from __future__ import annotations
+
+import ctypes as C
+
+import numpy as np
+
+from . import build as _build
+
+E4M3, E5M2 = 0, 1
+BF16, F32 = 0, 1
+PER_TENSOR, PER_ROW = 0, 1
+FP8_MAX = {E4M3: 448.0, E5M2: 57344.0}
+
+_lib = C.CDLL(_build.build())
+
+_i64, _f32, _i32 = C.c_int64, C.c_float, C.c_int
+_p = C.c_void_p
+
+_lib.orc_fp8_decode.restype = C.c_double
+_lib.orc_fp8_decode.argtypes = [C.c_uint8, _i32]
+_lib.orc_fp8_encode.restype = C.c_uint8
+_lib.orc_fp8_encode.argtypes = [_f32, _i32]
+_lib.orc_fp8_encode_array.restype = None
+_lib.orc_fp8_encode_array.argtypes = [_p, _i64, _i32, _p]
+_lib.orc_fp8_decode_array.restype = None
+_lib.orc_fp8_decode_array.argtypes = [_p, _i64, _i32, _p]
+_lib.orc_f32_to_bf16.restype = C.c_uint16
+_lib.orc_f32_to_bf16.argtypes = [_f32]
+_lib.orc_quantize.restype = _i32
+_lib.orc_quantize.argtypes = [_p, _i32, _i64, _i64, _i32, _i32, _p, _f32, _p, _p, _p]
+_lib.orc_forward_gemm.restype = _i32
+_lib.orc_forward_gemm.argtypes = [_p, _f32, _p, _f32, _i64, _i64, _i64, _i64, _p, _i64, _p, _i64, _p]
+_lib.orc_forward.restype = _i32
+_lib.orc_forward.argtypes = [_p, _f32, _p, _f32, _i64, _i64, _i64, _i64, _p, _p, _p]
+_lib.orc_dx_gemm.restype = _i32
+_lib.orc_dx_gemm.argtypes = [_p, _f32, _p, _f32, _i64, _i64, _i64, _p, _i64, _p, _i64, _p]
+_lib.orc_db_gemm.restype = _i32
+_lib.orc_db_gemm.argtypes = [_p, _f32, _p, _f32, _i64, _i64, _i64, _p, _i64, _p]
+_lib.orc_proxy_update.restype = _i32
+_lib.orc_proxy_update.argtypes = [_p, _p, _p, _f32, _i64, _i64, _i64, _i64, _p, _p]
+_lib.orc_num_threads.restype = _i32
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(_p)
+
+
+def _c(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _sel(s):
+    if s is None:
+        return None, 0
+    s = _c(s, np.int64)
+    return s, s.size
+
+
+def num_threads() -> int:
+    return int(_lib.orc_num_threads())
+
+
+def decode(code: int, fmt: int) -> float:
+    return float(_lib.orc_fp8_decode(int(code), fmt))
+
+
+def encode(value: float, fmt: int) -> int:
+    return int(_lib.orc_fp8_encode(float(np.float32(value)), fmt))
+
+
+def encode_array(values, fmt: int) -> np.ndarray:
+    v = _c(values, np.float32)
+    out = np.empty(v.shape, dtype=np.uint8)
+    _lib.orc_fp8_encode_array(_ptr(v), v.size, fmt, _ptr(out))
+    return out
+
+
+def decode_array(codes, fmt: int) -> np.ndarray:
+    c = _c(codes, np.uint8)
+    out = np.empty(c.shape, dtype=np.float64)
+    _lib.orc_fp8_decode_array(_ptr(c), c.size, fmt, _ptr(out))
+    return out
+
+
+def f32_to_bf16_bits(value: float) -> int:
+    return int(_lib.orc_f32_to_bf16(float(np.float32(value))))
+
+
+def bf16_bits(x) -> np.ndarray:
+    """fp32 array whose values are bf16-representable -> uint16 bf16 bit patterns (exact)."""
+    x = _c(x, np.float32)
+    bits = x.view(np.uint32)
+    assert not np.any(bits & 0xFFFF), "values are not bf16-representable"
+    return (bits >> 16).astype(np.uint16)
+
+
+def quantize(src, fmt: int, gran: int = PER_TENSOR, scale_in=None, premul: float = 1.0, src_is_bf16_bits=False):
+    """Q_fp8.  src: 2-D fp32 array, or uint16 bf16 bit patterns.  Returns (codes, scale, amax)."""
+    if src_is_bf16_bits:
+        a, dt = _c(src, np.uint16), BF16
+    else:
+        a, dt = _c(src, np.float32), F32
+    rows, cols = a.shape
+    groups = rows if gran == PER_ROW else 1
+    dst = np.empty((rows, cols), dtype=np.uint8)
+    scale_out = np.empty(groups, dtype=np.float32)
+    amax_out = np.empty(groups, dtype=np.float32)
+    s_in = None if scale_in is None else _c(np.atleast_1d(scale_in), np.float32)
+    rc = _lib.orc_quantize(_ptr(a), dt, rows, cols, fmt, gran, _ptr(s_in), float(np.float32(premul)),
+                           _ptr(dst), _ptr(scale_out), _ptr(amax_out))
+    assert rc == 0
+    if gran == PER_TENSOR:
+        return dst, np.float32(scale_out[0]), np.float32(amax_out[0])
+    return dst, scale_out, amax_out
+
+
+def forward_gemm(xq, s_x, wq, s_w, m: int, r: int, tsel=None, fsel=None) -> np.ndarray:
+    """Sampled O_merged: tokens tsel x merged features fsel (None = all), float64."""
+    xq, wq = _c(xq, np.uint8), _c(wq, np.uint8)
+    T, n = xq.shape
+    assert wq.shape == (m + r, n)
+    ts, nt = _sel(tsel)
+    fs, nf = _sel(fsel)
+    out = np.empty((nt if ts is not None else T, nf if fs is not None else m + r), dtype=np.float64)
+    rc = _lib.orc_forward_gemm(_ptr(xq), float(s_x), _ptr(wq), float(s_w), T, m, n, r,
+                               _ptr(ts), nt, _ptr(fs), nf, _ptr(out))
+    assert rc == 0
+    return out
+
+
+def forward(xq, s_x, wq, s_w, m: int, r: int):
+    """Returns (Y float64 [T,m], OA float32 [T,r], amax_oa float32)."""
+    xq, wq = _c(xq, np.uint8), _c(wq, np.uint8)
+    T, n = xq.shape
+    assert wq.shape == (m + r, n)
+    Y = np.empty((T, m), dtype=np.float64)
+    OA = np.empty((T, r), dtype=np.float32)
+    amax = np.zeros(1, dtype=np.float32)
+    rc = _lib.orc_forward(_ptr(xq), float(s_x), _ptr(wq), float(s_w), T, m, n, r, _ptr(Y), _ptr(OA), _ptr(amax))
+    assert rc == 0
+    return Y, OA, np.float32(amax[0])
+
+
+def dx_gemm(gq, s_g, wq, s_w, m: int, tsel=None, csel=None) -> np.ndarray:
+    gq, wq = _c(gq, np.uint8), _c(wq, np.uint8)
+    T = gq.shape[0]
+    n = wq.shape[1]
+    assert gq.shape == (T, m) and wq.shape[0] >= m
+    ts, nt = _sel(tsel)
+    cs, nc = _sel(csel)
+    out = np.empty((nt if ts is not None else T, nc if cs is not None else n), dtype=np.float64)
+    rc = _lib.orc_dx_gemm(_ptr(gq), float(s_g), _ptr(wq), float(s_w), T, m, n, _ptr(ts), nt, _ptr(cs), nc, _ptr(out))
+    assert rc == 0
+    return out
+
+
+def db_gemm(gq, s_g, oaq, s_oa, isel=None) -> np.ndarray:
+    gq, oaq = _c(gq, np.uint8), _c(oaq, np.uint8)
+    T, m = gq.shape
+    r = oaq.shape[1]
+    assert oaq.shape[0] == T
+    is_, ni = _sel(isel)
+    out = np.empty((ni if is_ is not None else m, r), dtype=np.float64)
+    rc = _lib.orc_db_gemm(_ptr(gq), float(s_g), _ptr(oaq), float(s_oa), T, m, r, _ptr(is_), ni, _ptr(out))
+    assert rc == 0
+    return out
+
+
+def proxy_update(wq, dbuf, dB, lr: float, k: int, m: int, r: int):
+    """In place on wq (uint8 [(m+r), n]) and dbuf (float32 [m, r]).  Returns (idx int32 [k], score float32 [m])."""
+    assert wq.dtype == np.uint8 and wq.flags.c_contiguous and wq.shape[0] == m + r
+    assert dbuf.dtype == np.float32 and dbuf.flags.c_contiguous and dbuf.shape == (m, r)
+    n = wq.shape[1]
+    g = None if dB is None else _c(dB, np.float32)
+    idx = np.empty(max(k, 0), dtype=np.int32)
+    score = np.empty(m, dtype=np.float32)
+    rc = _lib.orc_proxy_update(_ptr(wq), _ptr(dbuf), _ptr(g), float(np.float32(lr)), m, n, r, k, _ptr(idx), _ptr(score))
+    if rc != 0:
+        raise ValueError("orc_proxy_update rejected its arguments")
+    return idx, score
+
+
+# ---- whole-layer compositions in the paper's order (each step is one oracle call) ----
+
+def setup_layer(W, A, B, gamma: float):
+    """Alg. 1 without the SVD (A and B are given): W~, s_W = Q(W); A~ = Q(gamma*A; s_W);
+    W~' = [W~; A~]; the initial B is melded by the merge operator itself over all rows
+    (W + BA = W~ + B A~ in the scaled domain), leaving DeltaBuffer = 0."""
+    W = _c(W, np.float32)
+    A = _c(A, np.float32)
+    m, n = W.shape
+    r = A.shape[0]
+    wq_w, s_w, _ = quantize(W, E4M3)
+    aq, _, _ = quantize(A, E4M3, scale_in=s_w, premul=gamma)
+    wq = np.ascontiguousarray(np.concatenate([wq_w, aq], axis=0))
+    dbuf = np.zeros((m, r), dtype=np.float32)
+    if B is not None:
+        dbuf[:] = _c(B, np.float32)
+        proxy_update(wq, dbuf, None, 0.0, m, m, r)
+    return wq, s_w, dbuf
+
+
+def layer_forward(X, wq, s_w, m: int, r: int):
+    """Alg. 2 lines 5-9 for one layer.  Returns dict(xq, s_x, Y, OA, amax_oa)."""
+    xq, s_x, _ = quantize(X, E4M3)
+    Y, OA, amax_oa = forward(xq, s_x, wq, s_w, m, r)
+    return dict(xq=xq, s_x=s_x, Y=Y, OA=OA, amax_oa=amax_oa)
+
+
+def layer_backward(dY, OA, wq, s_w, m: int, r: int):
+    """Alg. 3 line 3 plus the implied input gradient.  Returns dict(gq, s_g, oaq, s_oa, dX, dB)."""
+    gq, s_g, _ = quantize(dY, E5M2)
+    oaq, s_oa, _ = quantize(OA, E4M3)
+    dX = dx_gemm(gq, s_g, wq, s_w, m)
+    dB = db_gemm(gq, s_g, oaq, s_oa)
+    return dict(gq=gq, s_g=s_g, oaq=oaq, s_oa=s_oa, dX=dX, dB=dB)
