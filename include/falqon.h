@@ -1,0 +1,152 @@
+/*
+ * falqon.h -- C ABI of the B200 (sm_100a) melded FP8-LoRA linear layer.
+ *
+ * One linear layer holds its LoRA adapter melded into an FP8 backbone: the E4M3
+ * matrix W~' = [W~; A~] of (m + r) rows by n columns, one fp32 scale s_W, and an
+ * fp32 DeltaBuffer of m x r that collects the optimizer's changes of B.  The four
+ * operations are the quantizer Q_fp8, the melded forward, the backward (input
+ * gradient and reformulated adapter gradient) and the row-wise proxy update.
+ *
+ * Conventions, for every entry point unless it says otherwise
+ *  - Layout: all matrices are dense and row-major.  Paper notation W in R^{m x n},
+ *    x in R^{n x d} maps to W[m][n] and X[T][n] with T = d tokens; O = Wx is Y[T][m].
+ *  - Pointers: everything named "device" is a device pointer to memory the CALLER
+ *    owns (including the workspace); the library allocates no device memory, keeps no
+ *    hidden per-layer state and frees nothing.  The falqon_layer struct itself is a
+ *    HOST struct.  Device pointers must be 16-byte aligned.
+ *  - Shapes: n and m must be multiples of 16 (bulk tensor copies need 16-byte row
+ *    pitches); r must be a multiple of 8 with 8 <= r <= 256; T >= 1.
+ *  - Execution: every call only enqueues work on `stream` and returns; results are
+ *    ready once the stream has drained.  Calls that touch the same layer or the same
+ *    workspace must be ordered on one stream.
+ *  - Errors: the return value is a falqon_status.  Bad arguments are detected on the
+ *    host before anything is launched (nothing is written).  CUDA launch failures map
+ *    to FALQON_ERR_CUDA.  Every device-side wait is bounded; a wait that runs out
+ *    records FALQON_ERR_TIMEOUT in a device status word that
+ *    falqon_last_device_status() returns.  Nothing traps or aborts.
+ *  - Scales follow the reading s = fp8max / amax: quantization multiplies by s,
+ *    de-quantization divides, and a product of two quantized operands is rescaled by
+ *    1 / (s_a * s_b)  (Eq. quantize, Eq. fp8_matmul of the paper).
+ */
+#ifndef FALQON_H_
+#define FALQON_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FALQON_OK = 0,
+  FALQON_ERR_INVALID_ARG = -1,
+  FALQON_ERR_UNSUPPORTED = -2,
+  FALQON_ERR_WORKSPACE = -3,
+  FALQON_ERR_CUDA = -4,
+  FALQON_ERR_TIMEOUT = -5
+} falqon_status;
+
+typedef enum { FALQON_E4M3 = 0, FALQON_E5M2 = 1 } falqon_fp8;        /* max 448 / max 57344 */
+typedef enum { FALQON_BF16 = 0, FALQON_F32 = 1 } falqon_dtype;
+typedef enum { FALQON_PER_TENSOR = 0, FALQON_PER_ROW = 1 } falqon_gran;
+
+/* A CUDA stream handle (the same pointer type as cudaStream_t); NULL is the default stream. */
+typedef struct CUstream_st *falqon_stream;
+
+/* One melded layer (Alg. 1 of the paper builds it; Eq. A_integ defines W~').  Host struct. */
+typedef struct {
+  int64_t m;      /* output features (rows of W)                                         */
+  int64_t n;      /* input features (columns of W)                                       */
+  int64_t r;      /* LoRA rank                                                           */
+  uint8_t *wq;    /* device [(m + r)][n] E4M3 codes; rows m..m+r-1 hold A~ = Q(A; s_W)   */
+  float *s_w;     /* device [1]: the per-tensor scale of W~, shared by A~                */
+  float *dbuf;    /* device [m][r] fp32 DeltaBuffer                                      */
+} falqon_layer;
+
+/* Names of the regions inside the workspace that hold staged intermediates of the last call
+ * (readable by a caller that wants to inspect or reuse them; see falqon_workspace_region). */
+typedef enum {
+  FALQON_WS_XQ = 0,       /* uint8 [T][n]   E4M3 codes of X       (after falqon_melded_forward)  */
+  FALQON_WS_GQ = 1,       /* uint8 [T][m]   E5M2 codes of dY      (after falqon_melded_backward) */
+  FALQON_WS_OAQ_T = 2,    /* uint8 [r16][T16] E4M3 codes of O_A, TRANSPOSED; r16 = r rounded up
+                             to 16, row pitch T16 = T rounded up to 16 (after backward)          */
+  FALQON_WS_SCALES = 3,   /* float [8]: 0 amax(X) 1 s_x 2 amax(dY) 3 s_g 4 amax(O_A) 5 s_OA      */
+  FALQON_WS_SCORE = 4,    /* float [m] row scores sum_j |DeltaBuffer[i][j]| (after proxy update)  */
+  FALQON_WS_DB_PART = 5   /* float [splits][m][r] split partial sums of dB (after backward)      */
+} falqon_ws_region;
+
+/* Host, pure.  Bytes of workspace that the calls below need for a layer of this shape with at
+ * most T_max tokens.  Returns 0 if the shape is not supported. */
+size_t falqon_workspace_bytes(int64_t m, int64_t n, int64_t r, int64_t T_max);
+
+/* Host, pure.  Byte offset and size of a region inside a workspace laid out for (m, n, r, T_max).
+ * Returns FALQON_OK or FALQON_ERR_INVALID_ARG. */
+int falqon_workspace_region(int64_t m, int64_t n, int64_t r, int64_t T_max, falqon_ws_region which,
+                            size_t *offset, size_t *bytes);
+
+/* Q_fp8 (Eq. quantize): absmax -> scale s = fp8max/amax -> saturating round-to-nearest-even cast.
+ *   src        device [rows][cols], bf16 or fp32 (src_dt), dense; cols a multiple of 16
+ *   fmt        E4M3 (weights, activations) or E5M2 (gradients)
+ *   gran       one scale for the tensor, or one per row
+ *   scale_in   device, nullable.  NULL: scale(s) come from the absmax and are written to scale_out.
+ *              Non-NULL ([1] or [rows]): cast with these scale(s) -- A~ = Q(gamma*A; s_W), Eq. A_integ.
+ *   premul     fp32 factor multiplied in first as its own rounded multiply (gamma = alpha/r); 1.0f = none
+ *   dst        device [rows][cols] uint8 codes
+ *   scale_out  device [1] or [rows], nullable when scale_in is given
+ *   amax_out   device [1] or [rows], nullable
+ *   ws         device scratch of at least 256 bytes (used only for per-tensor absmax scaling)
+ * amax == 0 gives scale 1.  NaN inputs are outside the contract. */
+int falqon_quantize(const void *src, falqon_dtype src_dt, int64_t rows, int64_t cols, falqon_fp8 fmt,
+                    falqon_gran gran, const float *scale_in, float premul, uint8_t *dst,
+                    float *scale_out, float *amax_out, void *ws, size_t ws_bytes, falqon_stream stream);
+
+/* Melded forward (Alg. 2 lines 5-9; Eq. o_split):  x~, s_x = Q_e4m3(X);
+ *   [Y | O_A] = x~ * W~'^T / (s_W * s_x)   accumulated in fp32 on the tensor cores.
+ *   X        device [T][n] bf16 or fp32
+ *   Y        device [T][m] bf16 or fp32 (y_dt)
+ *   OA       device [T][r] fp32: the one activation saved for backward
+ *   amax_oa  device [1]: max |O_A|, produced by the same kernel
+ *   s_x_out  device [1], nullable
+ * Leaves x~ and the scales in the workspace (FALQON_WS_XQ, FALQON_WS_SCALES). */
+int falqon_melded_forward(const falqon_layer *L, const void *X, falqon_dtype x_dt, int64_t T, void *Y,
+                          falqon_dtype y_dt, float *OA, float *amax_oa, float *s_x_out, void *ws,
+                          size_t ws_bytes, falqon_stream stream);
+
+/* Backward (Alg. 3 line 3 with Eq. lora_backward_modified, plus the input gradient the chain rule
+ * implies for O = W~ x~ / (s_W s_x)):   g~, s_g = Q_e5m2(dY);   O~_A, s_OA = Q_e4m3(O_A);
+ *   dX = g~ * W~ / (s_W * s_g)            (first m rows of W~' only; skipped when dX is NULL)
+ *   dB = g~^T * O~_A / (s_g * s_OA)       (fp32 [m][r], overwritten)
+ *   dY       device [T][m] bf16 or fp32
+ *   OA       device [T][r] fp32 and amax_oa device [1], as the forward produced them
+ *   dX       device [T][n] bf16 or fp32 (dx_dt), nullable
+ *   s_g_out  device [1], nullable */
+int falqon_melded_backward(const falqon_layer *L, const void *dY, falqon_dtype dy_dt, int64_t T,
+                           const float *OA, const float *amax_oa, void *dX, falqon_dtype dx_dt, float *dB,
+                           float *s_g_out, void *ws, size_t ws_bytes, falqon_stream stream);
+
+/* Row-wise proxy update (Alg. 3 lines 4-6; Eq. update):
+ *   DeltaBuffer <- fma(-lr, dB, DeltaBuffer)          (plain SGD form; skipped when dB is NULL, so a
+ *                                                      caller may run its own optimizer on dbuf)
+ *   score_i = sum_j |DeltaBuffer[i][j]|               (fp32, j ascending)
+ *   idx     = the k rows of largest score, ties to the lowest index, ascending
+ *   W~[i][:] <- sat_rne_e4m3( W~[i][:] + DeltaBuffer[i][:] * A~ )  for i in idx, as an fp32 fma chain
+ *              over j ascending (s_W cancels because A~ carries it); then DeltaBuffer[i][:] <- 0
+ *   idx_out  device [k] int32, nullable.   k == 0: optimizer step and scores only.  k > m: invalid.
+ * Mutates L->wq and L->dbuf.  With dB == NULL, lr == 0, k == m and dbuf preset to an initial B this
+ * is also the operation that melds that B into the backbone at set-up. */
+int falqon_proxy_update(const falqon_layer *L, const float *dB, float lr, int64_t k, int32_t *idx_out,
+                        void *ws, size_t ws_bytes, falqon_stream stream);
+
+/* Synchronizes `stream`, then returns and clears the device status word of the current device:
+ * FALQON_OK, FALQON_ERR_TIMEOUT (a bounded device-side wait ran out; results of that call are
+ * undefined) or FALQON_ERR_CUDA (the synchronize itself failed). */
+int falqon_last_device_status(falqon_stream stream);
+
+/* Host, pure.  Number of kernels the named call launches for this shape (for launch accounting). */
+int falqon_launch_count(const char *entry_point, int64_t m, int64_t n, int64_t r, int64_t T, int64_t k);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FALQON_H_ */

@@ -1,0 +1,208 @@
+"""ctypes binding of libfalqon.so: the same names as the C ABI in include/falqon.h.
+
+Argument marshalling only.  PyTorch supplies device memory (torch.empty) and the
+current CUDA stream; every step of the path runs in the library's kernels.  There
+is no fallback: importing this module raises if the library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfalqon.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+E4M3, E5M2 = 0, 1
+BF16, F32 = 0, 1
+PER_TENSOR, PER_ROW = 0, 1
+WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE, WS_DB_PART = range(6)
+
+EXPORTS = ["falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
+           "falqon_melded_backward", "falqon_proxy_update", "falqon_last_device_status", "falqon_launch_count"]
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2510_24061_b200.build` "
+                      "(there is no non-CUDA fallback)")
+lib = C.CDLL(LIB_PATH)
+
+
+class falqon_layer(C.Structure):
+    _fields_ = [("m", C.c_int64), ("n", C.c_int64), ("r", C.c_int64),
+                ("wq", C.c_void_p), ("s_w", C.c_void_p), ("dbuf", C.c_void_p)]
+
+
+_i64, _sz, _p, _f, _i = C.c_int64, C.c_size_t, C.c_void_p, C.c_float, C.c_int
+lib.falqon_workspace_bytes.restype = _sz
+lib.falqon_workspace_bytes.argtypes = [_i64, _i64, _i64, _i64]
+lib.falqon_workspace_region.restype = _i
+lib.falqon_workspace_region.argtypes = [_i64, _i64, _i64, _i64, _i, C.POINTER(_sz), C.POINTER(_sz)]
+lib.falqon_quantize.restype = _i
+lib.falqon_quantize.argtypes = [_p, _i, _i64, _i64, _i, _i, _p, _f, _p, _p, _p, _p, _sz, _p]
+lib.falqon_melded_forward.restype = _i
+lib.falqon_melded_forward.argtypes = [C.POINTER(falqon_layer), _p, _i, _i64, _p, _i, _p, _p, _p, _p, _sz, _p]
+lib.falqon_melded_backward.restype = _i
+lib.falqon_melded_backward.argtypes = [C.POINTER(falqon_layer), _p, _i, _i64, _p, _p, _p, _i, _p, _p, _p, _sz, _p]
+lib.falqon_proxy_update.restype = _i
+lib.falqon_proxy_update.argtypes = [C.POINTER(falqon_layer), _p, _f, _i64, _p, _p, _sz, _p]
+lib.falqon_last_device_status.restype = _i
+lib.falqon_last_device_status.argtypes = [_p]
+lib.falqon_launch_count.restype = _i
+lib.falqon_launch_count.argtypes = [C.c_char_p, _i64, _i64, _i64, _i64, _i64]
+
+
+class FalqonError(RuntimeError):
+    def __init__(self, call: str, status: int):
+        super().__init__(f"{call} returned status {status}")
+        self.status = status
+
+
+def _check(call: str, status: int):
+    if status != OK:
+        raise FalqonError(call, status)
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+class Layer:
+    """Owns the device tensors of one melded layer and the host struct that points at them."""
+
+    def __init__(self, wq: torch.Tensor, s_w: torch.Tensor, dbuf: torch.Tensor, r: int):
+        assert wq.dtype == torch.uint8 and wq.is_contiguous() and dbuf.dtype == torch.float32 and dbuf.is_contiguous()
+        self.wq, self.s_w, self.dbuf = wq, s_w, dbuf
+        self.m, self.n, self.r = wq.shape[0] - r, wq.shape[1], r
+        self.c = falqon_layer(self.m, self.n, self.r, wq.data_ptr(), s_w.data_ptr(), dbuf.data_ptr())
+        self._ws = None
+
+    def workspace(self, T: int) -> torch.Tensor:
+        need = workspace_bytes(self.m, self.n, self.r, T)
+        if need == 0:
+            raise FalqonError("falqon_workspace_bytes", ERR_INVALID_ARG)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.wq.device)
+        return self._ws
+
+
+def workspace_bytes(m: int, n: int, r: int, T: int) -> int:
+    return int(lib.falqon_workspace_bytes(m, n, r, T))
+
+
+def workspace_region(m: int, n: int, r: int, T: int, which: int):
+    off, size = _sz(), _sz()
+    _check("falqon_workspace_region", lib.falqon_workspace_region(m, n, r, T, which, C.byref(off), C.byref(size)))
+    return off.value, size.value
+
+
+def ws_view(layer: Layer, ws: torch.Tensor, T: int, which: int) -> torch.Tensor:
+    off, size = workspace_region(layer.m, layer.n, layer.r, T, which)
+    return ws[off:off + size]
+
+
+def launch_count(entry_point: str, m=0, n=0, r=0, T=0, k=0) -> int:
+    return int(lib.falqon_launch_count(entry_point.encode(), m, n, r, T, k))
+
+
+def last_device_status() -> int:
+    return int(lib.falqon_last_device_status(_stream()))
+
+
+def quantize(src: torch.Tensor, fmt: int, gran: int = PER_TENSOR, scale_in: torch.Tensor | None = None,
+             premul: float = 1.0, want_amax: bool = True, dst: torch.Tensor | None = None):
+    """falqon_quantize.  Returns (codes uint8 [rows, cols], scale fp32 [1] or [rows], amax or None)."""
+    assert src.dim() == 2 and src.is_contiguous()
+    rows, cols = src.shape
+    groups = rows if gran == PER_ROW else 1
+    dev = src.device
+    if dst is None:
+        dst = torch.empty((rows, cols), dtype=torch.uint8, device=dev)
+    scale_out = torch.empty(groups, dtype=torch.float32, device=dev)
+    amax_out = torch.empty(groups, dtype=torch.float32, device=dev) if want_amax else None
+    ws = torch.empty(256, dtype=torch.uint8, device=dev)
+    _check("falqon_quantize", lib.falqon_quantize(_ptr(src), _dt(src), rows, cols, fmt, gran, _ptr(scale_in), premul,
+                                                  _ptr(dst), _ptr(scale_out), _ptr(amax_out), _ptr(ws), ws.numel(),
+                                                  _stream()))
+    return dst, scale_out, amax_out
+
+
+def melded_forward(layer: Layer, X: torch.Tensor, y_dtype=torch.bfloat16, ws: torch.Tensor | None = None, out=None):
+    """falqon_melded_forward.  Returns (Y [T, m], OA fp32 [T, r], amax_oa fp32 [1], s_x fp32 [1])."""
+    assert X.dim() == 2 and X.is_contiguous() and X.shape[1] == layer.n
+    T = X.shape[0]
+    dev = X.device
+    ws = layer.workspace(T) if ws is None else ws
+    if out is None:
+        Y = torch.empty((T, layer.m), dtype=y_dtype, device=dev)
+        OA = torch.empty((T, layer.r), dtype=torch.float32, device=dev)
+        amax_oa = torch.empty(1, dtype=torch.float32, device=dev)
+        s_x = torch.empty(1, dtype=torch.float32, device=dev)
+    else:
+        Y, OA, amax_oa, s_x = out
+    _check("falqon_melded_forward", lib.falqon_melded_forward(C.byref(layer.c), _ptr(X), _dt(X), T, _ptr(Y), _dt(Y),
+                                                              _ptr(OA), _ptr(amax_oa), _ptr(s_x), _ptr(ws), ws.numel(),
+                                                              _stream()))
+    return Y, OA, amax_oa, s_x
+
+
+def melded_backward(layer: Layer, dY: torch.Tensor, OA: torch.Tensor, amax_oa: torch.Tensor, need_dx: bool = True,
+                    dx_dtype=torch.bfloat16, ws: torch.Tensor | None = None, out=None):
+    """falqon_melded_backward.  Returns (dX [T, n] or None, dB fp32 [m, r], s_g fp32 [1])."""
+    assert dY.dim() == 2 and dY.is_contiguous() and dY.shape[1] == layer.m
+    T = dY.shape[0]
+    dev = dY.device
+    ws = layer.workspace(T) if ws is None else ws
+    if out is None:
+        dX = torch.empty((T, layer.n), dtype=dx_dtype, device=dev) if need_dx else None
+        dB = torch.empty((layer.m, layer.r), dtype=torch.float32, device=dev)
+        s_g = torch.empty(1, dtype=torch.float32, device=dev)
+    else:
+        dX, dB, s_g = out
+    dx_dt = _dt(dX) if dX is not None else BF16
+    _check("falqon_melded_backward", lib.falqon_melded_backward(C.byref(layer.c), _ptr(dY), _dt(dY), T, _ptr(OA),
+                                                                _ptr(amax_oa), _ptr(dX), dx_dt, _ptr(dB), _ptr(s_g),
+                                                                _ptr(ws), ws.numel(), _stream()))
+    return dX, dB, s_g
+
+
+def proxy_update(layer: Layer, dB: torch.Tensor | None, lr: float, k: int, ws: torch.Tensor | None = None,
+                 idx_out: torch.Tensor | None = None):
+    """falqon_proxy_update (in place on layer.wq / layer.dbuf).  Returns idx int32 [k] ascending."""
+    ws = layer.workspace(1) if ws is None else ws
+    if idx_out is None and 0 < k <= layer.m:
+        idx_out = torch.empty(k, dtype=torch.int32, device=layer.wq.device)
+    _check("falqon_proxy_update", lib.falqon_proxy_update(C.byref(layer.c), _ptr(dB), lr, k, _ptr(idx_out), _ptr(ws),
+                                                          ws.numel(), _stream()))
+    return idx_out
+
+
+def setup_layer(W: torch.Tensor, A: torch.Tensor, B: torch.Tensor | None, gamma: float) -> Layer:
+    """Builds a melded layer from W [m, n], A [r, n] and an optional initial B [m, r] (all on the device):
+    W~, s_W = Q(W); A~ = Q(gamma*A; s_W); W~' = [W~; A~]; then melds B by the merge operator over all rows
+    (dbuf := B, falqon_proxy_update with dB = NULL, k = m), which leaves DeltaBuffer = 0."""
+    m, n = W.shape
+    r = A.shape[0]
+    dev = W.device
+    wq = torch.empty((m + r, n), dtype=torch.uint8, device=dev)
+    _, s_w, _ = quantize(W.contiguous(), E4M3, dst=wq[:m])
+    quantize(A.contiguous(), E4M3, scale_in=s_w, premul=gamma, want_amax=False, dst=wq[m:])
+    dbuf = torch.zeros((m, r), dtype=torch.float32, device=dev)
+    layer = Layer(wq, s_w, dbuf, r)
+    if B is not None:
+        dbuf.copy_(B.to(torch.float32))
+        proxy_update(layer, None, 0.0, m)
+    return layer

@@ -1,0 +1,269 @@
+// The C ABI of libfalqon (see include/falqon.h): argument validation, workspace layout, and the
+// sequence of kernel launches behind each entry point.  No device memory is allocated here.
+#include <cstring>
+
+#include "../../include/falqon.h"
+#include "internal.h"
+
+namespace falqon {
+namespace {
+
+__device__ int g_status_word;  // written by kernels whose bounded waits run out
+
+constexpr int kMaxDevices = 64;
+int* status_ptr() {
+  static int* ptrs[kMaxDevices] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  if (ptrs[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+    ptrs[dev] = static_cast<int*>(p);
+  }
+  return ptrs[dev];
+}
+
+struct WorkspaceLayout {
+  size_t scales, act8, oaq_t, db_part, score, sel_idx, total;
+  size_t act8_bytes, oaq_t_bytes, db_part_bytes, score_bytes, sel_idx_bytes;
+  int64_t r16, t16;
+  int splits;
+};
+
+constexpr size_t kHeaderBytes = 1024;
+
+bool shape_ok(int64_t m, int64_t n, int64_t r) {
+  return m >= 16 && n >= 16 && m % 16 == 0 && n % 16 == 0 && r >= 8 && r <= 256 && r % 8 == 0 &&
+         m < (1ll << 30) && n < (1ll << 30);
+}
+
+bool make_layout(int64_t m, int64_t n, int64_t r, int64_t T, WorkspaceLayout* w) {
+  if (!shape_ok(m, n, r) || T < 1 || T >= (1ll << 30)) return false;
+  w->r16 = round_up(r, 16);
+  w->t16 = round_up(T, 16);
+  w->splits = gemm_k_splits_for_db(m, T);
+  w->act8_bytes = static_cast<size_t>(T) * static_cast<size_t>(m > n ? m : n);
+  w->oaq_t_bytes = static_cast<size_t>(w->r16) * static_cast<size_t>(w->t16);
+  w->db_part_bytes = static_cast<size_t>(w->splits) * m * r * sizeof(float);
+  w->score_bytes = static_cast<size_t>(m) * sizeof(float);
+  w->sel_idx_bytes = static_cast<size_t>(m) * sizeof(int32_t);
+  size_t off = 0;
+  w->scales = off; off += kHeaderBytes;
+  w->score = off; off += round_up(w->score_bytes, 1024);      // token-independent regions first, so the
+  w->sel_idx = off; off += round_up(w->sel_idx_bytes, 1024);  // proxy update finds them for any T_max
+  w->act8 = off; off += round_up(w->act8_bytes, 1024);
+  w->oaq_t = off; off += round_up(w->oaq_t_bytes, 1024);
+  w->db_part = off; off += round_up(w->db_part_bytes, 1024);
+  w->total = off;
+  return true;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+inline bool dtype_ok(int dt) { return dt == FALQON_BF16 || dt == FALQON_F32; }
+
+bool layer_ok(const falqon_layer* L) {
+  return L != nullptr && shape_ok(L->m, L->n, L->r) && L->wq != nullptr && L->s_w != nullptr && L->dbuf != nullptr &&
+         aligned16(L->wq) && aligned16(L->dbuf);
+}
+
+#define FALQON_CUDA(expr)                                   \
+  do {                                                      \
+    cudaError_t e__ = (expr);                               \
+    if (e__ != cudaSuccess) return FALQON_ERR_CUDA;         \
+  } while (0)
+
+}  // namespace
+}  // namespace falqon
+
+using namespace falqon;
+
+extern "C" {
+
+size_t falqon_workspace_bytes(int64_t m, int64_t n, int64_t r, int64_t T_max) {
+  WorkspaceLayout w;
+  if (!make_layout(m, n, r, T_max, &w)) return 0;
+  return w.total;
+}
+
+int falqon_workspace_region(int64_t m, int64_t n, int64_t r, int64_t T_max, falqon_ws_region which, size_t* offset,
+                            size_t* bytes) {
+  WorkspaceLayout w;
+  if (offset == nullptr || bytes == nullptr || !make_layout(m, n, r, T_max, &w)) return FALQON_ERR_INVALID_ARG;
+  switch (which) {
+    case FALQON_WS_XQ: *offset = w.act8; *bytes = static_cast<size_t>(T_max) * n; break;
+    case FALQON_WS_GQ: *offset = w.act8; *bytes = static_cast<size_t>(T_max) * m; break;
+    case FALQON_WS_OAQ_T: *offset = w.oaq_t; *bytes = w.oaq_t_bytes; break;
+    case FALQON_WS_SCALES: *offset = w.scales; *bytes = 8 * sizeof(float); break;
+    case FALQON_WS_SCORE: *offset = w.score; *bytes = w.score_bytes; break;
+    case FALQON_WS_DB_PART: *offset = w.db_part; *bytes = w.db_part_bytes; break;
+    default: return FALQON_ERR_INVALID_ARG;
+  }
+  return FALQON_OK;
+}
+
+int falqon_quantize(const void* src, falqon_dtype src_dt, int64_t rows, int64_t cols, falqon_fp8 fmt, falqon_gran gran,
+                    const float* scale_in, float premul, uint8_t* dst, float* scale_out, float* amax_out, void* ws,
+                    size_t ws_bytes, falqon_stream stream) {
+  if (src == nullptr || dst == nullptr || rows < 1 || cols < 16 || cols % 16 != 0 || !dtype_ok(src_dt) ||
+      (fmt != FALQON_E4M3 && fmt != FALQON_E5M2) || (gran != FALQON_PER_TENSOR && gran != FALQON_PER_ROW) ||
+      !aligned16(src) || !aligned16(dst) || !(premul == premul) || rows * cols >= (1ll << 40))
+    return FALQON_ERR_INVALID_ARG;
+  if (scale_in == nullptr && scale_out == nullptr) return FALQON_ERR_INVALID_ARG;
+  if (gran == FALQON_PER_ROW) {
+    if (rows >= (1ll << 31)) return FALQON_ERR_INVALID_ARG;
+    FALQON_CUDA(launch_quantize_per_row(src, src_dt, rows, cols, fmt, premul, scale_in, dst, scale_out, amax_out, stream));
+    return FALQON_OK;
+  }
+  const int64_t count = rows * cols;
+  if (scale_in != nullptr) {
+    if (amax_out != nullptr) {
+      if (ws == nullptr || ws_bytes < 256) return FALQON_ERR_WORKSPACE;
+      FALQON_CUDA(launch_absmax(src, src_dt, count, premul, static_cast<uint32_t*>(ws), stream));
+      FALQON_CUDA(cudaMemcpyAsync(amax_out, ws, sizeof(float), cudaMemcpyDeviceToDevice, stream));
+    }
+    FALQON_CUDA(launch_cast_per_tensor(src, src_dt, count, fmt, premul, scale_in, false, dst, scale_out, nullptr, stream));
+    return FALQON_OK;
+  }
+  if (ws == nullptr || ws_bytes < 256 || !aligned16(ws)) return FALQON_ERR_WORKSPACE;
+  FALQON_CUDA(launch_absmax(src, src_dt, count, premul, static_cast<uint32_t*>(ws), stream));
+  FALQON_CUDA(launch_cast_per_tensor(src, src_dt, count, fmt, premul, static_cast<const float*>(ws), true, dst, scale_out,
+                                     amax_out, stream));
+  return FALQON_OK;
+}
+
+int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_dt, int64_t T, void* Y, falqon_dtype y_dt,
+                          float* OA, float* amax_oa, float* s_x_out, void* ws, size_t ws_bytes, falqon_stream stream) {
+  if (!layer_ok(L) || X == nullptr || Y == nullptr || OA == nullptr || amax_oa == nullptr || T < 1 || !dtype_ok(x_dt) ||
+      !dtype_ok(y_dt) || !aligned16(X) || !aligned16(Y) || !aligned16(OA))
+    return FALQON_ERR_INVALID_ARG;
+  WorkspaceLayout w;
+  if (!make_layout(L->m, L->n, L->r, T, &w)) return FALQON_ERR_INVALID_ARG;
+  if (ws == nullptr || !aligned16(ws) || ws_bytes < w.total) return FALQON_ERR_WORKSPACE;
+  int* status = status_ptr();
+  if (status == nullptr) return FALQON_ERR_CUDA;
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  float* scales = reinterpret_cast<float*>(base + w.scales);
+  uint8_t* xq = base + w.act8;
+  const int64_t m = L->m, n = L->n, r = L->r;
+
+  // S1: x~, s_x = Q_e4m3(X)
+  FALQON_CUDA(launch_absmax(X, x_dt, T * n, 1.0f, reinterpret_cast<uint32_t*>(scales + 0), stream));
+  FALQON_CUDA(launch_cast_per_tensor(X, x_dt, T * n, kE4M3, 1.0f, scales + 0, true, xq, scales + 1, nullptr, stream));
+  if (s_x_out != nullptr)
+    FALQON_CUDA(cudaMemcpyAsync(s_x_out, scales + 1, sizeof(float), cudaMemcpyDeviceToDevice, stream));
+  // S2: [Y | O_A] = x~ W~'^T / (s_W s_x), amax(O_A) from the epilogue
+  FALQON_CUDA(cudaMemsetAsync(amax_oa, 0, sizeof(float), stream));
+  GemmProblem g{};
+  g.M = T; g.N = m + r; g.K = n;
+  g.a = xq; g.lda = n; g.a_mn_major = false; g.a_fmt = kE4M3;
+  g.b = L->wq; g.ldb = n; g.b_mn_major = false; g.b_fmt = kE4M3;
+  g.block_n = 256; g.k_splits = 1;
+  g.c0 = Y; g.ldc0 = m; g.c0_dt = y_dt; g.n_split = m; g.c0_split_stride = 0;
+  g.c1 = OA; g.ldc1 = r; g.amax1_bits = reinterpret_cast<uint32_t*>(amax_oa);
+  g.scale_a = scales + 1; g.scale_b = L->s_w;
+  g.status = status;
+  FALQON_CUDA(launch_gemm_fp8(g, stream));
+  return FALQON_OK;
+}
+
+int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, int64_t T, const float* OA,
+                           const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, float* s_g_out, void* ws,
+                           size_t ws_bytes, falqon_stream stream) {
+  if (!layer_ok(L) || dY == nullptr || OA == nullptr || amax_oa == nullptr || dB == nullptr || T < 1 || !dtype_ok(dy_dt) ||
+      !dtype_ok(dx_dt) || !aligned16(dY) || !aligned16(OA) || !aligned16(dB) || (dX != nullptr && !aligned16(dX)))
+    return FALQON_ERR_INVALID_ARG;
+  WorkspaceLayout w;
+  if (!make_layout(L->m, L->n, L->r, T, &w)) return FALQON_ERR_INVALID_ARG;
+  if (ws == nullptr || !aligned16(ws) || ws_bytes < w.total) return FALQON_ERR_WORKSPACE;
+  int* status = status_ptr();
+  if (status == nullptr) return FALQON_ERR_CUDA;
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  float* scales = reinterpret_cast<float*>(base + w.scales);
+  uint8_t* gq = base + w.act8;
+  uint8_t* oaq_t = base + w.oaq_t;
+  float* part = reinterpret_cast<float*>(base + w.db_part);
+  const int64_t m = L->m, n = L->n, r = L->r;
+
+  // S3: g~, s_g = Q_e5m2(dY)
+  FALQON_CUDA(launch_absmax(dY, dy_dt, T * m, 1.0f, reinterpret_cast<uint32_t*>(scales + 2), stream));
+  FALQON_CUDA(launch_cast_per_tensor(dY, dy_dt, T * m, kE5M2, 1.0f, scales + 2, true, gq, scales + 3, nullptr, stream));
+  if (s_g_out != nullptr)
+    FALQON_CUDA(cudaMemcpyAsync(s_g_out, scales + 3, sizeof(float), cudaMemcpyDeviceToDevice, stream));
+  // S5a: O~_A, s_OA = Q_e4m3(O_A), written transposed for the dB product
+  FALQON_CUDA(cudaMemcpyAsync(scales + 4, amax_oa, sizeof(float), cudaMemcpyDeviceToDevice, stream));
+  FALQON_CUDA(launch_quantize_oa_transposed(OA, amax_oa, T, r, w.r16, w.t16, oaq_t, scales + 5, stream));
+  // S4: dX = g~ W~ / (s_W s_g)   (contraction over the m output channels; W~ read MN-major)
+  if (dX != nullptr) {
+    GemmProblem g{};
+    g.M = T; g.N = n; g.K = m;
+    g.a = gq; g.lda = m; g.a_mn_major = false; g.a_fmt = kE5M2;
+    g.b = L->wq; g.ldb = n; g.b_mn_major = true; g.b_fmt = kE4M3;
+    g.block_n = 256; g.k_splits = 1;
+    g.c0 = dX; g.ldc0 = n; g.c0_dt = dx_dt; g.n_split = n; g.c0_split_stride = 0;
+    g.c1 = nullptr; g.ldc1 = 0; g.amax1_bits = nullptr;
+    g.scale_a = scales + 3; g.scale_b = L->s_w;
+    g.status = status;
+    FALQON_CUDA(launch_gemm_fp8(g, stream));
+  }
+  // S5b: dB = g~^T O~_A / (s_g s_OA)   (contraction over tokens, split into slabs, fixed-order reduce)
+  {
+    GemmProblem g{};
+    g.M = m; g.N = r; g.K = T;
+    g.a = gq; g.lda = m; g.a_mn_major = true; g.a_fmt = kE5M2;
+    g.b = oaq_t; g.ldb = w.t16; g.b_mn_major = false; g.b_fmt = kE4M3;
+    g.block_n = static_cast<int>(w.r16); g.k_splits = w.splits;
+    g.c0 = part; g.ldc0 = r; g.c0_dt = kF32; g.n_split = r; g.c0_split_stride = m * r;
+    g.c1 = nullptr; g.ldc1 = 0; g.amax1_bits = nullptr;
+    g.scale_a = nullptr; g.scale_b = nullptr;
+    g.status = status;
+    FALQON_CUDA(launch_gemm_fp8(g, stream));
+    FALQON_CUDA(launch_reduce_db(part, w.splits, m * r, scales + 3, scales + 5, dB, stream));
+  }
+  return FALQON_OK;
+}
+
+int falqon_proxy_update(const falqon_layer* L, const float* dB, float lr, int64_t k, int32_t* idx_out, void* ws,
+                        size_t ws_bytes, falqon_stream stream) {
+  if (!layer_ok(L) || k < 0 || k > L->m || !(lr == lr) || (dB != nullptr && !aligned16(dB)))
+    return FALQON_ERR_INVALID_ARG;
+  WorkspaceLayout w;
+  if (!make_layout(L->m, L->n, L->r, 1, &w)) return FALQON_ERR_INVALID_ARG;  // score / index regions do not depend on T
+  if (ws == nullptr || !aligned16(ws) || ws_bytes < w.total) return FALQON_ERR_WORKSPACE;
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  float* score = reinterpret_cast<float*>(base + w.score);
+  int32_t* sel = reinterpret_cast<int32_t*>(base + w.sel_idx);
+  const int64_t m = L->m, n = L->n, r = L->r;
+  FALQON_CUDA(launch_sgd_score(L->dbuf, dB, lr, m, r, score, stream));
+  if (k > 0) {
+    FALQON_CUDA(launch_topk(score, m, k, sel, nullptr, stream));
+    FALQON_CUDA(launch_merge_rows(L->wq, L->dbuf, sel, k, m, n, r, stream));
+    if (idx_out != nullptr)
+      FALQON_CUDA(cudaMemcpyAsync(idx_out, sel, static_cast<size_t>(k) * sizeof(int32_t), cudaMemcpyDeviceToDevice, stream));
+  }
+  return FALQON_OK;
+}
+
+int falqon_last_device_status(falqon_stream stream) {
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return FALQON_ERR_CUDA;
+  int* p = status_ptr();
+  if (p == nullptr) return FALQON_ERR_CUDA;
+  int v = 0;
+  if (cudaMemcpy(&v, p, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FALQON_ERR_CUDA;
+  if (v != 0) {
+    const int zero = 0;
+    if (cudaMemcpy(p, &zero, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return FALQON_ERR_CUDA;
+  }
+  return v;
+}
+
+int falqon_launch_count(const char* entry_point, int64_t m, int64_t n, int64_t r, int64_t T, int64_t k) {
+  (void)m; (void)n; (void)r; (void)T;
+  if (entry_point == nullptr) return 0;
+  if (std::strcmp(entry_point, "falqon_quantize") == 0) return 2;           // absmax, cast
+  if (std::strcmp(entry_point, "falqon_melded_forward") == 0) return 3;     // absmax, cast, GEMM
+  if (std::strcmp(entry_point, "falqon_melded_backward") == 0) return 6;    // absmax, cast, O_A cast, dX, dB, reduce
+  if (std::strcmp(entry_point, "falqon_proxy_update") == 0) return k > 0 ? 4 : 1;  // score, top-k, merge, clear
+  return 0;
+}
+
+}  // extern "C"

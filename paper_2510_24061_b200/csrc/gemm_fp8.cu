@@ -1,0 +1,390 @@
+// FP8 GEMM on the 5th-generation tensor cores (tcgen05.mma kind::f8f6f4, fp32 accumulators in
+// tensor memory), operands staged by TMA into 128-byte-swizzled shared-memory tiles.
+//
+//   D[M][N] = A[M][K] * B[N][K]^T      A, B: E4M3 or E5M2 codes (mixed allowed), D: fp32 in TMEM
+//
+// One persistent CTA per SM walks a static list of 128 x block_n output tiles.  Warp roles:
+//   warp 0      TMA producer (one lane): fills a ring of (A,B) stages, signalled through mbarriers
+//   warp 1      allocates TMEM; one lane issues the MMAs and commits them to the barriers
+//   warps 2..5  epilogue: tcgen05.ld the accumulator, rescale by 1/(s_a*s_b), store
+// The accumulator is double buffered (2 x 256 TMEM columns), so the epilogue of tile i overlaps the
+// main loop of tile i+1.  Either operand may be K-major (rows along K) or MN-major (rows along M/N):
+// the melded forward reads both K-major, the input gradient reads W~ MN-major (no transposed copy of
+// the backbone exists), the adapter gradient reads the output gradient MN-major.
+// Every mbarrier wait is bounded; on a timeout the CTA records it, drains and frees its TMEM.
+#include <cuda.h>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace falqon {
+namespace {
+
+constexpr int kGemmThreads = 192;
+constexpr int kBlockM = 128;
+constexpr int kBlockKBytes = 128;          // one 128-byte swizzle row of FP8 = 128 elements of K
+constexpr int kUmmaK = 32;                 // K per tcgen05.mma for 8-bit operands
+constexpr uint32_t kATileBytes = kBlockM * kBlockKBytes;   // 16 KB
+constexpr uint32_t kMnChunkBytes = 128 * kBlockKBytes;     // a 128(K) x 128(M/N) chunk of an MN-major tile
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kAccCols = 256;
+constexpr int kMaxStages = 8;
+constexpr uint32_t kSmemBudget = 227 * 1024;
+constexpr uint32_t kBarrierBytes = 256;
+
+struct GemmParams {
+  int M, N, K;
+  int m_tiles, n_tiles, k_splits;
+  int kblocks_total, kblocks_per_split;
+  int block_n;
+  int num_stages;
+  uint32_t idesc;
+  // epilogue
+  void* c0; long long ldc0; int c0_dt; int n_split; long long c0_split_stride;
+  float* c1; long long ldc1; uint32_t* amax1_bits;
+  const float* scale_a; const float* scale_b;
+  int* status;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+template <bool kAMn, bool kBMn>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t smem_base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - raw_addr);
+
+  const uint32_t b_tile_bytes = static_cast<uint32_t>(p.block_n) * kBlockKBytes;
+  const uint32_t stage_bytes = kATileBytes + b_tile_bytes;
+  const int S = p.num_stages;
+  const uint32_t bars = smem_base + static_cast<uint32_t>(S) * stage_bytes;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (S + s); };
+  auto tmem_full_bar = [&](int a) { return bars + 8u * (2 * S + a); };
+  auto tmem_empty_bar = [&](int a) { return bars + 8u * (2 * S + 2 + a); };
+  const uint32_t slot_off = static_cast<uint32_t>(S) * stage_bytes + 8u * (2 * S + 4);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + slot_off);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    prefetch_tensor_map(&tmap_a);
+    prefetch_tensor_map(&tmap_b);
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tmem_full_bar(a), 1);
+      mbar_init(tmem_empty_bar(a), 4);
+    }
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_base + slot_off, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int tiles_per_split = p.m_tiles * p.n_tiles;
+  const int total_tiles = tiles_per_split * p.k_splits;
+  bool aborted = false;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int tile = blockIdx.x; tile < total_tiles && !aborted; tile += gridDim.x) {
+        const int split = tile / tiles_per_split;
+        const int rem = tile - split * tiles_per_split;
+        const int n_idx = rem / p.m_tiles;
+        const int m_idx = rem - n_idx * p.m_tiles;
+        const int kb_begin = split * p.kblocks_per_split;
+        const int kb_end = min(kb_begin + p.kblocks_per_split, p.kblocks_total);
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status)) { aborted = true; break; }
+          const uint32_t fb = full_bar(stage);
+          mbar_expect_tx(fb, stage_bytes);
+          const uint32_t a_dst = smem_base + static_cast<uint32_t>(stage) * stage_bytes;
+          const uint32_t b_dst = a_dst + kATileBytes;
+          if (!kAMn) tma_load_2d(a_dst, &tmap_a, fb, kb * kBlockKBytes, m_idx * kBlockM);
+          else       tma_load_2d(a_dst, &tmap_a, fb, m_idx * kBlockM, kb * kBlockKBytes);
+          if (!kBMn) {
+            tma_load_2d(b_dst, &tmap_b, fb, kb * kBlockKBytes, n_idx * p.block_n);
+          } else {
+            for (int c = 0; c < p.block_n / 128; ++c)
+              tma_load_2d(b_dst + c * kMnChunkBytes, &tmap_b, fb, n_idx * p.block_n + c * 128, kb * kBlockKBytes);
+          }
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      for (int tile = blockIdx.x; tile < total_tiles && !aborted; tile += gridDim.x) {
+        const int split = tile / tiles_per_split;
+        const int kb_begin = split * p.kblocks_per_split;
+        const int kb_end = min(kb_begin + p.kblocks_per_split, p.kblocks_total);
+        if (!mbar_wait(tmem_empty_bar(acc), acc_phase ^ 1u, p.status)) { aborted = true; break; }
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * kAccCols;
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, p.status)) { aborted = true; break; }
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_base + static_cast<uint32_t>(stage) * stage_bytes;
+          const uint32_t b_addr = a_addr + kATileBytes;
+#pragma unroll
+          for (int k = 0; k < kBlockKBytes / kUmmaK; ++k) {
+            const uint64_t adesc = kAMn ? make_smem_desc(a_addr + k * (kUmmaK * 128), kMnChunkBytes, 1024)
+                                        : make_smem_desc(a_addr + k * kUmmaK, 16, 1024);
+            const uint64_t bdesc = kBMn ? make_smem_desc(b_addr + k * (kUmmaK * 128), kMnChunkBytes, 1024)
+                                        : make_smem_desc(b_addr + k * kUmmaK, 16, 1024);
+            umma_f8(d_tmem, adesc, bdesc, p.idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
+          }
+          umma_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+        if (aborted) break;
+        umma_commit(tmem_full_bar(acc));  // accumulator complete
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int quad = warp & 3;  // TMEM lanes [32*quad, 32*quad+32) belong to this warp
+    const bool rescale = p.scale_a != nullptr;
+    const float inv = rescale ? 1.0f / (__ldg(p.scale_a) * __ldg(p.scale_b)) : 1.0f;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    uint32_t amax_bits = 0;
+    for (int tile = blockIdx.x; tile < total_tiles && !aborted; tile += gridDim.x) {
+      const int split = tile / tiles_per_split;
+      const int rem = tile - split * tiles_per_split;
+      const int n_idx = rem / p.m_tiles;
+      const int m_idx = rem - n_idx * p.m_tiles;
+      if (!mbar_wait(tmem_full_bar(acc), acc_phase, p.status)) { aborted = true; break; }
+      tc_fence_after_sync();
+      const int row = m_idx * kBlockM + quad * 32 + lane;
+      const bool row_ok = row < p.M;
+      const uint32_t t_row = tmem_base + static_cast<uint32_t>(acc) * kAccCols + (static_cast<uint32_t>(quad * 32) << 16);
+      const int n0 = n_idx * p.block_n;
+      for (int c = 0; c < p.block_n; c += 32) {
+        if (n0 + c >= p.N) break;  // warp-uniform
+        uint32_t v[32];
+        __syncwarp();
+        tmem_ld_32x32b_x32(t_row + c, v);
+        tmem_ld_wait();
+        const int col0 = n0 + c;
+        if (row_ok) {
+        float f[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * inv;
+        if (col0 + 32 <= p.n_split) {
+          if (p.c0_dt == kBF16) {
+            uint16_t* dst = static_cast<uint16_t*>(p.c0) + (long long)split * p.c0_split_stride + (long long)row * p.ldc0 + col0;
+            if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                uint4 o;
+                o.x = pack_bf16x2(f[8 * i + 0], f[8 * i + 1]);
+                o.y = pack_bf16x2(f[8 * i + 2], f[8 * i + 3]);
+                o.z = pack_bf16x2(f[8 * i + 4], f[8 * i + 5]);
+                o.w = pack_bf16x2(f[8 * i + 6], f[8 * i + 7]);
+                reinterpret_cast<uint4*>(dst)[i] = o;
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) dst[i] = static_cast<uint16_t>(pack_bf16x2(f[i], 0.0f) & 0xFFFF);
+            }
+          } else {
+            float* dst = static_cast<float*>(p.c0) + (long long)split * p.c0_split_stride + (long long)row * p.ldc0 + col0;
+            if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                reinterpret_cast<float4*>(dst)[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) dst[i] = f[i];
+            }
+          }
+        } else {
+          // chunk touches the O | O_A boundary or the ragged right edge: element by element
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int col = col0 + i;
+            if (col < p.n_split) {
+              const long long off = (long long)split * p.c0_split_stride + (long long)row * p.ldc0 + col;
+              if (p.c0_dt == kBF16) static_cast<uint16_t*>(p.c0)[off] = static_cast<uint16_t>(pack_bf16x2(f[i], 0.0f) & 0xFFFF);
+              else static_cast<float*>(p.c0)[off] = f[i];
+            } else if (col < p.N) {
+              p.c1[(long long)row * p.ldc1 + (col - p.n_split)] = f[i];
+              amax_bits = max(amax_bits, __float_as_uint(f[i]) & 0x7FFFFFFFu);
+            }
+          }
+        }
+        }  // row_ok
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tmem_empty_bar(acc));
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+    if (p.amax1_bits != nullptr) {
+      amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
+      if (lane == 0 && amax_bits != 0) atomicMax(p.amax1_bits, amax_bits);
+    }
+  }
+
+  // ------------------------------------------------------------ common exit
+  if (aborted) {
+    // give copies and MMAs in flight time to land before the shared memory and TMEM are released
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 200000ull) { }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------ host side
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      ptr = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(ptr);
+  }();
+  return fn;
+}
+
+// 2-D uint8 tensor [rows][cols] with row pitch ld bytes; box = box_cols x box_rows, 128-byte swizzle.
+bool make_tensor_map(CUtensorMap* map, const uint8_t* base, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols,
+                     uint32_t box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld)};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t elem_strides[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box, elem_strides,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int count = [] {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    return n;
+  }();
+  return count;
+}
+
+template <bool kAMn, bool kBMn>
+cudaError_t launch_variant(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& gp, int grid, size_t smem,
+                           cudaStream_t stream) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_fp8_kernel<kAMn, kBMn>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(kSmemBudget));
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  gemm_fp8_kernel<kAMn, kBMn><<<grid, kGemmThreads, smem, stream>>>(ta, tb, gp);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+int gemm_k_splits_for_db(int64_t m, int64_t T) {
+  const int64_t m_tiles = (m + kBlockM - 1) / kBlockM;
+  const int64_t kblocks = (T + kBlockKBytes - 1) / kBlockKBytes;
+  int64_t want = (2 * 148 + m_tiles - 1) / m_tiles;
+  if (want < 1) want = 1;
+  if (want > kblocks) want = kblocks;
+  const int64_t per = (kblocks + want - 1) / want;
+  return static_cast<int>((kblocks + per - 1) / per);
+}
+
+cudaError_t launch_gemm_fp8(const GemmProblem& q, cudaStream_t stream) {
+  if (q.M <= 0 || q.N <= 0 || q.K <= 0) return cudaErrorInvalidValue;
+  if (q.block_n < 16 || q.block_n > 256 || q.block_n % 16) return cudaErrorInvalidValue;
+  if (q.b_mn_major && q.block_n % 128) return cudaErrorInvalidValue;
+
+  GemmParams gp{};
+  gp.M = static_cast<int>(q.M); gp.N = static_cast<int>(q.N); gp.K = static_cast<int>(q.K);
+  gp.block_n = q.block_n;
+  gp.m_tiles = static_cast<int>((q.M + kBlockM - 1) / kBlockM);
+  gp.n_tiles = static_cast<int>((q.N + q.block_n - 1) / q.block_n);
+  gp.kblocks_total = static_cast<int>((q.K + kBlockKBytes - 1) / kBlockKBytes);
+  gp.k_splits = q.k_splits < 1 ? 1 : q.k_splits;
+  gp.kblocks_per_split = (gp.kblocks_total + gp.k_splits - 1) / gp.k_splits;
+  gp.k_splits = (gp.kblocks_total + gp.kblocks_per_split - 1) / gp.kblocks_per_split;  // no empty split
+  const uint32_t stage_bytes = kATileBytes + static_cast<uint32_t>(q.block_n) * kBlockKBytes;
+  int stages = static_cast<int>((kSmemBudget - 1024 - kBarrierBytes) / stage_bytes);
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 2) return cudaErrorInvalidValue;
+  gp.num_stages = stages;
+  // instruction descriptor: fp32 accumulate, operand formats and majors, N/8 at bit 17, M/16 at bit 24
+  gp.idesc = (1u << 4) | (static_cast<uint32_t>(q.a_fmt) << 7) | (static_cast<uint32_t>(q.b_fmt) << 10) |
+             ((q.a_mn_major ? 1u : 0u) << 15) | ((q.b_mn_major ? 1u : 0u) << 16) |
+             (static_cast<uint32_t>(q.block_n >> 3) << 17) | (static_cast<uint32_t>(kBlockM >> 4) << 24);
+  gp.c0 = q.c0; gp.ldc0 = q.ldc0; gp.c0_dt = q.c0_dt; gp.n_split = static_cast<int>(q.n_split);
+  gp.c0_split_stride = q.c0_split_stride;
+  gp.c1 = q.c1; gp.ldc1 = q.ldc1; gp.amax1_bits = q.amax1_bits;
+  gp.scale_a = q.scale_a; gp.scale_b = q.scale_b;
+  gp.status = q.status;
+
+  CUtensorMap ta, tb;
+  bool ok;
+  if (!q.a_mn_major) ok = make_tensor_map(&ta, q.a, q.M, q.K, q.lda, kBlockKBytes, kBlockM);
+  else               ok = make_tensor_map(&ta, q.a, q.K, q.M, q.lda, kBlockM, kBlockKBytes);
+  if (!ok) return cudaErrorInvalidValue;
+  if (!q.b_mn_major) ok = make_tensor_map(&tb, q.b, q.N, q.K, q.ldb, kBlockKBytes, static_cast<uint32_t>(q.block_n));
+  else               ok = make_tensor_map(&tb, q.b, q.K, q.N, q.ldb, 128, kBlockKBytes);
+  if (!ok) return cudaErrorInvalidValue;
+
+  const long long total_tiles = static_cast<long long>(gp.m_tiles) * gp.n_tiles * gp.k_splits;
+  int grid = sm_count();
+  if (total_tiles < grid) grid = static_cast<int>(total_tiles);
+  const size_t smem = static_cast<size_t>(stages) * stage_bytes + kBarrierBytes + 1024;
+  if (q.a_mn_major) {
+    if (q.b_mn_major) return launch_variant<true, true>(ta, tb, gp, grid, smem, stream);
+    return launch_variant<true, false>(ta, tb, gp, grid, smem, stream);
+  }
+  if (q.b_mn_major) return launch_variant<false, true>(ta, tb, gp, grid, smem, stream);
+  return launch_variant<false, false>(ta, tb, gp, grid, smem, stream);
+}
+
+}  // namespace falqon

@@ -1,0 +1,58 @@
+// Host-side declarations shared by the translation units of libfalqon (not part of the public ABI).
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace falqon {
+
+constexpr int kE4M3 = 0, kE5M2 = 1;
+constexpr int kBF16 = 0, kF32 = 1;
+
+inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+
+// ---- quantize.cu
+// amax_bits: device word holding the running max of |x| as an fp32 bit pattern (cleared by the call).
+cudaError_t launch_absmax(const void* src, int src_dt, int64_t count, float premul, uint32_t* amax_bits,
+                          cudaStream_t stream);
+// Cast with scale = fp8max / *amax (from_amax) or = *scale_ptr.  Also writes scale_out / amax_out if non-null.
+cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, int fmt, float premul,
+                                   const float* amax_or_scale, bool from_amax, uint8_t* dst, float* scale_out,
+                                   float* amax_out, cudaStream_t stream);
+cudaError_t launch_quantize_per_row(const void* src, int src_dt, int64_t rows, int64_t cols, int fmt, float premul,
+                                    const float* scale_in, uint8_t* dst, float* scale_out, float* amax_out,
+                                    cudaStream_t stream);
+// O_A [T][r] fp32 -> E4M3 codes written transposed as [r16][ldt] with s_OA = 448 / *amax_oa.
+cudaError_t launch_quantize_oa_transposed(const float* oa, const float* amax_oa, int64_t T, int64_t r, int64_t r16,
+                                          int64_t ldt, uint8_t* oaq_t, float* s_oa_out, cudaStream_t stream);
+
+// ---- gemm_fp8.cu
+struct GemmProblem {
+  // D[M][N] = A[M][K] * B[N][K]^T with fp32 accumulation on tcgen05
+  int64_t M, N, K;
+  const uint8_t* a; int64_t lda; bool a_mn_major; int a_fmt;  // K-major: a[M][lda]; MN-major: a[K][lda]
+  const uint8_t* b; int64_t ldb; bool b_mn_major; int b_fmt;  // K-major: b[N][ldb]; MN-major: b[K][ldb]
+  int block_n;                 // tile width (16..256, multiple of 16)
+  int k_splits;                // >1: partial sums, one output slab per split, no rescale
+  // epilogue: columns [0, n_split) -> c0 (bf16 or fp32), columns [n_split, N) -> c1 (fp32) with |max| -> amax1
+  void* c0; int64_t ldc0; int c0_dt; int64_t n_split; int64_t c0_split_stride;
+  float* c1; int64_t ldc1; uint32_t* amax1_bits;
+  const float* scale_a; const float* scale_b;  // device scalars; output *= 1/(sa*sb); null = no rescale
+  int* status;
+};
+cudaError_t launch_gemm_fp8(const GemmProblem& p, cudaStream_t stream);
+int gemm_k_splits_for_db(int64_t m, int64_t T);
+
+// ---- proxy_update.cu
+cudaError_t launch_reduce_db(const float* partials, int splits, int64_t count, const float* s_g, const float* s_oa,
+                             float* dB, cudaStream_t stream);
+cudaError_t launch_sgd_score(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, float* score,
+                             cudaStream_t stream);
+// scratch: at least topk_scratch_bytes(m).  idx (device [k], ascending) is always written to sel_idx.
+size_t topk_scratch_bytes(int64_t m);
+cudaError_t launch_topk(const float* score, int64_t m, int64_t k, int32_t* sel_idx, void* scratch, cudaStream_t stream);
+cudaError_t launch_merge_rows(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
+                              int64_t r, cudaStream_t stream);
+
+}  // namespace falqon

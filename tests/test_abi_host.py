@@ -1,0 +1,82 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every declared symbol,
+sizes its workspace sanely and rejects bad arguments before launching anything."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def fq():
+    from paper_2510_24061_b200 import build
+    build.build()
+    from paper_2510_24061_b200 import binding
+    return binding
+
+
+def test_library_exports_every_declared_symbol(fq):
+    header = open(os.path.join(ROOT, "include", "falqon.h")).read()
+    declared = set(re.findall(r"\b(falqon_[a-z_]+)\s*\(", header))
+    assert declared == set(fq.EXPORTS)
+    for name in declared:
+        assert hasattr(fq.lib, name), name
+
+
+def test_workspace_layout(fq):
+    m, n, r, T = 4096, 4096, 64, 4096
+    total = fq.workspace_bytes(m, n, r, T)
+    assert total >= T * max(m, n) + T * r
+    seen = []
+    for which in (fq.WS_XQ, fq.WS_OAQ_T, fq.WS_SCALES, fq.WS_SCORE, fq.WS_DB_PART):
+        off, size = fq.workspace_region(m, n, r, T, which)
+        assert off % 256 == 0 and off + size <= total
+        seen.append((off, off + size))
+    seen.sort()
+    assert all(a[1] <= b[0] for a, b in zip(seen, seen[1:]))          # regions do not overlap
+    # score region does not move with T, so a proxy update finds it in a workspace sized for any T
+    assert fq.workspace_region(m, n, r, 1, fq.WS_SCORE) == fq.workspace_region(m, n, r, T, fq.WS_SCORE)
+    for bad in [(4096, 4100, 64, 16), (4096, 4096, 12, 16), (4096, 4096, 512, 16), (8, 4096, 64, 16), (4096, 4096, 64, 0)]:
+        assert fq.workspace_bytes(*bad) == 0
+
+
+def test_bad_arguments_are_rejected_on_the_host(fq):
+    lib = fq.lib
+    fake = 0x10000  # an aligned non-null address that is never dereferenced on these paths
+    layer = fq.falqon_layer(256, 256, 16, fake, fake, fake)
+    big = 1 << 40
+    inv, wsp = fq.ERR_INVALID_ARG, fq.ERR_WORKSPACE
+    # quantize
+    assert lib.falqon_quantize(None, 0, 4, 16, 0, 0, None, 1.0, fake, fake, None, fake, 256, None) == inv
+    assert lib.falqon_quantize(fake, 0, 4, 20, 0, 0, None, 1.0, fake, fake, None, fake, 256, None) == inv   # cols % 16
+    assert lib.falqon_quantize(fake, 0, 4, 16, 7, 0, None, 1.0, fake, fake, None, fake, 256, None) == inv   # format
+    assert lib.falqon_quantize(fake + 4, 0, 4, 16, 0, 0, None, 1.0, fake, fake, None, fake, 256, None) == inv  # alignment
+    assert lib.falqon_quantize(fake, 0, 4, 16, 0, 0, None, 1.0, fake, None, None, fake, 256, None) == inv   # nowhere to put the scale
+    assert lib.falqon_quantize(fake, 0, 4, 16, 0, 0, None, 1.0, fake, fake, None, None, 0, None) == wsp
+    # forward
+    assert lib.falqon_melded_forward(None, fake, 0, 16, fake, 0, fake, fake, None, fake, big, None) == inv
+    assert lib.falqon_melded_forward(C.byref(layer), None, 0, 16, fake, 0, fake, fake, None, fake, big, None) == inv
+    assert lib.falqon_melded_forward(C.byref(layer), fake, 0, 0, fake, 0, fake, fake, None, fake, big, None) == inv
+    assert lib.falqon_melded_forward(C.byref(layer), fake, 3, 16, fake, 0, fake, fake, None, fake, big, None) == inv
+    assert lib.falqon_melded_forward(C.byref(layer), fake, 0, 16, fake, 0, fake, fake, None, fake, 1024, None) == wsp
+    odd = fq.falqon_layer(250, 256, 16, fake, fake, fake)
+    assert lib.falqon_melded_forward(C.byref(odd), fake, 0, 16, fake, 0, fake, fake, None, fake, big, None) == inv
+    # backward
+    assert lib.falqon_melded_backward(C.byref(layer), fake, 0, 16, None, fake, fake, 0, fake, None, fake, big, None) == inv
+    assert lib.falqon_melded_backward(C.byref(layer), fake, 0, 16, fake, fake, fake, 0, None, None, fake, big, None) == inv
+    assert lib.falqon_melded_backward(C.byref(layer), fake, 0, 16, fake, fake, None, 0, fake, None, fake, 16, None) == wsp
+    # proxy update
+    assert lib.falqon_proxy_update(C.byref(layer), None, 0.1, 257, None, fake, big, None) == inv            # k > m
+    assert lib.falqon_proxy_update(C.byref(layer), None, 0.1, -1, None, fake, big, None) == inv
+    assert lib.falqon_proxy_update(C.byref(layer), None, float("nan"), 1, None, fake, big, None) == inv
+    assert lib.falqon_proxy_update(C.byref(layer), None, 0.1, 1, None, fake, 64, None) == wsp
+    assert lib.falqon_proxy_update(None, None, 0.1, 1, None, fake, big, None) == inv
+
+
+def test_launch_counts(fq):
+    assert fq.launch_count("falqon_melded_forward") == 3
+    assert fq.launch_count("falqon_melded_backward") == 6
+    assert fq.launch_count("falqon_proxy_update", k=4) == 4 and fq.launch_count("falqon_proxy_update", k=0) == 1
+    assert fq.launch_count("nope") == 0

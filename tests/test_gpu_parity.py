@@ -1,0 +1,234 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, stage by stage.
+
+Each stage is teacher-forced: the oracle is fed the GPU's actual inputs of that stage, so the
+comparison isolates the stage.  Casts, scales, scores, top-k indices and merged rows must match bit
+for bit; tensor-core products must be within 2e-5 relative Frobenius error of the oracle's
+fp64-accumulated product of the identical FP8 operand bytes, taken on fp32 outputs.
+"""
+import numpy as np
+import pytest
+import torch
+
+from helpers import bits32, f32, layer_inputs, rel_fro, u8
+from paper_2510_24061_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+GEMM_TOL = 2e-5  # relative Frobenius error bound on tensor-core outputs
+
+
+@pytest.fixture(scope="module")
+def fq():
+    from paper_2510_24061_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def orc():
+    from oracle import falqon_oracle
+    return falqon_oracle
+
+
+DEV = "cuda:0"
+
+
+# ------------------------------------------------------------------ quantizer (S1 / S3 / S0)
+
+@pytest.mark.parametrize("fmt", [0, 1])
+@pytest.mark.parametrize("shape,dtype", [((512, 1024), torch.bfloat16), ((37, 48), torch.float32),
+                                         ((1, 16), torch.float32), ((1500, 4112), torch.bfloat16)])
+def test_quantize_per_tensor_bit_exact(fq, orc, fmt, shape, dtype):
+    x = synth.activations(5, 1, shape[0], shape[1], 4).to(dtype)
+    codes, scale, amax = fq.quantize(x.to(DEV), fmt)
+    q, s, a = orc.quantize(f32(x), fmt)
+    assert bits32(f32(amax))[0] == bits32(a) and bits32(f32(scale))[0] == bits32(s)
+    assert np.array_equal(u8(codes), q)
+    assert fq.last_device_status() == 0
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_cast_exhaustive_bf16_and_fp32_sample(fq, orc, fmt):
+    one = torch.ones(1, dtype=torch.float32, device=DEV)
+    bits = torch.arange(1 << 16, dtype=torch.int32).to(torch.int16).view(torch.bfloat16).reshape(4096, 16)
+    finite = torch.isfinite(bits.float())
+    x = torch.where(finite, bits, torch.zeros_like(bits))
+    codes, _, _ = fq.quantize(x.to(DEV), fmt, scale_in=one, want_amax=False)
+    assert np.array_equal(u8(codes), orc.encode_array(f32(x), fmt))
+    # every 64th fp32 bit pattern (2^26 values), NaN/inf replaced by 0
+    raw = (torch.arange(1 << 26, dtype=torch.int64) * 64 + 17).to(torch.int32).view(torch.float32)
+    raw = torch.where(torch.isfinite(raw), raw, torch.zeros_like(raw)).reshape(1 << 14, 1 << 12)
+    codes, _, _ = fq.quantize(raw.to(DEV), fmt, scale_in=one, want_amax=False)
+    assert np.array_equal(u8(codes), orc.encode_array(raw.numpy(), fmt))
+
+
+def test_quantize_given_scale_premul_and_per_row(fq, orc):
+    a = synth.adapter_a(3, 0, 16, 1024)
+    s_w = torch.tensor([4611.5], dtype=torch.float32)
+    codes, _, _ = fq.quantize(a.to(DEV), 0, scale_in=s_w.to(DEV), premul=2.0, want_amax=False)
+    q, _, _ = orc.quantize(f32(a), 0, scale_in=s_w.numpy(), premul=2.0)
+    assert np.array_equal(u8(codes), q)
+    w = synth.student_t3_bf16(3, 1, (96, 272), 0.02)
+    codes, scale, amax = fq.quantize(w.to(DEV), 0, gran=fq.PER_ROW)
+    q, s, am = orc.quantize(f32(w), 0, gran=orc.PER_ROW)
+    assert np.array_equal(bits32(f32(scale)), bits32(s)) and np.array_equal(bits32(f32(amax)), bits32(am))
+    assert np.array_equal(u8(codes), q)
+
+
+# ------------------------------------------------------------------ one layer, all stages
+
+def _run_layer_stages(fq, orc, seed, m, n, r, T, k, gamma, n_outliers, steps, lr, y_dtype=torch.float32):
+    W, A, B, X = layer_inputs(seed, 0, m, n, r, T, n_outliers)
+    # S0: set-up (quantize W, A; meld B over all rows)
+    layer = fq.setup_layer(W.to(DEV), A.to(DEV), B.to(DEV), gamma)
+    wq_o, s_w_o, dbuf_o = orc.setup_layer(f32(W), f32(A), f32(B), gamma)
+    assert bits32(f32(layer.s_w))[0] == bits32(s_w_o)
+    assert np.array_equal(u8(layer.wq), wq_o), "melded backbone codes differ after set-up"
+    assert not f32(layer.dbuf).any()
+    ws = layer.workspace(T)
+    Xd = X.to(DEV)
+    for step in range(steps):
+        # ---- forward
+        Y, OA, amax_oa, s_x = fq.melded_forward(layer, Xd, y_dtype=y_dtype, ws=ws)
+        xq_g = u8(fq.ws_view(layer, ws, T, fq.WS_XQ)).reshape(T, n)
+        xq_o, s_x_o, _ = orc.quantize(f32(X), orc.E4M3)
+        assert bits32(f32(s_x))[0] == bits32(s_x_o) and np.array_equal(xq_g, xq_o)
+        wq_now = u8(layer.wq)
+        Y_o, OA_o, _ = orc.forward(xq_g, np.float32(f32(s_x)[0]), wq_now, np.float32(f32(layer.s_w)[0]), m, r)
+        OA_g = f32(OA)
+        assert rel_fro(f32(Y), Y_o) <= GEMM_TOL, f"Y step {step}"
+        assert rel_fro(OA_g, OA_o) <= GEMM_TOL, f"OA step {step}"
+        assert bits32(f32(amax_oa))[0] == bits32(np.abs(OA_g).max())
+        # ---- backward
+        dY = synth.out_grad(seed, 0, step, T, m)
+        dX, dB, s_g = fq.melded_backward(layer, dY.to(DEV), OA, amax_oa, dx_dtype=torch.float32, ws=ws)
+        gq_g = u8(fq.ws_view(layer, ws, T, fq.WS_GQ)).reshape(T, m)
+        gq_o, s_g_o, _ = orc.quantize(f32(dY), orc.E5M2)
+        assert bits32(f32(s_g))[0] == bits32(s_g_o) and np.array_equal(gq_g, gq_o)
+        oaq_o, s_oa_o, _ = orc.quantize(OA_g, orc.E4M3)
+        scales = f32(fq.ws_view(layer, ws, T, fq.WS_SCALES).view(torch.float32))
+        assert bits32(scales[5]) == bits32(s_oa_o)
+        r16, t16 = (r + 15) // 16 * 16, (T + 15) // 16 * 16
+        oaq_t = u8(fq.ws_view(layer, ws, T, fq.WS_OAQ_T)).reshape(r16, t16)
+        assert np.array_equal(oaq_t[:r, :T].T, oaq_o)
+        dX_o = orc.dx_gemm(gq_g, s_g_o, wq_now, np.float32(f32(layer.s_w)[0]), m)
+        dB_o = orc.db_gemm(gq_g, s_g_o, oaq_o, s_oa_o)
+        assert rel_fro(f32(dX), dX_o) <= GEMM_TOL, f"dX step {step}"
+        assert rel_fro(f32(dB), dB_o) <= GEMM_TOL, f"dB step {step}"
+        # ---- proxy update, fed the GPU's own dB
+        dbuf_o = f32(layer.dbuf).copy()
+        wq_o2 = wq_now.copy()
+        idx = fq.proxy_update(layer, dB, lr, k, ws=ws)
+        idx_o, score_o = orc.proxy_update(wq_o2, dbuf_o, f32(dB), lr, k, m, r)
+        score_g = f32(fq.ws_view(layer, ws, T, fq.WS_SCORE).view(torch.float32))
+        assert np.array_equal(bits32(score_g), bits32(score_o)), f"scores step {step}"
+        if k > 0:
+            assert np.array_equal(u8(idx), idx_o), f"top-k step {step}"
+        assert np.array_equal(u8(layer.wq), wq_o2), f"merged rows step {step}"
+        assert np.array_equal(bits32(f32(layer.dbuf)), bits32(dbuf_o)), f"DeltaBuffer step {step}"
+    assert fq.last_device_status() == 0
+    return layer
+
+
+@pytest.mark.parametrize("lr", [2e-4, 2e-2, 2e-1])
+def test_config0_three_steps_all_stages(fq, orc, lr):
+    c = synth.config0()
+    _run_layer_stages(fq, orc, c["seed"], c["m"], c["n"], c["r"], c["T"], c["k"], c["alpha"] / c["r"],
+                      c["n_outliers"], c["steps"], lr)
+
+
+@pytest.mark.parametrize("m,n,r,T,k", [(272, 208, 8, 200, 5), (128, 128, 16, 128, 0), (144, 400, 24, 77, 144),
+                                       (1040, 528, 72, 333, 1), (256, 1024, 128, 640, 31), (512, 256, 256, 130, 512)])
+def test_ragged_and_edge_shapes(fq, orc, m, n, r, T, k):
+    _run_layer_stages(fq, orc, 11, m, n, r, T, k, 1.0, 3, 2, 2e-2)
+
+
+def test_bf16_outputs_are_rounded_fp32_outputs(fq):
+    c = synth.config0()
+    W, A, B, X = layer_inputs(0, 0, c["m"], c["n"], c["r"], c["T"], c["n_outliers"])
+    layer = fq.setup_layer(W.to(DEV), A.to(DEV), B.to(DEV), 2.0)
+    Y32, OA, amax_oa, _ = fq.melded_forward(layer, X.to(DEV), y_dtype=torch.float32)
+    Y16, OA2, _, _ = fq.melded_forward(layer, X.to(DEV), y_dtype=torch.bfloat16)
+    assert torch.equal(Y32.to(torch.bfloat16), Y16) and torch.equal(OA, OA2)
+    dY = synth.out_grad(0, 0, 0, c["T"], c["m"]).to(DEV)
+    dX32, dB, _ = fq.melded_backward(layer, dY, OA, amax_oa, dx_dtype=torch.float32)
+    dX16, dB2, _ = fq.melded_backward(layer, dY, OA, amax_oa, dx_dtype=torch.bfloat16)
+    assert torch.equal(dX32.to(torch.bfloat16), dX16) and torch.equal(dB, dB2)   # run-to-run deterministic
+    _, dB3, _ = fq.melded_backward(layer, dY, OA, amax_oa, need_dx=False)
+    assert torch.equal(dB, dB3)
+
+
+def test_b_zero_leaves_plain_fp8_layer(fq):
+    c = synth.config0()
+    W, A, _, X = layer_inputs(0, 0, c["m"], c["n"], c["r"], c["T"], c["n_outliers"])
+    Wd, Ad = W.to(DEV), A.to(DEV)
+    plain = fq.setup_layer(Wd, Ad, None, 2.0)
+    melded = fq.setup_layer(Wd, Ad, torch.zeros(c["m"], c["r"], device=DEV), 2.0)
+    assert torch.equal(plain.wq, melded.wq)
+    Y0, _, _, _ = fq.melded_forward(plain, X.to(DEV), y_dtype=torch.float32)
+    Y1, _, _, _ = fq.melded_forward(melded, X.to(DEV), y_dtype=torch.float32)
+    assert torch.equal(Y0, Y1)
+
+
+def test_topk_ties_go_to_lowest_index(fq, orc):
+    m, n, r = 256, 128, 16
+    W, A, _, _ = layer_inputs(2, 0, m, n, r, 16, 0)
+    layer = fq.setup_layer(W.to(DEV), A.to(DEV), None, 1.0)
+    dB = synth.normal_bf16(2, 99, (m, r), 1.0).float()
+    dB[40] = dB[7]; dB[200] = dB[7]; dB[100] = -dB[7]
+    dB[[7, 40, 100, 200]] *= 50           # the four tied rows carry the largest score
+    for k in (1, 2, 3, 4, 5):
+        layer.dbuf.zero_()
+        wq_o, dbuf_o = u8(layer.wq).copy(), np.zeros((m, r), np.float32)
+        idx = fq.proxy_update(layer, dB.to(DEV), 0.01, k)
+        idx_o, _ = orc.proxy_update(wq_o, dbuf_o, dB.numpy(), 0.01, k, m, r)
+        assert u8(idx).tolist() == idx_o.tolist()
+        assert u8(idx).tolist()[:min(k, 4)] == [7, 40, 100, 200][:min(k, 4)]
+        assert np.array_equal(u8(layer.wq), wq_o)
+
+
+# ------------------------------------------------------------------ full-size projections, sampled
+
+@pytest.mark.parametrize("name,n,m", [("q", 4096, 4096), ("gate", 4096, 11008), ("down", 11008, 4096)])
+def test_config1_projection_sampled(fq, orc, name, n, m):
+    c = synth.config1()
+    T, r, k = c["T"], c["r"], c["k"]
+    n_out = round(c["outlier_frac"] * n)
+    matrix = {"q": 0, "gate": 4, "down": 6}[name]
+    W = synth.backbone(0, matrix, m, n, DEV)
+    A = synth.adapter_a(0, matrix, r, n, DEV)
+    B = synth.adapter_b(0, matrix, m, r, DEV)
+    X = synth.activations(0, matrix, T, n, n_out, DEV)
+    dY = synth.out_grad(0, matrix, 0, T, m, DEV)
+    layer = fq.setup_layer(W, A, B, 1.0)
+    ws = layer.workspace(T)
+    Y, OA, amax_oa, s_x = fq.melded_forward(layer, X, y_dtype=torch.float32, ws=ws)
+    xq_g = u8(fq.ws_view(layer, ws, T, fq.WS_XQ)).reshape(T, n)
+    xq_o, s_x_o, _ = orc.quantize(f32(X), orc.E4M3)
+    assert bits32(f32(s_x))[0] == bits32(s_x_o) and np.array_equal(xq_g, xq_o)
+    wq = u8(layer.wq)
+    s_w = np.float32(f32(layer.s_w)[0])
+    rng = np.random.default_rng(1)
+    tsel = np.sort(rng.choice(T, 48, replace=False))
+    fsel = np.sort(rng.choice(m, 48, replace=False))
+    merged = torch.cat([Y, OA], dim=1)
+    rows_o = orc.forward_gemm(xq_g, s_x_o, wq, s_w, m, r, tsel=tsel)                 # 48 token rows x all features
+    assert rel_fro(f32(merged[torch.from_numpy(tsel).to(DEV)]), rows_o) <= GEMM_TOL
+    cols_o = orc.forward_gemm(xq_g, s_x_o, wq, s_w, m, r, fsel=fsel)                 # all tokens x 48 features
+    assert rel_fro(f32(Y[:, torch.from_numpy(fsel).to(DEV)]), cols_o) <= GEMM_TOL
+    assert bits32(f32(amax_oa))[0] == bits32(f32(OA.abs().max()))
+    dX, dB, s_g = fq.melded_backward(layer, dY, OA, amax_oa, dx_dtype=torch.float32, ws=ws)
+    gq_g = u8(fq.ws_view(layer, ws, T, fq.WS_GQ)).reshape(T, m)
+    gq_o, s_g_o, _ = orc.quantize(f32(dY), orc.E5M2)
+    assert bits32(f32(s_g))[0] == bits32(s_g_o) and np.array_equal(gq_g, gq_o)
+    csel = np.sort(rng.choice(n, 48, replace=False))
+    assert rel_fro(f32(dX[torch.from_numpy(tsel).to(DEV)]), orc.dx_gemm(gq_g, s_g_o, wq, s_w, m, tsel=tsel)) <= GEMM_TOL
+    assert rel_fro(f32(dX[:, torch.from_numpy(csel).to(DEV)]), orc.dx_gemm(gq_g, s_g_o, wq, s_w, m, csel=csel)) <= GEMM_TOL
+    oaq_o, s_oa_o, _ = orc.quantize(f32(OA), orc.E4M3)
+    isel = np.sort(rng.choice(m, 96, replace=False))
+    assert rel_fro(f32(dB[torch.from_numpy(isel).to(DEV)]), orc.db_gemm(gq_g, s_g_o, oaq_o, s_oa_o, isel=isel)) <= GEMM_TOL
+    dbuf_o, wq_o = f32(layer.dbuf).copy(), wq.copy()
+    idx = fq.proxy_update(layer, dB, c["lr"], k, ws=ws)
+    idx_o, score_o = orc.proxy_update(wq_o, dbuf_o, f32(dB), c["lr"], k, m, r)
+    assert np.array_equal(u8(idx), idx_o)
+    assert np.array_equal(u8(layer.wq), wq_o) and np.array_equal(bits32(f32(layer.dbuf)), bits32(dbuf_o))
+    assert fq.last_device_status() == 0
