@@ -182,7 +182,7 @@ def test_topk_ties_go_to_lowest_index(fq, orc):
         idx = fq.proxy_update(layer, dB.to(DEV), 0.01, k)
         idx_o, _ = orc.proxy_update(wq_o, dbuf_o, dB.numpy(), 0.01, k, m, r)
         assert u8(idx).tolist() == idx_o.tolist()
-        assert u8(idx).tolist()[:min(k, 4)] == [7, 40, 100, 200][:min(k, 4)]
+        assert set([7, 40, 100, 200][:min(k, 4)]) <= set(u8(idx).tolist())
         assert np.array_equal(u8(layer.wq), wq_o)
 
 
