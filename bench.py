@@ -1,0 +1,343 @@
+#!/usr/bin/env python
+"""Benchmark of the melded FP8-LoRA hot path on B200.
+
+Workload (one "step"): forward, backward and row-wise proxy update of the seven linear layers of one
+LLaMA-7B decoder layer (q, k, v, o 4096->4096; gate, up 4096->11008; down 11008->4096) at 4096 tokens,
+rank 64, top-256 rows per matrix -- synthetic seeded inputs with 1% outlier channels.  The metric is
+the algorithmic fwd+bwd FLOP rate 2T[n(m+r) + mn + mr] summed over the matrices, divided by the time
+of the whole step (quantization of X, dY, O_A and the proxy update are inside the timed region, their
+arithmetic is not counted as useful FLOPs).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line.  N > 1 (under torchrun) runs independent replicas, one per GPU (the path has no
+exchange step); the reported value is the aggregate over ranks with the max-over-ranks time.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2510_24061_b200 import synth  # noqa: E402
+
+METRIC = "melded FP8-LoRA layer fwd+bwd TFLOP/s (7B projection set, T=4096, r=64)"
+UNIT = "TFLOP/s"
+FP8_OVER_BF16 = 2.0        # nominal dense FP8 : bf16 tensor throughput on B200 (4.5 : 2.25 PFLOP/s)
+FALLBACK_BF16_TFLOPS = 1590.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def layer_flops(T, n, m, r):
+    """Algorithmic FLOPs of one fwd+bwd of one matrix: forward 2Tn(m+r), dX 2Tmn, dB 2Tmr."""
+    return 2.0 * T * (n * (m + r) + m * n + m * r)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            d = json.load(fh)
+        return dict(bf16_sustained=float(d["bf16_tflops_sustained"]), bf16_burst=float(d["bf16_tflops"]),
+                    hbm=float(d["hbm_gbs"]), source="measured")
+    except Exception:
+        return dict(bf16_sustained=FALLBACK_BF16_TFLOPS * 1.4 / 1.59, bf16_burst=FALLBACK_BF16_TFLOPS,
+                    hbm=FALLBACK_HBM_GBS, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+
+        def pump():
+            for line in self.proc.stdout:
+                self.lines.append(line.strip())
+        self.thread = threading.Thread(target=pump, daemon=True)
+        self.thread.start()
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_workload(fq, device, seed, T, r, k, linears, outlier_frac):
+    layers = []
+    for idx, (name, n, m) in enumerate(linears):
+        W = synth.backbone(seed, idx, m, n, device)
+        A = synth.adapter_a(seed, idx, r, n, device)
+        B = synth.adapter_b(seed, idx, m, r, device)
+        layer = fq.setup_layer(W, A, B, 1.0)
+        del W
+        X = synth.activations(seed, idx, T, n, round(outlier_frac * n), device)
+        dY = synth.out_grad(seed, idx, 0, T, m, device)
+        out_f = (torch.empty((T, m), dtype=torch.bfloat16, device=device),
+                 torch.empty((T, r), dtype=torch.float32, device=device),
+                 torch.empty(1, dtype=torch.float32, device=device), torch.empty(1, dtype=torch.float32, device=device))
+        out_b = (torch.empty((T, n), dtype=torch.bfloat16, device=device),
+                 torch.empty((m, r), dtype=torch.float32, device=device), torch.empty(1, dtype=torch.float32, device=device))
+        idx_out = torch.empty(k, dtype=torch.int32, device=device)
+        layers.append(dict(name=name, n=n, m=m, layer=layer, X=X, dY=dY, out_f=out_f, out_b=out_b, idx=idx_out,
+                           ws=layer.workspace(T)))
+    return layers
+
+
+def run_step(fq, layers, lr, k):
+    for L in layers:
+        _, OA, amax_oa, _ = fq.melded_forward(L["layer"], L["X"], ws=L["ws"], out=L["out_f"])
+        _, dB, _ = fq.melded_backward(L["layer"], L["dY"], OA, amax_oa, ws=L["ws"], out=L["out_b"])
+        fq.proxy_update(L["layer"], dB, lr, k, ws=L["ws"], idx_out=L["idx"])
+
+
+def run_step_e2e(fq, layers, host, lr, k):
+    """Same step, but every input starts in pinned host memory and the results are read back."""
+    for L, H in zip(layers, host):
+        L["X"].copy_(H["X"], non_blocking=True)
+        L["dY"].copy_(H["dY"], non_blocking=True)
+        _, OA, amax_oa, _ = fq.melded_forward(L["layer"], L["X"], ws=L["ws"], out=L["out_f"])
+        _, dB, _ = fq.melded_backward(L["layer"], L["dY"], OA, amax_oa, ws=L["ws"], out=L["out_b"])
+        fq.proxy_update(L["layer"], dB, lr, k, ws=L["ws"], idx_out=L["idx"])
+        H["dB"].copy_(dB, non_blocking=True)
+        H["idx"].copy_(L["idx"], non_blocking=True)
+
+
+def time_oracle_sample(T_sample, r, k, lr, seed=0):
+    """The CPU oracle, as it stands, on a token slice of the q projection (4096 -> 4096): quantize,
+    forward, backward and proxy update.  Returns (TFLOP/s, seconds, threads, description)."""
+    import numpy as np
+    from oracle import falqon_oracle as orc
+    n = m = 4096
+    W = synth.backbone(seed, 0, m, n).float().numpy()
+    A = synth.adapter_a(seed, 0, r, n).float().numpy()
+    X = synth.activations(seed, 0, T_sample, n, round(0.01 * n)).float().numpy()
+    dY = synth.out_grad(seed, 0, 0, T_sample, m).float().numpy()
+    wq, s_w, dbuf = orc.setup_layer(W, A, None, 1.0)   # set-up is not timed (not on the per-step path)
+    t0 = time.perf_counter()
+    f = orc.layer_forward(X, wq, s_w, m, r)
+    b = orc.layer_backward(dY, f["OA"], wq, s_w, m, r)
+    orc.proxy_update(wq, dbuf, b["dB"].astype(np.float32), lr, k, m, r)
+    dt = time.perf_counter() - t0
+    flops = layer_flops(T_sample, n, m, r)
+    desc = f"q projection 4096->4096, first {T_sample} of 4096 tokens, r={r}, top-{k}: quantize+fwd+bwd+proxy update"
+    return flops / dt / 1e12, dt, orc.num_threads(), desc
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="falqon", choices=["falqon", "reference"])
+    ap.add_argument("--oracle-tokens", type=int, default=256)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    cfg = synth.config1()
+    T, r, k, lr = cfg["T"], cfg["r"], cfg["k"], cfg["lr"]
+    linears = cfg["linears"]
+    flops_step = sum(layer_flops(T, n, m, r) for _, n, m in linears)
+    workload = {"workload": "configs[1]: LLaMA-7B projection set (q,k,v,o,gate,up,down), tokens=4096, rank=64, top-k=256",
+                "tokens": T, "rank": r, "topk": k, "matrices": len(linears), "gflop_per_step": flops_step / 1e9,
+                "l2": "inputs larger than L2 (0.85 GB touched per step)", "parallelism": f"replicas x{world}"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        steps = max(1, min(args.steps, 3))
+        for _ in range(min(args.warmup, 1)):
+            time_oracle_sample(min(args.oracle_tokens, 64), r, k, lr)
+        vals = [time_oracle_sample(args.oracle_tokens, r, k, lr) for _ in range(steps)]
+        tf = statistics.mean(v[0] for v in vals)
+        secs = statistics.mean(v[1] for v in vals)
+        print(json.dumps({
+            "impl": "reference", "metric": METRIC, "value": tf, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+            "warmup": min(args.warmup, 1), "ms_per_step": secs * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "fp8 (software E4M3/E5M2, fp64 accumulate)", "data": "synthetic",
+            "config": workload,
+            "cpu_baseline": {"value": tf, "unit": UNIT, "cores": vals[0][2], "kind": "oracle", "sample": vals[0][3]},
+            "e2e": {"value": tf, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the melded FP8-LoRA path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    from paper_2510_24061_b200 import binding as fq
+
+    layers = build_workload(fq, device, cfg["seed"] + rank, T, r, k, linears, cfg["outlier_frac"])
+    torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident timing, with the tensor-core products bracketed by events
+    for _ in range(max(args.warmup, 3)):
+        run_step(fq, layers, lr, k)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    gemm_stages = ["gemm_fwd", "gemm_dx", "gemm_db"]
+    n_records = 3 * len(layers) * args.steps
+    fq.profile_start(n_records, gemm_stages)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        run_step(fq, layers, lr, k)
+    ev1.record()
+    barrier()
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+    clocks = sampler.stop()
+    records = fq.profile_stop(n_records)
+    status = fq.last_device_status()
+    ms_step = ms_total / args.steps
+    value = world * flops_step / (ms_step * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel: the tcgen05 FP8 GEMM in its two tensor-bound roles
+    peaks = measured_peaks()
+    per_rec = 3 * len(layers)
+    t_big = sum(ms for name, ms in records if name in ("gemm_fwd", "gemm_dx"))
+    f_big = args.steps * sum(2.0 * T * n * (m + r) + 2.0 * T * m * n for _, n, m in linears)
+    launches_big = sum(1 for name, _ in records if name in ("gemm_fwd", "gemm_dx"))
+    achieved = f_big / (t_big * 1e-3) / 1e12 if t_big > 0 else 0.0
+    peak = peaks["bf16_sustained"] * FP8_OVER_BF16
+    roofline = {"kernel": "gemm_fp8_kernel (forward and input-gradient products)", "bound": "tensor",
+                "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "peak_source": f"{peaks['source']} bf16 sustained x{FP8_OVER_BF16:g} (nominal FP8:bf16 ratio)",
+                "frac_of_burst_peak": achieved / (peaks["bf16_burst"] * FP8_OVER_BF16),
+                "frac_of_nominal_4500": achieved / 4500.0,
+                "launches": launches_big, "avg_launch_ms": t_big / max(launches_big, 1),
+                "gflop_per_launch": f_big / max(launches_big, 1) / 1e9, "traffic": None}
+    t_db = sum(ms for name, ms in records if name == "gemm_db")
+
+    # ---- stage breakdown (separate untimed-for-value pass with every stage bracketed)
+    fq.profile_start(10 * len(layers) * 3, None)
+    for _ in range(3):
+        run_step(fq, layers, lr, k)
+    torch.cuda.synchronize()
+    breakdown = {}
+    for name, ms in fq.profile_stop(10 * len(layers) * 3):
+        breakdown[name] = breakdown.get(name, 0.0) + ms / 3.0
+    hbm_bytes_quant = sum(T * n * 5 + T * m * 5 for _, n, m in linears)   # 2 B absmax read + 2 B cast read + 1 B write
+    t_quant = (breakdown.get("quant_x", 0) + breakdown.get("quant_dy", 0)) * 1e-3
+    quant_gbs = hbm_bytes_quant / t_quant / 1e9 if t_quant > 0 else 0.0
+
+    # ---- end to end: inputs in pinned host memory, results read back, every step
+    host = []
+    for L in layers:
+        host.append(dict(X=L["X"].cpu().pin_memory(), dY=L["dY"].cpu().pin_memory(),
+                         dB=torch.empty(L["out_b"][1].shape, dtype=torch.float32).pin_memory(),
+                         idx=torch.empty(k, dtype=torch.int32).pin_memory()))
+    h2d = sum(H["X"].numel() * 2 + H["dY"].numel() * 2 for H in host)
+    d2h = sum(H["dB"].numel() * 4 + H["idx"].numel() * 4 for H in host)
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(2):
+        run_step_e2e(fq, layers, host, lr, k)
+    barrier()
+    ev0.record()
+    for _ in range(e2e_steps):
+        run_step_e2e(fq, layers, host, lr, k)
+    ev1.record()
+    barrier()
+    ms_e2e = max_over_ranks(ev0.elapsed_time(ev1)) / e2e_steps
+    e2e_value = world * flops_step / (ms_e2e * 1e-3) / 1e12
+
+    launches_per_step = sum(fq.launch_count("falqon_melded_forward") + fq.launch_count("falqon_melded_backward") +
+                            fq.launch_count("falqon_proxy_update", k=k) for _ in layers)
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        tf, secs, threads, desc = time_oracle_sample(args.oracle_tokens, r, k, lr)
+        cpu_baseline = {"value": tf, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
+                        "seconds": secs, "host_cpus": os.cpu_count()}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8",
+        "data": "synthetic", "config": workload, "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e, "steps": e2e_steps,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": roofline,
+        "cpu_baseline": cpu_baseline,
+        "frac_of_fp8_peak": {"of_measured_sustained_x2": value / world / peak, "of_nominal_4500": value / world / 4500.0},
+        "stage_ms_per_step": {k_: round(v, 4) for k_, v in sorted(breakdown.items())},
+        "gemm_db_ms_per_step": t_db / args.steps,
+        "quantize": {"bound": "hbm", "achieved_gbs": quant_gbs, "peak_gbs": peaks["hbm"], "frac": quant_gbs / peaks["hbm"],
+                     "bytes_per_elt": 5, "note": "absmax pass + cast pass of X and dY, algorithmic bytes"},
+        "device_status": status,
+    }
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

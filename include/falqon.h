@@ -143,6 +143,31 @@ int falqon_proxy_update(const falqon_layer *L, const float *dB, float lr, int64_
  * undefined) or FALQON_ERR_CUDA (the synchronize itself failed). */
 int falqon_last_device_status(falqon_stream stream);
 
+/* Stages that the optional timing hook can bracket with CUDA events (bit i of the mask = stage i). */
+typedef enum {
+  FALQON_STAGE_QUANT_X = 0,   /* absmax + cast of X            (S1) */
+  FALQON_STAGE_GEMM_FWD = 1,  /* melded forward product        (S2) */
+  FALQON_STAGE_QUANT_DY = 2,  /* absmax + cast of dY           (S3) */
+  FALQON_STAGE_QUANT_OA = 3,  /* cast of O_A                   (S5a) */
+  FALQON_STAGE_GEMM_DX = 4,   /* input-gradient product        (S4) */
+  FALQON_STAGE_GEMM_DB = 5,   /* adapter-gradient product      (S5b) */
+  FALQON_STAGE_REDUCE_DB = 6, /* fixed-order sum of its slabs  (S5b) */
+  FALQON_STAGE_SGD_SCORE = 7, /* optimizer step + row scores   (S6, S7) */
+  FALQON_STAGE_TOPK = 8,      /* row selection                 (S7) */
+  FALQON_STAGE_MERGE = 9      /* merge + requantize + clear    (S8) */
+} falqon_stage;
+
+/* Timing hook for benchmarks (the paper reports the same forward / backward / quantization
+ * breakdown).  Host only; not thread safe; off by default.  falqon_profile_start makes the calls
+ * above record a pair of CUDA events, on their stream, around each stage whose bit is set in
+ * stage_mask, for at most max_records stages (later ones are not recorded).  The events are host
+ * objects owned by the library; no device memory is allocated.  falqon_profile_stop waits for the
+ * recorded events, writes the elapsed milliseconds and the stage id of each record, in call order,
+ * to the two HOST arrays (capacity entries each), releases the events and returns the number of
+ * records written (>= 0) or a negative falqon_status. */
+int falqon_profile_start(int max_records, unsigned stage_mask);
+int falqon_profile_stop(float *ms_out, int *stage_out, int capacity);
+
 /* Host, pure.  Number of kernels the named call launches for this shape (for launch accounting). */
 int falqon_launch_count(const char *entry_point, int64_t m, int64_t n, int64_t r, int64_t T, int64_t k);
 

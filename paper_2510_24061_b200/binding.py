@@ -21,7 +21,9 @@ PER_TENSOR, PER_ROW = 0, 1
 WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE, WS_DB_PART = range(6)
 
 EXPORTS = ["falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
-           "falqon_melded_backward", "falqon_proxy_update", "falqon_last_device_status", "falqon_launch_count"]
+           "falqon_melded_backward", "falqon_proxy_update", "falqon_last_device_status", "falqon_launch_count",
+           "falqon_profile_start", "falqon_profile_stop"]
+STAGES = ["quant_x", "gemm_fwd", "quant_dy", "quant_oa", "gemm_dx", "gemm_db", "reduce_db", "sgd_score", "topk", "merge"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2510_24061_b200.build` "
@@ -49,6 +51,10 @@ lib.falqon_proxy_update.restype = _i
 lib.falqon_proxy_update.argtypes = [C.POINTER(falqon_layer), _p, _f, _i64, _p, _p, _sz, _p]
 lib.falqon_last_device_status.restype = _i
 lib.falqon_last_device_status.argtypes = [_p]
+lib.falqon_profile_start.restype = _i
+lib.falqon_profile_start.argtypes = [_i, C.c_uint]
+lib.falqon_profile_stop.restype = _i
+lib.falqon_profile_stop.argtypes = [C.POINTER(_f), C.POINTER(_i), _i]
 lib.falqon_launch_count.restype = _i
 lib.falqon_launch_count.argtypes = [C.c_char_p, _i64, _i64, _i64, _i64, _i64]
 
@@ -120,6 +126,23 @@ def launch_count(entry_point: str, m=0, n=0, r=0, T=0, k=0) -> int:
 
 def last_device_status() -> int:
     return int(lib.falqon_last_device_status(_stream()))
+
+
+def profile_start(max_records: int, stages=None):
+    mask = 0
+    for s in (STAGES if stages is None else stages):
+        mask |= 1 << STAGES.index(s)
+    _check("falqon_profile_start", lib.falqon_profile_start(max_records, mask))
+
+
+def profile_stop(capacity: int):
+    """Returns a list of (stage name, milliseconds) in call order."""
+    ms = (_f * capacity)()
+    kinds = (_i * capacity)()
+    n = lib.falqon_profile_stop(ms, kinds, capacity)
+    if n < 0:
+        raise FalqonError("falqon_profile_stop", n)
+    return [(STAGES[kinds[i]], float(ms[i])) for i in range(n)]
 
 
 def quantize(src: torch.Tensor, fmt: int, gran: int = PER_TENSOR, scale_in: torch.Tensor | None = None,

@@ -72,6 +72,32 @@ bool layer_ok(const falqon_layer* L) {
     if (e__ != cudaSuccess) return FALQON_ERR_CUDA;         \
   } while (0)
 
+// ---- optional per-stage timing (host-side CUDA events owned by the library; off by default)
+struct ProfileState {
+  bool active = false;
+  unsigned mask = 0;
+  int capacity = 0, used = 0;
+  cudaEvent_t* start = nullptr;
+  cudaEvent_t* stop = nullptr;
+  int* kind = nullptr;
+};
+ProfileState g_prof;
+
+struct StageTimer {
+  int slot = -1;
+  cudaStream_t stream;
+  StageTimer(int kind, cudaStream_t s) : stream(s) {
+    if (g_prof.active && ((g_prof.mask >> kind) & 1u) && g_prof.used < g_prof.capacity) {
+      slot = g_prof.used++;
+      g_prof.kind[slot] = kind;
+      cudaEventRecord(g_prof.start[slot], stream);
+    }
+  }
+  ~StageTimer() {
+    if (slot >= 0) cudaEventRecord(g_prof.stop[slot], stream);
+  }
+};
+
 }  // namespace
 }  // namespace falqon
 
@@ -147,8 +173,11 @@ int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_d
   const int64_t m = L->m, n = L->n, r = L->r;
 
   // S1: x~, s_x = Q_e4m3(X)
-  FALQON_CUDA(launch_absmax(X, x_dt, T * n, 1.0f, reinterpret_cast<uint32_t*>(scales + 0), stream));
-  FALQON_CUDA(launch_cast_per_tensor(X, x_dt, T * n, kE4M3, 1.0f, scales + 0, true, xq, scales + 1, nullptr, stream));
+  {
+    StageTimer timer(FALQON_STAGE_QUANT_X, stream);
+    FALQON_CUDA(launch_absmax(X, x_dt, T * n, 1.0f, reinterpret_cast<uint32_t*>(scales + 0), stream));
+    FALQON_CUDA(launch_cast_per_tensor(X, x_dt, T * n, kE4M3, 1.0f, scales + 0, true, xq, scales + 1, nullptr, stream));
+  }
   if (s_x_out != nullptr)
     FALQON_CUDA(cudaMemcpyAsync(s_x_out, scales + 1, sizeof(float), cudaMemcpyDeviceToDevice, stream));
   // S2: [Y | O_A] = x~ W~'^T / (s_W s_x), amax(O_A) from the epilogue
@@ -162,7 +191,10 @@ int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_d
   g.c1 = OA; g.ldc1 = r; g.amax1_bits = reinterpret_cast<uint32_t*>(amax_oa);
   g.scale_a = scales + 1; g.scale_b = L->s_w;
   g.status = status;
-  FALQON_CUDA(launch_gemm_fp8(g, stream));
+  {
+    StageTimer timer(FALQON_STAGE_GEMM_FWD, stream);
+    FALQON_CUDA(launch_gemm_fp8(g, stream));
+  }
   return FALQON_OK;
 }
 
@@ -185,13 +217,19 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
   const int64_t m = L->m, n = L->n, r = L->r;
 
   // S3: g~, s_g = Q_e5m2(dY)
-  FALQON_CUDA(launch_absmax(dY, dy_dt, T * m, 1.0f, reinterpret_cast<uint32_t*>(scales + 2), stream));
-  FALQON_CUDA(launch_cast_per_tensor(dY, dy_dt, T * m, kE5M2, 1.0f, scales + 2, true, gq, scales + 3, nullptr, stream));
+  {
+    StageTimer timer(FALQON_STAGE_QUANT_DY, stream);
+    FALQON_CUDA(launch_absmax(dY, dy_dt, T * m, 1.0f, reinterpret_cast<uint32_t*>(scales + 2), stream));
+    FALQON_CUDA(launch_cast_per_tensor(dY, dy_dt, T * m, kE5M2, 1.0f, scales + 2, true, gq, scales + 3, nullptr, stream));
+  }
   if (s_g_out != nullptr)
     FALQON_CUDA(cudaMemcpyAsync(s_g_out, scales + 3, sizeof(float), cudaMemcpyDeviceToDevice, stream));
   // S5a: O~_A, s_OA = Q_e4m3(O_A), written transposed for the dB product
   FALQON_CUDA(cudaMemcpyAsync(scales + 4, amax_oa, sizeof(float), cudaMemcpyDeviceToDevice, stream));
-  FALQON_CUDA(launch_quantize_oa_transposed(OA, amax_oa, T, r, w.r16, w.t16, oaq_t, scales + 5, stream));
+  {
+    StageTimer timer(FALQON_STAGE_QUANT_OA, stream);
+    FALQON_CUDA(launch_quantize_oa_transposed(OA, amax_oa, T, r, w.r16, w.t16, oaq_t, scales + 5, stream));
+  }
   // S4: dX = g~ W~ / (s_W s_g)   (contraction over the m output channels; W~ read MN-major)
   if (dX != nullptr) {
     GemmProblem g{};
@@ -203,6 +241,7 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
     g.c1 = nullptr; g.ldc1 = 0; g.amax1_bits = nullptr;
     g.scale_a = scales + 3; g.scale_b = L->s_w;
     g.status = status;
+    StageTimer timer(FALQON_STAGE_GEMM_DX, stream);
     FALQON_CUDA(launch_gemm_fp8(g, stream));
   }
   // S5b: dB = g~^T O~_A / (s_g s_OA)   (contraction over tokens, split into slabs, fixed-order reduce)
@@ -216,7 +255,11 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
     g.c1 = nullptr; g.ldc1 = 0; g.amax1_bits = nullptr;
     g.scale_a = nullptr; g.scale_b = nullptr;
     g.status = status;
-    FALQON_CUDA(launch_gemm_fp8(g, stream));
+    {
+      StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
+      FALQON_CUDA(launch_gemm_fp8(g, stream));
+    }
+    StageTimer timer(FALQON_STAGE_REDUCE_DB, stream);
     FALQON_CUDA(launch_reduce_db(part, w.splits, m * r, scales + 3, scales + 5, dB, stream));
   }
   return FALQON_OK;
@@ -233,10 +276,19 @@ int falqon_proxy_update(const falqon_layer* L, const float* dB, float lr, int64_
   float* score = reinterpret_cast<float*>(base + w.score);
   int32_t* sel = reinterpret_cast<int32_t*>(base + w.sel_idx);
   const int64_t m = L->m, n = L->n, r = L->r;
-  FALQON_CUDA(launch_sgd_score(L->dbuf, dB, lr, m, r, score, stream));
+  {
+    StageTimer timer(FALQON_STAGE_SGD_SCORE, stream);
+    FALQON_CUDA(launch_sgd_score(L->dbuf, dB, lr, m, r, score, stream));
+  }
   if (k > 0) {
-    FALQON_CUDA(launch_topk(score, m, k, sel, nullptr, stream));
-    FALQON_CUDA(launch_merge_rows(L->wq, L->dbuf, sel, k, m, n, r, stream));
+    {
+      StageTimer timer(FALQON_STAGE_TOPK, stream);
+      FALQON_CUDA(launch_topk(score, m, k, sel, nullptr, stream));
+    }
+    {
+      StageTimer timer(FALQON_STAGE_MERGE, stream);
+      FALQON_CUDA(launch_merge_rows(L->wq, L->dbuf, sel, k, m, n, r, stream));
+    }
     if (idx_out != nullptr)
       FALQON_CUDA(cudaMemcpyAsync(idx_out, sel, static_cast<size_t>(k) * sizeof(int32_t), cudaMemcpyDeviceToDevice, stream));
   }
@@ -254,6 +306,46 @@ int falqon_last_device_status(falqon_stream stream) {
     if (cudaMemcpy(p, &zero, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return FALQON_ERR_CUDA;
   }
   return v;
+}
+
+int falqon_profile_start(int max_records, unsigned stage_mask) {
+  if (g_prof.active || max_records < 1 || max_records > (1 << 20)) return FALQON_ERR_INVALID_ARG;
+  g_prof.start = new cudaEvent_t[max_records];
+  g_prof.stop = new cudaEvent_t[max_records];
+  g_prof.kind = new int[max_records];
+  for (int i = 0; i < max_records; ++i) {
+    if (cudaEventCreate(&g_prof.start[i]) != cudaSuccess || cudaEventCreate(&g_prof.stop[i]) != cudaSuccess) {
+      for (int j = 0; j < i; ++j) { cudaEventDestroy(g_prof.start[j]); cudaEventDestroy(g_prof.stop[j]); }
+      delete[] g_prof.start; delete[] g_prof.stop; delete[] g_prof.kind;
+      g_prof = ProfileState{};
+      return FALQON_ERR_CUDA;
+    }
+  }
+  g_prof.capacity = max_records;
+  g_prof.used = 0;
+  g_prof.mask = stage_mask;
+  g_prof.active = true;
+  return FALQON_OK;
+}
+
+int falqon_profile_stop(float* ms_out, int* stage_out, int capacity) {
+  if (!g_prof.active) return FALQON_ERR_INVALID_ARG;
+  g_prof.active = false;
+  int count = g_prof.used < capacity ? g_prof.used : capacity;
+  if (ms_out == nullptr || stage_out == nullptr) count = 0;
+  int rc = count;
+  for (int i = 0; i < count; ++i) {
+    if (cudaEventSynchronize(g_prof.stop[i]) != cudaSuccess ||
+        cudaEventElapsedTime(&ms_out[i], g_prof.start[i], g_prof.stop[i]) != cudaSuccess) {
+      rc = FALQON_ERR_CUDA;
+      break;
+    }
+    stage_out[i] = g_prof.kind[i];
+  }
+  for (int i = 0; i < g_prof.capacity; ++i) { cudaEventDestroy(g_prof.start[i]); cudaEventDestroy(g_prof.stop[i]); }
+  delete[] g_prof.start; delete[] g_prof.stop; delete[] g_prof.kind;
+  g_prof = ProfileState{};
+  return rc;
 }
 
 int falqon_launch_count(const char* entry_point, int64_t m, int64_t n, int64_t r, int64_t T, int64_t k) {
