@@ -71,7 +71,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -172,11 +172,12 @@ def time_oracle_sample(T_sample, r, k, lr, seed=0):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="falqon", choices=["falqon", "reference"])
     ap.add_argument("--oracle-tokens", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", default=None, help="profiling aid: restrict the workload to one projection (q,k,v,o,gate,up,down)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -185,8 +186,11 @@ def main():
     cfg = synth.config1()
     T, r, k, lr = cfg["T"], cfg["r"], cfg["k"], cfg["lr"]
     linears = cfg["linears"]
+    if args.only is not None:
+        linears = [l for l in linears if l[0] == args.only]
     flops_step = sum(layer_flops(T, n, m, r) for _, n, m in linears)
-    workload = {"workload": "configs[1]: LLaMA-7B projection set (q,k,v,o,gate,up,down), tokens=4096, rank=64, top-k=256",
+    workload = {"workload": "configs[1]: LLaMA-7B projection set (q,k,v,o,gate,up,down), tokens=4096, rank=64, top-k=256"
+                            + ("" if args.only is None else f" -- RESTRICTED to '{args.only}' (profiling aid, not a bench line)"),
                 "tokens": T, "rank": r, "topk": k, "matrices": len(linears), "gflop_per_step": flops_step / 1e9,
                 "l2": "inputs larger than L2 (0.85 GB touched per step)", "parallelism": f"replicas x{world}"}
 
