@@ -138,6 +138,24 @@ int falqon_melded_backward(const falqon_layer *L, const void *dY, falqon_dtype d
 int falqon_proxy_update(const falqon_layer *L, const float *dB, float lr, int64_t k, int32_t *idx_out,
                         void *ws, size_t ws_bytes, falqon_stream stream);
 
+/* The proxy update for callers that cannot provide a workspace.  The paper has no counterpart: this
+ * is the same operation as falqon_proxy_update, with the same arguments minus the workspace, for code
+ * that runs as a guest inside another runtime (a framework's custom-op hook, a server's plug-in) whose
+ * allocator already owns the device's memory: such a guest has nothing to allocate from, and a
+ * cudaMalloc of its own would fail or stall the whole device mid-step.  The scratch (row scores and
+ * the selected-row list) is a fixed 128 KB array inside the library image, resident on every GPU that
+ * loads the library until the process exits.
+ *   - Limit: L->m <= FALQON_STATIC_MAX_ROWS, otherwise FALQON_ERR_UNSUPPORTED and nothing is launched.
+ *   - The first call on each device looks up the array's device address (that device must be current);
+ *     make that first call outside any stream capture.  Nothing is allocated or freed, ever.
+ *   - All calls on a device share the array, which keeps the previous call's contents; nothing needs to
+ *     start at zero, but calls whose kernels overlap on the GPU race on it: order them on one stream
+ *     or with events.
+ *   - The row scores are not exposed (there is no workspace region to read them from). */
+#define FALQON_STATIC_MAX_ROWS 16384
+int falqon_proxy_update_static(const falqon_layer *L, const float *dB, float lr, int64_t k, int32_t *idx_out,
+                               falqon_stream stream);
+
 /* Synchronizes `stream`, then returns and clears the device status word of the current device:
  * FALQON_OK, FALQON_ERR_TIMEOUT (a bounded device-side wait ran out; results of that call are
  * undefined) or FALQON_ERR_CUDA (the synchronize itself failed). */

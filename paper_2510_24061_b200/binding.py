@@ -22,7 +22,8 @@ WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE, WS_DB_PART = range(6)
 
 EXPORTS = ["falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_last_device_status", "falqon_launch_count",
-           "falqon_profile_start", "falqon_profile_stop"]
+           "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static"]
+STATIC_MAX_ROWS = 16384
 STAGES = ["quant_x", "gemm_fwd", "quant_dy", "quant_oa", "gemm_dx", "gemm_db", "reduce_db", "sgd_score", "topk", "merge"]
 
 if not os.path.exists(LIB_PATH):
@@ -49,6 +50,8 @@ lib.falqon_melded_backward.restype = _i
 lib.falqon_melded_backward.argtypes = [C.POINTER(falqon_layer), _p, _i, _i64, _p, _p, _p, _i, _p, _p, _p, _sz, _p]
 lib.falqon_proxy_update.restype = _i
 lib.falqon_proxy_update.argtypes = [C.POINTER(falqon_layer), _p, _f, _i64, _p, _p, _sz, _p]
+lib.falqon_proxy_update_static.restype = _i
+lib.falqon_proxy_update_static.argtypes = [C.POINTER(falqon_layer), _p, _f, _i64, _p, _p]
 lib.falqon_last_device_status.restype = _i
 lib.falqon_last_device_status.argtypes = [_p]
 lib.falqon_profile_start.restype = _i
@@ -229,3 +232,16 @@ def setup_layer(W: torch.Tensor, A: torch.Tensor, B: torch.Tensor | None, gamma:
         dbuf.copy_(B.to(torch.float32))
         proxy_update(layer, None, 0.0, m)
     return layer
+
+
+def proxy_update_static(layer: Layer, dB: torch.Tensor | None, lr: float, k: int, idx_out: torch.Tensor | None = None):
+    """falqon_proxy_update_static: the proxy update for callers that cannot supply a workspace (guests
+    of a runtime whose allocator owns the device's memory).  Scratch is a fixed array inside the
+    library, so layer.m may not exceed STATIC_MAX_ROWS, calls must not overlap on the GPU, and the
+    first call on a device should be made outside any stream capture.  The caller still passes every
+    input and output; here idx_out is created with torch only when the caller gave none."""
+    if idx_out is None and 0 < k <= layer.m:
+        idx_out = torch.empty(k, dtype=torch.int32, device=layer.wq.device)
+    _check("falqon_proxy_update_static",
+           lib.falqon_proxy_update_static(C.byref(layer.c), _ptr(dB), lr, k, _ptr(idx_out), _stream()))
+    return idx_out
