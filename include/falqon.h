@@ -95,8 +95,10 @@ int falqon_workspace_region(int64_t m, int64_t n, int64_t r, int64_t T_max, falq
  *   dst        device [rows][cols] uint8 codes
  *   scale_out  device [1] or [rows], nullable when scale_in is given
  *   amax_out   device [1] or [rows], nullable
- *   ws         device scratch of at least 256 bytes (used only for per-tensor absmax scaling)
+ *   ws         device scratch of at least FALQON_QUANTIZE_WS_BYTES (per-tensor mode with an absmax only);
+ *              it needs no initialisation
  * amax == 0 gives scale 1.  NaN inputs are outside the contract. */
+#define FALQON_QUANTIZE_WS_BYTES 8192
 int falqon_quantize(const void *src, falqon_dtype src_dt, int64_t rows, int64_t cols, falqon_fp8 fmt,
                     falqon_gran gran, const float *scale_in, float premul, uint8_t *dst,
                     float *scale_out, float *amax_out, void *ws, size_t ws_bytes, falqon_stream stream);

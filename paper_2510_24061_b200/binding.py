@@ -159,7 +159,7 @@ def quantize(src: torch.Tensor, fmt: int, gran: int = PER_TENSOR, scale_in: torc
         dst = torch.empty((rows, cols), dtype=torch.uint8, device=dev)
     scale_out = torch.empty(groups, dtype=torch.float32, device=dev)
     amax_out = torch.empty(groups, dtype=torch.float32, device=dev) if want_amax else None
-    ws = torch.empty(256, dtype=torch.uint8, device=dev)
+    ws = torch.empty(8192, dtype=torch.uint8, device=dev)
     _check("falqon_quantize", lib.falqon_quantize(_ptr(src), _dt(src), rows, cols, fmt, gran, _ptr(scale_in), premul,
                                                   _ptr(dst), _ptr(scale_out), _ptr(amax_out), _ptr(ws), ws.numel(),
                                                   _stream()))

@@ -30,7 +30,9 @@ struct WorkspaceLayout {
   int splits;
 };
 
-constexpr size_t kHeaderBytes = 1024;
+constexpr size_t kHeaderBytes = 8192;     // scales at 0, absmax partials at kPartialsOffset
+constexpr size_t kPartialsOffset = 1024;
+static_assert(kPartialsOffset + kMaxAbsmaxParts * sizeof(uint32_t) <= kHeaderBytes, "header too small");
 
 bool shape_ok(int64_t m, int64_t n, int64_t r) {
   return m >= 16 && n >= 16 && m % 16 == 0 && n % 16 == 0 && r >= 8 && r <= 256 && r % 8 == 0 &&
@@ -141,19 +143,25 @@ int falqon_quantize(const void* src, falqon_dtype src_dt, int64_t rows, int64_t 
     return FALQON_OK;
   }
   const int64_t count = rows * cols;
-  if (scale_in != nullptr) {
-    if (amax_out != nullptr) {
-      if (ws == nullptr || ws_bytes < 256) return FALQON_ERR_WORKSPACE;
-      FALQON_CUDA(launch_absmax(src, src_dt, count, premul, static_cast<uint32_t*>(ws), stream));
-      FALQON_CUDA(cudaMemcpyAsync(amax_out, ws, sizeof(float), cudaMemcpyDeviceToDevice, stream));
-    }
-    FALQON_CUDA(launch_cast_per_tensor(src, src_dt, count, fmt, premul, scale_in, false, dst, scale_out, nullptr, stream));
+  int nparts = 0;
+  if (scale_in != nullptr && amax_out == nullptr) {
+    FALQON_CUDA(launch_cast_per_tensor(src, src_dt, count, fmt, premul, nullptr, 0, scale_in, dst, scale_out, nullptr,
+                                       nullptr, nullptr, stream));
     return FALQON_OK;
   }
-  if (ws == nullptr || ws_bytes < 256 || !aligned16(ws)) return FALQON_ERR_WORKSPACE;
-  FALQON_CUDA(launch_absmax(src, src_dt, count, premul, static_cast<uint32_t*>(ws), stream));
-  FALQON_CUDA(launch_cast_per_tensor(src, src_dt, count, fmt, premul, static_cast<const float*>(ws), true, dst, scale_out,
-                                     amax_out, stream));
+  if (ws == nullptr || ws_bytes < FALQON_QUANTIZE_WS_BYTES || !aligned16(ws)) return FALQON_ERR_WORKSPACE;
+  uint32_t* partial = static_cast<uint32_t*>(ws);
+  FALQON_CUDA(launch_absmax(src, src_dt, count, premul, partial, &nparts, stream));
+  if (scale_in != nullptr) {
+    // given scale, but the caller also wants the absmax: a cast from the partials yields it; then the real cast
+    FALQON_CUDA(launch_cast_per_tensor(src, src_dt, count, fmt, premul, partial, nparts, nullptr, dst, nullptr, nullptr,
+                                       amax_out, nullptr, stream));
+    FALQON_CUDA(launch_cast_per_tensor(src, src_dt, count, fmt, premul, nullptr, 0, scale_in, dst, scale_out, nullptr,
+                                       nullptr, nullptr, stream));
+    return FALQON_OK;
+  }
+  FALQON_CUDA(launch_cast_per_tensor(src, src_dt, count, fmt, premul, partial, nparts, nullptr, dst, scale_out, nullptr,
+                                     amax_out, nullptr, stream));
   return FALQON_OK;
 }
 
@@ -172,16 +180,16 @@ int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_d
   uint8_t* xq = base + w.act8;
   const int64_t m = L->m, n = L->n, r = L->r;
 
-  // S1: x~, s_x = Q_e4m3(X)
+  // S1: x~, s_x = Q_e4m3(X); the cast also clears amax(O_A), which the product's epilogue accumulates
+  uint32_t* partial = reinterpret_cast<uint32_t*>(base + w.scales + kPartialsOffset);
   {
     StageTimer timer(FALQON_STAGE_QUANT_X, stream);
-    FALQON_CUDA(launch_absmax(X, x_dt, T * n, 1.0f, reinterpret_cast<uint32_t*>(scales + 0), stream));
-    FALQON_CUDA(launch_cast_per_tensor(X, x_dt, T * n, kE4M3, 1.0f, scales + 0, true, xq, scales + 1, nullptr, stream));
+    int nparts = 0;
+    FALQON_CUDA(launch_absmax(X, x_dt, T * n, 1.0f, partial, &nparts, stream));
+    FALQON_CUDA(launch_cast_per_tensor(X, x_dt, T * n, kE4M3, 1.0f, partial, nparts, nullptr, xq, scales + 1, s_x_out,
+                                       scales + 0, amax_oa, stream));
   }
-  if (s_x_out != nullptr)
-    FALQON_CUDA(cudaMemcpyAsync(s_x_out, scales + 1, sizeof(float), cudaMemcpyDeviceToDevice, stream));
   // S2: [Y | O_A] = x~ W~'^T / (s_W s_x), amax(O_A) from the epilogue
-  FALQON_CUDA(cudaMemsetAsync(amax_oa, 0, sizeof(float), stream));
   GemmProblem g{};
   g.M = T; g.N = m + r; g.K = n;
   g.a = xq; g.lda = n; g.a_mn_major = false; g.a_fmt = kE4M3;
@@ -217,18 +225,18 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
   const int64_t m = L->m, n = L->n, r = L->r;
 
   // S3: g~, s_g = Q_e5m2(dY)
+  uint32_t* partial = reinterpret_cast<uint32_t*>(base + w.scales + kPartialsOffset);
   {
     StageTimer timer(FALQON_STAGE_QUANT_DY, stream);
-    FALQON_CUDA(launch_absmax(dY, dy_dt, T * m, 1.0f, reinterpret_cast<uint32_t*>(scales + 2), stream));
-    FALQON_CUDA(launch_cast_per_tensor(dY, dy_dt, T * m, kE5M2, 1.0f, scales + 2, true, gq, scales + 3, nullptr, stream));
+    int nparts = 0;
+    FALQON_CUDA(launch_absmax(dY, dy_dt, T * m, 1.0f, partial, &nparts, stream));
+    FALQON_CUDA(launch_cast_per_tensor(dY, dy_dt, T * m, kE5M2, 1.0f, partial, nparts, nullptr, gq, scales + 3, s_g_out,
+                                       scales + 2, nullptr, stream));
   }
-  if (s_g_out != nullptr)
-    FALQON_CUDA(cudaMemcpyAsync(s_g_out, scales + 3, sizeof(float), cudaMemcpyDeviceToDevice, stream));
   // S5a: O~_A, s_OA = Q_e4m3(O_A), written transposed for the dB product
-  FALQON_CUDA(cudaMemcpyAsync(scales + 4, amax_oa, sizeof(float), cudaMemcpyDeviceToDevice, stream));
   {
     StageTimer timer(FALQON_STAGE_QUANT_OA, stream);
-    FALQON_CUDA(launch_quantize_oa_transposed(OA, amax_oa, T, r, w.r16, w.t16, oaq_t, scales + 5, stream));
+    FALQON_CUDA(launch_quantize_oa_transposed(OA, amax_oa, T, r, w.r16, w.t16, oaq_t, scales + 5, scales + 4, stream));
   }
   // S4: dX = g~ W~ / (s_W s_g)   (contraction over the m output channels; W~ read MN-major)
   if (dX != nullptr) {
@@ -283,14 +291,12 @@ int falqon_proxy_update(const falqon_layer* L, const float* dB, float lr, int64_
   if (k > 0) {
     {
       StageTimer timer(FALQON_STAGE_TOPK, stream);
-      FALQON_CUDA(launch_topk(score, m, k, sel, nullptr, stream));
+      FALQON_CUDA(launch_topk(score, m, k, sel, idx_out, stream));
     }
     {
       StageTimer timer(FALQON_STAGE_MERGE, stream);
       FALQON_CUDA(launch_merge_rows(L->wq, L->dbuf, sel, k, m, n, r, stream));
     }
-    if (idx_out != nullptr)
-      FALQON_CUDA(cudaMemcpyAsync(idx_out, sel, static_cast<size_t>(k) * sizeof(int32_t), cudaMemcpyDeviceToDevice, stream));
   }
   return FALQON_OK;
 }

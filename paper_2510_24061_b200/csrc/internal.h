@@ -13,19 +13,23 @@ constexpr int kBF16 = 0, kF32 = 1;
 inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
 
 // ---- quantize.cu
-// amax_bits: device word holding the running max of |x| as an fp32 bit pattern (cleared by the call).
-cudaError_t launch_absmax(const void* src, int src_dt, int64_t count, float premul, uint32_t* amax_bits,
+constexpr int kMaxAbsmaxParts = 148 * 8;   // upper bound of the absmax grid = number of partial maxima
+// Pass 1 of per-tensor absmax scaling: one partial max (fp32 bit pattern of |x|) per CTA into partial[0..*nparts).
+cudaError_t launch_absmax(const void* src, int src_dt, int64_t count, float premul, uint32_t* partial, int* nparts,
                           cudaStream_t stream);
-// Cast with scale = fp8max / *amax (from_amax) or = *scale_ptr.  Also writes scale_out / amax_out if non-null.
+// Pass 2: cast with scale = fp8max / max(partial[0..nparts)) when nparts > 0, else with *scale_in.  Writes the
+// scale to scale_out / scale_out2 and the absmax to amax_out when non-null; sets *clear_word = 0 when non-null.
 cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, int fmt, float premul,
-                                   const float* amax_or_scale, bool from_amax, uint8_t* dst, float* scale_out,
-                                   float* amax_out, cudaStream_t stream);
+                                   const uint32_t* partial, int nparts, const float* scale_in, uint8_t* dst,
+                                   float* scale_out, float* scale_out2, float* amax_out, float* clear_word,
+                                   cudaStream_t stream);
 cudaError_t launch_quantize_per_row(const void* src, int src_dt, int64_t rows, int64_t cols, int fmt, float premul,
                                     const float* scale_in, uint8_t* dst, float* scale_out, float* amax_out,
                                     cudaStream_t stream);
-// O_A [T][r] fp32 -> E4M3 codes written transposed as [r16][ldt] with s_OA = 448 / *amax_oa.
+// O_A [T][r] fp32 -> E4M3 codes written transposed as [r16][ldt] with s_OA = 448 / *amax_oa; *amax_copy = *amax_oa.
 cudaError_t launch_quantize_oa_transposed(const float* oa, const float* amax_oa, int64_t T, int64_t r, int64_t r16,
-                                          int64_t ldt, uint8_t* oaq_t, float* s_oa_out, cudaStream_t stream);
+                                          int64_t ldt, uint8_t* oaq_t, float* s_oa_out, float* amax_copy,
+                                          cudaStream_t stream);
 
 // ---- gemm_fp8.cu
 struct GemmProblem {
@@ -49,9 +53,9 @@ cudaError_t launch_reduce_db(const float* partials, int splits, int64_t count, c
                              float* dB, cudaStream_t stream);
 cudaError_t launch_sgd_score(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, float* score,
                              cudaStream_t stream);
-// scratch: at least topk_scratch_bytes(m).  idx (device [k], ascending) is always written to sel_idx.
+// The k selected rows (ascending) are written to sel_idx and, when idx_copy is non-null, to idx_copy (int32 [k]).
 size_t topk_scratch_bytes(int64_t m);
-cudaError_t launch_topk(const float* score, int64_t m, int64_t k, int32_t* sel_idx, void* scratch, cudaStream_t stream);
+cudaError_t launch_topk(const float* score, int64_t m, int64_t k, int32_t* sel_idx, void* idx_copy, cudaStream_t stream);
 cudaError_t launch_merge_rows(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
                               int64_t r, cudaStream_t stream);
 

@@ -1,7 +1,7 @@
 // Q_fp8 kernels (Eq. quantize of the paper): absmax reduction, scale = fp8max / amax, saturating
 // round-to-nearest-even cast to E4M3 / E5M2.  HBM-bound: 128-bit loads and stores, warp-shuffle
-// reductions, one atomicMax per CTA on the bit pattern of |x| (max is order-free, so the result is
-// bit-exact whatever the schedule).
+// reductions, one partial maximum per CTA on the bit pattern of |x| (max is order-free, so the result
+// is bit-exact whatever the schedule; nothing has to be cleared between calls).
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -83,10 +83,11 @@ __device__ __forceinline__ uint32_t block_max_u32(uint32_t v, uint32_t* smem /* 
   return out;
 }
 
-// ---- pass 1: running max of |premul * x| into *amax_bits (must be 0 on entry)
+// ---- pass 1: max of |premul * x| per CTA, written to partial[blockIdx.x] (no atomics, nothing to
+// clear beforehand; the consumer takes the max over the gridDim.x partials)
 template <int kDt>
 __global__ void __launch_bounds__(kThreads) absmax_kernel(const void* __restrict__ src, int64_t count, float premul,
-                                                          bool use_premul, uint32_t* __restrict__ amax_bits) {
+                                                          bool use_premul, uint32_t* __restrict__ partial) {
   __shared__ uint32_t red[32];
   const int64_t nvec = count / 16;
   uint32_t m = 0;
@@ -103,20 +104,37 @@ __global__ void __launch_bounds__(kThreads) absmax_kernel(const void* __restrict
     }
   }
   m = block_max_u32(m, red);
-  if (threadIdx.x == 0 && m != 0) atomicMax(amax_bits, m);
+  if (threadIdx.x == 0) partial[blockIdx.x] = m;
 }
 
-// ---- pass 2: cast with one scale for the whole tensor
+// ---- pass 2: cast with one scale for the whole tensor.  nparts > 0: the scale comes from the max of
+// the absmax partials; nparts == 0: *scale_in is used as given.
+struct CastOutputs {
+  float* scale_out;    // nullable: receives the scale
+  float* scale_out2;   // nullable: second copy of the scale (the caller's own output pointer)
+  float* amax_out;     // nullable: receives the absmax (only when it was computed)
+  float* clear_word;   // nullable: set to 0 (the next kernel accumulates a max into it)
+};
 template <int kDt, int kFmt>
 __global__ void __launch_bounds__(kThreads) cast_kernel(const void* __restrict__ src, int64_t count, float premul,
-                                                        bool use_premul, const float* __restrict__ amax_or_scale,
-                                                        bool from_amax, uint8_t* __restrict__ dst,
-                                                        float* __restrict__ scale_out, float* __restrict__ amax_out) {
-  const float in = *amax_or_scale;
-  const float s = from_amax ? scale_from_amax(in, kFmt) : in;
+                                                        bool use_premul, const uint32_t* __restrict__ partial, int nparts,
+                                                        const float* __restrict__ scale_in, uint8_t* __restrict__ dst,
+                                                        CastOutputs out) {
+  __shared__ uint32_t red[32];
+  float s, amax = 0.0f;
+  if (nparts > 0) {
+    uint32_t mb = 0;
+    for (int i = threadIdx.x; i < nparts; i += kThreads) mb = max(mb, partial[i]);
+    amax = __uint_as_float(block_max_u32(mb, red));
+    s = scale_from_amax(amax, kFmt);
+  } else {
+    s = *scale_in;
+  }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
-    if (scale_out) *scale_out = s;
-    if (amax_out && from_amax) *amax_out = in;
+    if (out.scale_out) *out.scale_out = s;
+    if (out.scale_out2) *out.scale_out2 = s;
+    if (out.amax_out && nparts > 0) *out.amax_out = amax;
+    if (out.clear_word) *out.clear_word = 0.0f;
   }
   const int64_t nvec = count / 16;
   for (int64_t v = blockIdx.x * (int64_t)kThreads + threadIdx.x; v < nvec; v += (int64_t)gridDim.x * kThreads) {
@@ -167,26 +185,47 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const void* __r
   }
 }
 
-// ---- O_A [T][r] fp32 -> E4M3 codes, transposed to [r][ldt] so the dB product reads it K-major
-constexpr int kOaTileT = 64;
+// ---- O_A [T][r] fp32 -> E4M3 codes, transposed to [r][ldt] so the dB product reads it K-major.
+// A CTA converts 32 tokens x r: float4 loads along r, byte transposition through shared memory,
+// 16-byte stores along the tokens.
+constexpr int kOaTileT = 32;
 __global__ void __launch_bounds__(256) quantize_oa_transposed_kernel(const float* __restrict__ oa,
                                                                      const float* __restrict__ amax_oa, int64_t T, int r,
                                                                      int64_t ldt, uint8_t* __restrict__ oaq_t,
-                                                                     float* __restrict__ s_oa_out) {
-  __shared__ uint8_t tile[256][kOaTileT + 16];
-  const float s = scale_from_amax(*amax_oa, kE4M3);
-  if (blockIdx.x == 0 && threadIdx.x == 0 && s_oa_out) *s_oa_out = s;
+                                                                     float* __restrict__ s_oa_out,
+                                                                     float* __restrict__ amax_copy) {
+  __shared__ __align__(16) uint8_t tile[256][kOaTileT + 16];
+  const float amax = *amax_oa;
+  const float s = scale_from_amax(amax, kE4M3);
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    if (s_oa_out) *s_oa_out = s;
+    if (amax_copy) *amax_copy = amax;
+  }
   const int64_t t0 = (int64_t)blockIdx.x * kOaTileT;
   const int tcount = static_cast<int>(min((int64_t)kOaTileT, T - t0));
-  for (int e = threadIdx.x; e < tcount * r; e += blockDim.x) {
-    const int tl = e / r, j = e - tl * r;
-    const float x = oa[(t0 + tl) * r + j];
-    tile[j][tl] = static_cast<uint8_t>(cvt_fp8x2<kE4M3>(__fmul_rn(x, s), 0.0f) & 0xFF);
+  const int r4 = r >> 2;                       // r is a multiple of 8
+  const int tx = threadIdx.x % r4, ty = threadIdx.x / r4;
+  const int rows_per_pass = blockDim.x / r4;
+  if (ty < rows_per_pass) {
+    for (int tl = ty; tl < kOaTileT; tl += rows_per_pass) {
+      uint32_t codes = 0;
+      if (tl < tcount) {
+        const float4 x = __ldg(reinterpret_cast<const float4*>(oa + (t0 + tl) * r) + tx);
+        codes = cvt_fp8x4<kE4M3>(__fmul_rn(x.x, s), __fmul_rn(x.y, s), __fmul_rn(x.z, s), __fmul_rn(x.w, s));
+      }
+      tile[4 * tx + 0][tl] = static_cast<uint8_t>(codes);
+      tile[4 * tx + 1][tl] = static_cast<uint8_t>(codes >> 8);
+      tile[4 * tx + 2][tl] = static_cast<uint8_t>(codes >> 16);
+      tile[4 * tx + 3][tl] = static_cast<uint8_t>(codes >> 24);
+    }
   }
   __syncthreads();
-  for (int e = threadIdx.x; e < r * kOaTileT; e += blockDim.x) {
-    const int j = e / kOaTileT, tl = e - j * kOaTileT;
-    if (tl < tcount) oaq_t[(int64_t)j * ldt + t0 + tl] = tile[j][tl];
+  // each row j of the tile is 32 bytes = two 16-byte stores (tokens beyond T are zero codes and land in
+  // the padding of the row pitch, which is a multiple of 16, or are skipped at the very end)
+  for (int e = threadIdx.x; e < r * 2; e += blockDim.x) {
+    const int j = e >> 1, half = e & 1;
+    if (t0 + half * 16 < ldt)
+      *reinterpret_cast<uint4*>(oaq_t + (int64_t)j * ldt + t0 + half * 16) = *reinterpret_cast<const uint4*>(&tile[j][half * 16]);
   }
 }
 
@@ -199,24 +238,27 @@ inline int grid_for(int64_t nvec) {
 
 }  // namespace
 
-cudaError_t launch_absmax(const void* src, int src_dt, int64_t count, float premul, uint32_t* amax_bits,
+int absmax_grid(int64_t count) { return grid_for(count / 16); }
+
+cudaError_t launch_absmax(const void* src, int src_dt, int64_t count, float premul, uint32_t* partial, int* nparts,
                           cudaStream_t stream) {
-  cudaError_t e = cudaMemsetAsync(amax_bits, 0, sizeof(uint32_t), stream);
-  if (e != cudaSuccess) return e;
-  const int grid = grid_for(count / 16);
+  const int grid = absmax_grid(count);
+  *nparts = grid;
   const bool use_premul = premul != 1.0f;
-  if (src_dt == kBF16) absmax_kernel<kBF16><<<grid, kThreads, 0, stream>>>(src, count, premul, use_premul, amax_bits);
-  else absmax_kernel<kF32><<<grid, kThreads, 0, stream>>>(src, count, premul, use_premul, amax_bits);
+  if (src_dt == kBF16) absmax_kernel<kBF16><<<grid, kThreads, 0, stream>>>(src, count, premul, use_premul, partial);
+  else absmax_kernel<kF32><<<grid, kThreads, 0, stream>>>(src, count, premul, use_premul, partial);
   return cudaGetLastError();
 }
 
 cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, int fmt, float premul,
-                                   const float* amax_or_scale, bool from_amax, uint8_t* dst, float* scale_out,
-                                   float* amax_out, cudaStream_t stream) {
+                                   const uint32_t* partial, int nparts, const float* scale_in, uint8_t* dst,
+                                   float* scale_out, float* scale_out2, float* amax_out, float* clear_word,
+                                   cudaStream_t stream) {
   const int grid = grid_for(count / 16);
   const bool up = premul != 1.0f;
+  const CastOutputs out{scale_out, scale_out2, amax_out, clear_word};
 #define FALQON_CAST(DT, FMT) \
-  cast_kernel<DT, FMT><<<grid, kThreads, 0, stream>>>(src, count, premul, up, amax_or_scale, from_amax, dst, scale_out, amax_out)
+  cast_kernel<DT, FMT><<<grid, kThreads, 0, stream>>>(src, count, premul, up, partial, nparts, scale_in, dst, out)
   if (src_dt == kBF16) { if (fmt == kE4M3) FALQON_CAST(kBF16, kE4M3); else FALQON_CAST(kBF16, kE5M2); }
   else { if (fmt == kE4M3) FALQON_CAST(kF32, kE4M3); else FALQON_CAST(kF32, kE5M2); }
 #undef FALQON_CAST
@@ -237,10 +279,12 @@ cudaError_t launch_quantize_per_row(const void* src, int src_dt, int64_t rows, i
 }
 
 cudaError_t launch_quantize_oa_transposed(const float* oa, const float* amax_oa, int64_t T, int64_t r, int64_t r16,
-                                          int64_t ldt, uint8_t* oaq_t, float* s_oa_out, cudaStream_t stream) {
+                                          int64_t ldt, uint8_t* oaq_t, float* s_oa_out, float* amax_copy,
+                                          cudaStream_t stream) {
   (void)r16;
   const int grid = static_cast<int>((T + kOaTileT - 1) / kOaTileT);
-  quantize_oa_transposed_kernel<<<grid, 256, 0, stream>>>(oa, amax_oa, T, static_cast<int>(r), ldt, oaq_t, s_oa_out);
+  quantize_oa_transposed_kernel<<<grid, 256, 0, stream>>>(oa, amax_oa, T, static_cast<int>(r), ldt, oaq_t, s_oa_out,
+                                                          amax_copy);
   return cudaGetLastError();
 }
 

@@ -49,11 +49,11 @@ def test_bad_arguments_are_rejected_on_the_host(fq):
     big = 1 << 40
     inv, wsp = fq.ERR_INVALID_ARG, fq.ERR_WORKSPACE
     # quantize
-    assert lib.falqon_quantize(None, 0, 4, 16, 0, 0, None, 1.0, fake, fake, None, fake, 256, None) == inv
-    assert lib.falqon_quantize(fake, 0, 4, 20, 0, 0, None, 1.0, fake, fake, None, fake, 256, None) == inv   # cols % 16
-    assert lib.falqon_quantize(fake, 0, 4, 16, 7, 0, None, 1.0, fake, fake, None, fake, 256, None) == inv   # format
-    assert lib.falqon_quantize(fake + 4, 0, 4, 16, 0, 0, None, 1.0, fake, fake, None, fake, 256, None) == inv  # alignment
-    assert lib.falqon_quantize(fake, 0, 4, 16, 0, 0, None, 1.0, fake, None, None, fake, 256, None) == inv   # nowhere to put the scale
+    assert lib.falqon_quantize(None, 0, 4, 16, 0, 0, None, 1.0, fake, fake, None, fake, 8192, None) == inv
+    assert lib.falqon_quantize(fake, 0, 4, 20, 0, 0, None, 1.0, fake, fake, None, fake, 8192, None) == inv   # cols % 16
+    assert lib.falqon_quantize(fake, 0, 4, 16, 7, 0, None, 1.0, fake, fake, None, fake, 8192, None) == inv   # format
+    assert lib.falqon_quantize(fake + 4, 0, 4, 16, 0, 0, None, 1.0, fake, fake, None, fake, 8192, None) == inv  # alignment
+    assert lib.falqon_quantize(fake, 0, 4, 16, 0, 0, None, 1.0, fake, None, None, fake, 8192, None) == inv   # nowhere to put the scale
     assert lib.falqon_quantize(fake, 0, 4, 16, 0, 0, None, 1.0, fake, fake, None, None, 0, None) == wsp
     # forward
     assert lib.falqon_melded_forward(None, fake, 0, 16, fake, 0, fake, fake, None, fake, big, None) == inv
