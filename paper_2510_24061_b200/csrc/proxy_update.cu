@@ -52,11 +52,12 @@ __global__ void __launch_bounds__(256) sgd_score_kernel(float* __restrict__ dbuf
 }
 
 // ---- top-k rows by score (scores are >= +0, so their bit patterns order like the values):
-// radix select of the k-th largest value (4 passes of 8 bits, histogram in shared memory, the digit
-// found with a parallel suffix scan), then an index-ordered compaction that takes every score above
-// it and the lowest-index rows among the ties.  One CTA; output ascending, written to sel_idx and,
-// when given, to idx_out.
+// radix select of the k-th largest value (4 passes of 8 bits), then an index-ordered compaction that
+// takes every score above it and the lowest-index rows among the ties.  One CTA.  Thread t owns the
+// contiguous rows [t*E, (t+1)*E), so thread order is index order and the compaction needs only two
+// CTA-wide scans of per-thread counts.  Output ascending, written to sel_idx and, when given, idx_out.
 constexpr int kTopkThreads = 1024;
+constexpr int kTopkSmemRows = 48 * 1024;   // scores are staged in shared memory up to this many rows
 
 // Exclusive prefix sum of one int per thread over the whole CTA (1024 threads); *total = CTA sum.
 __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums /* [32] */, int* total) {
@@ -81,141 +82,176 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums /* [32
     if (lane == 31) *total = wi;
   }
   __syncthreads();
-  const int out = warp_sums[warp] + incl - v;
-  __syncthreads();
-  return out;
+  return warp_sums[warp] + incl - v;
 }
 
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restrict__ score, int m, int k,
-                                                            int32_t* __restrict__ sel_idx, int32_t* __restrict__ idx_out) {
-  __shared__ int hist[256];
-  __shared__ int warp_sums[32];
-  __shared__ int s_total;
-  __shared__ uint32_t s_digit, s_remaining;
-  const uint32_t* bits = reinterpret_cast<const uint32_t*>(score);
-  const int tid = threadIdx.x;
+                                                            int32_t* __restrict__ sel_idx, int32_t* __restrict__ idx_out,
+                                                            int use_smem) {
+  extern __shared__ uint32_t s_bits[];          // [m] when use_smem
+  __shared__ int hist[4][256];
+  __shared__ int warp_sums_a[32], warp_sums_b[32];
+  __shared__ int s_total_a, s_total_b;
+  __shared__ uint32_t s_digit[4], s_remaining[4];
+  const uint32_t* gbits = reinterpret_cast<const uint32_t*>(score);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  for (int i = tid; i < 4 * 256; i += kTopkThreads) (&hist[0][0])[i] = 0;
+  if (use_smem)
+    for (int i = tid; i < m; i += kTopkThreads) s_bits[i] = gbits[i];
+  __syncthreads();
+  const uint32_t* bits = use_smem ? s_bits : gbits;
+  const int E = (m + kTopkThreads - 1) / kTopkThreads;
+  const int lo = min(tid * E, m), hi = min(lo + E, m);
 
   uint32_t prefix = 0, mask = 0, remaining = static_cast<uint32_t>(k);
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    if (tid < 256) hist[tid] = 0;
-    __syncthreads();
-    for (int i = tid; i < m; i += kTopkThreads) {
+#pragma unroll
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    for (int i = lo; i < hi; ++i) {
       const uint32_t b = bits[i];
-      if ((b & mask) == prefix) atomicAdd(&hist[(b >> shift) & 0xFF], 1);
+      if ((b & mask) == prefix) atomicAdd(&hist[pass][(b >> shift) & 0xFF], 1);
     }
     __syncthreads();
-    // thread t < 256 owns bin d = 255 - t, so an exclusive scan over t counts the rows in larger bins
-    const int mine = (tid < 256) ? hist[255 - tid] : 0;
-    const int above = block_exclusive_scan(mine, warp_sums, &s_total);
-    if (tid < 256 && static_cast<uint32_t>(above) < remaining && remaining <= static_cast<uint32_t>(above + mine)) {
-      s_digit = static_cast<uint32_t>(255 - tid);
-      s_remaining = remaining - static_cast<uint32_t>(above);
+    if (warp == 0) {
+      // lane l owns bins 255-8l .. 248-8l (descending); find the bin where the running count reaches `remaining`
+      int cnt[8], sum = 0;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) { cnt[q] = hist[pass][255 - (8 * lane + q)]; sum += cnt[q]; }
+      int incl = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      int above = incl - sum;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        if (static_cast<uint32_t>(above) < remaining && remaining <= static_cast<uint32_t>(above + cnt[q])) {
+          s_digit[pass] = static_cast<uint32_t>(255 - (8 * lane + q));
+          s_remaining[pass] = remaining - static_cast<uint32_t>(above);
+        }
+        above += cnt[q];
+      }
     }
     __syncthreads();
-    prefix |= s_digit << shift;
-    remaining = s_remaining;
+    prefix |= s_digit[pass] << shift;
+    remaining = s_remaining[pass];
     mask |= 0xFFu << shift;
-    __syncthreads();
   }
   const uint32_t tau = prefix;                      // bit pattern of the k-th largest score
   const int take_eq = static_cast<int>(remaining);  // how many rows with score == tau are taken
 
-  int run_eq = 0, run_sel = 0;
-  for (int base = 0; base < m; base += kTopkThreads) {
-    const int i = base + tid;
-    const uint32_t b = (i < m) ? bits[i] : 0u;
-    const bool is_gt = (i < m) && b > tau;
-    const bool is_eq = (i < m) && b == tau;
-    const int eq_rank = run_eq + block_exclusive_scan(is_eq ? 1 : 0, warp_sums, &s_total);
-    run_eq += s_total;
-    const bool selected = is_gt || (is_eq && eq_rank < take_eq);
-    __syncthreads();
-    const int pos = run_sel + block_exclusive_scan(selected ? 1 : 0, warp_sums, &s_total);
-    run_sel += s_total;
+  int my_eq = 0;
+  for (int i = lo; i < hi; ++i) my_eq += (bits[i] == tau) ? 1 : 0;
+  int eq_rank = block_exclusive_scan(my_eq, warp_sums_a, &s_total_a);
+  int my_sel = 0;
+  {
+    int e = eq_rank;
+    for (int i = lo; i < hi; ++i) {
+      const uint32_t b = bits[i];
+      if (b > tau) ++my_sel;
+      else if (b == tau) { if (e < take_eq) ++my_sel; ++e; }
+    }
+  }
+  int pos = block_exclusive_scan(my_sel, warp_sums_b, &s_total_b);
+  for (int i = lo; i < hi; ++i) {
+    const uint32_t b = bits[i];
+    bool selected = b > tau;
+    if (b == tau) { selected = eq_rank < take_eq; ++eq_rank; }
     if (selected) {
       sel_idx[pos] = i;
       if (idx_out != nullptr) idx_out[pos] = i;
+      ++pos;
     }
-    __syncthreads();
   }
 }
 
 // ---- W~[i][:] <- sat_rne_e4m3(W~[i][:] + DeltaBuffer[i][:] * A~) for the selected rows.
-// A CTA owns 8 selected rows x 512 columns.  It first stages the r x 512 tile of A~ in shared memory
-// with 16-byte loads that are all in flight together, then each thread runs the fp32 fma chains of
-// 4 rows x 8 columns, so every decoded A~ value feeds four chains.  The chain order (j ascending,
-// seeded with the decoded W~) is fixed.
+// A CTA owns 32 selected rows x 128 columns.  It decodes the r x 128 tile of A~ to fp32 in shared
+// memory once (the FP8 decode is the expensive part, so it is shared by all 32 rows), then each thread
+// runs the fp32 fma chains of 4 rows x 8 columns.  The chain order (j ascending, seeded with the
+// decoded W~) is fixed, so the result is bit-identical to the sequential definition.
 constexpr int kMergeRowsPerThread = 4;
-constexpr int kMergeRowGroups = 2;
-constexpr int kMergeRows = kMergeRowsPerThread * kMergeRowGroups;   // rows per CTA
-constexpr int kMergeColsPerThread = 8;
-constexpr int kMergeTx = 64;
-constexpr int kMergeThreads = kMergeTx * kMergeRowGroups;           // 128
-constexpr int kMergeCols = kMergeTx * kMergeColsPerThread;          // 512 columns per CTA
+constexpr int kMergeTy = 8;
+constexpr int kMergeRows = kMergeRowsPerThread * kMergeTy;          // 32 rows per CTA
+constexpr int kMergeTx = 16;
+constexpr int kMergeThreads = kMergeTx * kMergeTy;                  // 128
+constexpr int kMergeCols = 128;                                     // columns per CTA: thread tx owns 4tx..4tx+3 and 64+4tx..64+4tx+3
 
-__device__ __forceinline__ void decode8(uint2 w, float (&a)[8]) {
-  const float2 p0 = e4m3x2_to_float2(w.x), p1 = e4m3x2_to_float2(w.x >> 16);
-  const float2 p2 = e4m3x2_to_float2(w.y), p3 = e4m3x2_to_float2(w.y >> 16);
-  a[0] = p0.x; a[1] = p0.y; a[2] = p1.x; a[3] = p1.y; a[4] = p2.x; a[5] = p2.y; a[6] = p3.x; a[7] = p3.y;
+__device__ __forceinline__ void decode4(uint32_t w, float (&a)[4]) {
+  const float2 p0 = e4m3x2_to_float2(w), p1 = e4m3x2_to_float2(w >> 16);
+  a[0] = p0.x; a[1] = p0.y; a[2] = p1.x; a[3] = p1.y;
 }
 
 __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __restrict__ wq, const float* __restrict__ dbuf,
                                                                    const int32_t* __restrict__ sel_idx, int k, int64_t m,
                                                                    int64_t n, int r) {
-  extern __shared__ __align__(16) uint8_t merge_smem[];
-  uint8_t* a_tile = merge_smem;                                           // [r][kMergeCols] codes of A~
-  float* sdb = reinterpret_cast<float*>(merge_smem + (size_t)r * kMergeCols);  // [kMergeRows][r]
+  extern __shared__ __align__(16) float merge_smem[];
+  float* a_tile = merge_smem;                         // [r][kMergeCols] decoded A~
+  float* sdb = merge_smem + (size_t)r * kMergeCols;   // [kMergeRows][r]
   __shared__ int srow[kMergeRows];
   const int g0 = blockIdx.y * kMergeRows;
   const int nrows = min(kMergeRows, k - g0);
   const int64_t cta_c0 = (int64_t)blockIdx.x * kMergeCols;
   const int cta_cols = static_cast<int>(min((int64_t)kMergeCols, n - cta_c0));   // multiple of 16
   if (threadIdx.x < kMergeRows) srow[threadIdx.x] = (threadIdx.x < nrows) ? sel_idx[g0 + threadIdx.x] : -1;
-  // stage A~ (rows m.. of W~')
+  // decode A~ (rows m.. of W~') into shared memory; columns beyond the matrix edge become 0
   const uint8_t* aq = wq + m * n + cta_c0;
-  const int vec_per_row = cta_cols / 16;
-  for (int e = threadIdx.x; e < r * vec_per_row; e += kMergeThreads) {
-    const int j = e / vec_per_row, v = e - j * vec_per_row;
-    *reinterpret_cast<uint4*>(a_tile + (size_t)j * kMergeCols + v * 16) =
-        __ldg(reinterpret_cast<const uint4*>(aq + (int64_t)j * n + v * 16));
+  for (int e = threadIdx.x; e < r * (kMergeCols / 16); e += kMergeThreads) {
+    const int j = e / (kMergeCols / 16), v = e % (kMergeCols / 16);
+    uint4 w = make_uint4(0u, 0u, 0u, 0u);
+    if (v * 16 < cta_cols) w = __ldg(reinterpret_cast<const uint4*>(aq + (int64_t)j * n + v * 16));
+    float f[4];
+    float4* dst = reinterpret_cast<float4*>(a_tile + (size_t)j * kMergeCols + v * 16);
+    decode4(w.x, f); dst[0] = make_float4(f[0], f[1], f[2], f[3]);
+    decode4(w.y, f); dst[1] = make_float4(f[0], f[1], f[2], f[3]);
+    decode4(w.z, f); dst[2] = make_float4(f[0], f[1], f[2], f[3]);
+    decode4(w.w, f); dst[3] = make_float4(f[0], f[1], f[2], f[3]);
   }
-  __syncthreads();
+  __syncthreads();   // srow visible
   for (int e = threadIdx.x; e < kMergeRows * r; e += kMergeThreads) {
     const int q = e / r, j = e - q * r;
     sdb[e] = (q < nrows) ? dbuf[(int64_t)srow[q] * r + j] : 0.0f;
   }
   __syncthreads();
   const int tx = threadIdx.x % kMergeTx, ty = threadIdx.x / kMergeTx;
-  const int lc = tx * kMergeColsPerThread;
-  if (lc >= cta_cols) return;
-  const int64_t c0 = cta_c0 + lc;
+  const int lc0 = 4 * tx, lc1 = 64 + 4 * tx;
+  const bool ok0 = lc0 < cta_cols, ok1 = lc1 < cta_cols;
   const int q0 = ty * kMergeRowsPerThread;
-  float v[kMergeRowsPerThread][kMergeColsPerThread];
+  float v[kMergeRowsPerThread][8];
 #pragma unroll
   for (int q = 0; q < kMergeRowsPerThread; ++q) {
-    uint2 w = make_uint2(0u, 0u);
-    if (q0 + q < nrows) w = *reinterpret_cast<const uint2*>(wq + (int64_t)srow[q0 + q] * n + c0);
-    decode8(w, v[q]);
+    uint32_t w0 = 0u, w1 = 0u;
+    if (q0 + q < nrows) {
+      const uint8_t* row = wq + (int64_t)srow[q0 + q] * n + cta_c0;
+      if (ok0) w0 = *reinterpret_cast<const uint32_t*>(row + lc0);
+      if (ok1) w1 = *reinterpret_cast<const uint32_t*>(row + lc1);
+    }
+    float f[4];
+    decode4(w0, f); v[q][0] = f[0]; v[q][1] = f[1]; v[q][2] = f[2]; v[q][3] = f[3];
+    decode4(w1, f); v[q][4] = f[0]; v[q][5] = f[1]; v[q][6] = f[2]; v[q][7] = f[3];
   }
   const float* d0 = sdb + q0 * r;
 #pragma unroll 4
   for (int j = 0; j < r; ++j) {
-    float a[8];
-    decode8(*reinterpret_cast<const uint2*>(a_tile + (size_t)j * kMergeCols + lc), a);
+    const float4 a0 = *reinterpret_cast<const float4*>(a_tile + (size_t)j * kMergeCols + lc0);
+    const float4 a1 = *reinterpret_cast<const float4*>(a_tile + (size_t)j * kMergeCols + lc1);
 #pragma unroll
     for (int q = 0; q < kMergeRowsPerThread; ++q) {
       const float d = d0[q * r + j];
-#pragma unroll
-      for (int c = 0; c < kMergeColsPerThread; ++c) v[q][c] = __fmaf_rn(d, a[c], v[q][c]);
+      v[q][0] = __fmaf_rn(d, a0.x, v[q][0]); v[q][1] = __fmaf_rn(d, a0.y, v[q][1]);
+      v[q][2] = __fmaf_rn(d, a0.z, v[q][2]); v[q][3] = __fmaf_rn(d, a0.w, v[q][3]);
+      v[q][4] = __fmaf_rn(d, a1.x, v[q][4]); v[q][5] = __fmaf_rn(d, a1.y, v[q][5]);
+      v[q][6] = __fmaf_rn(d, a1.z, v[q][6]); v[q][7] = __fmaf_rn(d, a1.w, v[q][7]);
     }
   }
 #pragma unroll
   for (int q = 0; q < kMergeRowsPerThread; ++q) {
     if (q0 + q < nrows) {
-      uint2 o;
-      o.x = cvt_fp8x4<kE4M3>(v[q][0], v[q][1], v[q][2], v[q][3]);
-      o.y = cvt_fp8x4<kE4M3>(v[q][4], v[q][5], v[q][6], v[q][7]);
-      *reinterpret_cast<uint2*>(wq + (int64_t)srow[q0 + q] * n + c0) = o;
+      uint8_t* row = wq + (int64_t)srow[q0 + q] * n + cta_c0;
+      if (ok0) *reinterpret_cast<uint32_t*>(row + lc0) = cvt_fp8x4<kE4M3>(v[q][0], v[q][1], v[q][2], v[q][3]);
+      if (ok1) *reinterpret_cast<uint32_t*>(row + lc1) = cvt_fp8x4<kE4M3>(v[q][4], v[q][5], v[q][6], v[q][7]);
     }
   }
 }
@@ -249,9 +285,18 @@ cudaError_t launch_sgd_score(float* dbuf, const float* dB, float lr, int64_t m, 
 
 size_t topk_scratch_bytes(int64_t m) { (void)m; return 256; }
 
-cudaError_t launch_topk(const float* score, int64_t m, int64_t k, int32_t* sel_idx, void* scratch, cudaStream_t stream) {
-  topk_kernel<<<1, kTopkThreads, 0, stream>>>(score, static_cast<int>(m), static_cast<int>(k), sel_idx,
-                                              static_cast<int32_t*>(scratch));
+cudaError_t launch_topk(const float* score, int64_t m, int64_t k, int32_t* sel_idx, void* idx_copy, cudaStream_t stream) {
+  const int use_smem = m <= kTopkSmemRows ? 1 : 0;
+  const size_t smem = use_smem ? static_cast<size_t>(m) * sizeof(uint32_t) : 0;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t ea = cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(kTopkSmemRows * sizeof(uint32_t)));
+    if (ea != cudaSuccess) return ea;
+    configured = true;
+  }
+  topk_kernel<<<1, kTopkThreads, smem, stream>>>(score, static_cast<int>(m), static_cast<int>(k), sel_idx,
+                                                 static_cast<int32_t*>(idx_copy), use_smem);
   return cudaGetLastError();
 }
 
@@ -259,10 +304,10 @@ cudaError_t launch_merge_rows(uint8_t* wq, float* dbuf, const int32_t* sel_idx, 
                               int64_t r, cudaStream_t stream) {
   dim3 grid(static_cast<unsigned>((n + kMergeCols - 1) / kMergeCols),
             static_cast<unsigned>((k + kMergeRows - 1) / kMergeRows));
-  const size_t smem = static_cast<size_t>(r) * kMergeCols + sizeof(float) * kMergeRows * r;
+  const size_t smem = sizeof(float) * (static_cast<size_t>(r) * kMergeCols + static_cast<size_t>(kMergeRows) * r);
   static bool configured = false;
   if (!configured) {
-    cudaError_t ea = cudaFuncSetAttribute(merge_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    cudaError_t ea = cudaFuncSetAttribute(merge_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 176 * 1024);
     if (ea != cudaSuccess) return ea;
     configured = true;
   }
