@@ -14,6 +14,8 @@
 // Every mbarrier wait is bounded; on a timeout the CTA records it, drains and frees its TMEM.
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -50,6 +52,55 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
+}
+
+// Stores 32 consecutive output columns [col0, col0+32) of one row: columns below n_split go to c0 (bf16 or
+// fp32, 16-byte stores when aligned), the rest up to N go to c1 (fp32) and feed the running |max|.
+__device__ __forceinline__ void epilogue_store32(const GemmParams& p, int row, int col0, int split, const float (&f)[32],
+                                                 uint32_t& amax_bits) {
+  if (col0 + 32 <= p.n_split) {
+    if (p.c0_dt == kBF16) {
+      uint16_t* dst = static_cast<uint16_t*>(p.c0) + (long long)split * p.c0_split_stride + (long long)row * p.ldc0 + col0;
+      if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          uint4 o;
+          o.x = pack_bf16x2(f[8 * i + 0], f[8 * i + 1]);
+          o.y = pack_bf16x2(f[8 * i + 2], f[8 * i + 3]);
+          o.z = pack_bf16x2(f[8 * i + 4], f[8 * i + 5]);
+          o.w = pack_bf16x2(f[8 * i + 6], f[8 * i + 7]);
+          reinterpret_cast<uint4*>(dst)[i] = o;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) dst[i] = static_cast<uint16_t>(pack_bf16x2(f[i], 0.0f) & 0xFFFF);
+      }
+    } else {
+      float* dst = static_cast<float*>(p.c0) + (long long)split * p.c0_split_stride + (long long)row * p.ldc0 + col0;
+      if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          reinterpret_cast<float4*>(dst)[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) dst[i] = f[i];
+      }
+    }
+  } else {
+    // chunk touches the O | O_A boundary or the ragged right edge: element by element
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const int col = col0 + i;
+      if (col < p.n_split) {
+        const long long off = (long long)split * p.c0_split_stride + (long long)row * p.ldc0 + col;
+        if (p.c0_dt == kBF16) static_cast<uint16_t*>(p.c0)[off] = static_cast<uint16_t>(pack_bf16x2(f[i], 0.0f) & 0xFFFF);
+        else static_cast<float*>(p.c0)[off] = f[i];
+      } else if (col < p.N) {
+        p.c1[(long long)row * p.ldc1 + (col - p.n_split)] = f[i];
+        amax_bits = max(amax_bits, __float_as_uint(f[i]) & 0x7FFFFFFFu);
+      }
+    }
+  }
 }
 
 template <bool kAMn, bool kBMn>
@@ -197,49 +248,7 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         float f[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * inv;
-        if (col0 + 32 <= p.n_split) {
-          if (p.c0_dt == kBF16) {
-            uint16_t* dst = static_cast<uint16_t*>(p.c0) + (long long)split * p.c0_split_stride + (long long)row * p.ldc0 + col0;
-            if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                uint4 o;
-                o.x = pack_bf16x2(f[8 * i + 0], f[8 * i + 1]);
-                o.y = pack_bf16x2(f[8 * i + 2], f[8 * i + 3]);
-                o.z = pack_bf16x2(f[8 * i + 4], f[8 * i + 5]);
-                o.w = pack_bf16x2(f[8 * i + 6], f[8 * i + 7]);
-                reinterpret_cast<uint4*>(dst)[i] = o;
-              }
-            } else {
-#pragma unroll
-              for (int i = 0; i < 32; ++i) dst[i] = static_cast<uint16_t>(pack_bf16x2(f[i], 0.0f) & 0xFFFF);
-            }
-          } else {
-            float* dst = static_cast<float*>(p.c0) + (long long)split * p.c0_split_stride + (long long)row * p.ldc0 + col0;
-            if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
-#pragma unroll
-              for (int i = 0; i < 8; ++i)
-                reinterpret_cast<float4*>(dst)[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
-            } else {
-#pragma unroll
-              for (int i = 0; i < 32; ++i) dst[i] = f[i];
-            }
-          }
-        } else {
-          // chunk touches the O | O_A boundary or the ragged right edge: element by element
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int col = col0 + i;
-            if (col < p.n_split) {
-              const long long off = (long long)split * p.c0_split_stride + (long long)row * p.ldc0 + col;
-              if (p.c0_dt == kBF16) static_cast<uint16_t*>(p.c0)[off] = static_cast<uint16_t>(pack_bf16x2(f[i], 0.0f) & 0xFFFF);
-              else static_cast<float*>(p.c0)[off] = f[i];
-            } else if (col < p.N) {
-              p.c1[(long long)row * p.ldc1 + (col - p.n_split)] = f[i];
-              amax_bits = max(amax_bits, __float_as_uint(f[i]) & 0x7FFFFFFFu);
-            }
-          }
-        }
+        epilogue_store32(p, row, col0, split, f, amax_bits);
         }  // row_ok
       }
       tc_fence_before_sync();
@@ -265,6 +274,195 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+
+// ------------------------------------------------------------------ CTA-pair variant (tensor-bound roles)
+// Two CTAs of a cluster compute one 256 x 256 tile with tcgen05.mma cta_group::2: each CTA stages its own
+// 128 rows of A and only HALF of the B tile (128 of the 256 N rows), the hardware shares the B halves
+// between the two tensor cores, and each CTA keeps its 128 accumulator rows in its own TMEM.  Per MMA a
+// CTA now moves (128 + 128) x 32 bytes through shared memory instead of (128 + 256) x 32, which is what
+// lets the tensor pipe run ahead of the shared-memory port, and the smaller stage (32 KB) buys a deeper
+// ring.  The leader CTA (cluster rank 0) issues all MMAs; TMA loads of both CTAs count their bytes on the
+// leader's "full" barrier; MMA completion is multicast to both CTAs' "empty" / "accumulator full"
+// barriers; both CTAs' epilogue warps arrive on the leader's "accumulator empty" barrier.
+// A is K-major; B is K-major or MN-major.  The last N tile is issued with a narrower instruction N.
+constexpr uint32_t kPairStageBytes = kATileBytes + 128 * kBlockKBytes;   // 32 KB per CTA per stage
+
+template <bool kBMn>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                     const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t smem_base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - raw_addr);
+
+  const int S = p.num_stages;
+  const uint32_t bars = smem_base + static_cast<uint32_t>(S) * kPairStageBytes;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (S + s); };
+  auto tmem_full_bar = [&](int a) { return bars + 8u * (2 * S + a); };
+  auto tmem_empty_bar = [&](int a) { return bars + 8u * (2 * S + 2 + a); };
+  const uint32_t slot_off = static_cast<uint32_t>(S) * kPairStageBytes + 8u * (2 * S + 4);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + slot_off);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();       // 0 = leader
+  const bool leader = rank == 0;
+
+  if (threadIdx.x == 0) {
+    prefetch_tensor_map(&tmap_a);
+    prefetch_tensor_map(&tmap_b);
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full_bar(s), 1);      // the leader's arrive.expect_tx; bytes from both CTAs
+      mbar_init(empty_bar(s), 1);     // one multicast commit
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tmem_full_bar(a), 1);   // one multicast commit
+      mbar_init(tmem_empty_bar(a), 8);  // 4 epilogue warps of each CTA
+    }
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_base + slot_off, kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_arrive();      // the peer's barriers must be initialised before anything signals them
+  cluster_wait();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int num_pairs = gridDim.x >> 1;
+  const int pair = blockIdx.x >> 1;
+  const int total_tiles = p.m_tiles * p.n_tiles;   // m_tiles counts 256-row pair tiles here
+  bool aborted = false;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (one lane in each CTA)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int tile = pair; tile < total_tiles && !aborted; tile += num_pairs) {
+        const int n_idx = tile / p.m_tiles;
+        const int m_idx = tile - n_idx * p.m_tiles;
+        const int n0 = n_idx * 256;
+        const int n_inst = min(256, (p.N - n0 + 15) & ~15);        // instruction N of this tile
+        const int row0 = m_idx * 256 + static_cast<int>(rank) * kBlockM;
+        const int bn0 = n0 + static_cast<int>(rank) * (n_inst >> 1);  // this CTA's half of the B rows
+        for (int kb = 0; kb < p.kblocks_total; ++kb) {
+          if (!mbar_wait_cluster(empty_bar(stage), phase ^ 1u, p.status)) { aborted = true; break; }
+          if (leader) mbar_expect_tx(full_bar(stage), 2 * kPairStageBytes);
+          const uint32_t fb = map_to_cta(full_bar(stage), 0);
+          const uint32_t a_dst = smem_base + static_cast<uint32_t>(stage) * kPairStageBytes;
+          const uint32_t b_dst = a_dst + kATileBytes;
+          tma_load_2d_pair(a_dst, &tmap_a, fb, kb * kBlockKBytes, row0);
+          if (!kBMn) tma_load_2d_pair(b_dst, &tmap_b, fb, kb * kBlockKBytes, bn0);
+          else       tma_load_2d_pair(b_dst, &tmap_b, fb, bn0, kb * kBlockKBytes);
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+      }
+      // tail: wait until the MMAs have released every stage, so no completion signal can arrive at a CTA
+      // that has already left
+      for (int i = 0; i < S && !aborted; ++i) {
+        if (!mbar_wait_cluster(empty_bar(stage), phase ^ 1u, p.status)) aborted = true;
+        if (++stage == S) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (one lane of the leader CTA)
+    if (lane == 0 && leader) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      for (int tile = pair; tile < total_tiles && !aborted; tile += num_pairs) {
+        const int n_idx = tile / p.m_tiles;
+        const int n0 = n_idx * 256;
+        const int n_inst = min(256, (p.N - n0 + 15) & ~15);
+        const uint32_t idesc = p.idesc | (static_cast<uint32_t>(n_inst >> 3) << 17);
+        if (!mbar_wait_cluster(tmem_empty_bar(acc), acc_phase ^ 1u, p.status)) { aborted = true; break; }
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * kAccCols;
+        for (int kb = 0; kb < p.kblocks_total; ++kb) {
+          if (!mbar_wait_cluster(full_bar(stage), phase, p.status)) { aborted = true; break; }
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_base + static_cast<uint32_t>(stage) * kPairStageBytes;
+          const uint32_t b_addr = a_addr + kATileBytes;
+#pragma unroll
+          for (int k = 0; k < kBlockKBytes / kUmmaK; ++k) {
+            const uint64_t adesc = make_smem_desc(a_addr + k * kUmmaK, 16, 1024);
+            const uint64_t bdesc = kBMn ? make_smem_desc(b_addr + k * (kUmmaK * 128), kMnChunkBytes, 1024)
+                                        : make_smem_desc(b_addr + k * kUmmaK, 16, 1024);
+            umma_f8_pair(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit_pair(empty_bar(stage), 3);   // frees the stage in both CTAs
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+        if (aborted) break;
+        umma_commit_pair(tmem_full_bar(acc), 3);    // accumulators of both CTAs complete
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5 of each CTA)
+    const int quad = warp & 3;
+    const bool rescale = p.scale_a != nullptr;
+    const float inv = rescale ? 1.0f / (__ldg(p.scale_a) * __ldg(p.scale_b)) : 1.0f;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    uint32_t amax_bits = 0;
+    for (int tile = pair; tile < total_tiles && !aborted; tile += num_pairs) {
+      const int n_idx = tile / p.m_tiles;
+      const int m_idx = tile - n_idx * p.m_tiles;
+      if (!mbar_wait_cluster(tmem_full_bar(acc), acc_phase, p.status)) { aborted = true; break; }
+      tc_fence_after_sync();
+      const int row = m_idx * 256 + static_cast<int>(rank) * kBlockM + quad * 32 + lane;
+      const bool row_ok = row < p.M;
+      const uint32_t t_row = tmem_base + static_cast<uint32_t>(acc) * kAccCols + (static_cast<uint32_t>(quad * 32) << 16);
+      const int n0 = n_idx * 256;
+      for (int c = 0; c < 256; c += 32) {
+        if (n0 + c >= p.N) break;  // warp-uniform
+        uint32_t v[32];
+        __syncwarp();
+        tmem_ld_32x32b_x32(t_row + c, v);
+        tmem_ld_wait();
+        if (row_ok) {
+          float f[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * inv;
+          epilogue_store32(p, row, n0 + c, 0, f, amax_bits);
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(tmem_empty_bar(acc), 0));
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+    if (p.amax1_bits != nullptr) {
+      amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
+      if (lane == 0 && amax_bits != 0) atomicMax(p.amax1_bits, amax_bits);
+    }
+  }
+
+  // ------------------------------------------------------------ common exit
+  if (aborted) {
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 200000ull) { }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_arrive();      // neither CTA frees its TMEM or leaves while the other may still signal it
+  cluster_wait();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
   }
 }
 
@@ -325,6 +523,74 @@ cudaError_t launch_variant(const CUtensorMap& ta, const CUtensorMap& tb, const G
   return cudaGetLastError();
 }
 
+template <bool kBMn>
+cudaError_t launch_pair_variant(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& gp, int grid, size_t smem,
+                                cudaStream_t stream) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_fp8_pair_kernel<kBMn>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(kSmemBudget));
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
+  cfg.blockDim = dim3(kGemmThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_fp8_pair_kernel<kBMn>, ta, tb, gp);
+}
+
+bool pair_kernel_disabled() {
+  // debugging aid: FALQON_DEBUG_GEMM_1CTA=1 routes every product through the single-CTA kernel
+  static const bool off = [] {
+    const char* v = std::getenv("FALQON_DEBUG_GEMM_1CTA");
+    return v != nullptr && v[0] == '1';
+  }();
+  return off;
+}
+
+cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
+  GemmParams gp{};
+  gp.M = static_cast<int>(q.M); gp.N = static_cast<int>(q.N); gp.K = static_cast<int>(q.K);
+  gp.block_n = 256;
+  gp.m_tiles = static_cast<int>((q.M + 255) / 256);
+  gp.n_tiles = static_cast<int>((q.N + 255) / 256);
+  gp.kblocks_total = static_cast<int>((q.K + kBlockKBytes - 1) / kBlockKBytes);
+  gp.k_splits = 1;
+  gp.kblocks_per_split = gp.kblocks_total;
+  int stages = static_cast<int>((kSmemBudget - 1024 - kBarrierBytes) / kPairStageBytes);
+  if (stages > kMaxStages) stages = kMaxStages;
+  gp.num_stages = stages;
+  // instruction descriptor without N (set per tile): fp32 accumulate, formats, B major, M = 256
+  gp.idesc = (1u << 4) | (static_cast<uint32_t>(q.a_fmt) << 7) | (static_cast<uint32_t>(q.b_fmt) << 10) |
+             ((q.b_mn_major ? 1u : 0u) << 16) | (static_cast<uint32_t>(256 >> 4) << 24);
+  gp.c0 = q.c0; gp.ldc0 = q.ldc0; gp.c0_dt = q.c0_dt; gp.n_split = static_cast<int>(q.n_split);
+  gp.c0_split_stride = 0;
+  gp.c1 = q.c1; gp.ldc1 = q.ldc1; gp.amax1_bits = q.amax1_bits;
+  gp.scale_a = q.scale_a; gp.scale_b = q.scale_b;
+  gp.status = q.status;
+  CUtensorMap ta, tb;
+  if (!make_tensor_map(&ta, q.a, q.M, q.K, q.lda, kBlockKBytes, kBlockM)) return cudaErrorInvalidValue;
+  const bool ok = q.b_mn_major ? make_tensor_map(&tb, q.b, q.K, q.N, q.ldb, 128, kBlockKBytes)
+                               : make_tensor_map(&tb, q.b, q.N, q.K, q.ldb, kBlockKBytes, 128);
+  if (!ok) return cudaErrorInvalidValue;
+  const long long total_tiles = static_cast<long long>(gp.m_tiles) * gp.n_tiles;
+  long long pairs = sm_count() / 2;
+  if (total_tiles < pairs) pairs = total_tiles;
+  const int grid = static_cast<int>(pairs * 2);
+  const size_t smem = static_cast<size_t>(stages) * kPairStageBytes + kBarrierBytes + 1024;
+  if (q.b_mn_major) return launch_pair_variant<true>(ta, tb, gp, grid, smem, stream);
+  return launch_pair_variant<false>(ta, tb, gp, grid, smem, stream);
+}
+
 }  // namespace
 
 int gemm_k_splits_for_db(int64_t m, int64_t T) {
@@ -341,6 +607,9 @@ cudaError_t launch_gemm_fp8(const GemmProblem& q, cudaStream_t stream) {
   if (q.M <= 0 || q.N <= 0 || q.K <= 0) return cudaErrorInvalidValue;
   if (q.block_n < 16 || q.block_n > 256 || q.block_n % 16) return cudaErrorInvalidValue;
   if (q.b_mn_major && q.block_n % 128) return cudaErrorInvalidValue;
+  // the tensor-bound roles (K-major A, full-width tiles, no token slabs) run on CTA pairs
+  if (!q.a_mn_major && q.block_n == 256 && q.k_splits <= 1 && q.N % 16 == 0 && !pair_kernel_disabled())
+    return launch_gemm_fp8_pair(q, stream);
 
   GemmParams gp{};
   gp.M = static_cast<int>(q.M); gp.N = static_cast<int>(q.N); gp.K = static_cast<int>(q.K);
