@@ -290,6 +290,15 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 // A is K-major; B is K-major or MN-major.  The last N tile is issued with a narrower instruction N.
 constexpr uint32_t kPairStageBytes = kATileBytes + 128 * kBlockKBytes;   // 32 KB per CTA per stage
 
+// Instruction N of a pair tile with `remaining` valid columns: a multiple of 16 (each CTA supplies N/2 rows of
+// B, a whole number of 8-row swizzle groups); with an MN-major B each half must also start on a 16-byte
+// boundary of the N axis for the TMA copy, so N is a multiple of 32 there.
+template <bool kBMn>
+__device__ __forceinline__ int pair_instr_n(int remaining) {
+  const int gran = kBMn ? 32 : 16;
+  return min(256, (remaining + gran - 1) / gran * gran);
+}
+
 template <bool kBMn>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -351,7 +360,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         const int n_idx = tile / p.m_tiles;
         const int m_idx = tile - n_idx * p.m_tiles;
         const int n0 = n_idx * 256;
-        const int n_inst = min(256, (p.N - n0 + 15) & ~15);        // instruction N of this tile
+        const int n_inst = pair_instr_n<kBMn>(p.N - n0);        // instruction N of this tile
         const int row0 = m_idx * 256 + static_cast<int>(rank) * kBlockM;
         const int bn0 = n0 + static_cast<int>(rank) * (n_inst >> 1);  // this CTA's half of the B rows
         for (int kb = 0; kb < p.kblocks_total; ++kb) {
@@ -383,7 +392,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       for (int tile = pair; tile < total_tiles && !aborted; tile += num_pairs) {
         const int n_idx = tile / p.m_tiles;
         const int n0 = n_idx * 256;
-        const int n_inst = min(256, (p.N - n0 + 15) & ~15);
+        const int n_inst = pair_instr_n<kBMn>(p.N - n0);
         const uint32_t idesc = p.idesc | (static_cast<uint32_t>(n_inst >> 3) << 17);
         if (!mbar_wait_cluster(tmem_empty_bar(acc), acc_phase ^ 1u, p.status)) { aborted = true; break; }
         tc_fence_after_sync();
