@@ -153,19 +153,19 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   bool aborted = false;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      for (int tile = blockIdx.x; tile < total_tiles && !aborted; tile += gridDim.x) {
-        const int split = tile / tiles_per_split;
-        const int rem = tile - split * tiles_per_split;
-        const int n_idx = rem / p.m_tiles;
-        const int m_idx = rem - n_idx * p.m_tiles;
-        const int kb_begin = split * p.kblocks_per_split;
-        const int kb_end = min(kb_begin + p.kblocks_per_split, p.kblocks_total);
-        for (int kb = kb_begin; kb < kb_end; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status)) { aborted = true; break; }
+    // ------------------------------------------------------------ TMA producer (whole warp loops, one lane issues)
+    int stage = 0;
+    uint32_t phase = 0;
+    for (int tile = blockIdx.x; tile < total_tiles && !aborted; tile += gridDim.x) {
+      const int split = tile / tiles_per_split;
+      const int rem = tile - split * tiles_per_split;
+      const int n_idx = rem / p.m_tiles;
+      const int m_idx = rem - n_idx * p.m_tiles;
+      const int kb_begin = split * p.kblocks_per_split;
+      const int kb_end = min(kb_begin + p.kblocks_per_split, p.kblocks_total);
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
+        if (!mbar_wait_warp(empty_bar(stage), phase ^ 1u, p.status)) { aborted = true; break; }
+        if (elect_one()) {
           const uint32_t fb = full_bar(stage);
           mbar_expect_tx(fb, stage_bytes);
           const uint32_t a_dst = smem_base + static_cast<uint32_t>(stage) * stage_bytes;
@@ -178,45 +178,51 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             for (int c = 0; c < p.block_n / 128; ++c)
               tma_load_2d(b_dst + c * kMnChunkBytes, &tmap_b, fb, n_idx * p.block_n + c * 128, kb * kBlockKBytes);
           }
-          if (++stage == S) { stage = 0; phase ^= 1u; }
         }
+        __syncwarp();
+        if (++stage == S) { stage = 0; phase ^= 1u; }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      int acc = 0;
-      uint32_t acc_phase = 0;
-      for (int tile = blockIdx.x; tile < total_tiles && !aborted; tile += gridDim.x) {
-        const int split = tile / tiles_per_split;
-        const int kb_begin = split * p.kblocks_per_split;
-        const int kb_end = min(kb_begin + p.kblocks_per_split, p.kblocks_total);
-        if (!mbar_wait(tmem_empty_bar(acc), acc_phase ^ 1u, p.status)) { aborted = true; break; }
+    // ------------------------------------------------------------ MMA issuer (whole warp loops, one lane issues:
+    // warp-uniform control flow keeps the descriptor arithmetic on the uniform datapath)
+    int stage = 0;
+    uint32_t phase = 0;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    // descriptors differ between stages and K steps only in the 14-bit start-address field
+    const uint64_t a_desc0 = kAMn ? make_smem_desc(smem_base, kMnChunkBytes, 1024) : make_smem_desc(smem_base, 16, 1024);
+    const uint64_t b_desc0 = kBMn ? make_smem_desc(smem_base + kATileBytes, kMnChunkBytes, 1024)
+                                  : make_smem_desc(smem_base + kATileBytes, 16, 1024);
+    constexpr uint32_t kAStep = (kAMn ? kUmmaK * 128 : kUmmaK) >> 4;   // per K step, in 16-byte units
+    constexpr uint32_t kBStep = (kBMn ? kUmmaK * 128 : kUmmaK) >> 4;
+    for (int tile = blockIdx.x; tile < total_tiles && !aborted; tile += gridDim.x) {
+      const int split = tile / tiles_per_split;
+      const int kb_begin = split * p.kblocks_per_split;
+      const int kb_end = min(kb_begin + p.kblocks_per_split, p.kblocks_total);
+      if (!mbar_wait_warp(tmem_empty_bar(acc), acc_phase ^ 1u, p.status)) { aborted = true; break; }
+      tc_fence_after_sync();
+      const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * kAccCols;
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
+        if (!mbar_wait_warp(full_bar(stage), phase, p.status)) { aborted = true; break; }
         tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * kAccCols;
-        for (int kb = kb_begin; kb < kb_end; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, p.status)) { aborted = true; break; }
-          tc_fence_after_sync();
-          const uint32_t a_addr = smem_base + static_cast<uint32_t>(stage) * stage_bytes;
-          const uint32_t b_addr = a_addr + kATileBytes;
+        const uint32_t stage_off = (static_cast<uint32_t>(stage) * stage_bytes) >> 4;
+        if (elect_one()) {
 #pragma unroll
           for (int k = 0; k < kBlockKBytes / kUmmaK; ++k) {
-            const uint64_t adesc = kAMn ? make_smem_desc(a_addr + k * (kUmmaK * 128), kMnChunkBytes, 1024)
-                                        : make_smem_desc(a_addr + k * kUmmaK, 16, 1024);
-            const uint64_t bdesc = kBMn ? make_smem_desc(b_addr + k * (kUmmaK * 128), kMnChunkBytes, 1024)
-                                        : make_smem_desc(b_addr + k * kUmmaK, 16, 1024);
-            umma_f8(d_tmem, adesc, bdesc, p.idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
+            umma_f8(d_tmem, a_desc0 + stage_off + k * kAStep, b_desc0 + stage_off + k * kBStep, p.idesc,
+                    (kb > kb_begin || k > 0) ? 1u : 0u);
           }
           umma_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
-          if (++stage == S) { stage = 0; phase ^= 1u; }
         }
-        if (aborted) break;
-        umma_commit(tmem_full_bar(acc));  // accumulator complete
-        acc ^= 1;
-        if (acc == 0) acc_phase ^= 1u;
+        __syncwarp();
+        if (++stage == S) { stage = 0; phase ^= 1u; }
       }
+      if (aborted) break;
+      if (elect_one()) umma_commit(tmem_full_bar(acc));  // accumulator complete
+      __syncwarp();
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5)
@@ -352,19 +358,19 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   bool aborted = false;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer (one lane in each CTA)
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      for (int tile = pair; tile < total_tiles && !aborted; tile += num_pairs) {
-        const int n_idx = tile / p.m_tiles;
-        const int m_idx = tile - n_idx * p.m_tiles;
-        const int n0 = n_idx * 256;
-        const int n_inst = pair_instr_n<kBMn>(p.N - n0);        // instruction N of this tile
-        const int row0 = m_idx * 256 + static_cast<int>(rank) * kBlockM;
-        const int bn0 = n0 + static_cast<int>(rank) * (n_inst >> 1);  // this CTA's half of the B rows
-        for (int kb = 0; kb < p.kblocks_total; ++kb) {
-          if (!mbar_wait_cluster(empty_bar(stage), phase ^ 1u, p.status)) { aborted = true; break; }
+    // ------------------------------------------------------------ TMA producer (warp 0 of each CTA; one lane issues)
+    int stage = 0;
+    uint32_t phase = 0;
+    for (int tile = pair; tile < total_tiles && !aborted; tile += num_pairs) {
+      const int n_idx = tile / p.m_tiles;
+      const int m_idx = tile - n_idx * p.m_tiles;
+      const int n0 = n_idx * 256;
+      const int n_inst = pair_instr_n<kBMn>(p.N - n0);             // instruction N of this tile
+      const int row0 = m_idx * 256 + static_cast<int>(rank) * kBlockM;
+      const int bn0 = n0 + static_cast<int>(rank) * (n_inst >> 1);  // this CTA's half of the B rows
+      for (int kb = 0; kb < p.kblocks_total; ++kb) {
+        if (!mbar_wait_warp(empty_bar(stage), phase ^ 1u, p.status)) { aborted = true; break; }
+        if (elect_one()) {
           if (leader) mbar_expect_tx(full_bar(stage), 2 * kPairStageBytes);
           const uint32_t fb = map_to_cta(full_bar(stage), 0);
           const uint32_t a_dst = smem_base + static_cast<uint32_t>(stage) * kPairStageBytes;
@@ -372,48 +378,55 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
           tma_load_2d_pair(a_dst, &tmap_a, fb, kb * kBlockKBytes, row0);
           if (!kBMn) tma_load_2d_pair(b_dst, &tmap_b, fb, kb * kBlockKBytes, bn0);
           else       tma_load_2d_pair(b_dst, &tmap_b, fb, bn0, kb * kBlockKBytes);
-          if (++stage == S) { stage = 0; phase ^= 1u; }
         }
-      }
-      // tail: wait until the MMAs have released every stage, so no completion signal can arrive at a CTA
-      // that has already left
-      for (int i = 0; i < S && !aborted; ++i) {
-        if (!mbar_wait_cluster(empty_bar(stage), phase ^ 1u, p.status)) aborted = true;
+        __syncwarp();
         if (++stage == S) { stage = 0; phase ^= 1u; }
       }
     }
+    // tail: wait until the MMAs have released every stage, so no completion signal can arrive at a CTA
+    // that has already left
+    for (int i = 0; i < S && !aborted; ++i) {
+      if (!mbar_wait_warp(empty_bar(stage), phase ^ 1u, p.status)) aborted = true;
+      if (++stage == S) { stage = 0; phase ^= 1u; }
+    }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer (one lane of the leader CTA)
-    if (lane == 0 && leader) {
+    // ------------------------------------------------------------ MMA issuer (warp 1 of the leader CTA; one lane issues)
+    if (leader) {
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
+      const uint64_t a_desc0 = make_smem_desc(smem_base, 16, 1024);
+      const uint64_t b_desc0 = kBMn ? make_smem_desc(smem_base + kATileBytes, kMnChunkBytes, 1024)
+                                    : make_smem_desc(smem_base + kATileBytes, 16, 1024);
+      constexpr uint32_t kAStep = kUmmaK >> 4;
+      constexpr uint32_t kBStep = (kBMn ? kUmmaK * 128 : kUmmaK) >> 4;
       for (int tile = pair; tile < total_tiles && !aborted; tile += num_pairs) {
         const int n_idx = tile / p.m_tiles;
         const int n0 = n_idx * 256;
         const int n_inst = pair_instr_n<kBMn>(p.N - n0);
         const uint32_t idesc = p.idesc | (static_cast<uint32_t>(n_inst >> 3) << 17);
-        if (!mbar_wait_cluster(tmem_empty_bar(acc), acc_phase ^ 1u, p.status)) { aborted = true; break; }
+        if (!mbar_wait_warp(tmem_empty_bar(acc), acc_phase ^ 1u, p.status)) { aborted = true; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * kAccCols;
         for (int kb = 0; kb < p.kblocks_total; ++kb) {
-          if (!mbar_wait_cluster(full_bar(stage), phase, p.status)) { aborted = true; break; }
+          if (!mbar_wait_warp(full_bar(stage), phase, p.status)) { aborted = true; break; }
           tc_fence_after_sync();
-          const uint32_t a_addr = smem_base + static_cast<uint32_t>(stage) * kPairStageBytes;
-          const uint32_t b_addr = a_addr + kATileBytes;
+          const uint32_t stage_off = (static_cast<uint32_t>(stage) * kPairStageBytes) >> 4;
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < kBlockKBytes / kUmmaK; ++k) {
-            const uint64_t adesc = make_smem_desc(a_addr + k * kUmmaK, 16, 1024);
-            const uint64_t bdesc = kBMn ? make_smem_desc(b_addr + k * (kUmmaK * 128), kMnChunkBytes, 1024)
-                                        : make_smem_desc(b_addr + k * kUmmaK, 16, 1024);
-            umma_f8_pair(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            for (int k = 0; k < kBlockKBytes / kUmmaK; ++k) {
+              umma_f8_pair(d_tmem, a_desc0 + stage_off + k * kAStep, b_desc0 + stage_off + k * kBStep, idesc,
+                           (kb > 0 || k > 0) ? 1u : 0u);
+            }
+            umma_commit_pair(empty_bar(stage), 3);   // frees the stage in both CTAs
           }
-          umma_commit_pair(empty_bar(stage), 3);   // frees the stage in both CTAs
+          __syncwarp();
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
         if (aborted) break;
-        umma_commit_pair(tmem_full_bar(acc), 3);    // accumulators of both CTAs complete
+        if (elect_one()) umma_commit_pair(tmem_full_bar(acc), 3);    // accumulators of both CTAs complete
+        __syncwarp();
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
@@ -429,7 +442,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     for (int tile = pair; tile < total_tiles && !aborted; tile += num_pairs) {
       const int n_idx = tile / p.m_tiles;
       const int m_idx = tile - n_idx * p.m_tiles;
-      if (!mbar_wait_cluster(tmem_full_bar(acc), acc_phase, p.status)) { aborted = true; break; }
+      if (!mbar_wait(tmem_full_bar(acc), acc_phase, p.status)) { aborted = true; break; }
       tc_fence_after_sync();
       const int row = m_idx * 256 + static_cast<int>(rank) * kBlockM + quad * 32 + lane;
       const bool row_ok = row < p.M;

@@ -196,23 +196,52 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __re
   const int64_t cta_c0 = (int64_t)blockIdx.x * kMergeCols;
   const int cta_cols = static_cast<int>(min((int64_t)kMergeCols, n - cta_c0));   // multiple of 16
   if (threadIdx.x < kMergeRows) srow[threadIdx.x] = (threadIdx.x < nrows) ? sel_idx[g0 + threadIdx.x] : -1;
-  // decode A~ (rows m.. of W~') into shared memory; columns beyond the matrix edge become 0
+  // decode A~ (rows m.. of W~') into shared memory; columns beyond the matrix edge become 0.  The loads of
+  // four iterations are issued together so that their latencies overlap.
   const uint8_t* aq = wq + m * n + cta_c0;
-  for (int e = threadIdx.x; e < r * (kMergeCols / 16); e += kMergeThreads) {
-    const int j = e / (kMergeCols / 16), v = e % (kMergeCols / 16);
-    uint4 w = make_uint4(0u, 0u, 0u, 0u);
-    if (v * 16 < cta_cols) w = __ldg(reinterpret_cast<const uint4*>(aq + (int64_t)j * n + v * 16));
-    float f[4];
-    float4* dst = reinterpret_cast<float4*>(a_tile + (size_t)j * kMergeCols + v * 16);
-    decode4(w.x, f); dst[0] = make_float4(f[0], f[1], f[2], f[3]);
-    decode4(w.y, f); dst[1] = make_float4(f[0], f[1], f[2], f[3]);
-    decode4(w.z, f); dst[2] = make_float4(f[0], f[1], f[2], f[3]);
-    decode4(w.w, f); dst[3] = make_float4(f[0], f[1], f[2], f[3]);
+  constexpr int kVecPerRow = kMergeCols / 16;
+  const int a_vecs = r * kVecPerRow;
+  for (int e0 = threadIdx.x; e0 < a_vecs; e0 += 4 * kMergeThreads) {
+    uint4 w[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + u * kMergeThreads;
+      const int j = e / kVecPerRow, v = e % kVecPerRow;
+      w[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (e < a_vecs && v * 16 < cta_cols) w[u] = __ldg(reinterpret_cast<const uint4*>(aq + (int64_t)j * n + v * 16));
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + u * kMergeThreads;
+      if (e < a_vecs) {
+        const int j = e / kVecPerRow, v = e % kVecPerRow;
+        float f[4];
+        float4* dst = reinterpret_cast<float4*>(a_tile + (size_t)j * kMergeCols + v * 16);
+        decode4(w[u].x, f); dst[0] = make_float4(f[0], f[1], f[2], f[3]);
+        decode4(w[u].y, f); dst[1] = make_float4(f[0], f[1], f[2], f[3]);
+        decode4(w[u].z, f); dst[2] = make_float4(f[0], f[1], f[2], f[3]);
+        decode4(w[u].w, f); dst[3] = make_float4(f[0], f[1], f[2], f[3]);
+      }
+    }
   }
   __syncthreads();   // srow visible
-  for (int e = threadIdx.x; e < kMergeRows * r; e += kMergeThreads) {
-    const int q = e / r, j = e - q * r;
-    sdb[e] = (q < nrows) ? dbuf[(int64_t)srow[q] * r + j] : 0.0f;
+  // the 32 DeltaBuffer rows, as float4 (r is a multiple of 8), four loads in flight per thread
+  const int r4 = r >> 2;
+  const int d_vecs = kMergeRows * r4;
+  for (int e0 = threadIdx.x; e0 < d_vecs; e0 += 4 * kMergeThreads) {
+    float4 d[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + u * kMergeThreads;
+      const int q = e / r4, j4 = e - q * r4;
+      d[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (e < d_vecs && q < nrows) d[u] = *reinterpret_cast<const float4*>(dbuf + (int64_t)srow[q] * r + 4 * j4);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + u * kMergeThreads;
+      if (e < d_vecs) reinterpret_cast<float4*>(sdb)[e] = d[u];
+    }
   }
   __syncthreads();
   const int tx = threadIdx.x % kMergeTx, ty = threadIdx.x / kMergeTx;

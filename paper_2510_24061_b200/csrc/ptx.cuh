@@ -46,6 +46,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return done != 0;
 }
 
+// Warp-uniform election of one lane (all 32 lanes must execute it convergently).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xFFFFFFFF;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
+
 // Bounded wait: gives up after kWaitLimitNs of wall time, records the timeout in *status and
 // returns false.  Callers leave their loops on false and fall through to the common exit, so a
 // lost signal can never hang the device.
@@ -64,6 +75,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* st
       return false;
     }
   }
+}
+
+// The same wait executed by a whole converged warp; the verdict is made warp-uniform.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* status) {
+  const bool ok = mbar_wait(bar, parity, status);
+  return __all_sync(0xFFFFFFFFu, ok);
 }
 
 // ---------------------------------------------------------------- TMA (bulk tensor copy), 2-D tiles, no multicast
@@ -159,31 +176,6 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {  //
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
 
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t done;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(done)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return done != 0;
-}
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, int* status) {
-  if (mbar_try_wait_cluster(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 128; ++i) {
-      if (mbar_try_wait_cluster(bar, parity)) return true;
-    }
-    if (global_timer_ns() - t0 > kWaitLimitNs) {
-      atomicExch(status, kStatusTimeout);
-      return false;
-    }
-  }
-}
 // TMA tile load issued by either CTA of a pair; the completion bytes are counted on `bar_cluster`,
 // a shared::cluster barrier address (the leader CTA's barrier).  No multicast.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst_smem, const void* tensor_map, uint32_t bar_cluster, int x,
