@@ -6,7 +6,7 @@
 // One persistent CTA per SM walks a static list of 128 x block_n output tiles.  Warp roles:
 //   warp 0      TMA producer (one lane): fills a ring of (A,B) stages, signalled through mbarriers
 //   warp 1      allocates TMEM; one lane issues the MMAs and commits them to the barriers
-//   warps 2..5  epilogue: tcgen05.ld the accumulator, rescale by 1/(s_a*s_b), store
+//   warps 2..9  epilogue: tcgen05.ld the accumulator, rescale by 1/(s_a*s_b), store
 // The accumulator is double buffered (2 x 256 TMEM columns), so the epilogue of tile i overlaps the
 // main loop of tile i+1.  Either operand may be K-major (rows along K) or MN-major (rows along M/N):
 // the melded forward reads both K-major, the input gradient reads W~ MN-major (no transposed copy of
@@ -22,7 +22,8 @@
 namespace falqon {
 namespace {
 
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 320;          // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
+constexpr int kEpilogueWarps = 8;
 constexpr int kBlockM = 128;
 constexpr int kBlockKBytes = 128;          // one 128-byte swizzle row of FP8 = 128 elements of K
 constexpr int kUmmaK = 32;                 // K per tcgen05.mma for 8-bit operands
@@ -103,6 +104,39 @@ __device__ __forceinline__ void epilogue_store32(const GemmParams& p, int row, i
   }
 }
 
+// Drains columns [col_begin, col_end) of one accumulator tile for this warp's 32 rows: tcgen05.ld of the next
+// 32-column chunk is in flight while the current one is rescaled and stored.
+__device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_row, int row, bool row_ok, int n0,
+                                              int col_begin, int col_end, int split, float inv, uint32_t& amax_bits) {
+  int last = min(col_end, p.N - n0);          // warp-uniform: columns at or beyond N hold nothing
+  if (col_begin >= last) return;
+  uint32_t va[32], vb[32];
+  auto drain = [&](const uint32_t (&v)[32], int c) {
+    if (row_ok) {
+      float f[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * inv;
+      epilogue_store32(p, row, n0 + c, split, f, amax_bits);
+    }
+  };
+  __syncwarp();
+  tmem_ld_32x32b_x32(t_row + col_begin, va);
+  tmem_ld_wait();
+  for (int c = col_begin; c < last; c += 64) {
+    const bool more1 = c + 32 < last;      // warp-uniform
+    __syncwarp();
+    if (more1) tmem_ld_32x32b_x32(t_row + c + 32, vb);
+    drain(va, c);
+    if (!more1) break;
+    tmem_ld_wait();
+    const bool more2 = c + 64 < last;
+    __syncwarp();
+    if (more2) tmem_ld_32x32b_x32(t_row + c + 64, va);
+    drain(vb, c + 32);
+    if (more2) tmem_ld_wait();
+  }
+}
+
 template <bool kAMn, bool kBMn>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -135,7 +169,7 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tmem_full_bar(a), 1);
-      mbar_init(tmem_empty_bar(a), 4);
+      mbar_init(tmem_empty_bar(a), kEpilogueWarps);
     }
     mbar_fence_init();
   }
@@ -225,8 +259,9 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       if (acc == 0) acc_phase ^= 1u;
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------ epilogue (warps 2..9)
     const int quad = warp & 3;  // TMEM lanes [32*quad, 32*quad+32) belong to this warp
+    const int col_half = (warp - 2) >> 2;   // warps 2..5 drain the left half of the tile, 6..9 the right half
     const bool rescale = p.scale_a != nullptr;
     const float inv = rescale ? 1.0f / (__ldg(p.scale_a) * __ldg(p.scale_b)) : 1.0f;
     int acc = 0;
@@ -243,20 +278,8 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const bool row_ok = row < p.M;
       const uint32_t t_row = tmem_base + static_cast<uint32_t>(acc) * kAccCols + (static_cast<uint32_t>(quad * 32) << 16);
       const int n0 = n_idx * p.block_n;
-      for (int c = 0; c < p.block_n; c += 32) {
-        if (n0 + c >= p.N) break;  // warp-uniform
-        uint32_t v[32];
-        __syncwarp();
-        tmem_ld_32x32b_x32(t_row + c, v);
-        tmem_ld_wait();
-        const int col0 = n0 + c;
-        if (row_ok) {
-        float f[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * inv;
-        epilogue_store32(p, row, col0, split, f, amax_bits);
-        }  // row_ok
-      }
+      const int half = (((p.block_n + 1) / 2) + 31) & ~31;   // first-half warps take [0, half), the others [half, block_n)
+      epilogue_tile(p, t_row, row, row_ok, n0, col_half ? half : 0, col_half ? p.block_n : half, split, inv, amax_bits);
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(tmem_empty_bar(acc));
@@ -337,7 +360,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tmem_full_bar(a), 1);   // one multicast commit
-      mbar_init(tmem_empty_bar(a), 8);  // 4 epilogue warps of each CTA
+      mbar_init(tmem_empty_bar(a), 2 * kEpilogueWarps);  // the epilogue warps of both CTAs
     }
     mbar_fence_init();
   }
@@ -432,8 +455,9 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5 of each CTA)
+    // ------------------------------------------------------------ epilogue (warps 2..9 of each CTA)
     const int quad = warp & 3;
+    const int col_half = (warp - 2) >> 2;
     const bool rescale = p.scale_a != nullptr;
     const float inv = rescale ? 1.0f / (__ldg(p.scale_a) * __ldg(p.scale_b)) : 1.0f;
     int acc = 0;
@@ -448,19 +472,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       const bool row_ok = row < p.M;
       const uint32_t t_row = tmem_base + static_cast<uint32_t>(acc) * kAccCols + (static_cast<uint32_t>(quad * 32) << 16);
       const int n0 = n_idx * 256;
-      for (int c = 0; c < 256; c += 32) {
-        if (n0 + c >= p.N) break;  // warp-uniform
-        uint32_t v[32];
-        __syncwarp();
-        tmem_ld_32x32b_x32(t_row + c, v);
-        tmem_ld_wait();
-        if (row_ok) {
-          float f[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * inv;
-          epilogue_store32(p, row, n0 + c, 0, f, amax_bits);
-        }
-      }
+      epilogue_tile(p, t_row, row, row_ok, n0, col_half ? 128 : 0, col_half ? 256 : 128, 0, inv, amax_bits);
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(tmem_empty_bar(acc), 0));
