@@ -177,10 +177,12 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     tmem_alloc(smem_base + slot_off, kTmemCols);
     tmem_relinquish();
   }
+  pdl_trigger();
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();   // everything above is private set-up; operands and scales are read only from here on
 
   const int tiles_per_split = p.m_tiles * p.n_tiles;
   const int total_tiles = tiles_per_split * p.k_splits;
@@ -368,12 +370,14 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     tmem_alloc_pair(smem_base + slot_off, kTmemCols);
     tmem_relinquish_pair();
   }
+  pdl_trigger();
   tc_fence_before_sync();
   __syncthreads();
   cluster_arrive();      // the peer's barriers must be initialised before anything signals them
   cluster_wait();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();   // everything above is private set-up; operands and scales are read only from here on
 
   const int num_pairs = gridDim.x >> 1;
   const int pair = blockIdx.x >> 1;
@@ -553,8 +557,8 @@ cudaError_t launch_variant(const CUtensorMap& ta, const CUtensorMap& tb, const G
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  gemm_fp8_kernel<kAMn, kBMn><<<grid, kGemmThreads, smem, stream>>>(ta, tb, gp);
-  return cudaGetLastError();
+  return launch_pdl(gemm_fp8_kernel<kAMn, kBMn>, dim3(static_cast<unsigned>(grid)), dim3(kGemmThreads), smem, stream, 1, ta,
+                    tb, gp);
 }
 
 template <bool kBMn>
@@ -567,19 +571,8 @@ cudaError_t launch_pair_variant(const CUtensorMap& ta, const CUtensorMap& tb, co
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
-  cfg.blockDim = dim3(kGemmThreads, 1, 1);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_fp8_pair_kernel<kBMn>, ta, tb, gp);
+  return launch_pdl(gemm_fp8_pair_kernel<kBMn>, dim3(static_cast<unsigned>(grid)), dim3(kGemmThreads), smem, stream, 2, ta, tb,
+                    gp);
 }
 
 bool pair_kernel_disabled() {

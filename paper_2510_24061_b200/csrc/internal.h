@@ -12,6 +12,34 @@ constexpr int kBF16 = 0, kF32 = 1;
 
 inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
 
+// Launches `kernel` so that it may be scheduled before the previous kernel in the stream has drained
+// (programmatic stream serialization).  The kernel itself must call pdl_wait() before it reads or writes
+// anything another kernel touches.  cluster_x > 1 adds a thread-block-cluster dimension.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, int cluster_x,
+                       Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = static_cast<unsigned>(cluster_x);
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = static_cast<unsigned>(n);
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- quantize.cu
 constexpr int kMaxAbsmaxParts = 148 * 8;   // upper bound of the absmax grid = number of partial maxima
 // Pass 1 of per-tensor absmax scaling: one partial max (fp32 bit pattern of |x|) per CTA into partial[0..*nparts).

@@ -12,6 +12,8 @@ namespace {
 __global__ void __launch_bounds__(256) reduce_db_kernel(const float* __restrict__ partials, int splits, int64_t count,
                                                         const float* __restrict__ s_g, const float* __restrict__ s_oa,
                                                         float* __restrict__ dB) {
+  pdl_trigger();
+  pdl_wait();
   const float inv = 1.0f / (__ldg(s_g) * __ldg(s_oa));
   const int64_t nvec = count / 4;
   for (int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; v < nvec; v += (int64_t)gridDim.x * blockDim.x) {
@@ -30,6 +32,8 @@ constexpr int kScoreRows = 32;
 __global__ void __launch_bounds__(256) sgd_score_kernel(float* __restrict__ dbuf, const float* __restrict__ dB,
                                                         float neg_lr, int64_t m, int r, float* __restrict__ score) {
   extern __shared__ float sabs[];  // [kScoreRows][r + 1]
+  pdl_trigger();
+  pdl_wait();
   const int64_t row0 = (int64_t)blockIdx.x * kScoreRows;
   const int rows = static_cast<int>(min((int64_t)kScoreRows, m - row0));
   const int64_t base = row0 * r;
@@ -95,6 +99,8 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
   __shared__ uint32_t s_digit[4], s_remaining[4];
   const uint32_t* gbits = reinterpret_cast<const uint32_t*>(score);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_trigger();
+  pdl_wait();
 
   for (int i = tid; i < 4 * 256; i += kTopkThreads) (&hist[0][0])[i] = 0;
   if (use_smem)
@@ -191,6 +197,8 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __re
   float* a_tile = merge_smem;                         // [r][kMergeCols] decoded A~
   float* sdb = merge_smem + (size_t)r * kMergeCols;   // [kMergeRows][r]
   __shared__ int srow[kMergeRows];
+  pdl_trigger();
+  pdl_wait();
   const int g0 = blockIdx.y * kMergeRows;
   const int nrows = min(kMergeRows, k - g0);
   const int64_t cta_c0 = (int64_t)blockIdx.x * kMergeCols;
@@ -287,6 +295,8 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __re
 
 __global__ void __launch_bounds__(256) zero_rows_kernel(float* __restrict__ dbuf, const int32_t* __restrict__ sel_idx,
                                                         int k, int r) {
+  pdl_trigger();
+  pdl_wait();
   for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < k * r; e += gridDim.x * blockDim.x) {
     const int s = e / r, j = e - s * r;
     dbuf[(int64_t)sel_idx[s] * r + j] = 0.0f;
@@ -300,16 +310,15 @@ cudaError_t launch_reduce_db(const float* partials, int splits, int64_t count, c
   int64_t blocks = (count / 4 + 255) / 256;
   if (blocks > 148 * 8) blocks = 148 * 8;
   if (blocks < 1) blocks = 1;
-  reduce_db_kernel<<<static_cast<int>(blocks), 256, 0, stream>>>(partials, splits, count, s_g, s_oa, dB);
-  return cudaGetLastError();
+  return launch_pdl(reduce_db_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream, 1, partials, splits, count,
+                    s_g, s_oa, dB);
 }
 
 cudaError_t launch_sgd_score(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, float* score,
                              cudaStream_t stream) {
   const int grid = static_cast<int>((m + kScoreRows - 1) / kScoreRows);
   const size_t smem = sizeof(float) * kScoreRows * (r + 1);
-  sgd_score_kernel<<<grid, 256, smem, stream>>>(dbuf, dB, -lr, m, static_cast<int>(r), score);
-  return cudaGetLastError();
+  return launch_pdl(sgd_score_kernel, dim3(grid), dim3(256), smem, stream, 1, dbuf, dB, -lr, m, static_cast<int>(r), score);
 }
 
 size_t topk_scratch_bytes(int64_t m) { (void)m; return 256; }
@@ -324,9 +333,8 @@ cudaError_t launch_topk(const float* score, int64_t m, int64_t k, int32_t* sel_i
     if (ea != cudaSuccess) return ea;
     configured = true;
   }
-  topk_kernel<<<1, kTopkThreads, smem, stream>>>(score, static_cast<int>(m), static_cast<int>(k), sel_idx,
-                                                 static_cast<int32_t*>(idx_copy), use_smem);
-  return cudaGetLastError();
+  return launch_pdl(topk_kernel, dim3(1), dim3(kTopkThreads), smem, stream, 1, score, static_cast<int>(m),
+                    static_cast<int>(k), sel_idx, static_cast<int32_t*>(idx_copy), use_smem);
 }
 
 cudaError_t launch_merge_rows(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
@@ -340,14 +348,13 @@ cudaError_t launch_merge_rows(uint8_t* wq, float* dbuf, const int32_t* sel_idx, 
     if (ea != cudaSuccess) return ea;
     configured = true;
   }
-  merge_rows_kernel<<<grid, kMergeThreads, smem, stream>>>(wq, dbuf, sel_idx, static_cast<int>(k), m, n,
-                                                           static_cast<int>(r));
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = launch_pdl(merge_rows_kernel, grid, dim3(kMergeThreads), smem, stream, 1, wq, dbuf, sel_idx,
+                             static_cast<int>(k), m, n, static_cast<int>(r));
   if (e != cudaSuccess) return e;
   int64_t zb = (k * r + 255) / 256;
   if (zb > 1024) zb = 1024;
-  zero_rows_kernel<<<static_cast<int>(zb), 256, 0, stream>>>(dbuf, sel_idx, static_cast<int>(k), static_cast<int>(r));
-  return cudaGetLastError();
+  return launch_pdl(zero_rows_kernel, dim3(static_cast<unsigned>(zb)), dim3(256), 0, stream, 1, dbuf, sel_idx,
+                    static_cast<int>(k), static_cast<int>(r));
 }
 
 }  // namespace falqon

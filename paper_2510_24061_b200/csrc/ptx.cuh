@@ -21,6 +21,14 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Every kernel of the library starts with pdl_trigger(); pdl_wait();  The trigger lets the next kernel in the
+// stream be scheduled (and run its set-up) while this one is still computing; the wait returns once the
+// previous kernel in the stream has completed and its writes are visible.  Nothing before pdl_wait() may
+// touch global memory that another kernel writes.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");

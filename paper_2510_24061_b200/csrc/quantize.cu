@@ -89,6 +89,8 @@ template <int kDt>
 __global__ void __launch_bounds__(kThreads) absmax_kernel(const void* __restrict__ src, int64_t count, float premul,
                                                           bool use_premul, uint32_t* __restrict__ partial) {
   __shared__ uint32_t red[32];
+  pdl_trigger();
+  pdl_wait();
   const int64_t nvec = count / 16;
   uint32_t m = 0;
   for (int64_t v = blockIdx.x * (int64_t)kThreads + threadIdx.x; v < nvec; v += (int64_t)gridDim.x * kThreads) {
@@ -121,6 +123,8 @@ __global__ void __launch_bounds__(kThreads) cast_kernel(const void* __restrict__
                                                         const float* __restrict__ scale_in, uint8_t* __restrict__ dst,
                                                         CastOutputs out) {
   __shared__ uint32_t red[32];
+  pdl_trigger();
+  pdl_wait();
   float s, amax = 0.0f;
   if (nparts > 0) {
     uint32_t mb = 0;
@@ -158,6 +162,8 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const void* __r
                                                                  uint8_t* __restrict__ dst, float* __restrict__ scale_out,
                                                                  float* __restrict__ amax_out) {
   __shared__ uint32_t red[32];
+  pdl_trigger();
+  pdl_wait();
   const int64_t row = blockIdx.x;
   const int64_t base = row * cols;
   const int64_t nvec = cols / 16;
@@ -195,6 +201,8 @@ __global__ void __launch_bounds__(256) quantize_oa_transposed_kernel(const float
                                                                      float* __restrict__ s_oa_out,
                                                                      float* __restrict__ amax_copy) {
   __shared__ __align__(16) uint8_t tile[256][kOaTileT + 16];
+  pdl_trigger();
+  pdl_wait();
   const float amax = *amax_oa;
   const float s = scale_from_amax(amax, kE4M3);
   if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -245,9 +253,9 @@ cudaError_t launch_absmax(const void* src, int src_dt, int64_t count, float prem
   const int grid = absmax_grid(count);
   *nparts = grid;
   const bool use_premul = premul != 1.0f;
-  if (src_dt == kBF16) absmax_kernel<kBF16><<<grid, kThreads, 0, stream>>>(src, count, premul, use_premul, partial);
-  else absmax_kernel<kF32><<<grid, kThreads, 0, stream>>>(src, count, premul, use_premul, partial);
-  return cudaGetLastError();
+  if (src_dt == kBF16)
+    return launch_pdl(absmax_kernel<kBF16>, dim3(grid), dim3(kThreads), 0, stream, 1, src, count, premul, use_premul, partial);
+  return launch_pdl(absmax_kernel<kF32>, dim3(grid), dim3(kThreads), 0, stream, 1, src, count, premul, use_premul, partial);
 }
 
 cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, int fmt, float premul,
@@ -258,11 +266,11 @@ cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, i
   const bool up = premul != 1.0f;
   const CastOutputs out{scale_out, scale_out2, amax_out, clear_word};
 #define FALQON_CAST(DT, FMT) \
-  cast_kernel<DT, FMT><<<grid, kThreads, 0, stream>>>(src, count, premul, up, partial, nparts, scale_in, dst, out)
+  return launch_pdl(cast_kernel<DT, FMT>, dim3(grid), dim3(kThreads), 0, stream, 1, src, count, premul, up, partial, nparts, \
+                    scale_in, dst, out)
   if (src_dt == kBF16) { if (fmt == kE4M3) FALQON_CAST(kBF16, kE4M3); else FALQON_CAST(kBF16, kE5M2); }
   else { if (fmt == kE4M3) FALQON_CAST(kF32, kE4M3); else FALQON_CAST(kF32, kE5M2); }
 #undef FALQON_CAST
-  return cudaGetLastError();
 }
 
 cudaError_t launch_quantize_per_row(const void* src, int src_dt, int64_t rows, int64_t cols, int fmt, float premul,
@@ -271,11 +279,11 @@ cudaError_t launch_quantize_per_row(const void* src, int src_dt, int64_t rows, i
   const bool up = premul != 1.0f;
   const int grid = static_cast<int>(rows);
 #define FALQON_ROWS(DT, FMT) \
-  quantize_rows_kernel<DT, FMT><<<grid, kThreads, 0, stream>>>(src, cols, premul, up, scale_in, dst, scale_out, amax_out)
+  return launch_pdl(quantize_rows_kernel<DT, FMT>, dim3(grid), dim3(kThreads), 0, stream, 1, src, cols, premul, up, \
+                    scale_in, dst, scale_out, amax_out)
   if (src_dt == kBF16) { if (fmt == kE4M3) FALQON_ROWS(kBF16, kE4M3); else FALQON_ROWS(kBF16, kE5M2); }
   else { if (fmt == kE4M3) FALQON_ROWS(kF32, kE4M3); else FALQON_ROWS(kF32, kE5M2); }
 #undef FALQON_ROWS
-  return cudaGetLastError();
 }
 
 cudaError_t launch_quantize_oa_transposed(const float* oa, const float* amax_oa, int64_t T, int64_t r, int64_t r16,
@@ -283,9 +291,8 @@ cudaError_t launch_quantize_oa_transposed(const float* oa, const float* amax_oa,
                                           cudaStream_t stream) {
   (void)r16;
   const int grid = static_cast<int>((T + kOaTileT - 1) / kOaTileT);
-  quantize_oa_transposed_kernel<<<grid, 256, 0, stream>>>(oa, amax_oa, T, static_cast<int>(r), ldt, oaq_t, s_oa_out,
-                                                          amax_copy);
-  return cudaGetLastError();
+  return launch_pdl(quantize_oa_transposed_kernel, dim3(grid), dim3(256), 0, stream, 1, oa, amax_oa, T, static_cast<int>(r),
+                    ldt, oaq_t, s_oa_out, amax_copy);
 }
 
 }  // namespace falqon
