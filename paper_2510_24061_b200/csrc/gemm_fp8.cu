@@ -23,7 +23,7 @@ namespace falqon {
 namespace {
 
 constexpr int kGemmThreads = 320;          // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
-constexpr int kEpilogueWarps = 8;
+constexpr uint32_t kEpilogueWarps = 8;
 constexpr int kBlockM = 128;
 constexpr int kBlockKBytes = 128;          // one 128-byte swizzle row of FP8 = 128 elements of K
 constexpr int kUmmaK = 32;                 // K per tcgen05.mma for 8-bit operands
@@ -34,6 +34,8 @@ constexpr uint32_t kAccCols = 256;
 constexpr int kMaxStages = 8;
 constexpr uint32_t kSmemBudget = 227 * 1024;
 constexpr uint32_t kBarrierBytes = 256;
+constexpr uint32_t kStageOutBytes = 32 * 128;                       // per epilogue warp: 32 rows x 128 B
+constexpr uint32_t kStagingBytes = kEpilogueWarps * kStageOutBytes;  // 32 KB behind the barriers
 
 struct GemmParams {
   int M, N, K;
@@ -104,21 +106,79 @@ __device__ __forceinline__ void epilogue_store32(const GemmParams& p, int row, i
   }
 }
 
-// Drains columns [col_begin, col_end) of one accumulator tile for this warp's 32 rows: tcgen05.ld of the next
-// 32-column chunk is in flight while the current one is rescaled and stored.
+// Drains columns [col_begin, col_end) of one accumulator tile for this warp's 32 rows.  tcgen05.ld of the next
+// 32-column chunk is in flight while the current one is rescaled.  Chunks that lie wholly inside the main
+// output (c0) are transposed through a 32 x 128-byte per-warp staging buffer in shared memory (16-byte pieces
+// XOR-swizzled by row, so neither side has bank conflicts) and leave as full 128-byte lines: a store
+// instruction then covers 4 rows x 128 B instead of 32 rows x 16 B.  Chunks that touch the O | O_A boundary
+// or the ragged right edge take the element-wise path.
 __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_row, int row, bool row_ok, int n0,
-                                              int col_begin, int col_end, int split, float inv, uint32_t& amax_bits) {
-  int last = min(col_end, p.N - n0);          // warp-uniform: columns at or beyond N hold nothing
+                                              int col_begin, int col_end, int split, float inv, uint32_t& amax_bits,
+                                              uint8_t* stage_out) {
+  const int last = min(col_end, p.N - n0);    // warp-uniform: columns at or beyond N hold nothing
   if (col_begin >= last) return;
-  uint32_t va[32], vb[32];
+  const int lane = threadIdx.x & 31;
+  const bool bf16 = p.c0_dt == kBF16;
+  const int esize = bf16 ? 2 : 4;
+  const int chunks_per_flush = bf16 ? 2 : 1;  // 64 bf16 or 32 fp32 columns fill the 128-byte rows
+  int pending = 0;                            // chunks staged and not yet flushed
+  int flush_col = 0;                          // first output column of the staged data
+
+  auto flush = [&]() {
+    if (pending == 0) return;
+    __syncwarp();
+    const int row_base = row - lane;
+    const int bytes_per_row = pending * 32 * esize;       // 64 or 128
+    const int lanes_per_row = bytes_per_row >> 4;          // 4 or 8
+    const int rows_per_inst = 32 / lanes_per_row;          // 8 or 4
+    const int piece = lane % lanes_per_row;
+    uint8_t* c0 = static_cast<uint8_t*>(p.c0) +
+                  ((long long)split * p.c0_split_stride + flush_col) * esize + (long long)piece * 16;
+    for (int r0 = 0; r0 < 32; r0 += rows_per_inst) {
+      const int r = r0 + lane / lanes_per_row;
+      const uint4 val = *reinterpret_cast<const uint4*>(stage_out + r * 128 + ((piece ^ (r & 7)) << 4));
+      if (row_base + r < p.M) *reinterpret_cast<uint4*>(c0 + (long long)(row_base + r) * p.ldc0 * esize) = val;
+    }
+    __syncwarp();
+    pending = 0;
+  };
+
   auto drain = [&](const uint32_t (&v)[32], int c) {
-    if (row_ok) {
-      float f[32];
+    const int col0 = n0 + c;
+    float f[32];
 #pragma unroll
-      for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * inv;
-      epilogue_store32(p, row, n0 + c, split, f, amax_bits);
+    for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * inv;
+    const bool fast = col0 + 32 <= p.n_split && ((p.ldc0 * esize) & 15) == 0 &&
+                      ((reinterpret_cast<uintptr_t>(p.c0) + (long long)split * p.c0_split_stride * esize) & 15) == 0;
+    if (fast) {   // warp-uniform
+      if (pending == 0) flush_col = col0;
+      uint8_t* my = stage_out + lane * 128;
+      const int sw = lane & 7;
+      if (bf16) {
+        const int base_piece = pending * 4;               // this chunk's 64 bytes
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint4 o;
+          o.x = pack_bf16x2(f[8 * j + 0], f[8 * j + 1]);
+          o.y = pack_bf16x2(f[8 * j + 2], f[8 * j + 3]);
+          o.z = pack_bf16x2(f[8 * j + 4], f[8 * j + 5]);
+          o.w = pack_bf16x2(f[8 * j + 6], f[8 * j + 7]);
+          *reinterpret_cast<uint4*>(my + (((base_piece + j) ^ sw) << 4)) = o;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          *reinterpret_cast<float4*>(my + ((j ^ sw) << 4)) = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
+      }
+      ++pending;
+      if (pending == chunks_per_flush) flush();
+    } else {
+      flush();
+      if (row_ok) epilogue_store32(p, row, col0, split, f, amax_bits);
     }
   };
+
+  uint32_t va[32], vb[32];
   __syncwarp();
   tmem_ld_32x32b_x32(t_row + col_begin, va);
   tmem_ld_wait();
@@ -135,6 +195,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ro
     drain(vb, c + 32);
     if (more2) tmem_ld_wait();
   }
+  flush();
 }
 
 template <bool kAMn, bool kBMn>
@@ -264,6 +325,7 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     // ------------------------------------------------------------ epilogue (warps 2..9)
     const int quad = warp & 3;  // TMEM lanes [32*quad, 32*quad+32) belong to this warp
     const int col_half = (warp - 2) >> 2;   // warps 2..5 drain the left half of the tile, 6..9 the right half
+    uint8_t* stage_out = smem_gen + static_cast<uint32_t>(S) * stage_bytes + kBarrierBytes + (warp - 2) * kStageOutBytes;
     const bool rescale = p.scale_a != nullptr;
     const float inv = rescale ? 1.0f / (__ldg(p.scale_a) * __ldg(p.scale_b)) : 1.0f;
     int acc = 0;
@@ -281,7 +343,8 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const uint32_t t_row = tmem_base + static_cast<uint32_t>(acc) * kAccCols + (static_cast<uint32_t>(quad * 32) << 16);
       const int n0 = n_idx * p.block_n;
       const int half = (((p.block_n + 1) / 2) + 31) & ~31;   // first-half warps take [0, half), the others [half, block_n)
-      epilogue_tile(p, t_row, row, row_ok, n0, col_half ? half : 0, col_half ? p.block_n : half, split, inv, amax_bits);
+      epilogue_tile(p, t_row, row, row_ok, n0, col_half ? half : 0, col_half ? p.block_n : half, split, inv, amax_bits,
+                    stage_out);
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(tmem_empty_bar(acc));
@@ -462,6 +525,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     // ------------------------------------------------------------ epilogue (warps 2..9 of each CTA)
     const int quad = warp & 3;
     const int col_half = (warp - 2) >> 2;
+    uint8_t* stage_out = smem_gen + static_cast<uint32_t>(S) * kPairStageBytes + kBarrierBytes + (warp - 2) * kStageOutBytes;
     const bool rescale = p.scale_a != nullptr;
     const float inv = rescale ? 1.0f / (__ldg(p.scale_a) * __ldg(p.scale_b)) : 1.0f;
     int acc = 0;
@@ -476,7 +540,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       const bool row_ok = row < p.M;
       const uint32_t t_row = tmem_base + static_cast<uint32_t>(acc) * kAccCols + (static_cast<uint32_t>(quad * 32) << 16);
       const int n0 = n_idx * 256;
-      epilogue_tile(p, t_row, row, row_ok, n0, col_half ? 128 : 0, col_half ? 256 : 128, 0, inv, amax_bits);
+      epilogue_tile(p, t_row, row, row_ok, n0, col_half ? 128 : 0, col_half ? 256 : 128, 0, inv, amax_bits, stage_out);
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(tmem_empty_bar(acc), 0));
@@ -593,7 +657,7 @@ cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
   gp.kblocks_total = static_cast<int>((q.K + kBlockKBytes - 1) / kBlockKBytes);
   gp.k_splits = 1;
   gp.kblocks_per_split = gp.kblocks_total;
-  int stages = static_cast<int>((kSmemBudget - 1024 - kBarrierBytes) / kPairStageBytes);
+  int stages = static_cast<int>((kSmemBudget - 1024 - kBarrierBytes - kStagingBytes) / kPairStageBytes);
   if (stages > kMaxStages) stages = kMaxStages;
   gp.num_stages = stages;
   // instruction descriptor without N (set per tile): fp32 accumulate, formats, B major, M = 256
@@ -613,7 +677,7 @@ cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
   long long pairs = sm_count() / 2;
   if (total_tiles < pairs) pairs = total_tiles;
   const int grid = static_cast<int>(pairs * 2);
-  const size_t smem = static_cast<size_t>(stages) * kPairStageBytes + kBarrierBytes + 1024;
+  const size_t smem = static_cast<size_t>(stages) * kPairStageBytes + kBarrierBytes + kStagingBytes + 1024;
   if (q.b_mn_major) return launch_pair_variant<true>(ta, tb, gp, grid, smem, stream);
   return launch_pair_variant<false>(ta, tb, gp, grid, smem, stream);
 }
@@ -648,7 +712,7 @@ cudaError_t launch_gemm_fp8(const GemmProblem& q, cudaStream_t stream) {
   gp.kblocks_per_split = (gp.kblocks_total + gp.k_splits - 1) / gp.k_splits;
   gp.k_splits = (gp.kblocks_total + gp.kblocks_per_split - 1) / gp.kblocks_per_split;  // no empty split
   const uint32_t stage_bytes = kATileBytes + static_cast<uint32_t>(q.block_n) * kBlockKBytes;
-  int stages = static_cast<int>((kSmemBudget - 1024 - kBarrierBytes) / stage_bytes);
+  int stages = static_cast<int>((kSmemBudget - 1024 - kBarrierBytes - kStagingBytes) / stage_bytes);
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2) return cudaErrorInvalidValue;
   gp.num_stages = stages;
@@ -674,7 +738,7 @@ cudaError_t launch_gemm_fp8(const GemmProblem& q, cudaStream_t stream) {
   const long long total_tiles = static_cast<long long>(gp.m_tiles) * gp.n_tiles * gp.k_splits;
   int grid = sm_count();
   if (total_tiles < grid) grid = static_cast<int>(total_tiles);
-  const size_t smem = static_cast<size_t>(stages) * stage_bytes + kBarrierBytes + 1024;
+  const size_t smem = static_cast<size_t>(stages) * stage_bytes + kBarrierBytes + kStagingBytes + 1024;
   if (q.a_mn_major) {
     if (q.b_mn_major) return launch_variant<true, true>(ta, tb, gp, grid, smem, stream);
     return launch_variant<true, false>(ta, tb, gp, grid, smem, stream);
