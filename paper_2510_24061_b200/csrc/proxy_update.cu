@@ -50,7 +50,8 @@ __global__ void __launch_bounds__(256) sgd_score_kernel(float* __restrict__ dbuf
   if (threadIdx.x < rows) {
     const float* a = sabs + threadIdx.x * (r + 1);
     float s = 0.0f;
-    for (int j = 0; j < r; ++j) s = __fadd_rn(s, a[j]);
+#pragma unroll 8
+    for (int j = 0; j < r; ++j) s = __fadd_rn(s, a[j]);   // strictly left to right; the loads run ahead
     score[row0 + threadIdx.x] = s;
   }
 }
@@ -114,9 +115,12 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
 #pragma unroll
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
-    for (int i = lo; i < hi; ++i) {
-      const uint32_t b = bits[i];
-      if ((b & mask) == prefix) atomicAdd(&hist[pass][(b >> shift) & 0xFF], 1);
+    // scores of one layer cluster in a few bins, so lanes that hit the same bin add once for all of them
+    for (int i0 = lo; i0 < lo + E; ++i0) {          // E iterations for every thread: the warp stays converged
+      const bool live = i0 < hi && ((bits[i0] & mask) == prefix);
+      const uint32_t bin = live ? ((bits[i0] >> shift) & 0xFF) : 0x100u + lane;   // dead lanes match nobody
+      const uint32_t peers = __match_any_sync(0xFFFFFFFFu, bin);
+      if (live && lane == __ffs(peers) - 1) atomicAdd(&hist[pass][bin], __popc(peers));
     }
     __syncthreads();
     if (warp == 0) {

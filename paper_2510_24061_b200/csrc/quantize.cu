@@ -140,8 +140,10 @@ __global__ void __launch_bounds__(kThreads) cast_kernel(const void* __restrict__
     if (out.amax_out && nparts > 0) *out.amax_out = amax;
     if (out.clear_word) *out.clear_word = 0.0f;
   }
+  // walk the tensor from its end: the absmax pass read it front to back, so its tail is what is still in L2
   const int64_t nvec = count / 16;
-  for (int64_t v = blockIdx.x * (int64_t)kThreads + threadIdx.x; v < nvec; v += (int64_t)gridDim.x * kThreads) {
+  for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < nvec; i += (int64_t)gridDim.x * kThreads) {
+    const int64_t v = nvec - 1 - i;
     float x[16];
     load16<kDt>(src, v * 16, x);
     reinterpret_cast<uint4*>(dst)[v] = cast16<kFmt>(x, premul, use_premul, s);
