@@ -115,20 +115,9 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
 #pragma unroll
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
-    // scores of one layer cluster in one or two bins: the lanes that share the first live lane's bin add
-    // once for all of them, the rest add individually
-    for (int i0 = lo; i0 < lo + E; ++i0) {          // E iterations for every thread: the warp stays converged
-      const uint32_t b = i0 < hi ? bits[i0] : 0u;
-      const bool live = i0 < hi && ((b & mask) == prefix);
-      const uint32_t bin = (b >> shift) & 0xFF;
-      const uint32_t act = __ballot_sync(0xFFFFFFFFu, live);
-      if (act != 0) {
-        const int leader = __ffs(act) - 1;
-        const uint32_t lead_bin = __shfl_sync(0xFFFFFFFFu, bin, leader);
-        const uint32_t same = __ballot_sync(0xFFFFFFFFu, live && bin == lead_bin);
-        if (lane == leader) atomicAdd(&hist[pass][lead_bin], __popc(same));
-        else if (live && bin != lead_bin) atomicAdd(&hist[pass][bin], 1);
-      }
+    for (int i = lo; i < hi; ++i) {
+      const uint32_t b = bits[i];
+      if ((b & mask) == prefix) atomicAdd(&hist[pass][(b >> shift) & 0xFF], 1);
     }
     __syncthreads();
     if (warp == 0) {
