@@ -37,6 +37,9 @@ UNIT = "TFLOP/s"
 FP8_OVER_BF16 = 2.0        # nominal dense FP8 : bf16 tensor throughput on B200 (4.5 : 2.25 PFLOP/s)
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read+write of the forward and dX launches on the q projection (36.93 + 37.61 MB) over their FP8 operand
+# bytes (33.82 + 33.55 MB); the ncu summary is under profiles/.  Traffic grows in proportion to the operands.
+DRAM_OVER_OPERAND_BYTES = (36.93 + 37.61) / (33.82 + 33.55)
 
 
 def layer_flops(T, n, m, r):
@@ -284,7 +287,11 @@ def main():
                 "frac_of_burst_peak": achieved / (peaks["bf16_burst"] * FP8_OVER_BF16),
                 "frac_of_nominal_4500": achieved / 4500.0,
                 "launches": launches_big, "avg_launch_ms": t_big / max(launches_big, 1),
-                "gflop_per_launch": f_big / max(launches_big, 1) / 1e9, "traffic": None}
+                "gflop_per_launch": f_big / max(launches_big, 1) / 1e9,
+                "traffic": DRAM_OVER_OPERAND_BYTES * sum((T * n + (m + r) * n) + (T * m + m * n) for _, n, m in linears)
+                / (2.0 * len(linears)),
+                "traffic_note": "bytes per average launch: FP8 operand bytes x 1.106, the dram read+write / operand ratio "
+                                "ncu measured on the q projection (profiles/gemm_fp8_pair_kernel__q_projection_T4096.md)"}
     t_db = sum(ms for name, ms in records if name == "gemm_db")
 
     # ---- stage breakdown (separate untimed-for-value pass with every stage bracketed)
