@@ -172,6 +172,79 @@ def time_oracle_sample(T_sample, r, k, lr, seed=0):
     return flops / dt / 1e12, dt, orc.num_threads(), desc
 
 
+def run_sweep(args):
+    """configs[4]: 4096 -> 11008, rank x tokens x top-k.  Forward and backward depend on (rank, tokens), the proxy
+    update on (rank, top-k); each is timed alone with CUDA events (warm L2 state of a step loop: the calls run back
+    to back on one stream) and set against the FP8 tensor roofline or the HBM / fp32-ALU rooflines."""
+    from paper_2510_24061_b200 import binding as fq
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks = measured_peaks()
+    tensor_peak = peaks["bf16_burst"] * FP8_OVER_BF16          # kernels timed in isolation: burst figure
+    n, m = 4096, 11008
+    ranks = [8, 16, 32, 64, 128]
+    tokens = [512, 2048, 8192, 32768]
+    topks = [0, 64, 512, 4096]
+    iters = 10
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    W = synth.backbone(0, 4, m, n, dev)
+    for r in ranks:
+        A = synth.adapter_a(0, 4, r, n, dev)
+        layer = fq.setup_layer(W, A, None, 1.0)
+        for T in tokens:
+            X = synth.activations(0, 4, T, n, round(0.01 * n), dev)
+            dY = synth.out_grad(0, 4, 0, T, m, dev)
+            ws = layer.workspace(T)
+            out_f = (torch.empty((T, m), dtype=torch.bfloat16, device=dev), torch.empty((T, r), dtype=torch.float32, device=dev),
+                     torch.empty(1, dtype=torch.float32, device=dev), torch.empty(1, dtype=torch.float32, device=dev))
+            out_b = (torch.empty((T, n), dtype=torch.bfloat16, device=dev), torch.empty((m, r), dtype=torch.float32, device=dev),
+                     torch.empty(1, dtype=torch.float32, device=dev))
+            t_f = timed(lambda: fq.melded_forward(layer, X, ws=ws, out=out_f))
+            _, OA, amax_oa, _ = out_f
+            t_b = timed(lambda: fq.melded_backward(layer, dY, OA, amax_oa, ws=ws, out=out_b))
+            f_f = 2.0 * T * n * (m + r)
+            f_b = 2.0 * T * m * n + 2.0 * T * m * r
+            print(json.dumps({"sweep": "fwd_bwd", "n": n, "m": m, "rank": r, "tokens": T,
+                              "fwd_ms": t_f, "fwd_tflops": f_f / t_f / 1e9, "fwd_frac_tensor_peak": f_f / t_f / 1e9 / tensor_peak,
+                              "bwd_ms": t_b, "bwd_tflops": f_b / t_b / 1e9, "bwd_frac_tensor_peak": f_b / t_b / 1e9 / tensor_peak,
+                              "tensor_peak_tflops": tensor_peak}), flush=True)
+            del X, dY, out_f, out_b, ws
+            layer._ws = None
+            torch.cuda.empty_cache()
+        dB = synth.normal_bf16(0, 77, (m, r), 1e-3, dev).float()
+        ws = layer.workspace(1)
+        for k in topks:
+            idx = torch.empty(max(k, 1), dtype=torch.int32, device=dev)
+            t_p = timed(lambda: fq.proxy_update(layer, dB, 2e-4, k, ws=ws, idx_out=idx if k > 0 else None))
+            bytes_p = 12.0 * m * r + 4.0 * m + k * (2.0 * n + 8.0 * r) + r * n   # optimizer+score pass, merged rows, A~ once
+            fma = float(k) * n * r
+            alu_peak = 148 * 128 * peaks_clock_ghz() * 1e9                    # fp32 fma per second
+            print(json.dumps({"sweep": "proxy", "n": n, "m": m, "rank": r, "topk": k, "proxy_ms": t_p,
+                              "algorithmic_gbs": bytes_p / t_p / 1e6, "frac_hbm_peak": bytes_p / t_p / 1e6 / peaks["hbm"],
+                              "merge_gfma_per_s": fma / t_p / 1e6, "frac_fp32_fma_peak": fma / (t_p * 1e-3) / alu_peak,
+                              "hbm_peak_gbs": peaks["hbm"]}), flush=True)
+
+
+def peaks_clock_ghz():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            return float(json.load(fh)["sm_max_mhz"]) / 1e3
+    except Exception:
+        return 1.965
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -180,6 +253,8 @@ def main():
     ap.add_argument("--impl", default="falqon", choices=["falqon", "reference"])
     ap.add_argument("--oracle-tokens", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="configs[4]: sweep rank x tokens x top-k on the 4096->11008 projection; one JSON line per point")
     ap.add_argument("--only", default=None, help="profiling aid: restrict the workload to one projection (q,k,v,o,gate,up,down)")
     args = ap.parse_args()
 
@@ -196,6 +271,11 @@ def main():
                             + ("" if args.only is None else f" -- RESTRICTED to '{args.only}' (profiling aid, not a bench line)"),
                 "tokens": T, "rank": r, "topk": k, "matrices": len(linears), "gflop_per_step": flops_step / 1e9,
                 "l2": "inputs larger than L2 (0.85 GB touched per step)", "parallelism": f"replicas x{world}"}
+
+    if args.sweep:
+        if rank == 0:
+            run_sweep(args)
+        return
 
     if args.impl == "reference":
         if rank != 0:
