@@ -80,6 +80,12 @@ typedef enum {
  * most T_max tokens.  Returns 0 if the shape is not supported. */
 size_t falqon_workspace_bytes(int64_t m, int64_t n, int64_t r, int64_t T_max);
 
+/* Clears the control words at the start of a workspace (the counters of the in-kernel barriers; 1 KB).
+ * Call it once after allocating a workspace, before the first falqon_melded_forward / _backward that uses it, and
+ * again after a call reported FALQON_ERR_TIMEOUT.  The calls leave those words cleared, so a workspace that is
+ * only ever passed to this library needs it once.  Enqueues a memset on `stream`. */
+int falqon_workspace_init(void *ws, size_t ws_bytes, falqon_stream stream);
+
 /* Host, pure.  Byte offset and size of a region inside a workspace laid out for (m, n, r, T_max).
  * Returns FALQON_OK or FALQON_ERR_INVALID_ARG. */
 int falqon_workspace_region(int64_t m, int64_t n, int64_t r, int64_t T_max, falqon_ws_region which,

@@ -22,7 +22,7 @@ WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE, WS_DB_PART = range(6)
 
 EXPORTS = ["falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_last_device_status", "falqon_launch_count",
-           "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static"]
+           "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static", "falqon_workspace_init"]
 STATIC_MAX_ROWS = 16384
 STAGES = ["quant_x", "gemm_fwd", "quant_dy", "quant_oa", "gemm_dx", "gemm_db", "reduce_db", "sgd_score", "topk", "merge"]
 
@@ -42,6 +42,8 @@ lib.falqon_workspace_bytes.restype = _sz
 lib.falqon_workspace_bytes.argtypes = [_i64, _i64, _i64, _i64]
 lib.falqon_workspace_region.restype = _i
 lib.falqon_workspace_region.argtypes = [_i64, _i64, _i64, _i64, _i, C.POINTER(_sz), C.POINTER(_sz)]
+lib.falqon_workspace_init.restype = _i
+lib.falqon_workspace_init.argtypes = [_p, _sz, _p]
 lib.falqon_quantize.restype = _i
 lib.falqon_quantize.argtypes = [_p, _i, _i64, _i64, _i, _i, _p, _f, _p, _p, _p, _p, _sz, _p]
 lib.falqon_melded_forward.restype = _i
@@ -105,7 +107,13 @@ class Layer:
             raise FalqonError("falqon_workspace_bytes", ERR_INVALID_ARG)
         if self._ws is None or self._ws.numel() < need:
             self._ws = torch.empty(need, dtype=torch.uint8, device=self.wq.device)
+            workspace_init(self._ws)
         return self._ws
+
+
+def workspace_init(ws: torch.Tensor):
+    """falqon_workspace_init: clears the control words of a freshly allocated workspace."""
+    _check("falqon_workspace_init", lib.falqon_workspace_init(_ptr(ws), ws.numel(), _stream()))
 
 
 def workspace_bytes(m: int, n: int, r: int, T: int) -> int:

@@ -32,6 +32,8 @@ struct WorkspaceLayout {
 
 constexpr size_t kHeaderBytes = 8192;     // scales at 0, absmax partials at kPartialsOffset
 constexpr size_t kPartialsOffset = 1024;
+constexpr size_t kSyncOffset = 256;       // counters of the in-kernel barriers: zero between calls (falqon_workspace_init)
+constexpr size_t kInitBytes = 1024;       // what falqon_workspace_init clears
 static_assert(kPartialsOffset + kMaxAbsmaxParts * sizeof(uint32_t) <= kHeaderBytes, "header too small");
 
 bool shape_ok(int64_t m, int64_t n, int64_t r) {
@@ -165,6 +167,12 @@ int falqon_quantize(const void* src, falqon_dtype src_dt, int64_t rows, int64_t 
   return FALQON_OK;
 }
 
+int falqon_workspace_init(void* ws, size_t ws_bytes, falqon_stream stream) {
+  if (ws == nullptr || !aligned16(ws) || ws_bytes < kInitBytes) return FALQON_ERR_WORKSPACE;
+  FALQON_CUDA(cudaMemsetAsync(ws, 0, kInitBytes, stream));
+  return FALQON_OK;
+}
+
 int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_dt, int64_t T, void* Y, falqon_dtype y_dt,
                           float* OA, float* amax_oa, float* s_x_out, void* ws, size_t ws_bytes, falqon_stream stream) {
   if (!layer_ok(L) || X == nullptr || Y == nullptr || OA == nullptr || amax_oa == nullptr || T < 1 || !dtype_ok(x_dt) ||
@@ -184,10 +192,8 @@ int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_d
   uint32_t* partial = reinterpret_cast<uint32_t*>(base + w.scales + kPartialsOffset);
   {
     StageTimer timer(FALQON_STAGE_QUANT_X, stream);
-    int nparts = 0;
-    FALQON_CUDA(launch_absmax(X, x_dt, T * n, 1.0f, partial, &nparts, stream));
-    FALQON_CUDA(launch_cast_per_tensor(X, x_dt, T * n, kE4M3, 1.0f, partial, nparts, nullptr, xq, scales + 1, s_x_out,
-                                       scales + 0, amax_oa, stream));
+    FALQON_CUDA(launch_quantize_fused(X, x_dt, T * n, kE4M3, xq, partial, base + w.scales + kSyncOffset, scales + 1, s_x_out,
+                                      scales + 0, amax_oa, status, stream));
   }
   // S2: [Y | O_A] = x~ W~'^T / (s_W s_x), amax(O_A) from the epilogue
   GemmProblem g{};
@@ -228,10 +234,8 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
   uint32_t* partial = reinterpret_cast<uint32_t*>(base + w.scales + kPartialsOffset);
   {
     StageTimer timer(FALQON_STAGE_QUANT_DY, stream);
-    int nparts = 0;
-    FALQON_CUDA(launch_absmax(dY, dy_dt, T * m, 1.0f, partial, &nparts, stream));
-    FALQON_CUDA(launch_cast_per_tensor(dY, dy_dt, T * m, kE5M2, 1.0f, partial, nparts, nullptr, gq, scales + 3, s_g_out,
-                                       scales + 2, nullptr, stream));
+    FALQON_CUDA(launch_quantize_fused(dY, dy_dt, T * m, kE5M2, gq, partial, base + w.scales + kSyncOffset, scales + 3, s_g_out,
+                                      scales + 2, nullptr, status, stream));
   }
   // S5a: O~_A, s_OA = Q_e4m3(O_A), written transposed for the dB product
   {

@@ -51,6 +51,11 @@ cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, i
                                    const uint32_t* partial, int nparts, const float* scale_in, uint8_t* dst,
                                    float* scale_out, float* scale_out2, float* amax_out, float* clear_word,
                                    cudaStream_t stream);
+// Per-tensor absmax scaling in one kernel (absmax, grid barrier, cast).  `sync` points at 8 bytes of workspace that
+// are zero before the call and are left zero by it; `partial` holds up to kMaxAbsmaxParts words.
+cudaError_t launch_quantize_fused(const void* src, int src_dt, int64_t count, int fmt, uint8_t* dst, uint32_t* partial,
+                                  void* sync, float* scale_out, float* scale_out2, float* amax_out, float* clear_word,
+                                  int* status, cudaStream_t stream);
 cudaError_t launch_quantize_per_row(const void* src, int src_dt, int64_t rows, int64_t cols, int fmt, float premul,
                                     const float* scale_in, uint8_t* dst, float* scale_out, float* amax_out,
                                     cudaStream_t stream);

@@ -157,6 +157,151 @@ __global__ void __launch_bounds__(kThreads) cast_kernel(const void* __restrict__
   }
 }
 
+// ---- fused per-tensor quantizer: absmax, a grid-wide barrier, then the cast, in ONE kernel.
+// All CTAs are co-resident (the host sizes the grid from the occupancy), so a CTA can wait for the others.
+// Each thread keeps the first kCache 16-element vectors it read in registers, so for tensors up to
+// grid x 256 x kCache x 16 elements the cast never touches memory again; what does not fit is re-read, most
+// recent first (that is what L2 still holds).  The barrier is two counters in the caller's workspace that
+// start at zero and are put back to zero by the last CTA to leave, and its wait is bounded.
+struct GridSync {
+  unsigned int arrive;
+  unsigned int depart;
+};
+
+__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+template <int kDt> struct RawVec;
+template <> struct RawVec<kBF16> { uint4 a, b; };              // 16 bf16
+template <> struct RawVec<kF32> { float4 a, b, c, d; };        // 16 fp32
+
+template <int kDt>
+__device__ __forceinline__ RawVec<kDt> load_raw(const void* src, int64_t elem);
+template <>
+__device__ __forceinline__ RawVec<kBF16> load_raw<kBF16>(const void* src, int64_t elem) {
+  const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(src) + elem);
+  RawVec<kBF16> r; r.a = __ldg(p); r.b = __ldg(p + 1); return r;
+}
+template <>
+__device__ __forceinline__ RawVec<kF32> load_raw<kF32>(const void* src, int64_t elem) {
+  const float4* p = reinterpret_cast<const float4*>(static_cast<const float*>(src) + elem);
+  RawVec<kF32> r; r.a = __ldg(p); r.b = __ldg(p + 1); r.c = __ldg(p + 2); r.d = __ldg(p + 3); return r;
+}
+__device__ __forceinline__ void unpack_raw(const RawVec<kBF16>& r, float (&v)[16]) {
+  const uint32_t w[8] = {r.a.x, r.a.y, r.a.z, r.a.w, r.b.x, r.b.y, r.b.z, r.b.w};
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+__device__ __forceinline__ void unpack_raw(const RawVec<kF32>& r, float (&v)[16]) {
+  v[0] = r.a.x; v[1] = r.a.y; v[2] = r.a.z; v[3] = r.a.w; v[4] = r.b.x; v[5] = r.b.y; v[6] = r.b.z; v[7] = r.b.w;
+  v[8] = r.c.x; v[9] = r.c.y; v[10] = r.c.z; v[11] = r.c.w; v[12] = r.d.x; v[13] = r.d.y; v[14] = r.d.z; v[15] = r.d.w;
+}
+
+template <int kDt, int kFmt>
+__global__ void __launch_bounds__(kThreads) quantize_fused_kernel(const void* __restrict__ src, int64_t count,
+                                                                  uint8_t* __restrict__ dst, uint32_t* __restrict__ partial,
+                                                                  GridSync* __restrict__ sync, CastOutputs out,
+                                                                  int* __restrict__ status) {
+  constexpr int kCache = (kDt == kBF16) ? 4 : 2;
+  __shared__ uint32_t red[32];
+  __shared__ int s_ok;
+  pdl_trigger();
+  pdl_wait();
+  const int64_t nvec = count / 16;
+  const int64_t stride = (int64_t)gridDim.x * kThreads;
+  const int64_t first = blockIdx.x * (int64_t)kThreads + threadIdx.x;
+  RawVec<kDt> cache[kCache];
+  uint32_t m = 0;
+  float x[16];
+#pragma unroll
+  for (int i = 0; i < kCache; ++i) {
+    const int64_t v = first + i * stride;
+    if (v < nvec) cache[i] = load_raw<kDt>(src, v * 16);
+  }
+#pragma unroll
+  for (int i = 0; i < kCache; ++i) {
+    const int64_t v = first + i * stride;
+    if (v < nvec) {
+      unpack_raw(cache[i], x);
+#pragma unroll
+      for (int e = 0; e < 16; ++e) m = max(m, abs_bits(x[e]));
+    }
+  }
+  int64_t v_last = first + (int64_t)(kCache - 1) * stride;   // last vector index visited by this thread
+  for (int64_t v = first + (int64_t)kCache * stride; v < nvec; v += stride) {
+    load16<kDt>(src, v * 16, x);
+#pragma unroll
+    for (int e = 0; e < 16; ++e) m = max(m, abs_bits(x[e]));
+    v_last = v;
+  }
+  if (blockIdx.x == 0) {  // ragged tail (count not a multiple of 16)
+    for (int64_t e = nvec * 16 + threadIdx.x; e < count; e += kThreads) m = max(m, abs_bits(load1<kDt>(src, e)));
+  }
+  m = block_max_u32(m, red);
+  // ---- grid barrier
+  if (threadIdx.x == 0) {
+    partial[blockIdx.x] = m;
+    __threadfence();
+    atomicAdd(&sync->arrive, 1u);
+    int ok = 1;
+    if (ld_acquire_gpu(&sync->arrive) < gridDim.x) {
+      const uint64_t t0 = global_timer_ns();
+      for (;;) {
+        if (ld_acquire_gpu(&sync->arrive) >= gridDim.x) break;
+        __nanosleep(40);
+        if (global_timer_ns() - t0 > kWaitLimitNs) { ok = 0; atomicExch(status, kStatusTimeout); break; }
+      }
+    }
+    s_ok = ok;
+  }
+  __syncthreads();
+  if (s_ok) {
+    uint32_t mb = 0;
+    for (int i = threadIdx.x; i < (int)gridDim.x; i += kThreads) mb = max(mb, __ldcg(partial + i));
+    const float amax = __uint_as_float(block_max_u32(mb, red));
+    const float s = scale_from_amax(amax, kFmt);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+      if (out.scale_out) *out.scale_out = s;
+      if (out.scale_out2) *out.scale_out2 = s;
+      if (out.amax_out) *out.amax_out = amax;
+      if (out.clear_word) *out.clear_word = 0.0f;
+    }
+    // streamed part, most recent first
+    for (int64_t v = v_last; v >= first + (int64_t)kCache * stride; v -= stride) {
+      load16<kDt>(src, v * 16, x);
+      reinterpret_cast<uint4*>(dst)[v] = cast16<kFmt>(x, 1.0f, false, s);
+    }
+#pragma unroll
+    for (int i = kCache - 1; i >= 0; --i) {
+      const int64_t v = first + i * stride;
+      if (v < nvec) {
+        unpack_raw(cache[i], x);
+        reinterpret_cast<uint4*>(dst)[v] = cast16<kFmt>(x, 1.0f, false, s);
+      }
+    }
+    if (blockIdx.x == 0) {
+      for (int64_t e = nvec * 16 + threadIdx.x; e < count; e += kThreads)
+        dst[e] = static_cast<uint8_t>(cvt_fp8x2<kFmt>(__fmul_rn(load1<kDt>(src, e), s), 0.0f) & 0xFF);
+    }
+  }
+  // ---- leave: the last CTA puts the counters back to zero for the next call
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned int prev = atomicAdd(&sync->depart, 1u);
+    if (prev == gridDim.x - 1) {
+      sync->arrive = 0u;
+      sync->depart = 0u;
+      __threadfence();
+    }
+  }
+}
+
 // ---- per-row scaling: one CTA per row, the row is read twice (second time from L1/L2)
 template <int kDt, int kFmt>
 __global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const void* __restrict__ src, int64_t cols, float premul,
@@ -273,6 +418,39 @@ cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, i
   if (src_dt == kBF16) { if (fmt == kE4M3) FALQON_CAST(kBF16, kE4M3); else FALQON_CAST(kBF16, kE5M2); }
   else { if (fmt == kE4M3) FALQON_CAST(kF32, kE4M3); else FALQON_CAST(kF32, kE5M2); }
 #undef FALQON_CAST
+}
+
+template <int kDt, int kFmt>
+cudaError_t launch_fused_variant(const void* src, int64_t count, uint8_t* dst, uint32_t* partial, void* sync,
+                                 const CastOutputs& out, int* status, cudaStream_t stream) {
+  static int blocks_per_sm = 0;
+  if (blocks_per_sm == 0) {
+    int b = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, quantize_fused_kernel<kDt, kFmt>, kThreads, 0);
+    if (e != cudaSuccess) return e;
+    blocks_per_sm = b < 1 ? 1 : b;
+  }
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  int64_t grid = (count / 16 + kThreads - 1) / kThreads;
+  const int64_t resident = static_cast<int64_t>(blocks_per_sm) * sms;
+  if (grid > resident) grid = resident;
+  if (grid > kMaxAbsmaxParts) grid = kMaxAbsmaxParts;
+  if (grid < 1) grid = 1;
+  return launch_pdl(quantize_fused_kernel<kDt, kFmt>, dim3(static_cast<unsigned>(grid)), dim3(kThreads), 0, stream, 1, src,
+                    count, dst, partial, static_cast<GridSync*>(sync), out, status);
+}
+
+cudaError_t launch_quantize_fused(const void* src, int src_dt, int64_t count, int fmt, uint8_t* dst, uint32_t* partial,
+                                  void* sync, float* scale_out, float* scale_out2, float* amax_out, float* clear_word,
+                                  int* status, cudaStream_t stream) {
+  const CastOutputs out{scale_out, scale_out2, amax_out, clear_word};
+  if (src_dt == kBF16) {
+    if (fmt == kE4M3) return launch_fused_variant<kBF16, kE4M3>(src, count, dst, partial, sync, out, status, stream);
+    return launch_fused_variant<kBF16, kE5M2>(src, count, dst, partial, sync, out, status, stream);
+  }
+  if (fmt == kE4M3) return launch_fused_variant<kF32, kE4M3>(src, count, dst, partial, sync, out, status, stream);
+  return launch_fused_variant<kF32, kE5M2>(src, count, dst, partial, sync, out, status, stream);
 }
 
 cudaError_t launch_quantize_per_row(const void* src, int src_dt, int64_t rows, int64_t cols, int fmt, float premul,
