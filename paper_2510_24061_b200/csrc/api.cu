@@ -33,7 +33,10 @@ struct WorkspaceLayout {
 constexpr size_t kHeaderBytes = 8192;     // scales at 0, absmax partials at kPartialsOffset
 constexpr size_t kPartialsOffset = 1024;
 constexpr size_t kSyncOffset = 256;       // counters of the in-kernel barriers: zero between calls (falqon_workspace_init)
-constexpr size_t kInitBytes = 1024;       // what falqon_workspace_init clears
+constexpr size_t kDoneOffset = 320;       // last-CTA counter of the fused optimizer/score/selection kernel
+constexpr size_t kGroupCountersOffset = 6144;   // row-group counters of the merge (2 KB: up to 512 groups of 32 rows)
+constexpr size_t kMaxMergeGroups = (kHeaderBytes - kGroupCountersOffset) / sizeof(unsigned int);
+constexpr size_t kInitBytes = kHeaderBytes;  // what falqon_workspace_init clears
 static_assert(kPartialsOffset + kMaxAbsmaxParts * sizeof(uint32_t) <= kHeaderBytes, "header too small");
 
 bool shape_ok(int64_t m, int64_t n, int64_t r) {
@@ -288,19 +291,17 @@ int falqon_proxy_update(const falqon_layer* L, const float* dB, float lr, int64_
   float* score = reinterpret_cast<float*>(base + w.score);
   int32_t* sel = reinterpret_cast<int32_t*>(base + w.sel_idx);
   const int64_t m = L->m, n = L->n, r = L->r;
+  unsigned int* done_counter = reinterpret_cast<unsigned int*>(base + w.scales + kDoneOffset);
+  unsigned int* group_counters = reinterpret_cast<unsigned int*>(base + w.scales + kGroupCountersOffset);
+  const bool fused_merge = static_cast<size_t>(merge_group_count(k)) <= kMaxMergeGroups;
   {
-    StageTimer timer(FALQON_STAGE_SGD_SCORE, stream);
-    FALQON_CUDA(launch_sgd_score(L->dbuf, dB, lr, m, r, score, stream));
+    StageTimer timer(FALQON_STAGE_SGD_SCORE, stream);   // optimizer step, scores and (k > 0) the selection: one kernel
+    FALQON_CUDA(launch_sgd_score_topk(L->dbuf, dB, lr, m, r, k, score, sel, idx_out, done_counter, stream));
   }
   if (k > 0) {
-    {
-      StageTimer timer(FALQON_STAGE_TOPK, stream);
-      FALQON_CUDA(launch_topk(score, m, k, sel, idx_out, stream));
-    }
-    {
-      StageTimer timer(FALQON_STAGE_MERGE, stream);
-      FALQON_CUDA(launch_merge_rows(L->wq, L->dbuf, sel, k, m, n, r, stream));
-    }
+    StageTimer timer(FALQON_STAGE_MERGE, stream);
+    if (fused_merge) FALQON_CUDA(launch_merge_rows_fused(L->wq, L->dbuf, sel, k, m, n, r, group_counters, stream));
+    else FALQON_CUDA(launch_merge_rows(L->wq, L->dbuf, sel, k, m, n, r, stream));
   }
   return FALQON_OK;
 }
@@ -362,9 +363,9 @@ int falqon_launch_count(const char* entry_point, int64_t m, int64_t n, int64_t r
   (void)m; (void)n; (void)r; (void)T;
   if (entry_point == nullptr) return 0;
   if (std::strcmp(entry_point, "falqon_quantize") == 0) return 2;           // absmax, cast
-  if (std::strcmp(entry_point, "falqon_melded_forward") == 0) return 3;     // absmax, cast, GEMM
-  if (std::strcmp(entry_point, "falqon_melded_backward") == 0) return 6;    // absmax, cast, O_A cast, dX, dB, reduce
-  if (std::strcmp(entry_point, "falqon_proxy_update") == 0) return k > 0 ? 4 : 1;  // score, top-k, merge, clear
+  if (std::strcmp(entry_point, "falqon_melded_forward") == 0) return 2;     // fused quantize, GEMM
+  if (std::strcmp(entry_point, "falqon_melded_backward") == 0) return 5;    // fused quantize, O_A cast, dX, dB, reduce
+  if (std::strcmp(entry_point, "falqon_proxy_update") == 0) return k > 0 ? 2 : 1;  // optimizer+score+top-k, merge+clear
   return 0;
 }
 

@@ -91,5 +91,13 @@ size_t topk_scratch_bytes(int64_t m);
 cudaError_t launch_topk(const float* score, int64_t m, int64_t k, int32_t* sel_idx, void* idx_copy, cudaStream_t stream);
 cudaError_t launch_merge_rows(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
                               int64_t r, cudaStream_t stream);
+// Fused forms used with an initialised workspace: optimizer step + scores + selection in one kernel (done_counter:
+// one word, zero between calls), and the merge that also clears the merged DeltaBuffer rows (group_counters:
+// merge_group_count(k) words, zero between calls).
+int merge_group_count(int64_t k);
+cudaError_t launch_sgd_score_topk(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, int64_t k, float* score,
+                                  int32_t* sel_idx, int32_t* idx_copy, unsigned int* done_counter, cudaStream_t stream);
+cudaError_t launch_merge_rows_fused(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
+                                    int64_t r, unsigned int* group_counters, cudaStream_t stream);
 
 }  // namespace falqon

@@ -64,9 +64,11 @@ __global__ void __launch_bounds__(256) sgd_score_kernel(float* __restrict__ dbuf
 constexpr int kTopkThreads = 1024;
 constexpr int kTopkSmemRows = 48 * 1024;   // scores are staged in shared memory up to this many rows
 
-// Exclusive prefix sum of one int per thread over the whole CTA (1024 threads); *total = CTA sum.
+// Exclusive prefix sum of one int per thread over the whole CTA (any multiple of 32 threads up to 1024);
+// *total = CTA sum.
 __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums /* [32] */, int* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nwarps = blockDim.x >> 5;
   int incl = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -76,7 +78,7 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums /* [32
   if (lane == 31) warp_sums[warp] = incl;
   __syncthreads();
   if (warp == 0) {
-    const int w = warp_sums[lane];
+    const int w = lane < nwarps ? warp_sums[lane] : 0;
     int wi = w;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -90,25 +92,24 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums /* [32
   return warp_sums[warp] + incl - v;
 }
 
-__global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restrict__ score, int m, int k,
-                                                            int32_t* __restrict__ sel_idx, int32_t* __restrict__ idx_out,
-                                                            int use_smem) {
-  extern __shared__ uint32_t s_bits[];          // [m] when use_smem
+// The whole selection, run by one CTA (all of its threads).  s_bits: shared-memory staging for the m scores, or
+// null to read them from global memory every time.
+__device__ __forceinline__ void topk_block(const float* __restrict__ score, int m, int k, int32_t* __restrict__ sel_idx,
+                                           int32_t* __restrict__ idx_out, uint32_t* s_bits) {
   __shared__ int hist[4][256];
   __shared__ int warp_sums_a[32], warp_sums_b[32];
   __shared__ int s_total_a, s_total_b;
   __shared__ uint32_t s_digit[4], s_remaining[4];
   const uint32_t* gbits = reinterpret_cast<const uint32_t*>(score);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  pdl_trigger();
-  pdl_wait();
+  const int nthreads = blockDim.x;
 
-  for (int i = tid; i < 4 * 256; i += kTopkThreads) (&hist[0][0])[i] = 0;
-  if (use_smem)
-    for (int i = tid; i < m; i += kTopkThreads) s_bits[i] = gbits[i];
+  for (int i = tid; i < 4 * 256; i += nthreads) (&hist[0][0])[i] = 0;
+  if (s_bits != nullptr)
+    for (int i = tid; i < m; i += nthreads) s_bits[i] = __ldcg(gbits + i);
   __syncthreads();
-  const uint32_t* bits = use_smem ? s_bits : gbits;
-  const int E = (m + kTopkThreads - 1) / kTopkThreads;
+  const uint32_t* bits = s_bits != nullptr ? s_bits : gbits;
+  const int E = (m + nthreads - 1) / nthreads;
   const int lo = min(tid * E, m), hi = min(lo + E, m);
 
   uint32_t prefix = 0, mask = 0, remaining = static_cast<uint32_t>(k);
@@ -174,6 +175,61 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
   }
 }
 
+__global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restrict__ score, int m, int k,
+                                                            int32_t* __restrict__ sel_idx, int32_t* __restrict__ idx_out,
+                                                            int use_smem) {
+  extern __shared__ uint32_t s_bits_dyn[];          // [m] when use_smem
+  pdl_trigger();
+  pdl_wait();
+  topk_block(score, m, k, sel_idx, idx_out, use_smem ? s_bits_dyn : nullptr);
+}
+
+// ---- optimizer step + row scores + selection in ONE kernel: CTAs of 1024 threads take 128 rows each; the CTA
+// that finishes last (a counter in the workspace that is zero between calls) runs the selection on all scores.
+constexpr int kFusedScoreRows = 128;
+__global__ void __launch_bounds__(kTopkThreads) sgd_score_topk_kernel(float* __restrict__ dbuf, const float* __restrict__ dB,
+                                                                      float neg_lr, int m, int r, int k,
+                                                                      float* __restrict__ score, int32_t* __restrict__ sel_idx,
+                                                                      int32_t* __restrict__ idx_out,
+                                                                      unsigned int* __restrict__ done_counter, int use_smem) {
+  extern __shared__ float fused_smem[];  // [kFusedScoreRows][r + 1] floats, later the m staged scores
+  __shared__ int s_last;
+  pdl_trigger();
+  pdl_wait();
+  const int row0 = blockIdx.x * kFusedScoreRows;
+  const int rows = min(kFusedScoreRows, m - row0);
+  const int64_t base = (int64_t)row0 * r;
+  for (int e = threadIdx.x; e < rows * r; e += blockDim.x) {
+    float d = dbuf[base + e];
+    if (dB != nullptr) {
+      d = __fmaf_rn(neg_lr, dB[base + e], d);
+      dbuf[base + e] = d;
+    }
+    const int i = e / r, j = e - i * r;
+    fused_smem[i * (r + 1) + j] = fabsf(d);
+  }
+  __syncthreads();
+  if (threadIdx.x < rows) {
+    const float* a = fused_smem + threadIdx.x * (r + 1);
+    float s = 0.0f;
+#pragma unroll 8
+    for (int j = 0; j < r; ++j) s = __fadd_rn(s, a[j]);   // strictly left to right; the loads run ahead
+    score[row0 + threadIdx.x] = s;
+  }
+  if (k <= 0) return;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned int prev = atomicAdd(done_counter, 1u);
+    s_last = (prev == gridDim.x - 1) ? 1 : 0;
+    if (s_last) *done_counter = 0u;       // back to zero for the next call
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  topk_block(score, m, k, sel_idx, idx_out, use_smem ? reinterpret_cast<uint32_t*>(fused_smem) : nullptr);
+}
+
 // ---- W~[i][:] <- sat_rne_e4m3(W~[i][:] + DeltaBuffer[i][:] * A~) for the selected rows.
 // A CTA owns 32 selected rows x 128 columns.  It decodes the r x 128 tile of A~ to fp32 in shared
 // memory once (the FP8 decode is the expensive part, so it is shared by all 32 rows), then each thread
@@ -191,9 +247,9 @@ __device__ __forceinline__ void decode4(uint32_t w, float (&a)[4]) {
   a[0] = p0.x; a[1] = p0.y; a[2] = p1.x; a[3] = p1.y;
 }
 
-__global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __restrict__ wq, const float* __restrict__ dbuf,
+__global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __restrict__ wq, float* dbuf,
                                                                    const int32_t* __restrict__ sel_idx, int k, int64_t m,
-                                                                   int64_t n, int r) {
+                                                                   int64_t n, int r, unsigned int* group_counters) {
   extern __shared__ __align__(16) float merge_smem[];
   float* a_tile = merge_smem;                         // [r][kMergeCols] decoded A~
   float* sdb = merge_smem + (size_t)r * kMergeCols;   // [kMergeRows][r]
@@ -253,6 +309,23 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __re
     }
   }
   __syncthreads();
+  // With group counters (zero between calls) the CTA that is last to have copied a row group's DeltaBuffer rows
+  // clears those rows, which saves a separate kernel; every CTA of the group has its copy by then.
+  if (group_counters != nullptr) {
+    __shared__ int s_clear;
+    if (threadIdx.x == 0) {
+      const unsigned int prev = atomicAdd(&group_counters[blockIdx.y], 1u);
+      s_clear = (prev == gridDim.x - 1) ? 1 : 0;
+      if (s_clear) group_counters[blockIdx.y] = 0u;
+    }
+    __syncthreads();
+    if (s_clear) {
+      for (int e = threadIdx.x; e < nrows * r4; e += kMergeThreads) {
+        const int q = e / r4, j4 = e - q * r4;
+        *reinterpret_cast<float4*>(dbuf + (int64_t)srow[q] * r + 4 * j4) = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+  }
   const int tx = threadIdx.x % kMergeTx, ty = threadIdx.x / kMergeTx;
   const int lc0 = 4 * tx, lc1 = 64 + 4 * tx;
   const bool ok0 = lc0 < cta_cols, ok1 = lc1 < cta_cols;
@@ -338,8 +411,9 @@ cudaError_t launch_topk(const float* score, int64_t m, int64_t k, int32_t* sel_i
                     static_cast<int>(k), sel_idx, static_cast<int32_t*>(idx_copy), use_smem);
 }
 
-cudaError_t launch_merge_rows(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
-                              int64_t r, cudaStream_t stream) {
+namespace {
+cudaError_t launch_merge_only(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n, int64_t r,
+                              unsigned int* group_counters, cudaStream_t stream) {
   dim3 grid(static_cast<unsigned>((n + kMergeCols - 1) / kMergeCols),
             static_cast<unsigned>((k + kMergeRows - 1) / kMergeRows));
   const size_t smem = sizeof(float) * (static_cast<size_t>(r) * kMergeCols + static_cast<size_t>(kMergeRows) * r);
@@ -349,13 +423,44 @@ cudaError_t launch_merge_rows(uint8_t* wq, float* dbuf, const int32_t* sel_idx, 
     if (ea != cudaSuccess) return ea;
     configured = true;
   }
-  cudaError_t e = launch_pdl(merge_rows_kernel, grid, dim3(kMergeThreads), smem, stream, 1, wq, dbuf, sel_idx,
-                             static_cast<int>(k), m, n, static_cast<int>(r));
+  return launch_pdl(merge_rows_kernel, grid, dim3(kMergeThreads), smem, stream, 1, wq, dbuf, sel_idx, static_cast<int>(k), m,
+                    n, static_cast<int>(r), group_counters);
+}
+}  // namespace
+
+cudaError_t launch_merge_rows(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
+                              int64_t r, cudaStream_t stream) {
+  cudaError_t e = launch_merge_only(wq, dbuf, sel_idx, k, m, n, r, nullptr, stream);
   if (e != cudaSuccess) return e;
   int64_t zb = (k * r + 255) / 256;
   if (zb > 1024) zb = 1024;
   return launch_pdl(zero_rows_kernel, dim3(static_cast<unsigned>(zb)), dim3(256), 0, stream, 1, dbuf, sel_idx,
                     static_cast<int>(k), static_cast<int>(r));
+}
+
+int merge_group_count(int64_t k) { return static_cast<int>((k + kMergeRows - 1) / kMergeRows); }
+
+cudaError_t launch_merge_rows_fused(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
+                                    int64_t r, unsigned int* group_counters, cudaStream_t stream) {
+  return launch_merge_only(wq, dbuf, sel_idx, k, m, n, r, group_counters, stream);
+}
+
+cudaError_t launch_sgd_score_topk(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, int64_t k, float* score,
+                                  int32_t* sel_idx, int32_t* idx_copy, unsigned int* done_counter, cudaStream_t stream) {
+  const int use_smem = m <= kTopkSmemRows ? 1 : 0;
+  size_t smem = sizeof(float) * kFusedScoreRows * (r + 1);
+  if (use_smem && static_cast<size_t>(m) * sizeof(uint32_t) > smem) smem = static_cast<size_t>(m) * sizeof(uint32_t);
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t ea = cudaFuncSetAttribute(sgd_score_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(kTopkSmemRows * sizeof(uint32_t)));
+    if (ea != cudaSuccess) return ea;
+    configured = true;
+  }
+  const int grid = static_cast<int>((m + kFusedScoreRows - 1) / kFusedScoreRows);
+  return launch_pdl(sgd_score_topk_kernel, dim3(grid), dim3(kTopkThreads), smem, stream, 1, dbuf, dB, -lr,
+                    static_cast<int>(m), static_cast<int>(r), static_cast<int>(k), score, sel_idx, idx_copy, done_counter,
+                    use_smem);
 }
 
 }  // namespace falqon

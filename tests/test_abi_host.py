@@ -76,7 +76,7 @@ def test_bad_arguments_are_rejected_on_the_host(fq):
 
 
 def test_launch_counts(fq):
-    assert fq.launch_count("falqon_melded_forward") == 3
-    assert fq.launch_count("falqon_melded_backward") == 6
-    assert fq.launch_count("falqon_proxy_update", k=4) == 4 and fq.launch_count("falqon_proxy_update", k=0) == 1
+    assert fq.launch_count("falqon_melded_forward") == 2
+    assert fq.launch_count("falqon_melded_backward") == 5
+    assert fq.launch_count("falqon_proxy_update", k=4) == 2 and fq.launch_count("falqon_proxy_update", k=0) == 1
     assert fq.launch_count("nope") == 0
