@@ -112,13 +112,36 @@ __device__ __forceinline__ void topk_block(const float* __restrict__ score, int 
   const int E = (m + nthreads - 1) / nthreads;
   const int lo = min(tid * E, m), hi = min(lo + E, m);
 
-  uint32_t prefix = 0, mask = 0, remaining = static_cast<uint32_t>(k);
-#pragma unroll
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
+  // The scores of a layer lie in a narrow range, so their top bits agree: find the highest bit in which any two
+  // differ (from the CTA-wide min and max) and run the radix passes only over the bits from there down.  This
+  // also keeps the first histogram from collapsing into one or two bins.
+  uint32_t lmin = 0xFFFFFFFFu, lmax = 0u;
+  for (int i = lo; i < hi; ++i) { const uint32_t b = bits[i]; lmin = min(lmin, b); lmax = max(lmax, b); }
+  lmin = __reduce_min_sync(0xFFFFFFFFu, lmin);
+  lmax = __reduce_max_sync(0xFFFFFFFFu, lmax);
+  if (lane == 0) { warp_sums_a[warp] = static_cast<int>(lmin); warp_sums_b[warp] = static_cast<int>(lmax); }
+  __syncthreads();
+  {
+    const int nwarps = nthreads >> 5;
+    uint32_t a = lane < nwarps ? static_cast<uint32_t>(warp_sums_a[lane]) : 0xFFFFFFFFu;
+    uint32_t b = lane < nwarps ? static_cast<uint32_t>(warp_sums_b[lane]) : 0u;
+    lmin = __reduce_min_sync(0xFFFFFFFFu, a);
+    lmax = __reduce_max_sync(0xFFFFFFFFu, b);
+  }
+  __syncthreads();   // warp_sums_* are reused by the scans below
+  const uint32_t diff = lmin ^ lmax;
+  int top_bits = diff == 0 ? 0 : 32 - __clz(diff);          // number of low bits that can differ
+  uint32_t prefix = top_bits >= 32 ? 0u : (lmax >> top_bits) << top_bits;   // the common high bits
+  uint32_t mask = top_bits >= 32 ? 0u : ~((1u << top_bits) - 1u);
+  uint32_t remaining = static_cast<uint32_t>(k);
+  int pass = 0;
+  for (int shift = top_bits; shift > 0; ++pass) {
+    const int nb = min(8, shift);
+    shift -= nb;
+    const uint32_t dmask = (1u << nb) - 1u;
     for (int i = lo; i < hi; ++i) {
       const uint32_t b = bits[i];
-      if ((b & mask) == prefix) atomicAdd(&hist[pass][(b >> shift) & 0xFF], 1);
+      if ((b & mask) == prefix) atomicAdd(&hist[pass][(b >> shift) & dmask], 1);
     }
     __syncthreads();
     if (warp == 0) {
@@ -145,7 +168,7 @@ __device__ __forceinline__ void topk_block(const float* __restrict__ score, int 
     __syncthreads();
     prefix |= s_digit[pass] << shift;
     remaining = s_remaining[pass];
-    mask |= 0xFFu << shift;
+    mask |= dmask << shift;
   }
   const uint32_t tau = prefix;                      // bit pattern of the k-th largest score
   const int take_eq = static_cast<int>(remaining);  // how many rows with score == tau are taken
@@ -231,13 +254,14 @@ __global__ void __launch_bounds__(kTopkThreads) sgd_score_topk_kernel(float* __r
 }
 
 // ---- W~[i][:] <- sat_rne_e4m3(W~[i][:] + DeltaBuffer[i][:] * A~) for the selected rows.
-// A CTA owns 32 selected rows x 128 columns.  It decodes the r x 128 tile of A~ to fp32 in shared
-// memory once (the FP8 decode is the expensive part, so it is shared by all 32 rows), then each thread
-// runs the fp32 fma chains of 4 rows x 8 columns.  The chain order (j ascending, seeded with the
+// A CTA owns 16 selected rows x 128 columns.  It decodes the r x 128 tile of A~ to fp32 in shared
+// memory once (the FP8 decode is the expensive part, so it is shared by all 16 rows), then each thread
+// runs the fp32 fma chains of 2 rows x 8 columns (small per-thread tiles: the chains are latency-bound, so
+// the kernel wants many threads rather than much work per thread).  The chain order (j ascending, seeded with the
 // decoded W~) is fixed, so the result is bit-identical to the sequential definition.
-constexpr int kMergeRowsPerThread = 4;
+constexpr int kMergeRowsPerThread = 2;
 constexpr int kMergeTy = 8;
-constexpr int kMergeRows = kMergeRowsPerThread * kMergeTy;          // 32 rows per CTA
+constexpr int kMergeRows = kMergeRowsPerThread * kMergeTy;          // 16 rows per CTA
 constexpr int kMergeTx = 16;
 constexpr int kMergeThreads = kMergeTx * kMergeTy;                  // 128
 constexpr int kMergeCols = 128;                                     // columns per CTA: thread tx owns 4tx..4tx+3 and 64+4tx..64+4tx+3
@@ -290,7 +314,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __re
     }
   }
   __syncthreads();   // srow visible
-  // the 32 DeltaBuffer rows, as float4 (r is a multiple of 8), four loads in flight per thread
+  // the DeltaBuffer rows of this CTA, as float4 (r is a multiple of 8), four loads in flight per thread
   const int r4 = r >> 2;
   const int d_vecs = kMergeRows * r4;
   for (int e0 = threadIdx.x; e0 < d_vecs; e0 += 4 * kMergeThreads) {
