@@ -254,14 +254,13 @@ __global__ void __launch_bounds__(kTopkThreads) sgd_score_topk_kernel(float* __r
 }
 
 // ---- W~[i][:] <- sat_rne_e4m3(W~[i][:] + DeltaBuffer[i][:] * A~) for the selected rows.
-// A CTA owns 16 selected rows x 128 columns.  It decodes the r x 128 tile of A~ to fp32 in shared
-// memory once (the FP8 decode is the expensive part, so it is shared by all 16 rows), then each thread
-// runs the fp32 fma chains of 2 rows x 8 columns (small per-thread tiles: the chains are latency-bound, so
-// the kernel wants many threads rather than much work per thread).  The chain order (j ascending, seeded with the
+// A CTA owns 32 selected rows x 128 columns.  It decodes the r x 128 tile of A~ to fp32 in shared
+// memory once (the FP8 decode is the expensive part, so it is shared by all 32 rows), then each thread
+// runs the fp32 fma chains of 4 rows x 8 columns (2 x 8 tiles with twice the threads measured slower).  The chain order (j ascending, seeded with the
 // decoded W~) is fixed, so the result is bit-identical to the sequential definition.
-constexpr int kMergeRowsPerThread = 2;
+constexpr int kMergeRowsPerThread = 4;
 constexpr int kMergeTy = 8;
-constexpr int kMergeRows = kMergeRowsPerThread * kMergeTy;          // 16 rows per CTA
+constexpr int kMergeRows = kMergeRowsPerThread * kMergeTy;          // 32 rows per CTA
 constexpr int kMergeTx = 16;
 constexpr int kMergeThreads = kMergeTx * kMergeTy;                  // 128
 constexpr int kMergeCols = 128;                                     // columns per CTA: thread tx owns 4tx..4tx+3 and 64+4tx..64+4tx+3
