@@ -192,17 +192,38 @@ int orc_quantize(const void* src, int src_dt, int64_t rows, int64_t cols, int fm
   return 0;
 }
 
+// Q_fp8 of dY in the per-row-scaled-backbone mode: column i of dY is first multiplied by 1 / s_w[i] (one fp32
+// reciprocal, one rounded fp32 multiply), then the tensor is quantized per tensor as in orc_quantize.
+int orc_quantize_colscaled(const void* src, int src_dt, int64_t rows, int64_t cols, int fmt, const float* col_div,
+                           uint8_t* dst, float* scale_out, float* amax_out) {
+  std::vector<float> inv((size_t)cols);
+  for (int64_t c = 0; c < cols; ++c) inv[c] = 1.0f / col_div[c];
+  float amax = 0.0f;
+  for (int64_t t = 0; t < rows; ++t)
+    for (int64_t c = 0; c < cols; ++c) amax = std::max(amax, std::fabs(load_elem(src, src_dt, t * cols + c) * inv[c]));
+  const float s = scale_from_amax(amax, fmt);
+  if (scale_out) *scale_out = s;
+  if (amax_out) *amax_out = amax;
+  for (int64_t t = 0; t < rows; ++t)
+    for (int64_t c = 0; c < cols; ++c) {
+      const float x = load_elem(src, src_dt, t * cols + c) * inv[c];
+      dst[t * cols + c] = fp8_encode(x * s, fmt);
+    }
+  return 0;
+}
+
 // Melded forward GEMM (Eq. o_split, Alg. 2): O_merged = W~' x~ / (s_W s_x).
 // Computes the outputs for tokens tsel[0..nt) x merged features fsel[0..nf)
 // (feature index i < m is O, i >= m is O_A); a null selection means "all".
 //   out[a*nf + b] = sum_c dec(xq[t_a][c]) * dec(wq[i_b][c]) / ((double)s_w * (double)s_x)
-int orc_forward_gemm(const uint8_t* xq, float s_x, const uint8_t* wq, float s_w,
+// Scales: per tensor, s_w[0] serves every row (the paper's scheme).  Per row (an extension for
+// heavy-tailed backbones): s_w[i] is the scale of row i < m and s_w[m] the one scale of the A~ block.
+int orc_forward_gemm(const uint8_t* xq, float s_x, const uint8_t* wq, const float* s_w, int gran,
                      int64_t T, int64_t m, int64_t n, int64_t r,
                      const int64_t* tsel, int64_t nt, const int64_t* fsel, int64_t nf, double* out) {
   const DecodeTable e4(FMT_E4M3);
   if (!tsel) nt = T;
   if (!fsel) nf = m + r;
-  const double d = (double)s_w * (double)s_x;
 #pragma omp parallel for collapse(2) schedule(static)
   for (int64_t a = 0; a < nt; ++a) {
     for (int64_t b = 0; b < nf; ++b) {
@@ -212,7 +233,8 @@ int orc_forward_gemm(const uint8_t* xq, float s_x, const uint8_t* wq, float s_w,
       const uint8_t* wr = wq + i * n;
       double acc = 0.0;
       for (int64_t c = 0; c < n; ++c) acc += e4.v[xr[c]] * e4.v[wr[c]];
-      out[a * nf + b] = acc / d;
+      const float sw = (gran == GRAN_ROW) ? s_w[i < m ? i : m] : s_w[0];
+      out[a * nf + b] = acc / ((double)sw * (double)s_x);
     }
   }
   return 0;
@@ -221,10 +243,10 @@ int orc_forward_gemm(const uint8_t* xq, float s_x, const uint8_t* wq, float s_w,
 // Full forward of one layer on already-quantized activations: splits O_merged
 // into Y[T][m] (double) and the saved O_A[T][r] (rounded once to fp32), and
 // reports amax(O_A) over the fp32 values.
-int orc_forward(const uint8_t* xq, float s_x, const uint8_t* wq, float s_w,
+int orc_forward(const uint8_t* xq, float s_x, const uint8_t* wq, const float* s_w, int gran,
                 int64_t T, int64_t m, int64_t n, int64_t r, double* Y, float* OA, float* amax_oa) {
   std::vector<double> merged((size_t)T * (size_t)(m + r));
-  orc_forward_gemm(xq, s_x, wq, s_w, T, m, n, r, nullptr, 0, nullptr, 0, merged.data());
+  orc_forward_gemm(xq, s_x, wq, s_w, gran, T, m, n, r, nullptr, 0, nullptr, 0, merged.data());
   float amax = 0.0f;
   for (int64_t t = 0; t < T; ++t) {
     for (int64_t i = 0; i < m; ++i) Y[t * m + i] = merged[t * (m + r) + i];
@@ -242,13 +264,15 @@ int orc_forward(const uint8_t* xq, float s_x, const uint8_t* wq, float s_w,
 // gradients; only the first m rows of W~' carry gradient to x):
 //   dX[t][c] = sum_{i<m} dec5(gq[t][i]) * dec4(wq[i][c]) / ((double)s_w * (double)s_g)
 // for tokens tsel x input channels csel (null = all).
-int orc_dx_gemm(const uint8_t* gq, float s_g, const uint8_t* wq, float s_w,
+// Per-row scales sit on the contraction axis here, so in that mode they were divided out of dY before its
+// E5M2 cast (see orc_quantize_colscaled) and only s_g remains: dX = sum_i dec5(gq) dec4(wq) / s_g.
+int orc_dx_gemm(const uint8_t* gq, float s_g, const uint8_t* wq, const float* s_w, int gran,
                 int64_t T, int64_t m, int64_t n,
                 const int64_t* tsel, int64_t nt, const int64_t* csel, int64_t nc, double* out) {
   const DecodeTable e4(FMT_E4M3), e5(FMT_E5M2);
   if (!tsel) nt = T;
   if (!csel) nc = n;
-  const double d = (double)s_w * (double)s_g;
+  const double d = (gran == GRAN_ROW) ? (double)s_g : (double)s_w[0] * (double)s_g;
 #pragma omp parallel for collapse(2) schedule(static)
   for (int64_t a = 0; a < nt; ++a) {
     for (int64_t b = 0; b < nc; ++b) {
@@ -264,8 +288,9 @@ int orc_dx_gemm(const uint8_t* gq, float s_g, const uint8_t* wq, float s_w,
 
 // Reformulated adapter gradient (Eq. lora_backward_modified, Alg. 3 line 3):
 //   dB[i][j] = sum_t dec5(gq[t][i]) * dec4(oaq[t][j]) / ((double)s_g * (double)s_oa)
-// for rows isel (null = all m rows), all r columns.
-int orc_db_gemm(const uint8_t* gq, float s_g, const uint8_t* oaq, float s_oa,
+// for rows isel (null = all m rows), all r columns.  row_scale (nullable): in the per-row mode gq carries
+// dY / s_w[i], so row i of the result is multiplied back by s_w[i].
+int orc_db_gemm(const uint8_t* gq, float s_g, const uint8_t* oaq, float s_oa, const float* row_scale,
                 int64_t T, int64_t m, int64_t r, const int64_t* isel, int64_t ni, double* out) {
   const DecodeTable e4(FMT_E4M3), e5(FMT_E5M2);
   if (!isel) ni = m;
@@ -276,7 +301,7 @@ int orc_db_gemm(const uint8_t* gq, float s_g, const uint8_t* oaq, float s_oa,
       const int64_t i = isel ? isel[a] : a;
       double acc = 0.0;
       for (int64_t t = 0; t < T; ++t) acc += e5.v[gq[t * m + i]] * e4.v[oaq[t * r + j]];
-      out[a * r + j] = acc / d;
+      out[a * r + j] = row_scale ? (acc / d) * (double)row_scale[i] : acc / d;
     }
   }
   return 0;
@@ -290,7 +315,10 @@ int orc_db_gemm(const uint8_t* gq, float s_g, const uint8_t* oaq, float s_oa,
 //      W~[i][c] = encode_e4m3(v)  -- the scale s_W cancels because A~ carries it (Eq. A_integ)
 //   5. the merged rows of dbuf are cleared (their change now lives in W~)
 // score_out (nullable) receives all m scores; idx_out (nullable) the k indices.
-int orc_proxy_update(uint8_t* wq, float* dbuf, const float* dB, float lr,
+// row_scales (nullable, m+1 entries): per-row mode.  The merge then works in row i's own scaled domain, where
+// A~ (scaled by s_w[m]) enters with the coefficient c_i = s_w[i] / s_w[m] (one fp32 division), applied to the
+// DeltaBuffer entry as its own rounded multiply before the chain.
+int orc_proxy_update(uint8_t* wq, float* dbuf, const float* dB, float lr, const float* row_scales,
                      int64_t m, int64_t n, int64_t r, int64_t k, int32_t* idx_out, float* score_out) {
   if (k < 0 || k > m) return -1;
   const DecodeTable e4(FMT_E4M3);
@@ -315,9 +343,13 @@ int orc_proxy_update(uint8_t* wq, float* dbuf, const float* dB, float lr,
 #pragma omp parallel for schedule(static)
   for (int64_t s = 0; s < k; ++s) {
     const int64_t i = sel[s];
+    const float coef = row_scales ? row_scales[i] / row_scales[m] : 1.0f;
     for (int64_t c = 0; c < n; ++c) {
       float v = (float)e4.v[wq[i * n + c]];
-      for (int64_t j = 0; j < r; ++j) v = std::fmaf(dbuf[i * r + j], (float)e4.v[aq[j * n + c]], v);
+      for (int64_t j = 0; j < r; ++j) {
+        const float d = row_scales ? dbuf[i * r + j] * coef : dbuf[i * r + j];
+        v = std::fmaf(d, (float)e4.v[aq[j * n + c]], v);
+      }
       wq[i * n + c] = fp8_encode(v, FMT_E4M3);
     }
   }

@@ -35,15 +35,17 @@ _lib.orc_f32_to_bf16.argtypes = [_f32]
 _lib.orc_quantize.restype = _i32
 _lib.orc_quantize.argtypes = [_p, _i32, _i64, _i64, _i32, _i32, _p, _f32, _p, _p, _p]
 _lib.orc_forward_gemm.restype = _i32
-_lib.orc_forward_gemm.argtypes = [_p, _f32, _p, _f32, _i64, _i64, _i64, _i64, _p, _i64, _p, _i64, _p]
+_lib.orc_forward_gemm.argtypes = [_p, _f32, _p, _p, _i32, _i64, _i64, _i64, _i64, _p, _i64, _p, _i64, _p]
 _lib.orc_forward.restype = _i32
-_lib.orc_forward.argtypes = [_p, _f32, _p, _f32, _i64, _i64, _i64, _i64, _p, _p, _p]
+_lib.orc_forward.argtypes = [_p, _f32, _p, _p, _i32, _i64, _i64, _i64, _i64, _p, _p, _p]
 _lib.orc_dx_gemm.restype = _i32
-_lib.orc_dx_gemm.argtypes = [_p, _f32, _p, _f32, _i64, _i64, _i64, _p, _i64, _p, _i64, _p]
+_lib.orc_dx_gemm.argtypes = [_p, _f32, _p, _p, _i32, _i64, _i64, _i64, _p, _i64, _p, _i64, _p]
 _lib.orc_db_gemm.restype = _i32
-_lib.orc_db_gemm.argtypes = [_p, _f32, _p, _f32, _i64, _i64, _i64, _p, _i64, _p]
+_lib.orc_db_gemm.argtypes = [_p, _f32, _p, _f32, _p, _i64, _i64, _i64, _p, _i64, _p]
 _lib.orc_proxy_update.restype = _i32
-_lib.orc_proxy_update.argtypes = [_p, _p, _p, _f32, _i64, _i64, _i64, _i64, _p, _p]
+_lib.orc_proxy_update.argtypes = [_p, _p, _p, _f32, _p, _i64, _i64, _i64, _i64, _p, _p]
+_lib.orc_quantize_colscaled.restype = _i32
+_lib.orc_quantize_colscaled.argtypes = [_p, _i32, _i64, _i64, _i32, _p, _p, _p, _p]
 _lib.orc_num_threads.restype = _i32
 
 
@@ -53,6 +55,12 @@ def _ptr(a):
 
 def _c(a, dtype):
     return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _sw(s_w):
+    """Scale argument -> (float32 array, granularity): a scalar is per tensor, an array of m+1 is per row."""
+    a = _c(np.atleast_1d(s_w), np.float32)
+    return a, (PER_ROW if a.size > 1 else PER_TENSOR)
 
 
 def _sel(s):
@@ -120,6 +128,20 @@ def quantize(src, fmt: int, gran: int = PER_TENSOR, scale_in=None, premul: float
     return dst, scale_out, amax_out
 
 
+def quantize_colscaled(src, fmt: int, col_div):
+    """Q_fp8 of a tensor whose column c is first multiplied by 1/col_div[c] (dY in the per-row mode)."""
+    a = _c(src, np.float32)
+    rows, cols = a.shape
+    div = _c(col_div, np.float32)
+    assert div.size >= cols
+    dst = np.empty((rows, cols), dtype=np.uint8)
+    scale_out = np.empty(1, dtype=np.float32)
+    amax_out = np.empty(1, dtype=np.float32)
+    rc = _lib.orc_quantize_colscaled(_ptr(a), F32, rows, cols, fmt, _ptr(div), _ptr(dst), _ptr(scale_out), _ptr(amax_out))
+    assert rc == 0
+    return dst, np.float32(scale_out[0]), np.float32(amax_out[0])
+
+
 def forward_gemm(xq, s_x, wq, s_w, m: int, r: int, tsel=None, fsel=None) -> np.ndarray:
     """Sampled O_merged: tokens tsel x merged features fsel (None = all), float64."""
     xq, wq = _c(xq, np.uint8), _c(wq, np.uint8)
@@ -128,7 +150,9 @@ def forward_gemm(xq, s_x, wq, s_w, m: int, r: int, tsel=None, fsel=None) -> np.n
     ts, nt = _sel(tsel)
     fs, nf = _sel(fsel)
     out = np.empty((nt if ts is not None else T, nf if fs is not None else m + r), dtype=np.float64)
-    rc = _lib.orc_forward_gemm(_ptr(xq), float(s_x), _ptr(wq), float(s_w), T, m, n, r,
+    sw, gran = _sw(s_w)
+    assert gran == PER_TENSOR or sw.size == m + 1
+    rc = _lib.orc_forward_gemm(_ptr(xq), float(s_x), _ptr(wq), _ptr(sw), gran, T, m, n, r,
                                _ptr(ts), nt, _ptr(fs), nf, _ptr(out))
     assert rc == 0
     return out
@@ -142,7 +166,9 @@ def forward(xq, s_x, wq, s_w, m: int, r: int):
     Y = np.empty((T, m), dtype=np.float64)
     OA = np.empty((T, r), dtype=np.float32)
     amax = np.zeros(1, dtype=np.float32)
-    rc = _lib.orc_forward(_ptr(xq), float(s_x), _ptr(wq), float(s_w), T, m, n, r, _ptr(Y), _ptr(OA), _ptr(amax))
+    sw, gran = _sw(s_w)
+    assert gran == PER_TENSOR or sw.size == m + 1
+    rc = _lib.orc_forward(_ptr(xq), float(s_x), _ptr(wq), _ptr(sw), gran, T, m, n, r, _ptr(Y), _ptr(OA), _ptr(amax))
     assert rc == 0
     return Y, OA, np.float32(amax[0])
 
@@ -155,24 +181,26 @@ def dx_gemm(gq, s_g, wq, s_w, m: int, tsel=None, csel=None) -> np.ndarray:
     ts, nt = _sel(tsel)
     cs, nc = _sel(csel)
     out = np.empty((nt if ts is not None else T, nc if cs is not None else n), dtype=np.float64)
-    rc = _lib.orc_dx_gemm(_ptr(gq), float(s_g), _ptr(wq), float(s_w), T, m, n, _ptr(ts), nt, _ptr(cs), nc, _ptr(out))
+    sw, gran = _sw(s_w)
+    rc = _lib.orc_dx_gemm(_ptr(gq), float(s_g), _ptr(wq), _ptr(sw), gran, T, m, n, _ptr(ts), nt, _ptr(cs), nc, _ptr(out))
     assert rc == 0
     return out
 
 
-def db_gemm(gq, s_g, oaq, s_oa, isel=None) -> np.ndarray:
+def db_gemm(gq, s_g, oaq, s_oa, isel=None, row_scale=None) -> np.ndarray:
     gq, oaq = _c(gq, np.uint8), _c(oaq, np.uint8)
     T, m = gq.shape
     r = oaq.shape[1]
     assert oaq.shape[0] == T
     is_, ni = _sel(isel)
     out = np.empty((ni if is_ is not None else m, r), dtype=np.float64)
-    rc = _lib.orc_db_gemm(_ptr(gq), float(s_g), _ptr(oaq), float(s_oa), T, m, r, _ptr(is_), ni, _ptr(out))
+    rs = None if row_scale is None else _c(row_scale, np.float32)
+    rc = _lib.orc_db_gemm(_ptr(gq), float(s_g), _ptr(oaq), float(s_oa), _ptr(rs), T, m, r, _ptr(is_), ni, _ptr(out))
     assert rc == 0
     return out
 
 
-def proxy_update(wq, dbuf, dB, lr: float, k: int, m: int, r: int):
+def proxy_update(wq, dbuf, dB, lr: float, k: int, m: int, r: int, row_scales=None):
     """In place on wq (uint8 [(m+r), n]) and dbuf (float32 [m, r]).  Returns (idx int32 [k], score float32 [m])."""
     assert wq.dtype == np.uint8 and wq.flags.c_contiguous and wq.shape[0] == m + r
     assert dbuf.dtype == np.float32 and dbuf.flags.c_contiguous and dbuf.shape == (m, r)
@@ -180,7 +208,10 @@ def proxy_update(wq, dbuf, dB, lr: float, k: int, m: int, r: int):
     g = None if dB is None else _c(dB, np.float32)
     idx = np.empty(max(k, 0), dtype=np.int32)
     score = np.empty(m, dtype=np.float32)
-    rc = _lib.orc_proxy_update(_ptr(wq), _ptr(dbuf), _ptr(g), float(np.float32(lr)), m, n, r, k, _ptr(idx), _ptr(score))
+    rs = None if row_scales is None else _c(row_scales, np.float32)
+    assert rs is None or rs.size == m + 1
+    rc = _lib.orc_proxy_update(_ptr(wq), _ptr(dbuf), _ptr(g), float(np.float32(lr)), _ptr(rs), m, n, r, k, _ptr(idx),
+                               _ptr(score))
     if rc != 0:
         raise ValueError("orc_proxy_update rejected its arguments")
     return idx, score
@@ -188,21 +219,28 @@ def proxy_update(wq, dbuf, dB, lr: float, k: int, m: int, r: int):
 
 # ---- whole-layer compositions in the paper's order (each step is one oracle call) ----
 
-def setup_layer(W, A, B, gamma: float):
+def setup_layer(W, A, B, gamma: float, per_row: bool = False):
     """Alg. 1 without the SVD (A and B are given): W~, s_W = Q(W); A~ = Q(gamma*A; s_W);
     W~' = [W~; A~]; the initial B is melded by the merge operator itself over all rows
-    (W + BA = W~ + B A~ in the scaled domain), leaving DeltaBuffer = 0."""
+    (W + BA = W~ + B A~ in the scaled domain), leaving DeltaBuffer = 0.
+    per_row: every row of W gets its own absmax scale and the A~ block one absmax scale of its own;
+    s_w is then an array of m + 1 scales."""
     W = _c(W, np.float32)
     A = _c(A, np.float32)
     m, n = W.shape
     r = A.shape[0]
-    wq_w, s_w, _ = quantize(W, E4M3)
-    aq, _, _ = quantize(A, E4M3, scale_in=s_w, premul=gamma)
+    if per_row:
+        wq_w, s_rows, _ = quantize(W, E4M3, gran=PER_ROW)
+        aq, s_a, _ = quantize(A, E4M3, premul=gamma)
+        s_w = np.concatenate([s_rows, [s_a]]).astype(np.float32)
+    else:
+        wq_w, s_w, _ = quantize(W, E4M3)
+        aq, _, _ = quantize(A, E4M3, scale_in=s_w, premul=gamma)
     wq = np.ascontiguousarray(np.concatenate([wq_w, aq], axis=0))
     dbuf = np.zeros((m, r), dtype=np.float32)
     if B is not None:
         dbuf[:] = _c(B, np.float32)
-        proxy_update(wq, dbuf, None, 0.0, m, m, r)
+        proxy_update(wq, dbuf, None, 0.0, m, m, r, row_scales=s_w if per_row else None)
     return wq, s_w, dbuf
 
 
@@ -215,8 +253,12 @@ def layer_forward(X, wq, s_w, m: int, r: int):
 
 def layer_backward(dY, OA, wq, s_w, m: int, r: int):
     """Alg. 3 line 3 plus the implied input gradient.  Returns dict(gq, s_g, oaq, s_oa, dX, dB)."""
-    gq, s_g, _ = quantize(dY, E5M2)
+    per_row = np.atleast_1d(s_w).size > 1
+    if per_row:
+        gq, s_g, _ = quantize_colscaled(dY, E5M2, np.asarray(s_w)[:m])
+    else:
+        gq, s_g, _ = quantize(dY, E5M2)
     oaq, s_oa, _ = quantize(OA, E4M3)
     dX = dx_gemm(gq, s_g, wq, s_w, m)
-    dB = db_gemm(gq, s_g, oaq, s_oa)
+    dB = db_gemm(gq, s_g, oaq, s_oa, row_scale=np.asarray(s_w)[:m] if per_row else None)
     return dict(gq=gq, s_g=s_g, oaq=oaq, s_oa=s_oa, dX=dX, dB=dB)
