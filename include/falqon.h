@@ -60,8 +60,16 @@ typedef struct {
   int64_t n;      /* input features (columns of W)                                       */
   int64_t r;      /* LoRA rank                                                           */
   uint8_t *wq;    /* device [(m + r)][n] E4M3 codes; rows m..m+r-1 hold A~ = Q(A; s_W)   */
-  float *s_w;     /* device [1]: the per-tensor scale of W~, shared by A~                */
+  float *s_w;     /* device [1]: the per-tensor scale of W~, shared by A~ (FALQON_PER_TENSOR, the
+                     paper's scheme); or device [m + 1] (FALQON_PER_ROW): s_w[i] = absmax scale of
+                     row i of W~, s_w[m] = the one absmax scale of the A~ block                 */
   float *dbuf;    /* device [m][r] fp32 DeltaBuffer                                      */
+  int32_t gran;   /* falqon_gran of s_w.  PER_ROW is an extension for heavy-tailed backbones:
+                     the forward rescales per output column; backward divides column i of dY by
+                     s_w[i] before its E5M2 cast (the row scales lie on dX's contraction axis) and
+                     multiplies row i of dB back; the merge weighs DeltaBuffer row i by
+                     s_w[i] / s_w[m].  Scales stay frozen after set-up in both modes.          */
+  int32_t reserved_;
 } falqon_layer;
 
 /* Names of the regions inside the workspace that hold staged intermediates of the last call

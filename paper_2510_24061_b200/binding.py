@@ -34,7 +34,8 @@ lib = C.CDLL(LIB_PATH)
 
 class falqon_layer(C.Structure):
     _fields_ = [("m", C.c_int64), ("n", C.c_int64), ("r", C.c_int64),
-                ("wq", C.c_void_p), ("s_w", C.c_void_p), ("dbuf", C.c_void_p)]
+                ("wq", C.c_void_p), ("s_w", C.c_void_p), ("dbuf", C.c_void_p),
+                ("gran", C.c_int32), ("reserved_", C.c_int32)]
 
 
 _i64, _sz, _p, _f, _i = C.c_int64, C.c_size_t, C.c_void_p, C.c_float, C.c_int
@@ -98,7 +99,9 @@ class Layer:
         assert wq.dtype == torch.uint8 and wq.is_contiguous() and dbuf.dtype == torch.float32 and dbuf.is_contiguous()
         self.wq, self.s_w, self.dbuf = wq, s_w, dbuf
         self.m, self.n, self.r = wq.shape[0] - r, wq.shape[1], r
-        self.c = falqon_layer(self.m, self.n, self.r, wq.data_ptr(), s_w.data_ptr(), dbuf.data_ptr())
+        assert s_w.numel() in (1, self.m + 1) and s_w.dtype == torch.float32 and s_w.is_contiguous()
+        self.gran = PER_ROW if s_w.numel() == self.m + 1 else PER_TENSOR
+        self.c = falqon_layer(self.m, self.n, self.r, wq.data_ptr(), s_w.data_ptr(), dbuf.data_ptr(), self.gran, 0)
         self._ws = None
 
     def workspace(self, T: int) -> torch.Tensor:
@@ -224,16 +227,22 @@ def proxy_update(layer: Layer, dB: torch.Tensor | None, lr: float, k: int, ws: t
     return idx_out
 
 
-def setup_layer(W: torch.Tensor, A: torch.Tensor, B: torch.Tensor | None, gamma: float) -> Layer:
+def setup_layer(W: torch.Tensor, A: torch.Tensor, B: torch.Tensor | None, gamma: float, per_row: bool = False) -> Layer:
     """Builds a melded layer from W [m, n], A [r, n] and an optional initial B [m, r] (all on the device):
     W~, s_W = Q(W); A~ = Q(gamma*A; s_W); W~' = [W~; A~]; then melds B by the merge operator over all rows
-    (dbuf := B, falqon_proxy_update with dB = NULL, k = m), which leaves DeltaBuffer = 0."""
+    (dbuf := B, falqon_proxy_update with dB = NULL, k = m), which leaves DeltaBuffer = 0.
+    per_row: each row of W gets its own absmax scale and the A~ block one absmax scale of its own."""
     m, n = W.shape
     r = A.shape[0]
     dev = W.device
     wq = torch.empty((m + r, n), dtype=torch.uint8, device=dev)
-    _, s_w, _ = quantize(W.contiguous(), E4M3, dst=wq[:m])
-    quantize(A.contiguous(), E4M3, scale_in=s_w, premul=gamma, want_amax=False, dst=wq[m:])
+    if per_row:
+        _, s_rows, _ = quantize(W.contiguous(), E4M3, gran=PER_ROW, dst=wq[:m])
+        _, s_a, _ = quantize(A.contiguous(), E4M3, premul=gamma, dst=wq[m:])
+        s_w = torch.cat([s_rows, s_a]).contiguous()
+    else:
+        _, s_w, _ = quantize(W.contiguous(), E4M3, dst=wq[:m])
+        quantize(A.contiguous(), E4M3, scale_in=s_w, premul=gamma, want_amax=False, dst=wq[m:])
     dbuf = torch.zeros((m, r), dtype=torch.float32, device=dev)
     layer = Layer(wq, s_w, dbuf, r)
     if B is not None:

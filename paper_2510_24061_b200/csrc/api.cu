@@ -24,8 +24,9 @@ int* status_ptr() {
 }
 
 struct WorkspaceLayout {
-  size_t scales, act8, oaq_t, db_part, score, sel_idx, total;
-  size_t act8_bytes, oaq_t_bytes, db_part_bytes, score_bytes, sel_idx_bytes;
+  size_t scales, act8, oaq_t, db_part, score, sel_idx, inv_sw, col_scale, total;
+  size_t act8_bytes, oaq_t_bytes, db_part_bytes, score_bytes, sel_idx_bytes, inv_sw_bytes, col_scale_bytes;
+  int64_t inv_sw_len, col_scale_len;   // table lengths, padded to a multiple of 32 (+32) so vector reads stay inside
   int64_t r16, t16;
   int splits;
 };
@@ -54,10 +55,16 @@ bool make_layout(int64_t m, int64_t n, int64_t r, int64_t T, WorkspaceLayout* w)
   w->db_part_bytes = static_cast<size_t>(w->splits) * m * r * sizeof(float);
   w->score_bytes = static_cast<size_t>(m) * sizeof(float);
   w->sel_idx_bytes = static_cast<size_t>(m) * sizeof(int32_t);
+  w->inv_sw_len = round_up(m, 32) + 32;
+  w->col_scale_len = round_up(m + r, 32) + 32;
+  w->inv_sw_bytes = static_cast<size_t>(w->inv_sw_len) * sizeof(float);
+  w->col_scale_bytes = static_cast<size_t>(w->col_scale_len) * sizeof(float);
   size_t off = 0;
   w->scales = off; off += kHeaderBytes;
   w->score = off; off += round_up(w->score_bytes, 1024);      // token-independent regions first, so the
   w->sel_idx = off; off += round_up(w->sel_idx_bytes, 1024);  // proxy update finds them for any T_max
+  w->inv_sw = off; off += round_up(w->inv_sw_bytes, 1024);        // per-row mode: 1/s_w[i]
+  w->col_scale = off; off += round_up(w->col_scale_bytes, 1024);  // per-row mode: 1/(s_w[c] s_x)
   w->act8 = off; off += round_up(w->act8_bytes, 1024);
   w->oaq_t = off; off += round_up(w->oaq_t_bytes, 1024);
   w->db_part = off; off += round_up(w->db_part_bytes, 1024);
@@ -70,7 +77,7 @@ inline bool dtype_ok(int dt) { return dt == FALQON_BF16 || dt == FALQON_F32; }
 
 bool layer_ok(const falqon_layer* L) {
   return L != nullptr && shape_ok(L->m, L->n, L->r) && L->wq != nullptr && L->s_w != nullptr && L->dbuf != nullptr &&
-         aligned16(L->wq) && aligned16(L->dbuf);
+         aligned16(L->wq) && aligned16(L->dbuf) && (L->gran == FALQON_PER_TENSOR || L->gran == FALQON_PER_ROW);
 }
 
 #define FALQON_CUDA(expr)                                   \
@@ -196,8 +203,12 @@ int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_d
   {
     StageTimer timer(FALQON_STAGE_QUANT_X, stream);
     FALQON_CUDA(launch_quantize_fused(X, x_dt, T * n, kE4M3, xq, partial, base + w.scales + kSyncOffset, scales + 1, s_x_out,
-                                      scales + 0, amax_oa, status, stream));
+                                      scales + 0, amax_oa, status, nullptr, 0, stream));
   }
+  const bool per_row = L->gran == FALQON_PER_ROW;
+  float* col_scale = reinterpret_cast<float*>(base + w.col_scale);
+  if (per_row)   // epilogue factors 1 / (s_w[column] * s_x); s_w[m] serves the O_A columns
+    FALQON_CUDA(launch_scale_table(1, L->s_w, m, r, scales + 1, col_scale, w.col_scale_len, stream));
   // S2: [Y | O_A] = x~ W~'^T / (s_W s_x), amax(O_A) from the epilogue
   GemmProblem g{};
   g.M = T; g.N = m + r; g.K = n;
@@ -206,7 +217,8 @@ int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_d
   g.block_n = 256; g.k_splits = 1;
   g.c0 = Y; g.ldc0 = m; g.c0_dt = y_dt; g.n_split = m; g.c0_split_stride = 0;
   g.c1 = OA; g.ldc1 = r; g.amax1_bits = reinterpret_cast<uint32_t*>(amax_oa);
-  g.scale_a = scales + 1; g.scale_b = L->s_w;
+  g.scale_a = per_row ? nullptr : scales + 1; g.scale_b = per_row ? nullptr : L->s_w;
+  g.col_scale = per_row ? col_scale : nullptr;
   g.status = status;
   {
     StageTimer timer(FALQON_STAGE_GEMM_FWD, stream);
@@ -235,10 +247,14 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
 
   // S3: g~, s_g = Q_e5m2(dY)
   uint32_t* partial = reinterpret_cast<uint32_t*>(base + w.scales + kPartialsOffset);
+  const bool per_row = L->gran == FALQON_PER_ROW;
+  float* inv_sw = reinterpret_cast<float*>(base + w.inv_sw);
+  if (per_row)   // the row scales lie on dX's contraction axis: divide them out of dY before its cast
+    FALQON_CUDA(launch_scale_table(0, L->s_w, m, r, nullptr, inv_sw, w.inv_sw_len, stream));
   {
     StageTimer timer(FALQON_STAGE_QUANT_DY, stream);
     FALQON_CUDA(launch_quantize_fused(dY, dy_dt, T * m, kE5M2, gq, partial, base + w.scales + kSyncOffset, scales + 3, s_g_out,
-                                      scales + 2, nullptr, status, stream));
+                                      scales + 2, nullptr, status, per_row ? inv_sw : nullptr, static_cast<int>(m), stream));
   }
   // S5a: O~_A, s_OA = Q_e4m3(O_A), written transposed for the dB product
   {
@@ -254,7 +270,8 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
     g.block_n = 256; g.k_splits = 1;
     g.c0 = dX; g.ldc0 = n; g.c0_dt = dx_dt; g.n_split = n; g.c0_split_stride = 0;
     g.c1 = nullptr; g.ldc1 = 0; g.amax1_bits = nullptr;
-    g.scale_a = scales + 3; g.scale_b = L->s_w;
+    g.scale_a = scales + 3; g.scale_b = per_row ? nullptr : L->s_w;
+    g.col_scale = nullptr;
     g.status = status;
     StageTimer timer(FALQON_STAGE_GEMM_DX, stream);
     FALQON_CUDA(launch_gemm_fp8(g, stream));
@@ -268,14 +285,14 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
     g.block_n = static_cast<int>(w.r16); g.k_splits = w.splits;
     g.c0 = part; g.ldc0 = r; g.c0_dt = kF32; g.n_split = r; g.c0_split_stride = m * r;
     g.c1 = nullptr; g.ldc1 = 0; g.amax1_bits = nullptr;
-    g.scale_a = nullptr; g.scale_b = nullptr;
+    g.scale_a = nullptr; g.scale_b = nullptr; g.col_scale = nullptr;
     g.status = status;
     {
       StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
       FALQON_CUDA(launch_gemm_fp8(g, stream));
     }
     StageTimer timer(FALQON_STAGE_REDUCE_DB, stream);
-    FALQON_CUDA(launch_reduce_db(part, w.splits, m * r, scales + 3, scales + 5, dB, stream));
+    FALQON_CUDA(launch_reduce_db(part, w.splits, m * r, scales + 3, scales + 5, per_row ? L->s_w : nullptr, r, dB, stream));
   }
   return FALQON_OK;
 }
@@ -300,8 +317,15 @@ int falqon_proxy_update(const falqon_layer* L, const float* dB, float lr, int64_
   }
   if (k > 0) {
     StageTimer timer(FALQON_STAGE_MERGE, stream);
-    if (fused_merge) FALQON_CUDA(launch_merge_rows_fused(L->wq, L->dbuf, sel, k, m, n, r, group_counters, stream));
-    else FALQON_CUDA(launch_merge_rows(L->wq, L->dbuf, sel, k, m, n, r, stream));
+    const float* row_scales = L->gran == FALQON_PER_ROW ? L->s_w : nullptr;
+    if (fused_merge) {
+      FALQON_CUDA(launch_merge_rows_fused(L->wq, L->dbuf, sel, k, m, n, r, group_counters, row_scales, stream));
+    } else if (row_scales == nullptr) {
+      FALQON_CUDA(launch_merge_rows(L->wq, L->dbuf, sel, k, m, n, r, stream));
+    } else {   // more row groups than counters: merge without the fused clearing, then clear
+      FALQON_CUDA(launch_merge_rows_fused(L->wq, L->dbuf, sel, k, m, n, r, nullptr, row_scales, stream));
+      FALQON_CUDA(launch_zero_rows(L->dbuf, sel, k, r, stream));
+    }
   }
   return FALQON_OK;
 }

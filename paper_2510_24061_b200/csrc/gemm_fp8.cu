@@ -48,6 +48,7 @@ struct GemmParams {
   void* c0; long long ldc0; int c0_dt; int n_split; long long c0_split_stride;
   float* c1; long long ldc1; uint32_t* amax1_bits;
   const float* scale_a; const float* scale_b;
+  const float* col_scale;
   int* status;
 };
 
@@ -146,8 +147,18 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ro
   auto drain = [&](const uint32_t (&v)[32], int c) {
     const int col0 = n0 + c;
     float f[32];
+    if (p.col_scale != nullptr) {   // per-column factors (table padded to a multiple of 32 beyond N)
+      const float4* cs = reinterpret_cast<const float4*>(p.col_scale + col0);
 #pragma unroll
-    for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * inv;
+      for (int i = 0; i < 8; ++i) {
+        const float4 s4 = __ldg(cs + i);
+        f[4 * i] = __uint_as_float(v[4 * i]) * s4.x; f[4 * i + 1] = __uint_as_float(v[4 * i + 1]) * s4.y;
+        f[4 * i + 2] = __uint_as_float(v[4 * i + 2]) * s4.z; f[4 * i + 3] = __uint_as_float(v[4 * i + 3]) * s4.w;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * inv;
+    }
     const bool fast = col0 + 32 <= p.n_split && ((p.ldc0 * esize) & 15) == 0 &&
                       ((reinterpret_cast<uintptr_t>(p.c0) + (long long)split * p.c0_split_stride * esize) & 15) == 0;
     if (fast) {   // warp-uniform
@@ -327,7 +338,7 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     const int col_half = (warp - 2) >> 2;   // warps 2..5 drain the left half of the tile, 6..9 the right half
     uint8_t* stage_out = smem_gen + static_cast<uint32_t>(S) * stage_bytes + kBarrierBytes + (warp - 2) * kStageOutBytes;
     const bool rescale = p.scale_a != nullptr;
-    const float inv = rescale ? 1.0f / (__ldg(p.scale_a) * __ldg(p.scale_b)) : 1.0f;
+    const float inv = rescale ? 1.0f / (p.scale_b != nullptr ? __ldg(p.scale_a) * __ldg(p.scale_b) : __ldg(p.scale_a)) : 1.0f;
     int acc = 0;
     uint32_t acc_phase = 0;
     uint32_t amax_bits = 0;
@@ -527,7 +538,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     const int col_half = (warp - 2) >> 2;
     uint8_t* stage_out = smem_gen + static_cast<uint32_t>(S) * kPairStageBytes + kBarrierBytes + (warp - 2) * kStageOutBytes;
     const bool rescale = p.scale_a != nullptr;
-    const float inv = rescale ? 1.0f / (__ldg(p.scale_a) * __ldg(p.scale_b)) : 1.0f;
+    const float inv = rescale ? 1.0f / (p.scale_b != nullptr ? __ldg(p.scale_a) * __ldg(p.scale_b) : __ldg(p.scale_a)) : 1.0f;
     int acc = 0;
     uint32_t acc_phase = 0;
     uint32_t amax_bits = 0;
@@ -666,7 +677,7 @@ cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
   gp.c0 = q.c0; gp.ldc0 = q.ldc0; gp.c0_dt = q.c0_dt; gp.n_split = static_cast<int>(q.n_split);
   gp.c0_split_stride = 0;
   gp.c1 = q.c1; gp.ldc1 = q.ldc1; gp.amax1_bits = q.amax1_bits;
-  gp.scale_a = q.scale_a; gp.scale_b = q.scale_b;
+  gp.scale_a = q.scale_a; gp.scale_b = q.scale_b; gp.col_scale = q.col_scale;
   gp.status = q.status;
   CUtensorMap ta, tb;
   if (!make_tensor_map(&ta, q.a, q.M, q.K, q.lda, kBlockKBytes, kBlockM)) return cudaErrorInvalidValue;
@@ -723,7 +734,7 @@ cudaError_t launch_gemm_fp8(const GemmProblem& q, cudaStream_t stream) {
   gp.c0 = q.c0; gp.ldc0 = q.ldc0; gp.c0_dt = q.c0_dt; gp.n_split = static_cast<int>(q.n_split);
   gp.c0_split_stride = q.c0_split_stride;
   gp.c1 = q.c1; gp.ldc1 = q.ldc1; gp.amax1_bits = q.amax1_bits;
-  gp.scale_a = q.scale_a; gp.scale_b = q.scale_b;
+  gp.scale_a = q.scale_a; gp.scale_b = q.scale_b; gp.col_scale = q.col_scale;
   gp.status = q.status;
 
   CUtensorMap ta, tb;

@@ -53,9 +53,14 @@ cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, i
                                    cudaStream_t stream);
 // Per-tensor absmax scaling in one kernel (absmax, grid barrier, cast).  `sync` points at 8 bytes of workspace that
 // are zero before the call and are left zero by it; `partial` holds up to kMaxAbsmaxParts words.
+// col_mul (nullable): column c of the [count / cols][cols] tensor is multiplied by col_mul[c] before everything else.
 cudaError_t launch_quantize_fused(const void* src, int src_dt, int64_t count, int fmt, uint8_t* dst, uint32_t* partial,
                                   void* sync, float* scale_out, float* scale_out2, float* amax_out, float* clear_word,
-                                  int* status, cudaStream_t stream);
+                                  int* status, const float* col_mul, int cols, cudaStream_t stream);
+// Tables for a per-row-scaled backbone (s_w has m + 1 entries): mode 0 -> out[i] = 1/s_w[i]; mode 1 ->
+// out[c] = 1/(s_w[min(c,m)] * *s_x) for c < m + r.  Entries up to `padded` are written (zero beyond the table).
+cudaError_t launch_scale_table(int mode, const float* s_w, int64_t m, int64_t r, const float* s_x, float* out, int64_t padded,
+                               cudaStream_t stream);
 cudaError_t launch_quantize_per_row(const void* src, int src_dt, int64_t rows, int64_t cols, int fmt, float premul,
                                     const float* scale_in, uint8_t* dst, float* scale_out, float* amax_out,
                                     cudaStream_t stream);
@@ -75,15 +80,17 @@ struct GemmProblem {
   // epilogue: columns [0, n_split) -> c0 (bf16 or fp32), columns [n_split, N) -> c1 (fp32) with |max| -> amax1
   void* c0; int64_t ldc0; int c0_dt; int64_t n_split; int64_t c0_split_stride;
   float* c1; int64_t ldc1; uint32_t* amax1_bits;
-  const float* scale_a; const float* scale_b;  // device scalars; output *= 1/(sa*sb); null = no rescale
+  const float* scale_a; const float* scale_b;  // device scalars; output *= 1/(sa*sb); scale_b null: 1/sa; both null: none
+  const float* col_scale;                      // nullable: per-column factors (N rounded up to 32 entries) instead
   int* status;
 };
 cudaError_t launch_gemm_fp8(const GemmProblem& p, cudaStream_t stream);
 int gemm_k_splits_for_db(int64_t m, int64_t T);
 
 // ---- proxy_update.cu
+// row_mul (nullable, one factor per row of r entries): dB[i][:] is also multiplied by row_mul[i].
 cudaError_t launch_reduce_db(const float* partials, int splits, int64_t count, const float* s_g, const float* s_oa,
-                             float* dB, cudaStream_t stream);
+                             const float* row_mul, int64_t r, float* dB, cudaStream_t stream);
 cudaError_t launch_sgd_score(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, float* score,
                              cudaStream_t stream);
 // The k selected rows (ascending) are written to sel_idx and, when idx_copy is non-null, to idx_copy (int32 [k]).
@@ -95,9 +102,11 @@ cudaError_t launch_merge_rows(uint8_t* wq, float* dbuf, const int32_t* sel_idx, 
 // one word, zero between calls), and the merge that also clears the merged DeltaBuffer rows (group_counters:
 // merge_group_count(k) words, zero between calls).
 int merge_group_count(int64_t k);
+cudaError_t launch_zero_rows(float* dbuf, const int32_t* sel_idx, int64_t k, int64_t r, cudaStream_t stream);
 cudaError_t launch_sgd_score_topk(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, int64_t k, float* score,
                                   int32_t* sel_idx, int32_t* idx_copy, unsigned int* done_counter, cudaStream_t stream);
+// row_scales (nullable, m + 1 entries): per-row mode, DeltaBuffer row i enters the chain times s_w[i] / s_w[m].
 cudaError_t launch_merge_rows_fused(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
-                                    int64_t r, unsigned int* group_counters, cudaStream_t stream);
+                                    int64_t r, unsigned int* group_counters, const float* row_scales, cudaStream_t stream);
 
 }  // namespace falqon

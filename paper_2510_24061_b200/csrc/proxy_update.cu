@@ -11,7 +11,7 @@ namespace {
 // ---- dB = (sum over splits, in split order) / (s_g * s_OA)
 __global__ void __launch_bounds__(256) reduce_db_kernel(const float* __restrict__ partials, int splits, int64_t count,
                                                         const float* __restrict__ s_g, const float* __restrict__ s_oa,
-                                                        float* __restrict__ dB) {
+                                                        const float* __restrict__ row_mul, int r, float* __restrict__ dB) {
   pdl_trigger();
   pdl_wait();
   const float inv = 1.0f / (__ldg(s_g) * __ldg(s_oa));
@@ -23,6 +23,10 @@ __global__ void __launch_bounds__(256) reduce_db_kernel(const float* __restrict_
       acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
     }
     acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+    if (row_mul != nullptr) {   // per-row-scaled backbone: give row i its scale back (r is a multiple of 4)
+      const float f = __ldg(row_mul + (v * 4) / r);
+      acc.x *= f; acc.y *= f; acc.z *= f; acc.w *= f;
+    }
     reinterpret_cast<float4*>(dB)[v] = acc;
   }
 }
@@ -272,7 +276,8 @@ __device__ __forceinline__ void decode4(uint32_t w, float (&a)[4]) {
 
 __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __restrict__ wq, float* dbuf,
                                                                    const int32_t* __restrict__ sel_idx, int k, int64_t m,
-                                                                   int64_t n, int r, unsigned int* group_counters) {
+                                                                   int64_t n, int r, unsigned int* group_counters,
+                                                                   const float* __restrict__ row_scales) {
   extern __shared__ __align__(16) float merge_smem[];
   float* a_tile = merge_smem;                         // [r][kMergeCols] decoded A~
   float* sdb = merge_smem + (size_t)r * kMergeCols;   // [kMergeRows][r]
@@ -323,7 +328,14 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __re
       const int e = e0 + u * kMergeThreads;
       const int q = e / r4, j4 = e - q * r4;
       d[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (e < d_vecs && q < nrows) d[u] = *reinterpret_cast<const float4*>(dbuf + (int64_t)srow[q] * r + 4 * j4);
+      if (e < d_vecs && q < nrows) {
+        d[u] = *reinterpret_cast<const float4*>(dbuf + (int64_t)srow[q] * r + 4 * j4);
+        if (row_scales != nullptr) {   // per-row mode: c_i = s_w[i] / s_w[m], applied as its own rounded multiply
+          const float c = __fdiv_rn(__ldg(row_scales + srow[q]), __ldg(row_scales + m));
+          d[u].x = __fmul_rn(d[u].x, c); d[u].y = __fmul_rn(d[u].y, c);
+          d[u].z = __fmul_rn(d[u].z, c); d[u].w = __fmul_rn(d[u].w, c);
+        }
+      }
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
@@ -403,12 +415,12 @@ __global__ void __launch_bounds__(256) zero_rows_kernel(float* __restrict__ dbuf
 }  // namespace
 
 cudaError_t launch_reduce_db(const float* partials, int splits, int64_t count, const float* s_g, const float* s_oa,
-                             float* dB, cudaStream_t stream) {
+                             const float* row_mul, int64_t r, float* dB, cudaStream_t stream) {
   int64_t blocks = (count / 4 + 255) / 256;
   if (blocks > 148 * 8) blocks = 148 * 8;
   if (blocks < 1) blocks = 1;
   return launch_pdl(reduce_db_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream, 1, partials, splits, count,
-                    s_g, s_oa, dB);
+                    s_g, s_oa, row_mul, static_cast<int>(r), dB);
 }
 
 cudaError_t launch_sgd_score(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, float* score,
@@ -436,7 +448,7 @@ cudaError_t launch_topk(const float* score, int64_t m, int64_t k, int32_t* sel_i
 
 namespace {
 cudaError_t launch_merge_only(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n, int64_t r,
-                              unsigned int* group_counters, cudaStream_t stream) {
+                              unsigned int* group_counters, const float* row_scales, cudaStream_t stream) {
   dim3 grid(static_cast<unsigned>((n + kMergeCols - 1) / kMergeCols),
             static_cast<unsigned>((k + kMergeRows - 1) / kMergeRows));
   const size_t smem = sizeof(float) * (static_cast<size_t>(r) * kMergeCols + static_cast<size_t>(kMergeRows) * r);
@@ -447,14 +459,21 @@ cudaError_t launch_merge_only(uint8_t* wq, float* dbuf, const int32_t* sel_idx, 
     configured = true;
   }
   return launch_pdl(merge_rows_kernel, grid, dim3(kMergeThreads), smem, stream, 1, wq, dbuf, sel_idx, static_cast<int>(k), m,
-                    n, static_cast<int>(r), group_counters);
+                    n, static_cast<int>(r), group_counters, row_scales);
 }
 }  // namespace
 
 cudaError_t launch_merge_rows(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
                               int64_t r, cudaStream_t stream) {
-  cudaError_t e = launch_merge_only(wq, dbuf, sel_idx, k, m, n, r, nullptr, stream);
+  cudaError_t e = launch_merge_only(wq, dbuf, sel_idx, k, m, n, r, nullptr, nullptr, stream);
   if (e != cudaSuccess) return e;
+  int64_t zb = (k * r + 255) / 256;
+  if (zb > 1024) zb = 1024;
+  return launch_pdl(zero_rows_kernel, dim3(static_cast<unsigned>(zb)), dim3(256), 0, stream, 1, dbuf, sel_idx,
+                    static_cast<int>(k), static_cast<int>(r));
+}
+
+cudaError_t launch_zero_rows(float* dbuf, const int32_t* sel_idx, int64_t k, int64_t r, cudaStream_t stream) {
   int64_t zb = (k * r + 255) / 256;
   if (zb > 1024) zb = 1024;
   return launch_pdl(zero_rows_kernel, dim3(static_cast<unsigned>(zb)), dim3(256), 0, stream, 1, dbuf, sel_idx,
@@ -464,8 +483,8 @@ cudaError_t launch_merge_rows(uint8_t* wq, float* dbuf, const int32_t* sel_idx, 
 int merge_group_count(int64_t k) { return static_cast<int>((k + kMergeRows - 1) / kMergeRows); }
 
 cudaError_t launch_merge_rows_fused(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
-                                    int64_t r, unsigned int* group_counters, cudaStream_t stream) {
-  return launch_merge_only(wq, dbuf, sel_idx, k, m, n, r, group_counters, stream);
+                                    int64_t r, unsigned int* group_counters, const float* row_scales, cudaStream_t stream) {
+  return launch_merge_only(wq, dbuf, sel_idx, k, m, n, r, group_counters, row_scales, stream);
 }
 
 cudaError_t launch_sgd_score_topk(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, int64_t k, float* score,

@@ -63,6 +63,7 @@ extern "C" int falqon_proxy_update_static(const falqon_layer* L, const float* dB
       L->r % 8 != 0 || L->n >= (1ll << 30) || k < 0 || k > L->m || !(lr == lr) || (dB != nullptr && !aligned16(dB)))
     return FALQON_ERR_INVALID_ARG;
   if (L->m > kMaxRows) return FALQON_ERR_UNSUPPORTED;   // the built-in scratch holds FALQON_STATIC_MAX_ROWS rows
+  if (L->gran != FALQON_PER_TENSOR) return FALQON_ERR_UNSUPPORTED;   // per-tensor scaled layers only
   unsigned char* scratch = scratch_on_current_device();
   if (scratch == nullptr) return FALQON_ERR_CUDA;
   float* score = reinterpret_cast<float*>(scratch);

@@ -203,11 +203,27 @@ __device__ __forceinline__ void unpack_raw(const RawVec<kF32>& r, float (&v)[16]
   v[8] = r.c.x; v[9] = r.c.y; v[10] = r.c.z; v[11] = r.c.w; v[12] = r.d.x; v[13] = r.d.y; v[14] = r.d.z; v[15] = r.d.w;
 }
 
-template <int kDt, int kFmt>
+// Multiplies the 16 values of one vector by the per-column factors col_mul[col .. col+15] (each its own
+// rounded multiply); a vector never straddles a row because the row length is a multiple of 16.
+__device__ __forceinline__ void apply_col_mul(float (&x)[16], const float* __restrict__ col_mul, int64_t elem, int cols) {
+  const int col = static_cast<int>(elem % cols);
+  const float4* p = reinterpret_cast<const float4*>(col_mul + col);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float4 f = __ldg(p + i);
+    x[4 * i] = __fmul_rn(x[4 * i], f.x); x[4 * i + 1] = __fmul_rn(x[4 * i + 1], f.y);
+    x[4 * i + 2] = __fmul_rn(x[4 * i + 2], f.z); x[4 * i + 3] = __fmul_rn(x[4 * i + 3], f.w);
+  }
+}
+
+// kColMul: every column c of the [rows][cols] tensor is first multiplied by col_mul[c] (the output gradient
+// of a layer whose backbone rows carry their own scales: col_mul[c] = 1 / s_w[c]).
+template <int kDt, int kFmt, bool kColMul>
 __global__ void __launch_bounds__(kThreads) quantize_fused_kernel(const void* __restrict__ src, int64_t count,
                                                                   uint8_t* __restrict__ dst, uint32_t* __restrict__ partial,
                                                                   GridSync* __restrict__ sync, CastOutputs out,
-                                                                  int* __restrict__ status) {
+                                                                  int* __restrict__ status,
+                                                                  const float* __restrict__ col_mul, int cols) {
   constexpr int kCache = (kDt == kBF16) ? 4 : 2;
   __shared__ uint32_t red[32];
   __shared__ int s_ok;
@@ -229,6 +245,7 @@ __global__ void __launch_bounds__(kThreads) quantize_fused_kernel(const void* __
     const int64_t v = first + i * stride;
     if (v < nvec) {
       unpack_raw(cache[i], x);
+      if (kColMul) apply_col_mul(x, col_mul, v * 16, cols);
 #pragma unroll
       for (int e = 0; e < 16; ++e) m = max(m, abs_bits(x[e]));
     }
@@ -236,6 +253,7 @@ __global__ void __launch_bounds__(kThreads) quantize_fused_kernel(const void* __
   int64_t v_last = first + (int64_t)(kCache - 1) * stride;   // last vector index visited by this thread
   for (int64_t v = first + (int64_t)kCache * stride; v < nvec; v += stride) {
     load16<kDt>(src, v * 16, x);
+    if (kColMul) apply_col_mul(x, col_mul, v * 16, cols);
 #pragma unroll
     for (int e = 0; e < 16; ++e) m = max(m, abs_bits(x[e]));
     v_last = v;
@@ -275,6 +293,7 @@ __global__ void __launch_bounds__(kThreads) quantize_fused_kernel(const void* __
     // streamed part, most recent first
     for (int64_t v = v_last; v >= first + (int64_t)kCache * stride; v -= stride) {
       load16<kDt>(src, v * 16, x);
+      if (kColMul) apply_col_mul(x, col_mul, v * 16, cols);
       reinterpret_cast<uint4*>(dst)[v] = cast16<kFmt>(x, 1.0f, false, s);
     }
 #pragma unroll
@@ -282,6 +301,7 @@ __global__ void __launch_bounds__(kThreads) quantize_fused_kernel(const void* __
       const int64_t v = first + i * stride;
       if (v < nvec) {
         unpack_raw(cache[i], x);
+        if (kColMul) apply_col_mul(x, col_mul, v * 16, cols);
         reinterpret_cast<uint4*>(dst)[v] = cast16<kFmt>(x, 1.0f, false, s);
       }
     }
@@ -300,6 +320,19 @@ __global__ void __launch_bounds__(kThreads) quantize_fused_kernel(const void* __
       __threadfence();
     }
   }
+}
+
+// ---- per-row-scaled backbone: small tables derived from the row scales s_w[0..m] (s_w[m] = scale of the A~ block)
+//   mode 0: out[i] = 1 / s_w[i], i < m                      (column factors of dY before its E5M2 cast)
+//   mode 1: out[c] = 1 / (s_w[min(c, m)] * s_x), c < m + r  (column factors of the forward epilogue); zero beyond
+__global__ void __launch_bounds__(256) scale_table_kernel(int mode, const float* __restrict__ s_w, int m, int r,
+                                                          const float* __restrict__ s_x, float* __restrict__ out, int padded) {
+  pdl_trigger();
+  pdl_wait();
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= padded) return;
+  if (mode == 0) out[c] = c < m ? __fdiv_rn(1.0f, s_w[c]) : 0.0f;
+  else out[c] = c < m + r ? __fdiv_rn(1.0f, __fmul_rn(s_w[c < m ? c : m], *s_x)) : 0.0f;
 }
 
 // ---- per-row scaling: one CTA per row, the row is read twice (second time from L1/L2)
@@ -420,13 +453,13 @@ cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, i
 #undef FALQON_CAST
 }
 
-template <int kDt, int kFmt>
+template <int kDt, int kFmt, bool kColMul>
 cudaError_t launch_fused_variant(const void* src, int64_t count, uint8_t* dst, uint32_t* partial, void* sync,
-                                 const CastOutputs& out, int* status, cudaStream_t stream) {
+                                 const CastOutputs& out, int* status, const float* col_mul, int cols, cudaStream_t stream) {
   static int blocks_per_sm = 0;
   if (blocks_per_sm == 0) {
     int b = 0;
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, quantize_fused_kernel<kDt, kFmt>, kThreads, 0);
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, quantize_fused_kernel<kDt, kFmt, kColMul>, kThreads, 0);
     if (e != cudaSuccess) return e;
     blocks_per_sm = b < 1 ? 1 : b;
   }
@@ -437,20 +470,34 @@ cudaError_t launch_fused_variant(const void* src, int64_t count, uint8_t* dst, u
   if (grid > resident) grid = resident;
   if (grid > kMaxAbsmaxParts) grid = kMaxAbsmaxParts;
   if (grid < 1) grid = 1;
-  return launch_pdl(quantize_fused_kernel<kDt, kFmt>, dim3(static_cast<unsigned>(grid)), dim3(kThreads), 0, stream, 1, src,
-                    count, dst, partial, static_cast<GridSync*>(sync), out, status);
+  return launch_pdl(quantize_fused_kernel<kDt, kFmt, kColMul>, dim3(static_cast<unsigned>(grid)), dim3(kThreads), 0, stream,
+                    1, src, count, dst, partial, static_cast<GridSync*>(sync), out, status, col_mul, cols);
 }
 
 cudaError_t launch_quantize_fused(const void* src, int src_dt, int64_t count, int fmt, uint8_t* dst, uint32_t* partial,
                                   void* sync, float* scale_out, float* scale_out2, float* amax_out, float* clear_word,
-                                  int* status, cudaStream_t stream) {
+                                  int* status, const float* col_mul, int cols, cudaStream_t stream) {
   const CastOutputs out{scale_out, scale_out2, amax_out, clear_word};
+#define FALQON_FUSED(DT, FMT)                                                                                              \
+  do {                                                                                                                     \
+    if (col_mul != nullptr)                                                                                                \
+      return launch_fused_variant<DT, FMT, true>(src, count, dst, partial, sync, out, status, col_mul, cols, stream);       \
+    return launch_fused_variant<DT, FMT, false>(src, count, dst, partial, sync, out, status, nullptr, 0, stream);           \
+  } while (0)
   if (src_dt == kBF16) {
-    if (fmt == kE4M3) return launch_fused_variant<kBF16, kE4M3>(src, count, dst, partial, sync, out, status, stream);
-    return launch_fused_variant<kBF16, kE5M2>(src, count, dst, partial, sync, out, status, stream);
+    if (fmt == kE4M3) FALQON_FUSED(kBF16, kE4M3);
+    FALQON_FUSED(kBF16, kE5M2);
   }
-  if (fmt == kE4M3) return launch_fused_variant<kF32, kE4M3>(src, count, dst, partial, sync, out, status, stream);
-  return launch_fused_variant<kF32, kE5M2>(src, count, dst, partial, sync, out, status, stream);
+  if (fmt == kE4M3) FALQON_FUSED(kF32, kE4M3);
+  FALQON_FUSED(kF32, kE5M2);
+#undef FALQON_FUSED
+}
+
+cudaError_t launch_scale_table(int mode, const float* s_w, int64_t m, int64_t r, const float* s_x, float* out, int64_t padded,
+                               cudaStream_t stream) {
+  const int grid = static_cast<int>((padded + 255) / 256);
+  return launch_pdl(scale_table_kernel, dim3(grid), dim3(256), 0, stream, 1, mode, s_w, static_cast<int>(m),
+                    static_cast<int>(r), s_x, out, static_cast<int>(padded));
 }
 
 cudaError_t launch_quantize_per_row(const void* src, int src_dt, int64_t rows, int64_t cols, int fmt, float premul,

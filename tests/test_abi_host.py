@@ -45,7 +45,7 @@ def test_workspace_layout(fq):
 def test_bad_arguments_are_rejected_on_the_host(fq):
     lib = fq.lib
     fake = 0x10000  # an aligned non-null address that is never dereferenced on these paths
-    layer = fq.falqon_layer(256, 256, 16, fake, fake, fake)
+    layer = fq.falqon_layer(256, 256, 16, fake, fake, fake, 0, 0)
     big = 1 << 40
     inv, wsp = fq.ERR_INVALID_ARG, fq.ERR_WORKSPACE
     # quantize
@@ -61,7 +61,9 @@ def test_bad_arguments_are_rejected_on_the_host(fq):
     assert lib.falqon_melded_forward(C.byref(layer), fake, 0, 0, fake, 0, fake, fake, None, fake, big, None) == inv
     assert lib.falqon_melded_forward(C.byref(layer), fake, 3, 16, fake, 0, fake, fake, None, fake, big, None) == inv
     assert lib.falqon_melded_forward(C.byref(layer), fake, 0, 16, fake, 0, fake, fake, None, fake, 1024, None) == wsp
-    odd = fq.falqon_layer(250, 256, 16, fake, fake, fake)
+    bad_gran = fq.falqon_layer(256, 256, 16, fake, fake, fake, 2, 0)
+    assert lib.falqon_melded_forward(C.byref(bad_gran), fake, 0, 16, fake, 0, fake, fake, None, fake, big, None) == inv
+    odd = fq.falqon_layer(250, 256, 16, fake, fake, fake, 0, 0)
     assert lib.falqon_melded_forward(C.byref(odd), fake, 0, 16, fake, 0, fake, fake, None, fake, big, None) == inv
     # backward
     assert lib.falqon_melded_backward(C.byref(layer), fake, 0, 16, None, fake, fake, 0, fake, None, fake, big, None) == inv

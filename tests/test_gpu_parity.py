@@ -76,12 +76,17 @@ def test_quantize_given_scale_premul_and_per_row(fq, orc):
 
 # ------------------------------------------------------------------ one layer, all stages
 
-def _run_layer_stages(fq, orc, seed, m, n, r, T, k, gamma, n_outliers, steps, lr, y_dtype=torch.float32):
+def _run_layer_stages(fq, orc, seed, m, n, r, T, k, gamma, n_outliers, steps, lr, y_dtype=torch.float32,
+                      per_row=False, heavy_tailed=False):
     W, A, B, X = layer_inputs(seed, 0, m, n, r, T, n_outliers)
+    if heavy_tailed:
+        W = synth.backbone(seed, 0, m, n, heavy_tailed=True)
     # S0: set-up (quantize W, A; meld B over all rows)
-    layer = fq.setup_layer(W.to(DEV), A.to(DEV), B.to(DEV), gamma)
-    wq_o, s_w_o, dbuf_o = orc.setup_layer(f32(W), f32(A), f32(B), gamma)
-    assert bits32(f32(layer.s_w))[0] == bits32(s_w_o)
+    layer = fq.setup_layer(W.to(DEV), A.to(DEV), B.to(DEV), gamma, per_row=per_row)
+    wq_o, s_w_o, dbuf_o = orc.setup_layer(f32(W), f32(A), f32(B), gamma, per_row=per_row)
+    assert np.array_equal(bits32(f32(layer.s_w)), bits32(np.atleast_1d(s_w_o)))
+    s_w_g = f32(layer.s_w) if per_row else np.float32(f32(layer.s_w)[0])
+    row_scales = s_w_g if per_row else None
     assert np.array_equal(u8(layer.wq), wq_o), "melded backbone codes differ after set-up"
     assert not f32(layer.dbuf).any()
     ws = layer.workspace(T)
@@ -93,7 +98,7 @@ def _run_layer_stages(fq, orc, seed, m, n, r, T, k, gamma, n_outliers, steps, lr
         xq_o, s_x_o, _ = orc.quantize(f32(X), orc.E4M3)
         assert bits32(f32(s_x))[0] == bits32(s_x_o) and np.array_equal(xq_g, xq_o)
         wq_now = u8(layer.wq)
-        Y_o, OA_o, _ = orc.forward(xq_g, np.float32(f32(s_x)[0]), wq_now, np.float32(f32(layer.s_w)[0]), m, r)
+        Y_o, OA_o, _ = orc.forward(xq_g, np.float32(f32(s_x)[0]), wq_now, s_w_g, m, r)
         OA_g = f32(OA)
         assert rel_fro(f32(Y), Y_o) <= GEMM_TOL, f"Y step {step}"
         assert rel_fro(OA_g, OA_o) <= GEMM_TOL, f"OA step {step}"
@@ -102,7 +107,10 @@ def _run_layer_stages(fq, orc, seed, m, n, r, T, k, gamma, n_outliers, steps, lr
         dY = synth.out_grad(seed, 0, step, T, m)
         dX, dB, s_g = fq.melded_backward(layer, dY.to(DEV), OA, amax_oa, dx_dtype=torch.float32, ws=ws)
         gq_g = u8(fq.ws_view(layer, ws, T, fq.WS_GQ)).reshape(T, m)
-        gq_o, s_g_o, _ = orc.quantize(f32(dY), orc.E5M2)
+        if per_row:
+            gq_o, s_g_o, _ = orc.quantize_colscaled(f32(dY), orc.E5M2, s_w_g[:m])
+        else:
+            gq_o, s_g_o, _ = orc.quantize(f32(dY), orc.E5M2)
         assert bits32(f32(s_g))[0] == bits32(s_g_o) and np.array_equal(gq_g, gq_o)
         oaq_o, s_oa_o, _ = orc.quantize(OA_g, orc.E4M3)
         scales = f32(fq.ws_view(layer, ws, T, fq.WS_SCALES).view(torch.float32))
@@ -110,15 +118,15 @@ def _run_layer_stages(fq, orc, seed, m, n, r, T, k, gamma, n_outliers, steps, lr
         r16, t16 = (r + 15) // 16 * 16, (T + 15) // 16 * 16
         oaq_t = u8(fq.ws_view(layer, ws, T, fq.WS_OAQ_T)).reshape(r16, t16)
         assert np.array_equal(oaq_t[:r, :T].T, oaq_o)
-        dX_o = orc.dx_gemm(gq_g, s_g_o, wq_now, np.float32(f32(layer.s_w)[0]), m)
-        dB_o = orc.db_gemm(gq_g, s_g_o, oaq_o, s_oa_o)
+        dX_o = orc.dx_gemm(gq_g, s_g_o, wq_now, s_w_g, m)
+        dB_o = orc.db_gemm(gq_g, s_g_o, oaq_o, s_oa_o, row_scale=s_w_g[:m] if per_row else None)
         assert rel_fro(f32(dX), dX_o) <= GEMM_TOL, f"dX step {step}"
         assert rel_fro(f32(dB), dB_o) <= GEMM_TOL, f"dB step {step}"
         # ---- proxy update, fed the GPU's own dB
         dbuf_o = f32(layer.dbuf).copy()
         wq_o2 = wq_now.copy()
         idx = fq.proxy_update(layer, dB, lr, k, ws=ws)
-        idx_o, score_o = orc.proxy_update(wq_o2, dbuf_o, f32(dB), lr, k, m, r)
+        idx_o, score_o = orc.proxy_update(wq_o2, dbuf_o, f32(dB), lr, k, m, r, row_scales=row_scales)
         score_g = f32(fq.ws_view(layer, ws, T, fq.WS_SCORE).view(torch.float32))
         assert np.array_equal(bits32(score_g), bits32(score_o)), f"scores step {step}"
         if k > 0:
@@ -140,6 +148,12 @@ def test_config0_three_steps_all_stages(fq, orc, lr):
                                        (1040, 528, 72, 333, 1), (256, 1024, 128, 640, 31), (512, 256, 256, 130, 512)])
 def test_ragged_and_edge_shapes(fq, orc, m, n, r, T, k):
     _run_layer_stages(fq, orc, 11, m, n, r, T, k, 1.0, 3, 2, 2e-2)
+
+
+@pytest.mark.parametrize("m,n,r,T,k", [(1024, 768, 16, 512, 32), (272, 208, 8, 200, 272), (640, 1280, 64, 300, 17)])
+def test_per_row_scaled_backbone_all_stages(fq, orc, m, n, r, T, k):
+    """Heavy-tailed backbone rows (Student-t, 3 degrees of freedom) with one scale per row."""
+    _run_layer_stages(fq, orc, 13, m, n, r, T, k, 1.0, 4, 2, 2e-2, per_row=True, heavy_tailed=True)
 
 
 def test_bf16_outputs_are_rounded_fp32_outputs(fq):

@@ -24,9 +24,9 @@ def _fq():
 def test_static_variant_rejects_oversized_and_bad_arguments():
     fq = _fq()
     fake = 0x10000
-    too_big = fq.falqon_layer(fq.STATIC_MAX_ROWS + 16, 256, 16, fake, fake, fake)
+    too_big = fq.falqon_layer(fq.STATIC_MAX_ROWS + 16, 256, 16, fake, fake, fake, 0, 0)
     assert fq.lib.falqon_proxy_update_static(C.byref(too_big), None, 0.1, 1, None, None) == fq.ERR_UNSUPPORTED
-    ok_shape = fq.falqon_layer(256, 256, 16, fake, fake, fake)
+    ok_shape = fq.falqon_layer(256, 256, 16, fake, fake, fake, 0, 0)
     assert fq.lib.falqon_proxy_update_static(C.byref(ok_shape), None, 0.1, 257, None, None) == fq.ERR_INVALID_ARG
     assert fq.lib.falqon_proxy_update_static(None, None, 0.1, 1, None, None) == fq.ERR_INVALID_ARG
 
