@@ -202,25 +202,22 @@ def test_topk_ties_go_to_lowest_index(fq, orc):
 
 # ------------------------------------------------------------------ full-size projections, sampled
 
-@pytest.mark.parametrize("name,n,m", [("q", 4096, 4096), ("gate", 4096, 11008), ("down", 11008, 4096)])
-def test_config1_projection_sampled(fq, orc, name, n, m):
-    c = synth.config1()
-    T, r, k = c["T"], c["r"], c["k"]
-    n_out = round(c["outlier_frac"] * n)
-    matrix = {"q": 0, "gate": 4, "down": 6}[name]
-    W = synth.backbone(0, matrix, m, n, DEV)
+def _sampled_projection(fq, orc, matrix, n, m, T, r, k, lr, outlier_frac, per_row=False, heavy_tailed=False):
+    """One full-size projection: bit-exact stages on every element, tensor-core outputs on sampled rows / columns."""
+    n_out = round(outlier_frac * n)
+    W = synth.backbone(0, matrix, m, n, DEV, heavy_tailed=heavy_tailed)
     A = synth.adapter_a(0, matrix, r, n, DEV)
     B = synth.adapter_b(0, matrix, m, r, DEV)
     X = synth.activations(0, matrix, T, n, n_out, DEV)
     dY = synth.out_grad(0, matrix, 0, T, m, DEV)
-    layer = fq.setup_layer(W, A, B, 1.0)
+    layer = fq.setup_layer(W, A, B, 1.0, per_row=per_row)
     ws = layer.workspace(T)
     Y, OA, amax_oa, s_x = fq.melded_forward(layer, X, y_dtype=torch.float32, ws=ws)
     xq_g = u8(fq.ws_view(layer, ws, T, fq.WS_XQ)).reshape(T, n)
     xq_o, s_x_o, _ = orc.quantize(f32(X), orc.E4M3)
     assert bits32(f32(s_x))[0] == bits32(s_x_o) and np.array_equal(xq_g, xq_o)
     wq = u8(layer.wq)
-    s_w = np.float32(f32(layer.s_w)[0])
+    s_w = f32(layer.s_w) if per_row else np.float32(f32(layer.s_w)[0])
     rng = np.random.default_rng(1)
     tsel = np.sort(rng.choice(T, 48, replace=False))
     fsel = np.sort(rng.choice(m, 48, replace=False))
@@ -232,17 +229,44 @@ def test_config1_projection_sampled(fq, orc, name, n, m):
     assert bits32(f32(amax_oa))[0] == bits32(f32(OA.abs().max()))
     dX, dB, s_g = fq.melded_backward(layer, dY, OA, amax_oa, dx_dtype=torch.float32, ws=ws)
     gq_g = u8(fq.ws_view(layer, ws, T, fq.WS_GQ)).reshape(T, m)
-    gq_o, s_g_o, _ = orc.quantize(f32(dY), orc.E5M2)
+    if per_row:
+        gq_o, s_g_o, _ = orc.quantize_colscaled(f32(dY), orc.E5M2, s_w[:m])
+    else:
+        gq_o, s_g_o, _ = orc.quantize(f32(dY), orc.E5M2)
     assert bits32(f32(s_g))[0] == bits32(s_g_o) and np.array_equal(gq_g, gq_o)
     csel = np.sort(rng.choice(n, 48, replace=False))
     assert rel_fro(f32(dX[torch.from_numpy(tsel).to(DEV)]), orc.dx_gemm(gq_g, s_g_o, wq, s_w, m, tsel=tsel)) <= GEMM_TOL
     assert rel_fro(f32(dX[:, torch.from_numpy(csel).to(DEV)]), orc.dx_gemm(gq_g, s_g_o, wq, s_w, m, csel=csel)) <= GEMM_TOL
     oaq_o, s_oa_o, _ = orc.quantize(f32(OA), orc.E4M3)
     isel = np.sort(rng.choice(m, 96, replace=False))
-    assert rel_fro(f32(dB[torch.from_numpy(isel).to(DEV)]), orc.db_gemm(gq_g, s_g_o, oaq_o, s_oa_o, isel=isel)) <= GEMM_TOL
+    dB_o = orc.db_gemm(gq_g, s_g_o, oaq_o, s_oa_o, isel=isel, row_scale=s_w[:m] if per_row else None)
+    assert rel_fro(f32(dB[torch.from_numpy(isel).to(DEV)]), dB_o) <= GEMM_TOL
     dbuf_o, wq_o = f32(layer.dbuf).copy(), wq.copy()
-    idx = fq.proxy_update(layer, dB, c["lr"], k, ws=ws)
-    idx_o, score_o = orc.proxy_update(wq_o, dbuf_o, f32(dB), c["lr"], k, m, r)
+    idx = fq.proxy_update(layer, dB, lr, k, ws=ws)
+    idx_o, score_o = orc.proxy_update(wq_o, dbuf_o, f32(dB), lr, k, m, r, row_scales=s_w if per_row else None)
     assert np.array_equal(u8(idx), idx_o)
     assert np.array_equal(u8(layer.wq), wq_o) and np.array_equal(bits32(f32(layer.dbuf)), bits32(dbuf_o))
     assert fq.last_device_status() == 0
+
+
+@pytest.mark.parametrize("name,n,m", [("q", 4096, 4096), ("gate", 4096, 11008), ("down", 11008, 4096)])
+def test_config1_projection_sampled(fq, orc, name, n, m):
+    c = synth.config1()
+    _sampled_projection(fq, orc, {"q": 0, "gate": 4, "down": 6}[name], n, m, c["T"], c["r"], c["k"], c["lr"],
+                        c["outlier_frac"])
+
+
+@pytest.mark.parametrize("name,n,m", [("q", 5120, 5120), ("down", 13824, 5120)])
+def test_config3_projection_sampled_per_row(fq, orc, name, n, m):
+    """LLaMA-13B shapes, 8192 tokens, heavy-tailed rows (0.02 * t_3) with per-row scales, top-512."""
+    _sampled_projection(fq, orc, {"q": 0, "down": 6}[name], n, m, 8192, 64, 512, 2e-4, 0.01, per_row=True,
+                        heavy_tailed=True)
+
+
+@pytest.mark.parametrize("r,T,k", [(8, 512, 4096), (128, 2048, 64), (32, 512, 0)])
+def test_config4_sweep_corner_shapes(fq, orc, r, T, k):
+    """Corners of the rank x tokens x top-k sweep on the 4096 -> 11008 projection."""
+    if k == 0:
+        _run_layer_stages(fq, orc, 0, 11008, 4096, r, T, 0, 1.0, 41, 1, 2e-4)
+    else:
+        _sampled_projection(fq, orc, 4, 4096, 11008, T, r, k, 2e-4, 0.01)
