@@ -360,6 +360,42 @@ int orc_proxy_update(uint8_t* wq, float* dbuf, const float* dB, float lr, const 
   return 0;
 }
 
+// AdamW on the DeltaBuffer (the optimizer the paper trains with; Alg. 3 line 4 leaves "Optimizer" generic).
+// One step t >= 1 for every element, all in fp32 in this order (decoupled weight decay first):
+//   p  = p * decay                          decay     = (float)(1 - lr*wd)
+//   m  = fma(beta1, m, (1-beta1) * g)
+//   v  = fma(beta2, v, (1-beta2) * (g*g))
+//   p  = fma(-step_size, m / (sqrt(v) / sqrt_bc2 + eps), p)
+//                                           step_size = (float)(lr / (1 - beta1^t)),  sqrt_bc2 = (float)sqrt(1 - beta2^t)
+// The three derived constants are evaluated in double and rounded once to fp32.
+void orc_adamw_constants(float lr, float beta1, float beta2, float weight_decay, int64_t step, float* decay,
+                         float* one_minus_b1, float* one_minus_b2, float* step_size, float* sqrt_bc2) {
+  *decay = (float)(1.0 - (double)lr * (double)weight_decay);
+  *one_minus_b1 = (float)(1.0 - (double)beta1);
+  *one_minus_b2 = (float)(1.0 - (double)beta2);
+  *step_size = (float)((double)lr / (1.0 - std::pow((double)beta1, (double)step)));
+  *sqrt_bc2 = (float)std::sqrt(1.0 - std::pow((double)beta2, (double)step));
+}
+
+int orc_adamw_step(float* p, const float* g, float* exp_avg, float* exp_avg_sq, int64_t count, float lr, float beta1,
+                   float beta2, float eps, float weight_decay, int64_t step) {
+  if (step < 1) return -1;
+  float decay, omb1, omb2, step_size, sqrt_bc2;
+  orc_adamw_constants(lr, beta1, beta2, weight_decay, step, &decay, &omb1, &omb2, &step_size, &sqrt_bc2);
+  for (int64_t e = 0; e < count; ++e) {
+    const float gi = g[e];
+    const float p1 = p[e] * decay;
+    const float m1 = std::fmaf(beta1, exp_avg[e], omb1 * gi);
+    const float g2 = gi * gi;
+    const float v1 = std::fmaf(beta2, exp_avg_sq[e], omb2 * g2);
+    const float denom = std::sqrt(v1) / sqrt_bc2 + eps;
+    p[e] = std::fmaf(-step_size, m1 / denom, p1);
+    exp_avg[e] = m1;
+    exp_avg_sq[e] = v1;
+  }
+  return 0;
+}
+
 int orc_num_threads(void) {
   int nthreads = 1;
 #ifdef _OPENMP

@@ -46,6 +46,8 @@ _lib.orc_proxy_update.restype = _i32
 _lib.orc_proxy_update.argtypes = [_p, _p, _p, _f32, _p, _i64, _i64, _i64, _i64, _p, _p]
 _lib.orc_quantize_colscaled.restype = _i32
 _lib.orc_quantize_colscaled.argtypes = [_p, _i32, _i64, _i64, _i32, _p, _p, _p, _p]
+_lib.orc_adamw_step.restype = _i32
+_lib.orc_adamw_step.argtypes = [_p, _p, _p, _p, _i64, _f32, _f32, _f32, _f32, _f32, _i64]
 _lib.orc_num_threads.restype = _i32
 
 
@@ -215,6 +217,18 @@ def proxy_update(wq, dbuf, dB, lr: float, k: int, m: int, r: int, row_scales=Non
     if rc != 0:
         raise ValueError("orc_proxy_update rejected its arguments")
     return idx, score
+
+
+def adamw_step(p, g, exp_avg, exp_avg_sq, lr, beta1, beta2, eps, weight_decay, step: int):
+    """AdamW on the DeltaBuffer, in place on p, exp_avg, exp_avg_sq (float32, contiguous)."""
+    for a in (p, exp_avg, exp_avg_sq):
+        assert a.dtype == np.float32 and a.flags.c_contiguous
+    g = _c(g, np.float32)
+    rc = _lib.orc_adamw_step(_ptr(p), _ptr(g), _ptr(exp_avg), _ptr(exp_avg_sq), p.size, float(np.float32(lr)),
+                             float(np.float32(beta1)), float(np.float32(beta2)), float(np.float32(eps)),
+                             float(np.float32(weight_decay)), int(step))
+    if rc != 0:
+        raise ValueError("orc_adamw_step rejected its arguments")
 
 
 # ---- whole-layer compositions in the paper's order (each step is one oracle call) ----
