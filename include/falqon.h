@@ -154,6 +154,22 @@ int falqon_melded_backward(const falqon_layer *L, const void *dY, falqon_dtype d
 int falqon_proxy_update(const falqon_layer *L, const float *dB, float lr, int64_t k, int32_t *idx_out,
                         void *ws, size_t ws_bytes, falqon_stream stream);
 
+/* The same update with AdamW as the optimizer -- the one the paper trains with (its Alg. 3 leaves "Optimizer"
+ * generic).  exp_avg and exp_avg_sq are device [m][r] fp32 state, zero before step 1, updated in place; they are NOT
+ * cleared when a row is merged (only DeltaBuffer rows are).  For every element, in fp32 and in this order:
+ *   p = p * (1 - lr*weight_decay);   m = fma(beta1, m, (1-beta1) * g);   v = fma(beta2, v, (1-beta2) * (g*g));
+ *   p = fma(-lr / (1 - beta1^step), m / (sqrt(v) / sqrt(1 - beta2^step) + eps), p)
+ * where the constants (1 - lr*weight_decay), (1-beta), lr / (1 - beta1^step), sqrt(1 - beta2^step) are evaluated in
+ * double from the fp32 hyper-parameters and rounded once to fp32.  step counts from 1.  Everything after the
+ * optimizer (scores, top-k, merge, clearing) is as in falqon_proxy_update. */
+typedef struct {
+  float lr, beta1, beta2, eps, weight_decay;
+  int64_t step;
+} falqon_adamw;
+int falqon_proxy_update_adamw(const falqon_layer *L, const float *dB, float *exp_avg, float *exp_avg_sq,
+                              const falqon_adamw *hp, int64_t k, int32_t *idx_out, void *ws, size_t ws_bytes,
+                              falqon_stream stream);
+
 /* The proxy update for callers that cannot provide a workspace.  The paper has no counterpart: this
  * is the same operation as falqon_proxy_update, with the same arguments minus the workspace, for code
  * that runs as a guest inside another runtime (a framework's custom-op hook, a server's plug-in) whose

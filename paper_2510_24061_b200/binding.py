@@ -22,7 +22,7 @@ WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE, WS_DB_PART = range(6)
 
 EXPORTS = ["falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_last_device_status", "falqon_launch_count",
-           "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static", "falqon_workspace_init"]
+           "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static", "falqon_workspace_init", "falqon_proxy_update_adamw"]
 STATIC_MAX_ROWS = 16384
 STAGES = ["quant_x", "gemm_fwd", "quant_dy", "quant_oa", "gemm_dx", "gemm_db", "reduce_db", "sgd_score", "topk", "merge"]
 
@@ -53,6 +53,13 @@ lib.falqon_melded_backward.restype = _i
 lib.falqon_melded_backward.argtypes = [C.POINTER(falqon_layer), _p, _i, _i64, _p, _p, _p, _i, _p, _p, _p, _sz, _p]
 lib.falqon_proxy_update.restype = _i
 lib.falqon_proxy_update.argtypes = [C.POINTER(falqon_layer), _p, _f, _i64, _p, _p, _sz, _p]
+class falqon_adamw(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("weight_decay", C.c_float), ("step", C.c_int64)]
+
+
+lib.falqon_proxy_update_adamw.restype = _i
+lib.falqon_proxy_update_adamw.argtypes = [C.POINTER(falqon_layer), _p, _p, _p, C.POINTER(falqon_adamw), _i64, _p, _p, _sz, _p]
 lib.falqon_proxy_update_static.restype = _i
 lib.falqon_proxy_update_static.argtypes = [C.POINTER(falqon_layer), _p, _f, _i64, _p, _p]
 lib.falqon_last_device_status.restype = _i
@@ -261,4 +268,19 @@ def proxy_update_static(layer: Layer, dB: torch.Tensor | None, lr: float, k: int
         idx_out = torch.empty(k, dtype=torch.int32, device=layer.wq.device)
     _check("falqon_proxy_update_static",
            lib.falqon_proxy_update_static(C.byref(layer.c), _ptr(dB), lr, k, _ptr(idx_out), _stream()))
+    return idx_out
+
+
+def proxy_update_adamw(layer: Layer, dB: torch.Tensor, exp_avg: torch.Tensor, exp_avg_sq: torch.Tensor, step: int, k: int,
+                       lr: float = 2e-4, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+                       weight_decay: float = 0.0, ws: torch.Tensor | None = None, idx_out: torch.Tensor | None = None):
+    """falqon_proxy_update_adamw: AdamW step on the DeltaBuffer (state in exp_avg / exp_avg_sq, fp32 [m, r], zero before
+    step 1), then scores, top-k, merge and clearing as in proxy_update.  Returns idx int32 [k] ascending."""
+    ws = layer.workspace(1) if ws is None else ws
+    if idx_out is None and 0 < k <= layer.m:
+        idx_out = torch.empty(k, dtype=torch.int32, device=layer.wq.device)
+    hp = falqon_adamw(lr, beta1, beta2, eps, weight_decay, step)
+    _check("falqon_proxy_update_adamw",
+           lib.falqon_proxy_update_adamw(C.byref(layer.c), _ptr(dB), _ptr(exp_avg), _ptr(exp_avg_sq), C.byref(hp), k,
+                                         _ptr(idx_out), _ptr(ws), ws.numel(), _stream()))
     return idx_out

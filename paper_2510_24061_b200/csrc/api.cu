@@ -297,8 +297,10 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
   return FALQON_OK;
 }
 
-int falqon_proxy_update(const falqon_layer* L, const float* dB, float lr, int64_t k, int32_t* idx_out, void* ws,
-                        size_t ws_bytes, falqon_stream stream) {
+namespace {
+// Shared tail of the two proxy-update entry points.  adamw == nullptr: plain SGD with `lr` (or no optimizer when dB is null).
+int proxy_update_impl(const falqon_layer* L, const float* dB, float lr, const falqon_adamw* adamw, float* exp_avg,
+                      float* exp_avg_sq, int64_t k, int32_t* idx_out, void* ws, size_t ws_bytes, falqon_stream stream) {
   if (!layer_ok(L) || k < 0 || k > L->m || !(lr == lr) || (dB != nullptr && !aligned16(dB)))
     return FALQON_ERR_INVALID_ARG;
   WorkspaceLayout w;
@@ -313,7 +315,12 @@ int falqon_proxy_update(const falqon_layer* L, const float* dB, float lr, int64_
   const bool fused_merge = static_cast<size_t>(merge_group_count(k)) <= kMaxMergeGroups;
   {
     StageTimer timer(FALQON_STAGE_SGD_SCORE, stream);   // optimizer step, scores and (k > 0) the selection: one kernel
-    FALQON_CUDA(launch_sgd_score_topk(L->dbuf, dB, lr, m, r, k, score, sel, idx_out, done_counter, stream));
+    if (adamw != nullptr) {
+      FALQON_CUDA(launch_adamw_score_topk(L->dbuf, dB, exp_avg, exp_avg_sq, adamw->lr, adamw->beta1, adamw->beta2, adamw->eps,
+                                          adamw->weight_decay, adamw->step, m, r, k, score, sel, idx_out, done_counter, stream));
+    } else {
+      FALQON_CUDA(launch_sgd_score_topk(L->dbuf, dB, lr, m, r, k, score, sel, idx_out, done_counter, stream));
+    }
   }
   if (k > 0) {
     StageTimer timer(FALQON_STAGE_MERGE, stream);
@@ -328,6 +335,22 @@ int falqon_proxy_update(const falqon_layer* L, const float* dB, float lr, int64_
     }
   }
   return FALQON_OK;
+}
+}  // namespace
+
+int falqon_proxy_update(const falqon_layer* L, const float* dB, float lr, int64_t k, int32_t* idx_out, void* ws,
+                        size_t ws_bytes, falqon_stream stream) {
+  return proxy_update_impl(L, dB, lr, nullptr, nullptr, nullptr, k, idx_out, ws, ws_bytes, stream);
+}
+
+int falqon_proxy_update_adamw(const falqon_layer* L, const float* dB, float* exp_avg, float* exp_avg_sq,
+                              const falqon_adamw* hp, int64_t k, int32_t* idx_out, void* ws, size_t ws_bytes,
+                              falqon_stream stream) {
+  if (hp == nullptr || dB == nullptr || exp_avg == nullptr || exp_avg_sq == nullptr || !aligned16(exp_avg) ||
+      !aligned16(exp_avg_sq) || hp->step < 1 || !(hp->lr == hp->lr) || !(hp->beta1 >= 0.0f && hp->beta1 < 1.0f) ||
+      !(hp->beta2 >= 0.0f && hp->beta2 < 1.0f) || !(hp->eps >= 0.0f) || !(hp->weight_decay == hp->weight_decay))
+    return FALQON_ERR_INVALID_ARG;
+  return proxy_update_impl(L, dB, hp->lr, hp, exp_avg, exp_avg_sq, k, idx_out, ws, ws_bytes, stream);
 }
 
 int falqon_last_device_status(falqon_stream stream) {

@@ -106,6 +106,11 @@ cudaError_t launch_zero_rows(float* dbuf, const int32_t* sel_idx, int64_t k, int
 cudaError_t launch_sgd_score_topk(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, int64_t k, float* score,
                                   int32_t* sel_idx, int32_t* idx_copy, unsigned int* done_counter, cudaStream_t stream);
 // row_scales (nullable, m + 1 entries): per-row mode, DeltaBuffer row i enters the chain times s_w[i] / s_w[m].
+// The same kernel with AdamW (decoupled weight decay) as the optimizer; exp_avg / exp_avg_sq are [m][r] fp32 state.
+cudaError_t launch_adamw_score_topk(float* dbuf, const float* dB, float* exp_avg, float* exp_avg_sq, float lr, float beta1,
+                                    float beta2, float eps, float weight_decay, int64_t step, int64_t m, int64_t r, int64_t k,
+                                    float* score, int32_t* sel_idx, int32_t* idx_copy, unsigned int* done_counter,
+                                    cudaStream_t stream);
 cudaError_t launch_merge_rows_fused(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
                                     int64_t r, unsigned int* group_counters, const float* row_scales, cudaStream_t stream);
 

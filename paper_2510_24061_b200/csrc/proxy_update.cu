@@ -2,6 +2,8 @@
 // the split adapter-gradient partial sums.  Everything that feeds a bit-exact stage is done in fp32
 // with an explicit operation order: one fma per DeltaBuffer element, left-to-right row sums, and the
 // merge as an fma chain over the rank index.
+#include <cmath>
+
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -211,11 +213,37 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
   topk_block(score, m, k, sel_idx, idx_out, use_smem ? s_bits_dyn : nullptr);
 }
 
+// ---- the optimizer step on one DeltaBuffer element.  kind 0: none (the caller ran its own optimizer), 1: plain
+// SGD d = fma(-lr, g, d), 2: AdamW with decoupled weight decay, all fp32 in this order:
+//   p = p * decay;  m = fma(beta1, m, (1-beta1) * g);  v = fma(beta2, v, (1-beta2) * (g*g));
+//   p = fma(-step_size, m / (sqrt(v) / sqrt_bc2 + eps), p)
+struct OptimizerArgs {
+  int kind;
+  float neg_lr;                                   // SGD
+  float beta1, beta2, eps, decay, one_minus_b1, one_minus_b2, neg_step_size, sqrt_bc2;   // AdamW
+  float* exp_avg;
+  float* exp_avg_sq;
+};
+__device__ __forceinline__ float optimizer_update(const OptimizerArgs& o, float d, const float* __restrict__ dB, int64_t e) {
+  if (o.kind == 1) return __fmaf_rn(o.neg_lr, dB[e], d);
+  if (o.kind == 2) {
+    const float g = dB[e];
+    const float p1 = __fmul_rn(d, o.decay);
+    const float m1 = __fmaf_rn(o.beta1, o.exp_avg[e], __fmul_rn(o.one_minus_b1, g));
+    const float v1 = __fmaf_rn(o.beta2, o.exp_avg_sq[e], __fmul_rn(o.one_minus_b2, __fmul_rn(g, g)));
+    const float denom = __fadd_rn(__fdiv_rn(__fsqrt_rn(v1), o.sqrt_bc2), o.eps);
+    o.exp_avg[e] = m1;
+    o.exp_avg_sq[e] = v1;
+    return __fmaf_rn(o.neg_step_size, __fdiv_rn(m1, denom), p1);
+  }
+  return d;
+}
+
 // ---- optimizer step + row scores + selection in ONE kernel: CTAs of 1024 threads take 128 rows each; the CTA
 // that finishes last (a counter in the workspace that is zero between calls) runs the selection on all scores.
 constexpr int kFusedScoreRows = 128;
 __global__ void __launch_bounds__(kTopkThreads) sgd_score_topk_kernel(float* __restrict__ dbuf, const float* __restrict__ dB,
-                                                                      float neg_lr, int m, int r, int k,
+                                                                      OptimizerArgs opt, int m, int r, int k,
                                                                       float* __restrict__ score, int32_t* __restrict__ sel_idx,
                                                                       int32_t* __restrict__ idx_out,
                                                                       unsigned int* __restrict__ done_counter, int use_smem) {
@@ -228,8 +256,8 @@ __global__ void __launch_bounds__(kTopkThreads) sgd_score_topk_kernel(float* __r
   const int64_t base = (int64_t)row0 * r;
   for (int e = threadIdx.x; e < rows * r; e += blockDim.x) {
     float d = dbuf[base + e];
-    if (dB != nullptr) {
-      d = __fmaf_rn(neg_lr, dB[base + e], d);
+    if (opt.kind != 0) {
+      d = optimizer_update(opt, d, dB, base + e);
       dbuf[base + e] = d;
     }
     const int i = e / r, j = e - i * r;
@@ -487,8 +515,10 @@ cudaError_t launch_merge_rows_fused(uint8_t* wq, float* dbuf, const int32_t* sel
   return launch_merge_only(wq, dbuf, sel_idx, k, m, n, r, group_counters, row_scales, stream);
 }
 
-cudaError_t launch_sgd_score_topk(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, int64_t k, float* score,
-                                  int32_t* sel_idx, int32_t* idx_copy, unsigned int* done_counter, cudaStream_t stream) {
+namespace {
+cudaError_t launch_opt_score_topk(float* dbuf, const float* dB, const OptimizerArgs& opt, int64_t m, int64_t r, int64_t k,
+                                  float* score, int32_t* sel_idx, int32_t* idx_copy, unsigned int* done_counter,
+                                  cudaStream_t stream) {
   const int use_smem = m <= kTopkSmemRows ? 1 : 0;
   size_t smem = sizeof(float) * kFusedScoreRows * (r + 1);
   if (use_smem && static_cast<size_t>(m) * sizeof(uint32_t) > smem) smem = static_cast<size_t>(m) * sizeof(uint32_t);
@@ -500,9 +530,36 @@ cudaError_t launch_sgd_score_topk(float* dbuf, const float* dB, float lr, int64_
     configured = true;
   }
   const int grid = static_cast<int>((m + kFusedScoreRows - 1) / kFusedScoreRows);
-  return launch_pdl(sgd_score_topk_kernel, dim3(grid), dim3(kTopkThreads), smem, stream, 1, dbuf, dB, -lr,
+  return launch_pdl(sgd_score_topk_kernel, dim3(grid), dim3(kTopkThreads), smem, stream, 1, dbuf, dB, opt,
                     static_cast<int>(m), static_cast<int>(r), static_cast<int>(k), score, sel_idx, idx_copy, done_counter,
                     use_smem);
+}
+}  // namespace
+
+cudaError_t launch_sgd_score_topk(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, int64_t k, float* score,
+                                  int32_t* sel_idx, int32_t* idx_copy, unsigned int* done_counter, cudaStream_t stream) {
+  OptimizerArgs opt{};
+  opt.kind = dB != nullptr ? 1 : 0;
+  opt.neg_lr = -lr;
+  return launch_opt_score_topk(dbuf, dB, opt, m, r, k, score, sel_idx, idx_copy, done_counter, stream);
+}
+
+cudaError_t launch_adamw_score_topk(float* dbuf, const float* dB, float* exp_avg, float* exp_avg_sq, float lr, float beta1,
+                                    float beta2, float eps, float weight_decay, int64_t step, int64_t m, int64_t r, int64_t k,
+                                    float* score, int32_t* sel_idx, int32_t* idx_copy, unsigned int* done_counter,
+                                    cudaStream_t stream) {
+  OptimizerArgs opt{};
+  opt.kind = 2;
+  opt.beta1 = beta1; opt.beta2 = beta2; opt.eps = eps;
+  // derived constants: evaluated in double, rounded once to fp32
+  opt.decay = static_cast<float>(1.0 - static_cast<double>(lr) * static_cast<double>(weight_decay));
+  opt.one_minus_b1 = static_cast<float>(1.0 - static_cast<double>(beta1));
+  opt.one_minus_b2 = static_cast<float>(1.0 - static_cast<double>(beta2));
+  opt.neg_step_size = -static_cast<float>(static_cast<double>(lr) / (1.0 - std::pow(static_cast<double>(beta1), static_cast<double>(step))));
+  opt.sqrt_bc2 = static_cast<float>(std::sqrt(1.0 - std::pow(static_cast<double>(beta2), static_cast<double>(step))));
+  opt.exp_avg = exp_avg;
+  opt.exp_avg_sq = exp_avg_sq;
+  return launch_opt_score_topk(dbuf, dB, opt, m, r, k, score, sel_idx, idx_copy, done_counter, stream);
 }
 
 }  // namespace falqon

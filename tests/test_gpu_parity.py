@@ -270,3 +270,25 @@ def test_config4_sweep_corner_shapes(fq, orc, r, T, k):
         _run_layer_stages(fq, orc, 0, 11008, 4096, r, T, 0, 1.0, 41, 1, 2e-4)
     else:
         _sampled_projection(fq, orc, 4, 4096, 11008, T, r, k, 2e-4, 0.01)
+
+
+def test_adamw_proxy_update_bit_exact(fq, orc):
+    """AdamW on the DeltaBuffer (the optimizer the paper trains with), three steps with merges in between."""
+    m, n, r, k = 1024, 512, 32, 48
+    W, A, B, _ = layer_inputs(17, 0, m, n, r, 16, 0)
+    layer = fq.setup_layer(W.to(DEV), A.to(DEV), B.to(DEV), 1.0)
+    wq_o, dbuf_o = u8(layer.wq).copy(), f32(layer.dbuf).copy()
+    m_g = torch.zeros((m, r), dtype=torch.float32, device=DEV)
+    v_g = torch.zeros((m, r), dtype=torch.float32, device=DEV)
+    m_o, v_o = np.zeros((m, r), np.float32), np.zeros((m, r), np.float32)
+    hp = dict(lr=2e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    for step in range(1, 4):
+        dB = synth.normal_bf16(17, 40 + step, (m, r), 1e-2).float()
+        idx = fq.proxy_update_adamw(layer, dB.to(DEV), m_g, v_g, step, k, **hp)
+        orc.adamw_step(dbuf_o, dB.numpy(), m_o, v_o, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"], step)
+        idx_o, _ = orc.proxy_update(wq_o, dbuf_o, None, 0.0, k, m, r)
+        assert np.array_equal(u8(idx), idx_o), step
+        assert np.array_equal(bits32(f32(m_g)), bits32(m_o)) and np.array_equal(bits32(f32(v_g)), bits32(v_o)), step
+        assert np.array_equal(bits32(f32(layer.dbuf)), bits32(dbuf_o)), step
+        assert np.array_equal(u8(layer.wq), wq_o), step
+    assert fq.last_device_status() == 0
