@@ -151,7 +151,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ro
       const float4* cs = reinterpret_cast<const float4*>(p.col_scale + col0);
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        const float4 s4 = __ldg(cs + i);
+        const float4 s4 = ld_stream(cs + i);
         f[4 * i] = __uint_as_float(v[4 * i]) * s4.x; f[4 * i + 1] = __uint_as_float(v[4 * i + 1]) * s4.y;
         f[4 * i + 2] = __uint_as_float(v[4 * i + 2]) * s4.z; f[4 * i + 3] = __uint_as_float(v[4 * i + 3]) * s4.w;
       }
@@ -338,7 +338,7 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     const int col_half = (warp - 2) >> 2;   // warps 2..5 drain the left half of the tile, 6..9 the right half
     uint8_t* stage_out = smem_gen + static_cast<uint32_t>(S) * stage_bytes + kBarrierBytes + (warp - 2) * kStageOutBytes;
     const bool rescale = p.scale_a != nullptr;
-    const float inv = rescale ? 1.0f / (p.scale_b != nullptr ? __ldg(p.scale_a) * __ldg(p.scale_b) : __ldg(p.scale_a)) : 1.0f;
+    const float inv = rescale ? 1.0f / (p.scale_b != nullptr ? ld_stream(p.scale_a) * ld_stream(p.scale_b) : ld_stream(p.scale_a)) : 1.0f;
     int acc = 0;
     uint32_t acc_phase = 0;
     uint32_t amax_bits = 0;
@@ -538,7 +538,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     const int col_half = (warp - 2) >> 2;
     uint8_t* stage_out = smem_gen + static_cast<uint32_t>(S) * kPairStageBytes + kBarrierBytes + (warp - 2) * kStageOutBytes;
     const bool rescale = p.scale_a != nullptr;
-    const float inv = rescale ? 1.0f / (p.scale_b != nullptr ? __ldg(p.scale_a) * __ldg(p.scale_b) : __ldg(p.scale_a)) : 1.0f;
+    const float inv = rescale ? 1.0f / (p.scale_b != nullptr ? ld_stream(p.scale_a) * ld_stream(p.scale_b) : ld_stream(p.scale_a)) : 1.0f;
     int acc = 0;
     uint32_t acc_phase = 0;
     uint32_t amax_bits = 0;

@@ -11,12 +11,12 @@ namespace falqon {
 namespace {
 
 // ---- dB = (sum over splits, in split order) / (s_g * s_OA)
-__global__ void __launch_bounds__(256) reduce_db_kernel(const float* __restrict__ partials, int splits, int64_t count,
-                                                        const float* __restrict__ s_g, const float* __restrict__ s_oa,
-                                                        const float* __restrict__ row_mul, int r, float* __restrict__ dB) {
+__global__ void __launch_bounds__(256) reduce_db_kernel(const float* partials, int splits, int64_t count,
+                                                        const float* s_g, const float* s_oa,
+                                                        const float* row_mul, int r, float* dB) {
   pdl_trigger();
   pdl_wait();
-  const float inv = 1.0f / (__ldg(s_g) * __ldg(s_oa));
+  const float inv = 1.0f / (ld_stream(s_g) * ld_stream(s_oa));
   const int64_t nvec = count / 4;
   for (int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; v < nvec; v += (int64_t)gridDim.x * blockDim.x) {
     float4 acc = reinterpret_cast<const float4*>(partials)[v];
@@ -26,7 +26,7 @@ __global__ void __launch_bounds__(256) reduce_db_kernel(const float* __restrict_
     }
     acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
     if (row_mul != nullptr) {   // per-row-scaled backbone: give row i its scale back (r is a multiple of 4)
-      const float f = __ldg(row_mul + (v * 4) / r);
+      const float f = ld_stream(row_mul + (v * 4) / r);
       acc.x *= f; acc.y *= f; acc.z *= f; acc.w *= f;
     }
     reinterpret_cast<float4*>(dB)[v] = acc;
@@ -35,8 +35,8 @@ __global__ void __launch_bounds__(256) reduce_db_kernel(const float* __restrict_
 
 // ---- DeltaBuffer <- fma(-lr, dB, DeltaBuffer); score_i = ((|d_i0| + |d_i1|) + ...) in fp32
 constexpr int kScoreRows = 32;
-__global__ void __launch_bounds__(256) sgd_score_kernel(float* __restrict__ dbuf, const float* __restrict__ dB,
-                                                        float neg_lr, int64_t m, int r, float* __restrict__ score) {
+__global__ void __launch_bounds__(256) sgd_score_kernel(float* dbuf, const float* dB,
+                                                        float neg_lr, int64_t m, int r, float* score) {
   extern __shared__ float sabs[];  // [kScoreRows][r + 1]
   pdl_trigger();
   pdl_wait();
@@ -100,8 +100,8 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums /* [32
 
 // The whole selection, run by one CTA (all of its threads).  s_bits: shared-memory staging for the m scores, or
 // null to read them from global memory every time.
-__device__ __forceinline__ void topk_block(const float* __restrict__ score, int m, int k, int32_t* __restrict__ sel_idx,
-                                           int32_t* __restrict__ idx_out, uint32_t* s_bits) {
+__device__ __forceinline__ void topk_block(const float* score, int m, int k, int32_t* sel_idx,
+                                           int32_t* idx_out, uint32_t* s_bits) {
   __shared__ int hist[4][256];
   __shared__ int warp_sums_a[32], warp_sums_b[32];
   __shared__ int s_total_a, s_total_b;
@@ -204,8 +204,8 @@ __device__ __forceinline__ void topk_block(const float* __restrict__ score, int 
   }
 }
 
-__global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restrict__ score, int m, int k,
-                                                            int32_t* __restrict__ sel_idx, int32_t* __restrict__ idx_out,
+__global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* score, int m, int k,
+                                                            int32_t* sel_idx, int32_t* idx_out,
                                                             int use_smem) {
   extern __shared__ uint32_t s_bits_dyn[];          // [m] when use_smem
   pdl_trigger();
@@ -224,7 +224,7 @@ struct OptimizerArgs {
   float* exp_avg;
   float* exp_avg_sq;
 };
-__device__ __forceinline__ float optimizer_update(const OptimizerArgs& o, float d, const float* __restrict__ dB, int64_t e) {
+__device__ __forceinline__ float optimizer_update(const OptimizerArgs& o, float d, const float* dB, int64_t e) {
   if (o.kind == 1) return __fmaf_rn(o.neg_lr, dB[e], d);
   if (o.kind == 2) {
     const float g = dB[e];
@@ -242,11 +242,11 @@ __device__ __forceinline__ float optimizer_update(const OptimizerArgs& o, float 
 // ---- optimizer step + row scores + selection in ONE kernel: CTAs of 1024 threads take 128 rows each; the CTA
 // that finishes last (a counter in the workspace that is zero between calls) runs the selection on all scores.
 constexpr int kFusedScoreRows = 128;
-__global__ void __launch_bounds__(kTopkThreads) sgd_score_topk_kernel(float* __restrict__ dbuf, const float* __restrict__ dB,
+__global__ void __launch_bounds__(kTopkThreads) sgd_score_topk_kernel(float* dbuf, const float* dB,
                                                                       OptimizerArgs opt, int m, int r, int k,
-                                                                      float* __restrict__ score, int32_t* __restrict__ sel_idx,
-                                                                      int32_t* __restrict__ idx_out,
-                                                                      unsigned int* __restrict__ done_counter, int use_smem) {
+                                                                      float* score, int32_t* sel_idx,
+                                                                      int32_t* idx_out,
+                                                                      unsigned int* done_counter, int use_smem) {
   extern __shared__ float fused_smem[];  // [kFusedScoreRows][r + 1] floats, later the m staged scores
   __shared__ int s_last;
   pdl_trigger();
@@ -302,10 +302,10 @@ __device__ __forceinline__ void decode4(uint32_t w, float (&a)[4]) {
   a[0] = p0.x; a[1] = p0.y; a[2] = p1.x; a[3] = p1.y;
 }
 
-__global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __restrict__ wq, float* dbuf,
-                                                                   const int32_t* __restrict__ sel_idx, int k, int64_t m,
+__global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* wq, float* dbuf,
+                                                                   const int32_t* sel_idx, int k, int64_t m,
                                                                    int64_t n, int r, unsigned int* group_counters,
-                                                                   const float* __restrict__ row_scales) {
+                                                                   const float* row_scales) {
   extern __shared__ __align__(16) float merge_smem[];
   float* a_tile = merge_smem;                         // [r][kMergeCols] decoded A~
   float* sdb = merge_smem + (size_t)r * kMergeCols;   // [kMergeRows][r]
@@ -329,7 +329,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __re
       const int e = e0 + u * kMergeThreads;
       const int j = e / kVecPerRow, v = e % kVecPerRow;
       w[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (e < a_vecs && v * 16 < cta_cols) w[u] = __ldg(reinterpret_cast<const uint4*>(aq + (int64_t)j * n + v * 16));
+      if (e < a_vecs && v * 16 < cta_cols) w[u] = ld_stream(reinterpret_cast<const uint4*>(aq + (int64_t)j * n + v * 16));
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
@@ -359,7 +359,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __re
       if (e < d_vecs && q < nrows) {
         d[u] = *reinterpret_cast<const float4*>(dbuf + (int64_t)srow[q] * r + 4 * j4);
         if (row_scales != nullptr) {   // per-row mode: c_i = s_w[i] / s_w[m], applied as its own rounded multiply
-          const float c = __fdiv_rn(__ldg(row_scales + srow[q]), __ldg(row_scales + m));
+          const float c = __fdiv_rn(ld_stream(row_scales + srow[q]), ld_stream(row_scales + m));
           d[u].x = __fmul_rn(d[u].x, c); d[u].y = __fmul_rn(d[u].y, c);
           d[u].z = __fmul_rn(d[u].z, c); d[u].w = __fmul_rn(d[u].w, c);
         }
@@ -430,7 +430,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* __re
   }
 }
 
-__global__ void __launch_bounds__(256) zero_rows_kernel(float* __restrict__ dbuf, const int32_t* __restrict__ sel_idx,
+__global__ void __launch_bounds__(256) zero_rows_kernel(float* dbuf, const int32_t* sel_idx,
                                                         int k, int r) {
   pdl_trigger();
   pdl_wait();

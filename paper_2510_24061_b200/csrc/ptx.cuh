@@ -29,6 +29,13 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// Because a kernel may start (and its SM may cache lines) while the kernel before it is still writing, data that
+// another kernel of the stream produces must never be read through the non-coherent path (__ldg / LDG.NC, which
+// the compiler also picks for const __restrict__ pointers) nor be served from this SM's L1: every global load in
+// this library goes to L2 (ld.global.cg).  The whole library is additionally built with -Xptxas -dlcm=cg.
+template <typename T>
+__device__ __forceinline__ T ld_stream(const T* p) { return __ldcg(p); }
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");

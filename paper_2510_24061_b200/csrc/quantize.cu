@@ -26,7 +26,7 @@ template <int kDt>
 __device__ __forceinline__ void load16(const void* src, int64_t elem, float (&v)[16]) {
   if (kDt == kBF16) {
     const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(src) + elem);
-    uint4 a = __ldg(p), b = __ldg(p + 1);
+    uint4 a = ld_stream(p), b = ld_stream(p + 1);
     const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -37,7 +37,7 @@ __device__ __forceinline__ void load16(const void* src, int64_t elem, float (&v)
     const float4* p = reinterpret_cast<const float4*>(static_cast<const float*>(src) + elem);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      float4 f = __ldg(p + i);
+      float4 f = ld_stream(p + i);
       v[4 * i] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
     }
   }
@@ -86,8 +86,8 @@ __device__ __forceinline__ uint32_t block_max_u32(uint32_t v, uint32_t* smem /* 
 // ---- pass 1: max of |premul * x| per CTA, written to partial[blockIdx.x] (no atomics, nothing to
 // clear beforehand; the consumer takes the max over the gridDim.x partials)
 template <int kDt>
-__global__ void __launch_bounds__(kThreads) absmax_kernel(const void* __restrict__ src, int64_t count, float premul,
-                                                          bool use_premul, uint32_t* __restrict__ partial) {
+__global__ void __launch_bounds__(kThreads) absmax_kernel(const void* src, int64_t count, float premul,
+                                                          bool use_premul, uint32_t* partial) {
   __shared__ uint32_t red[32];
   pdl_trigger();
   pdl_wait();
@@ -118,9 +118,9 @@ struct CastOutputs {
   float* clear_word;   // nullable: set to 0 (the next kernel accumulates a max into it)
 };
 template <int kDt, int kFmt>
-__global__ void __launch_bounds__(kThreads) cast_kernel(const void* __restrict__ src, int64_t count, float premul,
-                                                        bool use_premul, const uint32_t* __restrict__ partial, int nparts,
-                                                        const float* __restrict__ scale_in, uint8_t* __restrict__ dst,
+__global__ void __launch_bounds__(kThreads) cast_kernel(const void* src, int64_t count, float premul,
+                                                        bool use_premul, const uint32_t* partial, int nparts,
+                                                        const float* scale_in, uint8_t* dst,
                                                         CastOutputs out) {
   __shared__ uint32_t red[32];
   pdl_trigger();
@@ -183,12 +183,12 @@ __device__ __forceinline__ RawVec<kDt> load_raw(const void* src, int64_t elem);
 template <>
 __device__ __forceinline__ RawVec<kBF16> load_raw<kBF16>(const void* src, int64_t elem) {
   const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(src) + elem);
-  RawVec<kBF16> r; r.a = __ldg(p); r.b = __ldg(p + 1); return r;
+  RawVec<kBF16> r; r.a = ld_stream(p); r.b = ld_stream(p + 1); return r;
 }
 template <>
 __device__ __forceinline__ RawVec<kF32> load_raw<kF32>(const void* src, int64_t elem) {
   const float4* p = reinterpret_cast<const float4*>(static_cast<const float*>(src) + elem);
-  RawVec<kF32> r; r.a = __ldg(p); r.b = __ldg(p + 1); r.c = __ldg(p + 2); r.d = __ldg(p + 3); return r;
+  RawVec<kF32> r; r.a = ld_stream(p); r.b = ld_stream(p + 1); r.c = ld_stream(p + 2); r.d = ld_stream(p + 3); return r;
 }
 __device__ __forceinline__ void unpack_raw(const RawVec<kBF16>& r, float (&v)[16]) {
   const uint32_t w[8] = {r.a.x, r.a.y, r.a.z, r.a.w, r.b.x, r.b.y, r.b.z, r.b.w};
@@ -205,12 +205,12 @@ __device__ __forceinline__ void unpack_raw(const RawVec<kF32>& r, float (&v)[16]
 
 // Multiplies the 16 values of one vector by the per-column factors col_mul[col .. col+15] (each its own
 // rounded multiply); a vector never straddles a row because the row length is a multiple of 16.
-__device__ __forceinline__ void apply_col_mul(float (&x)[16], const float* __restrict__ col_mul, int64_t elem, int cols) {
+__device__ __forceinline__ void apply_col_mul(float (&x)[16], const float* col_mul, int64_t elem, int cols) {
   const int col = static_cast<int>(elem % cols);
   const float4* p = reinterpret_cast<const float4*>(col_mul + col);
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const float4 f = __ldg(p + i);
+    const float4 f = ld_stream(p + i);
     x[4 * i] = __fmul_rn(x[4 * i], f.x); x[4 * i + 1] = __fmul_rn(x[4 * i + 1], f.y);
     x[4 * i + 2] = __fmul_rn(x[4 * i + 2], f.z); x[4 * i + 3] = __fmul_rn(x[4 * i + 3], f.w);
   }
@@ -219,11 +219,11 @@ __device__ __forceinline__ void apply_col_mul(float (&x)[16], const float* __res
 // kColMul: every column c of the [rows][cols] tensor is first multiplied by col_mul[c] (the output gradient
 // of a layer whose backbone rows carry their own scales: col_mul[c] = 1 / s_w[c]).
 template <int kDt, int kFmt, bool kColMul>
-__global__ void __launch_bounds__(kThreads) quantize_fused_kernel(const void* __restrict__ src, int64_t count,
-                                                                  uint8_t* __restrict__ dst, uint32_t* __restrict__ partial,
-                                                                  GridSync* __restrict__ sync, CastOutputs out,
-                                                                  int* __restrict__ status,
-                                                                  const float* __restrict__ col_mul, int cols) {
+__global__ void __launch_bounds__(kThreads) quantize_fused_kernel(const void* src, int64_t count,
+                                                                  uint8_t* dst, uint32_t* partial,
+                                                                  GridSync* sync, CastOutputs out,
+                                                                  int* status,
+                                                                  const float* col_mul, int cols) {
   constexpr int kCache = (kDt == kBF16) ? 4 : 2;
   __shared__ uint32_t red[32];
   __shared__ int s_ok;
@@ -325,8 +325,8 @@ __global__ void __launch_bounds__(kThreads) quantize_fused_kernel(const void* __
 // ---- per-row-scaled backbone: small tables derived from the row scales s_w[0..m] (s_w[m] = scale of the A~ block)
 //   mode 0: out[i] = 1 / s_w[i], i < m                      (column factors of dY before its E5M2 cast)
 //   mode 1: out[c] = 1 / (s_w[min(c, m)] * s_x), c < m + r  (column factors of the forward epilogue); zero beyond
-__global__ void __launch_bounds__(256) scale_table_kernel(int mode, const float* __restrict__ s_w, int m, int r,
-                                                          const float* __restrict__ s_x, float* __restrict__ out, int padded) {
+__global__ void __launch_bounds__(256) scale_table_kernel(int mode, const float* s_w, int m, int r,
+                                                          const float* s_x, float* out, int padded) {
   pdl_trigger();
   pdl_wait();
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
@@ -337,10 +337,10 @@ __global__ void __launch_bounds__(256) scale_table_kernel(int mode, const float*
 
 // ---- per-row scaling: one CTA per row, the row is read twice (second time from L1/L2)
 template <int kDt, int kFmt>
-__global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const void* __restrict__ src, int64_t cols, float premul,
-                                                                 bool use_premul, const float* __restrict__ scale_in,
-                                                                 uint8_t* __restrict__ dst, float* __restrict__ scale_out,
-                                                                 float* __restrict__ amax_out) {
+__global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const void* src, int64_t cols, float premul,
+                                                                 bool use_premul, const float* scale_in,
+                                                                 uint8_t* dst, float* scale_out,
+                                                                 float* amax_out) {
   __shared__ uint32_t red[32];
   pdl_trigger();
   pdl_wait();
@@ -375,11 +375,11 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const void* __r
 // A CTA converts 32 tokens x r: float4 loads along r, byte transposition through shared memory,
 // 16-byte stores along the tokens.
 constexpr int kOaTileT = 32;
-__global__ void __launch_bounds__(256) quantize_oa_transposed_kernel(const float* __restrict__ oa,
-                                                                     const float* __restrict__ amax_oa, int64_t T, int r,
-                                                                     int64_t ldt, uint8_t* __restrict__ oaq_t,
-                                                                     float* __restrict__ s_oa_out,
-                                                                     float* __restrict__ amax_copy) {
+__global__ void __launch_bounds__(256) quantize_oa_transposed_kernel(const float* oa,
+                                                                     const float* amax_oa, int64_t T, int r,
+                                                                     int64_t ldt, uint8_t* oaq_t,
+                                                                     float* s_oa_out,
+                                                                     float* amax_copy) {
   __shared__ __align__(16) uint8_t tile[256][kOaTileT + 16];
   pdl_trigger();
   pdl_wait();
@@ -398,7 +398,7 @@ __global__ void __launch_bounds__(256) quantize_oa_transposed_kernel(const float
     for (int tl = ty; tl < kOaTileT; tl += rows_per_pass) {
       uint32_t codes = 0;
       if (tl < tcount) {
-        const float4 x = __ldg(reinterpret_cast<const float4*>(oa + (t0 + tl) * r) + tx);
+        const float4 x = ld_stream(reinterpret_cast<const float4*>(oa + (t0 + tl) * r) + tx);
         codes = cvt_fp8x4<kE4M3>(__fmul_rn(x.x, s), __fmul_rn(x.y, s), __fmul_rn(x.z, s), __fmul_rn(x.w, s));
       }
       tile[4 * tx + 0][tl] = static_cast<uint8_t>(codes);
