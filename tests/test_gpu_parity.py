@@ -156,6 +156,13 @@ def test_per_row_scaled_backbone_all_stages(fq, orc, m, n, r, T, k):
     _run_layer_stages(fq, orc, 13, m, n, r, T, k, 1.0, 4, 2, 2e-2, per_row=True, heavy_tailed=True)
 
 
+@pytest.mark.parametrize("per_row", [False, True])
+def test_many_steps_keep_every_stage_fresh(fq, orc, per_row):
+    """Twenty-five steps with a new output gradient each: every kernel overlaps the launch of the next one, so a
+    stage that read anything stale (a scale, a slab, a score from the step before) would show up here."""
+    _run_layer_stages(fq, orc, 23, 640, 1280, 64, 300, 17, 1.0, 4, 25, 2e-2, per_row=per_row, heavy_tailed=per_row)
+
+
 def test_bf16_outputs_are_rounded_fp32_outputs(fq):
     c = synth.config0()
     W, A, B, X = layer_inputs(0, 0, c["m"], c["n"], c["r"], c["T"], c["n_outliers"])
