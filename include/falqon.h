@@ -18,7 +18,11 @@
  *    pitches); r must be a multiple of 8 with 8 <= r <= 256; T >= 1.
  *  - Execution: every call only enqueues work on `stream` and returns; results are
  *    ready once the stream has drained.  Calls that touch the same layer or the same
- *    workspace must be ordered on one stream.
+ *    workspace must be ordered on one stream.  A workspace must have been through
+ *    falqon_workspace_init once before its first use.  The kernels are launched with
+ *    programmatic stream serialization (each may be scheduled while its predecessor in
+ *    the stream still runs and waits on the device for it to finish); a caller's own
+ *    kernels placed between two calls are ordinary stream work and need nothing special.
  *  - Errors: the return value is a falqon_status.  Bad arguments are detected on the
  *    host before anything is launched (nothing is written).  CUDA launch failures map
  *    to FALQON_ERR_CUDA.  Every device-side wait is bounded; a wait that runs out
@@ -88,10 +92,11 @@ typedef enum {
  * most T_max tokens.  Returns 0 if the shape is not supported. */
 size_t falqon_workspace_bytes(int64_t m, int64_t n, int64_t r, int64_t T_max);
 
-/* Clears the control words at the start of a workspace (the counters of the in-kernel barriers; 1 KB).
- * Call it once after allocating a workspace, before the first falqon_melded_forward / _backward that uses it, and
- * again after a call reported FALQON_ERR_TIMEOUT.  The calls leave those words cleared, so a workspace that is
- * only ever passed to this library needs it once.  Enqueues a memset on `stream`. */
+/* Clears the control words at the start of a workspace (8 KB: the counters of the in-kernel grid barrier, of the
+ * "last CTA finishes the job" hand-overs and of the merge's row groups).  Call it once after allocating a
+ * workspace, before the first falqon_melded_forward / _backward / _proxy_update that uses it, and again after a
+ * call reported FALQON_ERR_TIMEOUT.  The calls leave those words cleared, so a workspace that is only ever passed
+ * to this library needs it once.  Enqueues a memset on `stream`. */
 int falqon_workspace_init(void *ws, size_t ws_bytes, falqon_stream stream);
 
 /* Host, pure.  Byte offset and size of a region inside a workspace laid out for (m, n, r, T_max).
