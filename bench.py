@@ -111,6 +111,19 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def aggregate_over_ranks(ms_local: float, flops_per_rank: float, dist=None, device=None):
+    """Replica aggregation: every rank runs its own batch; the job's time is the slowest rank's (max-reduce of the
+    device-timed milliseconds), the job's work is the sum over ranks.  Returns (ms, TFLOP/s of the whole job)."""
+    world = 1
+    ms = float(ms_local)
+    if dist is not None and dist.is_initialized():
+        world = dist.get_world_size()
+        t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms, world * flops_per_rank / (ms * 1e-3) / 1e12
+
+
 def build_workload(fq, device, seed, T, r, k, linears, outlier_frac):
     layers = []
     for idx, (name, n, m) in enumerate(linears):
@@ -314,11 +327,7 @@ def main():
         torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return aggregate_over_ranks(ms, 0.0, dist, device)[0]
 
     # ---- device-resident timing: EXACTLY --steps steps between two events, nothing else in the stream
     for _ in range(max(args.warmup, 3)):
