@@ -105,6 +105,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const void* tenso
       ::"r"(dst_smem), "l"(tensor_map), "r"(bar), "r"(x), "r"(y)
       : "memory");
 }
+// Untiled bulk copy global -> shared of `bytes` (a multiple of 16; both addresses 16-byte aligned), completing on
+// the mbarrier of the issuing CTA.
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
 __device__ __forceinline__ void prefetch_tensor_map(const void* tensor_map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tensor_map) : "memory");
 }

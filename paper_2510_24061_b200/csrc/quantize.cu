@@ -157,12 +157,8 @@ __global__ void __launch_bounds__(kThreads) cast_kernel(const void* src, int64_t
   }
 }
 
-// ---- fused per-tensor quantizer: absmax, a grid-wide barrier, then the cast, in ONE kernel.
-// All CTAs are co-resident (the host sizes the grid from the occupancy), so a CTA can wait for the others.
-// Each thread keeps the first kCache 16-element vectors it read in registers, so for tensors up to
-// grid x 256 x kCache x 16 elements the cast never touches memory again; what does not fit is re-read, most
-// recent first (that is what L2 still holds).  The barrier is two counters in the caller's workspace that
-// start at zero and are put back to zero by the last CTA to leave, and its wait is bounded.
+// The grid-wide barrier of the fused quantizer: two counters in the caller's workspace that start at zero and are
+// put back to zero by the last CTA to leave.
 struct GridSync {
   unsigned int arrive;
   unsigned int depart;
@@ -174,106 +170,126 @@ __device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
   return v;
 }
 
-template <int kDt> struct RawVec;
-template <> struct RawVec<kBF16> { uint4 a, b; };              // 16 bf16
-template <> struct RawVec<kF32> { float4 a, b, c, d; };        // 16 fp32
+// ---- fused per-tensor quantizer: absmax, a grid-wide barrier, then the cast, in ONE kernel, with the tensor held
+// in shared memory across the barrier.  All CTAs are co-resident (one per SM; the host sizes the grid from the
+// occupancy), so a CTA can wait for the others; the wait is bounded.  Each CTA streams its 16 KB chunks (chunk c belongs to CTA c mod grid)
+// through a ring of kStagedSlots bulk-copy targets, so up to 224 KB per SM are in flight or resident without
+// costing a register.  After the barrier the chunks still in the ring (the last kStagedSlots of the CTA) are cast
+// straight from shared memory; earlier ones are fetched again, most recent first (what L2 still holds), into the
+// slots as they free up.  Tensors up to 148 x 224 KB are read from memory exactly once.
+constexpr int kStagedThreads = 512;
+constexpr int kChunkBytes = 16384;
+constexpr int kStagedSlots = 14;
 
-template <int kDt>
-__device__ __forceinline__ RawVec<kDt> load_raw(const void* src, int64_t elem);
-template <>
-__device__ __forceinline__ RawVec<kBF16> load_raw<kBF16>(const void* src, int64_t elem) {
-  const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(src) + elem);
-  RawVec<kBF16> r; r.a = ld_stream(p); r.b = ld_stream(p + 1); return r;
-}
-template <>
-__device__ __forceinline__ RawVec<kF32> load_raw<kF32>(const void* src, int64_t elem) {
-  const float4* p = reinterpret_cast<const float4*>(static_cast<const float*>(src) + elem);
-  RawVec<kF32> r; r.a = ld_stream(p); r.b = ld_stream(p + 1); r.c = ld_stream(p + 2); r.d = ld_stream(p + 3); return r;
-}
-__device__ __forceinline__ void unpack_raw(const RawVec<kBF16>& r, float (&v)[16]) {
-  const uint32_t w[8] = {r.a.x, r.a.y, r.a.z, r.a.w, r.b.x, r.b.y, r.b.z, r.b.w};
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    v[2 * i] = __uint_as_float(w[i] << 16);
-    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-  }
-}
-__device__ __forceinline__ void unpack_raw(const RawVec<kF32>& r, float (&v)[16]) {
-  v[0] = r.a.x; v[1] = r.a.y; v[2] = r.a.z; v[3] = r.a.w; v[4] = r.b.x; v[5] = r.b.y; v[6] = r.b.z; v[7] = r.b.w;
-  v[8] = r.c.x; v[9] = r.c.y; v[10] = r.c.z; v[11] = r.c.w; v[12] = r.d.x; v[13] = r.d.y; v[14] = r.d.z; v[15] = r.d.w;
-}
+template <int kDt> struct Unit { static constexpr int kElems = kDt == kBF16 ? 8 : 4; };
 
-// Multiplies the 16 values of one vector by the per-column factors col_mul[col .. col+15] (each its own
-// rounded multiply); a vector never straddles a row because the row length is a multiple of 16.
-__device__ __forceinline__ void apply_col_mul(float (&x)[16], const float* col_mul, int64_t elem, int cols) {
-  const int col = static_cast<int>(elem % cols);
-  const float4* p = reinterpret_cast<const float4*>(col_mul + col);
+// The elements of one 16-byte unit as fp32, times their column factors when kColMul.
+template <int kDt, bool kColMul>
+__device__ __forceinline__ void unit_values(const uint4& q, const float* col_mul, int col, float (&x)[Unit<kDt>::kElems]) {
+  if (kDt == kBF16) {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float4 f = ld_stream(p + i);
-    x[4 * i] = __fmul_rn(x[4 * i], f.x); x[4 * i + 1] = __fmul_rn(x[4 * i + 1], f.y);
-    x[4 * i + 2] = __fmul_rn(x[4 * i + 2], f.z); x[4 * i + 3] = __fmul_rn(x[4 * i + 3], f.w);
+    for (int i = 0; i < 4; ++i) {
+      x[2 * i] = __uint_as_float(w[i] << 16);
+      x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  } else {
+    x[0] = __uint_as_float(q.x); x[1] = __uint_as_float(q.y); x[2] = __uint_as_float(q.z); x[3] = __uint_as_float(q.w);
   }
-}
-
-// kColMul: every column c of the [rows][cols] tensor is first multiplied by col_mul[c] (the output gradient
-// of a layer whose backbone rows carry their own scales: col_mul[c] = 1 / s_w[c]).
-template <int kDt, int kFmt, bool kColMul>
-__global__ void __launch_bounds__(kThreads) quantize_fused_kernel(const void* src, int64_t count,
-                                                                  uint8_t* dst, uint32_t* partial,
-                                                                  GridSync* sync, CastOutputs out,
-                                                                  int* status,
-                                                                  const float* col_mul, int cols) {
-  constexpr int kCache = (kDt == kBF16) ? 4 : 2;
-  __shared__ uint32_t red[32];
-  __shared__ int s_ok;
-  pdl_trigger();
-  pdl_wait();
-  const int64_t nvec = count / 16;
-  const int64_t stride = (int64_t)gridDim.x * kThreads;
-  const int64_t first = blockIdx.x * (int64_t)kThreads + threadIdx.x;
-  RawVec<kDt> cache[kCache];
-  uint32_t m = 0;
-  float x[16];
+  if (kColMul) {
+    const float4* f = reinterpret_cast<const float4*>(col_mul + col);
 #pragma unroll
-  for (int i = 0; i < kCache; ++i) {
-    const int64_t v = first + i * stride;
-    if (v < nvec) cache[i] = load_raw<kDt>(src, v * 16);
-  }
-#pragma unroll
-  for (int i = 0; i < kCache; ++i) {
-    const int64_t v = first + i * stride;
-    if (v < nvec) {
-      unpack_raw(cache[i], x);
-      if (kColMul) apply_col_mul(x, col_mul, v * 16, cols);
-#pragma unroll
-      for (int e = 0; e < 16; ++e) m = max(m, abs_bits(x[e]));
+    for (int i = 0; i < Unit<kDt>::kElems / 4; ++i) {
+      const float4 c = ld_stream(f + i);
+      x[4 * i] = __fmul_rn(x[4 * i], c.x); x[4 * i + 1] = __fmul_rn(x[4 * i + 1], c.y);
+      x[4 * i + 2] = __fmul_rn(x[4 * i + 2], c.z); x[4 * i + 3] = __fmul_rn(x[4 * i + 3], c.w);
     }
   }
-  int64_t v_last = first + (int64_t)(kCache - 1) * stride;   // last vector index visited by this thread
-  for (int64_t v = first + (int64_t)kCache * stride; v < nvec; v += stride) {
-    load16<kDt>(src, v * 16, x);
-    if (kColMul) apply_col_mul(x, col_mul, v * 16, cols);
-#pragma unroll
-    for (int e = 0; e < 16; ++e) m = max(m, abs_bits(x[e]));
-    v_last = v;
+}
+
+template <int kDt, int kFmt, bool kColMul>
+__global__ void __launch_bounds__(kStagedThreads, 1)
+quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* partial, GridSync* sync, CastOutputs out,
+                       int* status, const float* col_mul, int cols) {
+  constexpr int kEsize = kDt == kBF16 ? 2 : 4;
+  constexpr int kUnit = Unit<kDt>::kElems;
+  constexpr int64_t kChunkElems = kChunkBytes / kEsize;
+  extern __shared__ __align__(128) uint8_t stage[];
+  __shared__ __align__(8) uint64_t bars[kStagedSlots];
+  __shared__ uint32_t red[32];
+  __shared__ int s_ok;
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    for (int s = 0; s < kStagedSlots; ++s) mbar_init(smem_u32(&bars[s]), 1);
+    mbar_fence_init();
   }
-  if (blockIdx.x == 0) {  // ragged tail (count not a multiple of 16)
-    for (int64_t e = nvec * 16 + threadIdx.x; e < count; e += kThreads) m = max(m, abs_bits(load1<kDt>(src, e)));
+  pdl_trigger();
+  __syncthreads();
+  pdl_wait();
+
+  const int64_t bulk_elems = (count / 16) * 16;      // the rest (fewer than 16 elements) goes element by element
+  const int64_t n_chunks = (bulk_elems + kChunkElems - 1) / kChunkElems;
+  const int grid = static_cast<int>(gridDim.x);
+  const int n_my = blockIdx.x < n_chunks ? static_cast<int>((n_chunks - blockIdx.x + grid - 1) / grid) : 0;
+  auto chunk_of = [&](int i) -> int64_t { return blockIdx.x + static_cast<int64_t>(i) * grid; };
+  auto chunk_elems = [&](int64_t c) -> int {
+    const int64_t rem = bulk_elems - c * kChunkElems;
+    return static_cast<int>(rem < kChunkElems ? rem : kChunkElems);
+  };
+  auto issue = [&](int i) {   // one thread: fetch the CTA's i-th chunk into slot i mod kStagedSlots
+    const int s = i % kStagedSlots;
+    const int64_t c = chunk_of(i);
+    const uint32_t bytes = static_cast<uint32_t>(chunk_elems(c)) * kEsize;   // a multiple of 32
+    const uint32_t bar = smem_u32(&bars[s]);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier reads of the slot come first
+    mbar_expect_tx(bar, bytes);
+    bulk_load_1d(smem_u32(stage + s * kChunkBytes), static_cast<const uint8_t*>(src) + c * kChunkBytes, bytes, bar);
+  };
+
+  // ---- pass 1: absmax
+  if (tid == 0)
+    for (int i = 0; i < n_my && i < kStagedSlots; ++i) issue(i);
+  uint32_t phase_bits = 0;   // bit s: parity of the next completion of slot s
+  uint32_t m = 0;
+  bool failed = false;
+  for (int i = 0; i < n_my; ++i) {
+    const int s = i % kStagedSlots;
+    const bool ok = mbar_wait(smem_u32(&bars[s]), (phase_bits >> s) & 1u, status);
+    phase_bits ^= 1u << s;
+    const int64_t e0 = chunk_of(i) * kChunkElems;
+    const int units = chunk_elems(chunk_of(i)) / kUnit;
+    const uint4* sp = reinterpret_cast<const uint4*>(stage + s * kChunkBytes);
+    for (int u = tid; u < units; u += kStagedThreads) {
+      float x[kUnit];
+      unit_values<kDt, kColMul>(sp[u], col_mul, kColMul ? static_cast<int>((e0 + static_cast<int64_t>(u) * kUnit) % cols) : 0, x);
+#pragma unroll
+      for (int e = 0; e < kUnit; ++e) m = max(m, abs_bits(x[e]));
+    }
+    if (!__syncthreads_and(ok)) { failed = true; break; }   // block-uniform; also: the slot is free again
+    if (tid == 0 && i + kStagedSlots < n_my) issue(i + kStagedSlots);
+  }
+  if (blockIdx.x == 0) {   // ragged tail
+    for (int64_t e = bulk_elems + tid; e < count; e += kStagedThreads) {
+      float x = load1<kDt>(src, e);
+      if (kColMul) x = __fmul_rn(x, ld_stream(col_mul + static_cast<int>(e % cols)));
+      m = max(m, abs_bits(x));
+    }
   }
   m = block_max_u32(m, red);
-  // ---- grid barrier
-  if (threadIdx.x == 0) {
-    partial[blockIdx.x] = m;
-    __threadfence();
-    atomicAdd(&sync->arrive, 1u);
-    int ok = 1;
-    if (ld_acquire_gpu(&sync->arrive) < gridDim.x) {
-      const uint64_t t0 = global_timer_ns();
-      for (;;) {
-        if (ld_acquire_gpu(&sync->arrive) >= gridDim.x) break;
-        __nanosleep(40);
-        if (global_timer_ns() - t0 > kWaitLimitNs) { ok = 0; atomicExch(status, kStatusTimeout); break; }
+  // ---- grid barrier (a CTA that gave up above does not arrive: the others time out and report it)
+  if (tid == 0) {
+    int ok = failed ? 0 : 1;
+    if (ok) {
+      partial[blockIdx.x] = m;
+      __threadfence();
+      atomicAdd(&sync->arrive, 1u);
+      if (ld_acquire_gpu(&sync->arrive) < gridDim.x) {
+        const uint64_t t0 = global_timer_ns();
+        for (;;) {
+          if (ld_acquire_gpu(&sync->arrive) >= gridDim.x) break;
+          __nanosleep(40);
+          if (global_timer_ns() - t0 > kWaitLimitNs) { ok = 0; atomicExch(status, kStatusTimeout); break; }
+        }
       }
     }
     s_ok = ok;
@@ -281,38 +297,62 @@ __global__ void __launch_bounds__(kThreads) quantize_fused_kernel(const void* sr
   __syncthreads();
   if (s_ok) {
     uint32_t mb = 0;
-    for (int i = threadIdx.x; i < (int)gridDim.x; i += kThreads) mb = max(mb, __ldcg(partial + i));
+    for (int i = tid; i < grid; i += kStagedThreads) mb = max(mb, __ldcg(partial + i));
     const float amax = __uint_as_float(block_max_u32(mb, red));
-    const float s = scale_from_amax(amax, kFmt);
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-      if (out.scale_out) *out.scale_out = s;
-      if (out.scale_out2) *out.scale_out2 = s;
+    const float sc = scale_from_amax(amax, kFmt);
+    if (blockIdx.x == 0 && tid == 0) {
+      if (out.scale_out) *out.scale_out = sc;
+      if (out.scale_out2) *out.scale_out2 = sc;
       if (out.amax_out) *out.amax_out = amax;
       if (out.clear_word) *out.clear_word = 0.0f;
     }
-    // streamed part, most recent first
-    for (int64_t v = v_last; v >= first + (int64_t)kCache * stride; v -= stride) {
-      load16<kDt>(src, v * 16, x);
-      if (kColMul) apply_col_mul(x, col_mul, v * 16, cols);
-      reinterpret_cast<uint4*>(dst)[v] = cast16<kFmt>(x, 1.0f, false, s);
-    }
+    // ---- pass 2: cast, most recent chunk first
+    for (int t = 0; t < n_my; ++t) {
+      const int i = n_my - 1 - t;
+      const int s = i % kStagedSlots;
+      bool ok = true;
+      if (t >= kStagedSlots) {   // this chunk had left the ring and was fetched again
+        ok = mbar_wait(smem_u32(&bars[s]), (phase_bits >> s) & 1u, status);
+        phase_bits ^= 1u << s;
+      }
+      const int64_t e0 = chunk_of(i) * kChunkElems;
+      const int units = chunk_elems(chunk_of(i)) / kUnit;
+      const uint4* sp = reinterpret_cast<const uint4*>(stage + s * kChunkBytes);
+      for (int u = tid; u < units; u += kStagedThreads) {
+        float x[kUnit];
+        const int64_t e = e0 + static_cast<int64_t>(u) * kUnit;
+        unit_values<kDt, kColMul>(sp[u], col_mul, kColMul ? static_cast<int>(e % cols) : 0, x);
 #pragma unroll
-    for (int i = kCache - 1; i >= 0; --i) {
-      const int64_t v = first + i * stride;
-      if (v < nvec) {
-        unpack_raw(cache[i], x);
-        if (kColMul) apply_col_mul(x, col_mul, v * 16, cols);
-        reinterpret_cast<uint4*>(dst)[v] = cast16<kFmt>(x, 1.0f, false, s);
+        for (int k = 0; k < kUnit; ++k) x[k] = __fmul_rn(x[k], sc);
+        if (kDt == kBF16) {
+          uint2 o;
+          o.x = cvt_fp8x4<kFmt>(x[0], x[1], x[2], x[3]);
+          o.y = cvt_fp8x4<kFmt>(x[kUnit - 4], x[kUnit - 3], x[kUnit - 2], x[kUnit - 1]);
+          *reinterpret_cast<uint2*>(dst + e) = o;
+        } else {
+          *reinterpret_cast<uint32_t*>(dst + e) = cvt_fp8x4<kFmt>(x[0], x[1], x[2], x[3]);
+        }
+      }
+      if (t + kStagedSlots < n_my) {
+        if (!__syncthreads_and(ok)) { failed = true; break; }
+        if (tid == 0) issue(i - kStagedSlots);
       }
     }
     if (blockIdx.x == 0) {
-      for (int64_t e = nvec * 16 + threadIdx.x; e < count; e += kThreads)
-        dst[e] = static_cast<uint8_t>(cvt_fp8x2<kFmt>(__fmul_rn(load1<kDt>(src, e), s), 0.0f) & 0xFF);
+      for (int64_t e = bulk_elems + tid; e < count; e += kStagedThreads) {
+        float x = load1<kDt>(src, e);
+        if (kColMul) x = __fmul_rn(x, ld_stream(col_mul + static_cast<int>(e % cols)));
+        dst[e] = static_cast<uint8_t>(cvt_fp8x2<kFmt>(__fmul_rn(x, sc), 0.0f) & 0xFF);
+      }
     }
   }
   // ---- leave: the last CTA puts the counters back to zero for the next call
+  if (failed) {   // copies may still be in flight towards this CTA's shared memory: give them time to land
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 200000ull) { }
+  }
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (tid == 0 && !failed) {
     const unsigned int prev = atomicAdd(&sync->depart, 1u);
     if (prev == gridDim.x - 1) {
       sync->arrive = 0u;
@@ -454,24 +494,30 @@ cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, i
 }
 
 template <int kDt, int kFmt, bool kColMul>
-cudaError_t launch_fused_variant(const void* src, int64_t count, uint8_t* dst, uint32_t* partial, void* sync,
-                                 const CastOutputs& out, int* status, const float* col_mul, int cols, cudaStream_t stream) {
+cudaError_t launch_staged_variant(const void* src, int64_t count, uint8_t* dst, uint32_t* partial, void* sync,
+                                  const CastOutputs& out, int* status, const float* col_mul, int cols, cudaStream_t stream) {
+  constexpr size_t kSmem = static_cast<size_t>(kStagedSlots) * kChunkBytes;
   static int blocks_per_sm = 0;
   if (blocks_per_sm == 0) {
-    int b = 0;
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, quantize_fused_kernel<kDt, kFmt, kColMul>, kThreads, 0);
+    cudaError_t e = cudaFuncSetAttribute(quantize_staged_kernel<kDt, kFmt, kColMul>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmem));
     if (e != cudaSuccess) return e;
-    blocks_per_sm = b < 1 ? 1 : b;
+    int b = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, quantize_staged_kernel<kDt, kFmt, kColMul>, kStagedThreads, kSmem);
+    if (e != cudaSuccess) return e;
+    if (b < 1) return cudaErrorLaunchOutOfResources;
+    blocks_per_sm = b;
   }
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  int64_t grid = (count / 16 + kThreads - 1) / kThreads;
-  const int64_t resident = static_cast<int64_t>(blocks_per_sm) * sms;
+  const int64_t chunk_elems = kChunkBytes / (kDt == kBF16 ? 2 : 4);
+  int64_t grid = (count / 16 * 16 + chunk_elems - 1) / chunk_elems;
+  const int64_t resident = static_cast<int64_t>(blocks_per_sm) * sms;   // all CTAs must be resident together
   if (grid > resident) grid = resident;
   if (grid > kMaxAbsmaxParts) grid = kMaxAbsmaxParts;
   if (grid < 1) grid = 1;
-  return launch_pdl(quantize_fused_kernel<kDt, kFmt, kColMul>, dim3(static_cast<unsigned>(grid)), dim3(kThreads), 0, stream,
-                    1, src, count, dst, partial, static_cast<GridSync*>(sync), out, status, col_mul, cols);
+  return launch_pdl(quantize_staged_kernel<kDt, kFmt, kColMul>, dim3(static_cast<unsigned>(grid)), dim3(kStagedThreads), kSmem,
+                    stream, 1, src, count, dst, partial, static_cast<GridSync*>(sync), out, status, col_mul, cols);
 }
 
 cudaError_t launch_quantize_fused(const void* src, int src_dt, int64_t count, int fmt, uint8_t* dst, uint32_t* partial,
@@ -481,8 +527,8 @@ cudaError_t launch_quantize_fused(const void* src, int src_dt, int64_t count, in
 #define FALQON_FUSED(DT, FMT)                                                                                              \
   do {                                                                                                                     \
     if (col_mul != nullptr)                                                                                                \
-      return launch_fused_variant<DT, FMT, true>(src, count, dst, partial, sync, out, status, col_mul, cols, stream);       \
-    return launch_fused_variant<DT, FMT, false>(src, count, dst, partial, sync, out, status, nullptr, 0, stream);           \
+      return launch_staged_variant<DT, FMT, true>(src, count, dst, partial, sync, out, status, col_mul, cols, stream);     \
+    return launch_staged_variant<DT, FMT, false>(src, count, dst, partial, sync, out, status, nullptr, 0, stream);         \
   } while (0)
   if (src_dt == kBF16) {
     if (fmt == kE4M3) FALQON_FUSED(kBF16, kE4M3);

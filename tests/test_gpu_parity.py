@@ -156,6 +156,46 @@ def test_per_row_scaled_backbone_all_stages(fq, orc, m, n, r, T, k):
     _run_layer_stages(fq, orc, 13, m, n, r, T, k, 1.0, 4, 2, 2e-2, per_row=True, heavy_tailed=True)
 
 
+@pytest.mark.parametrize("m,n,r,T,k", [(3840, 1024, 64, 1280, 64), (1024, 3872, 64, 1200, 16)])
+def test_more_tiles_than_cta_pairs_all_stages(fq, orc, m, n, r, T, k):
+    """80 output tiles for 74 CTA pairs, element by element: the forward product (first shape) and the
+    input-gradient product (second shape, with a ragged last tile row and column) give some pairs two tiles."""
+    _run_layer_stages(fq, orc, 29, m, n, r, T, k, 1.0, 3, 2, 2e-2)
+
+
+@pytest.mark.parametrize("per_row", [False, True])
+def test_fp32_inputs_larger_than_the_staging_ring(fq, orc, per_row):
+    """fp32 activations and output gradients of 49 MB each: more than the fused quantizer keeps on chip, so part
+    of the tensor is fetched a second time for the cast; the last 16 KB chunk is partial.  Codes and scales
+    must match bit for bit (per-row mode: the gradient is divided by the row scales before its cast)."""
+    T, big, small, r = 3001, 4112, 128, 16
+    # forward: X is [T][big]
+    W, A, B, _ = layer_inputs(31, 0, small, big, r, 16, 0)
+    layer = fq.setup_layer(W.to(DEV), A.to(DEV), B.to(DEV), 1.0, per_row=per_row)
+    X = synth.normal_bf16(31, 7, (T, big), 1.0).float() * 1.0009765625 + 3.0e-4   # not bf16-representable
+    ws = layer.workspace(T)
+    _, _, _, s_x = fq.melded_forward(layer, X.to(DEV), y_dtype=torch.float32, ws=ws)
+    xq_o, s_x_o, _ = orc.quantize(f32(X), orc.E4M3)
+    assert bits32(f32(s_x))[0] == bits32(s_x_o)
+    assert np.array_equal(u8(fq.ws_view(layer, ws, T, fq.WS_XQ)).reshape(T, big), xq_o)
+    # backward: dY is [T][big]
+    W, A, B, X2 = layer_inputs(32, 0, big, small, r, T, 0)
+    if per_row:
+        W = synth.backbone(32, 0, big, small, heavy_tailed=True)
+    layer = fq.setup_layer(W.to(DEV), A.to(DEV), B.to(DEV), 1.0, per_row=per_row)
+    ws = layer.workspace(T)
+    _, OA, amax_oa, _ = fq.melded_forward(layer, X2.to(DEV), y_dtype=torch.float32, ws=ws)
+    dY = synth.normal_bf16(32, 9, (T, big), 1.0e-3).float() * 0.99951171875 - 1.0e-7
+    _, _, s_g = fq.melded_backward(layer, dY.to(DEV), OA, amax_oa, dx_dtype=torch.float32, ws=ws)
+    if per_row:
+        gq_o, s_g_o, _ = orc.quantize_colscaled(f32(dY), orc.E5M2, f32(layer.s_w)[:big])
+    else:
+        gq_o, s_g_o, _ = orc.quantize(f32(dY), orc.E5M2)
+    assert bits32(f32(s_g))[0] == bits32(s_g_o)
+    assert np.array_equal(u8(fq.ws_view(layer, ws, T, fq.WS_GQ)).reshape(T, big), gq_o)
+    assert fq.last_device_status() == 0
+
+
 @pytest.mark.parametrize("per_row", [False, True])
 def test_many_steps_keep_every_stage_fresh(fq, orc, per_row):
     """Twenty-five steps with a new output gradient each: every kernel overlaps the launch of the next one, so a
