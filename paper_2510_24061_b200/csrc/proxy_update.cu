@@ -208,8 +208,8 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* score, 
                                                             int32_t* sel_idx, int32_t* idx_out,
                                                             int use_smem) {
   extern __shared__ uint32_t s_bits_dyn[];          // [m] when use_smem
+  pdl_wait();      // before the trigger, for the sake of the merge that follows (it reads A~ ahead of its wait)
   pdl_trigger();
-  pdl_wait();
   topk_block(score, m, k, sel_idx, idx_out, use_smem ? s_bits_dyn : nullptr);
 }
 
@@ -224,16 +224,15 @@ struct OptimizerArgs {
   float* exp_avg;
   float* exp_avg_sq;
 };
-__device__ __forceinline__ float optimizer_update(const OptimizerArgs& o, float d, const float* dB, int64_t e) {
-  if (o.kind == 1) return __fmaf_rn(o.neg_lr, dB[e], d);
+__device__ __forceinline__ float optimizer_update(const OptimizerArgs& o, float d, float g, float& ea, float& es) {
+  if (o.kind == 1) return __fmaf_rn(o.neg_lr, g, d);
   if (o.kind == 2) {
-    const float g = dB[e];
     const float p1 = __fmul_rn(d, o.decay);
-    const float m1 = __fmaf_rn(o.beta1, o.exp_avg[e], __fmul_rn(o.one_minus_b1, g));
-    const float v1 = __fmaf_rn(o.beta2, o.exp_avg_sq[e], __fmul_rn(o.one_minus_b2, __fmul_rn(g, g)));
+    const float m1 = __fmaf_rn(o.beta1, ea, __fmul_rn(o.one_minus_b1, g));
+    const float v1 = __fmaf_rn(o.beta2, es, __fmul_rn(o.one_minus_b2, __fmul_rn(g, g)));
     const float denom = __fadd_rn(__fdiv_rn(__fsqrt_rn(v1), o.sqrt_bc2), o.eps);
-    o.exp_avg[e] = m1;
-    o.exp_avg_sq[e] = v1;
+    ea = m1;
+    es = v1;
     return __fmaf_rn(o.neg_step_size, __fdiv_rn(m1, denom), p1);
   }
   return d;
@@ -249,19 +248,41 @@ __global__ void __launch_bounds__(kTopkThreads) sgd_score_topk_kernel(float* dbu
                                                                       unsigned int* done_counter, int use_smem) {
   extern __shared__ float fused_smem[];  // [kFusedScoreRows][r + 1] floats, later the m staged scores
   __shared__ int s_last;
-  pdl_trigger();
+  // The wait comes first: the merge that follows reads the A~ rows before its own wait, which is only safe
+  // once every earlier kernel on the stream has finished, i.e. once this kernel is past this point.
   pdl_wait();
+  pdl_trigger();
   const int row0 = blockIdx.x * kFusedScoreRows;
   const int rows = min(kFusedScoreRows, m - row0);
   const int64_t base = (int64_t)row0 * r;
-  for (int e = threadIdx.x; e < rows * r; e += blockDim.x) {
-    float d = dbuf[base + e];
-    if (opt.kind != 0) {
-      d = optimizer_update(opt, d, dB, base + e);
-      dbuf[base + e] = d;
+  const int total = rows * r;
+  constexpr int kBatch = 4;   // loads of four elements per thread are in flight together
+  for (int e0 = threadIdx.x; e0 < total; e0 += kBatch * blockDim.x) {
+    float d[kBatch], g[kBatch], ea[kBatch], es[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int e = e0 + u * blockDim.x;
+      d[u] = 0.0f; g[u] = 0.0f; ea[u] = 0.0f; es[u] = 0.0f;
+      if (e < total) {
+        d[u] = ld_stream(dbuf + base + e);
+        if (opt.kind != 0) g[u] = ld_stream(dB + base + e);
+        if (opt.kind == 2) { ea[u] = ld_stream(opt.exp_avg + base + e); es[u] = ld_stream(opt.exp_avg_sq + base + e); }
+      }
     }
-    const int i = e / r, j = e - i * r;
-    fused_smem[i * (r + 1) + j] = fabsf(d);
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int e = e0 + u * blockDim.x;
+      if (e < total) {
+        float v = d[u];
+        if (opt.kind != 0) {
+          v = optimizer_update(opt, v, g[u], ea[u], es[u]);
+          dbuf[base + e] = v;
+          if (opt.kind == 2) { opt.exp_avg[base + e] = ea[u]; opt.exp_avg_sq[base + e] = es[u]; }
+        }
+        const int i = e / r, j = e - i * r;
+        fused_smem[i * (r + 1) + j] = fabsf(v);
+      }
+    }
   }
   __syncthreads();
   if (threadIdx.x < rows) {
@@ -311,12 +332,13 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* wq, 
   float* sdb = merge_smem + (size_t)r * kMergeCols;   // [kMergeRows][r]
   __shared__ int srow[kMergeRows];
   pdl_trigger();
-  pdl_wait();
   const int g0 = blockIdx.y * kMergeRows;
   const int nrows = min(kMergeRows, k - g0);
   const int64_t cta_c0 = (int64_t)blockIdx.x * kMergeCols;
   const int cta_cols = static_cast<int>(min((int64_t)kMergeCols, n - cta_c0));   // multiple of 16
-  if (threadIdx.x < kMergeRows) srow[threadIdx.x] = (threadIdx.x < nrows) ? sel_idx[g0 + threadIdx.x] : -1;
+  // The A~ rows are decoded BEFORE the wait, while the selection kernel is still running: nothing on the proxy
+  // update's path writes them, and the kernel launched before this one (the selection) releases this launch
+  // only after its own wait, i.e. after everything earlier on the stream (a set-up cast of A~, say) is done.
   // decode A~ (rows m.. of W~') into shared memory; columns beyond the matrix edge become 0.  The loads of
   // four iterations are issued together so that their latencies overlap.
   const uint8_t* aq = wq + m * n + cta_c0;
@@ -345,7 +367,9 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* wq, 
       }
     }
   }
-  __syncthreads();   // srow visible
+  pdl_wait();
+  if (threadIdx.x < kMergeRows) srow[threadIdx.x] = (threadIdx.x < nrows) ? ld_stream(sel_idx + g0 + threadIdx.x) : -1;
+  __syncthreads();   // srow and the A~ tile visible
   // the DeltaBuffer rows of this CTA, as float4 (r is a multiple of 8), four loads in flight per thread
   const int r4 = r >> 2;
   const int d_vecs = kMergeRows * r4;
