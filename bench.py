@@ -415,8 +415,9 @@ def main():
     ms_e2e = max_over_ranks(ev0.elapsed_time(ev1)) / e2e_steps
     e2e_value = world * flops_step / (ms_e2e * 1e-3) / 1e12
 
-    launches_per_step = sum(fq.launch_count("falqon_melded_forward") + fq.launch_count("falqon_melded_backward") +
-                            fq.launch_count("falqon_proxy_update", k=k) for _ in layers)
+    launches_per_step = sum(fq.launch_count("falqon_melded_forward") +
+                            fq.launch_count("falqon_melded_backward") +
+                            fq.launch_count("falqon_proxy_update", k=k) for L in layers)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()

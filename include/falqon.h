@@ -84,8 +84,7 @@ typedef enum {
   FALQON_WS_OAQ_T = 2,    /* uint8 [r16][T16] E4M3 codes of O_A, TRANSPOSED; r16 = r rounded up
                              to 16, row pitch T16 = T rounded up to 16 (after backward)          */
   FALQON_WS_SCALES = 3,   /* float [8]: 0 amax(X) 1 s_x 2 amax(dY) 3 s_g 4 amax(O_A) 5 s_OA      */
-  FALQON_WS_SCORE = 4,    /* float [m] row scores sum_j |DeltaBuffer[i][j]| (after proxy update)  */
-  FALQON_WS_DB_PART = 5   /* float [splits][m][r] split partial sums of dB (after backward)      */
+  FALQON_WS_SCORE = 4     /* float [m] row scores sum_j |DeltaBuffer[i][j]| (after proxy update)  */
 } falqon_ws_region;
 
 /* Host, pure.  Bytes of workspace that the calls below need for a layer of this shape with at
@@ -202,13 +201,13 @@ int falqon_last_device_status(falqon_stream stream);
 typedef enum {
   FALQON_STAGE_QUANT_X = 0,   /* absmax + cast of X            (S1) */
   FALQON_STAGE_GEMM_FWD = 1,  /* melded forward product        (S2) */
-  FALQON_STAGE_QUANT_DY = 2,  /* absmax + cast of dY           (S3) */
-  FALQON_STAGE_QUANT_OA = 3,  /* cast of O_A                   (S5a) */
+  FALQON_STAGE_QUANT_DY = 2,  /* absmax + cast of dY, with the cast of O_A riding along (S3, S5a) */
+  FALQON_STAGE_QUANT_OA = 3,  /* unused: the cast of O_A runs inside stage 2 */
   FALQON_STAGE_GEMM_DX = 4,   /* input-gradient product        (S4) */
-  FALQON_STAGE_GEMM_DB = 5,   /* adapter-gradient product      (S5b) */
-  FALQON_STAGE_REDUCE_DB = 6, /* fixed-order sum of its slabs  (S5b) */
-  FALQON_STAGE_SGD_SCORE = 7, /* optimizer step + row scores   (S6, S7) */
-  FALQON_STAGE_TOPK = 8,      /* row selection                 (S7) */
+  FALQON_STAGE_GEMM_DB = 5,   /* adapter-gradient product with the slab sum (S5b) */
+  FALQON_STAGE_REDUCE_DB = 6, /* unused: the slab sum runs inside stage 5 */
+  FALQON_STAGE_SGD_SCORE = 7, /* optimizer step, row scores and row selection (S6, S7) */
+  FALQON_STAGE_TOPK = 8,      /* row selection when it runs as its own kernel (falqon_proxy_update_static) */
   FALQON_STAGE_MERGE = 9      /* merge + requantize + clear    (S8) */
 } falqon_stage;
 

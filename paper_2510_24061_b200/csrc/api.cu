@@ -24,11 +24,10 @@ int* status_ptr() {
 }
 
 struct WorkspaceLayout {
-  size_t scales, act8, oaq_t, db_part, score, sel_idx, inv_sw, col_scale, total;
-  size_t act8_bytes, oaq_t_bytes, db_part_bytes, score_bytes, sel_idx_bytes, inv_sw_bytes, col_scale_bytes;
+  size_t scales, act8, oaq_t, score, sel_idx, inv_sw, col_scale, total;
+  size_t act8_bytes, oaq_t_bytes, score_bytes, sel_idx_bytes, inv_sw_bytes, col_scale_bytes;
   int64_t inv_sw_len, col_scale_len;   // table lengths, padded to a multiple of 32 (+32) so vector reads stay inside
   int64_t r16, t16;
-  int splits;
 };
 
 constexpr size_t kHeaderBytes = 8192;     // scales at 0, absmax partials at kPartialsOffset
@@ -49,10 +48,8 @@ bool make_layout(int64_t m, int64_t n, int64_t r, int64_t T, WorkspaceLayout* w)
   if (!shape_ok(m, n, r) || T < 1 || T >= (1ll << 30)) return false;
   w->r16 = round_up(r, 16);
   w->t16 = round_up(T, 16);
-  w->splits = gemm_k_splits_for_db(m, T);
   w->act8_bytes = static_cast<size_t>(T) * static_cast<size_t>(m > n ? m : n);
   w->oaq_t_bytes = static_cast<size_t>(w->r16) * static_cast<size_t>(w->t16);
-  w->db_part_bytes = static_cast<size_t>(w->splits) * m * r * sizeof(float);
   w->score_bytes = static_cast<size_t>(m) * sizeof(float);
   w->sel_idx_bytes = static_cast<size_t>(m) * sizeof(int32_t);
   w->inv_sw_len = round_up(m, 32) + 32;
@@ -67,7 +64,6 @@ bool make_layout(int64_t m, int64_t n, int64_t r, int64_t T, WorkspaceLayout* w)
   w->col_scale = off; off += round_up(w->col_scale_bytes, 1024);  // per-row mode: 1/(s_w[c] s_x)
   w->act8 = off; off += round_up(w->act8_bytes, 1024);
   w->oaq_t = off; off += round_up(w->oaq_t_bytes, 1024);
-  w->db_part = off; off += round_up(w->db_part_bytes, 1024);
   w->total = off;
   return true;
 }
@@ -135,7 +131,6 @@ int falqon_workspace_region(int64_t m, int64_t n, int64_t r, int64_t T_max, falq
     case FALQON_WS_OAQ_T: *offset = w.oaq_t; *bytes = w.oaq_t_bytes; break;
     case FALQON_WS_SCALES: *offset = w.scales; *bytes = 8 * sizeof(float); break;
     case FALQON_WS_SCORE: *offset = w.score; *bytes = w.score_bytes; break;
-    case FALQON_WS_DB_PART: *offset = w.db_part; *bytes = w.db_part_bytes; break;
     default: return FALQON_ERR_INVALID_ARG;
   }
   return FALQON_OK;
@@ -203,7 +198,7 @@ int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_d
   {
     StageTimer timer(FALQON_STAGE_QUANT_X, stream);
     FALQON_CUDA(launch_quantize_fused(X, x_dt, T * n, kE4M3, xq, partial, base + w.scales + kSyncOffset, scales + 1, s_x_out,
-                                      scales + 0, amax_oa, status, nullptr, 0, stream));
+                                      scales + 0, amax_oa, status, nullptr, 0, nullptr, stream));
   }
   const bool per_row = L->gran == FALQON_PER_ROW;
   float* col_scale = reinterpret_cast<float*>(base + w.col_scale);
@@ -212,10 +207,10 @@ int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_d
   // S2: [Y | O_A] = x~ W~'^T / (s_W s_x), amax(O_A) from the epilogue
   GemmProblem g{};
   g.M = T; g.N = m + r; g.K = n;
-  g.a = xq; g.lda = n; g.a_mn_major = false; g.a_fmt = kE4M3;
+  g.a = xq; g.lda = n; g.a_fmt = kE4M3;
   g.b = L->wq; g.ldb = n; g.b_mn_major = false; g.b_fmt = kE4M3;
-  g.block_n = 256; g.k_splits = 1;
-  g.c0 = Y; g.ldc0 = m; g.c0_dt = y_dt; g.n_split = m; g.c0_split_stride = 0;
+  g.block_n = 256;
+  g.c0 = Y; g.ldc0 = m; g.c0_dt = y_dt; g.n_split = m;
   g.c1 = OA; g.ldc1 = r; g.amax1_bits = reinterpret_cast<uint32_t*>(amax_oa);
   g.scale_a = per_row ? nullptr : scales + 1; g.scale_b = per_row ? nullptr : L->s_w;
   g.col_scale = per_row ? col_scale : nullptr;
@@ -242,7 +237,6 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
   float* scales = reinterpret_cast<float*>(base + w.scales);
   uint8_t* gq = base + w.act8;
   uint8_t* oaq_t = base + w.oaq_t;
-  float* part = reinterpret_cast<float*>(base + w.db_part);
   const int64_t m = L->m, n = L->n, r = L->r;
 
   // S3: g~, s_g = Q_e5m2(dY)
@@ -253,46 +247,36 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
     FALQON_CUDA(launch_scale_table(0, L->s_w, m, r, nullptr, inv_sw, w.inv_sw_len, stream));
   {
     StageTimer timer(FALQON_STAGE_QUANT_DY, stream);
+    // S5a rides along: O~_A = Q_e4m3(O_A) with s_OA from the forward's amax, written transposed for the dB product
+    const OaCastJob oa_cast{OA, amax_oa, T, static_cast<int>(r), w.t16, oaq_t, scales + 5, scales + 4};
     FALQON_CUDA(launch_quantize_fused(dY, dy_dt, T * m, kE5M2, gq, partial, base + w.scales + kSyncOffset, scales + 3, s_g_out,
-                                      scales + 2, nullptr, status, per_row ? inv_sw : nullptr, static_cast<int>(m), stream));
+                                      scales + 2, nullptr, status, per_row ? inv_sw : nullptr, static_cast<int>(m), &oa_cast,
+                                      stream));
   }
-  // S5a: O~_A, s_OA = Q_e4m3(O_A), written transposed for the dB product
+  // S5b: dB = g~^T O~_A / (s_g s_OA) over token slabs, slab sum in slab order across a thread-block cluster.  It runs
+  // before S4 (neither needs the other): g~ was written a moment ago and is still in L2.
   {
-    StageTimer timer(FALQON_STAGE_QUANT_OA, stream);
-    FALQON_CUDA(launch_quantize_oa_transposed(OA, amax_oa, T, r, w.r16, w.t16, oaq_t, scales + 5, scales + 4, stream));
+    DbFusedProblem d{};
+    d.m = m; d.r = r; d.T = T;
+    d.gq = gq; d.oaq_t = oaq_t; d.ldt = w.t16; d.s_oa = scales + 5;
+    d.s_g = scales + 3; d.row_mul = per_row ? L->s_w : nullptr; d.dB = dB; d.status = status;
+    StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
+    FALQON_CUDA(launch_db_fused(d, stream));
   }
   // S4: dX = g~ W~ / (s_W s_g)   (contraction over the m output channels; W~ read MN-major)
   if (dX != nullptr) {
     GemmProblem g{};
     g.M = T; g.N = n; g.K = m;
-    g.a = gq; g.lda = m; g.a_mn_major = false; g.a_fmt = kE5M2;
+    g.a = gq; g.lda = m; g.a_fmt = kE5M2;
     g.b = L->wq; g.ldb = n; g.b_mn_major = true; g.b_fmt = kE4M3;
-    g.block_n = 256; g.k_splits = 1;
-    g.c0 = dX; g.ldc0 = n; g.c0_dt = dx_dt; g.n_split = n; g.c0_split_stride = 0;
+    g.block_n = 256;
+    g.c0 = dX; g.ldc0 = n; g.c0_dt = dx_dt; g.n_split = n;
     g.c1 = nullptr; g.ldc1 = 0; g.amax1_bits = nullptr;
     g.scale_a = scales + 3; g.scale_b = per_row ? nullptr : L->s_w;
     g.col_scale = nullptr;
     g.status = status;
     StageTimer timer(FALQON_STAGE_GEMM_DX, stream);
     FALQON_CUDA(launch_gemm_fp8(g, stream));
-  }
-  // S5b: dB = g~^T O~_A / (s_g s_OA)   (contraction over tokens, split into slabs, fixed-order reduce)
-  {
-    GemmProblem g{};
-    g.M = m; g.N = r; g.K = T;
-    g.a = gq; g.lda = m; g.a_mn_major = true; g.a_fmt = kE5M2;
-    g.b = oaq_t; g.ldb = w.t16; g.b_mn_major = false; g.b_fmt = kE4M3;
-    g.block_n = static_cast<int>(w.r16); g.k_splits = w.splits;
-    g.c0 = part; g.ldc0 = r; g.c0_dt = kF32; g.n_split = r; g.c0_split_stride = m * r;
-    g.c1 = nullptr; g.ldc1 = 0; g.amax1_bits = nullptr;
-    g.scale_a = nullptr; g.scale_b = nullptr; g.col_scale = nullptr;
-    g.status = status;
-    {
-      StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
-      FALQON_CUDA(launch_gemm_fp8(g, stream));
-    }
-    StageTimer timer(FALQON_STAGE_REDUCE_DB, stream);
-    FALQON_CUDA(launch_reduce_db(part, w.splits, m * r, scales + 3, scales + 5, per_row ? L->s_w : nullptr, r, dB, stream));
   }
   return FALQON_OK;
 }
@@ -411,7 +395,7 @@ int falqon_launch_count(const char* entry_point, int64_t m, int64_t n, int64_t r
   if (entry_point == nullptr) return 0;
   if (std::strcmp(entry_point, "falqon_quantize") == 0) return 2;           // absmax, cast
   if (std::strcmp(entry_point, "falqon_melded_forward") == 0) return 2;     // fused quantize, GEMM
-  if (std::strcmp(entry_point, "falqon_melded_backward") == 0) return 5;    // fused quantize, O_A cast, dX, dB, reduce
+  if (std::strcmp(entry_point, "falqon_melded_backward") == 0) return 3;    // fused quantize, dX, fused dB
   if (std::strcmp(entry_point, "falqon_proxy_update") == 0) return k > 0 ? 2 : 1;  // optimizer+score+top-k, merge+clear
   return 0;
 }

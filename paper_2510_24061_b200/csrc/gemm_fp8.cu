@@ -8,9 +8,9 @@
 //   warp 1      allocates TMEM; one lane issues the MMAs and commits them to the barriers
 //   warps 2..9  epilogue: tcgen05.ld the accumulator, rescale by 1/(s_a*s_b), store
 // The accumulator is double buffered (2 x 256 TMEM columns), so the epilogue of tile i overlaps the
-// main loop of tile i+1.  Either operand may be K-major (rows along K) or MN-major (rows along M/N):
-// the melded forward reads both K-major, the input gradient reads W~ MN-major (no transposed copy of
-// the backbone exists), the adapter gradient reads the output gradient MN-major.
+// main loop of tile i+1.  A is K-major (rows along K); B may be K-major or MN-major (rows along N): the
+// melded forward reads both K-major, the input gradient reads W~ MN-major (no transposed copy of the
+// backbone exists).  (The adapter gradient, which reads the output gradient MN-major, has its own kernel.)
 // Every mbarrier wait is bounded; on a timeout the CTA records it, drains and frees its TMEM.
 #include <cuda.h>
 
@@ -39,13 +39,13 @@ constexpr uint32_t kStagingBytes = kEpilogueWarps * kStageOutBytes;  // 32 KB be
 
 struct GemmParams {
   int M, N, K;
-  int m_tiles, n_tiles, k_splits;
-  int kblocks_total, kblocks_per_split;
+  int m_tiles, n_tiles;
+  int kblocks_total;
   int block_n;
   int num_stages;
   uint32_t idesc;
   // epilogue
-  void* c0; long long ldc0; int c0_dt; int n_split; long long c0_split_stride;
+  void* c0; long long ldc0; int c0_dt; int n_split;
   float* c1; long long ldc1; uint32_t* amax1_bits;
   const float* scale_a; const float* scale_b;
   const float* col_scale;
@@ -60,11 +60,11 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 // Stores 32 consecutive output columns [col0, col0+32) of one row: columns below n_split go to c0 (bf16 or
 // fp32, 16-byte stores when aligned), the rest up to N go to c1 (fp32) and feed the running |max|.
-__device__ __forceinline__ void epilogue_store32(const GemmParams& p, int row, int col0, int split, const float (&f)[32],
+__device__ __forceinline__ void epilogue_store32(const GemmParams& p, int row, int col0, const float (&f)[32],
                                                  uint32_t& amax_bits) {
   if (col0 + 32 <= p.n_split) {
     if (p.c0_dt == kBF16) {
-      uint16_t* dst = static_cast<uint16_t*>(p.c0) + (long long)split * p.c0_split_stride + (long long)row * p.ldc0 + col0;
+      uint16_t* dst = static_cast<uint16_t*>(p.c0) + (long long)row * p.ldc0 + col0;
       if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -80,7 +80,7 @@ __device__ __forceinline__ void epilogue_store32(const GemmParams& p, int row, i
         for (int i = 0; i < 32; ++i) dst[i] = static_cast<uint16_t>(pack_bf16x2(f[i], 0.0f) & 0xFFFF);
       }
     } else {
-      float* dst = static_cast<float*>(p.c0) + (long long)split * p.c0_split_stride + (long long)row * p.ldc0 + col0;
+      float* dst = static_cast<float*>(p.c0) + (long long)row * p.ldc0 + col0;
       if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
 #pragma unroll
         for (int i = 0; i < 8; ++i)
@@ -96,7 +96,7 @@ __device__ __forceinline__ void epilogue_store32(const GemmParams& p, int row, i
     for (int i = 0; i < 32; ++i) {
       const int col = col0 + i;
       if (col < p.n_split) {
-        const long long off = (long long)split * p.c0_split_stride + (long long)row * p.ldc0 + col;
+        const long long off = (long long)row * p.ldc0 + col;
         if (p.c0_dt == kBF16) static_cast<uint16_t*>(p.c0)[off] = static_cast<uint16_t>(pack_bf16x2(f[i], 0.0f) & 0xFFFF);
         else static_cast<float*>(p.c0)[off] = f[i];
       } else if (col < p.N) {
@@ -114,7 +114,7 @@ __device__ __forceinline__ void epilogue_store32(const GemmParams& p, int row, i
 // instruction then covers 4 rows x 128 B instead of 32 rows x 16 B.  Chunks that touch the O | O_A boundary
 // or the ragged right edge take the element-wise path.
 __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_row, int row, bool row_ok, int n0,
-                                              int col_begin, int col_end, int split, float inv, uint32_t& amax_bits,
+                                              int col_begin, int col_end, float inv, uint32_t& amax_bits,
                                               uint8_t* stage_out) {
   const int last = min(col_end, p.N - n0);    // warp-uniform: columns at or beyond N hold nothing
   if (col_begin >= last) return;
@@ -134,7 +134,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ro
     const int rows_per_inst = 32 / lanes_per_row;          // 8 or 4
     const int piece = lane % lanes_per_row;
     uint8_t* c0 = static_cast<uint8_t*>(p.c0) +
-                  ((long long)split * p.c0_split_stride + flush_col) * esize + (long long)piece * 16;
+                  (long long)flush_col * esize + (long long)piece * 16;
     for (int r0 = 0; r0 < 32; r0 += rows_per_inst) {
       const int r = r0 + lane / lanes_per_row;
       const uint4 val = *reinterpret_cast<const uint4*>(stage_out + r * 128 + ((piece ^ (r & 7)) << 4));
@@ -160,7 +160,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ro
       for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * inv;
     }
     const bool fast = col0 + 32 <= p.n_split && ((p.ldc0 * esize) & 15) == 0 &&
-                      ((reinterpret_cast<uintptr_t>(p.c0) + (long long)split * p.c0_split_stride * esize) & 15) == 0;
+                      (reinterpret_cast<uintptr_t>(p.c0) & 15) == 0;
     if (fast) {   // warp-uniform
       if (pending == 0) flush_col = col0;
       uint8_t* my = stage_out + lane * 128;
@@ -185,7 +185,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ro
       if (pending == chunks_per_flush) flush();
     } else {
       flush();
-      if (row_ok) epilogue_store32(p, row, col0, split, f, amax_bits);
+      if (row_ok) epilogue_store32(p, row, col0, f, amax_bits);
     }
   };
 
@@ -209,7 +209,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ro
   flush();
 }
 
-template <bool kAMn, bool kBMn>
+template <bool kBMn>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                 const GemmParams p) {
@@ -256,8 +256,7 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();   // everything above is private set-up; operands and scales are read only from here on
 
-  const int tiles_per_split = p.m_tiles * p.n_tiles;
-  const int total_tiles = tiles_per_split * p.k_splits;
+  const int total_tiles = p.m_tiles * p.n_tiles;
   bool aborted = false;
 
   if (warp == 0) {
@@ -265,21 +264,16 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     int stage = 0;
     uint32_t phase = 0;
     for (int tile = blockIdx.x; tile < total_tiles && !aborted; tile += gridDim.x) {
-      const int split = tile / tiles_per_split;
-      const int rem = tile - split * tiles_per_split;
-      const int n_idx = rem / p.m_tiles;
-      const int m_idx = rem - n_idx * p.m_tiles;
-      const int kb_begin = split * p.kblocks_per_split;
-      const int kb_end = min(kb_begin + p.kblocks_per_split, p.kblocks_total);
-      for (int kb = kb_begin; kb < kb_end; ++kb) {
+      const int n_idx = tile / p.m_tiles;
+      const int m_idx = tile - n_idx * p.m_tiles;
+      for (int kb = 0; kb < p.kblocks_total; ++kb) {
         if (!mbar_wait_warp(empty_bar(stage), phase ^ 1u, p.status)) { aborted = true; break; }
         if (elect_one()) {
           const uint32_t fb = full_bar(stage);
           mbar_expect_tx(fb, stage_bytes);
           const uint32_t a_dst = smem_base + static_cast<uint32_t>(stage) * stage_bytes;
           const uint32_t b_dst = a_dst + kATileBytes;
-          if (!kAMn) tma_load_2d(a_dst, &tmap_a, fb, kb * kBlockKBytes, m_idx * kBlockM);
-          else       tma_load_2d(a_dst, &tmap_a, fb, m_idx * kBlockM, kb * kBlockKBytes);
+          tma_load_2d(a_dst, &tmap_a, fb, kb * kBlockKBytes, m_idx * kBlockM);
           if (!kBMn) {
             tma_load_2d(b_dst, &tmap_b, fb, kb * kBlockKBytes, n_idx * p.block_n);
           } else {
@@ -299,19 +293,16 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     int acc = 0;
     uint32_t acc_phase = 0;
     // descriptors differ between stages and K steps only in the 14-bit start-address field
-    const uint64_t a_desc0 = kAMn ? make_smem_desc(smem_base, kMnChunkBytes, 1024) : make_smem_desc(smem_base, 16, 1024);
+    const uint64_t a_desc0 = make_smem_desc(smem_base, 16, 1024);
     const uint64_t b_desc0 = kBMn ? make_smem_desc(smem_base + kATileBytes, kMnChunkBytes, 1024)
                                   : make_smem_desc(smem_base + kATileBytes, 16, 1024);
-    constexpr uint32_t kAStep = (kAMn ? kUmmaK * 128 : kUmmaK) >> 4;   // per K step, in 16-byte units
+    constexpr uint32_t kAStep = kUmmaK >> 4;   // per K step, in 16-byte units
     constexpr uint32_t kBStep = (kBMn ? kUmmaK * 128 : kUmmaK) >> 4;
     for (int tile = blockIdx.x; tile < total_tiles && !aborted; tile += gridDim.x) {
-      const int split = tile / tiles_per_split;
-      const int kb_begin = split * p.kblocks_per_split;
-      const int kb_end = min(kb_begin + p.kblocks_per_split, p.kblocks_total);
       if (!mbar_wait_warp(tmem_empty_bar(acc), acc_phase ^ 1u, p.status)) { aborted = true; break; }
       tc_fence_after_sync();
       const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * kAccCols;
-      for (int kb = kb_begin; kb < kb_end; ++kb) {
+      for (int kb = 0; kb < p.kblocks_total; ++kb) {
         if (!mbar_wait_warp(full_bar(stage), phase, p.status)) { aborted = true; break; }
         tc_fence_after_sync();
         const uint32_t stage_off = (static_cast<uint32_t>(stage) * stage_bytes) >> 4;
@@ -319,7 +310,7 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 #pragma unroll
           for (int k = 0; k < kBlockKBytes / kUmmaK; ++k) {
             umma_f8(d_tmem, a_desc0 + stage_off + k * kAStep, b_desc0 + stage_off + k * kBStep, p.idesc,
-                    (kb > kb_begin || k > 0) ? 1u : 0u);
+                    (kb > 0 || k > 0) ? 1u : 0u);
           }
           umma_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
         }
@@ -343,10 +334,8 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     uint32_t acc_phase = 0;
     uint32_t amax_bits = 0;
     for (int tile = blockIdx.x; tile < total_tiles && !aborted; tile += gridDim.x) {
-      const int split = tile / tiles_per_split;
-      const int rem = tile - split * tiles_per_split;
-      const int n_idx = rem / p.m_tiles;
-      const int m_idx = rem - n_idx * p.m_tiles;
+      const int n_idx = tile / p.m_tiles;
+      const int m_idx = tile - n_idx * p.m_tiles;
       if (!mbar_wait(tmem_full_bar(acc), acc_phase, p.status)) { aborted = true; break; }
       tc_fence_after_sync();
       const int row = m_idx * kBlockM + quad * 32 + lane;
@@ -354,8 +343,7 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const uint32_t t_row = tmem_base + static_cast<uint32_t>(acc) * kAccCols + (static_cast<uint32_t>(quad * 32) << 16);
       const int n0 = n_idx * p.block_n;
       const int half = (((p.block_n + 1) / 2) + 31) & ~31;   // first-half warps take [0, half), the others [half, block_n)
-      epilogue_tile(p, t_row, row, row_ok, n0, col_half ? half : 0, col_half ? p.block_n : half, split, inv, amax_bits,
-                    stage_out);
+      epilogue_tile(p, t_row, row, row_ok, n0, col_half ? half : 0, col_half ? p.block_n : half, inv, amax_bits, stage_out);
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(tmem_empty_bar(acc));
@@ -551,7 +539,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       const bool row_ok = row < p.M;
       const uint32_t t_row = tmem_base + static_cast<uint32_t>(acc) * kAccCols + (static_cast<uint32_t>(quad * 32) << 16);
       const int n0 = n_idx * 256;
-      epilogue_tile(p, t_row, row, row_ok, n0, col_half ? 128 : 0, col_half ? 256 : 128, 0, inv, amax_bits, stage_out);
+      epilogue_tile(p, t_row, row, row_ok, n0, col_half ? 128 : 0, col_half ? 256 : 128, inv, amax_bits, stage_out);
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(tmem_empty_bar(acc), 0));
@@ -597,6 +585,8 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
+}  // namespace
+
 // 2-D uint8 tensor [rows][cols] with row pitch ld bytes; box = box_cols x box_rows, 128-byte swizzle.
 bool make_tensor_map(CUtensorMap* map, const uint8_t* base, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols,
                      uint32_t box_rows) {
@@ -622,17 +612,19 @@ int sm_count() {
   return count;
 }
 
-template <bool kAMn, bool kBMn>
+namespace {
+
+template <bool kBMn>
 cudaError_t launch_variant(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& gp, int grid, size_t smem,
                            cudaStream_t stream) {
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_fp8_kernel<kAMn, kBMn>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(gemm_fp8_kernel<kBMn>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(kSmemBudget));
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  return launch_pdl(gemm_fp8_kernel<kAMn, kBMn>, dim3(static_cast<unsigned>(grid)), dim3(kGemmThreads), smem, stream, 1, ta,
+  return launch_pdl(gemm_fp8_kernel<kBMn>, dim3(static_cast<unsigned>(grid)), dim3(kGemmThreads), smem, stream, 1, ta,
                     tb, gp);
 }
 
@@ -666,8 +658,6 @@ cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
   gp.m_tiles = static_cast<int>((q.M + 255) / 256);
   gp.n_tiles = static_cast<int>((q.N + 255) / 256);
   gp.kblocks_total = static_cast<int>((q.K + kBlockKBytes - 1) / kBlockKBytes);
-  gp.k_splits = 1;
-  gp.kblocks_per_split = gp.kblocks_total;
   int stages = static_cast<int>((kSmemBudget - 1024 - kBarrierBytes - kStagingBytes) / kPairStageBytes);
   if (stages > kMaxStages) stages = kMaxStages;
   gp.num_stages = stages;
@@ -675,7 +665,6 @@ cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
   gp.idesc = (1u << 4) | (static_cast<uint32_t>(q.a_fmt) << 7) | (static_cast<uint32_t>(q.b_fmt) << 10) |
              ((q.b_mn_major ? 1u : 0u) << 16) | (static_cast<uint32_t>(256 >> 4) << 24);
   gp.c0 = q.c0; gp.ldc0 = q.ldc0; gp.c0_dt = q.c0_dt; gp.n_split = static_cast<int>(q.n_split);
-  gp.c0_split_stride = 0;
   gp.c1 = q.c1; gp.ldc1 = q.ldc1; gp.amax1_bits = q.amax1_bits;
   gp.scale_a = q.scale_a; gp.scale_b = q.scale_b; gp.col_scale = q.col_scale;
   gp.status = q.status;
@@ -695,22 +684,12 @@ cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
 
 }  // namespace
 
-int gemm_k_splits_for_db(int64_t m, int64_t T) {
-  const int64_t m_tiles = (m + kBlockM - 1) / kBlockM;
-  const int64_t kblocks = (T + kBlockKBytes - 1) / kBlockKBytes;
-  int64_t want = (2 * 148 + m_tiles - 1) / m_tiles;
-  if (want < 1) want = 1;
-  if (want > kblocks) want = kblocks;
-  const int64_t per = (kblocks + want - 1) / want;
-  return static_cast<int>((kblocks + per - 1) / per);
-}
-
 cudaError_t launch_gemm_fp8(const GemmProblem& q, cudaStream_t stream) {
   if (q.M <= 0 || q.N <= 0 || q.K <= 0) return cudaErrorInvalidValue;
   if (q.block_n < 16 || q.block_n > 256 || q.block_n % 16) return cudaErrorInvalidValue;
   if (q.b_mn_major && q.block_n % 128) return cudaErrorInvalidValue;
   // the tensor-bound roles (K-major A, full-width tiles, no token slabs) run on CTA pairs
-  if (!q.a_mn_major && q.block_n == 256 && q.k_splits <= 1 && q.N % 16 == 0 && !pair_kernel_disabled())
+  if (q.block_n == 256 && q.N % 16 == 0 && !pair_kernel_disabled())
     return launch_gemm_fp8_pair(q, stream);
 
   GemmParams gp{};
@@ -719,9 +698,6 @@ cudaError_t launch_gemm_fp8(const GemmProblem& q, cudaStream_t stream) {
   gp.m_tiles = static_cast<int>((q.M + kBlockM - 1) / kBlockM);
   gp.n_tiles = static_cast<int>((q.N + q.block_n - 1) / q.block_n);
   gp.kblocks_total = static_cast<int>((q.K + kBlockKBytes - 1) / kBlockKBytes);
-  gp.k_splits = q.k_splits < 1 ? 1 : q.k_splits;
-  gp.kblocks_per_split = (gp.kblocks_total + gp.k_splits - 1) / gp.k_splits;
-  gp.k_splits = (gp.kblocks_total + gp.kblocks_per_split - 1) / gp.kblocks_per_split;  // no empty split
   const uint32_t stage_bytes = kATileBytes + static_cast<uint32_t>(q.block_n) * kBlockKBytes;
   int stages = static_cast<int>((kSmemBudget - 1024 - kBarrierBytes - kStagingBytes) / stage_bytes);
   if (stages > kMaxStages) stages = kMaxStages;
@@ -729,33 +705,27 @@ cudaError_t launch_gemm_fp8(const GemmProblem& q, cudaStream_t stream) {
   gp.num_stages = stages;
   // instruction descriptor: fp32 accumulate, operand formats and majors, N/8 at bit 17, M/16 at bit 24
   gp.idesc = (1u << 4) | (static_cast<uint32_t>(q.a_fmt) << 7) | (static_cast<uint32_t>(q.b_fmt) << 10) |
-             ((q.a_mn_major ? 1u : 0u) << 15) | ((q.b_mn_major ? 1u : 0u) << 16) |
+             ((q.b_mn_major ? 1u : 0u) << 16) |
              (static_cast<uint32_t>(q.block_n >> 3) << 17) | (static_cast<uint32_t>(kBlockM >> 4) << 24);
   gp.c0 = q.c0; gp.ldc0 = q.ldc0; gp.c0_dt = q.c0_dt; gp.n_split = static_cast<int>(q.n_split);
-  gp.c0_split_stride = q.c0_split_stride;
   gp.c1 = q.c1; gp.ldc1 = q.ldc1; gp.amax1_bits = q.amax1_bits;
   gp.scale_a = q.scale_a; gp.scale_b = q.scale_b; gp.col_scale = q.col_scale;
   gp.status = q.status;
 
   CUtensorMap ta, tb;
   bool ok;
-  if (!q.a_mn_major) ok = make_tensor_map(&ta, q.a, q.M, q.K, q.lda, kBlockKBytes, kBlockM);
-  else               ok = make_tensor_map(&ta, q.a, q.K, q.M, q.lda, kBlockM, kBlockKBytes);
+  ok = make_tensor_map(&ta, q.a, q.M, q.K, q.lda, kBlockKBytes, kBlockM);
   if (!ok) return cudaErrorInvalidValue;
   if (!q.b_mn_major) ok = make_tensor_map(&tb, q.b, q.N, q.K, q.ldb, kBlockKBytes, static_cast<uint32_t>(q.block_n));
   else               ok = make_tensor_map(&tb, q.b, q.K, q.N, q.ldb, 128, kBlockKBytes);
   if (!ok) return cudaErrorInvalidValue;
 
-  const long long total_tiles = static_cast<long long>(gp.m_tiles) * gp.n_tiles * gp.k_splits;
+  const long long total_tiles = static_cast<long long>(gp.m_tiles) * gp.n_tiles;
   int grid = sm_count();
   if (total_tiles < grid) grid = static_cast<int>(total_tiles);
   const size_t smem = static_cast<size_t>(stages) * stage_bytes + kBarrierBytes + kStagingBytes + 1024;
-  if (q.a_mn_major) {
-    if (q.b_mn_major) return launch_variant<true, true>(ta, tb, gp, grid, smem, stream);
-    return launch_variant<true, false>(ta, tb, gp, grid, smem, stream);
-  }
-  if (q.b_mn_major) return launch_variant<false, true>(ta, tb, gp, grid, smem, stream);
-  return launch_variant<false, false>(ta, tb, gp, grid, smem, stream);
+  if (q.b_mn_major) return launch_variant<true>(ta, tb, gp, grid, smem, stream);
+  return launch_variant<false>(ta, tb, gp, grid, smem, stream);
 }
 
 }  // namespace falqon

@@ -5,6 +5,8 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+struct CUtensorMap_st;
+
 namespace falqon {
 
 constexpr int kE4M3 = 0, kE5M2 = 1;
@@ -51,12 +53,25 @@ cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, i
                                    const uint32_t* partial, int nparts, const float* scale_in, uint8_t* dst,
                                    float* scale_out, float* scale_out2, float* amax_out, float* clear_word,
                                    cudaStream_t stream);
+// A small cast that rides along with a fused quantizer launch (S5a inside S3's kernel): O_A [T][r] fp32 -> E4M3 codes
+// written transposed as [r][ldt] with s_OA = 448 / *amax_oa; *amax_copy = *amax_oa.  oa == nullptr: none.
+struct OaCastJob {
+  const float* oa;
+  const float* amax_oa;
+  long long T;
+  int r;
+  long long ldt;
+  uint8_t* oaq_t;
+  float* s_oa_out;
+  float* amax_copy;   // nullable
+};
 // Per-tensor absmax scaling in one kernel (absmax, grid barrier, cast).  `sync` points at 8 bytes of workspace that
 // are zero before the call and are left zero by it; `partial` holds up to kMaxAbsmaxParts words.
 // col_mul (nullable): column c of the [count / cols][cols] tensor is multiplied by col_mul[c] before everything else.
+// oa_cast (nullable): see OaCastJob.
 cudaError_t launch_quantize_fused(const void* src, int src_dt, int64_t count, int fmt, uint8_t* dst, uint32_t* partial,
                                   void* sync, float* scale_out, float* scale_out2, float* amax_out, float* clear_word,
-                                  int* status, const float* col_mul, int cols, cudaStream_t stream);
+                                  int* status, const float* col_mul, int cols, const OaCastJob* oa_cast, cudaStream_t stream);
 // Tables for a per-row-scaled backbone (s_w has m + 1 entries): mode 0 -> out[i] = 1/s_w[i]; mode 1 ->
 // out[c] = 1/(s_w[min(c,m)] * *s_x) for c < m + r.  Entries up to `padded` are written (zero beyond the table).
 cudaError_t launch_scale_table(int mode, const float* s_w, int64_t m, int64_t r, const float* s_x, float* out, int64_t padded,
@@ -64,33 +79,42 @@ cudaError_t launch_scale_table(int mode, const float* s_w, int64_t m, int64_t r,
 cudaError_t launch_quantize_per_row(const void* src, int src_dt, int64_t rows, int64_t cols, int fmt, float premul,
                                     const float* scale_in, uint8_t* dst, float* scale_out, float* amax_out,
                                     cudaStream_t stream);
-// O_A [T][r] fp32 -> E4M3 codes written transposed as [r16][ldt] with s_OA = 448 / *amax_oa; *amax_copy = *amax_oa.
-cudaError_t launch_quantize_oa_transposed(const float* oa, const float* amax_oa, int64_t T, int64_t r, int64_t r16,
-                                          int64_t ldt, uint8_t* oaq_t, float* s_oa_out, float* amax_copy,
-                                          cudaStream_t stream);
 
 // ---- gemm_fp8.cu
 struct GemmProblem {
   // D[M][N] = A[M][K] * B[N][K]^T with fp32 accumulation on tcgen05
   int64_t M, N, K;
-  const uint8_t* a; int64_t lda; bool a_mn_major; int a_fmt;  // K-major: a[M][lda]; MN-major: a[K][lda]
+  const uint8_t* a; int64_t lda; int a_fmt;                   // K-major: a[M][lda]
   const uint8_t* b; int64_t ldb; bool b_mn_major; int b_fmt;  // K-major: b[N][ldb]; MN-major: b[K][ldb]
   int block_n;                 // tile width (16..256, multiple of 16)
-  int k_splits;                // >1: partial sums, one output slab per split, no rescale
   // epilogue: columns [0, n_split) -> c0 (bf16 or fp32), columns [n_split, N) -> c1 (fp32) with |max| -> amax1
-  void* c0; int64_t ldc0; int c0_dt; int64_t n_split; int64_t c0_split_stride;
+  void* c0; int64_t ldc0; int c0_dt; int64_t n_split;
   float* c1; int64_t ldc1; uint32_t* amax1_bits;
   const float* scale_a; const float* scale_b;  // device scalars; output *= 1/(sa*sb); scale_b null: 1/sa; both null: none
   const float* col_scale;                      // nullable: per-column factors (N rounded up to 32 entries) instead
   int* status;
 };
 cudaError_t launch_gemm_fp8(const GemmProblem& p, cudaStream_t stream);
-int gemm_k_splits_for_db(int64_t m, int64_t T);
+// 2-D uint8 tensor [rows][cols] with row pitch ld bytes; box = box_cols x box_rows, 128-byte swizzle.
+bool make_tensor_map(CUtensorMap_st* map, const uint8_t* base, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols,
+                     uint32_t box_rows);
+int sm_count();
+
+// ---- gemm_db.cu: S5b in one kernel -- dB = g~^T O~_A / (s_g s_OA) over token slabs, the slab sum taken in slab
+// order across a thread-block cluster.
+struct DbFusedProblem {
+  int64_t m, r, T;
+  const uint8_t* gq;           // [T][m] E5M2
+  const uint8_t* oaq_t; int64_t ldt;   // [r16][ldt] E4M3 codes of O_A, transposed (rows r.. may hold anything)
+  const float* s_oa;           // [1]
+  const float* s_g;            // [1]
+  const float* row_mul;        // nullable [m]: dB row i is also multiplied by row_mul[i]
+  float* dB;                   // [m][r]
+  int* status;
+};
+cudaError_t launch_db_fused(const DbFusedProblem& p, cudaStream_t stream);
 
 // ---- proxy_update.cu
-// row_mul (nullable, one factor per row of r entries): dB[i][:] is also multiplied by row_mul[i].
-cudaError_t launch_reduce_db(const float* partials, int splits, int64_t count, const float* s_g, const float* s_oa,
-                             const float* row_mul, int64_t r, float* dB, cudaStream_t stream);
 cudaError_t launch_sgd_score(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, float* score,
                              cudaStream_t stream);
 // The k selected rows (ascending) are written to sel_idx and, when idx_copy is non-null, to idx_copy (int32 [k]).

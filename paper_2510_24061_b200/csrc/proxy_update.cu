@@ -10,29 +10,6 @@
 namespace falqon {
 namespace {
 
-// ---- dB = (sum over splits, in split order) / (s_g * s_OA)
-__global__ void __launch_bounds__(256) reduce_db_kernel(const float* partials, int splits, int64_t count,
-                                                        const float* s_g, const float* s_oa,
-                                                        const float* row_mul, int r, float* dB) {
-  pdl_trigger();
-  pdl_wait();
-  const float inv = 1.0f / (ld_stream(s_g) * ld_stream(s_oa));
-  const int64_t nvec = count / 4;
-  for (int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; v < nvec; v += (int64_t)gridDim.x * blockDim.x) {
-    float4 acc = reinterpret_cast<const float4*>(partials)[v];
-    for (int s = 1; s < splits; ++s) {
-      const float4 x = reinterpret_cast<const float4*>(partials + (int64_t)s * count)[v];
-      acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
-    }
-    acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-    if (row_mul != nullptr) {   // per-row-scaled backbone: give row i its scale back (r is a multiple of 4)
-      const float f = ld_stream(row_mul + (v * 4) / r);
-      acc.x *= f; acc.y *= f; acc.z *= f; acc.w *= f;
-    }
-    reinterpret_cast<float4*>(dB)[v] = acc;
-  }
-}
-
 // ---- DeltaBuffer <- fma(-lr, dB, DeltaBuffer); score_i = ((|d_i0| + |d_i1|) + ...) in fp32
 constexpr int kScoreRows = 32;
 __global__ void __launch_bounds__(256) sgd_score_kernel(float* dbuf, const float* dB,
@@ -465,15 +442,6 @@ __global__ void __launch_bounds__(256) zero_rows_kernel(float* dbuf, const int32
 }
 
 }  // namespace
-
-cudaError_t launch_reduce_db(const float* partials, int splits, int64_t count, const float* s_g, const float* s_oa,
-                             const float* row_mul, int64_t r, float* dB, cudaStream_t stream) {
-  int64_t blocks = (count / 4 + 255) / 256;
-  if (blocks > 148 * 8) blocks = 148 * 8;
-  if (blocks < 1) blocks = 1;
-  return launch_pdl(reduce_db_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream, 1, partials, splits, count,
-                    s_g, s_oa, row_mul, static_cast<int>(r), dB);
-}
 
 cudaError_t launch_sgd_score(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, float* score,
                              cudaStream_t stream) {

@@ -192,6 +192,12 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
   return r;
 }
+__device__ __forceinline__ float4 ld_shared_cluster_f32x4(uint32_t cluster_addr) {   // any CTA's shared memory
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr) : "memory");
+  return v;
+}
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {  // may target the peer CTA's barrier
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
@@ -261,6 +267,16 @@ __device__ __forceinline__ float2 e4m3x2_to_float2(uint32_t pair) {
       : "=f"(out.x), "=f"(out.y)
       : "r"(h2));
   return out;
+}
+
+// Eq. quantize: scale = fp8max / amax as one IEEE fp32 division; amax == 0 -> 1; an infinite quotient -> FLT_MAX.
+// fmt: 0 = E4M3 (max 448), 1 = E5M2 (max 57344).
+__device__ __forceinline__ float fp8_max(int fmt) { return fmt == 0 ? 448.0f : 57344.0f; }
+__device__ __forceinline__ float scale_from_amax(float amax, int fmt) {
+  if (!(amax > 0.0f)) return 1.0f;
+  float s = __fdiv_rn(fp8_max(fmt), amax);
+  if (isinf(s)) s = 3.402823466e+38f;
+  return s;
 }
 
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }

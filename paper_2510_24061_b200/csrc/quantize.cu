@@ -11,16 +11,6 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kMaxBlocks = 148 * 8;
 
-__device__ __forceinline__ float fp8_max(int fmt) { return fmt == kE4M3 ? 448.0f : 57344.0f; }
-
-// scale = fp8max / amax as one IEEE fp32 division; amax == 0 -> 1; an infinite quotient -> FLT_MAX.
-__device__ __forceinline__ float scale_from_amax(float amax, int fmt) {
-  if (!(amax > 0.0f)) return 1.0f;
-  float s = __fdiv_rn(fp8_max(fmt), amax);
-  if (isinf(s)) s = 3.402823466e+38f;
-  return s;
-}
-
 // Loads 16 consecutive elements as fp32 (element index must be a multiple of 16).
 template <int kDt>
 __device__ __forceinline__ void load16(const void* src, int64_t elem, float (&v)[16]) {
@@ -207,10 +197,62 @@ __device__ __forceinline__ void unit_values(const uint4& q, const float* col_mul
   }
 }
 
+// A rider of the output-gradient quantizer (S5a): O_A [T][r] fp32 -> E4M3 codes with s_OA = 448 / amax(O_A), stored
+// TRANSPOSED as [r][ldt] so that the adapter-gradient product reads them K-major.  One warp converts a tile of
+// 32 tokens (only the upper half of a CTA's warps call this): lane (tg, jq) takes tokens 4 tg .. 4 tg + 3 and columns 16 jq .. 16 jq + 15 of every block of 64
+// columns, so the codes of four consecutive tokens of one column form one 32-bit store.  Tokens at or beyond T
+// give zero codes (they land in the padding of the row pitch, a multiple of 16).
+__device__ __forceinline__ void cast_oa_transposed(const OaCastJob& job) {
+  const int lane = threadIdx.x & 31;
+  const int tg = lane >> 2, jq = lane & 3;
+  const float amax = ld_stream(job.amax_oa);
+  const float s_oa = scale_from_amax(amax, kE4M3);
+  if (blockIdx.x == 0 && threadIdx.x == blockDim.x / 2) {
+    *job.s_oa_out = s_oa;
+    if (job.amax_copy != nullptr) *job.amax_copy = amax;
+  }
+  const long long n_tiles = (job.T + 31) / 32;
+  const int rider_warps = blockDim.x >> 6;                      // the upper half of the CTA's warps
+  const int w = (threadIdx.x >> 5) - rider_warps;               // 0 .. rider_warps - 1
+  const int r16 = (job.r + 15) & ~15;
+  // consecutive tiles go to different CTAs, so a small O_A costs every CTA at most one tile on one warp
+  for (long long tile = static_cast<long long>(w) * gridDim.x + blockIdx.x; tile < n_tiles;
+       tile += static_cast<long long>(rider_warps) * gridDim.x) {
+    const long long t0 = tile * 32 + 4 * tg;
+    for (int jb = 0; jb < r16; jb += 64) {
+      const int j0 = jb + 16 * jq;
+      if (j0 >= job.r) continue;
+      float4 x[4][4];
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          x[a][q] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (t0 + a < job.T && j0 + 4 * q < job.r)    // r is a multiple of 8: a float4 is all inside or all outside
+            x[a][q] = ld_stream(reinterpret_cast<const float4*>(job.oa + (t0 + a) * job.r + j0) + q);
+        }
+      }
+      if (t0 >= job.ldt) continue;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float c[4][4] = {{x[0][q].x, x[1][q].x, x[2][q].x, x[3][q].x}, {x[0][q].y, x[1][q].y, x[2][q].y, x[3][q].y},
+                               {x[0][q].z, x[1][q].z, x[2][q].z, x[3][q].z}, {x[0][q].w, x[1][q].w, x[2][q].w, x[3][q].w}};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int j = j0 + 4 * q + e;
+          if (j < job.r)
+            *reinterpret_cast<uint32_t*>(job.oaq_t + static_cast<long long>(j) * job.ldt + t0) =
+                cvt_fp8x4<kE4M3>(__fmul_rn(c[e][0], s_oa), __fmul_rn(c[e][1], s_oa), __fmul_rn(c[e][2], s_oa), __fmul_rn(c[e][3], s_oa));
+        }
+      }
+    }
+  }
+}
+
 template <int kDt, int kFmt, bool kColMul>
 __global__ void __launch_bounds__(kStagedThreads, 1)
 quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* partial, GridSync* sync, CastOutputs out,
-                       int* status, const float* col_mul, int cols) {
+                       int* status, const float* col_mul, int cols, OaCastJob oa_job) {
   constexpr int kEsize = kDt == kBF16 ? 2 : 4;
   constexpr int kUnit = Unit<kDt>::kElems;
   constexpr int64_t kChunkElems = kChunkBytes / kEsize;
@@ -276,6 +318,9 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
     }
   }
   m = block_max_u32(m, red);
+  // the rider runs here, on warps that would otherwise idle while thread 0 waits at the grid barrier: this CTA's
+  // bulk copies have landed, so the rider's loads do not queue behind them
+  if (oa_job.oa != nullptr && tid >= kStagedThreads / 2) cast_oa_transposed(oa_job);
   // ---- grid barrier (a CTA that gave up above does not arrive: the others time out and report it)
   if (tid == 0) {
     int ok = failed ? 0 : 1;
@@ -411,52 +456,6 @@ __global__ void __launch_bounds__(kThreads) quantize_rows_kernel(const void* src
   }
 }
 
-// ---- O_A [T][r] fp32 -> E4M3 codes, transposed to [r][ldt] so the dB product reads it K-major.
-// A CTA converts 32 tokens x r: float4 loads along r, byte transposition through shared memory,
-// 16-byte stores along the tokens.
-constexpr int kOaTileT = 32;
-__global__ void __launch_bounds__(256) quantize_oa_transposed_kernel(const float* oa,
-                                                                     const float* amax_oa, int64_t T, int r,
-                                                                     int64_t ldt, uint8_t* oaq_t,
-                                                                     float* s_oa_out,
-                                                                     float* amax_copy) {
-  __shared__ __align__(16) uint8_t tile[256][kOaTileT + 16];
-  pdl_trigger();
-  pdl_wait();
-  const float amax = *amax_oa;
-  const float s = scale_from_amax(amax, kE4M3);
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
-    if (s_oa_out) *s_oa_out = s;
-    if (amax_copy) *amax_copy = amax;
-  }
-  const int64_t t0 = (int64_t)blockIdx.x * kOaTileT;
-  const int tcount = static_cast<int>(min((int64_t)kOaTileT, T - t0));
-  const int r4 = r >> 2;                       // r is a multiple of 8
-  const int tx = threadIdx.x % r4, ty = threadIdx.x / r4;
-  const int rows_per_pass = blockDim.x / r4;
-  if (ty < rows_per_pass) {
-    for (int tl = ty; tl < kOaTileT; tl += rows_per_pass) {
-      uint32_t codes = 0;
-      if (tl < tcount) {
-        const float4 x = ld_stream(reinterpret_cast<const float4*>(oa + (t0 + tl) * r) + tx);
-        codes = cvt_fp8x4<kE4M3>(__fmul_rn(x.x, s), __fmul_rn(x.y, s), __fmul_rn(x.z, s), __fmul_rn(x.w, s));
-      }
-      tile[4 * tx + 0][tl] = static_cast<uint8_t>(codes);
-      tile[4 * tx + 1][tl] = static_cast<uint8_t>(codes >> 8);
-      tile[4 * tx + 2][tl] = static_cast<uint8_t>(codes >> 16);
-      tile[4 * tx + 3][tl] = static_cast<uint8_t>(codes >> 24);
-    }
-  }
-  __syncthreads();
-  // each row j of the tile is 32 bytes = two 16-byte stores (tokens beyond T are zero codes and land in
-  // the padding of the row pitch, which is a multiple of 16, or are skipped at the very end)
-  for (int e = threadIdx.x; e < r * 2; e += blockDim.x) {
-    const int j = e >> 1, half = e & 1;
-    if (t0 + half * 16 < ldt)
-      *reinterpret_cast<uint4*>(oaq_t + (int64_t)j * ldt + t0 + half * 16) = *reinterpret_cast<const uint4*>(&tile[j][half * 16]);
-  }
-}
-
 inline int grid_for(int64_t nvec) {
   int64_t blocks = (nvec + kThreads - 1) / kThreads;
   if (blocks < 1) blocks = 1;
@@ -495,7 +494,8 @@ cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, i
 
 template <int kDt, int kFmt, bool kColMul>
 cudaError_t launch_staged_variant(const void* src, int64_t count, uint8_t* dst, uint32_t* partial, void* sync,
-                                  const CastOutputs& out, int* status, const float* col_mul, int cols, cudaStream_t stream) {
+                                  const CastOutputs& out, int* status, const float* col_mul, int cols, const OaCastJob& oa_job,
+                                  cudaStream_t stream) {
   constexpr size_t kSmem = static_cast<size_t>(kStagedSlots) * kChunkBytes;
   static int blocks_per_sm = 0;
   if (blocks_per_sm == 0) {
@@ -517,18 +517,19 @@ cudaError_t launch_staged_variant(const void* src, int64_t count, uint8_t* dst, 
   if (grid > kMaxAbsmaxParts) grid = kMaxAbsmaxParts;
   if (grid < 1) grid = 1;
   return launch_pdl(quantize_staged_kernel<kDt, kFmt, kColMul>, dim3(static_cast<unsigned>(grid)), dim3(kStagedThreads), kSmem,
-                    stream, 1, src, count, dst, partial, static_cast<GridSync*>(sync), out, status, col_mul, cols);
+                    stream, 1, src, count, dst, partial, static_cast<GridSync*>(sync), out, status, col_mul, cols, oa_job);
 }
 
 cudaError_t launch_quantize_fused(const void* src, int src_dt, int64_t count, int fmt, uint8_t* dst, uint32_t* partial,
                                   void* sync, float* scale_out, float* scale_out2, float* amax_out, float* clear_word,
-                                  int* status, const float* col_mul, int cols, cudaStream_t stream) {
+                                  int* status, const float* col_mul, int cols, const OaCastJob* oa_cast, cudaStream_t stream) {
   const CastOutputs out{scale_out, scale_out2, amax_out, clear_word};
+  const OaCastJob oa_job = oa_cast != nullptr ? *oa_cast : OaCastJob{};
 #define FALQON_FUSED(DT, FMT)                                                                                              \
   do {                                                                                                                     \
     if (col_mul != nullptr)                                                                                                \
-      return launch_staged_variant<DT, FMT, true>(src, count, dst, partial, sync, out, status, col_mul, cols, stream);     \
-    return launch_staged_variant<DT, FMT, false>(src, count, dst, partial, sync, out, status, nullptr, 0, stream);         \
+      return launch_staged_variant<DT, FMT, true>(src, count, dst, partial, sync, out, status, col_mul, cols, oa_job, stream); \
+    return launch_staged_variant<DT, FMT, false>(src, count, dst, partial, sync, out, status, nullptr, 0, oa_job, stream); \
   } while (0)
   if (src_dt == kBF16) {
     if (fmt == kE4M3) FALQON_FUSED(kBF16, kE4M3);
@@ -557,15 +558,6 @@ cudaError_t launch_quantize_per_row(const void* src, int src_dt, int64_t rows, i
   if (src_dt == kBF16) { if (fmt == kE4M3) FALQON_ROWS(kBF16, kE4M3); else FALQON_ROWS(kBF16, kE5M2); }
   else { if (fmt == kE4M3) FALQON_ROWS(kF32, kE4M3); else FALQON_ROWS(kF32, kE5M2); }
 #undef FALQON_ROWS
-}
-
-cudaError_t launch_quantize_oa_transposed(const float* oa, const float* amax_oa, int64_t T, int64_t r, int64_t r16,
-                                          int64_t ldt, uint8_t* oaq_t, float* s_oa_out, float* amax_copy,
-                                          cudaStream_t stream) {
-  (void)r16;
-  const int grid = static_cast<int>((T + kOaTileT - 1) / kOaTileT);
-  return launch_pdl(quantize_oa_transposed_kernel, dim3(grid), dim3(256), 0, stream, 1, oa, amax_oa, T, static_cast<int>(r),
-                    ldt, oaq_t, s_oa_out, amax_copy);
 }
 
 }  // namespace falqon
