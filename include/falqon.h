@@ -133,6 +133,16 @@ int falqon_melded_forward(const falqon_layer *L, const void *X, falqon_dtype x_d
                           falqon_dtype y_dt, float *OA, float *amax_oa, float *s_x_out, void *ws,
                           size_t ws_bytes, falqon_stream stream);
 
+/* The product of the melded forward alone, for inputs that are already quantized: several layers that read the
+ * same activations (the q, k and v projections of a block; gate and up) share one x~.
+ *   xq   device [T][n] E4M3 codes, e.g. the FALQON_WS_XQ region of the workspace of the layer that ran
+ *        falqon_melded_forward on the same X
+ *   s_x  device [1], the scale the codes were cast with (entry 1 of that workspace's FALQON_WS_SCALES)
+ * Everything else as falqon_melded_forward; this call's workspace holds no x~ afterwards. */
+int falqon_melded_forward_codes(const falqon_layer *L, const uint8_t *xq, const float *s_x, int64_t T, void *Y,
+                                falqon_dtype y_dt, float *OA, float *amax_oa, void *ws, size_t ws_bytes,
+                                falqon_stream stream);
+
 /* Backward (Alg. 3 line 3 with Eq. lora_backward_modified, plus the input gradient the chain rule
  * implies for O = W~ x~ / (s_W s_x)):   g~, s_g = Q_e5m2(dY);   O~_A, s_OA = Q_e4m3(O_A);
  *   dX = g~ * W~ / (s_W * s_g)            (first m rows of W~' only; skipped when dX is NULL)

@@ -21,6 +21,7 @@ PER_TENSOR, PER_ROW = 0, 1
 WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 
 EXPORTS = ["falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
+           "falqon_melded_forward_codes",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_last_device_status", "falqon_launch_count",
            "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static", "falqon_workspace_init", "falqon_proxy_update_adamw"]
 STATIC_MAX_ROWS = 16384
@@ -49,6 +50,8 @@ lib.falqon_quantize.restype = _i
 lib.falqon_quantize.argtypes = [_p, _i, _i64, _i64, _i, _i, _p, _f, _p, _p, _p, _p, _sz, _p]
 lib.falqon_melded_forward.restype = _i
 lib.falqon_melded_forward.argtypes = [C.POINTER(falqon_layer), _p, _i, _i64, _p, _i, _p, _p, _p, _p, _sz, _p]
+lib.falqon_melded_forward_codes.restype = _i
+lib.falqon_melded_forward_codes.argtypes = [C.POINTER(falqon_layer), _p, _p, _i64, _p, _i, _p, _p, _p, _sz, _p]
 lib.falqon_melded_backward.restype = _i
 lib.falqon_melded_backward.argtypes = [C.POINTER(falqon_layer), _p, _i, _i64, _p, _p, _p, _i, _p, _p, _p, _sz, _p]
 lib.falqon_proxy_update.restype = _i
@@ -201,6 +204,27 @@ def melded_forward(layer: Layer, X: torch.Tensor, y_dtype=torch.bfloat16, ws: to
                                                               _ptr(OA), _ptr(amax_oa), _ptr(s_x), _ptr(ws), ws.numel(),
                                                               _stream()))
     return Y, OA, amax_oa, s_x
+
+
+def melded_forward_codes(layer: Layer, xq: torch.Tensor, s_x: torch.Tensor, y_dtype=torch.bfloat16,
+                         ws: torch.Tensor | None = None, out=None):
+    """falqon_melded_forward_codes: the forward product on activations another layer already quantized
+    (xq uint8 [T, n], s_x fp32 [1]).  Returns (Y [T, m], OA fp32 [T, r], amax_oa fp32 [1])."""
+    assert xq.dim() == 2 and xq.is_contiguous() and xq.shape[1] == layer.n and xq.dtype == torch.uint8
+    assert s_x.dtype == torch.float32 and s_x.numel() == 1
+    T = xq.shape[0]
+    dev = xq.device
+    ws = layer.workspace(T) if ws is None else ws
+    if out is None:
+        Y = torch.empty((T, layer.m), dtype=y_dtype, device=dev)
+        OA = torch.empty((T, layer.r), dtype=torch.float32, device=dev)
+        amax_oa = torch.empty(1, dtype=torch.float32, device=dev)
+    else:
+        Y, OA, amax_oa = out
+    _check("falqon_melded_forward_codes", lib.falqon_melded_forward_codes(C.byref(layer.c), _ptr(xq), _ptr(s_x), T, _ptr(Y),
+                                                                          _dt(Y), _ptr(OA), _ptr(amax_oa), _ptr(ws),
+                                                                          ws.numel(), _stream()))
+    return Y, OA, amax_oa
 
 
 def melded_backward(layer: Layer, dY: torch.Tensor, OA: torch.Tensor, amax_oa: torch.Tensor, need_dx: bool = True,

@@ -108,6 +108,29 @@ struct StageTimer {
   }
 };
 
+// S2: [Y | O_A] = x~ W~'^T / (s_W s_x), amax(O_A) from the epilogue (which accumulates into *amax_oa: zero beforehand)
+int forward_product(const falqon_layer* L, const uint8_t* xq, const float* s_x, int64_t T, void* Y, int y_dt, float* OA,
+                    float* amax_oa, uint8_t* base, const WorkspaceLayout& w, int* status, cudaStream_t stream) {
+  const int64_t m = L->m, n = L->n, r = L->r;
+  const bool per_row = L->gran == FALQON_PER_ROW;
+  float* col_scale = reinterpret_cast<float*>(base + w.col_scale);
+  if (per_row)   // epilogue factors 1 / (s_w[column] * s_x); s_w[m] serves the O_A columns
+    FALQON_CUDA(launch_scale_table(1, L->s_w, m, r, s_x, col_scale, w.col_scale_len, stream));
+  GemmProblem g{};
+  g.M = T; g.N = m + r; g.K = n;
+  g.a = xq; g.lda = n; g.a_fmt = kE4M3;
+  g.b = L->wq; g.ldb = n; g.b_mn_major = false; g.b_fmt = kE4M3;
+  g.block_n = 256;
+  g.c0 = Y; g.ldc0 = m; g.c0_dt = y_dt; g.n_split = m;
+  g.c1 = OA; g.ldc1 = r; g.amax1_bits = reinterpret_cast<uint32_t*>(amax_oa);
+  g.scale_a = per_row ? nullptr : s_x; g.scale_b = per_row ? nullptr : L->s_w;
+  g.col_scale = per_row ? col_scale : nullptr;
+  g.status = status;
+  StageTimer timer(FALQON_STAGE_GEMM_FWD, stream);
+  FALQON_CUDA(launch_gemm_fp8(g, stream));
+  return FALQON_OK;
+}
+
 }  // namespace
 }  // namespace falqon
 
@@ -191,7 +214,7 @@ int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_d
   uint8_t* base = static_cast<uint8_t*>(ws);
   float* scales = reinterpret_cast<float*>(base + w.scales);
   uint8_t* xq = base + w.act8;
-  const int64_t m = L->m, n = L->n, r = L->r;
+  const int64_t n = L->n;
 
   // S1: x~, s_x = Q_e4m3(X); the cast also clears amax(O_A), which the product's epilogue accumulates
   uint32_t* partial = reinterpret_cast<uint32_t*>(base + w.scales + kPartialsOffset);
@@ -200,26 +223,21 @@ int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_d
     FALQON_CUDA(launch_quantize_fused(X, x_dt, T * n, kE4M3, xq, partial, base + w.scales + kSyncOffset, scales + 1, s_x_out,
                                       scales + 0, amax_oa, status, nullptr, 0, nullptr, stream));
   }
-  const bool per_row = L->gran == FALQON_PER_ROW;
-  float* col_scale = reinterpret_cast<float*>(base + w.col_scale);
-  if (per_row)   // epilogue factors 1 / (s_w[column] * s_x); s_w[m] serves the O_A columns
-    FALQON_CUDA(launch_scale_table(1, L->s_w, m, r, scales + 1, col_scale, w.col_scale_len, stream));
-  // S2: [Y | O_A] = x~ W~'^T / (s_W s_x), amax(O_A) from the epilogue
-  GemmProblem g{};
-  g.M = T; g.N = m + r; g.K = n;
-  g.a = xq; g.lda = n; g.a_fmt = kE4M3;
-  g.b = L->wq; g.ldb = n; g.b_mn_major = false; g.b_fmt = kE4M3;
-  g.block_n = 256;
-  g.c0 = Y; g.ldc0 = m; g.c0_dt = y_dt; g.n_split = m;
-  g.c1 = OA; g.ldc1 = r; g.amax1_bits = reinterpret_cast<uint32_t*>(amax_oa);
-  g.scale_a = per_row ? nullptr : scales + 1; g.scale_b = per_row ? nullptr : L->s_w;
-  g.col_scale = per_row ? col_scale : nullptr;
-  g.status = status;
-  {
-    StageTimer timer(FALQON_STAGE_GEMM_FWD, stream);
-    FALQON_CUDA(launch_gemm_fp8(g, stream));
-  }
-  return FALQON_OK;
+  return forward_product(L, xq, scales + 1, T, Y, y_dt, OA, amax_oa, base, w, status, stream);
+}
+
+int falqon_melded_forward_codes(const falqon_layer* L, const uint8_t* xq, const float* s_x, int64_t T, void* Y,
+                                falqon_dtype y_dt, float* OA, float* amax_oa, void* ws, size_t ws_bytes, falqon_stream stream) {
+  if (!layer_ok(L) || xq == nullptr || s_x == nullptr || Y == nullptr || OA == nullptr || amax_oa == nullptr || T < 1 ||
+      !dtype_ok(y_dt) || !aligned16(xq) || !aligned16(Y) || !aligned16(OA))
+    return FALQON_ERR_INVALID_ARG;
+  WorkspaceLayout w;
+  if (!make_layout(L->m, L->n, L->r, T, &w)) return FALQON_ERR_INVALID_ARG;
+  if (ws == nullptr || !aligned16(ws) || ws_bytes < w.total) return FALQON_ERR_WORKSPACE;
+  int* status = status_ptr();
+  if (status == nullptr) return FALQON_ERR_CUDA;
+  FALQON_CUDA(cudaMemsetAsync(amax_oa, 0, sizeof(float), stream));   // the product's epilogue accumulates a max into it
+  return forward_product(L, xq, s_x, T, Y, y_dt, OA, amax_oa, static_cast<uint8_t*>(ws), w, status, stream);
 }
 
 int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, int64_t T, const float* OA,

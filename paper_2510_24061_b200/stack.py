@@ -1,0 +1,241 @@
+"""A chain of decoder-shaped blocks built from melded FP8-LoRA linear layers: the workload of the "32-layer stack"
+configuration.  It exists to run the layer in the launch pattern of a training step -- seven projections per block,
+q/k/v and gate/up sharing one quantized input, each block's backward followed by its seven proxy updates -- not to
+model attention: the token mixing is a stand-in.
+
+Per block (T tokens, hidden H, MLP width F; every linear is a melded layer, everything between them is a bf16
+kernel of falqon_chain.h):
+    x1 = rmsnorm(h);   q, k, v = L_q(x1), L_k(x1), L_v(x1)      one shared x~
+    a  = (q + k + v) / sqrt(3)                                    stand-in for the attention mixing
+    h' = h + L_o(a)
+    x2 = rmsnorm(h');  g, u = L_gate(x2), L_up(x2)               one shared x~
+    z  = silu(g) * u
+    h_next = (h' + L_down(z)) / sqrt(2)
+Loss = <h_last, G>.  The backward mirrors this; kept for it per block are h, h' (for the norms), g, u (for the
+gate) and each projection's O_A -- the melded layer needs neither its input nor A for its gradients.  (Without the
+norms the gated MLP squares the scale of the residual stream in every block and bf16 overflows within a few.)
+
+Only argument marshalling and buffer bookkeeping happen here; every arithmetic step runs in the library's kernels.
+"""
+import ctypes as C
+import math
+
+import torch
+
+from . import binding as fq
+from . import synth
+
+lib = fq.lib
+_p, _f, _i64 = C.c_void_p, C.c_float, C.c_int64
+lib.falqon_chain_combine.restype = C.c_int
+lib.falqon_chain_combine.argtypes = [_p, _p, _f, _p, _f, _p, _f, _p, _f, _i64, _p]
+lib.falqon_chain_silu_mul.restype = C.c_int
+lib.falqon_chain_silu_mul.argtypes = [_p, _p, _p, _i64, _p]
+lib.falqon_chain_silu_mul_grad.restype = C.c_int
+lib.falqon_chain_silu_mul_grad.argtypes = [_p, _p, _p, _p, _p, _i64, _p]
+lib.falqon_chain_rmsnorm.restype = C.c_int
+lib.falqon_chain_rmsnorm.argtypes = [_p, _p, _p, _i64, _i64, _f, _p]
+lib.falqon_chain_rmsnorm_grad.restype = C.c_int
+lib.falqon_chain_rmsnorm_grad.argtypes = [_p, _p, _p, _p, _i64, _i64, _p]
+CHAIN_EXPORTS = ["falqon_chain_combine", "falqon_chain_silu_mul", "falqon_chain_silu_mul_grad", "falqon_chain_rmsnorm",
+                 "falqon_chain_rmsnorm_grad"]
+NORM_EPS = 1e-6
+
+PROJ = ["q", "k", "v", "o", "gate", "up", "down"]
+INV_SQRT3 = 1.0 / math.sqrt(3.0)
+INV_SQRT2 = 1.0 / math.sqrt(2.0)
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def combine(out, a, sa=1.0, b=None, sb=1.0, c=None, sc=1.0, d=None, sd=1.0):
+    """out = bf16(sa*a + sb*b + sc*c + sd*d); b, c, d optional."""
+    for t in (out, a, b, c, d):
+        assert t is None or (t.dtype == torch.bfloat16 and t.is_contiguous() and t.numel() == out.numel())
+    fq._check("falqon_chain_combine", lib.falqon_chain_combine(_ptr(out), _ptr(a), sa, _ptr(b), sb, _ptr(c), sc, _ptr(d), sd,
+                                                                out.numel(), fq._stream()))
+    return out
+
+
+def silu_mul(z, g, u):
+    for t in (z, g, u):
+        assert t.dtype == torch.bfloat16 and t.is_contiguous() and t.numel() == z.numel()
+    fq._check("falqon_chain_silu_mul", lib.falqon_chain_silu_mul(_ptr(z), _ptr(g), _ptr(u), z.numel(), fq._stream()))
+    return z
+
+
+def silu_mul_grad(dg, du, g, u, dz):
+    for t in (dg, du, g, u, dz):
+        assert t.dtype == torch.bfloat16 and t.is_contiguous() and t.numel() == g.numel()
+    fq._check("falqon_chain_silu_mul_grad", lib.falqon_chain_silu_mul_grad(_ptr(dg), _ptr(du), _ptr(g), _ptr(u), _ptr(dz),
+                                                                            g.numel(), fq._stream()))
+    return dg, du
+
+
+def rmsnorm(y, inv_rms, x):
+    assert x.dtype == torch.bfloat16 and x.dim() == 2 and x.is_contiguous() and y.shape == x.shape and y.is_contiguous()
+    assert inv_rms.dtype == torch.float32 and inv_rms.numel() == x.shape[0]
+    fq._check("falqon_chain_rmsnorm", lib.falqon_chain_rmsnorm(_ptr(y), _ptr(inv_rms), _ptr(x), x.shape[0], x.shape[1],
+                                                                NORM_EPS, fq._stream()))
+    return y
+
+
+def rmsnorm_grad(dx, dy, x, inv_rms):
+    for t in (dx, dy, x):
+        assert t.dtype == torch.bfloat16 and t.is_contiguous() and t.shape == x.shape
+    fq._check("falqon_chain_rmsnorm_grad", lib.falqon_chain_rmsnorm_grad(_ptr(dx), _ptr(dy), _ptr(x), _ptr(inv_rms), x.shape[0],
+                                                                          x.shape[1], fq._stream()))
+    return dx
+
+
+class Stack:
+    """n_layers blocks with hidden size H and MLP width F, T tokens per step, LoRA rank r, top-k rows per update."""
+
+    def __init__(self, n_layers: int, H: int, F: int, T: int, r: int, k: int, seed: int, device, lr: float = 2e-4):
+        self.n_layers, self.H, self.F, self.T, self.r, self.k, self.lr = n_layers, H, F, T, r, k, lr
+        self.device = torch.device(device)
+        self.seed = seed
+        self.shapes = {"q": (H, H), "k": (H, H), "v": (H, H), "o": (H, H), "gate": (H, F), "up": (H, F), "down": (F, H)}  # n -> m
+        self.layers = []
+        for l in range(n_layers):
+            block = {}
+            for pi, name in enumerate(PROJ):
+                n, m = self.shapes[name]
+                mat = l * len(PROJ) + pi
+                W = synth.backbone(seed, mat, m, n, self.device)
+                A = synth.adapter_a(seed, mat, r, n, self.device)
+                B = synth.adapter_b(seed, mat, m, r, self.device)
+                block[name] = fq.setup_layer(W, A, B, 1.0)
+                del W, A, B
+            self.layers.append(block)
+        dev, bf = self.device, torch.bfloat16
+        # one workspace per projection kind, shared by all blocks (the stream serialises their use)
+        self.ws = {}
+        for name in PROJ:
+            n, m = self.shapes[name]
+            self.ws[name] = torch.empty(fq.workspace_bytes(m, n, r, T), dtype=torch.uint8, device=dev)
+            fq.workspace_init(self.ws[name])
+        # saved for the backward, per block: h, h' and their row norms, g, u, and every projection's O_A (+ its amax)
+        self.saved = [dict(g=torch.empty((T, F), dtype=bf, device=dev), u=torch.empty((T, F), dtype=bf, device=dev),
+                           h=torch.empty((T, H), dtype=bf, device=dev), hp=torch.empty((T, H), dtype=bf, device=dev),
+                           inv1=torch.empty(T, dtype=torch.float32, device=dev),
+                           inv2=torch.empty(T, dtype=torch.float32, device=dev),
+                           oa={p: torch.empty((T, r), dtype=torch.float32, device=dev) for p in PROJ},
+                           amax={p: torch.empty(1, dtype=torch.float32, device=dev) for p in PROJ})
+                      for _ in range(n_layers)]
+        # transients, reused by every block
+        e = lambda cols: torch.empty((T, cols), dtype=bf, device=dev)
+        self.x1, self.x2 = e(H), e(H)
+        self.q, self.kk, self.v, self.a, self.o, self.dn = e(H), e(H), e(H), e(H), e(H), e(H)
+        self.h_out = e(H)
+        self.z = e(F)
+        self.dh, self.dhp, self.da, self.dqkv = e(H), e(H), e(H), e(H)
+        self.dx = [e(H), e(H), e(H)]
+        self.dz, self.dg, self.du, self.ddn = e(F), e(F), e(F), e(H)
+        self.s_x = torch.empty(1, dtype=torch.float32, device=dev)
+        self.s_g = torch.empty(1, dtype=torch.float32, device=dev)
+        self.dB = {p: torch.empty((self.shapes[p][1], r), dtype=torch.float32, device=dev) for p in PROJ}
+        self.idx = torch.empty(max(k, 1), dtype=torch.int32, device=dev)
+        self.capture = None   # optional: {(block, proj): dict} filled with references / copies for parity checks
+
+    # ---- one linear: forward on X (quantizing it) or on another projection's codes
+    def _fwd(self, l, name, X, Y):
+        sv = self.saved[l]
+        fq.melded_forward(self.layers[l][name], X, ws=self.ws[name], out=(Y, sv["oa"][name], sv["amax"][name], self.s_x))
+        self._cap(l, name, X=X, Y=Y)
+
+    def _fwd_shared(self, l, name, owner, X, Y):
+        n, _ = self.shapes[name]
+        lo = self.layers[l][owner]
+        xq = fq.ws_view(lo, self.ws[owner], self.T, fq.WS_XQ)[: self.T * n].view(self.T, n)
+        s_x = fq.ws_view(lo, self.ws[owner], self.T, fq.WS_SCALES).view(torch.float32)[1:2]
+        sv = self.saved[l]
+        fq.melded_forward_codes(self.layers[l][name], xq, s_x, ws=self.ws[name], out=(Y, sv["oa"][name], sv["amax"][name]))
+        self._cap(l, name, X=X, Y=Y)
+
+    def _bwd(self, l, name, dY, dX):
+        sv = self.saved[l]
+        fq.melded_backward(self.layers[l][name], dY, sv["oa"][name], sv["amax"][name], ws=self.ws[name],
+                           out=(dX, self.dB[name], self.s_g))
+        self._cap(l, name, dY=dY, dX=dX, dB=self.dB[name], OA=sv["oa"][name])
+        fq.proxy_update(self.layers[l][name], self.dB[name], self.lr, self.k, ws=self.ws[name],
+                        idx_out=self.idx if self.k > 0 else None)
+
+    def _cap(self, l, name, **tensors):
+        if self.capture is not None and (l, name) in self.capture:
+            self.capture[(l, name)].update({k2: v.clone() for k2, v in tensors.items()})
+
+    def forward(self, h0: torch.Tensor) -> torch.Tensor:
+        for l in range(self.n_layers):
+            sv = self.saved[l]
+            if l == 0:
+                sv["h"].copy_(h0)
+            h, hp = sv["h"], sv["hp"]
+            rmsnorm(self.x1, sv["inv1"], h)
+            self._fwd(l, "q", self.x1, self.q)
+            self._fwd_shared(l, "k", "q", self.x1, self.kk)
+            self._fwd_shared(l, "v", "q", self.x1, self.v)
+            combine(self.a, self.q, INV_SQRT3, self.kk, INV_SQRT3, self.v, INV_SQRT3)
+            self._fwd(l, "o", self.a, self.o)
+            combine(hp, h, 1.0, self.o, 1.0)
+            rmsnorm(self.x2, sv["inv2"], hp)
+            self._fwd(l, "gate", self.x2, sv["g"])
+            self._fwd_shared(l, "up", "gate", self.x2, sv["u"])
+            silu_mul(self.z, sv["g"], sv["u"])
+            self._fwd(l, "down", self.z, self.dn)
+            out = self.saved[l + 1]["h"] if l + 1 < self.n_layers else self.h_out   # the next block's saved input
+            combine(out, hp, INV_SQRT2, self.dn, INV_SQRT2)
+        return self.h_out
+
+    def backward(self, G: torch.Tensor):
+        """G = d loss / d h_last.  Each block's backward is followed at once by the proxy updates of its layers
+        (inside _bwd), as in the paper's training loop."""
+        dh = G
+        for l in reversed(range(self.n_layers)):
+            sv = self.saved[l]
+            combine(self.ddn, dh, INV_SQRT2)                                   # d(down output) = dh / sqrt(2)
+            self._bwd(l, "down", self.ddn, self.dz)
+            silu_mul_grad(self.dg, self.du, sv["g"], sv["u"], self.dz)
+            self._bwd(l, "gate", self.dg, self.dx[0])
+            self._bwd(l, "up", self.du, self.dx[1])
+            combine(self.dx[0], self.dx[0], 1.0, self.dx[1], 1.0)               # d x2
+            rmsnorm_grad(self.dx[1], self.dx[0], sv["hp"], sv["inv2"])
+            combine(self.dhp, dh, INV_SQRT2, self.dx[1], 1.0)                   # dh' = dh/sqrt(2) + norm'(d x2)
+            self._bwd(l, "o", self.dhp, self.da)
+            combine(self.dqkv, self.da, INV_SQRT3)                              # dq = dk = dv = da / sqrt(3)
+            self._bwd(l, "q", self.dqkv, self.dx[0])
+            self._bwd(l, "k", self.dqkv, self.dx[1])
+            self._bwd(l, "v", self.dqkv, self.dx[2])
+            combine(self.dx[0], self.dx[0], 1.0, self.dx[1], 1.0, self.dx[2], 1.0)   # d x1
+            rmsnorm_grad(self.dx[1], self.dx[0], sv["h"], sv["inv1"])
+            combine(self.dh, self.dhp, 1.0, self.dx[1], 1.0)
+            dh = self.dh
+        return dh
+
+    def step(self, h0: torch.Tensor, G: torch.Tensor):
+        h = self.forward(h0)
+        self.backward(G)
+        return h
+
+    # ---- bookkeeping for the benchmark line
+    def flops_per_step(self) -> float:
+        T, r = self.T, self.r
+        return float(self.n_layers * sum(2 * T * (n * (m + r) + m * n + m * r) for n, m in self.shapes.values()))
+
+    def launches_per_step(self) -> int:
+        per_block = 0
+        for name in PROJ:
+            shared = name in ("k", "v", "up")
+            per_block += (1 if shared else fq.launch_count("falqon_melded_forward"))   # codes: the product alone
+            per_block += fq.launch_count("falqon_melded_backward") + fq.launch_count("falqon_proxy_update", k=self.k)
+        per_block += 6 + 9   # chain kernels: forward 6 (2 norms, mix, 2 residuals, gate), backward 9
+        return per_block * self.n_layers
+
+    def bytes_resident(self) -> int:
+        tot = 0
+        for block in self.layers:
+            for L in block.values():
+                tot += L.wq.numel() + 4 * L.s_w.numel() + 4 * L.dbuf.numel()
+        return tot

@@ -25,6 +25,19 @@ def test_library_exports_every_declared_symbol(fq):
         assert hasattr(fq.lib, name), name
 
 
+def test_chain_header_symbols_are_exported(fq):
+    header = open(os.path.join(ROOT, "include", "falqon_chain.h")).read()
+    declared = set(re.findall(r"\b(falqon_chain_[a-z_]+)\s*\(", header))
+    from paper_2510_24061_b200 import stack
+    assert declared == set(stack.CHAIN_EXPORTS)
+    for name in declared:
+        assert hasattr(fq.lib, name), name
+    fake = 0x10000
+    assert fq.lib.falqon_chain_combine(fake, None, C.c_float(1), None, C.c_float(1), None, C.c_float(1), None, C.c_float(1),
+                                       64, None) == fq.ERR_INVALID_ARG
+    assert stack.lib.falqon_chain_rmsnorm(fake, fake, fake, 4, 12, C.c_float(1e-6), None) == fq.ERR_INVALID_ARG   # cols % 8
+
+
 def test_workspace_layout(fq):
     m, n, r, T = 4096, 4096, 64, 4096
     total = fq.workspace_bytes(m, n, r, T)

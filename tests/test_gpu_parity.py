@@ -218,6 +218,25 @@ def test_bf16_outputs_are_rounded_fp32_outputs(fq):
     assert torch.equal(dB, dB3)
 
 
+@pytest.mark.parametrize("per_row", [False, True])
+def test_forward_on_shared_codes_equals_forward(fq, per_row):
+    """Two layers that read the same activations (q and k of a block): the second one takes the first one's x~ and
+    s_x from its workspace and must produce what a forward of its own on X produces, bit for bit."""
+    m, n, r, T = 640, 1280, 64, 300
+    W1, A1, B1, X = layer_inputs(41, 0, m, n, r, T, 4)
+    W2, A2, B2, _ = layer_inputs(41, 1, m, n, r, T, 4)
+    first = fq.setup_layer(W1.to(DEV), A1.to(DEV), B1.to(DEV), 1.0, per_row=per_row)
+    second = fq.setup_layer(W2.to(DEV), A2.to(DEV), B2.to(DEV), 1.0, per_row=per_row)
+    ws1, ws2 = first.workspace(T), second.workspace(T)
+    fq.melded_forward(first, X.to(DEV), y_dtype=torch.float32, ws=ws1)
+    xq = fq.ws_view(first, ws1, T, fq.WS_XQ)[:T * n].reshape(T, n)
+    s_x = fq.ws_view(first, ws1, T, fq.WS_SCALES).view(torch.float32)[1:2]
+    Y_c, OA_c, amax_c = fq.melded_forward_codes(second, xq, s_x, y_dtype=torch.float32, ws=ws2)
+    Y, OA, amax, _ = fq.melded_forward(second, X.to(DEV), y_dtype=torch.float32, ws=ws2)
+    assert torch.equal(Y_c, Y) and torch.equal(OA_c, OA) and torch.equal(amax_c, amax)
+    assert fq.last_device_status() == 0
+
+
 def test_b_zero_leaves_plain_fp8_layer(fq):
     c = synth.config0()
     W, A, _, X = layer_inputs(0, 0, c["m"], c["n"], c["r"], c["T"], c["n_outliers"])

@@ -1,0 +1,163 @@
+"""GPU parity of the decoder-shaped chain of melded layers (the "32-layer stack" configuration).
+
+The element-wise chain kernels are checked against the same formulas in fp32 on the CPU.  Every checked
+projection inside the chain is teacher-forced like the single-layer tests: the oracle is fed the tensors the GPU
+actually saw at that point of the step (captured copies), so each stage is compared in isolation.  Outputs
+inside the chain are bf16, so tensor-core results are compared with the oracle's fp32 result at bf16 resolution:
+within one bf16 step of it, and equal to its bf16 rounding on all but a small fraction of elements.
+"""
+import numpy as np
+import pytest
+import torch
+
+from helpers import bits32, f32, rel_fro, u8
+from paper_2510_24061_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def fq():
+    from paper_2510_24061_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def st():
+    from paper_2510_24061_b200 import stack
+    return stack
+
+
+@pytest.fixture(scope="module")
+def orc():
+    from oracle import falqon_oracle
+    return falqon_oracle
+
+
+def _bf16_steps(a: torch.Tensor, b: torch.Tensor) -> torch.Tensor:
+    """Distance between two bf16 tensors in representable steps (monotone integer mapping of the bit patterns)."""
+    def key(t):
+        i = t.contiguous().view(torch.int16).to(torch.int32)
+        return torch.where(i < 0, -(i & 0x7FFF), i)
+    return (key(a) - key(b)).abs()
+
+
+def test_chain_elementwise_kernels(st):
+    torch.manual_seed(0)
+    n = 8 * 4099
+    a, b, c, d = [(torch.randn(n) * s).to(torch.bfloat16) for s in (1.0, 0.5, 2.0, 0.1)]
+    ad, bd, cd, dd = [t.to(DEV) for t in (a, b, c, d)]
+    out = torch.empty_like(ad)
+    st.combine(out, ad, 0.5, bd, -1.25, cd, 3.0 ** -0.5, dd, 1.0)
+    acc = a.double() * np.float32(0.5)
+    for s, t in ((np.float32(-1.25), b), (np.float32(3.0 ** -0.5), c), (np.float32(1.0), d)):
+        acc = (acc.float().double() + float(s) * t.double())      # fp32 fma chain: one rounding per step
+    ref = acc.float().to(torch.bfloat16)
+    assert int(_bf16_steps(out.cpu(), ref).max()) <= 1 and float((out.cpu() != ref).float().mean()) < 1e-3
+    st.combine(out, ad, 2.0 ** -0.5)
+    assert torch.equal(out.cpu(), (a.float() * np.float32(2.0 ** -0.5)).to(torch.bfloat16))
+    z = torch.empty_like(ad)
+    st.silu_mul(z, ad, bd)
+    ref = (a.float() * torch.sigmoid(a.float()) * b.float()).to(torch.bfloat16)
+    assert int(_bf16_steps(z.cpu(), ref).max()) <= 1 and float((z.cpu() != ref).float().mean()) < 2e-2
+    dg, du = torch.empty_like(ad), torch.empty_like(ad)
+    st.silu_mul_grad(dg, du, ad, bd, cd)
+    s = torch.sigmoid(a.float())
+    ref_u = (c.float() * a.float() * s).to(torch.bfloat16)
+    ref_g = (c.float() * b.float() * s * (1 + a.float() * (1 - s))).to(torch.bfloat16)
+    for got, ref in ((du, ref_u), (dg, ref_g)):
+        assert int(_bf16_steps(got.cpu(), ref).max()) <= 1 and float((got.cpu() != ref).float().mean()) < 2e-2
+
+
+def test_chain_rmsnorm_and_its_gradient(st):
+    torch.manual_seed(1)
+    rows, cols = 37, 8 * 131
+    x = (torch.randn(rows, cols) * 3.0).to(torch.bfloat16)
+    dy = torch.randn(rows, cols).to(torch.bfloat16)
+    y, inv = torch.empty_like(x, device=DEV), torch.empty(rows, dtype=torch.float32, device=DEV)
+    st.rmsnorm(y, inv, x.to(DEV))
+    xf = x.double()
+    inv_ref = 1.0 / torch.sqrt((xf * xf).mean(dim=1) + st.NORM_EPS)
+    assert torch.allclose(inv.cpu().double(), inv_ref, rtol=1e-5)
+    ref = (xf * inv_ref[:, None]).float().to(torch.bfloat16)
+    assert int(_bf16_steps(y.cpu(), ref).max()) <= 1 and float((y.cpu() != ref).float().mean()) < 1e-2
+    dx = torch.empty_like(y)
+    st.rmsnorm_grad(dx, dy.to(DEV), x.to(DEV), inv)
+    xh = xf * inv_ref[:, None]
+    ref = (inv_ref[:, None] * (dy.double() - xh * (dy.double() * xh).mean(dim=1, keepdim=True))).float().to(torch.bfloat16)
+    assert int(_bf16_steps(dx.cpu(), ref).max()) <= 1 and float((dx.cpu() != ref).float().mean()) < 1e-2
+    # against autograd of the same function
+    xa = x.double().requires_grad_(True)
+    (xa / torch.sqrt((xa * xa).mean(dim=1, keepdim=True) + st.NORM_EPS) * dy.double()).sum().backward()
+    assert torch.allclose(dx.cpu().double(), xa.grad, rtol=2e-2, atol=1e-3)
+
+
+def _close_bf16(gpu: torch.Tensor, ref_f32: np.ndarray, what: str):
+    """A bf16 tensor-core output against the oracle's fp32 result: every element within one bf16 step of the
+    oracle's value (plus a floor of 2e-5 of the tensor's rms for elements that cancel to almost nothing), and
+    the whole tensor within the rounding noise of bf16."""
+    got = gpu.detach().float().cpu().numpy().astype(np.float64)
+    ref = ref_f32.astype(np.float64)
+    rms = np.sqrt(np.mean(ref * ref))
+    assert np.all(np.abs(got - ref) <= np.abs(ref) * 2.0 ** -8 + 2e-5 * rms), f"{what}: element out of tolerance"
+    assert np.linalg.norm(got - ref) <= 2.0 ** -8 * np.linalg.norm(ref), f"{what}: tensor out of tolerance"
+    ref16 = torch.from_numpy(np.ascontiguousarray(ref_f32)).to(torch.bfloat16)
+    assert float((gpu.detach().cpu() != ref16).float().mean()) < 0.02, f"{what}: too many elements differ from the rounded oracle"
+
+
+def _check_projection(fq, orc, cap, layer, name, T, r, k, lr, n_rows):
+    """cap: what the GPU saw for this projection (X, Y, OA, dY, dX, dB, wq and dbuf before its update)."""
+    m, n = layer.m, layer.n
+    wq, s_w = u8(cap["wq"]), np.float32(f32(layer.s_w)[0])
+    rng = np.random.default_rng(5)
+    tsel = np.sort(rng.choice(T, min(n_rows, T), replace=False))
+    tdev = torch.from_numpy(tsel).to(DEV)
+    # S1 + S2 (for k, v, up the codes came from the neighbouring projection's cast of the same X)
+    xq_o, s_x_o, _ = orc.quantize(f32(cap["X"]), orc.E4M3)
+    rows_o = orc.forward_gemm(xq_o, s_x_o, wq, s_w, m, r, tsel=tsel)
+    _close_bf16(cap["Y"][tdev], rows_o[:, :m], f"{name} Y")
+    assert rel_fro(f32(cap["OA"][tdev]), rows_o[:, m:]) <= 2e-5, f"{name} OA"
+    # S3 + S4 + S5
+    gq_o, s_g_o, _ = orc.quantize(f32(cap["dY"]), orc.E5M2)
+    _close_bf16(cap["dX"][tdev], orc.dx_gemm(gq_o, s_g_o, wq, s_w, m, tsel=tsel), f"{name} dX")
+    oaq_o, s_oa_o, _ = orc.quantize(f32(cap["OA"]), orc.E4M3)
+    isel = np.sort(rng.choice(m, min(2 * n_rows, m), replace=False))
+    dB_o = orc.db_gemm(gq_o, s_g_o, oaq_o, s_oa_o, isel=isel)
+    dB_g = f32(cap["dB"][torch.from_numpy(isel).to(DEV)])
+    assert rel_fro(dB_g, dB_o) <= 2e-5, f"{name} dB"
+    # S6..S8, fed the GPU's own dB: bit-exact
+    wq_o, dbuf_o = wq.copy(), f32(cap["dbuf"]).copy()
+    orc.proxy_update(wq_o, dbuf_o, f32(cap["dB"]), lr, k, m, r)
+    assert np.array_equal(u8(layer.wq), wq_o), f"{name} merged rows"
+    assert np.array_equal(bits32(f32(layer.dbuf)), bits32(dbuf_o)), f"{name} DeltaBuffer"
+
+
+def _run_and_check(fq, st, orc, n_layers, H, F, T, r, k, check_blocks, n_rows):
+    stack = st.Stack(n_layers, H, F, T, r, k, seed=7, device=DEV, lr=2e-2)
+    h0 = synth.normal_bf16(7, 9001, (T, H), 1.0, DEV)
+    G = synth.normal_bf16(7, 9002, (T, H), 1.0e-2, DEV)
+    stack.capture = {(l, p): {} for l in check_blocks for p in st.PROJ}
+    # the layer state each checked projection starts from (one step: a layer is updated once, after its backward)
+    for (l, p), cap in stack.capture.items():
+        cap["wq"] = stack.layers[l][p].wq.clone()
+        cap["dbuf"] = stack.layers[l][p].dbuf.clone()
+    h = stack.step(h0, G)
+    torch.cuda.synchronize()
+    assert fq.last_device_status() == 0
+    assert bool(torch.isfinite(h.float()).all())
+    for (l, p), cap in stack.capture.items():
+        _check_projection(fq, orc, cap, stack.layers[l][p], f"block {l} {p}", T, r, k, 2e-2, n_rows)
+    return stack
+
+
+def test_small_stack_every_projection(fq, st, orc):
+    """Three blocks of a narrow chain, every projection of every block checked on all token rows."""
+    _run_and_check(fq, st, orc, 3, 256, 640, 192, 16, 8, check_blocks=[0, 1, 2], n_rows=192)
+
+
+def test_stack_7b_shapes_sampled(fq, st, orc):
+    """The 7B shapes (hidden 4096, MLP 11008, 4096 tokens, rank 64, top-256), 32 blocks in one step: the first, the
+    last and two other blocks are checked on sampled rows."""
+    stack = _run_and_check(fq, st, orc, 32, 4096, 11008, 4096, 64, 256, check_blocks=[0, 11, 22, 31], n_rows=24)
+    assert stack.flops_per_step() == pytest.approx(107.41e12, rel=1e-3)
