@@ -250,6 +250,61 @@ def run_sweep(args):
                               "hbm_peak_gbs": peaks["hbm"]}), flush=True)
 
 
+def run_stack(args):
+    """configs[2]: 32 decoder-shaped blocks of the 7B projection set, activations chained (see
+    paper_2510_24061_b200/stack.py), one training step = forward through all blocks, backward, and each block's
+    seven proxy updates right after its backward.  One JSON line: step ms, TFLOP/s over the algorithmic FLOP of the
+    224 melded layers, both peak fractions, memory in use."""
+    from paper_2510_24061_b200 import binding as fq
+    from paper_2510_24061_b200 import stack as st
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    cfg = synth.config1()
+    T, r, k, lr = cfg["T"], cfg["r"], cfg["k"], cfg["lr"]
+    H, F, n_layers = 4096, 11008, args.stack_layers
+    peaks = measured_peaks()
+    stack = st.Stack(n_layers, H, F, T, r, k, seed=cfg["seed"], device=dev, lr=lr)
+    h0 = synth.normal_bf16(cfg["seed"], 9001, (T, H), 1.0, dev)
+    G = synth.normal_bf16(cfg["seed"], 9002, (T, H), 1.0e-2, dev)
+    steps, warmup = max(1, min(args.steps, 20)), max(3, min(args.warmup, 5))
+    for _ in range(warmup):
+        stack.step(h0, G)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        stack.step(h0, G)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / steps
+    # forward alone and backward (+ updates) alone, same protocol
+    e0.record()
+    for _ in range(steps):
+        stack.forward(h0)
+    e1.record()
+    torch.cuda.synchronize()
+    ms_f = e0.elapsed_time(e1) / steps
+    flops = stack.flops_per_step()
+    tf = flops / (ms * 1e-3) / 1e12
+    print(json.dumps({
+        "metric": METRIC, "value": tf, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warmup, "ms_per_step": ms,
+        "forward_ms": ms_f, "backward_and_updates_ms": ms - ms_f, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "fp8", "data": "synthetic",
+        "config": {"workload": f"configs[2]: {n_layers} chained blocks of the LLaMA-7B projection set, tokens=4096, rank=64, "
+                               "top-k=256, q/k/v and gate/up share one quantized input, bf16 chain kernels between the layers",
+                   "tokens": T, "rank": r, "topk": k, "matrices": 7 * n_layers, "tflop_per_step": flops / 1e12,
+                   "l2": "working set far larger than L2 (every step touches the whole stack)", "parallelism": "single GPU"},
+        "clocks": clocks, "gpu_launches": stack.launches_per_step() * steps,
+        "frac_of_fp8_peak": {"of_measured_sustained_x2": tf / (peaks["bf16_sustained"] * FP8_OVER_BF16),
+                             "of_nominal_4500": tf / 4500.0},
+        "memory": {"layers_bytes": stack.bytes_resident(), "allocated_bytes": torch.cuda.memory_allocated(dev),
+                   "peak_allocated_bytes": torch.cuda.max_memory_allocated(dev)},
+        "device_status": fq.last_device_status()}))
+
+
 def peaks_clock_ghz():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
@@ -268,6 +323,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true",
                     help="configs[4]: sweep rank x tokens x top-k on the 4096->11008 projection; one JSON line per point")
+    ap.add_argument("--stack", action="store_true",
+                    help="configs[2]: the 32-block chained stack of the 7B projection set; one JSON line")
+    ap.add_argument("--stack-layers", type=int, default=32)
     ap.add_argument("--only", default=None, help="profiling aid: restrict the workload to one projection (q,k,v,o,gate,up,down)")
     args = ap.parse_args()
 
@@ -288,6 +346,10 @@ def main():
     if args.sweep:
         if rank == 0:
             run_sweep(args)
+        return
+    if args.stack:
+        if rank == 0:
+            run_stack(args)
         return
 
     if args.impl == "reference":
