@@ -163,6 +163,12 @@ def test_more_tiles_than_cta_pairs_all_stages(fq, orc, m, n, r, T, k):
     _run_layer_stages(fq, orc, 29, m, n, r, T, k, 1.0, 3, 2, 2e-2)
 
 
+@pytest.mark.parametrize("T", [1, 5, 17])
+def test_a_handful_of_tokens(fq, orc, T):
+    """Fewer tokens than one tile row, than one 16-byte vector of codes, than one k-block of the adapter gradient."""
+    _run_layer_stages(fq, orc, 37, 272, 208, 24, T, 9, 1.0, 2, 2, 2e-2)
+
+
 @pytest.mark.parametrize("per_row", [False, True])
 def test_fp32_inputs_larger_than_the_staging_ring(fq, orc, per_row):
     """fp32 activations and output gradients of 49 MB each: more than the fused quantizer keeps on chip, so part
@@ -329,9 +335,10 @@ def test_config3_projection_sampled_per_row(fq, orc, name, n, m):
                         heavy_tailed=True)
 
 
-@pytest.mark.parametrize("r,T,k", [(8, 512, 4096), (128, 2048, 64), (32, 512, 0)])
+@pytest.mark.parametrize("r,T,k", [(8, 512, 4096), (128, 2048, 64), (32, 512, 0), (128, 32768, 4096)])
 def test_config4_sweep_corner_shapes(fq, orc, r, T, k):
-    """Corners of the rank x tokens x top-k sweep on the 4096 -> 11008 projection."""
+    """Corners of the rank x tokens x top-k sweep on the 4096 -> 11008 projection (the last one is its largest point:
+    268 MB of activations, 721 MB of output gradients, 2.1 G fma in the merge)."""
     if k == 0:
         _run_layer_stages(fq, orc, 0, 11008, 4096, r, T, 0, 1.0, 41, 1, 2e-4)
     else:
