@@ -118,7 +118,6 @@ cudaError_t launch_db_fused(const DbFusedProblem& p, cudaStream_t stream);
 cudaError_t launch_sgd_score(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, float* score,
                              cudaStream_t stream);
 // The k selected rows (ascending) are written to sel_idx and, when idx_copy is non-null, to idx_copy (int32 [k]).
-size_t topk_scratch_bytes(int64_t m);
 cudaError_t launch_topk(const float* score, int64_t m, int64_t k, int32_t* sel_idx, void* idx_copy, cudaStream_t stream);
 cudaError_t launch_merge_rows(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
                               int64_t r, cudaStream_t stream);

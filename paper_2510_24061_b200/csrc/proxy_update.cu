@@ -450,8 +450,6 @@ cudaError_t launch_sgd_score(float* dbuf, const float* dB, float lr, int64_t m, 
   return launch_pdl(sgd_score_kernel, dim3(grid), dim3(256), smem, stream, 1, dbuf, dB, -lr, m, static_cast<int>(r), score);
 }
 
-size_t topk_scratch_bytes(int64_t m) { (void)m; return 256; }
-
 cudaError_t launch_topk(const float* score, int64_t m, int64_t k, int32_t* sel_idx, void* idx_copy, cudaStream_t stream) {
   const int use_smem = m <= kTopkSmemRows ? 1 : 0;
   const size_t smem = use_smem ? static_cast<size_t>(m) * sizeof(uint32_t) : 0;

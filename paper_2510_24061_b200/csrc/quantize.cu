@@ -249,6 +249,24 @@ __device__ __forceinline__ void cast_oa_transposed(const OaCastJob& job) {
   }
 }
 
+// Casts the elements of one 16-byte unit (element index e of the tensor) and stores their codes.
+template <int kDt, int kFmt, bool kColMul>
+__device__ __forceinline__ void cast_unit(const uint4& q, int64_t e, const float* col_mul, int cols, float sc, uint8_t* dst) {
+  constexpr int kUnit = Unit<kDt>::kElems;
+  float x[kUnit];
+  unit_values<kDt, kColMul>(q, col_mul, kColMul ? static_cast<int>(e % cols) : 0, x);
+#pragma unroll
+  for (int k = 0; k < kUnit; ++k) x[k] = __fmul_rn(x[k], sc);
+  if (kDt == kBF16) {
+    uint2 o;
+    o.x = cvt_fp8x4<kFmt>(x[0], x[1], x[2], x[3]);
+    o.y = cvt_fp8x4<kFmt>(x[kUnit - 4], x[kUnit - 3], x[kUnit - 2], x[kUnit - 1]);
+    *reinterpret_cast<uint2*>(dst + e) = o;
+  } else {
+    *reinterpret_cast<uint32_t*>(dst + e) = cvt_fp8x4<kFmt>(x[0], x[1], x[2], x[3]);
+  }
+}
+
 template <int kDt, int kFmt, bool kColMul>
 __global__ void __launch_bounds__(kStagedThreads, 1)
 quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* partial, GridSync* sync, CastOutputs out,
@@ -363,20 +381,15 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
       const int64_t e0 = chunk_of(i) * kChunkElems;
       const int units = chunk_elems(chunk_of(i)) / kUnit;
       const uint4* sp = reinterpret_cast<const uint4*>(stage + s * kChunkBytes);
-      for (int u = tid; u < units; u += kStagedThreads) {
-        float x[kUnit];
-        const int64_t e = e0 + static_cast<int64_t>(u) * kUnit;
-        unit_values<kDt, kColMul>(sp[u], col_mul, kColMul ? static_cast<int>(e % cols) : 0, x);
-#pragma unroll
-        for (int k = 0; k < kUnit; ++k) x[k] = __fmul_rn(x[k], sc);
-        if (kDt == kBF16) {
-          uint2 o;
-          o.x = cvt_fp8x4<kFmt>(x[0], x[1], x[2], x[3]);
-          o.y = cvt_fp8x4<kFmt>(x[kUnit - 4], x[kUnit - 3], x[kUnit - 2], x[kUnit - 1]);
-          *reinterpret_cast<uint2*>(dst + e) = o;
-        } else {
-          *reinterpret_cast<uint32_t*>(dst + e) = cvt_fp8x4<kFmt>(x[0], x[1], x[2], x[3]);
-        }
+      // two units per thread and iteration (a full chunk is exactly one iteration): both shared-memory loads are
+      // issued before either conversion chain starts
+      for (int u = tid; u < units; u += 2 * kStagedThreads) {
+        const int u1 = u + kStagedThreads;
+        const bool has1 = u1 < units;
+        const uint4 q0 = sp[u];
+        const uint4 q1 = has1 ? sp[u1] : make_uint4(0u, 0u, 0u, 0u);
+        cast_unit<kDt, kFmt, kColMul>(q0, e0 + static_cast<int64_t>(u) * kUnit, col_mul, cols, sc, dst);
+        if (has1) cast_unit<kDt, kFmt, kColMul>(q1, e0 + static_cast<int64_t>(u1) * kUnit, col_mul, cols, sc, dst);
       }
       if (t + kStagedSlots < n_my) {
         if (!__syncthreads_and(ok)) { failed = true; break; }
