@@ -137,6 +137,70 @@ inline float scale_from_amax(float amax, int fmt) {
   return s;
 }
 
+// ---- exact merge arithmetic (the correctly rounded variant of the merge, an extension beyond the paper's text):
+// every E4M3 value is an integer multiple of 2^-9 and every fp32 value an integer multiple of 2^-149, so each term
+// DeltaBuffer * A~ and the backbone code itself are integer multiples of 2^-158.  The sum is held exactly as a big
+// integer in that unit (radix 2^32 digits in 64-bit bins, so hundreds of terms can be added before a carry pass),
+// and rounded ONCE to E4M3: nearest, ties to the even code, saturating at +-448; a sum that rounds to zero keeps
+// its sign, an exact zero is +0.
+struct ExactSum {
+  static constexpr int kBins = 12;       // 384 bits: 2^-158 .. beyond 2^127 * 2^18
+  int64_t bin[kBins];
+  ExactSum() { for (int i = 0; i < kBins; ++i) bin[i] = 0; }
+  // adds p * 2^shift (in units of 2^-158); |p| < 2^62, shift >= 0
+  void add_shifted(int64_t p, int shift) {
+    const int k = shift >> 5, t = shift & 31;
+    const __int128 v = (__int128)p << t;
+    bin[k] += (int64_t)(uint64_t)((unsigned __int128)v & 0xFFFFFFFFu);
+    bin[k + 1] += (int64_t)(uint64_t)(((unsigned __int128)v >> 32) & 0xFFFFFFFFu);
+    bin[k + 2] += (int64_t)(v >> 64);    // arithmetic shift: carries the sign
+  }
+  // d * (a_int * 2^-9) for an fp32 d (finite) and an E4M3 value a_int * 2^-9
+  void add_product(float d, int32_t a_int) {
+    uint32_t b;
+    std::memcpy(&b, &d, 4);
+    const int ef = (int)((b >> 23) & 0xFF);
+    const int64_t frac = (int64_t)(b & 0x7FFFFFu);
+    int64_t mant = ef == 0 ? frac : (frac | 0x800000);
+    const int e = ef == 0 ? -149 : ef - 150;          // d = +-mant * 2^e
+    if (b >> 31) mant = -mant;
+    if (mant == 0 || a_int == 0) return;
+    add_shifted(mant * (int64_t)a_int, e + 149);      // unit 2^-158 = 2^(e-9) / 2^(e+149)
+  }
+  void add_code_value(int32_t w_int) { if (w_int) add_shifted((int64_t)w_int, 149); }   // w_int * 2^-9
+  uint8_t round_to_e4m3() const {
+    int64_t d[kBins];
+    int64_t carry = 0;
+    for (int i = 0; i < kBins; ++i) {                 // normalise to digits in [0, 2^32), sign in the last carry
+      const int64_t t = bin[i] + carry;
+      d[i] = t & 0xFFFFFFFFll;
+      carry = t >> 32;                                 // arithmetic shift: floor division
+    }
+    const bool negative = carry < 0;                   // value = digits - 2^(32 kBins) when negative
+    if (negative) {                                    // magnitude = two's complement
+      int64_t c = 1;
+      for (int i = 0; i < kBins; ++i) { const int64_t t = (~d[i] & 0xFFFFFFFFll) + c; d[i] = t & 0xFFFFFFFFll; c = t >> 32; }
+    }
+    int top = -1;                                      // index of the highest set bit of the magnitude
+    for (int i = kBins - 1; i >= 0 && top < 0; --i)
+      if (d[i]) for (int bit = 31; bit >= 0; --bit) if ((d[i] >> bit) & 1) { top = i * 32 + bit; break; }
+    if (top < 0) return 0x00;                          // exact zero: +0
+    auto bit_at = [&](int pos) -> int { return pos < 0 ? 0 : (int)((d[pos >> 5] >> (pos & 31)) & 1); };
+    // quantum 2^q: 2^-9 (bit 149 of the unit) up to and including the binade [2^-6, 2^-5), then three bits below the top
+    const int q = std::max(149, top - 3);
+    int Q = 0;
+    for (int pos = top; pos >= q; --pos) Q = (Q << 1) | bit_at(pos);
+    const int half = bit_at(q - 1);
+    bool sticky = false;
+    for (int pos = q - 2; pos >= 0 && !sticky; --pos) sticky = bit_at(pos) != 0;
+    if (half && (sticky || (Q & 1))) ++Q;
+    double mag = std::ldexp((double)Q, q - 158);
+    if (mag > 448.0) mag = 448.0;
+    const uint8_t code = fp8_encode((float)mag, FMT_E4M3);     // exactly representable: no further rounding
+    return negative ? (uint8_t)(code | 0x80) : code;
+  }
+};
+
 struct DecodeTable {
   double v[256];
   explicit DecodeTable(int fmt) { for (int c = 0; c < 256; ++c) v[c] = fp8_decode((uint8_t)c, fmt); }
@@ -318,8 +382,9 @@ int orc_db_gemm(const uint8_t* gq, float s_g, const uint8_t* oaq, float s_oa, co
 // row_scales (nullable, m+1 entries): per-row mode.  The merge then works in row i's own scaled domain, where
 // A~ (scaled by s_w[m]) enters with the coefficient c_i = s_w[i] / s_w[m] (one fp32 division), applied to the
 // DeltaBuffer entry as its own rounded multiply before the chain.
-int orc_proxy_update(uint8_t* wq, float* dbuf, const float* dB, float lr, const float* row_scales,
-                     int64_t m, int64_t n, int64_t r, int64_t k, int32_t* idx_out, float* score_out) {
+static int proxy_update_impl(uint8_t* wq, float* dbuf, const float* dB, float lr, const float* row_scales,
+                             int64_t m, int64_t n, int64_t r, int64_t k, int32_t* idx_out, float* score_out,
+                             bool exact_merge) {
   if (k < 0 || k > m) return -1;
   const DecodeTable e4(FMT_E4M3);
   if (dB) {
@@ -345,6 +410,16 @@ int orc_proxy_update(uint8_t* wq, float* dbuf, const float* dB, float lr, const 
     const int64_t i = sel[s];
     const float coef = row_scales ? row_scales[i] / row_scales[m] : 1.0f;
     for (int64_t c = 0; c < n; ++c) {
+      if (exact_merge) {   // one rounding of the exact sum (the coefficient is still its own rounded fp32 multiply)
+        ExactSum acc;
+        acc.add_code_value((int32_t)std::lrint(e4.v[wq[i * n + c]] * 512.0));
+        for (int64_t j = 0; j < r; ++j) {
+          const float d = row_scales ? dbuf[i * r + j] * coef : dbuf[i * r + j];
+          acc.add_product(d, (int32_t)std::lrint(e4.v[aq[j * n + c]] * 512.0));
+        }
+        wq[i * n + c] = acc.round_to_e4m3();
+        continue;
+      }
       float v = (float)e4.v[wq[i * n + c]];
       for (int64_t j = 0; j < r; ++j) {
         const float d = row_scales ? dbuf[i * r + j] * coef : dbuf[i * r + j];
@@ -358,6 +433,28 @@ int orc_proxy_update(uint8_t* wq, float* dbuf, const float* dB, float lr, const 
     if (idx_out) idx_out[s] = (int32_t)sel[s];
   }
   return 0;
+}
+
+int orc_proxy_update(uint8_t* wq, float* dbuf, const float* dB, float lr, const float* row_scales,
+                     int64_t m, int64_t n, int64_t r, int64_t k, int32_t* idx_out, float* score_out) {
+  return proxy_update_impl(wq, dbuf, dB, lr, row_scales, m, n, r, k, idx_out, score_out, false);
+}
+
+// The same update with the correctly rounded merge: W~[i][c] <- sat_rne_e4m3(W~[i][c] + sum_j d'_ij * A~[j][c]) where
+// the sum is exact and rounded once (d'_ij = DeltaBuffer entry, times the row coefficient as its own fp32 multiply
+// in per-row mode).  Steps 1-3 and 5 are unchanged.
+int orc_proxy_update_exact(uint8_t* wq, float* dbuf, const float* dB, float lr, const float* row_scales,
+                           int64_t m, int64_t n, int64_t r, int64_t k, int32_t* idx_out, float* score_out) {
+  return proxy_update_impl(wq, dbuf, dB, lr, row_scales, m, n, r, k, idx_out, score_out, true);
+}
+
+// One exactly rounded dot product, for pins: code of sat_rne_e4m3(dec(w) + sum_j d[j] * dec(a[j])).
+uint8_t orc_exact_merge_element(uint8_t w, const float* d, const uint8_t* a, int64_t r) {
+  const DecodeTable e4(FMT_E4M3);
+  ExactSum acc;
+  acc.add_code_value((int32_t)std::lrint(e4.v[w] * 512.0));
+  for (int64_t j = 0; j < r; ++j) acc.add_product(d[j], (int32_t)std::lrint(e4.v[a[j]] * 512.0));
+  return acc.round_to_e4m3();
 }
 
 // AdamW on the DeltaBuffer (the optimizer the paper trains with; Alg. 3 line 4 leaves "Optimizer" generic).

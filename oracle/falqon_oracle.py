@@ -44,6 +44,10 @@ _lib.orc_db_gemm.restype = _i32
 _lib.orc_db_gemm.argtypes = [_p, _f32, _p, _f32, _p, _i64, _i64, _i64, _p, _i64, _p]
 _lib.orc_proxy_update.restype = _i32
 _lib.orc_proxy_update.argtypes = [_p, _p, _p, _f32, _p, _i64, _i64, _i64, _i64, _p, _p]
+_lib.orc_proxy_update_exact.restype = _i32
+_lib.orc_proxy_update_exact.argtypes = [_p, _p, _p, _f32, _p, _i64, _i64, _i64, _i64, _p, _p]
+_lib.orc_exact_merge_element.restype = C.c_uint8
+_lib.orc_exact_merge_element.argtypes = [C.c_uint8, _p, _p, _i64]
 _lib.orc_quantize_colscaled.restype = _i32
 _lib.orc_quantize_colscaled.argtypes = [_p, _i32, _i64, _i64, _i32, _p, _p, _p, _p]
 _lib.orc_adamw_step.restype = _i32
@@ -217,6 +221,31 @@ def proxy_update(wq, dbuf, dB, lr: float, k: int, m: int, r: int, row_scales=Non
     if rc != 0:
         raise ValueError("orc_proxy_update rejected its arguments")
     return idx, score
+
+
+def proxy_update_exact(wq, dbuf, dB, lr: float, k: int, m: int, r: int, row_scales=None):
+    """proxy_update with the correctly rounded merge (exact sum, one rounding to E4M3)."""
+    assert wq.dtype == np.uint8 and wq.flags.c_contiguous and wq.shape[0] == m + r
+    assert dbuf.dtype == np.float32 and dbuf.flags.c_contiguous and dbuf.shape == (m, r)
+    n = wq.shape[1]
+    g = None if dB is None else _c(dB, np.float32)
+    idx = np.empty(max(k, 0), dtype=np.int32)
+    score = np.empty(m, dtype=np.float32)
+    rs = None if row_scales is None else _c(row_scales, np.float32)
+    assert rs is None or rs.size == m + 1
+    rc = _lib.orc_proxy_update_exact(_ptr(wq), _ptr(dbuf), _ptr(g), float(np.float32(lr)), _ptr(rs), m, n, r, k, _ptr(idx),
+                                     _ptr(score))
+    if rc != 0:
+        raise ValueError("orc_proxy_update_exact rejected its arguments")
+    return idx, score
+
+
+def exact_merge_element(w: int, d, a) -> int:
+    """Code of sat_rne_e4m3(dec(w) + sum_j d[j] * dec(a[j])) with the sum exact (d float32, a uint8 codes)."""
+    d = _c(d, np.float32)
+    a = _c(a, np.uint8)
+    assert d.size == a.size
+    return int(_lib.orc_exact_merge_element(int(w), _ptr(d), _ptr(a), d.size))
 
 
 def adamw_step(p, g, exp_avg, exp_avg_sq, lr, beta1, beta2, eps, weight_decay, step: int):
