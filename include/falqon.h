@@ -202,6 +202,24 @@ int falqon_proxy_update_adamw(const falqon_layer *L, const float *dB, float *exp
 int falqon_proxy_update_static(const falqon_layer *L, const float *dB, float lr, int64_t k, int32_t *idx_out,
                                falqon_stream stream);
 
+/* The proxy update with a CORRECTLY ROUNDED merge (an extension: the paper does not fix the merge arithmetic, and
+ * falqon_proxy_update reads it as an fp32 fma chain).  Steps 1-3 (optimizer, scores, top-k) and the clearing are the
+ * same; the merge becomes
+ *     W~[i][c] <- sat_rne_e4m3( W~[i][c] + sum_j d'_ij * A~[j][c] )      sum exact, ONE rounding
+ * (nearest, ties to the even code, saturating at +-448; a sum that rounds to zero keeps its sign, an exact zero is
+ * +0; d'_ij = DeltaBuffer entry, in per-row mode times s_w[i] / s_w[m] as its own fp32 multiply).  The sums are
+ * formed on the tensor cores from exact bf16 limbs; an element whose sum lies within the accumulation error bound of
+ * a rounding boundary is recomputed in exact integer arithmetic, so the result does not depend on summation order.
+ *   scratch        device, falqon_exact_merge_scratch_bytes(m, n, r) bytes, no initialisation needed
+ *   sums_out       device [k][n] fp32, nullable: the tensor-core sums before rounding (diagnostics)
+ *   fix_count_out  device [1], nullable: number of elements that took the exact path
+ * Other arguments and return values as falqon_proxy_update; FALQON_ERR_WORKSPACE also for a scratch that is too
+ * small. */
+size_t falqon_exact_merge_scratch_bytes(int64_t m, int64_t n, int64_t r);
+int falqon_proxy_update_exact(const falqon_layer *L, const float *dB, float lr, int64_t k, int32_t *idx_out, void *ws,
+                              size_t ws_bytes, void *scratch, size_t scratch_bytes, float *sums_out,
+                              uint32_t *fix_count_out, falqon_stream stream);
+
 /* Synchronizes `stream`, then returns and clears the device status word of the current device:
  * FALQON_OK, FALQON_ERR_TIMEOUT (a bounded device-side wait ran out; results of that call are
  * undefined) or FALQON_ERR_CUDA (the synchronize itself failed). */

@@ -21,7 +21,7 @@ PER_TENSOR, PER_ROW = 0, 1
 WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 
 EXPORTS = ["falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
-           "falqon_melded_forward_codes",
+           "falqon_melded_forward_codes", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_last_device_status", "falqon_launch_count",
            "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static", "falqon_workspace_init", "falqon_proxy_update_adamw"]
 STATIC_MAX_ROWS = 16384
@@ -63,6 +63,10 @@ class falqon_adamw(C.Structure):
 
 lib.falqon_proxy_update_adamw.restype = _i
 lib.falqon_proxy_update_adamw.argtypes = [C.POINTER(falqon_layer), _p, _p, _p, C.POINTER(falqon_adamw), _i64, _p, _p, _sz, _p]
+lib.falqon_exact_merge_scratch_bytes.restype = _sz
+lib.falqon_exact_merge_scratch_bytes.argtypes = [_i64, _i64, _i64]
+lib.falqon_proxy_update_exact.restype = _i
+lib.falqon_proxy_update_exact.argtypes = [C.POINTER(falqon_layer), _p, _f, _i64, _p, _p, _sz, _p, _sz, _p, _p, _p]
 lib.falqon_proxy_update_static.restype = _i
 lib.falqon_proxy_update_static.argtypes = [C.POINTER(falqon_layer), _p, _f, _i64, _p, _p]
 lib.falqon_last_device_status.restype = _i
@@ -256,6 +260,25 @@ def proxy_update(layer: Layer, dB: torch.Tensor | None, lr: float, k: int, ws: t
     _check("falqon_proxy_update", lib.falqon_proxy_update(C.byref(layer.c), _ptr(dB), lr, k, _ptr(idx_out), _ptr(ws),
                                                           ws.numel(), _stream()))
     return idx_out
+
+
+def proxy_update_exact(layer: Layer, dB: torch.Tensor | None, lr: float, k: int, ws: torch.Tensor | None = None,
+                       idx_out: torch.Tensor | None = None, scratch: torch.Tensor | None = None, want_sums: bool = False,
+                       want_count: bool = True):
+    """falqon_proxy_update_exact: the proxy update with the correctly rounded merge.  Returns (idx int32 [k] ascending,
+    number of elements that took the exact path as a device int32 [1] or None, the tensor-core sums fp32 [k, n] or None)."""
+    ws = layer.workspace(1) if ws is None else ws
+    dev = layer.wq.device
+    if idx_out is None and 0 < k <= layer.m:
+        idx_out = torch.empty(k, dtype=torch.int32, device=dev)
+    if scratch is None:
+        scratch = torch.empty(int(lib.falqon_exact_merge_scratch_bytes(layer.m, layer.n, layer.r)), dtype=torch.uint8, device=dev)
+    fixed = torch.zeros(1, dtype=torch.int32, device=dev) if want_count else None
+    sums = torch.empty((k, layer.n), dtype=torch.float32, device=dev) if want_sums and k > 0 else None
+    _check("falqon_proxy_update_exact",
+           lib.falqon_proxy_update_exact(C.byref(layer.c), _ptr(dB), lr, k, _ptr(idx_out), _ptr(ws), ws.numel(), _ptr(scratch),
+                                         scratch.numel(), _ptr(sums), _ptr(fixed), _stream()))
+    return idx_out, fixed, sums
 
 
 def setup_layer(W: torch.Tensor, A: torch.Tensor, B: torch.Tensor | None, gamma: float, per_row: bool = False) -> Layer:

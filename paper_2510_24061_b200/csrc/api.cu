@@ -301,8 +301,15 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
 
 namespace {
 // Shared tail of the two proxy-update entry points.  adamw == nullptr: plain SGD with `lr` (or no optimizer when dB is null).
+// exact != nullptr: the merge runs in its correctly rounded form with the caller's scratch.
+struct ExactMergeArgs {
+  void* scratch;
+  float* sums_out;
+  unsigned int* fix_count_out;
+};
 int proxy_update_impl(const falqon_layer* L, const float* dB, float lr, const falqon_adamw* adamw, float* exp_avg,
-                      float* exp_avg_sq, int64_t k, int32_t* idx_out, void* ws, size_t ws_bytes, falqon_stream stream) {
+                      float* exp_avg_sq, int64_t k, int32_t* idx_out, void* ws, size_t ws_bytes, falqon_stream stream,
+                      const ExactMergeArgs* exact = nullptr) {
   if (!layer_ok(L) || k < 0 || k > L->m || !(lr == lr) || (dB != nullptr && !aligned16(dB)))
     return FALQON_ERR_INVALID_ARG;
   WorkspaceLayout w;
@@ -327,7 +334,12 @@ int proxy_update_impl(const falqon_layer* L, const float* dB, float lr, const fa
   if (k > 0) {
     StageTimer timer(FALQON_STAGE_MERGE, stream);
     const float* row_scales = L->gran == FALQON_PER_ROW ? L->s_w : nullptr;
-    if (fused_merge) {
+    if (exact != nullptr) {
+      int* status = status_ptr();
+      if (status == nullptr) return FALQON_ERR_CUDA;
+      FALQON_CUDA(launch_merge_exact(L->wq, L->dbuf, sel, k, m, n, r, row_scales, exact->scratch, exact->sums_out,
+                                     exact->fix_count_out, status, stream));
+    } else if (fused_merge) {
       FALQON_CUDA(launch_merge_rows_fused(L->wq, L->dbuf, sel, k, m, n, r, group_counters, row_scales, stream));
     } else if (row_scales == nullptr) {
       FALQON_CUDA(launch_merge_rows(L->wq, L->dbuf, sel, k, m, n, r, stream));
@@ -353,6 +365,22 @@ int falqon_proxy_update_adamw(const falqon_layer* L, const float* dB, float* exp
       !(hp->beta2 >= 0.0f && hp->beta2 < 1.0f) || !(hp->eps >= 0.0f) || !(hp->weight_decay == hp->weight_decay))
     return FALQON_ERR_INVALID_ARG;
   return proxy_update_impl(L, dB, hp->lr, hp, exp_avg, exp_avg_sq, k, idx_out, ws, ws_bytes, stream);
+}
+
+size_t falqon_exact_merge_scratch_bytes(int64_t m, int64_t n, int64_t r) {
+  if (!shape_ok(m, n, r)) return 0;
+  return exact_merge_scratch_bytes(m, n, r);
+}
+
+int falqon_proxy_update_exact(const falqon_layer* L, const float* dB, float lr, int64_t k, int32_t* idx_out, void* ws,
+                              size_t ws_bytes, void* scratch, size_t scratch_bytes, float* sums_out, uint32_t* fix_count_out,
+                              falqon_stream stream) {
+  if (!layer_ok(L)) return FALQON_ERR_INVALID_ARG;
+  if (scratch == nullptr || !aligned16(scratch) || scratch_bytes < exact_merge_scratch_bytes(L->m, L->n, L->r))
+    return FALQON_ERR_WORKSPACE;
+  if (sums_out != nullptr && !aligned16(sums_out)) return FALQON_ERR_INVALID_ARG;
+  const ExactMergeArgs exact{scratch, sums_out, fix_count_out};
+  return proxy_update_impl(L, dB, lr, nullptr, nullptr, nullptr, k, idx_out, ws, ws_bytes, stream, &exact);
 }
 
 int falqon_last_device_status(falqon_stream stream) {

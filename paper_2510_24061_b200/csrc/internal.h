@@ -114,6 +114,15 @@ struct DbFusedProblem {
 };
 cudaError_t launch_db_fused(const DbFusedProblem& p, cudaStream_t stream);
 
+// ---- merge_exact.cu: the correctly rounded merge of the selected rows on the tensor cores (guard band + exact fallback).
+// scratch: exact_merge_scratch_bytes(m, n, r) bytes, no initialisation needed.  Clears the merged DeltaBuffer rows.
+// sums_out (nullable [k][n] fp32): the accumulated sums before rounding; fix_count_out (nullable device [1]): how many
+// elements went through the exact fallback.
+size_t exact_merge_scratch_bytes(int64_t m, int64_t n, int64_t r);
+cudaError_t launch_merge_exact(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n, int64_t r,
+                               const float* row_scales, void* scratch, float* sums_out, unsigned int* fix_count_out, int* status,
+                               cudaStream_t stream);
+
 // ---- proxy_update.cu
 cudaError_t launch_sgd_score(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, float* score,
                              cudaStream_t stream);
