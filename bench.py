@@ -259,10 +259,15 @@ def run_sweep(args):
         for k in topks:
             idx = torch.empty(max(k, 1), dtype=torch.int32, device=dev)
             t_p = timed(lambda: fq.proxy_update(layer, dB, 2e-4, k, ws=ws, idx_out=idx if k > 0 else None))
+            t_x = None
+            if k > 0:   # the same update with the correctly rounded merge on the tensor cores
+                scratch = torch.empty(int(fq.lib.falqon_exact_merge_scratch_bytes(m, n, r)), dtype=torch.uint8, device=dev)
+                t_x = timed(lambda: fq.proxy_update_exact(layer, dB, 2e-4, k, ws=ws, idx_out=idx, scratch=scratch, want_count=False))
+                del scratch
             bytes_p = 12.0 * m * r + 4.0 * m + k * (2.0 * n + 8.0 * r) + r * n   # optimizer+score pass, merged rows, A~ once
             fma = float(k) * n * r
             alu_peak = 148 * 128 * peaks_clock_ghz() * 1e9                    # fp32 fma per second
-            print(json.dumps({"sweep": "proxy", "n": n, "m": m, "rank": r, "topk": k, "proxy_ms": t_p,
+            print(json.dumps({"sweep": "proxy", "n": n, "m": m, "rank": r, "topk": k, "proxy_ms": t_p, "proxy_exact_merge_ms": t_x,
                               "algorithmic_gbs": bytes_p / t_p / 1e6, "frac_hbm_peak": bytes_p / t_p / 1e6 / peaks["hbm"],
                               "merge_gfma_per_s": fma / t_p / 1e6, "frac_fp32_fma_peak": fma / (t_p * 1e-3) / alu_peak,
                               "hbm_peak_gbs": peaks["hbm"]}), flush=True)
