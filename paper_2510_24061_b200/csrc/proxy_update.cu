@@ -47,32 +47,34 @@ __global__ void __launch_bounds__(256) sgd_score_kernel(float* dbuf, const float
 constexpr int kTopkThreads = 1024;
 constexpr int kTopkSmemRows = 48 * 1024;   // scores are staged in shared memory up to this many rows
 
-// Exclusive prefix sum of one int per thread over the whole CTA (any multiple of 32 threads up to 1024);
-// *total = CTA sum.
-__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums /* [32] */, int* total) {
+// Exclusive prefix sums of two ints per thread over the whole CTA (any multiple of 32 threads up to 1024), one pass of
+// synchronisation for both.
+__device__ __forceinline__ void block_exclusive_scan2(int a, int b, int* sums_a /* [32] */, int* sums_b /* [32] */, int& ex_a,
+                                                      int& ex_b) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nwarps = blockDim.x >> 5;
-  int incl = v;
+  int ia = a, ib = b;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-    if (lane >= o) incl += t;
+    const int ta = __shfl_up_sync(0xFFFFFFFFu, ia, o), tb = __shfl_up_sync(0xFFFFFFFFu, ib, o);
+    if (lane >= o) { ia += ta; ib += tb; }
   }
-  if (lane == 31) warp_sums[warp] = incl;
+  if (lane == 31) { sums_a[warp] = ia; sums_b[warp] = ib; }
   __syncthreads();
   if (warp == 0) {
-    const int w = lane < nwarps ? warp_sums[lane] : 0;
-    int wi = w;
+    const int wa = lane < nwarps ? sums_a[lane] : 0, wb = lane < nwarps ? sums_b[lane] : 0;
+    int xa = wa, xb = wb;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int t = __shfl_up_sync(0xFFFFFFFFu, wi, o);
-      if (lane >= o) wi += t;
+      const int ta = __shfl_up_sync(0xFFFFFFFFu, xa, o), tb = __shfl_up_sync(0xFFFFFFFFu, xb, o);
+      if (lane >= o) { xa += ta; xb += tb; }
     }
-    warp_sums[lane] = wi - w;                 // exclusive offset of each warp
-    if (lane == 31) *total = wi;
+    sums_a[lane] = xa - wa;
+    sums_b[lane] = xb - wb;
   }
   __syncthreads();
-  return warp_sums[warp] + incl - v;
+  ex_a = sums_a[warp] + ia - a;
+  ex_b = sums_b[warp] + ib - b;
 }
 
 // The whole selection, run by one CTA (all of its threads).  s_bits: shared-memory staging for the m scores, or
@@ -81,16 +83,20 @@ __device__ __forceinline__ void topk_block(const float* score, int m, int k, int
                                            int32_t* idx_out, uint32_t* s_bits) {
   __shared__ int hist[4][256];
   __shared__ int warp_sums_a[32], warp_sums_b[32];
-  __shared__ int s_total_a, s_total_b;
   __shared__ uint32_t s_digit[4], s_remaining[4];
   const uint32_t* gbits = reinterpret_cast<const uint32_t*>(score);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nthreads = blockDim.x;
 
   for (int i = tid; i < 4 * 256; i += nthreads) (&hist[0][0])[i] = 0;
-  if (s_bits != nullptr)
-    for (int i = tid; i < m; i += nthreads) s_bits[i] = __ldcg(gbits + i);
-  __syncthreads();
+  // the minimum and maximum are taken while the scores stream in (any assignment of elements to threads will do)
+  uint32_t lmin = 0xFFFFFFFFu, lmax = 0u;
+  for (int i = tid; i < m; i += nthreads) {
+    const uint32_t b = __ldcg(gbits + i);
+    if (s_bits != nullptr) s_bits[i] = b;
+    lmin = min(lmin, b);
+    lmax = max(lmax, b);
+  }
   const uint32_t* bits = s_bits != nullptr ? s_bits : gbits;
   const int E = (m + nthreads - 1) / nthreads;
   const int lo = min(tid * E, m), hi = min(lo + E, m);
@@ -98,8 +104,6 @@ __device__ __forceinline__ void topk_block(const float* score, int m, int k, int
   // The scores of a layer lie in a narrow range, so their top bits agree: find the highest bit in which any two
   // differ (from the CTA-wide min and max) and run the radix passes only over the bits from there down.  This
   // also keeps the first histogram from collapsing into one or two bins.
-  uint32_t lmin = 0xFFFFFFFFu, lmax = 0u;
-  for (int i = lo; i < hi; ++i) { const uint32_t b = bits[i]; lmin = min(lmin, b); lmax = max(lmax, b); }
   lmin = __reduce_min_sync(0xFFFFFFFFu, lmin);
   lmax = __reduce_max_sync(0xFFFFFFFFu, lmax);
   if (lane == 0) { warp_sums_a[warp] = static_cast<int>(lmin); warp_sums_b[warp] = static_cast<int>(lmax); }
@@ -156,19 +160,18 @@ __device__ __forceinline__ void topk_block(const float* score, int m, int k, int
   const uint32_t tau = prefix;                      // bit pattern of the k-th largest score
   const int take_eq = static_cast<int>(remaining);  // how many rows with score == tau are taken
 
-  int my_eq = 0;
-  for (int i = lo; i < hi; ++i) my_eq += (bits[i] == tau) ? 1 : 0;
-  int eq_rank = block_exclusive_scan(my_eq, warp_sums_a, &s_total_a);
-  int my_sel = 0;
-  {
-    int e = eq_rank;
-    for (int i = lo; i < hi; ++i) {
-      const uint32_t b = bits[i];
-      if (b > tau) ++my_sel;
-      else if (b == tau) { if (e < take_eq) ++my_sel; ++e; }
-    }
+  // index-ordered compaction with ONE scan: rows above tau that precede this thread's range, and rows equal to tau
+  // that precede it (of which the first take_eq overall are taken)
+  int my_gt = 0, my_eq = 0;
+  for (int i = lo; i < hi; ++i) {
+    const uint32_t b = bits[i];
+    my_gt += b > tau ? 1 : 0;
+    my_eq += b == tau ? 1 : 0;
   }
-  int pos = block_exclusive_scan(my_sel, warp_sums_b, &s_total_b);
+  int gt_before, eq_before;
+  block_exclusive_scan2(my_gt, my_eq, warp_sums_a, warp_sums_b, gt_before, eq_before);
+  int pos = gt_before + min(eq_before, take_eq);
+  int eq_rank = eq_before;
   for (int i = lo; i < hi; ++i) {
     const uint32_t b = bits[i];
     bool selected = b > tau;
