@@ -286,7 +286,7 @@ def run_stack(args):
     T, r, k, lr = cfg["T"], cfg["r"], cfg["k"], cfg["lr"]
     H, F, n_layers = 4096, 11008, args.stack_layers
     peaks = measured_peaks()
-    stack = st.Stack(n_layers, H, F, T, r, k, seed=cfg["seed"], device=dev, lr=lr)
+    stack = st.Stack(n_layers, H, F, T, r, k, seed=cfg["seed"], device=dev, lr=lr, producer_amax=not args.stack_own_absmax)
     h0 = synth.normal_bf16(cfg["seed"], 9001, (T, H), 1.0, dev)
     G = synth.normal_bf16(cfg["seed"], 9002, (T, H), 1.0e-2, dev)
     steps, warmup = max(1, min(args.steps, 20)), max(3, min(args.warmup, 5))
@@ -349,6 +349,8 @@ def main():
     ap.add_argument("--stack", action="store_true",
                     help="configs[2]: the 32-block chained stack of the 7B projection set; one JSON line")
     ap.add_argument("--stack-layers", type=int, default=32)
+    ap.add_argument("--stack-own-absmax", action="store_true",
+                    help="with --stack: every layer takes the absmax of its input itself (the chain kernels do not hand it over)")
     ap.add_argument("--only", default=None, help="profiling aid: restrict the workload to one projection (q,k,v,o,gate,up,down)")
     args = ap.parse_args()
 

@@ -133,6 +133,13 @@ int falqon_melded_forward(const falqon_layer *L, const void *X, falqon_dtype x_d
                           falqon_dtype y_dt, float *OA, float *amax_oa, float *s_x_out, void *ws,
                           size_t ws_bytes, falqon_stream stream);
 
+/* falqon_melded_forward for a caller that already knows amax_x = max |X| (device [1], fp32, exactly the maximum of the
+ * absolute values of the tensor as stored): the kernel that produced X took it on the way out.  The cast is then a
+ * single pass -- no absmax reduction, no grid-wide barrier.  Everything else as falqon_melded_forward. */
+int falqon_melded_forward_amax(const falqon_layer *L, const void *X, falqon_dtype x_dt, const float *amax_x, int64_t T,
+                               void *Y, falqon_dtype y_dt, float *OA, float *amax_oa, float *s_x_out, void *ws,
+                               size_t ws_bytes, falqon_stream stream);
+
 /* The product of the melded forward alone, for inputs that are already quantized: several layers that read the
  * same activations (the q, k and v projections of a block; gate and up) share one x~.
  *   xq   device [T][n] E4M3 codes, e.g. the FALQON_WS_XQ region of the workspace of the layer that ran
@@ -154,6 +161,12 @@ int falqon_melded_forward_codes(const falqon_layer *L, const uint8_t *xq, const 
 int falqon_melded_backward(const falqon_layer *L, const void *dY, falqon_dtype dy_dt, int64_t T,
                            const float *OA, const float *amax_oa, void *dX, falqon_dtype dx_dt, float *dB,
                            float *s_g_out, void *ws, size_t ws_bytes, falqon_stream stream);
+
+/* falqon_melded_backward for a caller that already knows amax_dy = max |dY| (device [1]); per-tensor layers only
+ * (FALQON_ERR_UNSUPPORTED for FALQON_PER_ROW, whose cast input is dY divided by the row scales). */
+int falqon_melded_backward_amax(const falqon_layer *L, const void *dY, falqon_dtype dy_dt, const float *amax_dy, int64_t T,
+                                const float *OA, const float *amax_oa, void *dX, falqon_dtype dx_dt, float *dB,
+                                float *s_g_out, void *ws, size_t ws_bytes, falqon_stream stream);
 
 /* Row-wise proxy update (Alg. 3 lines 4-6; Eq. update):
  *   DeltaBuffer <- fma(-lr, dB, DeltaBuffer)          (plain SGD form; skipped when dB is NULL, so a

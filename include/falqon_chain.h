@@ -4,7 +4,10 @@
  * Harness code: none of this is part of the paper's method, which is the linear layer alone (falqon.h).
  * Every tensor is a dense device array of `count` bf16 values, 16-byte aligned, count a multiple of 8;
  * arithmetic is fp32, results rounded to nearest even.  Calls are asynchronous on `stream` and return
- * FALQON_OK, FALQON_ERR_INVALID_ARG or FALQON_ERR_CUDA. */
+ * FALQON_OK, FALQON_ERR_INVALID_ARG or FALQON_ERR_CUDA.
+ * amax_out arguments (device [1] fp32, nullable): the kernel raises the word to the largest |value| it stored (an
+ * atomic max on the bit pattern, so the word must hold 0, or any lower bound >= 0, beforehand).  A melded layer that
+ * consumes the tensor can then skip its own absmax pass (falqon_melded_forward_amax / _backward_amax). */
 #ifndef FALQON_CHAIN_H
 #define FALQON_CHAIN_H
 
@@ -17,20 +20,20 @@ extern "C" {
 /* out = bf16(sa*a + sb*b + sc*c + sd*d), accumulated left to right with fma; b, c, d may be NULL (skipped).
  * out may alias any input. */
 int falqon_chain_combine(void *out, const void *a, float sa, const void *b, float sb, const void *c, float sc,
-                         const void *d, float sd, int64_t count, falqon_stream stream);
+                         const void *d, float sd, int64_t count, float *amax_out, falqon_stream stream);
 
 /* z = bf16(silu(g) * u), silu(x) = x / (1 + exp(-x)). */
-int falqon_chain_silu_mul(void *z, const void *g, const void *u, int64_t count, falqon_stream stream);
+int falqon_chain_silu_mul(void *z, const void *g, const void *u, int64_t count, float *amax_out, falqon_stream stream);
 
 /* Gradient of the above: with s = 1 / (1 + exp(-g)):  du = dz * g * s,  dg = dz * u * s * (1 + g * (1 - s)).
  * dg may alias g or dz, du may alias u. */
 int falqon_chain_silu_mul_grad(void *dg, void *du, const void *g, const void *u, const void *dz, int64_t count,
-                               falqon_stream stream);
+                               float *amax_dg, float *amax_du, falqon_stream stream);
 
 /* Per-row RMS normalisation without a gain: y[t][:] = bf16(x[t][:] * inv_rms[t]), inv_rms[t] = 1 / sqrt(mean(x[t][:]^2) + eps).
  * x, y: [rows][cols] bf16, cols a multiple of 8 and at most 16384; inv_rms: device [rows] fp32, kept for the gradient. */
 int falqon_chain_rmsnorm(void *y, float *inv_rms, const void *x, int64_t rows, int64_t cols, float eps,
-                         falqon_stream stream);
+                         float *amax_out, falqon_stream stream);
 
 /* Gradient of the above: with xh = x * inv_rms:  dx = inv_rms * (dy - xh * mean(dy * xh)), one row at a time. */
 int falqon_chain_rmsnorm_grad(void *dx, const void *dy, const void *x, const float *inv_rms, int64_t rows,

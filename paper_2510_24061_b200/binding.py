@@ -21,7 +21,7 @@ PER_TENSOR, PER_ROW = 0, 1
 WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 
 EXPORTS = ["falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
-           "falqon_melded_forward_codes", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
+           "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_last_device_status", "falqon_launch_count",
            "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static", "falqon_workspace_init", "falqon_proxy_update_adamw"]
 STATIC_MAX_ROWS = 16384
@@ -50,6 +50,10 @@ lib.falqon_quantize.restype = _i
 lib.falqon_quantize.argtypes = [_p, _i, _i64, _i64, _i, _i, _p, _f, _p, _p, _p, _p, _sz, _p]
 lib.falqon_melded_forward.restype = _i
 lib.falqon_melded_forward.argtypes = [C.POINTER(falqon_layer), _p, _i, _i64, _p, _i, _p, _p, _p, _p, _sz, _p]
+lib.falqon_melded_forward_amax.restype = _i
+lib.falqon_melded_forward_amax.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _i, _p, _p, _p, _p, _sz, _p]
+lib.falqon_melded_backward_amax.restype = _i
+lib.falqon_melded_backward_amax.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _p, _p, _i, _p, _p, _p, _sz, _p]
 lib.falqon_melded_forward_codes.restype = _i
 lib.falqon_melded_forward_codes.argtypes = [C.POINTER(falqon_layer), _p, _p, _i64, _p, _i, _p, _p, _p, _sz, _p]
 lib.falqon_melded_backward.restype = _i
@@ -191,8 +195,10 @@ def quantize(src: torch.Tensor, fmt: int, gran: int = PER_TENSOR, scale_in: torc
     return dst, scale_out, amax_out
 
 
-def melded_forward(layer: Layer, X: torch.Tensor, y_dtype=torch.bfloat16, ws: torch.Tensor | None = None, out=None):
-    """falqon_melded_forward.  Returns (Y [T, m], OA fp32 [T, r], amax_oa fp32 [1], s_x fp32 [1])."""
+def melded_forward(layer: Layer, X: torch.Tensor, y_dtype=torch.bfloat16, ws: torch.Tensor | None = None, out=None,
+                   amax_x: torch.Tensor | None = None):
+    """falqon_melded_forward (falqon_melded_forward_amax when amax_x, fp32 [1] = max |X|, is given).
+    Returns (Y [T, m], OA fp32 [T, r], amax_oa fp32 [1], s_x fp32 [1])."""
     assert X.dim() == 2 and X.is_contiguous() and X.shape[1] == layer.n
     T = X.shape[0]
     dev = X.device
@@ -204,6 +210,12 @@ def melded_forward(layer: Layer, X: torch.Tensor, y_dtype=torch.bfloat16, ws: to
         s_x = torch.empty(1, dtype=torch.float32, device=dev)
     else:
         Y, OA, amax_oa, s_x = out
+    if amax_x is not None:
+        assert amax_x.dtype == torch.float32 and amax_x.numel() == 1
+        _check("falqon_melded_forward_amax",
+               lib.falqon_melded_forward_amax(C.byref(layer.c), _ptr(X), _dt(X), _ptr(amax_x), T, _ptr(Y), _dt(Y), _ptr(OA),
+                                              _ptr(amax_oa), _ptr(s_x), _ptr(ws), ws.numel(), _stream()))
+        return Y, OA, amax_oa, s_x
     _check("falqon_melded_forward", lib.falqon_melded_forward(C.byref(layer.c), _ptr(X), _dt(X), T, _ptr(Y), _dt(Y),
                                                               _ptr(OA), _ptr(amax_oa), _ptr(s_x), _ptr(ws), ws.numel(),
                                                               _stream()))
@@ -232,8 +244,9 @@ def melded_forward_codes(layer: Layer, xq: torch.Tensor, s_x: torch.Tensor, y_dt
 
 
 def melded_backward(layer: Layer, dY: torch.Tensor, OA: torch.Tensor, amax_oa: torch.Tensor, need_dx: bool = True,
-                    dx_dtype=torch.bfloat16, ws: torch.Tensor | None = None, out=None):
-    """falqon_melded_backward.  Returns (dX [T, n] or None, dB fp32 [m, r], s_g fp32 [1])."""
+                    dx_dtype=torch.bfloat16, ws: torch.Tensor | None = None, out=None, amax_dy: torch.Tensor | None = None):
+    """falqon_melded_backward (falqon_melded_backward_amax when amax_dy, fp32 [1] = max |dY|, is given).
+    Returns (dX [T, n] or None, dB fp32 [m, r], s_g fp32 [1])."""
     assert dY.dim() == 2 and dY.is_contiguous() and dY.shape[1] == layer.m
     T = dY.shape[0]
     dev = dY.device
@@ -245,6 +258,12 @@ def melded_backward(layer: Layer, dY: torch.Tensor, OA: torch.Tensor, amax_oa: t
     else:
         dX, dB, s_g = out
     dx_dt = _dt(dX) if dX is not None else BF16
+    if amax_dy is not None:
+        assert amax_dy.dtype == torch.float32 and amax_dy.numel() == 1
+        _check("falqon_melded_backward_amax",
+               lib.falqon_melded_backward_amax(C.byref(layer.c), _ptr(dY), _dt(dY), _ptr(amax_dy), T, _ptr(OA), _ptr(amax_oa),
+                                               _ptr(dX), dx_dt, _ptr(dB), _ptr(s_g), _ptr(ws), ws.numel(), _stream()))
+        return dX, dB, s_g
     _check("falqon_melded_backward", lib.falqon_melded_backward(C.byref(layer.c), _ptr(dY), _dt(dY), T, _ptr(OA),
                                                                 _ptr(amax_oa), _ptr(dX), dx_dt, _ptr(dB), _ptr(s_g),
                                                                 _ptr(ws), ws.numel(), _stream()))

@@ -201,8 +201,11 @@ int falqon_workspace_init(void* ws, size_t ws_bytes, falqon_stream stream) {
   return FALQON_OK;
 }
 
-int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_dt, int64_t T, void* Y, falqon_dtype y_dt,
-                          float* OA, float* amax_oa, float* s_x_out, void* ws, size_t ws_bytes, falqon_stream stream) {
+namespace {
+// amax_x (nullable, device [1]): the caller already knows max |X| (the kernel that produced X took it), so the cast is a
+// single pass with no reduction and no grid barrier.
+int forward_impl(const falqon_layer* L, const void* X, falqon_dtype x_dt, const float* amax_x, int64_t T, void* Y,
+                 falqon_dtype y_dt, float* OA, float* amax_oa, float* s_x_out, void* ws, size_t ws_bytes, falqon_stream stream) {
   if (!layer_ok(L) || X == nullptr || Y == nullptr || OA == nullptr || amax_oa == nullptr || T < 1 || !dtype_ok(x_dt) ||
       !dtype_ok(y_dt) || !aligned16(X) || !aligned16(Y) || !aligned16(OA))
     return FALQON_ERR_INVALID_ARG;
@@ -220,10 +223,28 @@ int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_d
   uint32_t* partial = reinterpret_cast<uint32_t*>(base + w.scales + kPartialsOffset);
   {
     StageTimer timer(FALQON_STAGE_QUANT_X, stream);
-    FALQON_CUDA(launch_quantize_fused(X, x_dt, T * n, kE4M3, xq, partial, base + w.scales + kSyncOffset, scales + 1, s_x_out,
-                                      scales + 0, amax_oa, status, nullptr, 0, nullptr, stream));
+    if (amax_x != nullptr) {
+      FALQON_CUDA(launch_cast_per_tensor(X, x_dt, T * n, kE4M3, 1.0f, reinterpret_cast<const uint32_t*>(amax_x), 1, nullptr, xq,
+                                         scales + 1, s_x_out, scales + 0, amax_oa, stream));
+    } else {
+      FALQON_CUDA(launch_quantize_fused(X, x_dt, T * n, kE4M3, xq, partial, base + w.scales + kSyncOffset, scales + 1, s_x_out,
+                                        scales + 0, amax_oa, status, nullptr, 0, nullptr, stream));
+    }
   }
   return forward_product(L, xq, scales + 1, T, Y, y_dt, OA, amax_oa, base, w, status, stream);
+}
+}  // namespace
+
+int falqon_melded_forward(const falqon_layer* L, const void* X, falqon_dtype x_dt, int64_t T, void* Y, falqon_dtype y_dt,
+                          float* OA, float* amax_oa, float* s_x_out, void* ws, size_t ws_bytes, falqon_stream stream) {
+  return forward_impl(L, X, x_dt, nullptr, T, Y, y_dt, OA, amax_oa, s_x_out, ws, ws_bytes, stream);
+}
+
+int falqon_melded_forward_amax(const falqon_layer* L, const void* X, falqon_dtype x_dt, const float* amax_x, int64_t T, void* Y,
+                               falqon_dtype y_dt, float* OA, float* amax_oa, float* s_x_out, void* ws, size_t ws_bytes,
+                               falqon_stream stream) {
+  if (amax_x == nullptr) return FALQON_ERR_INVALID_ARG;
+  return forward_impl(L, X, x_dt, amax_x, T, Y, y_dt, OA, amax_oa, s_x_out, ws, ws_bytes, stream);
 }
 
 int falqon_melded_forward_codes(const falqon_layer* L, const uint8_t* xq, const float* s_x, int64_t T, void* Y,
@@ -240,9 +261,11 @@ int falqon_melded_forward_codes(const falqon_layer* L, const uint8_t* xq, const 
   return forward_product(L, xq, s_x, T, Y, y_dt, OA, amax_oa, static_cast<uint8_t*>(ws), w, status, stream);
 }
 
-int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, int64_t T, const float* OA,
-                           const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, float* s_g_out, void* ws,
-                           size_t ws_bytes, falqon_stream stream) {
+namespace {
+// amax_dy (nullable, device [1]; per-tensor layers only): max |dY| is already known, see forward_impl.
+int backward_impl(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, const float* amax_dy, int64_t T, const float* OA,
+                  const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, float* s_g_out, void* ws, size_t ws_bytes,
+                  falqon_stream stream) {
   if (!layer_ok(L) || dY == nullptr || OA == nullptr || amax_oa == nullptr || dB == nullptr || T < 1 || !dtype_ok(dy_dt) ||
       !dtype_ok(dx_dt) || !aligned16(dY) || !aligned16(OA) || !aligned16(dB) || (dX != nullptr && !aligned16(dX)))
     return FALQON_ERR_INVALID_ARG;
@@ -267,9 +290,15 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
     StageTimer timer(FALQON_STAGE_QUANT_DY, stream);
     // S5a rides along: O~_A = Q_e4m3(O_A) with s_OA from the forward's amax, written transposed for the dB product
     const OaCastJob oa_cast{OA, amax_oa, T, static_cast<int>(r), w.t16, oaq_t, scales + 5, scales + 4};
-    FALQON_CUDA(launch_quantize_fused(dY, dy_dt, T * m, kE5M2, gq, partial, base + w.scales + kSyncOffset, scales + 3, s_g_out,
-                                      scales + 2, nullptr, status, per_row ? inv_sw : nullptr, static_cast<int>(m), &oa_cast,
-                                      stream));
+    if (amax_dy != nullptr) {   // single-pass cast; the O_A cast has no fused launch to ride on and runs by itself
+      FALQON_CUDA(launch_cast_per_tensor(dY, dy_dt, T * m, kE5M2, 1.0f, reinterpret_cast<const uint32_t*>(amax_dy), 1, nullptr, gq,
+                                         scales + 3, s_g_out, scales + 2, nullptr, stream));
+      FALQON_CUDA(launch_oa_cast(oa_cast, stream));
+    } else {
+      FALQON_CUDA(launch_quantize_fused(dY, dy_dt, T * m, kE5M2, gq, partial, base + w.scales + kSyncOffset, scales + 3, s_g_out,
+                                        scales + 2, nullptr, status, per_row ? inv_sw : nullptr, static_cast<int>(m), &oa_cast,
+                                        stream));
+    }
   }
   // S5b: dB = g~^T O~_A / (s_g s_OA) over token slabs, slab sum in slab order across a thread-block cluster.  It runs
   // before S4 (neither needs the other): g~ was written a moment ago and is still in L2.
@@ -297,6 +326,21 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
     FALQON_CUDA(launch_gemm_fp8(g, stream));
   }
   return FALQON_OK;
+}
+}  // namespace
+
+int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, int64_t T, const float* OA,
+                           const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, float* s_g_out, void* ws,
+                           size_t ws_bytes, falqon_stream stream) {
+  return backward_impl(L, dY, dy_dt, nullptr, T, OA, amax_oa, dX, dx_dt, dB, s_g_out, ws, ws_bytes, stream);
+}
+
+int falqon_melded_backward_amax(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, const float* amax_dy, int64_t T,
+                                const float* OA, const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, float* s_g_out,
+                                void* ws, size_t ws_bytes, falqon_stream stream) {
+  if (amax_dy == nullptr) return FALQON_ERR_INVALID_ARG;
+  if (L != nullptr && L->gran == FALQON_PER_ROW) return FALQON_ERR_UNSUPPORTED;   // the cast input is dY / s_w[column] there
+  return backward_impl(L, dY, dy_dt, amax_dy, T, OA, amax_oa, dX, dx_dt, dB, s_g_out, ws, ws_bytes, stream);
 }
 
 namespace {

@@ -26,11 +26,30 @@ __device__ __forceinline__ uint4 pack8(const float (&x)[8]) {
   return make_uint4(pack2(x[0], x[1]), pack2(x[2], x[3]), pack2(x[4], x[5]), pack2(x[6], x[7]));
 }
 
+// Largest |bf16| bit pattern (15 bits) among the two halves of each word.
+__device__ __forceinline__ uint32_t max_abs_bf16(const uint4& q, uint32_t m) {
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) m = max(m, max(w[i] & 0x7FFFu, (w[i] >> 16) & 0x7FFFu));
+  return m;
+}
+// Raises *amax (the fp32 bit pattern of a non-negative value) to the CTA's largest |bf16| with one atomic per CTA.
+__device__ __forceinline__ void publish_amax(uint32_t m, float* amax) {
+  __shared__ uint32_t s_max;
+  if (threadIdx.x == 0) s_max = 0u;
+  __syncthreads();
+  m = __reduce_max_sync(0xFFFFFFFFu, m);
+  if ((threadIdx.x & 31) == 0 && m != 0u) atomicMax(&s_max, m);
+  __syncthreads();
+  if (threadIdx.x == 0 && s_max != 0u) atomicMax(reinterpret_cast<unsigned int*>(amax), s_max << 16);
+}
+
 __global__ void __launch_bounds__(kChainThreads) combine_kernel(uint4* out, const uint4* a, float sa, const uint4* b, float sb,
                                                                 const uint4* c, float sc, const uint4* d, float sd,
-                                                                int64_t nvec) {
+                                                                int64_t nvec, float* amax) {
   pdl_trigger();
   pdl_wait();
+  uint32_t mx = 0;
   for (int64_t v = blockIdx.x * (int64_t)kChainThreads + threadIdx.x; v < nvec; v += (int64_t)gridDim.x * kChainThreads) {
     float x[8], y[8], acc[8];
     unpack8(ld_stream(a + v), x);
@@ -51,29 +70,39 @@ __global__ void __launch_bounds__(kChainThreads) combine_kernel(uint4* out, cons
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[i] = __fmaf_rn(sd, y[i], acc[i]);
     }
-    out[v] = pack8(acc);
+    const uint4 o = pack8(acc);
+    out[v] = o;
+    mx = max_abs_bf16(o, mx);
   }
+  if (amax != nullptr) publish_amax(mx, amax);
 }
 
 __device__ __forceinline__ float sigmoidf(float x) { return 1.0f / (1.0f + expf(-x)); }
 
-__global__ void __launch_bounds__(kChainThreads) silu_mul_kernel(uint4* z, const uint4* g, const uint4* u, int64_t nvec) {
+__global__ void __launch_bounds__(kChainThreads) silu_mul_kernel(uint4* z, const uint4* g, const uint4* u, int64_t nvec,
+                                                                 float* amax) {
   pdl_trigger();
   pdl_wait();
+  uint32_t mx = 0;
   for (int64_t v = blockIdx.x * (int64_t)kChainThreads + threadIdx.x; v < nvec; v += (int64_t)gridDim.x * kChainThreads) {
     float x[8], y[8], o[8];
     unpack8(ld_stream(g + v), x);
     unpack8(ld_stream(u + v), y);
 #pragma unroll
     for (int i = 0; i < 8; ++i) o[i] = x[i] * sigmoidf(x[i]) * y[i];
-    z[v] = pack8(o);
+    const uint4 q = pack8(o);
+    z[v] = q;
+    mx = max_abs_bf16(q, mx);
   }
+  if (amax != nullptr) publish_amax(mx, amax);
 }
 
 __global__ void __launch_bounds__(kChainThreads) silu_mul_grad_kernel(uint4* dg, uint4* du, const uint4* g, const uint4* u,
-                                                                      const uint4* dz, int64_t nvec) {
+                                                                      const uint4* dz, int64_t nvec, float* amax_dg,
+                                                                      float* amax_du) {
   pdl_trigger();
   pdl_wait();
+  uint32_t mg = 0, mu = 0;
   for (int64_t v = blockIdx.x * (int64_t)kChainThreads + threadIdx.x; v < nvec; v += (int64_t)gridDim.x * kChainThreads) {
     float x[8], y[8], t[8], og[8], ou[8];
     unpack8(ld_stream(g + v), x);
@@ -85,9 +114,14 @@ __global__ void __launch_bounds__(kChainThreads) silu_mul_grad_kernel(uint4* dg,
       ou[i] = t[i] * x[i] * s;
       og[i] = t[i] * y[i] * s * (1.0f + x[i] * (1.0f - s));
     }
-    dg[v] = pack8(og);
-    du[v] = pack8(ou);
+    const uint4 qg = pack8(og), qu = pack8(ou);
+    dg[v] = qg;
+    du[v] = qu;
+    mg = max_abs_bf16(qg, mg);
+    mu = max_abs_bf16(qu, mu);
   }
+  if (amax_dg != nullptr) publish_amax(mg, amax_dg);
+  if (amax_du != nullptr) publish_amax(mu, amax_du);
 }
 
 // One CTA of 128 threads per row; a thread keeps its elements (up to 16 vectors of 8) in registers between the
@@ -106,7 +140,7 @@ __device__ __forceinline__ float block_sum_128(float v, float* red /* [4] */) {
 }
 
 __global__ void __launch_bounds__(kNormThreads) rmsnorm_kernel(uint4* y, float* inv_rms, const uint4* x, int vec_per_row,
-                                                               float inv_cols, float eps) {
+                                                               float inv_cols, float eps, float* amax) {
   __shared__ float red[4];
   pdl_trigger();
   pdl_wait();
@@ -127,6 +161,7 @@ __global__ void __launch_bounds__(kNormThreads) rmsnorm_kernel(uint4* y, float* 
   }
   const float inv = rsqrtf(block_sum_128(ss, red) * inv_cols + eps);
   if (threadIdx.x == 0) inv_rms[blockIdx.x] = inv;
+  uint32_t mx = 0;
 #pragma unroll
   for (int i = 0; i < kNormMaxVec; ++i) {
     const int v = threadIdx.x + i * kNormThreads;
@@ -135,9 +170,12 @@ __global__ void __launch_bounds__(kNormThreads) rmsnorm_kernel(uint4* y, float* 
       unpack8(raw[i], f);
 #pragma unroll
       for (int e = 0; e < 8; ++e) f[e] *= inv;
-      yr[v] = pack8(f);
+      const uint4 o = pack8(f);
+      yr[v] = o;
+      mx = max_abs_bf16(o, mx);
     }
   }
+  if (amax != nullptr) publish_amax(mx, amax);
 }
 
 __global__ void __launch_bounds__(kNormThreads) rmsnorm_grad_kernel(uint4* dx, const uint4* dy, const uint4* x,
@@ -193,44 +231,46 @@ using namespace falqon;
 extern "C" {
 
 int falqon_chain_combine(void* out, const void* a, float sa, const void* b, float sb, const void* c, float sc, const void* d,
-                         float sd, int64_t count, falqon_stream stream) {
+                         float sd, int64_t count, float* amax_out, falqon_stream stream) {
   if (out == nullptr || a == nullptr || count < 8 || count % 8 || !ok16(out) || !ok16(a) || !ok16(b) || !ok16(c) || !ok16(d))
     return FALQON_ERR_INVALID_ARG;
   const int64_t nvec = count / 8;
   cudaError_t e = launch_pdl(combine_kernel, dim3(chain_grid(nvec)), dim3(kChainThreads), 0, static_cast<cudaStream_t>(stream), 1,
                              static_cast<uint4*>(out), static_cast<const uint4*>(a), sa, static_cast<const uint4*>(b), sb,
-                             static_cast<const uint4*>(c), sc, static_cast<const uint4*>(d), sd, nvec);
+                             static_cast<const uint4*>(c), sc, static_cast<const uint4*>(d), sd, nvec, amax_out);
   return e == cudaSuccess ? FALQON_OK : FALQON_ERR_CUDA;
 }
 
-int falqon_chain_silu_mul(void* z, const void* g, const void* u, int64_t count, falqon_stream stream) {
+int falqon_chain_silu_mul(void* z, const void* g, const void* u, int64_t count, float* amax_out, falqon_stream stream) {
   if (z == nullptr || g == nullptr || u == nullptr || count < 8 || count % 8 || !ok16(z) || !ok16(g) || !ok16(u))
     return FALQON_ERR_INVALID_ARG;
   const int64_t nvec = count / 8;
   cudaError_t e = launch_pdl(silu_mul_kernel, dim3(chain_grid(nvec)), dim3(kChainThreads), 0, static_cast<cudaStream_t>(stream), 1,
-                             static_cast<uint4*>(z), static_cast<const uint4*>(g), static_cast<const uint4*>(u), nvec);
+                             static_cast<uint4*>(z), static_cast<const uint4*>(g), static_cast<const uint4*>(u), nvec, amax_out);
   return e == cudaSuccess ? FALQON_OK : FALQON_ERR_CUDA;
 }
 
 int falqon_chain_silu_mul_grad(void* dg, void* du, const void* g, const void* u, const void* dz, int64_t count,
-                               falqon_stream stream) {
+                               float* amax_dg, float* amax_du, falqon_stream stream) {
   if (dg == nullptr || du == nullptr || g == nullptr || u == nullptr || dz == nullptr || count < 8 || count % 8 || !ok16(dg) ||
       !ok16(du) || !ok16(g) || !ok16(u) || !ok16(dz))
     return FALQON_ERR_INVALID_ARG;
   const int64_t nvec = count / 8;
   cudaError_t e = launch_pdl(silu_mul_grad_kernel, dim3(chain_grid(nvec)), dim3(kChainThreads), 0,
                              static_cast<cudaStream_t>(stream), 1, static_cast<uint4*>(dg), static_cast<uint4*>(du),
-                             static_cast<const uint4*>(g), static_cast<const uint4*>(u), static_cast<const uint4*>(dz), nvec);
+                             static_cast<const uint4*>(g), static_cast<const uint4*>(u), static_cast<const uint4*>(dz), nvec,
+                             amax_dg, amax_du);
   return e == cudaSuccess ? FALQON_OK : FALQON_ERR_CUDA;
 }
 
-int falqon_chain_rmsnorm(void* y, float* inv_rms, const void* x, int64_t rows, int64_t cols, float eps, falqon_stream stream) {
+int falqon_chain_rmsnorm(void* y, float* inv_rms, const void* x, int64_t rows, int64_t cols, float eps, float* amax_out,
+                         falqon_stream stream) {
   if (y == nullptr || inv_rms == nullptr || x == nullptr || rows < 1 || rows > (1ll << 30) || cols < 8 || cols % 8 ||
       cols > kNormThreads * kNormMaxVec * 8 || !ok16(y) || !ok16(x) || !(eps >= 0.0f))
     return FALQON_ERR_INVALID_ARG;
   cudaError_t e = launch_pdl(rmsnorm_kernel, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
                              static_cast<cudaStream_t>(stream), 1, static_cast<uint4*>(y), inv_rms, static_cast<const uint4*>(x),
-                             static_cast<int>(cols / 8), 1.0f / static_cast<float>(cols), eps);
+                             static_cast<int>(cols / 8), 1.0f / static_cast<float>(cols), eps, amax_out);
   return e == cudaSuccess ? FALQON_OK : FALQON_ERR_CUDA;
 }
 

@@ -65,6 +65,7 @@ struct OaCastJob {
   float* s_oa_out;
   float* amax_copy;   // nullable
 };
+cudaError_t launch_oa_cast(const OaCastJob& job, cudaStream_t stream);   // the same cast as a kernel of its own
 // Per-tensor absmax scaling in one kernel (absmax, grid barrier, cast).  `sync` points at 8 bytes of workspace that
 // are zero before the call and are left zero by it; `partial` holds up to kMaxAbsmaxParts words.
 // col_mul (nullable): column c of the [count / cols][cols] tensor is multiplied by col_mul[c] before everything else.

@@ -199,21 +199,19 @@ __device__ __forceinline__ void unit_values(const uint4& q, const float* col_mul
 
 // A rider of the output-gradient quantizer (S5a): O_A [T][r] fp32 -> E4M3 codes with s_OA = 448 / amax(O_A), stored
 // TRANSPOSED as [r][ldt] so that the adapter-gradient product reads them K-major.  One warp converts a tile of
-// 32 tokens (only the upper half of a CTA's warps call this): lane (tg, jq) takes tokens 4 tg .. 4 tg + 3 and columns 16 jq .. 16 jq + 15 of every block of 64
+// 32 tokens (warp w of the rider_warps warps of a CTA that take part): lane (tg, jq) takes tokens 4 tg .. 4 tg + 3 and columns 16 jq .. 16 jq + 15 of every block of 64
 // columns, so the codes of four consecutive tokens of one column form one 32-bit store.  Tokens at or beyond T
 // give zero codes (they land in the padding of the row pitch, a multiple of 16).
-__device__ __forceinline__ void cast_oa_transposed(const OaCastJob& job) {
+__device__ __forceinline__ void cast_oa_transposed(const OaCastJob& job, int w, int rider_warps) {
   const int lane = threadIdx.x & 31;
   const int tg = lane >> 2, jq = lane & 3;
   const float amax = ld_stream(job.amax_oa);
   const float s_oa = scale_from_amax(amax, kE4M3);
-  if (blockIdx.x == 0 && threadIdx.x == blockDim.x / 2) {
+  if (blockIdx.x == 0 && w == 0 && lane == 0) {
     *job.s_oa_out = s_oa;
     if (job.amax_copy != nullptr) *job.amax_copy = amax;
   }
   const long long n_tiles = (job.T + 31) / 32;
-  const int rider_warps = blockDim.x >> 6;                      // the upper half of the CTA's warps
-  const int w = (threadIdx.x >> 5) - rider_warps;               // 0 .. rider_warps - 1
   const int r16 = (job.r + 15) & ~15;
   // consecutive tiles go to different CTAs, so a small O_A costs every CTA at most one tile on one warp
   for (long long tile = static_cast<long long>(w) * gridDim.x + blockIdx.x; tile < n_tiles;
@@ -338,7 +336,8 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
   m = block_max_u32(m, red);
   // the rider runs here, on warps that would otherwise idle while thread 0 waits at the grid barrier: this CTA's
   // bulk copies have landed, so the rider's loads do not queue behind them
-  if (oa_job.oa != nullptr && tid >= kStagedThreads / 2) cast_oa_transposed(oa_job);
+  if (oa_job.oa != nullptr && tid >= kStagedThreads / 2)   // the upper half of the CTA's warps
+    cast_oa_transposed(oa_job, (tid >> 5) - kStagedThreads / 64, kStagedThreads / 64);
   // ---- grid barrier (a CTA that gave up above does not arrive: the others time out and report it)
   if (tid == 0) {
     int ok = failed ? 0 : 1;
@@ -505,6 +504,14 @@ cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, i
 #undef FALQON_CAST
 }
 
+// The O_A cast as a kernel of its own (for a backward whose output-gradient absmax is already known, so that no fused
+// quantizer launch exists for it to ride on).
+__global__ void __launch_bounds__(256) oa_cast_kernel(OaCastJob job) {
+  pdl_trigger();
+  pdl_wait();
+  cast_oa_transposed(job, threadIdx.x >> 5, 8);
+}
+
 template <int kDt, int kFmt, bool kColMul>
 cudaError_t launch_staged_variant(const void* src, int64_t count, uint8_t* dst, uint32_t* partial, void* sync,
                                   const CastOutputs& out, int* status, const float* col_mul, int cols, const OaCastJob& oa_job,
@@ -551,6 +558,13 @@ cudaError_t launch_quantize_fused(const void* src, int src_dt, int64_t count, in
   if (fmt == kE4M3) FALQON_FUSED(kF32, kE4M3);
   FALQON_FUSED(kF32, kE5M2);
 #undef FALQON_FUSED
+}
+
+cudaError_t launch_oa_cast(const OaCastJob& job, cudaStream_t stream) {
+  const long long tiles = (job.T + 31) / 32;
+  long long grid = (tiles + 7) / 8;
+  if (grid > 148 * 8) grid = 148 * 8;
+  return launch_pdl(oa_cast_kernel, dim3(static_cast<unsigned>(grid)), dim3(256), 0, stream, 1, job);
 }
 
 cudaError_t launch_scale_table(int mode, const float* s_w, int64_t m, int64_t r, const float* s_x, float* out, int64_t padded,

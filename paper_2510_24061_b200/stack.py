@@ -28,13 +28,13 @@ from . import synth
 lib = fq.lib
 _p, _f, _i64 = C.c_void_p, C.c_float, C.c_int64
 lib.falqon_chain_combine.restype = C.c_int
-lib.falqon_chain_combine.argtypes = [_p, _p, _f, _p, _f, _p, _f, _p, _f, _i64, _p]
+lib.falqon_chain_combine.argtypes = [_p, _p, _f, _p, _f, _p, _f, _p, _f, _i64, _p, _p]
 lib.falqon_chain_silu_mul.restype = C.c_int
-lib.falqon_chain_silu_mul.argtypes = [_p, _p, _p, _i64, _p]
+lib.falqon_chain_silu_mul.argtypes = [_p, _p, _p, _i64, _p, _p]
 lib.falqon_chain_silu_mul_grad.restype = C.c_int
-lib.falqon_chain_silu_mul_grad.argtypes = [_p, _p, _p, _p, _p, _i64, _p]
+lib.falqon_chain_silu_mul_grad.argtypes = [_p, _p, _p, _p, _p, _i64, _p, _p, _p]
 lib.falqon_chain_rmsnorm.restype = C.c_int
-lib.falqon_chain_rmsnorm.argtypes = [_p, _p, _p, _i64, _i64, _f, _p]
+lib.falqon_chain_rmsnorm.argtypes = [_p, _p, _p, _i64, _i64, _f, _p, _p]
 lib.falqon_chain_rmsnorm_grad.restype = C.c_int
 lib.falqon_chain_rmsnorm_grad.argtypes = [_p, _p, _p, _p, _i64, _i64, _p]
 CHAIN_EXPORTS = ["falqon_chain_combine", "falqon_chain_silu_mul", "falqon_chain_silu_mul_grad", "falqon_chain_rmsnorm",
@@ -50,35 +50,36 @@ def _ptr(t):
     return None if t is None else t.data_ptr()
 
 
-def combine(out, a, sa=1.0, b=None, sb=1.0, c=None, sc=1.0, d=None, sd=1.0):
-    """out = bf16(sa*a + sb*b + sc*c + sd*d); b, c, d optional."""
+def combine(out, a, sa=1.0, b=None, sb=1.0, c=None, sc=1.0, d=None, sd=1.0, amax=None):
+    """out = bf16(sa*a + sb*b + sc*c + sd*d); b, c, d optional.  amax (fp32 [1], zero beforehand): raised to max |out|."""
     for t in (out, a, b, c, d):
         assert t is None or (t.dtype == torch.bfloat16 and t.is_contiguous() and t.numel() == out.numel())
     fq._check("falqon_chain_combine", lib.falqon_chain_combine(_ptr(out), _ptr(a), sa, _ptr(b), sb, _ptr(c), sc, _ptr(d), sd,
-                                                                out.numel(), fq._stream()))
+                                                                out.numel(), _ptr(amax), fq._stream()))
     return out
 
 
-def silu_mul(z, g, u):
+def silu_mul(z, g, u, amax=None):
     for t in (z, g, u):
         assert t.dtype == torch.bfloat16 and t.is_contiguous() and t.numel() == z.numel()
-    fq._check("falqon_chain_silu_mul", lib.falqon_chain_silu_mul(_ptr(z), _ptr(g), _ptr(u), z.numel(), fq._stream()))
+    fq._check("falqon_chain_silu_mul", lib.falqon_chain_silu_mul(_ptr(z), _ptr(g), _ptr(u), z.numel(), _ptr(amax), fq._stream()))
     return z
 
 
-def silu_mul_grad(dg, du, g, u, dz):
+def silu_mul_grad(dg, du, g, u, dz, amax_dg=None, amax_du=None):
     for t in (dg, du, g, u, dz):
         assert t.dtype == torch.bfloat16 and t.is_contiguous() and t.numel() == g.numel()
     fq._check("falqon_chain_silu_mul_grad", lib.falqon_chain_silu_mul_grad(_ptr(dg), _ptr(du), _ptr(g), _ptr(u), _ptr(dz),
-                                                                            g.numel(), fq._stream()))
+                                                                            g.numel(), _ptr(amax_dg), _ptr(amax_du),
+                                                                            fq._stream()))
     return dg, du
 
 
-def rmsnorm(y, inv_rms, x):
+def rmsnorm(y, inv_rms, x, amax=None):
     assert x.dtype == torch.bfloat16 and x.dim() == 2 and x.is_contiguous() and y.shape == x.shape and y.is_contiguous()
     assert inv_rms.dtype == torch.float32 and inv_rms.numel() == x.shape[0]
     fq._check("falqon_chain_rmsnorm", lib.falqon_chain_rmsnorm(_ptr(y), _ptr(inv_rms), _ptr(x), x.shape[0], x.shape[1],
-                                                                NORM_EPS, fq._stream()))
+                                                                NORM_EPS, _ptr(amax), fq._stream()))
     return y
 
 
@@ -93,8 +94,12 @@ def rmsnorm_grad(dx, dy, x, inv_rms):
 class Stack:
     """n_layers blocks with hidden size H and MLP width F, T tokens per step, LoRA rank r, top-k rows per update."""
 
-    def __init__(self, n_layers: int, H: int, F: int, T: int, r: int, k: int, seed: int, device, lr: float = 2e-4):
+    def __init__(self, n_layers: int, H: int, F: int, T: int, r: int, k: int, seed: int, device, lr: float = 2e-4,
+                 producer_amax: bool = True):
+        """producer_amax: the chain kernels hand the absmax of their outputs to the layers that consume them, whose
+        input casts are then single-pass (False: every layer takes the absmax of its input itself)."""
         self.n_layers, self.H, self.F, self.T, self.r, self.k, self.lr = n_layers, H, F, T, r, k, lr
+        self.producer_amax = producer_amax
         self.device = torch.device(device)
         self.seed = seed
         self.shapes = {"q": (H, H), "k": (H, H), "v": (H, H), "o": (H, H), "gate": (H, F), "up": (H, F), "down": (F, H)}  # n -> m
@@ -138,12 +143,18 @@ class Stack:
         self.s_g = torch.empty(1, dtype=torch.float32, device=dev)
         self.dB = {p: torch.empty((self.shapes[p][1], r), dtype=torch.float32, device=dev) for p in PROJ}
         self.idx = torch.empty(max(k, 1), dtype=torch.int32, device=dev)
+        # absmax words of the chain's outputs, one row per block: x1, a, x2, z | ddn, dg, du, dhp, dqkv (cleared every step)
+        self.amax = torch.zeros((n_layers, 16), dtype=torch.float32, device=dev)
         self.capture = None   # optional: {(block, proj): dict} filled with references / copies for parity checks
 
     # ---- one linear: forward on X (quantizing it) or on another projection's codes
-    def _fwd(self, l, name, X, Y):
+    def _am(self, l, slot):
+        return self.amax[l, slot:slot + 1] if self.producer_amax else None
+
+    def _fwd(self, l, name, X, Y, amax_x=None):
         sv = self.saved[l]
-        fq.melded_forward(self.layers[l][name], X, ws=self.ws[name], out=(Y, sv["oa"][name], sv["amax"][name], self.s_x))
+        fq.melded_forward(self.layers[l][name], X, ws=self.ws[name], out=(Y, sv["oa"][name], sv["amax"][name], self.s_x),
+                          amax_x=amax_x)
         self._cap(l, name, X=X, Y=Y)
 
     def _fwd_shared(self, l, name, owner, X, Y):
@@ -155,10 +166,10 @@ class Stack:
         fq.melded_forward_codes(self.layers[l][name], xq, s_x, ws=self.ws[name], out=(Y, sv["oa"][name], sv["amax"][name]))
         self._cap(l, name, X=X, Y=Y)
 
-    def _bwd(self, l, name, dY, dX):
+    def _bwd(self, l, name, dY, dX, amax_dy=None):
         sv = self.saved[l]
         fq.melded_backward(self.layers[l][name], dY, sv["oa"][name], sv["amax"][name], ws=self.ws[name],
-                           out=(dX, self.dB[name], self.s_g))
+                           out=(dX, self.dB[name], self.s_g), amax_dy=amax_dy)
         self._cap(l, name, dY=dY, dX=dX, dB=self.dB[name], OA=sv["oa"][name])
         fq.proxy_update(self.layers[l][name], self.dB[name], self.lr, self.k, ws=self.ws[name],
                         idx_out=self.idx if self.k > 0 else None)
@@ -168,23 +179,25 @@ class Stack:
             self.capture[(l, name)].update({k2: v.clone() for k2, v in tensors.items()})
 
     def forward(self, h0: torch.Tensor) -> torch.Tensor:
+        if self.producer_amax:
+            self.amax.zero_()
         for l in range(self.n_layers):
             sv = self.saved[l]
             if l == 0:
                 sv["h"].copy_(h0)
             h, hp = sv["h"], sv["hp"]
-            rmsnorm(self.x1, sv["inv1"], h)
-            self._fwd(l, "q", self.x1, self.q)
+            rmsnorm(self.x1, sv["inv1"], h, amax=self._am(l, 0))
+            self._fwd(l, "q", self.x1, self.q, self._am(l, 0))
             self._fwd_shared(l, "k", "q", self.x1, self.kk)
             self._fwd_shared(l, "v", "q", self.x1, self.v)
-            combine(self.a, self.q, INV_SQRT3, self.kk, INV_SQRT3, self.v, INV_SQRT3)
-            self._fwd(l, "o", self.a, self.o)
+            combine(self.a, self.q, INV_SQRT3, self.kk, INV_SQRT3, self.v, INV_SQRT3, amax=self._am(l, 1))
+            self._fwd(l, "o", self.a, self.o, self._am(l, 1))
             combine(hp, h, 1.0, self.o, 1.0)
-            rmsnorm(self.x2, sv["inv2"], hp)
-            self._fwd(l, "gate", self.x2, sv["g"])
+            rmsnorm(self.x2, sv["inv2"], hp, amax=self._am(l, 2))
+            self._fwd(l, "gate", self.x2, sv["g"], self._am(l, 2))
             self._fwd_shared(l, "up", "gate", self.x2, sv["u"])
-            silu_mul(self.z, sv["g"], sv["u"])
-            self._fwd(l, "down", self.z, self.dn)
+            silu_mul(self.z, sv["g"], sv["u"], amax=self._am(l, 3))
+            self._fwd(l, "down", self.z, self.dn, self._am(l, 3))
             out = self.saved[l + 1]["h"] if l + 1 < self.n_layers else self.h_out   # the next block's saved input
             combine(out, hp, INV_SQRT2, self.dn, INV_SQRT2)
         return self.h_out
@@ -195,19 +208,19 @@ class Stack:
         dh = G
         for l in reversed(range(self.n_layers)):
             sv = self.saved[l]
-            combine(self.ddn, dh, INV_SQRT2)                                   # d(down output) = dh / sqrt(2)
-            self._bwd(l, "down", self.ddn, self.dz)
-            silu_mul_grad(self.dg, self.du, sv["g"], sv["u"], self.dz)
-            self._bwd(l, "gate", self.dg, self.dx[0])
-            self._bwd(l, "up", self.du, self.dx[1])
+            combine(self.ddn, dh, INV_SQRT2, amax=self._am(l, 4))               # d(down output) = dh / sqrt(2)
+            self._bwd(l, "down", self.ddn, self.dz, self._am(l, 4))
+            silu_mul_grad(self.dg, self.du, sv["g"], sv["u"], self.dz, self._am(l, 5), self._am(l, 6))
+            self._bwd(l, "gate", self.dg, self.dx[0], self._am(l, 5))
+            self._bwd(l, "up", self.du, self.dx[1], self._am(l, 6))
             combine(self.dx[0], self.dx[0], 1.0, self.dx[1], 1.0)               # d x2
             rmsnorm_grad(self.dx[1], self.dx[0], sv["hp"], sv["inv2"])
-            combine(self.dhp, dh, INV_SQRT2, self.dx[1], 1.0)                   # dh' = dh/sqrt(2) + norm'(d x2)
-            self._bwd(l, "o", self.dhp, self.da)
-            combine(self.dqkv, self.da, INV_SQRT3)                              # dq = dk = dv = da / sqrt(3)
-            self._bwd(l, "q", self.dqkv, self.dx[0])
-            self._bwd(l, "k", self.dqkv, self.dx[1])
-            self._bwd(l, "v", self.dqkv, self.dx[2])
+            combine(self.dhp, dh, INV_SQRT2, self.dx[1], 1.0, amax=self._am(l, 7))   # dh' = dh/sqrt(2) + norm'(d x2)
+            self._bwd(l, "o", self.dhp, self.da, self._am(l, 7))
+            combine(self.dqkv, self.da, INV_SQRT3, amax=self._am(l, 8))         # dq = dk = dv = da / sqrt(3)
+            self._bwd(l, "q", self.dqkv, self.dx[0], self._am(l, 8))
+            self._bwd(l, "k", self.dqkv, self.dx[1], self._am(l, 8))
+            self._bwd(l, "v", self.dqkv, self.dx[2], self._am(l, 8))
             combine(self.dx[0], self.dx[0], 1.0, self.dx[1], 1.0, self.dx[2], 1.0)   # d x1
             rmsnorm_grad(self.dx[1], self.dx[0], sv["h"], sv["inv1"])
             combine(self.dh, self.dhp, 1.0, self.dx[1], 1.0)
@@ -229,7 +242,8 @@ class Stack:
         for name in PROJ:
             shared = name in ("k", "v", "up")
             per_block += (1 if shared else fq.launch_count("falqon_melded_forward"))   # codes: the product alone
-            per_block += fq.launch_count("falqon_melded_backward") + fq.launch_count("falqon_proxy_update", k=self.k)
+            per_block += fq.launch_count("falqon_melded_backward") + (1 if self.producer_amax else 0)   # + the O_A cast
+            per_block += fq.launch_count("falqon_proxy_update", k=self.k)
         per_block += 6 + 9   # chain kernels: forward 6 (2 norms, mix, 2 residuals, gate), backward 9
         return per_block * self.n_layers
 

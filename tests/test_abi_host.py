@@ -34,8 +34,8 @@ def test_chain_header_symbols_are_exported(fq):
         assert hasattr(fq.lib, name), name
     fake = 0x10000
     assert fq.lib.falqon_chain_combine(fake, None, C.c_float(1), None, C.c_float(1), None, C.c_float(1), None, C.c_float(1),
-                                       64, None) == fq.ERR_INVALID_ARG
-    assert stack.lib.falqon_chain_rmsnorm(fake, fake, fake, 4, 12, C.c_float(1e-6), None) == fq.ERR_INVALID_ARG   # cols % 8
+                                       64, None, None) == fq.ERR_INVALID_ARG
+    assert stack.lib.falqon_chain_rmsnorm(fake, fake, fake, 4, 12, C.c_float(1e-6), None, None) == fq.ERR_INVALID_ARG   # cols % 8
 
 
 def test_workspace_layout(fq):

@@ -243,6 +243,36 @@ def test_forward_on_shared_codes_equals_forward(fq, per_row):
     assert fq.last_device_status() == 0
 
 
+def test_known_absmax_variants_equal_the_plain_calls(fq):
+    """A caller that knows max |X| and max |dY| gets single-pass casts; every output must equal the plain calls' bit for
+    bit (same scale, same codes, same products).  Per-row layers reject the backward variant."""
+    m, n, r, T = 640, 1280, 64, 300
+    W, A, B, X = layer_inputs(43, 0, m, n, r, T, 4)
+    dY = synth.out_grad(43, 0, 0, T, m).to(DEV)
+    Xd = X.to(DEV)
+    layer = fq.setup_layer(W.to(DEV), A.to(DEV), B.to(DEV), 1.0)
+    ws = layer.workspace(T)
+    Y, OA, amax_oa, s_x = [t.clone() for t in fq.melded_forward(layer, Xd, y_dtype=torch.float32, ws=ws)]
+    xq = fq.ws_view(layer, ws, T, fq.WS_XQ).clone()
+    dX, dB, s_g = [t.clone() for t in fq.melded_backward(layer, dY, OA, amax_oa, dx_dtype=torch.float32, ws=ws)]
+    gq = fq.ws_view(layer, ws, T, fq.WS_GQ).clone()
+    oaq = fq.ws_view(layer, ws, T, fq.WS_OAQ_T).clone()
+    ws2 = torch.empty_like(ws)
+    fq.workspace_init(ws2)
+    Y2, OA2, amax2, s_x2 = fq.melded_forward(layer, Xd, y_dtype=torch.float32, ws=ws2, amax_x=Xd.float().abs().max().reshape(1))
+    assert torch.equal(fq.ws_view(layer, ws2, T, fq.WS_XQ), xq) and torch.equal(s_x2, s_x)
+    assert torch.equal(Y2, Y) and torch.equal(OA2, OA) and torch.equal(amax2, amax_oa)
+    dX2, dB2, s_g2 = fq.melded_backward(layer, dY, OA2, amax2, dx_dtype=torch.float32, ws=ws2,
+                                        amax_dy=dY.float().abs().max().reshape(1))
+    assert torch.equal(fq.ws_view(layer, ws2, T, fq.WS_GQ), gq) and torch.equal(s_g2, s_g)
+    assert torch.equal(fq.ws_view(layer, ws2, T, fq.WS_OAQ_T)[: r * ((T + 15) // 16 * 16)], oaq[: r * ((T + 15) // 16 * 16)])
+    assert torch.equal(dX2, dX) and torch.equal(dB2, dB)
+    per_row = fq.setup_layer(W.to(DEV), A.to(DEV), None, 1.0, per_row=True)
+    with pytest.raises(fq.FalqonError):
+        fq.melded_backward(per_row, dY, OA, amax_oa, amax_dy=dY.float().abs().max().reshape(1))
+    assert fq.last_device_status() == 0
+
+
 def test_b_zero_leaves_plain_fp8_layer(fq):
     c = synth.config0()
     W, A, _, X = layer_inputs(0, 0, c["m"], c["n"], c["r"], c["T"], c["n_outliers"])

@@ -49,7 +49,9 @@ def test_chain_elementwise_kernels(st):
     a, b, c, d = [(torch.randn(n) * s).to(torch.bfloat16) for s in (1.0, 0.5, 2.0, 0.1)]
     ad, bd, cd, dd = [t.to(DEV) for t in (a, b, c, d)]
     out = torch.empty_like(ad)
-    st.combine(out, ad, 0.5, bd, -1.25, cd, 3.0 ** -0.5, dd, 1.0)
+    amax = torch.zeros(4, dtype=torch.float32, device=DEV)
+    st.combine(out, ad, 0.5, bd, -1.25, cd, 3.0 ** -0.5, dd, 1.0, amax=amax[0:1])
+    assert float(amax[0]) == float(out.float().abs().max())
     acc = a.double() * np.float32(0.5)
     for s, t in ((np.float32(-1.25), b), (np.float32(3.0 ** -0.5), c), (np.float32(1.0), d)):
         acc = (acc.float().double() + float(s) * t.double())      # fp32 fma chain: one rounding per step
@@ -58,11 +60,13 @@ def test_chain_elementwise_kernels(st):
     st.combine(out, ad, 2.0 ** -0.5)
     assert torch.equal(out.cpu(), (a.float() * np.float32(2.0 ** -0.5)).to(torch.bfloat16))
     z = torch.empty_like(ad)
-    st.silu_mul(z, ad, bd)
+    st.silu_mul(z, ad, bd, amax=amax[1:2])
+    assert float(amax[1]) == float(z.float().abs().max())
     ref = (a.float() * torch.sigmoid(a.float()) * b.float()).to(torch.bfloat16)
     assert int(_bf16_steps(z.cpu(), ref).max()) <= 1 and float((z.cpu() != ref).float().mean()) < 2e-2
     dg, du = torch.empty_like(ad), torch.empty_like(ad)
-    st.silu_mul_grad(dg, du, ad, bd, cd)
+    st.silu_mul_grad(dg, du, ad, bd, cd, amax[2:3], amax[3:4])
+    assert float(amax[2]) == float(dg.float().abs().max()) and float(amax[3]) == float(du.float().abs().max())
     s = torch.sigmoid(a.float())
     ref_u = (c.float() * a.float() * s).to(torch.bfloat16)
     ref_g = (c.float() * b.float() * s * (1 + a.float() * (1 - s))).to(torch.bfloat16)
@@ -76,7 +80,9 @@ def test_chain_rmsnorm_and_its_gradient(st):
     x = (torch.randn(rows, cols) * 3.0).to(torch.bfloat16)
     dy = torch.randn(rows, cols).to(torch.bfloat16)
     y, inv = torch.empty_like(x, device=DEV), torch.empty(rows, dtype=torch.float32, device=DEV)
-    st.rmsnorm(y, inv, x.to(DEV))
+    amax = torch.zeros(1, dtype=torch.float32, device=DEV)
+    st.rmsnorm(y, inv, x.to(DEV), amax=amax)
+    assert float(amax[0]) == float(y.float().abs().max())
     xf = x.double()
     inv_ref = 1.0 / torch.sqrt((xf * xf).mean(dim=1) + st.NORM_EPS)
     assert torch.allclose(inv.cpu().double(), inv_ref, rtol=1e-5)
@@ -133,8 +139,8 @@ def _check_projection(fq, orc, cap, layer, name, T, r, k, lr, n_rows):
     assert np.array_equal(bits32(f32(layer.dbuf)), bits32(dbuf_o)), f"{name} DeltaBuffer"
 
 
-def _run_and_check(fq, st, orc, n_layers, H, F, T, r, k, check_blocks, n_rows):
-    stack = st.Stack(n_layers, H, F, T, r, k, seed=7, device=DEV, lr=2e-2)
+def _run_and_check(fq, st, orc, n_layers, H, F, T, r, k, check_blocks, n_rows, producer_amax=True):
+    stack = st.Stack(n_layers, H, F, T, r, k, seed=7, device=DEV, lr=2e-2, producer_amax=producer_amax)
     h0 = synth.normal_bf16(7, 9001, (T, H), 1.0, DEV)
     G = synth.normal_bf16(7, 9002, (T, H), 1.0e-2, DEV)
     stack.capture = {(l, p): {} for l in check_blocks for p in st.PROJ}
@@ -151,9 +157,11 @@ def _run_and_check(fq, st, orc, n_layers, H, F, T, r, k, check_blocks, n_rows):
     return stack
 
 
-def test_small_stack_every_projection(fq, st, orc):
-    """Three blocks of a narrow chain, every projection of every block checked on all token rows."""
-    _run_and_check(fq, st, orc, 3, 256, 640, 192, 16, 8, check_blocks=[0, 1, 2], n_rows=192)
+@pytest.mark.parametrize("producer_amax", [True, False])
+def test_small_stack_every_projection(fq, st, orc, producer_amax):
+    """Three blocks of a narrow chain, every projection of every block checked on all token rows; with the chain
+    kernels handing the absmax of their outputs to the layers (single-pass input casts) and without."""
+    _run_and_check(fq, st, orc, 3, 256, 640, 192, 16, 8, check_blocks=[0, 1, 2], n_rows=192, producer_amax=producer_amax)
 
 
 def test_stack_7b_shapes_sampled(fq, st, orc):
