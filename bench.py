@@ -457,7 +457,7 @@ def main():
     launches_big = sum(1 for name, _ in records if name in ("gemm_fwd", "gemm_dx"))
     achieved = f_big / (t_big * 1e-3) / 1e12 if t_big > 0 else 0.0
     peak = peaks["bf16_sustained"] * FP8_OVER_BF16
-    roofline = {"kernel": "gemm_fp8_kernel (forward and input-gradient products)", "bound": "tensor",
+    roofline = {"kernel": "gemm_fp8_pair_kernel (forward and input-gradient products)", "bound": "tensor",
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                 "peak_source": f"{peaks['source']} bf16 sustained x{FP8_OVER_BF16:g} (nominal FP8:bf16 ratio)",
                 "frac_of_burst_peak": achieved / (peaks["bf16_burst"] * FP8_OVER_BF16),
