@@ -37,9 +37,13 @@ UNIT = "TFLOP/s"
 FP8_OVER_BF16 = 2.0        # nominal dense FP8 : bf16 tensor throughput on B200 (4.5 : 2.25 PFLOP/s)
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read+write of the forward and dX launches on the q projection (36.93 + 37.61 MB) over their FP8 operand
-# bytes (33.82 + 33.55 MB); the ncu summary is under profiles/.  Traffic grows in proportion to the operands.
-DRAM_OVER_OPERAND_BYTES = (36.93 + 37.61) / (33.82 + 33.55)
+# dram__bytes_read.sum + dram__bytes_write.sum of one forward and one dX launch of gemm_fp8_pair_kernel, measured with ncu on
+# the three projection shapes of the workload (profiles/gemm_fp8_pair_kernel__traffic_by_shape.md), in bytes:
+GEMM_DRAM_BYTES = {   # (n, m): (forward, dX)
+    (4096, 4096): (33950976 + 2122240, 33630720 + 351488),
+    (4096, 11008): (62336256 + 53340160, 136442624 + 18720512),
+    (11008, 4096): (139000064 + 23043328, 62110720 + 49093120),
+}
 
 
 def layer_flops(T, n, m, r):
@@ -464,10 +468,11 @@ def main():
                 "frac_of_nominal_4500": achieved / 4500.0,
                 "launches": launches_big, "avg_launch_ms": t_big / max(launches_big, 1),
                 "gflop_per_launch": f_big / max(launches_big, 1) / 1e9,
-                "traffic": DRAM_OVER_OPERAND_BYTES * sum((T * n + (m + r) * n) + (T * m + m * n) for _, n, m in linears)
-                / (2.0 * len(linears)),
-                "traffic_note": "bytes per average launch: FP8 operand bytes x 1.106, the dram read+write / operand ratio "
-                                "ncu measured on the q projection (profiles/gemm_fp8_pair_kernel__q_projection_T4096.md)"}
+                "traffic": sum(sum(GEMM_DRAM_BYTES.get((n, m), (0, 0))) for _, n, m in linears) / (2.0 * len(linears)),
+                "traffic_note": "dram read+write bytes per average launch, from the ncu capture of the forward and dX "
+                                "launch of each projection shape (profiles/gemm_fp8_pair_kernel__traffic_by_shape.md); "
+                                "algorithmic operand bytes per average launch: %.1f MB" %
+                                (sum((T * n + (m + r) * n) + (T * m + m * n) for _, n, m in linears) / (2.0 * len(linears)) / 1e6)}
     t_db = sum(ms for name, ms in records if name == "gemm_db")
 
     # ---- stage breakdown (separate untimed-for-value pass with every stage bracketed)
