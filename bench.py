@@ -128,13 +128,13 @@ def aggregate_over_ranks(ms_local: float, flops_per_rank: float, dist=None, devi
     return ms, world * flops_per_rank / (ms * 1e-3) / 1e12
 
 
-def build_workload(fq, device, seed, T, r, k, linears, outlier_frac):
+def build_workload(fq, device, seed, T, r, k, linears, outlier_frac, per_row=False, heavy_tailed=False):
     layers = []
     for idx, (name, n, m) in enumerate(linears):
-        W = synth.backbone(seed, idx, m, n, device)
+        W = synth.backbone(seed, idx, m, n, device, heavy_tailed=heavy_tailed)
         A = synth.adapter_a(seed, idx, r, n, device)
         B = synth.adapter_b(seed, idx, m, r, device)
-        layer = fq.setup_layer(W, A, B, 1.0)
+        layer = fq.setup_layer(W, A, B, 1.0, per_row=per_row)
         del W
         X = synth.activations(seed, idx, T, n, round(outlier_frac * n), device)
         dY = synth.out_grad(seed, idx, 0, T, m, device)
@@ -355,22 +355,29 @@ def main():
     ap.add_argument("--stack-layers", type=int, default=32)
     ap.add_argument("--stack-own-absmax", action="store_true",
                     help="with --stack: every layer takes the absmax of its input itself (the chain kernels do not hand it over)")
+    ap.add_argument("--config3", action="store_true",
+                    help="configs[3] instead of configs[1]: the LLaMA-13B projection set, 8192 tokens, per-row-scaled "
+                         "heavy-tailed backbone, top-512 (not the headline line)")
     ap.add_argument("--only", default=None, help="profiling aid: restrict the workload to one projection (q,k,v,o,gate,up,down)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    cfg = synth.config1()
+    cfg = synth.config3() if args.config3 else synth.config1()
     T, r, k, lr = cfg["T"], cfg["r"], cfg["k"], cfg["lr"]
     linears = cfg["linears"]
     if args.only is not None:
         linears = [l for l in linears if l[0] == args.only]
     flops_step = sum(layer_flops(T, n, m, r) for _, n, m in linears)
-    workload = {"workload": "configs[1]: LLaMA-7B projection set (q,k,v,o,gate,up,down), tokens=4096, rank=64, top-k=256"
+    workload = {"workload": ("configs[3]: LLaMA-13B projection set (q,k,v,o,gate,up,down), tokens=8192, rank=64, top-k=512, "
+                             "per-row-scaled heavy-tailed backbone" if args.config3 else
+                             "configs[1]: LLaMA-7B projection set (q,k,v,o,gate,up,down), tokens=4096, rank=64, top-k=256")
                             + ("" if args.only is None else f" -- RESTRICTED to '{args.only}' (profiling aid, not a bench line)"),
                 "tokens": T, "rank": r, "topk": k, "matrices": len(linears), "gflop_per_step": flops_step / 1e9,
-                "l2": "inputs larger than L2 (0.85 GB touched per step)", "parallelism": f"replicas x{world}"}
+                "l2": "inputs larger than L2 (%.2f GB of inputs and outputs touched per step)" %
+                      (sum(2.0 * T * (n + m) * 2 for _, n, m in linears) / 1e9),
+                "parallelism": f"replicas x{world}"}
 
     if args.sweep:
         if rank == 0:
@@ -409,7 +416,8 @@ def main():
         dist.init_process_group("nccl", device_id=device)
     from paper_2510_24061_b200 import binding as fq
 
-    layers = build_workload(fq, device, cfg["seed"] + rank, T, r, k, linears, cfg["outlier_frac"])
+    layers = build_workload(fq, device, cfg["seed"] + rank, T, r, k, linears, cfg["outlier_frac"],
+                            per_row=cfg.get("per_row", False), heavy_tailed=cfg.get("heavy_tailed", False))
     torch.cuda.synchronize()
 
     def barrier():
@@ -468,7 +476,8 @@ def main():
                 "frac_of_nominal_4500": achieved / 4500.0,
                 "launches": launches_big, "avg_launch_ms": t_big / max(launches_big, 1),
                 "gflop_per_launch": f_big / max(launches_big, 1) / 1e9,
-                "traffic": sum(sum(GEMM_DRAM_BYTES.get((n, m), (0, 0))) for _, n, m in linears) / (2.0 * len(linears)),
+                "traffic": (sum(sum(GEMM_DRAM_BYTES[(n, m)]) for _, n, m in linears) / (2.0 * len(linears))
+                            if all((n, m) in GEMM_DRAM_BYTES for _, n, m in linears) else None),
                 "traffic_note": "dram read+write bytes per average launch, from the ncu capture of the forward and dX "
                                 "launch of each projection shape (profiles/gemm_fp8_pair_kernel__traffic_by_shape.md); "
                                 "algorithmic operand bytes per average launch: %.1f MB" %

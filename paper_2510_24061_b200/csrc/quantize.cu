@@ -175,7 +175,8 @@ template <int kDt> struct Unit { static constexpr int kElems = kDt == kBF16 ? 8 
 
 // The elements of one 16-byte unit as fp32, times their column factors when kColMul.
 template <int kDt, bool kColMul>
-__device__ __forceinline__ void unit_values(const uint4& q, const float* col_mul, int col, float (&x)[Unit<kDt>::kElems]) {
+__device__ __forceinline__ void unit_values(const uint4& q, const float* col_mul, const float* table, int col,
+                                            float (&x)[Unit<kDt>::kElems]) {
   if (kDt == kBF16) {
     const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
@@ -186,11 +187,11 @@ __device__ __forceinline__ void unit_values(const uint4& q, const float* col_mul
   } else {
     x[0] = __uint_as_float(q.x); x[1] = __uint_as_float(q.y); x[2] = __uint_as_float(q.z); x[3] = __uint_as_float(q.w);
   }
-  if (kColMul) {
-    const float4* f = reinterpret_cast<const float4*>(col_mul + col);
+  if (kColMul) {   // the factors come from the CTA's shared-memory copy when there is one
+    const float4* f = reinterpret_cast<const float4*>((table != nullptr ? table : col_mul) + col);
 #pragma unroll
     for (int i = 0; i < Unit<kDt>::kElems / 4; ++i) {
-      const float4 c = ld_stream(f + i);
+      const float4 c = table != nullptr ? f[i] : ld_stream(f + i);
       x[4 * i] = __fmul_rn(x[4 * i], c.x); x[4 * i + 1] = __fmul_rn(x[4 * i + 1], c.y);
       x[4 * i + 2] = __fmul_rn(x[4 * i + 2], c.z); x[4 * i + 3] = __fmul_rn(x[4 * i + 3], c.w);
     }
@@ -247,12 +248,20 @@ __device__ __forceinline__ void cast_oa_transposed(const OaCastJob& job, int w, 
   }
 }
 
+// x mod cols for x < cols + 8192 (a column offset inside one chunk): a compare and a subtract for the wide rows of
+// real layers, a division only for narrow ones.
+__device__ __forceinline__ uint32_t wrap_col(uint32_t x, uint32_t cols) {
+  if (cols >= 8192u) return x >= cols ? x - cols : x;
+  return x % cols;
+}
+
 // Casts the elements of one 16-byte unit (element index e of the tensor) and stores their codes.
 template <int kDt, int kFmt, bool kColMul>
-__device__ __forceinline__ void cast_unit(const uint4& q, int64_t e, const float* col_mul, int cols, float sc, uint8_t* dst) {
+__device__ __forceinline__ void cast_unit(const uint4& q, int64_t e, int col, const float* col_mul, const float* table, float sc,
+                                          uint8_t* dst) {
   constexpr int kUnit = Unit<kDt>::kElems;
   float x[kUnit];
-  unit_values<kDt, kColMul>(q, col_mul, kColMul ? static_cast<int>(e % cols) : 0, x);
+  unit_values<kDt, kColMul>(q, col_mul, table, col, x);
 #pragma unroll
   for (int k = 0; k < kUnit; ++k) x[k] = __fmul_rn(x[k], sc);
   if (kDt == kBF16) {
@@ -268,22 +277,30 @@ __device__ __forceinline__ void cast_unit(const uint4& q, int64_t e, const float
 template <int kDt, int kFmt, bool kColMul>
 __global__ void __launch_bounds__(kStagedThreads, 1)
 quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* partial, GridSync* sync, CastOutputs out,
-                       int* status, const float* col_mul, int cols, OaCastJob oa_job) {
+                       int* status, const float* col_mul, int cols, OaCastJob oa_job, int slots, int table_floats) {
   constexpr int kEsize = kDt == kBF16 ? 2 : 4;
   constexpr int kUnit = Unit<kDt>::kElems;
   constexpr int64_t kChunkElems = kChunkBytes / kEsize;
-  extern __shared__ __align__(128) uint8_t stage[];
+  // dynamic shared memory: [table_floats column factors, padded to whole chunks][slots x 16 KB ring]
+  extern __shared__ __align__(128) uint8_t staged_smem[];
+  const float* table = table_floats > 0 ? reinterpret_cast<const float*>(staged_smem) : nullptr;
+  uint8_t* stage = staged_smem + (static_cast<size_t>(table_floats) * 4 + kChunkBytes - 1) / kChunkBytes * kChunkBytes;
   __shared__ __align__(8) uint64_t bars[kStagedSlots];
   __shared__ uint32_t red[32];
   __shared__ int s_ok;
   const int tid = threadIdx.x;
   if (tid == 0) {
-    for (int s = 0; s < kStagedSlots; ++s) mbar_init(smem_u32(&bars[s]), 1);
+    for (int s = 0; s < slots; ++s) mbar_init(smem_u32(&bars[s]), 1);
     mbar_fence_init();
   }
   pdl_trigger();
   __syncthreads();
   pdl_wait();
+  if (table_floats > 0) {   // the column factors, once per CTA (they are read twice per element otherwise)
+    float* tw = reinterpret_cast<float*>(staged_smem);
+    for (int c = tid; c < table_floats; c += kStagedThreads) tw[c] = ld_stream(col_mul + c);
+    __syncthreads();
+  }
 
   const int64_t bulk_elems = (count / 16) * 16;      // the rest (fewer than 16 elements) goes element by element
   const int64_t n_chunks = (bulk_elems + kChunkElems - 1) / kChunkElems;
@@ -294,8 +311,8 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
     const int64_t rem = bulk_elems - c * kChunkElems;
     return static_cast<int>(rem < kChunkElems ? rem : kChunkElems);
   };
-  auto issue = [&](int i) {   // one thread: fetch the CTA's i-th chunk into slot i mod kStagedSlots
-    const int s = i % kStagedSlots;
+  auto issue = [&](int i) {   // one thread: fetch the CTA's i-th chunk into slot i mod slots
+    const int s = i % slots;
     const int64_t c = chunk_of(i);
     const uint32_t bytes = static_cast<uint32_t>(chunk_elems(c)) * kEsize;   // a multiple of 32
     const uint32_t bar = smem_u32(&bars[s]);
@@ -306,25 +323,26 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
 
   // ---- pass 1: absmax
   if (tid == 0)
-    for (int i = 0; i < n_my && i < kStagedSlots; ++i) issue(i);
+    for (int i = 0; i < n_my && i < slots; ++i) issue(i);
   uint32_t phase_bits = 0;   // bit s: parity of the next completion of slot s
   uint32_t m = 0;
   bool failed = false;
   for (int i = 0; i < n_my; ++i) {
-    const int s = i % kStagedSlots;
+    const int s = i % slots;
     const bool ok = mbar_wait(smem_u32(&bars[s]), (phase_bits >> s) & 1u, status);
     phase_bits ^= 1u << s;
     const int64_t e0 = chunk_of(i) * kChunkElems;
+    const uint32_t col0 = kColMul ? static_cast<uint32_t>(e0 % cols) : 0u;   // one 64-bit modulo per chunk, 32-bit ones per unit
     const int units = chunk_elems(chunk_of(i)) / kUnit;
     const uint4* sp = reinterpret_cast<const uint4*>(stage + s * kChunkBytes);
     for (int u = tid; u < units; u += kStagedThreads) {
       float x[kUnit];
-      unit_values<kDt, kColMul>(sp[u], col_mul, kColMul ? static_cast<int>((e0 + static_cast<int64_t>(u) * kUnit) % cols) : 0, x);
+      unit_values<kDt, kColMul>(sp[u], col_mul, table, kColMul ? static_cast<int>(wrap_col(col0 + static_cast<uint32_t>(u) * kUnit, static_cast<uint32_t>(cols))) : 0, x);
 #pragma unroll
       for (int e = 0; e < kUnit; ++e) m = max(m, abs_bits(x[e]));
     }
     if (!__syncthreads_and(ok)) { failed = true; break; }   // block-uniform; also: the slot is free again
-    if (tid == 0 && i + kStagedSlots < n_my) issue(i + kStagedSlots);
+    if (tid == 0 && i + slots < n_my) issue(i + slots);
   }
   if (blockIdx.x == 0) {   // ragged tail
     for (int64_t e = bulk_elems + tid; e < count; e += kStagedThreads) {
@@ -371,13 +389,15 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
     // ---- pass 2: cast, most recent chunk first
     for (int t = 0; t < n_my; ++t) {
       const int i = n_my - 1 - t;
-      const int s = i % kStagedSlots;
+      const int s = i % slots;
       bool ok = true;
-      if (t >= kStagedSlots) {   // this chunk had left the ring and was fetched again
+      if (t >= slots) {   // this chunk had left the ring and was fetched again
         ok = mbar_wait(smem_u32(&bars[s]), (phase_bits >> s) & 1u, status);
         phase_bits ^= 1u << s;
       }
       const int64_t e0 = chunk_of(i) * kChunkElems;
+      const uint32_t col0 = kColMul ? static_cast<uint32_t>(e0 % cols) : 0u;
+      const uint32_t ucols = kColMul ? static_cast<uint32_t>(cols) : 1u;
       const int units = chunk_elems(chunk_of(i)) / kUnit;
       const uint4* sp = reinterpret_cast<const uint4*>(stage + s * kChunkBytes);
       // two units per thread and iteration (a full chunk is exactly one iteration): both shared-memory loads are
@@ -387,12 +407,15 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
         const bool has1 = u1 < units;
         const uint4 q0 = sp[u];
         const uint4 q1 = has1 ? sp[u1] : make_uint4(0u, 0u, 0u, 0u);
-        cast_unit<kDt, kFmt, kColMul>(q0, e0 + static_cast<int64_t>(u) * kUnit, col_mul, cols, sc, dst);
-        if (has1) cast_unit<kDt, kFmt, kColMul>(q1, e0 + static_cast<int64_t>(u1) * kUnit, col_mul, cols, sc, dst);
+        cast_unit<kDt, kFmt, kColMul>(q0, e0 + static_cast<int64_t>(u) * kUnit,
+                                      kColMul ? static_cast<int>(wrap_col(col0 + static_cast<uint32_t>(u) * kUnit, ucols)) : 0, col_mul, table, sc, dst);
+        if (has1)
+          cast_unit<kDt, kFmt, kColMul>(q1, e0 + static_cast<int64_t>(u1) * kUnit,
+                                        kColMul ? static_cast<int>(wrap_col(col0 + static_cast<uint32_t>(u1) * kUnit, ucols)) : 0, col_mul, table, sc, dst);
       }
-      if (t + kStagedSlots < n_my) {
+      if (t + slots < n_my) {
         if (!__syncthreads_and(ok)) { failed = true; break; }
-        if (tid == 0) issue(i - kStagedSlots);
+        if (tid == 0) issue(i - slots);
       }
     }
     if (blockIdx.x == 0) {
@@ -536,8 +559,15 @@ cudaError_t launch_staged_variant(const void* src, int64_t count, uint8_t* dst, 
   if (grid > resident) grid = resident;
   if (grid > kMaxAbsmaxParts) grid = kMaxAbsmaxParts;
   if (grid < 1) grid = 1;
+  // per-row mode: the column factors live in shared memory too when they fit beside at least eight ring slots
+  int table_floats = 0, slots = kStagedSlots;
+  if (kColMul) {
+    const int table_chunks = static_cast<int>((static_cast<int64_t>(cols) * 4 + kChunkBytes - 1) / kChunkBytes);
+    if (table_chunks <= kStagedSlots - 8) { table_floats = cols; slots = kStagedSlots - table_chunks; }
+  }
   return launch_pdl(quantize_staged_kernel<kDt, kFmt, kColMul>, dim3(static_cast<unsigned>(grid)), dim3(kStagedThreads), kSmem,
-                    stream, 1, src, count, dst, partial, static_cast<GridSync*>(sync), out, status, col_mul, cols, oa_job);
+                    stream, 1, src, count, dst, partial, static_cast<GridSync*>(sync), out, status, col_mul, cols, oa_job, slots,
+                    table_floats);
 }
 
 cudaError_t launch_quantize_fused(const void* src, int src_dt, int64_t count, int fmt, uint8_t* dst, uint32_t* partial,

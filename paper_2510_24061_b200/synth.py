@@ -171,3 +171,11 @@ def config1():
     """LLaMA-7B projection set of one decoder layer: tokens 4096, rank 64, 1% outlier channels, top-256."""
     return dict(seed=0, linears=LLAMA_7B_LINEARS, T=4096, r=64, alpha=64.0, k=256, steps=10, lr=2e-4,
                 outlier_frac=0.01)
+
+
+def config3():
+    """LLaMA-13B projection set: hidden 5120, MLP 13824, tokens 8192, rank 64, top-512; heavy-tailed backbone rows
+    (0.02 * Student-t with 3 degrees of freedom) with one scale per row."""
+    return dict(seed=0, linears=LLAMA_13B_LINEARS, T=8192, r=64, alpha=64.0, k=512, steps=10, lr=2e-4,
+                outlier_frac=0.01, per_row=True, heavy_tailed=True)
+
