@@ -287,6 +287,20 @@ def setup_layer(W, A, B, gamma: float, per_row: bool = False):
     return wq, s_w, dbuf
 
 
+def svd_init(W, r: int):
+    """Alg. 1 lines 3-5 (Eq. q_error, Eq. reform): W~, s_W = Q(W); Delta W = W - W~ / s_W; (B^, A^) = the rank-r
+    truncated SVD of Delta W, the singular values split evenly: B^ = U_r sqrt(S_r), A^ = sqrt(S_r) V_r^T (the paper
+    does not say how they are split; only A^ enters the melded layer, and only up to the sign of each row).
+    fp64 throughout, numpy's LAPACK SVD as the library step.  Returns (wq [m, n] codes, s_W, A^ [r, n], B^ [m, r],
+    sigma [min(m, n)] all singular values)."""
+    W = _c(W, np.float32)
+    wq, s_w, _ = quantize(W, E4M3)
+    E = W.astype(np.float64) - decode_array(wq, E4M3).reshape(W.shape) / np.float64(s_w)
+    U, S, Vt = np.linalg.svd(E, full_matrices=False)
+    root = np.sqrt(S[:r])
+    return wq, s_w, root[:, None] * Vt[:r], U[:, :r] * root[None, :], S
+
+
 def layer_forward(X, wq, s_w, m: int, r: int):
     """Alg. 2 lines 5-9 for one layer.  Returns dict(xq, s_x, Y, OA, amax_oa)."""
     xq, s_x, _ = quantize(X, E4M3)
