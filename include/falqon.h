@@ -215,6 +215,26 @@ int falqon_proxy_update_adamw(const falqon_layer *L, const float *dB, float *exp
 int falqon_proxy_update_static(const falqon_layer *L, const float *dB, float lr, int64_t k, int32_t *idx_out,
                                falqon_stream stream);
 
+/* Initialisation of the adapter from the quantization error (Alg. 1 lines 4-5; Eq. q_error, Eq. reform):
+ *     Delta W = W - dec(W~) / s_W,      A^ = sqrt(S_r) V_r^T   of the rank-r truncated SVD  Delta W ~ U_r S_r V_r^T
+ * (the singular values split evenly between B^ = U_r sqrt(S_r) and A^; only A^ enters the melded layer, B^ is what
+ * quantization already did to W).  Computed by a randomized subspace iteration with `power_iters` power steps, fp32,
+ * set-up code off the per-step path; its accuracy is that of the method: excellent where the spectrum of Delta W
+ * decays, a near-optimal r-dimensional subspace where it is flat (the rows of A^ are then not individually
+ * meaningful).  Per-tensor scaled W~ only.
+ *   W        device [m][n] bf16 or fp32, the backbone that was quantized
+ *   wq, s_w  device [m][n] E4M3 codes and [1] scale from falqon_quantize(W)
+ *   omega    device [n][l] fp32, an i.i.d. standard normal test matrix drawn by the caller; l even, r <= l <= 160
+ *            (l = r + 16 is a good choice)
+ *   A_hat    device [r][n] fp32 out; each row is determined up to its sign
+ *   sigma    device [r] fp32 out: the leading singular values of Delta W
+ *   scratch  device, falqon_svd_init_scratch_bytes(m, n, l) bytes
+ * Returns FALQON_OK, FALQON_ERR_INVALID_ARG, FALQON_ERR_WORKSPACE or FALQON_ERR_CUDA. */
+size_t falqon_svd_init_scratch_bytes(int64_t m, int64_t n, int64_t l);
+int falqon_svd_init(const void *W, falqon_dtype w_dt, int64_t m, int64_t n, const uint8_t *wq, const float *s_w, int64_t r,
+                    const float *omega, int64_t l, int32_t power_iters, float *A_hat, float *sigma, void *scratch,
+                    size_t scratch_bytes, falqon_stream stream);
+
 /* The proxy update with a CORRECTLY ROUNDED merge (an extension: the paper does not fix the merge arithmetic, and
  * falqon_proxy_update reads it as an fp32 fma chain).  Steps 1-3 (optimizer, scores, top-k) and the clearing are the
  * same; the merge becomes

@@ -22,6 +22,7 @@ WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 
 EXPORTS = ["falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
+           "falqon_svd_init_scratch_bytes", "falqon_svd_init",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_last_device_status", "falqon_launch_count",
            "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static", "falqon_workspace_init", "falqon_proxy_update_adamw"]
 STATIC_MAX_ROWS = 16384
@@ -71,6 +72,10 @@ lib.falqon_exact_merge_scratch_bytes.restype = _sz
 lib.falqon_exact_merge_scratch_bytes.argtypes = [_i64, _i64, _i64]
 lib.falqon_proxy_update_exact.restype = _i
 lib.falqon_proxy_update_exact.argtypes = [C.POINTER(falqon_layer), _p, _f, _i64, _p, _p, _sz, _p, _sz, _p, _p, _p]
+lib.falqon_svd_init_scratch_bytes.restype = _sz
+lib.falqon_svd_init_scratch_bytes.argtypes = [_i64, _i64, _i64]
+lib.falqon_svd_init.restype = _i
+lib.falqon_svd_init.argtypes = [_p, _i, _i64, _i64, _p, _p, _i64, _p, _i64, C.c_int32, _p, _p, _p, _sz, _p]
 lib.falqon_proxy_update_static.restype = _i
 lib.falqon_proxy_update_static.argtypes = [C.POINTER(falqon_layer), _p, _f, _i64, _p, _p]
 lib.falqon_last_device_status.restype = _i
@@ -298,6 +303,33 @@ def proxy_update_exact(layer: Layer, dB: torch.Tensor | None, lr: float, k: int,
            lib.falqon_proxy_update_exact(C.byref(layer.c), _ptr(dB), lr, k, _ptr(idx_out), _ptr(ws), ws.numel(), _ptr(scratch),
                                          scratch.numel(), _ptr(sums), _ptr(fixed), _stream()))
     return idx_out, fixed, sums
+
+
+def svd_init(W: torch.Tensor, wq: torch.Tensor, s_w: torch.Tensor, r: int, omega: torch.Tensor, power_iters: int = 2):
+    """falqon_svd_init: A^ [r, n] fp32 and the r leading singular values of Delta W = W - dec(wq) / s_w.
+    wq: uint8 [m, n] codes of W (per-tensor scale s_w); omega: fp32 [n, l] standard normal, l even, r <= l <= 160."""
+    m, n = W.shape
+    l = omega.shape[1]
+    assert wq.shape == (m, n) and wq.dtype == torch.uint8 and wq.is_contiguous() and W.is_contiguous()
+    assert omega.shape[0] == n and omega.dtype == torch.float32 and omega.is_contiguous()
+    dev = W.device
+    A_hat = torch.empty((r, n), dtype=torch.float32, device=dev)
+    sigma = torch.empty(r, dtype=torch.float32, device=dev)
+    scratch = torch.empty(int(lib.falqon_svd_init_scratch_bytes(m, n, l)), dtype=torch.uint8, device=dev)
+    _check("falqon_svd_init", lib.falqon_svd_init(_ptr(W), _dt(W), m, n, _ptr(wq), _ptr(s_w), r, _ptr(omega), l, power_iters,
+                                                  _ptr(A_hat), _ptr(sigma), _ptr(scratch), scratch.numel(), _stream()))
+    return A_hat, sigma
+
+
+def setup_layer_svd(W: torch.Tensor, r: int, omega: torch.Tensor, power_iters: int = 2) -> Layer:
+    """Alg. 1 in full for one layer: W~, s_W = Q(W); A^ from the SVD of the quantization error; A~ = Q(A^; s_W);
+    W~' = [W~; A~]; DeltaBuffer = 0.  omega: fp32 [n, l] standard normal drawn by the caller."""
+    m, n = W.shape
+    wq = torch.empty((m + r, n), dtype=torch.uint8, device=W.device)
+    _, s_w, _ = quantize(W.contiguous(), E4M3, dst=wq[:m])
+    A_hat, _ = svd_init(W.contiguous(), wq[:m], s_w, r, omega, power_iters)
+    quantize(A_hat, E4M3, scale_in=s_w, want_amax=False, dst=wq[m:])
+    return Layer(wq, s_w, torch.zeros((m, r), dtype=torch.float32, device=W.device), r)
 
 
 def setup_layer(W: torch.Tensor, A: torch.Tensor, B: torch.Tensor | None, gamma: float, per_row: bool = False) -> Layer:

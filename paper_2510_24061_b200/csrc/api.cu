@@ -427,6 +427,23 @@ int falqon_proxy_update_exact(const falqon_layer* L, const float* dB, float lr, 
   return proxy_update_impl(L, dB, lr, nullptr, nullptr, nullptr, k, idx_out, ws, ws_bytes, stream, &exact);
 }
 
+size_t falqon_svd_init_scratch_bytes(int64_t m, int64_t n, int64_t l) {
+  if (m < 16 || n < 16 || m % 16 || n % 16 || l < 2 || l % 2 || l > 160) return 0;
+  return svd_init_scratch_bytes(m, n, l);
+}
+
+int falqon_svd_init(const void* W, falqon_dtype w_dt, int64_t m, int64_t n, const uint8_t* wq, const float* s_w, int64_t r,
+                    const float* omega, int64_t l, int32_t power_iters, float* A_hat, float* sigma, void* scratch,
+                    size_t scratch_bytes, falqon_stream stream) {
+  if (W == nullptr || wq == nullptr || s_w == nullptr || omega == nullptr || A_hat == nullptr || sigma == nullptr ||
+      !dtype_ok(w_dt) || m < 16 || n < 16 || m % 16 || n % 16 || r < 1 || l < r || l % 2 || l > 160 || l > m || l > n ||
+      power_iters < 0 || power_iters > 16 || !aligned16(W) || !aligned16(wq) || !aligned16(omega) || !aligned16(A_hat))
+    return FALQON_ERR_INVALID_ARG;
+  if (scratch == nullptr || !aligned16(scratch) || scratch_bytes < svd_init_scratch_bytes(m, n, l)) return FALQON_ERR_WORKSPACE;
+  FALQON_CUDA(launch_svd_init(W, w_dt, m, n, wq, s_w, r, omega, l, power_iters, A_hat, sigma, scratch, stream));
+  return FALQON_OK;
+}
+
 int falqon_last_device_status(falqon_stream stream) {
   if (cudaStreamSynchronize(stream) != cudaSuccess) return FALQON_ERR_CUDA;
   int* p = status_ptr();

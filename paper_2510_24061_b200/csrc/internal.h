@@ -124,6 +124,13 @@ cudaError_t launch_merge_exact(uint8_t* wq, float* dbuf, const int32_t* sel_idx,
                                const float* row_scales, void* scratch, float* sums_out, unsigned int* fix_count_out, int* status,
                                cudaStream_t stream);
 
+// ---- svd_init.cu: A^ = sqrt(S_r) V_r^T of Delta W = W - dec(W~) / s_W by randomized subspace iteration (set-up code).
+// omega: [n][l] fp32 Gaussian test matrix drawn by the caller, l even, r <= l <= 160; scratch: svd_init_scratch_bytes.
+size_t svd_init_scratch_bytes(int64_t m, int64_t n, int64_t l);
+cudaError_t launch_svd_init(const void* w, int w_dt, int64_t m, int64_t n, const uint8_t* wq, const float* s_w, int64_t r,
+                            const float* omega, int64_t l, int power_iters, float* a_hat, float* sigma, void* scratch,
+                            cudaStream_t stream);
+
 // ---- proxy_update.cu
 cudaError_t launch_sgd_score(float* dbuf, const float* dB, float lr, int64_t m, int64_t r, float* score,
                              cudaStream_t stream);
