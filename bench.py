@@ -149,14 +149,24 @@ def build_workload(fq, device, seed, T, r, k, linears, outlier_frac, per_row=Fal
     return layers
 
 
-def run_step(fq, layers, lr, k):
+def run_step(fq, layers, lr, k, batch=None):
+    """Forward and backward of every projection, and the proxy update of each: one batched call for the whole set
+    (batch: a ProxyBatch over the layers' gradient buffers), or one call per projection when batch is None."""
     for L in layers:
         _, OA, amax_oa, _ = fq.melded_forward(L["layer"], L["X"], ws=L["ws"], out=L["out_f"])
         _, dB, _ = fq.melded_backward(L["layer"], L["dY"], OA, amax_oa, ws=L["ws"], out=L["out_b"])
-        fq.proxy_update(L["layer"], dB, lr, k, ws=L["ws"], idx_out=L["idx"])
+        if batch is None:
+            fq.proxy_update(L["layer"], dB, lr, k, ws=L["ws"], idx_out=L["idx"])
+    if batch is not None:
+        batch.run(lr)
 
 
-def run_step_e2e(fq, layers, host, lr, k, pipe):
+def make_proxy_batch(fq, layers, k):
+    return fq.ProxyBatch([L["layer"] for L in layers], [L["out_b"][1] for L in layers], [k] * len(layers),
+                         wss=[L["ws"] for L in layers], idx_outs=[L["idx"] for L in layers])
+
+
+def run_step_e2e(fq, layers, host, lr, k, pipe, batch=None):
     """Same step, but every input starts in pinned host memory and the results are read back.  The uploads run on a
     copy stream one projection ahead of the compute stream (each projection has its own device buffers; an event
     per projection says when its inputs have landed, another when the compute no longer reads them)."""
@@ -173,9 +183,15 @@ def run_step_e2e(fq, layers, host, lr, k, pipe):
         _, OA, amax_oa, _ = fq.melded_forward(L["layer"], L["X"], ws=L["ws"], out=L["out_f"])
         _, dB, _ = fq.melded_backward(L["layer"], L["dY"], OA, amax_oa, ws=L["ws"], out=L["out_b"])
         pipe["consumed"][i].record(compute)
-        fq.proxy_update(L["layer"], dB, lr, k, ws=L["ws"], idx_out=L["idx"])
+        if batch is None:
+            fq.proxy_update(L["layer"], dB, lr, k, ws=L["ws"], idx_out=L["idx"])
         H["dB"].copy_(dB, non_blocking=True)
-        H["idx"].copy_(L["idx"], non_blocking=True)
+        if batch is None:
+            H["idx"].copy_(L["idx"], non_blocking=True)
+    if batch is not None:
+        batch.run(lr)
+        for L, H in zip(layers, host):
+            H["idx"].copy_(L["idx"], non_blocking=True)
 
 
 def make_e2e_pipe(n_layers):
@@ -290,7 +306,8 @@ def run_stack(args):
     T, r, k, lr = cfg["T"], cfg["r"], cfg["k"], cfg["lr"]
     H, F, n_layers = 4096, 11008, args.stack_layers
     peaks = measured_peaks()
-    stack = st.Stack(n_layers, H, F, T, r, k, seed=cfg["seed"], device=dev, lr=lr, producer_amax=not args.stack_own_absmax)
+    stack = st.Stack(n_layers, H, F, T, r, k, seed=cfg["seed"], device=dev, lr=lr, producer_amax=not args.stack_own_absmax,
+                     batched_proxy=not args.proxy_per_layer)
     h0 = synth.normal_bf16(cfg["seed"], 9001, (T, H), 1.0, dev)
     G = synth.normal_bf16(cfg["seed"], 9002, (T, H), 1.0e-2, dev)
     steps, warmup = max(1, min(args.steps, 20)), max(3, min(args.warmup, 5))
@@ -358,6 +375,8 @@ def main():
     ap.add_argument("--config3", action="store_true",
                     help="configs[3] instead of configs[1]: the LLaMA-13B projection set, 8192 tokens, per-row-scaled "
                          "heavy-tailed backbone, top-512 (not the headline line)")
+    ap.add_argument("--proxy-per-layer", action="store_true",
+                    help="run one falqon_proxy_update per projection instead of one falqon_proxy_update_batched per step")
     ap.add_argument("--only", default=None, help="profiling aid: restrict the workload to one projection (q,k,v,o,gate,up,down)")
     args = ap.parse_args()
 
@@ -377,7 +396,8 @@ def main():
                 "tokens": T, "rank": r, "topk": k, "matrices": len(linears), "gflop_per_step": flops_step / 1e9,
                 "l2": "inputs larger than L2 (%.2f GB of inputs and outputs touched per step)" %
                       (sum(2.0 * T * (n + m) * 2 for _, n, m in linears) / 1e9),
-                "parallelism": f"replicas x{world}"}
+                "parallelism": f"replicas x{world}",
+                "proxy_update": "one call per projection" if args.proxy_per_layer else "one batched call per step"}
 
     if args.sweep:
         if rank == 0:
@@ -428,9 +448,10 @@ def main():
     def max_over_ranks(ms):
         return aggregate_over_ranks(ms, 0.0, dist, device)[0]
 
+    batch = None if args.proxy_per_layer else make_proxy_batch(fq, layers, k)
     # ---- device-resident timing: EXACTLY --steps steps between two events, nothing else in the stream
     for _ in range(max(args.warmup, 3)):
-        run_step(fq, layers, lr, k)
+        run_step(fq, layers, lr, k, batch)
     barrier()
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -438,7 +459,7 @@ def main():
     barrier()
     ev0.record()
     for _ in range(args.steps):
-        run_step(fq, layers, lr, k)
+        run_step(fq, layers, lr, k, batch)
     ev1.record()
     barrier()
     ms_total = max_over_ranks(ev0.elapsed_time(ev1))
@@ -453,7 +474,7 @@ def main():
     barrier()
     ev0.record()
     for _ in range(args.steps):
-        run_step(fq, layers, lr, k)
+        run_step(fq, layers, lr, k, batch)
     ev1.record()
     barrier()
     ms_step_instrumented = max_over_ranks(ev0.elapsed_time(ev1)) / args.steps
@@ -487,7 +508,7 @@ def main():
     # ---- stage breakdown (separate untimed-for-value pass with every stage bracketed)
     fq.profile_start(10 * len(layers) * 3, None)
     for _ in range(3):
-        run_step(fq, layers, lr, k)
+        run_step(fq, layers, lr, k, batch)
     torch.cuda.synchronize()
     breakdown = {}
     for name, ms in fq.profile_stop(10 * len(layers) * 3):
@@ -507,19 +528,20 @@ def main():
     e2e_steps = max(3, min(args.steps, 20))
     pipe = make_e2e_pipe(len(layers))
     for _ in range(2):
-        run_step_e2e(fq, layers, host, lr, k, pipe)
+        run_step_e2e(fq, layers, host, lr, k, pipe, batch)
     barrier()
     ev0.record()
     for _ in range(e2e_steps):
-        run_step_e2e(fq, layers, host, lr, k, pipe)
+        run_step_e2e(fq, layers, host, lr, k, pipe, batch)
     ev1.record()
     barrier()
     ms_e2e = max_over_ranks(ev0.elapsed_time(ev1)) / e2e_steps
     e2e_value = world * flops_step / (ms_e2e * 1e-3) / 1e12
 
-    launches_per_step = sum(fq.launch_count("falqon_melded_forward") +
-                            fq.launch_count("falqon_melded_backward") +
-                            fq.launch_count("falqon_proxy_update", k=k) for L in layers)
+    launches_per_step = sum(fq.launch_count("falqon_melded_forward") + fq.launch_count("falqon_melded_backward") +
+                            (fq.launch_count("falqon_proxy_update", k=k) if batch is None else 0) for L in layers)
+    if batch is not None:
+        launches_per_step += fq.launch_count("falqon_proxy_update_batched", k=k) * ((len(layers) + 7) // 8)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()

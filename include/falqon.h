@@ -181,6 +181,20 @@ int falqon_melded_backward_amax(const falqon_layer *L, const void *dY, falqon_dt
 int falqon_proxy_update(const falqon_layer *L, const float *dB, float lr, int64_t k, int32_t *idx_out,
                         void *ws, size_t ws_bytes, falqon_stream stream);
 
+/* falqon_proxy_update for `count` layers in two launches instead of 2 x count (Alg. 3 lines 4-6, Eq. update, for each
+ * layer; the paper's layer-wise schedule runs the updates of a block's projections back to back, and one layer's update
+ * moves only a few MB, so a single call is bound by launch latency rather than by memory).  All arrays are HOST arrays
+ * of `count` entries: layers[i] (each with its own wq / s_w / dbuf), dB[i] (device [m_i][r_i] fp32, or NULL for that
+ * layer), k[i], idx_out (NULL, or entries that are device [k_i] int32 or NULL), ws[i] / ws_bytes[i] (each layer's own
+ * initialised workspace, as for falqon_proxy_update; two layers must not share one).  The layers may differ in shape,
+ * rank, granularity and k.  lr is shared.  The result for every layer is bit-identical to its own
+ * falqon_proxy_update call.  Any invalid entry rejects the whole call before anything is launched.  count == 0 is a
+ * no-op.  A layer whose k needs more row groups than a workspace has counters for (k > 16384) makes the call fall back
+ * to per-layer launches, with the same results. */
+int falqon_proxy_update_batched(const falqon_layer *layers, int32_t count, const float *const *dB, float lr,
+                                const int64_t *k, int32_t *const *idx_out, void *const *ws, const size_t *ws_bytes,
+                                falqon_stream stream);
+
 /* The same update with AdamW as the optimizer -- the one the paper trains with (its Alg. 3 leaves "Optimizer"
  * generic).  exp_avg and exp_avg_sq are device [m][r] fp32 state, zero before step 1, updated in place; they are NOT
  * cleared when a row is merged (only DeltaBuffer rows are).  For every element, in fp32 and in this order:

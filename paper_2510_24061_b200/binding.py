@@ -23,7 +23,7 @@ WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 EXPORTS = ["falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
            "falqon_svd_init_scratch_bytes", "falqon_svd_init",
-           "falqon_melded_backward", "falqon_proxy_update", "falqon_last_device_status", "falqon_launch_count",
+           "falqon_melded_backward", "falqon_proxy_update", "falqon_proxy_update_batched", "falqon_last_device_status", "falqon_launch_count",
            "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static", "falqon_workspace_init", "falqon_proxy_update_adamw"]
 STATIC_MAX_ROWS = 16384
 STAGES = ["quant_x", "gemm_fwd", "quant_dy", "quant_oa", "gemm_dx", "gemm_db", "reduce_db", "sgd_score", "topk", "merge"]
@@ -61,6 +61,9 @@ lib.falqon_melded_backward.restype = _i
 lib.falqon_melded_backward.argtypes = [C.POINTER(falqon_layer), _p, _i, _i64, _p, _p, _p, _i, _p, _p, _p, _sz, _p]
 lib.falqon_proxy_update.restype = _i
 lib.falqon_proxy_update.argtypes = [C.POINTER(falqon_layer), _p, _f, _i64, _p, _p, _sz, _p]
+lib.falqon_proxy_update_batched.restype = _i
+lib.falqon_proxy_update_batched.argtypes = [C.POINTER(falqon_layer), C.c_int32, C.POINTER(_p), _f, C.POINTER(_i64), C.POINTER(_p),
+                                            C.POINTER(_p), C.POINTER(_sz), _p]
 class falqon_adamw(C.Structure):
     _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
                 ("weight_decay", C.c_float), ("step", C.c_int64)]
@@ -284,6 +287,39 @@ def proxy_update(layer: Layer, dB: torch.Tensor | None, lr: float, k: int, ws: t
     _check("falqon_proxy_update", lib.falqon_proxy_update(C.byref(layer.c), _ptr(dB), lr, k, _ptr(idx_out), _ptr(ws),
                                                           ws.numel(), _stream()))
     return idx_out
+
+
+class ProxyBatch:
+    """The host arrays of one falqon_proxy_update_batched call, marshalled once and reusable while the tensors live:
+    layers, their adapter gradients (entries may be None), k per layer, workspaces and index outputs."""
+
+    def __init__(self, layers, dBs, ks, wss=None, idx_outs=None):
+        n = len(layers)
+        assert len(dBs) == n and len(ks) == n
+        self.layers, self.dBs, self.ks = list(layers), list(dBs), [int(k) for k in ks]
+        self.wss = [L.workspace(1) for L in layers] if wss is None else list(wss)
+        if idx_outs is None:
+            idx_outs = [torch.empty(k, dtype=torch.int32, device=L.wq.device) if 0 < k <= L.m else None
+                        for L, k in zip(self.layers, self.ks)]
+        self.idx_outs = list(idx_outs)
+        self.c_layers = (falqon_layer * max(n, 1))(*[L.c for L in self.layers])
+        self.c_dB = (_p * max(n, 1))(*[_ptr(t) for t in self.dBs])
+        self.c_k = (_i64 * max(n, 1))(*self.ks)
+        self.c_idx = (_p * max(n, 1))(*[_ptr(t) for t in self.idx_outs])
+        self.c_ws = (_p * max(n, 1))(*[_ptr(t) for t in self.wss])
+        self.c_ws_bytes = (_sz * max(n, 1))(*[t.numel() for t in self.wss])
+        self.count = n
+
+    def run(self, lr: float):
+        _check("falqon_proxy_update_batched",
+               lib.falqon_proxy_update_batched(self.c_layers, self.count, self.c_dB, lr, self.c_k, self.c_idx, self.c_ws,
+                                               self.c_ws_bytes, _stream()))
+        return self.idx_outs
+
+
+def proxy_update_batched(layers, dBs, lr: float, ks, wss=None, idx_outs=None):
+    """falqon_proxy_update_batched: the proxy update of several layers in two launches.  Returns the list of idx tensors."""
+    return ProxyBatch(layers, dBs, ks, wss, idx_outs).run(lr)
 
 
 def proxy_update_exact(layer: Layer, dB: torch.Tensor | None, lr: float, k: int, ws: torch.Tensor | None = None,

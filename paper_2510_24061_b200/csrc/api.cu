@@ -401,6 +401,64 @@ int falqon_proxy_update(const falqon_layer* L, const float* dB, float lr, int64_
   return proxy_update_impl(L, dB, lr, nullptr, nullptr, nullptr, k, idx_out, ws, ws_bytes, stream);
 }
 
+int falqon_proxy_update_batched(const falqon_layer* layers, int32_t count, const float* const* dB, float lr, const int64_t* k,
+                                int32_t* const* idx_out, void* const* ws, const size_t* ws_bytes, falqon_stream stream) {
+  if (count < 0 || !(lr == lr)) return FALQON_ERR_INVALID_ARG;
+  if (count == 0) return FALQON_OK;
+  if (layers == nullptr || dB == nullptr || k == nullptr || ws == nullptr || ws_bytes == nullptr) return FALQON_ERR_INVALID_ARG;
+  bool fused = true;
+  for (int32_t i = 0; i < count; ++i) {
+    const falqon_layer* L = &layers[i];
+    if (!layer_ok(L) || k[i] < 0 || k[i] > L->m || (dB[i] != nullptr && !aligned16(dB[i]))) return FALQON_ERR_INVALID_ARG;
+    WorkspaceLayout w;
+    if (!make_layout(L->m, L->n, L->r, 1, &w)) return FALQON_ERR_INVALID_ARG;
+    if (ws[i] == nullptr || !aligned16(ws[i]) || ws_bytes[i] < w.total) return FALQON_ERR_WORKSPACE;
+    for (int32_t j = 0; j < i; ++j)
+      if (ws[j] == ws[i] || layers[j].wq == L->wq || layers[j].dbuf == L->dbuf) return FALQON_ERR_INVALID_ARG;
+    if (static_cast<size_t>(merge_group_count(k[i])) > kMaxMergeGroups) fused = false;
+  }
+  if (!fused) {
+    for (int32_t i = 0; i < count; ++i) {
+      const int rc = proxy_update_impl(&layers[i], dB[i], lr, nullptr, nullptr, nullptr, k[i],
+                                       idx_out != nullptr ? idx_out[i] : nullptr, ws[i], ws_bytes[i], stream);
+      if (rc != FALQON_OK) return rc;
+    }
+    return FALQON_OK;
+  }
+  for (int32_t first = 0; first < count; first += kProxyBatchMax) {
+    const int chunk = count - first < kProxyBatchMax ? count - first : kProxyBatchMax;
+    ProxyBatchLayer b[kProxyBatchMax];
+    bool any_merge = false;
+    for (int c = 0; c < chunk; ++c) {
+      const int32_t i = first + c;
+      const falqon_layer* L = &layers[i];
+      WorkspaceLayout w;
+      make_layout(L->m, L->n, L->r, 1, &w);
+      uint8_t* base = static_cast<uint8_t*>(ws[i]);
+      b[c].wq = L->wq;
+      b[c].dbuf = L->dbuf;
+      b[c].dB = dB[i];
+      b[c].row_scales = L->gran == FALQON_PER_ROW ? L->s_w : nullptr;
+      b[c].score = reinterpret_cast<float*>(base + w.score);
+      b[c].sel_idx = reinterpret_cast<int32_t*>(base + w.sel_idx);
+      b[c].idx_out = idx_out != nullptr ? idx_out[i] : nullptr;
+      b[c].done_counter = reinterpret_cast<unsigned int*>(base + w.scales + kDoneOffset);
+      b[c].group_counters = reinterpret_cast<unsigned int*>(base + w.scales + kGroupCountersOffset);
+      b[c].m = L->m; b[c].n = L->n; b[c].r = L->r; b[c].k = k[i];
+      any_merge = any_merge || k[i] > 0;
+    }
+    {
+      StageTimer timer(FALQON_STAGE_SGD_SCORE, stream);
+      FALQON_CUDA(launch_proxy_update_batched(b, chunk, lr, 0, stream));
+    }
+    if (any_merge) {
+      StageTimer timer(FALQON_STAGE_MERGE, stream);
+      FALQON_CUDA(launch_proxy_update_batched(b, chunk, lr, 1, stream));
+    }
+  }
+  return FALQON_OK;
+}
+
 int falqon_proxy_update_adamw(const falqon_layer* L, const float* dB, float* exp_avg, float* exp_avg_sq,
                               const falqon_adamw* hp, int64_t k, int32_t* idx_out, void* ws, size_t ws_bytes,
                               falqon_stream stream) {
@@ -504,6 +562,7 @@ int falqon_launch_count(const char* entry_point, int64_t m, int64_t n, int64_t r
   if (std::strcmp(entry_point, "falqon_melded_forward") == 0) return 2;     // fused quantize, GEMM
   if (std::strcmp(entry_point, "falqon_melded_backward") == 0) return 3;    // fused quantize, dX, fused dB
   if (std::strcmp(entry_point, "falqon_proxy_update") == 0) return k > 0 ? 2 : 1;  // optimizer+score+top-k, merge+clear
+  if (std::strcmp(entry_point, "falqon_proxy_update_batched") == 0) return k > 0 ? 2 : 1;   // per 8 layers
   return 0;
 }
 

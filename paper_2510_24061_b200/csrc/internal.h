@@ -154,4 +154,22 @@ cudaError_t launch_adamw_score_topk(float* dbuf, const float* dB, float* exp_avg
 cudaError_t launch_merge_rows_fused(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n,
                                     int64_t r, unsigned int* group_counters, const float* row_scales, cudaStream_t stream);
 
+// The two fused kernels over up to kProxyBatchMax layers per launch (plain SGD; dB null = no optimizer step for that
+// layer).  Every layer brings its own score / selection regions and counters; results are those of the per-layer calls.
+constexpr int kProxyBatchMax = 8;
+struct ProxyBatchLayer {
+  uint8_t* wq;
+  float* dbuf;
+  const float* dB;
+  const float* row_scales;      // null for a per-tensor scale
+  float* score;
+  int32_t* sel_idx;
+  int32_t* idx_out;             // nullable
+  unsigned int* done_counter;
+  unsigned int* group_counters;
+  int64_t m, n, r, k;
+};
+// phase 0: optimizer step, scores and selection of every layer; phase 1: the merge of every layer with k > 0.
+cudaError_t launch_proxy_update_batched(const ProxyBatchLayer* layers, int count, float lr, int phase, cudaStream_t stream);
+
 }  // namespace falqon

@@ -221,18 +221,14 @@ __device__ __forceinline__ float optimizer_update(const OptimizerArgs& o, float 
 // ---- optimizer step + row scores + selection in ONE kernel: CTAs of 1024 threads take 128 rows each; the CTA
 // that finishes last (a counter in the workspace that is zero between calls) runs the selection on all scores.
 constexpr int kFusedScoreRows = 128;
-__global__ void __launch_bounds__(kTopkThreads) sgd_score_topk_kernel(float* dbuf, const float* dB,
-                                                                      OptimizerArgs opt, int m, int r, int k,
-                                                                      float* score, int32_t* sel_idx,
-                                                                      int32_t* idx_out,
-                                                                      unsigned int* done_counter, int use_smem) {
-  extern __shared__ float fused_smem[];  // [kFusedScoreRows][r + 1] floats, later the m staged scores
+// cta / n_ctas: this CTA's position among the CTAs that work on the layer.  fused_smem: [kFusedScoreRows][r + 1]
+// floats, later the m staged scores.
+__device__ __forceinline__ void score_topk_body(float* dbuf, const float* dB, const OptimizerArgs& opt, int m, int r, int k,
+                                                float* score, int32_t* sel_idx, int32_t* idx_out,
+                                                unsigned int* done_counter, int use_smem, int cta, int n_ctas,
+                                                float* fused_smem) {
   __shared__ int s_last;
-  // The wait comes first: the merge that follows reads the A~ rows before its own wait, which is only safe
-  // once every earlier kernel on the stream has finished, i.e. once this kernel is past this point.
-  pdl_wait();
-  pdl_trigger();
-  const int row0 = blockIdx.x * kFusedScoreRows;
+  const int row0 = cta * kFusedScoreRows;
   const int rows = min(kFusedScoreRows, m - row0);
   const int64_t base = (int64_t)row0 * r;
   const int total = rows * r;
@@ -277,13 +273,59 @@ __global__ void __launch_bounds__(kTopkThreads) sgd_score_topk_kernel(float* dbu
   __syncthreads();
   if (threadIdx.x == 0) {
     const unsigned int prev = atomicAdd(done_counter, 1u);
-    s_last = (prev == gridDim.x - 1) ? 1 : 0;
+    s_last = (prev == static_cast<unsigned int>(n_ctas) - 1u) ? 1 : 0;
     if (s_last) *done_counter = 0u;       // back to zero for the next call
   }
   __syncthreads();
   if (!s_last) return;
   __threadfence();
   topk_block(score, m, k, sel_idx, idx_out, use_smem ? reinterpret_cast<uint32_t*>(fused_smem) : nullptr);
+}
+
+__global__ void __launch_bounds__(kTopkThreads) sgd_score_topk_kernel(float* dbuf, const float* dB,
+                                                                      OptimizerArgs opt, int m, int r, int k,
+                                                                      float* score, int32_t* sel_idx,
+                                                                      int32_t* idx_out,
+                                                                      unsigned int* done_counter, int use_smem) {
+  extern __shared__ float fused_smem_dyn[];
+  // The wait comes first: the merge that follows reads the A~ rows before its own wait, which is only safe
+  // once every earlier kernel on the stream has finished, i.e. once this kernel is past this point.
+  pdl_wait();
+  pdl_trigger();
+  score_topk_body(dbuf, dB, opt, m, r, k, score, sel_idx, idx_out, done_counter, use_smem, blockIdx.x, gridDim.x,
+                  fused_smem_dyn);
+}
+
+// The same for several layers in one launch: the CTAs of all layers are laid end to end and each finds its layer
+// from the table of first-CTA indices.  Plain SGD (or none, where a layer's dB is null).
+struct BatchedScoreLayer {
+  float* dbuf;
+  const float* dB;
+  float* score;
+  int32_t* sel_idx;
+  int32_t* idx_out;
+  unsigned int* done_counter;
+  int m, r, k, cta_begin;
+};
+struct BatchedScoreArgs {
+  BatchedScoreLayer layer[kProxyBatchMax];
+  int count;
+  float neg_lr;
+};
+__global__ void __launch_bounds__(kTopkThreads) score_topk_batched_kernel(const __grid_constant__ BatchedScoreArgs args) {
+  extern __shared__ float fused_smem_dyn[];
+  pdl_wait();
+  pdl_trigger();
+  int l = 0;
+#pragma unroll 1
+  for (int i = 1; i < args.count; ++i) l = static_cast<int>(blockIdx.x) >= args.layer[i].cta_begin ? i : l;
+  const BatchedScoreLayer& a = args.layer[l];
+  const int n_ctas = (a.m + kFusedScoreRows - 1) / kFusedScoreRows;
+  OptimizerArgs opt{};
+  opt.kind = a.dB != nullptr ? 1 : 0;
+  opt.neg_lr = args.neg_lr;
+  score_topk_body(a.dbuf, a.dB, opt, a.m, a.r, a.k, a.score, a.sel_idx, a.idx_out, a.done_counter,
+                  a.m <= kTopkSmemRows ? 1 : 0, static_cast<int>(blockIdx.x) - a.cta_begin, n_ctas, fused_smem_dyn);
 }
 
 // ---- W~[i][:] <- sat_rne_e4m3(W~[i][:] + DeltaBuffer[i][:] * A~) for the selected rows.
@@ -303,18 +345,16 @@ __device__ __forceinline__ void decode4(uint32_t w, float (&a)[4]) {
   a[0] = p0.x; a[1] = p0.y; a[2] = p1.x; a[3] = p1.y;
 }
 
-__global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* wq, float* dbuf,
-                                                                   const int32_t* sel_idx, int k, int64_t m,
-                                                                   int64_t n, int r, unsigned int* group_counters,
-                                                                   const float* row_scales) {
-  extern __shared__ __align__(16) float merge_smem[];
+// col_tile / group: which 128 columns and which 32 selected rows this CTA owns; n_col_tiles: CTAs per row group.
+__device__ __forceinline__ void merge_rows_body(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int k, int64_t m, int64_t n,
+                                                int r, unsigned int* group_counters, const float* row_scales, int col_tile,
+                                                int group, int n_col_tiles, float* merge_smem) {
   float* a_tile = merge_smem;                         // [r][kMergeCols] decoded A~
   float* sdb = merge_smem + (size_t)r * kMergeCols;   // [kMergeRows][r]
   __shared__ int srow[kMergeRows];
-  pdl_trigger();
-  const int g0 = blockIdx.y * kMergeRows;
+  const int g0 = group * kMergeRows;
   const int nrows = min(kMergeRows, k - g0);
-  const int64_t cta_c0 = (int64_t)blockIdx.x * kMergeCols;
+  const int64_t cta_c0 = (int64_t)col_tile * kMergeCols;
   const int cta_cols = static_cast<int>(min((int64_t)kMergeCols, n - cta_c0));   // multiple of 16
   // The A~ rows are decoded BEFORE the wait, while the selection kernel is still running: nothing on the proxy
   // update's path writes them, and the kernel launched before this one (the selection) releases this launch
@@ -381,9 +421,9 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* wq, 
   if (group_counters != nullptr) {
     __shared__ int s_clear;
     if (threadIdx.x == 0) {
-      const unsigned int prev = atomicAdd(&group_counters[blockIdx.y], 1u);
-      s_clear = (prev == gridDim.x - 1) ? 1 : 0;
-      if (s_clear) group_counters[blockIdx.y] = 0u;
+      const unsigned int prev = atomicAdd(&group_counters[group], 1u);
+      s_clear = (prev == static_cast<unsigned int>(n_col_tiles) - 1u) ? 1 : 0;
+      if (s_clear) group_counters[group] = 0u;
     }
     __syncthreads();
     if (s_clear) {
@@ -432,6 +472,42 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* wq, 
       if (ok1) *reinterpret_cast<uint32_t*>(row + lc1) = cvt_fp8x4<kE4M3>(v[q][4], v[q][5], v[q][6], v[q][7]);
     }
   }
+}
+
+__global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* wq, float* dbuf,
+                                                                   const int32_t* sel_idx, int k, int64_t m,
+                                                                   int64_t n, int r, unsigned int* group_counters,
+                                                                   const float* row_scales) {
+  extern __shared__ __align__(16) float merge_smem_dyn[];
+  pdl_trigger();
+  merge_rows_body(wq, dbuf, sel_idx, k, m, n, r, group_counters, row_scales, blockIdx.x, blockIdx.y, gridDim.x,
+                  merge_smem_dyn);
+}
+
+// Several layers in one launch (see score_topk_batched_kernel): a layer's CTAs are numbered column tile fastest.
+struct BatchedMergeLayer {
+  uint8_t* wq;
+  float* dbuf;
+  const int32_t* sel_idx;
+  unsigned int* group_counters;
+  const float* row_scales;
+  int64_t m, n;
+  int r, k, cta_begin, col_tiles;
+};
+struct BatchedMergeArgs {
+  BatchedMergeLayer layer[kProxyBatchMax];
+  int count;
+};
+__global__ void __launch_bounds__(kMergeThreads) merge_rows_batched_kernel(const __grid_constant__ BatchedMergeArgs args) {
+  extern __shared__ __align__(16) float merge_smem_dyn[];
+  pdl_trigger();
+  int l = 0;
+#pragma unroll 1
+  for (int i = 1; i < args.count; ++i) l = static_cast<int>(blockIdx.x) >= args.layer[i].cta_begin ? i : l;
+  const BatchedMergeLayer& a = args.layer[l];
+  const int local = static_cast<int>(blockIdx.x) - a.cta_begin;
+  merge_rows_body(a.wq, a.dbuf, a.sel_idx, a.k, a.m, a.n, a.r, a.group_counters, a.row_scales, local % a.col_tiles,
+                  local / a.col_tiles, a.col_tiles, merge_smem_dyn);
 }
 
 __global__ void __launch_bounds__(256) zero_rows_kernel(float* dbuf, const int32_t* sel_idx,
@@ -553,6 +629,50 @@ cudaError_t launch_adamw_score_topk(float* dbuf, const float* dB, float* exp_avg
   opt.exp_avg = exp_avg;
   opt.exp_avg_sq = exp_avg_sq;
   return launch_opt_score_topk(dbuf, dB, opt, m, r, k, score, sel_idx, idx_copy, done_counter, stream);
+}
+
+cudaError_t launch_proxy_update_batched(const ProxyBatchLayer* layers, int count, float lr, int phase, cudaStream_t stream) {
+  if (count < 1 || count > kProxyBatchMax) return cudaErrorInvalidValue;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t ea = cudaFuncSetAttribute(score_topk_batched_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(kTopkSmemRows * sizeof(uint32_t)));
+    if (ea != cudaSuccess) return ea;
+    ea = cudaFuncSetAttribute(merge_rows_batched_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 176 * 1024);
+    if (ea != cudaSuccess) return ea;
+    configured = true;
+  }
+  BatchedScoreArgs sa{};
+  BatchedMergeArgs ma{};
+  sa.count = count;
+  sa.neg_lr = -lr;
+  int score_ctas = 0, merge_ctas = 0;
+  size_t score_smem = 0, merge_smem = 0;
+  for (int i = 0; i < count; ++i) {
+    const ProxyBatchLayer& L = layers[i];
+    BatchedScoreLayer& a = sa.layer[i];
+    a.dbuf = L.dbuf; a.dB = L.dB; a.score = L.score; a.sel_idx = L.sel_idx; a.idx_out = L.idx_out;
+    a.done_counter = L.done_counter;
+    a.m = static_cast<int>(L.m); a.r = static_cast<int>(L.r); a.k = static_cast<int>(L.k);
+    a.cta_begin = score_ctas;
+    score_ctas += static_cast<int>((L.m + kFusedScoreRows - 1) / kFusedScoreRows);
+    size_t smem = sizeof(float) * kFusedScoreRows * (L.r + 1);
+    if (L.m <= kTopkSmemRows && static_cast<size_t>(L.m) * sizeof(uint32_t) > smem) smem = static_cast<size_t>(L.m) * sizeof(uint32_t);
+    if (smem > score_smem) score_smem = smem;
+    if (L.k > 0) {
+      BatchedMergeLayer& b = ma.layer[ma.count++];
+      b.wq = L.wq; b.dbuf = L.dbuf; b.sel_idx = L.sel_idx; b.group_counters = L.group_counters; b.row_scales = L.row_scales;
+      b.m = L.m; b.n = L.n; b.r = static_cast<int>(L.r); b.k = static_cast<int>(L.k);
+      b.cta_begin = merge_ctas;
+      b.col_tiles = static_cast<int>((L.n + kMergeCols - 1) / kMergeCols);
+      merge_ctas += b.col_tiles * merge_group_count(L.k);
+      const size_t ms = sizeof(float) * (static_cast<size_t>(L.r) * kMergeCols + static_cast<size_t>(kMergeRows) * L.r);
+      if (ms > merge_smem) merge_smem = ms;
+    }
+  }
+  if (phase == 0) return launch_pdl(score_topk_batched_kernel, dim3(score_ctas), dim3(kTopkThreads), score_smem, stream, 1, sa);
+  if (ma.count == 0) return cudaSuccess;
+  return launch_pdl(merge_rows_batched_kernel, dim3(merge_ctas), dim3(kMergeThreads), merge_smem, stream, 1, ma);
 }
 
 }  // namespace falqon

@@ -95,9 +95,12 @@ class Stack:
     """n_layers blocks with hidden size H and MLP width F, T tokens per step, LoRA rank r, top-k rows per update."""
 
     def __init__(self, n_layers: int, H: int, F: int, T: int, r: int, k: int, seed: int, device, lr: float = 2e-4,
-                 producer_amax: bool = True):
+                 producer_amax: bool = True, batched_proxy: bool = True):
         """producer_amax: the chain kernels hand the absmax of their outputs to the layers that consume them, whose
-        input casts are then single-pass (False: every layer takes the absmax of its input itself)."""
+        input casts are then single-pass (False: every layer takes the absmax of its input itself).
+        batched_proxy: the seven proxy updates of a block run as one falqon_proxy_update_batched call at the end of
+        the block's backward (False: one falqon_proxy_update after every projection's backward; same results, since
+        nothing later in the backward reads an updated backbone)."""
         self.n_layers, self.H, self.F, self.T, self.r, self.k, self.lr = n_layers, H, F, T, r, k, lr
         self.producer_amax = producer_amax
         self.device = torch.device(device)
@@ -143,6 +146,12 @@ class Stack:
         self.s_g = torch.empty(1, dtype=torch.float32, device=dev)
         self.dB = {p: torch.empty((self.shapes[p][1], r), dtype=torch.float32, device=dev) for p in PROJ}
         self.idx = torch.empty(max(k, 1), dtype=torch.int32, device=dev)
+        # one batched proxy update per block (its seven projections), or None: one call after every backward
+        self.batches = None
+        if batched_proxy:
+            self.batches = [fq.ProxyBatch([self.layers[l][p] for p in PROJ], [self.dB[p] for p in PROJ], [k] * len(PROJ),
+                                          wss=[self.ws[p] for p in PROJ], idx_outs=[None] * len(PROJ))
+                            for l in range(n_layers)]
         # absmax words of the chain's outputs, one row per block: x1, a, x2, z | ddn, dg, du, dhp, dqkv (cleared every step)
         self.amax = torch.zeros((n_layers, 16), dtype=torch.float32, device=dev)
         self.capture = None   # optional: {(block, proj): dict} filled with references / copies for parity checks
@@ -171,8 +180,9 @@ class Stack:
         fq.melded_backward(self.layers[l][name], dY, sv["oa"][name], sv["amax"][name], ws=self.ws[name],
                            out=(dX, self.dB[name], self.s_g), amax_dy=amax_dy)
         self._cap(l, name, dY=dY, dX=dX, dB=self.dB[name], OA=sv["oa"][name])
-        fq.proxy_update(self.layers[l][name], self.dB[name], self.lr, self.k, ws=self.ws[name],
-                        idx_out=self.idx if self.k > 0 else None)
+        if self.batches is None:
+            fq.proxy_update(self.layers[l][name], self.dB[name], self.lr, self.k, ws=self.ws[name],
+                            idx_out=self.idx if self.k > 0 else None)
 
     def _cap(self, l, name, **tensors):
         if self.capture is not None and (l, name) in self.capture:
@@ -204,7 +214,7 @@ class Stack:
 
     def backward(self, G: torch.Tensor):
         """G = d loss / d h_last.  Each block's backward is followed at once by the proxy updates of its layers
-        (inside _bwd), as in the paper's training loop."""
+        (one batched call, or inside _bwd), as in the paper's layer-wise training loop."""
         dh = G
         for l in reversed(range(self.n_layers)):
             sv = self.saved[l]
@@ -225,6 +235,8 @@ class Stack:
             rmsnorm_grad(self.dx[1], self.dx[0], sv["h"], sv["inv1"])
             combine(self.dh, self.dhp, 1.0, self.dx[1], 1.0)
             dh = self.dh
+            if self.batches is not None:
+                self.batches[l].run(self.lr)
         return dh
 
     def step(self, h0: torch.Tensor, G: torch.Tensor):
@@ -243,7 +255,10 @@ class Stack:
             shared = name in ("k", "v", "up")
             per_block += (1 if shared else fq.launch_count("falqon_melded_forward"))   # codes: the product alone
             per_block += fq.launch_count("falqon_melded_backward") + (1 if self.producer_amax else 0)   # + the O_A cast
-            per_block += fq.launch_count("falqon_proxy_update", k=self.k)
+            if self.batches is None:
+                per_block += fq.launch_count("falqon_proxy_update", k=self.k)
+        if self.batches is not None:
+            per_block += fq.launch_count("falqon_proxy_update_batched", k=self.k)
         per_block += 6 + 9   # chain kernels: forward 6 (2 norms, mix, 2 residuals, gate), backward 9
         return per_block * self.n_layers
 

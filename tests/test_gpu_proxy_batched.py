@@ -1,0 +1,110 @@
+"""GPU parity of falqon_proxy_update_batched (the proxy update of several layers in two launches) against the
+oracle's proxy update run layer by layer: indices, every byte of every backbone and every DeltaBuffer bit."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import bits32, f32, layer_inputs, u8
+from paper_2510_24061_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def fq():
+    from paper_2510_24061_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def orc():
+    from oracle import falqon_oracle
+    return falqon_oracle
+
+
+def _make(fq, seed, i, m, n, r, per_row):
+    W, A, _, _ = layer_inputs(seed, i, m, n, r, 16, 0)
+    if per_row:
+        W = synth.backbone(seed, i, m, n, heavy_tailed=True)
+    layer = fq.setup_layer(W.to(DEV), A.to(DEV), None, 1.0, per_row=per_row)
+    layer.dbuf.copy_(synth.normal_bf16(seed, 50 + 16 * i, (m, r), 0.05).float().to(DEV))
+    dB = (synth.normal_bf16(seed, 51 + 16 * i, (m, r), 1.0).float() * 0.337).to(DEV)
+    return layer, dB
+
+
+def _check_against_oracle(fq, orc, specs, lr, seed, steps=1):
+    """specs: (m, n, r, k, per_row, with_dB) per layer."""
+    made = [_make(fq, seed, i, m, n, r, per_row) for i, (m, n, r, k, per_row, _) in enumerate(specs)]
+    layers = [l for l, _ in made]
+    dBs = [dB if spec[5] else None for (_, dB), spec in zip(made, specs)]
+    ks = [spec[3] for spec in specs]
+    batch = fq.ProxyBatch(layers, dBs, ks)
+    for step in range(steps):
+        before = [(u8(l.wq).copy(), f32(l.dbuf).copy()) for l in layers]
+        idxs = batch.run(lr)
+        for i, (layer, spec) in enumerate(zip(layers, specs)):
+            m, n, r, k, per_row, with_dB = spec
+            wq_o, dbuf_o = before[i]
+            idx_o, _ = orc.proxy_update(wq_o, dbuf_o, f32(dBs[i]) if with_dB else None, lr, k, m, r,
+                                        row_scales=f32(layer.s_w) if per_row else None)
+            if k > 0:
+                assert np.array_equal(u8(idxs[i]), idx_o), f"layer {i} step {step}: indices"
+            assert np.array_equal(u8(layer.wq), wq_o), f"layer {i} step {step}: backbone"
+            assert np.array_equal(bits32(f32(layer.dbuf)), bits32(dbuf_o)), f"layer {i} step {step}: DeltaBuffer"
+    assert fq.last_device_status() == 0
+
+
+def test_mixed_layers_match_the_oracle(fq, orc):
+    """Different shapes, ranks and k in one call; a per-row layer; a layer without an optimizer step; k = 0 and k = m;
+    a ragged last column tile and a ragged last row group; two steps, so the control words must be back at zero."""
+    specs = [(256, 128, 16, 40, False, True), (272, 208, 8, 272, False, True), (144, 400, 24, 0, False, True),
+             (640, 1280, 64, 133, True, True), (512, 256, 32, 17, False, False), (1040, 528, 72, 1, False, True)]
+    _check_against_oracle(fq, orc, specs, 2e-2, 71, steps=2)
+
+
+def test_more_layers_than_one_launch_takes(fq, orc):
+    specs = [(128 + 16 * i, 128 + 32 * (i % 3), 8 * (1 + i % 4), 5 + 3 * i, i % 5 == 4, True) for i in range(11)]
+    _check_against_oracle(fq, orc, specs, 5e-2, 72)
+
+
+def test_all_layers_with_k_zero_and_an_empty_call(fq, orc):
+    specs = [(256, 128, 16, 0, False, True), (128, 256, 8, 0, False, True)]
+    _check_against_oracle(fq, orc, specs, 1e-2, 73)
+    assert fq.proxy_update_batched([], [], 0.1, []) == []
+
+
+def test_batched_equals_per_layer_calls_on_the_7b_projection_set(fq):
+    """The seven projections of configs[1] (r = 64, k = 256): one batched call against seven single calls, bit for bit."""
+    c = synth.config1()
+    shapes = [(m, n) for _, n, m in c["linears"]]
+    r, k, lr = c["r"], c["k"], c["lr"]
+    a, b = [], []
+    for i, (m, n) in enumerate(shapes):
+        layer, dB = _make(fq, 74, i, m, n, r, False)
+        a.append((layer, dB))
+        twin = fq.Layer(layer.wq.clone(), layer.s_w.clone(), layer.dbuf.clone(), r)
+        b.append((twin, dB))
+    idx_a = fq.proxy_update_batched([l for l, _ in a], [d for _, d in a], lr, [k] * len(a))
+    for i, (twin, dB) in enumerate(b):
+        idx_b = fq.proxy_update(twin, dB, lr, k)
+        assert torch.equal(idx_a[i], idx_b)
+        assert torch.equal(a[i][0].wq, twin.wq)
+        assert torch.equal(a[i][0].dbuf.view(torch.int32), twin.dbuf.view(torch.int32))
+    assert fq.last_device_status() == 0
+
+
+def test_invalid_entries_reject_the_whole_call(fq):
+    l0, dB0 = _make(fq, 75, 0, 128, 128, 8, False)
+    l1, dB1 = _make(fq, 75, 1, 128, 128, 8, False)
+    wq_before = l0.wq.clone()
+    with pytest.raises(fq.FalqonError) as e:
+        fq.proxy_update_batched([l0, l1], [dB0, dB1], 0.1, [4, 129])          # k > m in the second layer
+    assert e.value.status == fq.ERR_INVALID_ARG
+    with pytest.raises(fq.FalqonError):
+        fq.proxy_update_batched([l0, l0], [dB0, dB0], 0.1, [4, 4])            # the same layer twice
+    ws = l0.workspace(1)
+    with pytest.raises(fq.FalqonError):
+        fq.proxy_update_batched([l0, l1], [dB0, dB1], 0.1, [4, 4], wss=[ws, ws])   # a shared workspace
+    torch.cuda.synchronize()
+    assert torch.equal(l0.wq, wq_before)

@@ -140,7 +140,8 @@ def _check_projection(fq, orc, cap, layer, name, T, r, k, lr, n_rows):
 
 
 def _run_and_check(fq, st, orc, n_layers, H, F, T, r, k, check_blocks, n_rows, producer_amax=True):
-    stack = st.Stack(n_layers, H, F, T, r, k, seed=7, device=DEV, lr=2e-2, producer_amax=producer_amax)
+    stack = st.Stack(n_layers, H, F, T, r, k, seed=7, device=DEV, lr=2e-2, producer_amax=producer_amax,
+                     batched_proxy=producer_amax)   # the second variant also keeps the per-projection proxy updates
     h0 = synth.normal_bf16(7, 9001, (T, H), 1.0, DEV)
     G = synth.normal_bf16(7, 9002, (T, H), 1.0e-2, DEV)
     stack.capture = {(l, p): {} for l in check_blocks for p in st.PROJ}
