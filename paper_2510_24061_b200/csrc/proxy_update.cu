@@ -329,13 +329,20 @@ __global__ void __launch_bounds__(kTopkThreads) score_topk_batched_kernel(const 
 }
 
 // ---- W~[i][:] <- sat_rne_e4m3(W~[i][:] + DeltaBuffer[i][:] * A~) for the selected rows.
-// A CTA owns 32 selected rows x 128 columns.  It decodes the r x 128 tile of A~ to fp32 in shared
-// memory once (the FP8 decode is the expensive part, so it is shared by all 32 rows), then each thread
-// runs the fp32 fma chains of 4 rows x 8 columns (2 x 8 tiles with twice the threads measured slower).  The chain order (j ascending, seeded with the
-// decoded W~) is fixed, so the result is bit-identical to the sequential definition.
+// A CTA owns 128 columns and every n_splits-th group of 32 selected rows.  It decodes the r x 128 tile of A~ to fp32 in
+// shared memory once (the FP8 decode is the expensive part, so it is shared by all of the CTA's rows), then walks
+// its row groups: each thread runs the fp32 fma chains of 4 rows x 8 columns
+// (8 x 8 tiles and a hand-pipelined j loop were measured and were no faster).  The chain order (j ascending, seeded
+// with the decoded W~) is fixed, so the result is bit-identical to the sequential definition.  The groups are software
+// pipelined: while one is in the fma loop, the next one's DeltaBuffer rows arrive by asynchronous copy, its backbone codes
+// are in flight to registers, and the row indices of the one after it are being fetched, so that a CTA pays the
+// memory latency once, not once per group.  The inner loop needs as many shared-memory wavefronts as it can get: the
+// DeltaBuffer rows are read four j at a time, and their pitch of r + 4 floats keeps the two row blocks a warp
+// touches in different banks.
 constexpr int kMergeRowsPerThread = 4;
 constexpr int kMergeTy = 8;
-constexpr int kMergeRows = kMergeRowsPerThread * kMergeTy;          // 32 rows per CTA
+constexpr int kMergeRows = kMergeRowsPerThread * kMergeTy;          // 32 rows per group
+constexpr int kMergeRing = 4;                                       // row-index slots: groups t - 1 .. t + 2
 constexpr int kMergeTx = 16;
 constexpr int kMergeThreads = kMergeTx * kMergeTy;                  // 128
 constexpr int kMergeCols = 128;                                     // columns per CTA: thread tx owns 4tx..4tx+3 and 64+4tx..64+4tx+3
@@ -345,17 +352,24 @@ __device__ __forceinline__ void decode4(uint32_t w, float (&a)[4]) {
   a[0] = p0.x; a[1] = p0.y; a[2] = p1.x; a[3] = p1.y;
 }
 
-// col_tile / group: which 128 columns and which 32 selected rows this CTA owns; n_col_tiles: CTAs per row group.
+__host__ __device__ constexpr size_t merge_smem_bytes(int64_t r) {
+  return sizeof(float) * (static_cast<size_t>(r) * kMergeCols + 2 * static_cast<size_t>(kMergeRows) * (r + 4));
+}
+
+// col_tile: which 128 columns; split / n_splits: this CTA takes the row groups split, split + n_splits, ...;
+// n_col_tiles: how many CTAs work on one row group.
 __device__ __forceinline__ void merge_rows_body(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int k, int64_t m, int64_t n,
                                                 int r, unsigned int* group_counters, const float* row_scales, int col_tile,
-                                                int group, int n_col_tiles, float* merge_smem) {
+                                                int split, int n_splits, int n_col_tiles, float* merge_smem) {
+  constexpr int kRPT = kMergeRowsPerThread;
+  const int pitch = r + 4;
   float* a_tile = merge_smem;                         // [r][kMergeCols] decoded A~
-  float* sdb = merge_smem + (size_t)r * kMergeCols;   // [kMergeRows][r]
-  __shared__ int srow[kMergeRows];
-  const int g0 = group * kMergeRows;
-  const int nrows = min(kMergeRows, k - g0);
+  float* sdb = merge_smem + (size_t)r * kMergeCols;   // [2][kMergeRows][r + 4]
+  __shared__ int srow[kMergeRing][kMergeRows];        // row indices of the groups t - 1 (late clearing) .. t + 2
   const int64_t cta_c0 = (int64_t)col_tile * kMergeCols;
   const int cta_cols = static_cast<int>(min((int64_t)kMergeCols, n - cta_c0));   // multiple of 16
+  const int groups = (k + kMergeRows - 1) / kMergeRows;
+  const int items = split < groups ? (groups - split + n_splits - 1) / n_splits : 0;
   // The A~ rows are decoded BEFORE the wait, while the selection kernel is still running: nothing on the proxy
   // update's path writes them, and the kernel launched before this one (the selection) releases this launch
   // only after its own wait, i.e. after everything earlier on the stream (a set-up cast of A~, say) is done.
@@ -388,89 +402,146 @@ __device__ __forceinline__ void merge_rows_body(uint8_t* wq, float* dbuf, const 
     }
   }
   pdl_wait();
-  if (threadIdx.x < kMergeRows) srow[threadIdx.x] = (threadIdx.x < nrows) ? ld_stream(sel_idx + g0 + threadIdx.x) : -1;
-  __syncthreads();   // srow and the A~ tile visible
-  // the DeltaBuffer rows of this CTA, as float4 (r is a multiple of 8), four loads in flight per thread
+  if (items == 0) return;
+  const int tid = threadIdx.x;
+  const int tx = tid % kMergeTx, ty = tid / kMergeTx;
+  const int lc0 = 4 * tx, lc1 = 64 + 4 * tx;
+  const bool ok0 = lc0 < cta_cols, ok1 = lc1 < cta_cols;
+  const int q0 = ty * kRPT;
   const int r4 = r >> 2;
   const int d_vecs = kMergeRows * r4;
-  for (int e0 = threadIdx.x; e0 < d_vecs; e0 += 4 * kMergeThreads) {
-    float4 d[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int e = e0 + u * kMergeThreads;
+  // index of selected row q of this CTA's item t (or -1 past the end of the selection / of the items)
+  auto fetch_index = [&](int t) -> int {
+    const int64_t pos = (int64_t)(split + t * n_splits) * kMergeRows + tid;
+    return (t < items && tid < kMergeRows && pos < k) ? ld_stream(sel_idx + pos) : -1;
+  };
+  // DeltaBuffer rows of the group whose indices are in srow[slot] -> sdb[buf], as asynchronous 16-byte copies
+  auto fetch_rows = [&](int slot, int buf) {
+    float* dst = sdb + (size_t)buf * kMergeRows * pitch;
+    for (int e = tid; e < d_vecs; e += kMergeThreads) {
       const int q = e / r4, j4 = e - q * r4;
-      d[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (e < d_vecs && q < nrows) {
-        d[u] = *reinterpret_cast<const float4*>(dbuf + (int64_t)srow[q] * r + 4 * j4);
-        if (row_scales != nullptr) {   // per-row mode: c_i = s_w[i] / s_w[m], applied as its own rounded multiply
-          const float c = __fdiv_rn(ld_stream(row_scales + srow[q]), ld_stream(row_scales + m));
-          d[u].x = __fmul_rn(d[u].x, c); d[u].y = __fmul_rn(d[u].y, c);
-          d[u].z = __fmul_rn(d[u].z, c); d[u].w = __fmul_rn(d[u].w, c);
+      const int row = srow[slot][q];
+      if (row >= 0) cp_async16(smem_u32(dst + q * pitch + 4 * j4), dbuf + (int64_t)row * r + 4 * j4);
+    }
+    cp_async_commit();
+  };
+  auto fetch_codes = [&](int slot, uint32_t (&w0)[kRPT], uint32_t (&w1)[kRPT]) {
+#pragma unroll
+    for (int q = 0; q < kRPT; ++q) {
+      w0[q] = 0u; w1[q] = 0u;
+      const int row = srow[slot][q0 + q];
+      if (row >= 0) {
+        const uint8_t* p = wq + (int64_t)row * n + cta_c0;
+        if (ok0) w0[q] = *reinterpret_cast<const uint32_t*>(p + lc0);
+        if (ok1) w1[q] = *reinterpret_cast<const uint32_t*>(p + lc1);
+      }
+    }
+  };
+  if (tid < kMergeRows) {
+    srow[0][tid] = fetch_index(0);
+    srow[1][tid] = fetch_index(1);
+  }
+  __syncthreads();   // the indices and the A~ tile are visible
+  uint32_t w0[kRPT], w1[kRPT];
+  fetch_rows(0, 0);
+  fetch_codes(0, w0, w1);
+  unsigned int pending = 0u;     // warp 0: the counter value its lane 0 drew for the previous group
+  bool has_pending = false;
+  for (int t = 0; t < items; ++t) {
+    const int slot = t % kMergeRing, buf = t & 1;
+    const int idx_ahead = fetch_index(t + 2);
+    uint32_t nw0[kRPT], nw1[kRPT];
+    if (t + 1 < items) {
+      fetch_rows((t + 1) % kMergeRing, buf ^ 1);
+      fetch_codes((t + 1) % kMergeRing, nw0, nw1);
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
+    }
+    float* db = sdb + (size_t)buf * kMergeRows * pitch;
+    if (row_scales != nullptr) {   // per-row mode: c_i = s_w[i] / s_w[m], applied as its own rounded multiply to the
+      const float s_a = ld_stream(row_scales + m);                       // chunks this thread copied itself
+      for (int e = tid; e < d_vecs; e += kMergeThreads) {
+        const int q = e / r4, j4 = e - q * r4;
+        const int row = srow[slot][q];
+        if (row >= 0) {
+          const float c = __fdiv_rn(ld_stream(row_scales + row), s_a);
+          float4* p = reinterpret_cast<float4*>(db + q * pitch + 4 * j4);
+          float4 d = *p;
+          d.x = __fmul_rn(d.x, c); d.y = __fmul_rn(d.y, c); d.z = __fmul_rn(d.z, c); d.w = __fmul_rn(d.w, c);
+          *p = d;
+        }
+      }
+    }
+    __syncthreads();   // this group's DeltaBuffer rows have landed for every thread
+    // accumulators as packed pairs of neighbouring columns: the chains run on the two-wide fp32 fma, every half
+    // of which is an ordinary round-to-nearest fma
+    uint64_t v[kRPT][4];
+#pragma unroll
+    for (int q = 0; q < kRPT; ++q) {
+      float f[4];
+      decode4(w0[q], f); v[q][0] = pack_f32x2(f[0], f[1]); v[q][1] = pack_f32x2(f[2], f[3]);
+      decode4(w1[q], f); v[q][2] = pack_f32x2(f[0], f[1]); v[q][3] = pack_f32x2(f[2], f[3]);
+    }
+    const float* d0 = db + q0 * pitch;
+#pragma unroll 1
+    for (int j = 0; j < r; j += 4) {
+      float4 d4[kRPT];
+#pragma unroll
+      for (int q = 0; q < kRPT; ++q) d4[q] = *reinterpret_cast<const float4*>(d0 + q * pitch + j);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const ulonglong2 a0 = *reinterpret_cast<const ulonglong2*>(a_tile + (size_t)(j + u) * kMergeCols + lc0);
+        const ulonglong2 a1 = *reinterpret_cast<const ulonglong2*>(a_tile + (size_t)(j + u) * kMergeCols + lc1);
+#pragma unroll
+        for (int q = 0; q < kRPT; ++q) {
+          const float d = u == 0 ? d4[q].x : u == 1 ? d4[q].y : u == 2 ? d4[q].z : d4[q].w;
+          const uint64_t dd = pack_f32x2(d, d);
+          fma_f32x2(v[q][0], dd, a0.x); fma_f32x2(v[q][1], dd, a0.y);
+          fma_f32x2(v[q][2], dd, a1.x); fma_f32x2(v[q][3], dd, a1.y);
         }
       }
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int e = e0 + u * kMergeThreads;
-      if (e < d_vecs) reinterpret_cast<float4*>(sdb)[e] = d[u];
-    }
-  }
-  __syncthreads();
-  // With group counters (zero between calls) the CTA that is last to have copied a row group's DeltaBuffer rows
-  // clears those rows, which saves a separate kernel; every CTA of the group has its copy by then.
-  if (group_counters != nullptr) {
-    __shared__ int s_clear;
-    if (threadIdx.x == 0) {
-      const unsigned int prev = atomicAdd(&group_counters[group], 1u);
-      s_clear = (prev == static_cast<unsigned int>(n_col_tiles) - 1u) ? 1 : 0;
-      if (s_clear) group_counters[group] = 0u;
-    }
-    __syncthreads();
-    if (s_clear) {
-      for (int e = threadIdx.x; e < nrows * r4; e += kMergeThreads) {
-        const int q = e / r4, j4 = e - q * r4;
-        *reinterpret_cast<float4*>(dbuf + (int64_t)srow[q] * r + 4 * j4) = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int q = 0; q < kRPT; ++q) {
+      const int row = srow[slot][q0 + q];
+      if (row >= 0) {
+        uint8_t* p = wq + (int64_t)row * n + cta_c0;
+        float f[8];
+        unpack_f32x2(v[q][0], f[0], f[1]); unpack_f32x2(v[q][1], f[2], f[3]);
+        unpack_f32x2(v[q][2], f[4], f[5]); unpack_f32x2(v[q][3], f[6], f[7]);
+        if (ok0) *reinterpret_cast<uint32_t*>(p + lc0) = cvt_fp8x4<kE4M3>(f[0], f[1], f[2], f[3]);
+        if (ok1) *reinterpret_cast<uint32_t*>(p + lc1) = cvt_fp8x4<kE4M3>(f[4], f[5], f[6], f[7]);
       }
     }
-  }
-  const int tx = threadIdx.x % kMergeTx, ty = threadIdx.x / kMergeTx;
-  const int lc0 = 4 * tx, lc1 = 64 + 4 * tx;
-  const bool ok0 = lc0 < cta_cols, ok1 = lc1 < cta_cols;
-  const int q0 = ty * kMergeRowsPerThread;
-  float v[kMergeRowsPerThread][8];
-#pragma unroll
-  for (int q = 0; q < kMergeRowsPerThread; ++q) {
-    uint32_t w0 = 0u, w1 = 0u;
-    if (q0 + q < nrows) {
-      const uint8_t* row = wq + (int64_t)srow[q0 + q] * n + cta_c0;
-      if (ok0) w0 = *reinterpret_cast<const uint32_t*>(row + lc0);
-      if (ok1) w1 = *reinterpret_cast<const uint32_t*>(row + lc1);
+    // With group counters (zero between calls) the CTA that is last to be done with a row group clears the group's
+    // DeltaBuffer rows, which saves a separate kernel; every CTA of the group has its copy of them by then.  Warp 0
+    // does this alone, and looks at the counter value one group late, so that nobody waits for the atomic.
+    if (group_counters != nullptr && tid < 32) {
+      auto clear_if_last = [&](int item) {
+        unsigned int prev = __shfl_sync(0xFFFFFFFFu, pending, 0);
+        if (prev == static_cast<unsigned int>(n_col_tiles) - 1u) {
+          const int g = split + item * n_splits;
+          if (tid == 0) group_counters[g] = 0u;
+          const int s3 = item % kMergeRing;
+          for (int e = tid; e < d_vecs; e += 32) {
+            const int q = e / r4, j4 = e - q * r4;
+            const int row = srow[s3][q];
+            if (row >= 0) *reinterpret_cast<float4*>(dbuf + (int64_t)row * r + 4 * j4) = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        }
+      };
+      if (has_pending) clear_if_last(t - 1);
+      if (tid == 0) pending = atomicAdd(&group_counters[split + t * n_splits], 1u);
+      has_pending = true;
+      if (t + 1 == items) clear_if_last(t);
     }
-    float f[4];
-    decode4(w0, f); v[q][0] = f[0]; v[q][1] = f[1]; v[q][2] = f[2]; v[q][3] = f[3];
-    decode4(w1, f); v[q][4] = f[0]; v[q][5] = f[1]; v[q][6] = f[2]; v[q][7] = f[3];
-  }
-  const float* d0 = sdb + q0 * r;
-#pragma unroll 4
-  for (int j = 0; j < r; ++j) {
-    const float4 a0 = *reinterpret_cast<const float4*>(a_tile + (size_t)j * kMergeCols + lc0);
-    const float4 a1 = *reinterpret_cast<const float4*>(a_tile + (size_t)j * kMergeCols + lc1);
+    // The indices of group t + 2 go into the slot that group t - 2 had; the late clearing of that group ran before
+    // the previous iteration's closing barrier.
+    if (tid < kMergeRows) srow[(t + 2) % kMergeRing][tid] = idx_ahead;
 #pragma unroll
-    for (int q = 0; q < kMergeRowsPerThread; ++q) {
-      const float d = d0[q * r + j];
-      v[q][0] = __fmaf_rn(d, a0.x, v[q][0]); v[q][1] = __fmaf_rn(d, a0.y, v[q][1]);
-      v[q][2] = __fmaf_rn(d, a0.z, v[q][2]); v[q][3] = __fmaf_rn(d, a0.w, v[q][3]);
-      v[q][4] = __fmaf_rn(d, a1.x, v[q][4]); v[q][5] = __fmaf_rn(d, a1.y, v[q][5]);
-      v[q][6] = __fmaf_rn(d, a1.z, v[q][6]); v[q][7] = __fmaf_rn(d, a1.w, v[q][7]);
-    }
-  }
-#pragma unroll
-  for (int q = 0; q < kMergeRowsPerThread; ++q) {
-    if (q0 + q < nrows) {
-      uint8_t* row = wq + (int64_t)srow[q0 + q] * n + cta_c0;
-      if (ok0) *reinterpret_cast<uint32_t*>(row + lc0) = cvt_fp8x4<kE4M3>(v[q][0], v[q][1], v[q][2], v[q][3]);
-      if (ok1) *reinterpret_cast<uint32_t*>(row + lc1) = cvt_fp8x4<kE4M3>(v[q][4], v[q][5], v[q][6], v[q][7]);
-    }
+    for (int q = 0; q < kRPT; ++q) { w0[q] = nw0[q]; w1[q] = nw1[q]; }
+    __syncthreads();   // everyone is done with sdb[buf]; the new indices are visible
   }
 }
 
@@ -480,7 +551,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_kernel(uint8_t* wq, 
                                                                    const float* row_scales) {
   extern __shared__ __align__(16) float merge_smem_dyn[];
   pdl_trigger();
-  merge_rows_body(wq, dbuf, sel_idx, k, m, n, r, group_counters, row_scales, blockIdx.x, blockIdx.y, gridDim.x,
+  merge_rows_body(wq, dbuf, sel_idx, k, m, n, r, group_counters, row_scales, blockIdx.x, blockIdx.y, gridDim.y, gridDim.x,
                   merge_smem_dyn);
 }
 
@@ -492,7 +563,7 @@ struct BatchedMergeLayer {
   unsigned int* group_counters;
   const float* row_scales;
   int64_t m, n;
-  int r, k, cta_begin, col_tiles;
+  int r, k, cta_begin, col_tiles, splits;
 };
 struct BatchedMergeArgs {
   BatchedMergeLayer layer[kProxyBatchMax];
@@ -507,7 +578,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_rows_batched_kernel(const
   const BatchedMergeLayer& a = args.layer[l];
   const int local = static_cast<int>(blockIdx.x) - a.cta_begin;
   merge_rows_body(a.wq, a.dbuf, a.sel_idx, a.k, a.m, a.n, a.r, a.group_counters, a.row_scales, local % a.col_tiles,
-                  local / a.col_tiles, a.col_tiles, merge_smem_dyn);
+                  local / a.col_tiles, a.splits, a.col_tiles, merge_smem_dyn);
 }
 
 __global__ void __launch_bounds__(256) zero_rows_kernel(float* dbuf, const int32_t* sel_idx,
@@ -544,19 +615,34 @@ cudaError_t launch_topk(const float* score, int64_t m, int64_t k, int32_t* sel_i
 }
 
 namespace {
+constexpr int kMergeSmemMax = 200 * 1024;   // r = 256: 128 KB of A~ and two buffers of 33 KB
+constexpr int kMergeCtasPerSm = 4;
+
+// How many CTAs may share one column tile (each takes every splits-th row group) so that the whole launch is about one
+// wave of resident CTAs: the fewer CTAs, the more groups each one pipelines through.
+int merge_splits_budget(int64_t col_tiles_total, int64_t r_max) {
+  int64_t per_sm = (227 * 1024) / static_cast<int64_t>(merge_smem_bytes(r_max) + 1024);
+  if (per_sm > kMergeCtasPerSm) per_sm = kMergeCtasPerSm;
+  if (per_sm < 1) per_sm = 1;
+  const int64_t budget = per_sm * sm_count() / (col_tiles_total > 0 ? col_tiles_total : 1);
+  return static_cast<int>(budget < 1 ? 1 : budget);
+}
+
 cudaError_t launch_merge_only(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n, int64_t r,
                               unsigned int* group_counters, const float* row_scales, cudaStream_t stream) {
-  dim3 grid(static_cast<unsigned>((n + kMergeCols - 1) / kMergeCols),
-            static_cast<unsigned>((k + kMergeRows - 1) / kMergeRows));
-  const size_t smem = sizeof(float) * (static_cast<size_t>(r) * kMergeCols + static_cast<size_t>(kMergeRows) * r);
   static bool configured = false;
   if (!configured) {
-    cudaError_t ea = cudaFuncSetAttribute(merge_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 176 * 1024);
+    cudaError_t ea = cudaFuncSetAttribute(merge_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeSmemMax);
     if (ea != cudaSuccess) return ea;
     configured = true;
   }
-  return launch_pdl(merge_rows_kernel, grid, dim3(kMergeThreads), smem, stream, 1, wq, dbuf, sel_idx, static_cast<int>(k), m,
-                    n, static_cast<int>(r), group_counters, row_scales);
+  const int64_t col_tiles = (n + kMergeCols - 1) / kMergeCols, groups = (k + kMergeRows - 1) / kMergeRows;
+  int64_t splits = merge_splits_budget(col_tiles, r);
+  if (splits > groups) splits = groups;
+  if (splits > 65535) splits = 65535;
+  dim3 grid(static_cast<unsigned>(col_tiles), static_cast<unsigned>(splits));
+  return launch_pdl(merge_rows_kernel, grid, dim3(kMergeThreads), merge_smem_bytes(r), stream, 1, wq, dbuf, sel_idx,
+                    static_cast<int>(k), m, n, static_cast<int>(r), group_counters, row_scales);
 }
 }  // namespace
 
@@ -631,23 +717,55 @@ cudaError_t launch_adamw_score_topk(float* dbuf, const float* dB, float* exp_avg
   return launch_opt_score_topk(dbuf, dB, opt, m, r, k, score, sel_idx, idx_copy, done_counter, stream);
 }
 
+namespace {
+cudaError_t launch_merge_batched(const ProxyBatchLayer* layers, int count, cudaStream_t stream) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t ea = cudaFuncSetAttribute(merge_rows_batched_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeSmemMax);
+    if (ea != cudaSuccess) return ea;
+    configured = true;
+  }
+  int64_t col_tiles_total = 0, r_max = 8;
+  for (int i = 0; i < count; ++i) {
+    if (layers[i].k <= 0) continue;
+    col_tiles_total += (layers[i].n + kMergeCols - 1) / kMergeCols;
+    if (layers[i].r > r_max) r_max = layers[i].r;
+  }
+  const int budget = merge_splits_budget(col_tiles_total, r_max);
+  BatchedMergeArgs ma{};
+  int ctas = 0;
+  for (int i = 0; i < count; ++i) {
+    const ProxyBatchLayer& L = layers[i];
+    if (L.k <= 0) continue;
+    BatchedMergeLayer& b = ma.layer[ma.count++];
+    b.wq = L.wq; b.dbuf = L.dbuf; b.sel_idx = L.sel_idx; b.group_counters = L.group_counters; b.row_scales = L.row_scales;
+    b.m = L.m; b.n = L.n; b.r = static_cast<int>(L.r); b.k = static_cast<int>(L.k);
+    b.cta_begin = ctas;
+    b.col_tiles = static_cast<int>((L.n + kMergeCols - 1) / kMergeCols);
+    const int groups = static_cast<int>((L.k + kMergeRows - 1) / kMergeRows);
+    b.splits = budget < groups ? budget : groups;
+    ctas += b.col_tiles * b.splits;
+  }
+  if (ma.count == 0) return cudaSuccess;
+  return launch_pdl(merge_rows_batched_kernel, dim3(ctas), dim3(kMergeThreads), merge_smem_bytes(r_max), stream, 1, ma);
+}
+}  // namespace
+
 cudaError_t launch_proxy_update_batched(const ProxyBatchLayer* layers, int count, float lr, int phase, cudaStream_t stream) {
   if (count < 1 || count > kProxyBatchMax) return cudaErrorInvalidValue;
+  if (phase != 0) return launch_merge_batched(layers, count, stream);
   static bool configured = false;
   if (!configured) {
     cudaError_t ea = cudaFuncSetAttribute(score_topk_batched_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(kTopkSmemRows * sizeof(uint32_t)));
     if (ea != cudaSuccess) return ea;
-    ea = cudaFuncSetAttribute(merge_rows_batched_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 176 * 1024);
-    if (ea != cudaSuccess) return ea;
     configured = true;
   }
   BatchedScoreArgs sa{};
-  BatchedMergeArgs ma{};
   sa.count = count;
   sa.neg_lr = -lr;
-  int score_ctas = 0, merge_ctas = 0;
-  size_t score_smem = 0, merge_smem = 0;
+  int score_ctas = 0;
+  size_t score_smem = 0;
   for (int i = 0; i < count; ++i) {
     const ProxyBatchLayer& L = layers[i];
     BatchedScoreLayer& a = sa.layer[i];
@@ -659,20 +777,8 @@ cudaError_t launch_proxy_update_batched(const ProxyBatchLayer* layers, int count
     size_t smem = sizeof(float) * kFusedScoreRows * (L.r + 1);
     if (L.m <= kTopkSmemRows && static_cast<size_t>(L.m) * sizeof(uint32_t) > smem) smem = static_cast<size_t>(L.m) * sizeof(uint32_t);
     if (smem > score_smem) score_smem = smem;
-    if (L.k > 0) {
-      BatchedMergeLayer& b = ma.layer[ma.count++];
-      b.wq = L.wq; b.dbuf = L.dbuf; b.sel_idx = L.sel_idx; b.group_counters = L.group_counters; b.row_scales = L.row_scales;
-      b.m = L.m; b.n = L.n; b.r = static_cast<int>(L.r); b.k = static_cast<int>(L.k);
-      b.cta_begin = merge_ctas;
-      b.col_tiles = static_cast<int>((L.n + kMergeCols - 1) / kMergeCols);
-      merge_ctas += b.col_tiles * merge_group_count(L.k);
-      const size_t ms = sizeof(float) * (static_cast<size_t>(L.r) * kMergeCols + static_cast<size_t>(kMergeRows) * L.r);
-      if (ms > merge_smem) merge_smem = ms;
-    }
   }
-  if (phase == 0) return launch_pdl(score_topk_batched_kernel, dim3(score_ctas), dim3(kTopkThreads), score_smem, stream, 1, sa);
-  if (ma.count == 0) return cudaSuccess;
-  return launch_pdl(merge_rows_batched_kernel, dim3(merge_ctas), dim3(kMergeThreads), merge_smem, stream, 1, ma);
+  return launch_pdl(score_topk_batched_kernel, dim3(score_ctas), dim3(kTopkThreads), score_smem, stream, 1, sa);
 }
 
 }  // namespace falqon
