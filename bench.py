@@ -293,6 +293,57 @@ def run_sweep(args):
                               "hbm_peak_gbs": peaks["hbm"]}), flush=True)
 
 
+def measure_tensor_ceiling(fq, seconds, fills, gpu_index=0):
+    """Back-to-back launches of the MMA-issue-only kernel (the product kernels' 256 x 256 x 32 E4M3 instruction on
+    operands resident in shared memory) for `seconds` per operand fill.  Per fill: the rate over the first ten launches
+    (burst), over the last second (sustained, under the power cap) and over the whole run, with the clocks seen."""
+    import time
+    dev = torch.device("cuda", torch.cuda.current_device())
+    sink = torch.zeros(4 * fq.tensor_ceiling_ctas(), dtype=torch.float32, device=dev)
+    kblocks = 20000            # about 10 ms per launch
+    out = {"kblocks_per_launch": kblocks, "seconds_per_fill": seconds, "ctas": fq.tensor_ceiling_ctas()}
+    codes = {"zeros": 0, "uniform_codes": 1, "bell_shaped_codes": 2}
+    for name in fills:
+        for _ in range(3):
+            flops = fq.tensor_ceiling(kblocks, 1, codes[name], sink)
+        torch.cuda.synchronize()
+        time.sleep(1.0)        # let the power average settle before the burst figure
+        sampler = ClockSampler(gpu_index)
+        sampler.start()
+        events = [torch.cuda.Event(enable_timing=True)]
+        events[0].record()
+        t0 = time.time()
+        while time.time() - t0 < seconds:
+            for _ in range(10):
+                fq.tensor_ceiling(kblocks, 1, codes[name], sink)
+            ev = torch.cuda.Event(enable_timing=True)
+            ev.record()
+            events.append(ev)
+            ev.synchronize()
+        clocks = sampler.stop()
+        ms = [events[i].elapsed_time(events[i + 1]) for i in range(len(events) - 1)]     # each: 10 launches
+        rate = lambda chunk: 10.0 * len(chunk) * flops / (sum(chunk) * 1e-3) / 1e12
+        n_last = max(1, int(len(ms) * min(1.0, 1.0 / seconds)))
+        out[name] = {"burst": rate(ms[:1]), "sustained": rate(ms[-n_last:]), "whole_run": rate(ms), "launches": 10 * len(ms),
+                     "clocks": clocks}
+    return out
+
+
+def run_tensor_ceiling(args):
+    """The FP8 tensor pipe with nothing else in the way, for zero operands, uniformly random codes and the codes of a
+    bell-shaped variable under absmax scaling.  One JSON line."""
+    from paper_2510_24061_b200 import binding as fq
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    out = {"metric": "FP8 tensor ceiling (tcgen05.mma kind::f8f6f4, 256x256x32 over CTA pairs, operands in shared memory)",
+           "unit": "TFLOP/s",
+           "bf16_x2_reference": {"burst": peaks["bf16_burst"] * FP8_OVER_BF16, "sustained": peaks["bf16_sustained"] * FP8_OVER_BF16,
+                                 "source": peaks["source"]}, "nominal": 4500.0}
+    out.update(measure_tensor_ceiling(fq, args.tensor_ceiling, ["zeros", "uniform_codes", "bell_shaped_codes"]))
+    out["device_status"] = fq.last_device_status()
+    print(json.dumps(out), flush=True)
+
+
 def run_stack(args):
     """configs[2]: 32 decoder-shaped blocks of the 7B projection set, activations chained (see
     paper_2510_24061_b200/stack.py), one training step = forward through all blocks, backward, and each block's
@@ -375,6 +426,10 @@ def main():
     ap.add_argument("--config3", action="store_true",
                     help="configs[3] instead of configs[1]: the LLaMA-13B projection set, 8192 tokens, per-row-scaled "
                          "heavy-tailed backbone, top-512 (not the headline line)")
+    ap.add_argument("--tensor-ceiling", type=float, default=0.0, metavar="SECONDS",
+                    help="measure the FP8 tensor pipe alone (MMA issue on shared-memory operands) for SECONDS per fill; one JSON line")
+    ap.add_argument("--no-tensor-ceiling", action="store_true",
+                    help="skip the 3 s measurement of the FP8 tensor pipe alone that the default line reports beside the roofline")
     ap.add_argument("--proxy-per-layer", action="store_true",
                     help="run one falqon_proxy_update per projection instead of one falqon_proxy_update_batched per step")
     ap.add_argument("--only", default=None, help="profiling aid: restrict the workload to one projection (q,k,v,o,gate,up,down)")
@@ -399,6 +454,10 @@ def main():
                 "parallelism": f"replicas x{world}",
                 "proxy_update": "one call per projection" if args.proxy_per_layer else "one batched call per step"}
 
+    if args.tensor_ceiling > 0:
+        if rank == 0:
+            run_tensor_ceiling(args)
+        return
     if args.sweep:
         if rank == 0:
             run_sweep(args)
@@ -552,6 +611,16 @@ def main():
         tf, secs, threads, desc = time_oracle_sample(args.oracle_tokens, r, k, lr)
         cpu_baseline = {"value": tf, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
                         "seconds": secs, "host_cpus": os.cpu_count()}
+
+    # ---- the FP8 tensor pipe alone (rank 0 at N = 1 only; at N > 1 the other ranks would be idle and the board power differs)
+    if not args.no_tensor_ceiling and world == 1:
+        tc = measure_tensor_ceiling(fq, 3.0, ["bell_shaped_codes"], local_rank)
+        ceiling = tc["bell_shaped_codes"]["sustained"]
+        roofline["mma_only_ceiling"] = {
+            "sustained": ceiling, "burst": tc["bell_shaped_codes"]["burst"], "unit": "TFLOP/s",
+            "clocks": tc["bell_shaped_codes"]["clocks"], "frac": achieved / ceiling if ceiling > 0 else None,
+            "note": "this GPU's tensor pipe issuing the products' own MMA on shared-memory operands (bell-shaped E4M3 codes) "
+                    "for 3 s under the power cap: no loads, no epilogue; python bench.py --tensor-ceiling 3 gives all fills"}
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),

@@ -272,6 +272,18 @@ int falqon_proxy_update_exact(const falqon_layer *L, const float *dB, float lr, 
  * undefined) or FALQON_ERR_CUDA (the synchronize itself failed). */
 int falqon_last_device_status(falqon_stream stream);
 
+/* Measurement aid (no counterpart in the paper): the ceiling of this GPU's FP8 tensor pipe.  One launch in which every
+ * SM pair issues kblocks x 4 of the 256 x 256 x 32 E4M3 MMAs that the forward and input-gradient products issue, on
+ * operand tiles that stay in shared memory (random_fill 0: zeros; 1: uniformly random codes drawn from `seed`; 2: the
+ * codes of a bell-shaped variable under absmax scaling, as quantized activations are; the data decide the power drawn
+ * and with it the clock).  Asynchronous on `stream`; the caller times a sequence of
+ * launches with events.  *flops_out (host, nullable) receives the floating-point operations of one launch.
+ * sink: device [4 * falqon_tensor_ceiling_ctas()] fp32 or NULL; receives partial sums of the accumulators (all zero
+ * for zero operands).  1 <= kblocks <= 2^20.  A wait that runs out sets the device status word. */
+int falqon_tensor_ceiling_ctas(void);
+int falqon_tensor_ceiling(int64_t kblocks, uint32_t seed, int32_t random_fill, float *sink, double *flops_out,
+                          falqon_stream stream);
+
 /* Stages that the optional timing hook can bracket with CUDA events (bit i of the mask = stage i). */
 typedef enum {
   FALQON_STAGE_QUANT_X = 0,   /* absmax + cast of X            (S1) */

@@ -22,7 +22,7 @@ WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 
 EXPORTS = ["falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
-           "falqon_svd_init_scratch_bytes", "falqon_svd_init",
+           "falqon_svd_init_scratch_bytes", "falqon_svd_init", "falqon_tensor_ceiling", "falqon_tensor_ceiling_ctas",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_proxy_update_batched", "falqon_last_device_status", "falqon_launch_count",
            "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static", "falqon_workspace_init", "falqon_proxy_update_adamw"]
 STATIC_MAX_ROWS = 16384
@@ -64,6 +64,10 @@ lib.falqon_proxy_update.argtypes = [C.POINTER(falqon_layer), _p, _f, _i64, _p, _
 lib.falqon_proxy_update_batched.restype = _i
 lib.falqon_proxy_update_batched.argtypes = [C.POINTER(falqon_layer), C.c_int32, C.POINTER(_p), _f, C.POINTER(_i64), C.POINTER(_p),
                                             C.POINTER(_p), C.POINTER(_sz), _p]
+lib.falqon_tensor_ceiling.restype = _i
+lib.falqon_tensor_ceiling.argtypes = [_i64, C.c_uint32, C.c_int32, _p, C.POINTER(C.c_double), _p]
+lib.falqon_tensor_ceiling_ctas.restype = _i
+lib.falqon_tensor_ceiling_ctas.argtypes = []
 class falqon_adamw(C.Structure):
     _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
                 ("weight_decay", C.c_float), ("step", C.c_int64)]
@@ -287,6 +291,19 @@ def proxy_update(layer: Layer, dB: torch.Tensor | None, lr: float, k: int, ws: t
     _check("falqon_proxy_update", lib.falqon_proxy_update(C.byref(layer.c), _ptr(dB), lr, k, _ptr(idx_out), _ptr(ws),
                                                           ws.numel(), _stream()))
     return idx_out
+
+
+def tensor_ceiling(kblocks: int, seed: int = 1, random_fill: int = 1, sink: torch.Tensor | None = None) -> float:
+    """falqon_tensor_ceiling: one launch of the MMA-issue-only measurement kernel on the current stream.  Returns the
+    floating-point operations of the launch (time a sequence of launches with events to get a rate)."""
+    flops = C.c_double()
+    _check("falqon_tensor_ceiling", lib.falqon_tensor_ceiling(kblocks, seed, int(random_fill), _ptr(sink), C.byref(flops),
+                                                             _stream()))
+    return flops.value
+
+
+def tensor_ceiling_ctas() -> int:
+    return int(lib.falqon_tensor_ceiling_ctas())
 
 
 class ProxyBatch:

@@ -172,4 +172,10 @@ struct ProxyBatchLayer {
 // phase 0: optimizer step, scores and selection of every layer; phase 1: the merge of every layer with k > 0.
 cudaError_t launch_proxy_update_batched(const ProxyBatchLayer* layers, int count, float lr, int phase, cudaStream_t stream);
 
+// Measurement aid: every SM pair issues kblocks x 4 FP8 MMAs (256 x 256 x 32, the product kernels' instruction) on
+// operands resident in shared memory.  sink: device [4 * tensor_ceiling_ctas()] floats or null.
+int tensor_ceiling_ctas();
+double tensor_ceiling_flops(int kblocks);
+cudaError_t launch_tensor_ceiling(int kblocks, uint32_t seed, int random_fill, float* sink, int* status, cudaStream_t stream);
+
 }  // namespace falqon
