@@ -242,11 +242,10 @@ cudaError_t launch_db_fused(const DbFusedProblem& q, cudaStream_t stream) {
   if (!make_tensor_map(&tg, q.gq, q.T, q.m, q.m, kDbBlock, kDbBlock)) return cudaErrorInvalidValue;
   if (!make_tensor_map(&toa, q.oaq_t, p.r16, q.T, q.ldt, kDbBlock, static_cast<uint32_t>(p.r16))) return cudaErrorInvalidValue;
   const size_t smem = static_cast<size_t>(kDbStages) * (kDbATileBytes + static_cast<size_t>(p.r16) * kDbBlock) + 128 + 1024;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(db_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e != cudaSuccess) return e;
-    configured = true;
+  static DeviceMask configured{0};
+  {
+    const cudaError_t ec = set_max_dynamic_smem(db_fused_kernel, 227 * 1024, configured);
+    if (ec != cudaSuccess) return ec;
   }
   const unsigned grid = static_cast<unsigned>(p.m_tiles) * static_cast<unsigned>(splits);
   return launch_pdl(db_fused_kernel, dim3(grid), dim3(kDbThreads), smem, stream, splits, tg, toa, p);

@@ -602,14 +602,15 @@ bool make_tensor_map(CUtensorMap* map, const uint8_t* base, int64_t rows, int64_
   return r == CUDA_SUCCESS;
 }
 
-int sm_count() {
-  static int count = [] {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
-    return n;
-  }();
-  return count;
+int sm_count() {   // of the current device
+  static std::atomic<int> counts[64];
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  const bool tracked = dev >= 0 && dev < 64;
+  if (tracked && (n = counts[dev].load()) > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+  if (tracked) counts[dev].store(n);
+  return n;
 }
 
 namespace {
@@ -617,12 +618,10 @@ namespace {
 template <bool kBMn>
 cudaError_t launch_variant(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& gp, int grid, size_t smem,
                            cudaStream_t stream) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_fp8_kernel<kBMn>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(kSmemBudget));
-    if (e != cudaSuccess) return e;
-    configured = true;
+  static DeviceMask configured{0};
+  {
+    const cudaError_t ec = set_max_dynamic_smem(gemm_fp8_kernel<kBMn>, static_cast<int>(kSmemBudget), configured);
+    if (ec != cudaSuccess) return ec;
   }
   return launch_pdl(gemm_fp8_kernel<kBMn>, dim3(static_cast<unsigned>(grid)), dim3(kGemmThreads), smem, stream, 1, ta,
                     tb, gp);
@@ -631,12 +630,10 @@ cudaError_t launch_variant(const CUtensorMap& ta, const CUtensorMap& tb, const G
 template <bool kBMn>
 cudaError_t launch_pair_variant(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& gp, int grid, size_t smem,
                                 cudaStream_t stream) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_fp8_pair_kernel<kBMn>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(kSmemBudget));
-    if (e != cudaSuccess) return e;
-    configured = true;
+  static DeviceMask configured{0};
+  {
+    const cudaError_t ec = set_max_dynamic_smem(gemm_fp8_pair_kernel<kBMn>, static_cast<int>(kSmemBudget), configured);
+    if (ec != cudaSuccess) return ec;
   }
   return launch_pdl(gemm_fp8_pair_kernel<kBMn>, dim3(static_cast<unsigned>(grid)), dim3(kGemmThreads), smem, stream, 2, ta, tb,
                     gp);

@@ -1,6 +1,7 @@
 // Host-side declarations shared by the translation units of libfalqon (not part of the public ABI).
 #pragma once
 
+#include <atomic>
 #include <cstddef>
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -13,6 +14,20 @@ constexpr int kE4M3 = 0, kE5M2 = 1;
 constexpr int kBF16 = 0, kF32 = 1;
 
 inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+
+// The largest dynamic shared-memory size of a kernel is a property of the (kernel, device) pair: set it the first time a
+// launch site is used on a device.  `done` is the launch site's own word, one bit per device.
+using DeviceMask = std::atomic<unsigned long long>;
+template <typename K>
+cudaError_t set_max_dynamic_smem(K kernel, int bytes, DeviceMask& done) {
+  int dev = 0;
+  const bool tracked = cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64;
+  const unsigned long long bit = tracked ? 1ull << dev : 0ull;
+  if (tracked && (done.load(std::memory_order_acquire) & bit) != 0) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && tracked) done.fetch_or(bit, std::memory_order_release);
+  return e;
+}
 
 // Launches `kernel` so that it may be scheduled before the previous kernel in the stream has drained
 // (programmatic stream serialization).  The kernel itself must call pdl_wait() before it reads or writes

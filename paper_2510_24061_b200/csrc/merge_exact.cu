@@ -515,11 +515,10 @@ cudaError_t launch_merge_exact(uint8_t* wq, float* dbuf, const int32_t* sel_idx,
                        static_cast<uint32_t>(block_n)))
     return cudaErrorInvalidValue;
   const size_t smem = static_cast<size_t>(kXStages) * (kXATile + static_cast<size_t>(block_n) * kXBlockKBytes) + 256 + 1024;
-  static bool configured = false;
-  if (!configured) {
-    e = cudaFuncSetAttribute(merge_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e != cudaSuccess) return e;
-    configured = true;
+  static DeviceMask configured{0};
+  {
+    const cudaError_t ec = set_max_dynamic_smem(merge_exact_kernel, 227 * 1024, configured);
+    if (ec != cudaSuccess) return ec;
   }
   int grid = 2 * sm_count();
   const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;

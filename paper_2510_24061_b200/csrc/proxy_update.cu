@@ -603,12 +603,10 @@ cudaError_t launch_sgd_score(float* dbuf, const float* dB, float lr, int64_t m, 
 cudaError_t launch_topk(const float* score, int64_t m, int64_t k, int32_t* sel_idx, void* idx_copy, cudaStream_t stream) {
   const int use_smem = m <= kTopkSmemRows ? 1 : 0;
   const size_t smem = use_smem ? static_cast<size_t>(m) * sizeof(uint32_t) : 0;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t ea = cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          static_cast<int>(kTopkSmemRows * sizeof(uint32_t)));
-    if (ea != cudaSuccess) return ea;
-    configured = true;
+  static DeviceMask configured{0};
+  {
+    const cudaError_t ec = set_max_dynamic_smem(topk_kernel, static_cast<int>(kTopkSmemRows * sizeof(uint32_t)), configured);
+    if (ec != cudaSuccess) return ec;
   }
   return launch_pdl(topk_kernel, dim3(1), dim3(kTopkThreads), smem, stream, 1, score, static_cast<int>(m),
                     static_cast<int>(k), sel_idx, static_cast<int32_t*>(idx_copy), use_smem);
@@ -630,11 +628,10 @@ int merge_splits_budget(int64_t col_tiles_total, int64_t r_max) {
 
 cudaError_t launch_merge_only(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n, int64_t r,
                               unsigned int* group_counters, const float* row_scales, cudaStream_t stream) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t ea = cudaFuncSetAttribute(merge_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeSmemMax);
-    if (ea != cudaSuccess) return ea;
-    configured = true;
+  static DeviceMask configured{0};
+  {
+    const cudaError_t ec = set_max_dynamic_smem(merge_rows_kernel, kMergeSmemMax, configured);
+    if (ec != cudaSuccess) return ec;
   }
   const int64_t col_tiles = (n + kMergeCols - 1) / kMergeCols, groups = (k + kMergeRows - 1) / kMergeRows;
   int64_t splits = merge_splits_budget(col_tiles, r);
@@ -677,12 +674,10 @@ cudaError_t launch_opt_score_topk(float* dbuf, const float* dB, const OptimizerA
   const int use_smem = m <= kTopkSmemRows ? 1 : 0;
   size_t smem = sizeof(float) * kFusedScoreRows * (r + 1);
   if (use_smem && static_cast<size_t>(m) * sizeof(uint32_t) > smem) smem = static_cast<size_t>(m) * sizeof(uint32_t);
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t ea = cudaFuncSetAttribute(sgd_score_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          static_cast<int>(kTopkSmemRows * sizeof(uint32_t)));
-    if (ea != cudaSuccess) return ea;
-    configured = true;
+  static DeviceMask configured{0};
+  {
+    const cudaError_t ec = set_max_dynamic_smem(sgd_score_topk_kernel, static_cast<int>(kTopkSmemRows * sizeof(uint32_t)), configured);
+    if (ec != cudaSuccess) return ec;
   }
   const int grid = static_cast<int>((m + kFusedScoreRows - 1) / kFusedScoreRows);
   return launch_pdl(sgd_score_topk_kernel, dim3(grid), dim3(kTopkThreads), smem, stream, 1, dbuf, dB, opt,
@@ -719,11 +714,10 @@ cudaError_t launch_adamw_score_topk(float* dbuf, const float* dB, float* exp_avg
 
 namespace {
 cudaError_t launch_merge_batched(const ProxyBatchLayer* layers, int count, cudaStream_t stream) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t ea = cudaFuncSetAttribute(merge_rows_batched_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeSmemMax);
-    if (ea != cudaSuccess) return ea;
-    configured = true;
+  static DeviceMask configured{0};
+  {
+    const cudaError_t ec = set_max_dynamic_smem(merge_rows_batched_kernel, kMergeSmemMax, configured);
+    if (ec != cudaSuccess) return ec;
   }
   int64_t col_tiles_total = 0, r_max = 8;
   for (int i = 0; i < count; ++i) {
@@ -754,12 +748,10 @@ cudaError_t launch_merge_batched(const ProxyBatchLayer* layers, int count, cudaS
 cudaError_t launch_proxy_update_batched(const ProxyBatchLayer* layers, int count, float lr, int phase, cudaStream_t stream) {
   if (count < 1 || count > kProxyBatchMax) return cudaErrorInvalidValue;
   if (phase != 0) return launch_merge_batched(layers, count, stream);
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t ea = cudaFuncSetAttribute(score_topk_batched_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          static_cast<int>(kTopkSmemRows * sizeof(uint32_t)));
-    if (ea != cudaSuccess) return ea;
-    configured = true;
+  static DeviceMask configured{0};
+  {
+    const cudaError_t ec = set_max_dynamic_smem(score_topk_batched_kernel, static_cast<int>(kTopkSmemRows * sizeof(uint32_t)), configured);
+    if (ec != cudaSuccess) return ec;
   }
   BatchedScoreArgs sa{};
   sa.count = count;

@@ -540,16 +540,19 @@ cudaError_t launch_staged_variant(const void* src, int64_t count, uint8_t* dst, 
                                   const CastOutputs& out, int* status, const float* col_mul, int cols, const OaCastJob& oa_job,
                                   cudaStream_t stream) {
   constexpr size_t kSmem = static_cast<size_t>(kStagedSlots) * kChunkBytes;
-  static int blocks_per_sm = 0;
-  if (blocks_per_sm == 0) {
-    cudaError_t e = cudaFuncSetAttribute(quantize_staged_kernel<kDt, kFmt, kColMul>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmem));
-    if (e != cudaSuccess) return e;
+  static DeviceMask configured{0};
+  {
+    const cudaError_t ec = set_max_dynamic_smem(quantize_staged_kernel<kDt, kFmt, kColMul>, static_cast<int>(kSmem), configured);
+    if (ec != cudaSuccess) return ec;
+  }
+  static std::atomic<int> blocks_per_sm{0};   // the kernel's grid barrier needs every CTA resident: checked once
+  if (blocks_per_sm.load() == 0) {
     int b = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, quantize_staged_kernel<kDt, kFmt, kColMul>, kStagedThreads, kSmem);
+    const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, quantize_staged_kernel<kDt, kFmt, kColMul>,
+                                                                        kStagedThreads, kSmem);
     if (e != cudaSuccess) return e;
     if (b < 1) return cudaErrorLaunchOutOfResources;
-    blocks_per_sm = b;
+    blocks_per_sm.store(b);
   }
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);

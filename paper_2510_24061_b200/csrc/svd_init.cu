@@ -245,12 +245,11 @@ cudaError_t launch_svd_init(const void* w, int w_dt, int64_t m, int64_t n, const
   float* lam = reinterpret_cast<float*>(base);
   const int L = static_cast<int>(l), M = static_cast<int>(m), N = static_cast<int>(n);
   const size_t small_smem = static_cast<size_t>(2) * l * l * sizeof(float);
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(svd_chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(svd_jacobi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024);
-    if (e != cudaSuccess) return e;
-    configured = true;
+  static DeviceMask configured_chol{0}, configured_jacobi{0};
+  {
+    cudaError_t ec = set_max_dynamic_smem(svd_chol_inv_kernel, 210 * 1024, configured_chol);
+    if (ec == cudaSuccess) ec = set_max_dynamic_smem(svd_jacobi_kernel, 210 * 1024, configured_jacobi);
+    if (ec != cudaSuccess) return ec;
   }
 #define SVD_TRY(expr) do { cudaError_t e__ = (expr); if (e__ != cudaSuccess) return e__; } while (0)
   int64_t blocks = (m * n / 4 + 255) / 256;

@@ -140,12 +140,10 @@ double tensor_ceiling_flops(int kblocks) {   // of one launch: every pair issues
 }
 
 cudaError_t launch_tensor_ceiling(int kblocks, uint32_t seed, int random_fill, float* sink, int* status, cudaStream_t stream) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(tensor_ceiling_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(kCeilSmem));
-    if (e != cudaSuccess) return e;
-    configured = true;
+  static DeviceMask configured{0};
+  {
+    const cudaError_t ec = set_max_dynamic_smem(tensor_ceiling_kernel, static_cast<int>(kCeilSmem), configured);
+    if (ec != cudaSuccess) return ec;
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(static_cast<unsigned>(tensor_ceiling_ctas()));
