@@ -303,9 +303,16 @@ def measure_tensor_ceiling(fq, seconds, fills, gpu_index=0):
     kblocks = 20000            # about 10 ms per launch
     out = {"kblocks_per_launch": kblocks, "seconds_per_fill": seconds, "ctas": fq.tensor_ceiling_ctas()}
     codes = {"zeros": 0, "uniform_codes": 1, "bell_shaped_codes": 2}
+    traffic = None
     for name in fills:
+        load_src = None
+        if name.endswith("+operand_traffic"):     # 64 MB of codes (stays in L2), streamed into the operand slots
+            if traffic is None:
+                traffic = torch.randint(0, 120, (64 << 20,), dtype=torch.uint8, device=dev)
+            load_src = traffic
+        fill = codes[name.split("+")[0]]
         for _ in range(3):
-            flops = fq.tensor_ceiling(kblocks, 1, codes[name], sink)
+            flops = fq.tensor_ceiling(kblocks, 1, fill, sink, load_src)
         torch.cuda.synchronize()
         time.sleep(1.0)        # let the power average settle before the burst figure
         sampler = ClockSampler(gpu_index)
@@ -315,7 +322,7 @@ def measure_tensor_ceiling(fq, seconds, fills, gpu_index=0):
         t0 = time.time()
         while time.time() - t0 < seconds:
             for _ in range(10):
-                fq.tensor_ceiling(kblocks, 1, codes[name], sink)
+                fq.tensor_ceiling(kblocks, 1, fill, sink, load_src)
             ev = torch.cuda.Event(enable_timing=True)
             ev.record()
             events.append(ev)
@@ -339,7 +346,8 @@ def run_tensor_ceiling(args):
            "unit": "TFLOP/s",
            "bf16_x2_reference": {"burst": peaks["bf16_burst"] * FP8_OVER_BF16, "sustained": peaks["bf16_sustained"] * FP8_OVER_BF16,
                                  "source": peaks["source"]}, "nominal": 4500.0}
-    out.update(measure_tensor_ceiling(fq, args.tensor_ceiling, ["zeros", "uniform_codes", "bell_shaped_codes"]))
+    out.update(measure_tensor_ceiling(fq, args.tensor_ceiling, ["zeros", "uniform_codes", "bell_shaped_codes",
+                                                                  "bell_shaped_codes+operand_traffic"]))
     out["device_status"] = fq.last_device_status()
     print(json.dumps(out), flush=True)
 

@@ -279,10 +279,14 @@ int falqon_last_device_status(falqon_stream stream);
  * and with it the clock).  Asynchronous on `stream`; the caller times a sequence of
  * launches with events.  *flops_out (host, nullable) receives the floating-point operations of one launch.
  * sink: device [4 * falqon_tensor_ceiling_ctas()] fp32 or NULL; receives partial sums of the accumulators (all zero
- * for zero operands).  1 <= kblocks <= 2^20.  A wait that runs out sets the device status word. */
+ * for zero operands).  1 <= kblocks <= 2^20.  A wait that runs out sets the device status word.
+ * load_src (device, nullable; load_bytes a multiple of 16384, at least 32768): when given, every CTA also streams
+ * 2 x 16 KB per k-block from that buffer into its operand slots through a 6-slot producer/consumer ring, i.e. the MMAs
+ * now wait for operand traffic from L2 as those of a real 256 x 256 tile pipeline do (a buffer that fits L2 stays
+ * there); the MMAs then multiply whatever the buffer holds, and the sums in `sink` follow from it. */
 int falqon_tensor_ceiling_ctas(void);
 int falqon_tensor_ceiling(int64_t kblocks, uint32_t seed, int32_t random_fill, float *sink, double *flops_out,
-                          falqon_stream stream);
+                          const void *load_src, size_t load_bytes, falqon_stream stream);
 
 /* Stages that the optional timing hook can bracket with CUDA events (bit i of the mask = stage i). */
 typedef enum {

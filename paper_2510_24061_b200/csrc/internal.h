@@ -191,6 +191,9 @@ cudaError_t launch_proxy_update_batched(const ProxyBatchLayer* layers, int count
 // operands resident in shared memory.  sink: device [4 * tensor_ceiling_ctas()] floats or null.
 int tensor_ceiling_ctas();
 double tensor_ceiling_flops(int kblocks);
-cudaError_t launch_tensor_ceiling(int kblocks, uint32_t seed, int random_fill, float* sink, int* status, cudaStream_t stream);
+// load_src / load_bytes: optional buffer (a multiple of 16 KB, at least 32 KB) streamed into the operand slots at the
+// rate of a real product's operand traffic.
+cudaError_t launch_tensor_ceiling(int kblocks, uint32_t seed, int random_fill, float* sink, int* status, const void* load_src,
+                                  size_t load_bytes, cudaStream_t stream);
 
 }  // namespace falqon

@@ -12,27 +12,33 @@ namespace falqon {
 namespace {
 
 constexpr int kCeilThreads = 128;
-constexpr int kCeilStages = 4;                       // operand slots the issuer cycles through, as a pipeline would
+constexpr int kCeilStages = 6;                       // operand slots the issuer cycles through, as the products' pipeline does
 constexpr uint32_t kCeilTileBytes = 128 * 128;       // 128 rows x 128 bytes of K (one swizzle row), per CTA
 constexpr uint32_t kCeilStageBytes = 2 * kCeilTileBytes;   // this CTA's half of A and of B
 constexpr uint32_t kCeilTmemCols = 512;              // two 256-column accumulators
 constexpr int kCeilKBlocksPerTile = 32;              // a fresh accumulation every 32 k-blocks (K = 4096)
-constexpr size_t kCeilSmem = kCeilStages * kCeilStageBytes + 64 + 1024;
+constexpr size_t kCeilSmem = kCeilStages * kCeilStageBytes + 128 + 1024;
 
 __device__ __forceinline__ uint32_t mix32(uint32_t x) {
   x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
   return x;
 }
 
+// load_src / load_chunks: optional.  When given, warp 0 of every CTA also streams 2 x 16 KB per k-block from that buffer
+// (load_chunks chunks of 16 KB) into the operand slots, paced by the MMAs like the producer of a real product is: the
+// traffic from L2 into shared memory of a 256 x 256 tile pipeline, without its dependencies (the MMAs read whatever the
+// slots hold, so the sums are then not reproducible).
 __global__ void __launch_bounds__(kCeilThreads, 1) tensor_ceiling_kernel(int kblocks, uint32_t seed, int random_fill,
-                                                                         float* sink, int* status) {
+                                                                         float* sink, int* status, const uint8_t* load_src,
+                                                                         uint32_t load_chunks) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t smem_base = (raw_addr + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - raw_addr);
   const uint32_t bars = smem_base + kCeilStages * kCeilStageBytes;
   auto done_bar = [&](int s) { return bars + 8u * s; };
-  const uint32_t slot_off = kCeilStages * kCeilStageBytes + 8u * kCeilStages;
+  auto load_bar = [&](int s) { return bars + 8u * (kCeilStages + s); };
+  const uint32_t slot_off = kCeilStages * kCeilStageBytes + 16u * kCeilStages;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + slot_off);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const bool leader = cluster_ctarank() == 0;
@@ -59,7 +65,7 @@ __global__ void __launch_bounds__(kCeilThreads, 1) tensor_ceiling_kernel(int kbl
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the tensor pipe
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kCeilStages; ++s) mbar_init(done_bar(s), 1);
+    for (int s = 0; s < kCeilStages; ++s) { mbar_init(done_bar(s), 1); mbar_init(load_bar(s), 1); }
     mbar_fence_init();
   }
   if (warp == 1) {
@@ -74,6 +80,34 @@ __global__ void __launch_bounds__(kCeilThreads, 1) tensor_ceiling_kernel(int kbl
   const uint32_t tmem_base = *tmem_slot;
 
   bool aborted = false;
+  if (warp == 0 && load_src != nullptr) {
+    // the stand-in for a TMA producer: slot s is refilled once the MMAs that used it are done (the same condition a
+    // real producer waits for) and its own previous copies have landed
+    int stage = 0;
+    uint32_t phase = 0, lphase = 0;
+    uint32_t chunk = (blockIdx.x * 2654435761u) % load_chunks;
+    for (int kb = 0; kb < kblocks && !aborted; ++kb) {
+      if (!mbar_wait_warp(done_bar(stage), phase ^ 1u, status)) { aborted = true; break; }
+      if (!mbar_wait_warp(load_bar(stage), lphase ^ 1u, status)) { aborted = true; break; }
+      if (elect_one()) {
+        const uint32_t dst = smem_base + static_cast<uint32_t>(stage) * kCeilStageBytes;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_expect_tx(load_bar(stage), 2 * kCeilTileBytes);
+        bulk_load_1d(dst, load_src + static_cast<size_t>(chunk) * kCeilTileBytes, kCeilTileBytes, load_bar(stage));
+        const uint32_t chunk2 = chunk + 1 < load_chunks ? chunk + 1 : 0;
+        bulk_load_1d(dst + kCeilTileBytes, load_src + static_cast<size_t>(chunk2) * kCeilTileBytes, kCeilTileBytes, load_bar(stage));
+      }
+      __syncwarp();
+      chunk += 2;
+      if (chunk >= load_chunks) chunk -= load_chunks;
+      if (++stage == kCeilStages) { stage = 0; phase ^= 1u; lphase ^= 1u; }
+    }
+    // every copy has landed before the CTA leaves
+    for (int i = 0; i < kCeilStages && !aborted; ++i) {
+      if (!mbar_wait_warp(load_bar(stage), lphase ^ 1u, status)) aborted = true;
+      if (++stage == kCeilStages) { stage = 0; lphase ^= 1u; }
+    }
+  }
   if (warp == 1) {
     int stage = 0;
     uint32_t phase = 0;
@@ -83,7 +117,10 @@ __global__ void __launch_bounds__(kCeilThreads, 1) tensor_ceiling_kernel(int kbl
       // E4M3 x E4M3 -> fp32, both operands K-major, N = 256, M = 256 over the pair
       const uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(256 >> 3) << 17) | (static_cast<uint32_t>(256 >> 4) << 24);
       for (int kb = 0; kb < kblocks; ++kb) {
-        if (!mbar_wait_warp(done_bar(stage), phase ^ 1u, status)) { aborted = true; break; }
+        // without the load stream: at most kCeilStages commits in flight; with it: the slot's copies have landed
+        const bool ok = load_src != nullptr ? mbar_wait_warp(load_bar(stage), phase, status)
+                                            : mbar_wait_warp(done_bar(stage), phase ^ 1u, status);
+        if (!ok) { aborted = true; break; }
         tc_fence_after_sync();
         const int in_tile = kb % kCeilKBlocksPerTile;
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>((kb / kCeilKBlocksPerTile) & 1) * 256u;
@@ -139,7 +176,8 @@ double tensor_ceiling_flops(int kblocks) {   // of one launch: every pair issues
   return static_cast<double>(tensor_ceiling_ctas() / 2) * kblocks * 4.0 * 2.0 * 256.0 * 256.0 * 32.0;
 }
 
-cudaError_t launch_tensor_ceiling(int kblocks, uint32_t seed, int random_fill, float* sink, int* status, cudaStream_t stream) {
+cudaError_t launch_tensor_ceiling(int kblocks, uint32_t seed, int random_fill, float* sink, int* status, const void* load_src,
+                                  size_t load_bytes, cudaStream_t stream) {
   static DeviceMask configured{0};
   {
     const cudaError_t ec = set_max_dynamic_smem(tensor_ceiling_kernel, static_cast<int>(kCeilSmem), configured);
@@ -157,7 +195,9 @@ cudaError_t launch_tensor_ceiling(int kblocks, uint32_t seed, int random_fill, f
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, tensor_ceiling_kernel, kblocks, seed, random_fill, sink, status);
+  const uint32_t load_chunks = load_src != nullptr ? static_cast<uint32_t>(load_bytes / kCeilTileBytes) : 0u;
+  return cudaLaunchKernelEx(&cfg, tensor_ceiling_kernel, kblocks, seed, random_fill, sink, status,
+                            load_chunks >= 2 ? static_cast<const uint8_t*>(load_src) : nullptr, load_chunks);
 }
 
 }  // namespace falqon

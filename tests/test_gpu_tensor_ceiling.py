@@ -69,3 +69,19 @@ def test_time_is_proportional_to_the_work_and_the_rate_is_plausible(fq):
     print(f"[tensor ceiling] {tflops:.0f} TFLOP/s over {t2 * 1e3:.1f} ms")
     assert 1000.0 < tflops < 4500.0 * 1.05          # above the nominal peak the kernel would not be doing the work
     assert fq.last_device_status() == 0
+
+
+def test_with_the_operand_stream(fq):
+    """The producer/consumer form (operands streamed from a buffer while the MMAs run) finishes cleanly for k-block counts
+    around the ring size, and the MMAs then see the buffer's contents: a buffer of zeros gives zero sums whatever the fill."""
+    src = torch.zeros(1 << 20, dtype=torch.uint8, device=DEV)
+    for kblocks in (1, 5, 6, 7, 40, 1000):
+        sink = _sink(fq)
+        fq.tensor_ceiling(kblocks, 3, 1, sink, src)
+        torch.cuda.synchronize()
+        assert fq.last_device_status() == 0
+        assert bool(torch.isfinite(sink).all())
+        if kblocks >= 40:
+            assert not bool(sink.any())      # the last accumulation ran entirely on streamed (zero) operands
+    with pytest.raises(fq.FalqonError):
+        fq.tensor_ceiling(8, 3, 1, None, src[:16384])
