@@ -89,9 +89,32 @@ def test_bad_arguments_are_rejected_on_the_host(fq):
     assert lib.falqon_proxy_update(C.byref(layer), None, 0.1, 1, None, fake, 64, None) == wsp
     assert lib.falqon_proxy_update(None, None, 0.1, 1, None, fake, big, None) == inv
 
+    # batched proxy update: host arrays; any bad entry rejects the whole call
+    two = (fq.falqon_layer * 2)(layer, fq.falqon_layer(128, 256, 8, fake + 0x100000, fake, fake + 0x200000, 0, 0))
+    p2, i2, z2 = (C.c_void_p * 2), (C.c_int64 * 2), (C.c_size_t * 2)
+    none2, ws2, big2 = p2(None, None), p2(fake + 0x300000, fake + 0x400000), z2(big, big)
+    call = lib.falqon_proxy_update_batched
+    assert call(two, 0, none2, 0.1, i2(1, 1), None, ws2, big2, None) == fq.OK                     # an empty call
+    assert call(two, -1, none2, 0.1, i2(1, 1), None, ws2, big2, None) == inv
+    assert call(None, 2, none2, 0.1, i2(1, 1), None, ws2, big2, None) == inv
+    assert call(two, 2, none2, 0.1, i2(1, 129), None, ws2, big2, None) == inv                     # k > m in the second layer
+    assert call(two, 2, none2, float("nan"), i2(1, 1), None, ws2, big2, None) == inv
+    assert call(two, 2, none2, 0.1, i2(1, 1), None, p2(fake + 0x300000, fake + 0x300000), big2, None) == inv   # shared workspace
+    assert call(two, 2, none2, 0.1, i2(1, 1), None, ws2, z2(big, 64), None) == wsp
+    assert call(two, 2, none2, 0.1, i2(1, 1), None, p2(fake + 0x300000, None), big2, None) == wsp
+    twice = (fq.falqon_layer * 2)(layer, layer)
+    assert call(twice, 2, none2, 0.1, i2(1, 1), None, ws2, big2, None) == inv                     # the same layer twice
+    # tensor ceiling
+    assert lib.falqon_tensor_ceiling(0, 1, 0, None, None, None, 0, None) == inv
+    assert lib.falqon_tensor_ceiling((1 << 20) + 1, 1, 0, None, None, None, 0, None) == inv
+    assert lib.falqon_tensor_ceiling(8, 1, 3, None, None, None, 0, None) == inv                   # no such fill
+    assert lib.falqon_tensor_ceiling(8, 1, 1, None, None, fake, 16384, None) == inv               # stream buffer too small
+    assert lib.falqon_tensor_ceiling(8, 1, 1, None, None, fake, 40000, None) == inv               # not whole chunks
+
 
 def test_launch_counts(fq):
     assert fq.launch_count("falqon_melded_forward") == 2
     assert fq.launch_count("falqon_melded_backward") == 3      # quantize, dX, fused dB
     assert fq.launch_count("falqon_proxy_update", k=4) == 2 and fq.launch_count("falqon_proxy_update", k=0) == 1
+    assert fq.launch_count("falqon_proxy_update_batched", k=4) == 2 and fq.launch_count("falqon_proxy_update_batched", k=0) == 1
     assert fq.launch_count("nope") == 0
