@@ -211,6 +211,14 @@ int falqon_proxy_update_adamw(const falqon_layer *L, const float *dB, float *exp
                               const falqon_adamw *hp, int64_t k, int32_t *idx_out, void *ws, size_t ws_bytes,
                               falqon_stream stream);
 
+/* falqon_proxy_update_adamw for `count` layers in two launches (falqon_proxy_update_batched with AdamW as the optimizer of
+ * every layer).  exp_avg[i], exp_avg_sq[i]: device [m_i][r_i] fp32 state of layer i; dB[i] must not be NULL.  The
+ * hyper-parameters (and the step count) are shared by the layers.  Bit-identical to the per-layer calls. */
+int falqon_proxy_update_batched_adamw(const falqon_layer *layers, int32_t count, const float *const *dB,
+                                      float *const *exp_avg, float *const *exp_avg_sq, const falqon_adamw *hp,
+                                      const int64_t *k, int32_t *const *idx_out, void *const *ws, const size_t *ws_bytes,
+                                      falqon_stream stream);
+
 /* The proxy update for callers that cannot provide a workspace.  The paper has no counterpart: this
  * is the same operation as falqon_proxy_update, with the same arguments minus the workspace, for code
  * that runs as a guest inside another runtime (a framework's custom-op hook, a server's plug-in) whose

@@ -23,7 +23,7 @@ WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 EXPORTS = ["falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
            "falqon_svd_init_scratch_bytes", "falqon_svd_init", "falqon_tensor_ceiling", "falqon_tensor_ceiling_ctas",
-           "falqon_melded_backward", "falqon_proxy_update", "falqon_proxy_update_batched", "falqon_last_device_status", "falqon_launch_count",
+           "falqon_melded_backward", "falqon_proxy_update", "falqon_proxy_update_batched", "falqon_proxy_update_batched_adamw", "falqon_last_device_status", "falqon_launch_count",
            "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static", "falqon_workspace_init", "falqon_proxy_update_adamw"]
 STATIC_MAX_ROWS = 16384
 STAGES = ["quant_x", "gemm_fwd", "quant_dy", "quant_oa", "gemm_dx", "gemm_db", "reduce_db", "sgd_score", "topk", "merge"]
@@ -64,6 +64,9 @@ lib.falqon_proxy_update.argtypes = [C.POINTER(falqon_layer), _p, _f, _i64, _p, _
 lib.falqon_proxy_update_batched.restype = _i
 lib.falqon_proxy_update_batched.argtypes = [C.POINTER(falqon_layer), C.c_int32, C.POINTER(_p), _f, C.POINTER(_i64), C.POINTER(_p),
                                             C.POINTER(_p), C.POINTER(_sz), _p]
+lib.falqon_proxy_update_batched_adamw.restype = _i
+lib.falqon_proxy_update_batched_adamw.argtypes = [C.POINTER(falqon_layer), C.c_int32, C.POINTER(_p), C.POINTER(_p), C.POINTER(_p),
+                                                  C.c_void_p, C.POINTER(_i64), C.POINTER(_p), C.POINTER(_p), C.POINTER(_sz), _p]
 lib.falqon_tensor_ceiling.restype = _i
 lib.falqon_tensor_ceiling.argtypes = [_i64, C.c_uint32, C.c_int32, _p, C.POINTER(C.c_double), _p, _sz, _p]
 lib.falqon_tensor_ceiling_ctas.restype = _i
@@ -329,6 +332,17 @@ class ProxyBatch:
         self.c_ws = (_p * max(n, 1))(*[_ptr(t) for t in self.wss])
         self.c_ws_bytes = (_sz * max(n, 1))(*[t.numel() for t in self.wss])
         self.count = n
+
+    def run_adamw(self, exp_avgs, exp_avg_sqs, lr: float, beta1: float, beta2: float, eps: float, weight_decay: float, step: int):
+        """falqon_proxy_update_batched_adamw with the per-layer state tensors exp_avgs / exp_avg_sqs (fp32 [m, r] each)."""
+        n = max(self.count, 1)
+        hp = falqon_adamw(lr, beta1, beta2, eps, weight_decay, step)
+        c_ea = (_p * n)(*[_ptr(t) for t in exp_avgs])
+        c_es = (_p * n)(*[_ptr(t) for t in exp_avg_sqs])
+        _check("falqon_proxy_update_batched_adamw",
+               lib.falqon_proxy_update_batched_adamw(self.c_layers, self.count, self.c_dB, c_ea, c_es, C.byref(hp), self.c_k,
+                                                     self.c_idx, self.c_ws, self.c_ws_bytes, _stream()))
+        return self.idx_outs
 
     def run(self, lr: float):
         _check("falqon_proxy_update_batched",

@@ -401,15 +401,27 @@ int falqon_proxy_update(const falqon_layer* L, const float* dB, float lr, int64_
   return proxy_update_impl(L, dB, lr, nullptr, nullptr, nullptr, k, idx_out, ws, ws_bytes, stream);
 }
 
-int falqon_proxy_update_batched(const falqon_layer* layers, int32_t count, const float* const* dB, float lr, const int64_t* k,
-                                int32_t* const* idx_out, void* const* ws, const size_t* ws_bytes, falqon_stream stream) {
+namespace {
+bool adamw_ok(const falqon_adamw* hp) {
+  return hp != nullptr && hp->step >= 1 && hp->lr == hp->lr && hp->beta1 >= 0.0f && hp->beta1 < 1.0f && hp->beta2 >= 0.0f &&
+         hp->beta2 < 1.0f && hp->eps >= 0.0f && hp->weight_decay == hp->weight_decay;
+}
+
+// hp == null: plain SGD with lr.  hp != null: AdamW on every layer (dB, exp_avg, exp_avg_sq all required).
+int proxy_update_batched_impl(const falqon_layer* layers, int32_t count, const float* const* dB, float lr, const falqon_adamw* hp,
+                              float* const* exp_avg, float* const* exp_avg_sq, const int64_t* k, int32_t* const* idx_out,
+                              void* const* ws, const size_t* ws_bytes, falqon_stream stream) {
   if (count < 0 || !(lr == lr)) return FALQON_ERR_INVALID_ARG;
   if (count == 0) return FALQON_OK;
   if (layers == nullptr || dB == nullptr || k == nullptr || ws == nullptr || ws_bytes == nullptr) return FALQON_ERR_INVALID_ARG;
+  if (hp != nullptr && (exp_avg == nullptr || exp_avg_sq == nullptr)) return FALQON_ERR_INVALID_ARG;
   bool fused = true;
   for (int32_t i = 0; i < count; ++i) {
     const falqon_layer* L = &layers[i];
     if (!layer_ok(L) || k[i] < 0 || k[i] > L->m || (dB[i] != nullptr && !aligned16(dB[i]))) return FALQON_ERR_INVALID_ARG;
+    if (hp != nullptr && (dB[i] == nullptr || exp_avg[i] == nullptr || exp_avg_sq[i] == nullptr || !aligned16(exp_avg[i]) ||
+                          !aligned16(exp_avg_sq[i])))
+      return FALQON_ERR_INVALID_ARG;
     WorkspaceLayout w;
     if (!make_layout(L->m, L->n, L->r, 1, &w)) return FALQON_ERR_INVALID_ARG;
     if (ws[i] == nullptr || !aligned16(ws[i]) || ws_bytes[i] < w.total) return FALQON_ERR_WORKSPACE;
@@ -419,12 +431,16 @@ int falqon_proxy_update_batched(const falqon_layer* layers, int32_t count, const
   }
   if (!fused) {
     for (int32_t i = 0; i < count; ++i) {
-      const int rc = proxy_update_impl(&layers[i], dB[i], lr, nullptr, nullptr, nullptr, k[i],
-                                       idx_out != nullptr ? idx_out[i] : nullptr, ws[i], ws_bytes[i], stream);
+      const int rc = proxy_update_impl(&layers[i], dB[i], lr, hp, hp != nullptr ? exp_avg[i] : nullptr,
+                                       hp != nullptr ? exp_avg_sq[i] : nullptr, k[i], idx_out != nullptr ? idx_out[i] : nullptr,
+                                       ws[i], ws_bytes[i], stream);
       if (rc != FALQON_OK) return rc;
     }
     return FALQON_OK;
   }
+  AdamwHyper hyper{};
+  if (hp != nullptr) hyper = AdamwHyper{hp->lr, hp->beta1, hp->beta2, hp->eps, hp->weight_decay, hp->step};
+  const AdamwHyper* adamw = hp != nullptr ? &hyper : nullptr;
   for (int32_t first = 0; first < count; first += kProxyBatchMax) {
     const int chunk = count - first < kProxyBatchMax ? count - first : kProxyBatchMax;
     ProxyBatchLayer b[kProxyBatchMax];
@@ -438,6 +454,8 @@ int falqon_proxy_update_batched(const falqon_layer* layers, int32_t count, const
       b[c].wq = L->wq;
       b[c].dbuf = L->dbuf;
       b[c].dB = dB[i];
+      b[c].exp_avg = hp != nullptr ? exp_avg[i] : nullptr;
+      b[c].exp_avg_sq = hp != nullptr ? exp_avg_sq[i] : nullptr;
       b[c].row_scales = L->gran == FALQON_PER_ROW ? L->s_w : nullptr;
       b[c].score = reinterpret_cast<float*>(base + w.score);
       b[c].sel_idx = reinterpret_cast<int32_t*>(base + w.sel_idx);
@@ -449,14 +467,28 @@ int falqon_proxy_update_batched(const falqon_layer* layers, int32_t count, const
     }
     {
       StageTimer timer(FALQON_STAGE_SGD_SCORE, stream);
-      FALQON_CUDA(launch_proxy_update_batched(b, chunk, lr, 0, stream));
+      FALQON_CUDA(launch_proxy_update_batched(b, chunk, lr, adamw, 0, stream));
     }
     if (any_merge) {
       StageTimer timer(FALQON_STAGE_MERGE, stream);
-      FALQON_CUDA(launch_proxy_update_batched(b, chunk, lr, 1, stream));
+      FALQON_CUDA(launch_proxy_update_batched(b, chunk, lr, adamw, 1, stream));
     }
   }
   return FALQON_OK;
+}
+
+}  // namespace
+
+int falqon_proxy_update_batched(const falqon_layer* layers, int32_t count, const float* const* dB, float lr, const int64_t* k,
+                                int32_t* const* idx_out, void* const* ws, const size_t* ws_bytes, falqon_stream stream) {
+  return proxy_update_batched_impl(layers, count, dB, lr, nullptr, nullptr, nullptr, k, idx_out, ws, ws_bytes, stream);
+}
+
+int falqon_proxy_update_batched_adamw(const falqon_layer* layers, int32_t count, const float* const* dB, float* const* exp_avg,
+                                      float* const* exp_avg_sq, const falqon_adamw* hp, const int64_t* k, int32_t* const* idx_out,
+                                      void* const* ws, const size_t* ws_bytes, falqon_stream stream) {
+  if (!adamw_ok(hp)) return FALQON_ERR_INVALID_ARG;
+  return proxy_update_batched_impl(layers, count, dB, hp->lr, hp, exp_avg, exp_avg_sq, k, idx_out, ws, ws_bytes, stream);
 }
 
 int falqon_proxy_update_adamw(const falqon_layer* L, const float* dB, float* exp_avg, float* exp_avg_sq,

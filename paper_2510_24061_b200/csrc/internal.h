@@ -176,6 +176,8 @@ struct ProxyBatchLayer {
   uint8_t* wq;
   float* dbuf;
   const float* dB;
+  float* exp_avg;               // AdamW state of this layer (both null for plain SGD)
+  float* exp_avg_sq;
   const float* row_scales;      // null for a per-tensor scale
   float* score;
   int32_t* sel_idx;
@@ -185,7 +187,13 @@ struct ProxyBatchLayer {
   int64_t m, n, r, k;
 };
 // phase 0: optimizer step, scores and selection of every layer; phase 1: the merge of every layer with k > 0.
-cudaError_t launch_proxy_update_batched(const ProxyBatchLayer* layers, int count, float lr, int phase, cudaStream_t stream);
+// adamw == null: plain SGD with `lr`; else AdamW with these hyper-parameters on every layer (lr is then ignored).
+struct AdamwHyper {
+  float lr, beta1, beta2, eps, weight_decay;
+  int64_t step;
+};
+cudaError_t launch_proxy_update_batched(const ProxyBatchLayer* layers, int count, float lr, const AdamwHyper* adamw, int phase,
+                                        cudaStream_t stream);
 
 // Measurement aid: every SM pair issues kblocks x 4 FP8 MMAs (256 x 256 x 32, the product kernels' instruction) on
 // operands resident in shared memory.  sink: device [4 * tensor_ceiling_ctas()] floats or null.

@@ -301,6 +301,8 @@ __global__ void __launch_bounds__(kTopkThreads) sgd_score_topk_kernel(float* dbu
 struct BatchedScoreLayer {
   float* dbuf;
   const float* dB;
+  float* exp_avg;
+  float* exp_avg_sq;
   float* score;
   int32_t* sel_idx;
   int32_t* idx_out;
@@ -310,7 +312,7 @@ struct BatchedScoreLayer {
 struct BatchedScoreArgs {
   BatchedScoreLayer layer[kProxyBatchMax];
   int count;
-  float neg_lr;
+  OptimizerArgs opt;     // the constants shared by all layers; kind and the state pointers are set per layer
 };
 __global__ void __launch_bounds__(kTopkThreads) score_topk_batched_kernel(const __grid_constant__ BatchedScoreArgs args) {
   extern __shared__ float fused_smem_dyn[];
@@ -321,9 +323,10 @@ __global__ void __launch_bounds__(kTopkThreads) score_topk_batched_kernel(const 
   for (int i = 1; i < args.count; ++i) l = static_cast<int>(blockIdx.x) >= args.layer[i].cta_begin ? i : l;
   const BatchedScoreLayer& a = args.layer[l];
   const int n_ctas = (a.m + kFusedScoreRows - 1) / kFusedScoreRows;
-  OptimizerArgs opt{};
-  opt.kind = a.dB != nullptr ? 1 : 0;
-  opt.neg_lr = args.neg_lr;
+  OptimizerArgs opt = args.opt;
+  if (a.dB == nullptr) opt.kind = 0;
+  opt.exp_avg = a.exp_avg;
+  opt.exp_avg_sq = a.exp_avg_sq;
   score_topk_body(a.dbuf, a.dB, opt, a.m, a.r, a.k, a.score, a.sel_idx, a.idx_out, a.done_counter,
                   a.m <= kTopkSmemRows ? 1 : 0, static_cast<int>(blockIdx.x) - a.cta_begin, n_ctas, fused_smem_dyn);
 }
@@ -694,10 +697,8 @@ cudaError_t launch_sgd_score_topk(float* dbuf, const float* dB, float lr, int64_
   return launch_opt_score_topk(dbuf, dB, opt, m, r, k, score, sel_idx, idx_copy, done_counter, stream);
 }
 
-cudaError_t launch_adamw_score_topk(float* dbuf, const float* dB, float* exp_avg, float* exp_avg_sq, float lr, float beta1,
-                                    float beta2, float eps, float weight_decay, int64_t step, int64_t m, int64_t r, int64_t k,
-                                    float* score, int32_t* sel_idx, int32_t* idx_copy, unsigned int* done_counter,
-                                    cudaStream_t stream) {
+namespace {
+OptimizerArgs adamw_args(float lr, float beta1, float beta2, float eps, float weight_decay, int64_t step) {
   OptimizerArgs opt{};
   opt.kind = 2;
   opt.beta1 = beta1; opt.beta2 = beta2; opt.eps = eps;
@@ -707,6 +708,15 @@ cudaError_t launch_adamw_score_topk(float* dbuf, const float* dB, float* exp_avg
   opt.one_minus_b2 = static_cast<float>(1.0 - static_cast<double>(beta2));
   opt.neg_step_size = -static_cast<float>(static_cast<double>(lr) / (1.0 - std::pow(static_cast<double>(beta1), static_cast<double>(step))));
   opt.sqrt_bc2 = static_cast<float>(std::sqrt(1.0 - std::pow(static_cast<double>(beta2), static_cast<double>(step))));
+  return opt;
+}
+}  // namespace
+
+cudaError_t launch_adamw_score_topk(float* dbuf, const float* dB, float* exp_avg, float* exp_avg_sq, float lr, float beta1,
+                                    float beta2, float eps, float weight_decay, int64_t step, int64_t m, int64_t r, int64_t k,
+                                    float* score, int32_t* sel_idx, int32_t* idx_copy, unsigned int* done_counter,
+                                    cudaStream_t stream) {
+  OptimizerArgs opt = adamw_args(lr, beta1, beta2, eps, weight_decay, step);
   opt.exp_avg = exp_avg;
   opt.exp_avg_sq = exp_avg_sq;
   return launch_opt_score_topk(dbuf, dB, opt, m, r, k, score, sel_idx, idx_copy, done_counter, stream);
@@ -745,7 +755,8 @@ cudaError_t launch_merge_batched(const ProxyBatchLayer* layers, int count, cudaS
 }
 }  // namespace
 
-cudaError_t launch_proxy_update_batched(const ProxyBatchLayer* layers, int count, float lr, int phase, cudaStream_t stream) {
+cudaError_t launch_proxy_update_batched(const ProxyBatchLayer* layers, int count, float lr, const AdamwHyper* adamw, int phase,
+                                        cudaStream_t stream) {
   if (count < 1 || count > kProxyBatchMax) return cudaErrorInvalidValue;
   if (phase != 0) return launch_merge_batched(layers, count, stream);
   static DeviceMask configured{0};
@@ -755,13 +766,18 @@ cudaError_t launch_proxy_update_batched(const ProxyBatchLayer* layers, int count
   }
   BatchedScoreArgs sa{};
   sa.count = count;
-  sa.neg_lr = -lr;
+  if (adamw != nullptr) {
+    sa.opt = adamw_args(adamw->lr, adamw->beta1, adamw->beta2, adamw->eps, adamw->weight_decay, adamw->step);
+  } else {
+    sa.opt.kind = 1;
+    sa.opt.neg_lr = -lr;
+  }
   int score_ctas = 0;
   size_t score_smem = 0;
   for (int i = 0; i < count; ++i) {
     const ProxyBatchLayer& L = layers[i];
     BatchedScoreLayer& a = sa.layer[i];
-    a.dbuf = L.dbuf; a.dB = L.dB; a.score = L.score; a.sel_idx = L.sel_idx; a.idx_out = L.idx_out;
+    a.dbuf = L.dbuf; a.dB = L.dB; a.exp_avg = L.exp_avg; a.exp_avg_sq = L.exp_avg_sq; a.score = L.score; a.sel_idx = L.sel_idx; a.idx_out = L.idx_out;
     a.done_counter = L.done_counter;
     a.m = static_cast<int>(L.m); a.r = static_cast<int>(L.r); a.k = static_cast<int>(L.k);
     a.cta_begin = score_ctas;

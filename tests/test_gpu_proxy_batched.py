@@ -108,3 +108,40 @@ def test_invalid_entries_reject_the_whole_call(fq):
         fq.proxy_update_batched([l0, l1], [dB0, dB1], 0.1, [4, 4], wss=[ws, ws])   # a shared workspace
     torch.cuda.synchronize()
     assert torch.equal(l0.wq, wq_before)
+
+
+def test_batched_adamw_equals_per_layer_calls_and_the_oracle(fq, orc):
+    """Three AdamW steps on four layers of different shapes: one batched call per step against one call per layer, bit
+    for bit (backbone, DeltaBuffer, both moments, indices); the first layer is also checked against the oracle."""
+    specs = [(256, 128, 16, 40), (640, 1280, 64, 133), (144, 400, 24, 0), (512, 256, 32, 512)]
+    hp = dict(lr=3e-3, beta1=0.9, beta2=0.99, eps=1e-8, weight_decay=0.01)
+    a, b = [], []
+    for i, (m, n, r, k) in enumerate(specs):
+        layer, _ = _make(fq, 76, i, m, n, r, False)
+        twin = fq.Layer(layer.wq.clone(), layer.s_w.clone(), layer.dbuf.clone(), r)
+        z = lambda: torch.zeros((m, r), dtype=torch.float32, device=DEV)
+        a.append(dict(layer=layer, ea=z(), es=z()))
+        b.append(dict(layer=twin, ea=z(), es=z()))
+    dBs = [torch.empty((m, r), dtype=torch.float32, device=DEV) for m, _, r, _ in specs]
+    batch = fq.ProxyBatch([x["layer"] for x in a], dBs, [s[3] for s in specs])
+    m0, n0, r0, k0 = specs[0]
+    wq_o, dbuf_o = u8(a[0]["layer"].wq).copy(), f32(a[0]["layer"].dbuf).copy()
+    ea_o, es_o = np.zeros((m0, r0), np.float32), np.zeros((m0, r0), np.float32)
+    for step in (1, 2, 3):
+        for i, (m, n, r, k) in enumerate(specs):
+            dBs[i].copy_((synth.normal_bf16(76, 300 + 16 * i + step, (m, r), 1.0).float() * 0.3).to(DEV))
+        idx_a = batch.run_adamw([x["ea"] for x in a], [x["es"] for x in a], step=step, **hp)
+        for i, (m, n, r, k) in enumerate(specs):
+            idx_b = fq.proxy_update_adamw(b[i]["layer"], dBs[i], b[i]["ea"], b[i]["es"], step, k, **hp)
+            if k > 0:
+                assert torch.equal(idx_a[i], idx_b), f"layer {i} step {step}: indices"
+            assert torch.equal(a[i]["layer"].wq, b[i]["layer"].wq), f"layer {i} step {step}: backbone"
+            for what, x, y in (("DeltaBuffer", a[i]["layer"].dbuf, b[i]["layer"].dbuf), ("exp_avg", a[i]["ea"], b[i]["ea"]),
+                               ("exp_avg_sq", a[i]["es"], b[i]["es"])):
+                assert torch.equal(x.view(torch.int32), y.view(torch.int32)), f"layer {i} step {step}: {what}"
+        orc.adamw_step(dbuf_o, f32(dBs[0]), ea_o, es_o, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"], step)
+        idx_o, _ = orc.proxy_update(wq_o, dbuf_o, None, 0.0, k0, m0, r0)
+        assert np.array_equal(u8(idx_a[0]), idx_o) and np.array_equal(u8(a[0]["layer"].wq), wq_o)
+        assert np.array_equal(bits32(f32(a[0]["layer"].dbuf)), bits32(dbuf_o))
+        assert np.array_equal(bits32(f32(a[0]["ea"])), bits32(ea_o)) and np.array_equal(bits32(f32(a[0]["es"])), bits32(es_o))
+    assert fq.last_device_status() == 0
