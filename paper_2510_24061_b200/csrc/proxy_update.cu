@@ -628,6 +628,16 @@ int merge_splits_budget(int64_t col_tiles_total, int64_t r_max) {
   const int64_t budget = per_sm * sm_count() / (col_tiles_total > 0 ? col_tiles_total : 1);
   return static_cast<int>(budget < 1 ? 1 : budget);
 }
+// ... but no CTA walks more than kMergeItemsMax groups: with many selected rows and a small rank the groups are short
+// and bound by memory latency, which more CTAs (several waves of them) hide better than a longer walk does.
+constexpr int kMergeItemsMax = 4;
+int merge_splits(int budget, int64_t groups) {
+  int64_t splits = (groups + kMergeItemsMax - 1) / kMergeItemsMax;
+  if (splits < budget) splits = budget;
+  if (splits > groups) splits = groups;
+  if (splits > 65535) splits = 65535;
+  return static_cast<int>(splits < 1 ? 1 : splits);
+}
 
 cudaError_t launch_merge_only(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n, int64_t r,
                               unsigned int* group_counters, const float* row_scales, cudaStream_t stream) {
@@ -637,9 +647,7 @@ cudaError_t launch_merge_only(uint8_t* wq, float* dbuf, const int32_t* sel_idx, 
     if (ec != cudaSuccess) return ec;
   }
   const int64_t col_tiles = (n + kMergeCols - 1) / kMergeCols, groups = (k + kMergeRows - 1) / kMergeRows;
-  int64_t splits = merge_splits_budget(col_tiles, r);
-  if (splits > groups) splits = groups;
-  if (splits > 65535) splits = 65535;
+  const int splits = merge_splits(merge_splits_budget(col_tiles, r), groups);
   dim3 grid(static_cast<unsigned>(col_tiles), static_cast<unsigned>(splits));
   return launch_pdl(merge_rows_kernel, grid, dim3(kMergeThreads), merge_smem_bytes(r), stream, 1, wq, dbuf, sel_idx,
                     static_cast<int>(k), m, n, static_cast<int>(r), group_counters, row_scales);
@@ -747,7 +755,7 @@ cudaError_t launch_merge_batched(const ProxyBatchLayer* layers, int count, cudaS
     b.cta_begin = ctas;
     b.col_tiles = static_cast<int>((L.n + kMergeCols - 1) / kMergeCols);
     const int groups = static_cast<int>((L.k + kMergeRows - 1) / kMergeRows);
-    b.splits = budget < groups ? budget : groups;
+    b.splits = merge_splits(budget, groups);
     ctas += b.col_tiles * b.splits;
   }
   if (ma.count == 0) return cudaSuccess;
