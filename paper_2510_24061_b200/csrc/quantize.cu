@@ -283,20 +283,23 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
   constexpr int64_t kChunkElems = kChunkBytes / kEsize;
   // dynamic shared memory: [table_floats column factors, padded to whole chunks][slots x 16 KB ring]
   extern __shared__ __align__(128) uint8_t staged_smem[];
-  const float* table = table_floats > 0 ? reinterpret_cast<const float*>(staged_smem) : nullptr;
-  uint8_t* stage = staged_smem + (static_cast<size_t>(table_floats) * 4 + kChunkBytes - 1) / kChunkBytes * kChunkBytes;
+  // (only the column-scaled form has a table; without one the ring is the whole array and its size a constant)
+  const float* table = kColMul && table_floats > 0 ? reinterpret_cast<const float*>(staged_smem) : nullptr;
+  uint8_t* stage = kColMul ? staged_smem + (static_cast<size_t>(table_floats) * 4 + kChunkBytes - 1) / kChunkBytes * kChunkBytes
+                           : staged_smem;
+  const int nslots = kColMul ? slots : kStagedSlots;
   __shared__ __align__(8) uint64_t bars[kStagedSlots];
   __shared__ uint32_t red[32];
   __shared__ int s_ok;
   const int tid = threadIdx.x;
   if (tid == 0) {
-    for (int s = 0; s < slots; ++s) mbar_init(smem_u32(&bars[s]), 1);
+    for (int s = 0; s < nslots; ++s) mbar_init(smem_u32(&bars[s]), 1);
     mbar_fence_init();
   }
   pdl_trigger();
   __syncthreads();
   pdl_wait();
-  if (table_floats > 0) {   // the column factors, once per CTA (they are read twice per element otherwise)
+  if (kColMul && table_floats > 0) {   // the column factors, once per CTA (they are read twice per element otherwise)
     float* tw = reinterpret_cast<float*>(staged_smem);
     for (int c = tid; c < table_floats; c += kStagedThreads) tw[c] = ld_stream(col_mul + c);
     __syncthreads();
@@ -311,8 +314,8 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
     const int64_t rem = bulk_elems - c * kChunkElems;
     return static_cast<int>(rem < kChunkElems ? rem : kChunkElems);
   };
-  auto issue = [&](int i) {   // one thread: fetch the CTA's i-th chunk into slot i mod slots
-    const int s = i % slots;
+  auto issue = [&](int i) {   // one thread: fetch the CTA's i-th chunk into slot i mod nslots
+    const int s = i % nslots;
     const int64_t c = chunk_of(i);
     const uint32_t bytes = static_cast<uint32_t>(chunk_elems(c)) * kEsize;   // a multiple of 32
     const uint32_t bar = smem_u32(&bars[s]);
@@ -323,12 +326,12 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
 
   // ---- pass 1: absmax
   if (tid == 0)
-    for (int i = 0; i < n_my && i < slots; ++i) issue(i);
+    for (int i = 0; i < n_my && i < nslots; ++i) issue(i);
   uint32_t phase_bits = 0;   // bit s: parity of the next completion of slot s
   uint32_t m = 0;
   bool failed = false;
-  for (int i = 0; i < n_my; ++i) {
-    const int s = i % slots;
+  // (the slot index is stepped along with i: an integer division per chunk costs as much as a third of the chunk's work)
+  for (int i = 0, s = 0; i < n_my; ++i, s = s + 1 == nslots ? 0 : s + 1) {
     const bool ok = mbar_wait(smem_u32(&bars[s]), (phase_bits >> s) & 1u, status);
     phase_bits ^= 1u << s;
     const int64_t e0 = chunk_of(i) * kChunkElems;
@@ -342,7 +345,7 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
       for (int e = 0; e < kUnit; ++e) m = max(m, abs_bits(x[e]));
     }
     if (!__syncthreads_and(ok)) { failed = true; break; }   // block-uniform; also: the slot is free again
-    if (tid == 0 && i + slots < n_my) issue(i + slots);
+    if (tid == 0 && i + nslots < n_my) issue(i + nslots);
   }
   if (blockIdx.x == 0) {   // ragged tail
     for (int64_t e = bulk_elems + tid; e < count; e += kStagedThreads) {
@@ -387,11 +390,10 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
       if (out.clear_word) *out.clear_word = 0.0f;
     }
     // ---- pass 2: cast, most recent chunk first
-    for (int t = 0; t < n_my; ++t) {
+    for (int t = 0, s = n_my > 0 ? (n_my - 1) % nslots : 0; t < n_my; ++t, s = (s == 0 ? nslots : s) - 1) {
       const int i = n_my - 1 - t;
-      const int s = i % slots;
       bool ok = true;
-      if (t >= slots) {   // this chunk had left the ring and was fetched again
+      if (t >= nslots) {   // this chunk had left the ring and was fetched again
         ok = mbar_wait(smem_u32(&bars[s]), (phase_bits >> s) & 1u, status);
         phase_bits ^= 1u << s;
       }
@@ -413,9 +415,9 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
           cast_unit<kDt, kFmt, kColMul>(q1, e0 + static_cast<int64_t>(u1) * kUnit,
                                         kColMul ? static_cast<int>(wrap_col(col0 + static_cast<uint32_t>(u1) * kUnit, ucols)) : 0, col_mul, table, sc, dst);
       }
-      if (t + slots < n_my) {
+      if (t + nslots < n_my) {
         if (!__syncthreads_and(ok)) { failed = true; break; }
-        if (tid == 0) issue(i - slots);
+        if (tid == 0) issue(i - nslots);
       }
     }
     if (blockIdx.x == 0) {
