@@ -291,10 +291,12 @@ int falqon_last_device_status(falqon_stream stream);
  * load_src (device, nullable; load_bytes a multiple of 16384, at least 32768): when given, every CTA also streams
  * 2 x 16 KB per k-block from that buffer into its operand slots through a 6-slot producer/consumer ring, i.e. the MMAs
  * now wait for operand traffic from L2 as those of a real 256 x 256 tile pipeline do (a buffer that fits L2 stays
- * there); the MMAs then multiply whatever the buffer holds, and the sums in `sink` follow from it. */
+ * there); the MMAs then multiply whatever the buffer holds, and the sums in `sink` follow from it.
+ * bytes_per_kblock: what one CTA fetches per k-block (four MMAs): 0 or 32768 for the traffic of 256 x 256 tiles, down to
+ * 16384 (a multiple of 16) to model tiles that share more of their operands. */
 int falqon_tensor_ceiling_ctas(void);
 int falqon_tensor_ceiling(int64_t kblocks, uint32_t seed, int32_t random_fill, float *sink, double *flops_out,
-                          const void *load_src, size_t load_bytes, falqon_stream stream);
+                          const void *load_src, size_t load_bytes, int32_t bytes_per_kblock, falqon_stream stream);
 
 /* Stages that the optional timing hook can bracket with CUDA events (bit i of the mask = stage i). */
 typedef enum {

@@ -68,7 +68,7 @@ lib.falqon_proxy_update_batched_adamw.restype = _i
 lib.falqon_proxy_update_batched_adamw.argtypes = [C.POINTER(falqon_layer), C.c_int32, C.POINTER(_p), C.POINTER(_p), C.POINTER(_p),
                                                   C.c_void_p, C.POINTER(_i64), C.POINTER(_p), C.POINTER(_p), C.POINTER(_sz), _p]
 lib.falqon_tensor_ceiling.restype = _i
-lib.falqon_tensor_ceiling.argtypes = [_i64, C.c_uint32, C.c_int32, _p, C.POINTER(C.c_double), _p, _sz, _p]
+lib.falqon_tensor_ceiling.argtypes = [_i64, C.c_uint32, C.c_int32, _p, C.POINTER(C.c_double), _p, _sz, C.c_int32, _p]
 lib.falqon_tensor_ceiling_ctas.restype = _i
 lib.falqon_tensor_ceiling_ctas.argtypes = []
 class falqon_adamw(C.Structure):
@@ -297,14 +297,14 @@ def proxy_update(layer: Layer, dB: torch.Tensor | None, lr: float, k: int, ws: t
 
 
 def tensor_ceiling(kblocks: int, seed: int = 1, random_fill: int = 1, sink: torch.Tensor | None = None,
-                   load_src: torch.Tensor | None = None) -> float:
+                   load_src: torch.Tensor | None = None, bytes_per_kblock: int = 0) -> float:
     """falqon_tensor_ceiling: one launch of the MMA-issue-only measurement kernel on the current stream.  Returns the
     floating-point operations of the launch (time a sequence of launches with events to get a rate).  load_src: an
     optional uint8 device buffer whose 16 KB chunks are streamed into the operand slots as a product's operands are."""
     flops = C.c_double()
     _check("falqon_tensor_ceiling", lib.falqon_tensor_ceiling(kblocks, seed, int(random_fill), _ptr(sink), C.byref(flops),
                                                              _ptr(load_src), 0 if load_src is None else load_src.numel(),
-                                                             _stream()))
+                                                             bytes_per_kblock, _stream()))
     return flops.value
 
 

@@ -537,14 +537,16 @@ int falqon_svd_init(const void* W, falqon_dtype w_dt, int64_t m, int64_t n, cons
 int falqon_tensor_ceiling_ctas(void) { return tensor_ceiling_ctas(); }
 
 int falqon_tensor_ceiling(int64_t kblocks, uint32_t seed, int32_t random_fill, float* sink, double* flops_out,
-                          const void* load_src, size_t load_bytes, falqon_stream stream) {
+                          const void* load_src, size_t load_bytes, int32_t bytes_per_kblock, falqon_stream stream) {
+  if (bytes_per_kblock == 0) bytes_per_kblock = 32768;
+  if (bytes_per_kblock < 16384 || bytes_per_kblock > 32768 || bytes_per_kblock % 16 != 0) return FALQON_ERR_INVALID_ARG;
   if (kblocks < 1 || kblocks > (1 << 20) || random_fill < 0 || random_fill > 2 || (sink != nullptr && !aligned16(sink)))
     return FALQON_ERR_INVALID_ARG;
   if (load_src != nullptr && (!aligned16(load_src) || load_bytes < 32768 || load_bytes % 16384 != 0)) return FALQON_ERR_INVALID_ARG;
   int* status = status_ptr();
   if (status == nullptr) return FALQON_ERR_CUDA;
   if (flops_out != nullptr) *flops_out = tensor_ceiling_flops(static_cast<int>(kblocks));
-  FALQON_CUDA(launch_tensor_ceiling(static_cast<int>(kblocks), seed, random_fill, sink, status, load_src, load_bytes, stream));
+  FALQON_CUDA(launch_tensor_ceiling(static_cast<int>(kblocks), seed, random_fill, sink, status, load_src, load_bytes, bytes_per_kblock, stream));
   return FALQON_OK;
 }
 

@@ -201,7 +201,8 @@ int tensor_ceiling_ctas();
 double tensor_ceiling_flops(int kblocks);
 // load_src / load_bytes: optional buffer (a multiple of 16 KB, at least 32 KB) streamed into the operand slots at the
 // rate of a real product's operand traffic.
+// bytes_per_kblock: 16384 .. 32768, a multiple of 16 (what one CTA fetches per four MMAs: 32768 for 256 x 256 tiles).
 cudaError_t launch_tensor_ceiling(int kblocks, uint32_t seed, int random_fill, float* sink, int* status, const void* load_src,
-                                  size_t load_bytes, cudaStream_t stream);
+                                  size_t load_bytes, int bytes_per_kblock, cudaStream_t stream);
 
 }  // namespace falqon

@@ -24,13 +24,14 @@ __device__ __forceinline__ uint32_t mix32(uint32_t x) {
   return x;
 }
 
-// load_src / load_chunks: optional.  When given, warp 0 of every CTA also streams 2 x 16 KB per k-block from that buffer
+// load_src / load_chunks: optional.  When given, warp 0 of every CTA also streams 16 KB + second_copy_bytes (2 x 16 KB
+// for the traffic of a 256 x 256 tile, less for that of wider tiles) per k-block from that buffer
 // (load_chunks chunks of 16 KB) into the operand slots, paced by the MMAs like the producer of a real product is: the
 // traffic from L2 into shared memory of a 256 x 256 tile pipeline, without its dependencies (the MMAs read whatever the
 // slots hold, so the sums are then not reproducible).
 __global__ void __launch_bounds__(kCeilThreads, 1) tensor_ceiling_kernel(int kblocks, uint32_t seed, int random_fill,
                                                                          float* sink, int* status, const uint8_t* load_src,
-                                                                         uint32_t load_chunks) {
+                                                                         uint32_t load_chunks, uint32_t second_copy_bytes) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t smem_base = (raw_addr + 1023u) & ~1023u;
@@ -92,10 +93,11 @@ __global__ void __launch_bounds__(kCeilThreads, 1) tensor_ceiling_kernel(int kbl
       if (elect_one()) {
         const uint32_t dst = smem_base + static_cast<uint32_t>(stage) * kCeilStageBytes;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_expect_tx(load_bar(stage), 2 * kCeilTileBytes);
+        mbar_expect_tx(load_bar(stage), kCeilTileBytes + second_copy_bytes);
         bulk_load_1d(dst, load_src + static_cast<size_t>(chunk) * kCeilTileBytes, kCeilTileBytes, load_bar(stage));
         const uint32_t chunk2 = chunk + 1 < load_chunks ? chunk + 1 : 0;
-        bulk_load_1d(dst + kCeilTileBytes, load_src + static_cast<size_t>(chunk2) * kCeilTileBytes, kCeilTileBytes, load_bar(stage));
+        if (second_copy_bytes > 0)
+          bulk_load_1d(dst + kCeilTileBytes, load_src + static_cast<size_t>(chunk2) * kCeilTileBytes, second_copy_bytes, load_bar(stage));
       }
       __syncwarp();
       chunk += 2;
@@ -177,7 +179,7 @@ double tensor_ceiling_flops(int kblocks) {   // of one launch: every pair issues
 }
 
 cudaError_t launch_tensor_ceiling(int kblocks, uint32_t seed, int random_fill, float* sink, int* status, const void* load_src,
-                                  size_t load_bytes, cudaStream_t stream) {
+                                  size_t load_bytes, int bytes_per_kblock, cudaStream_t stream) {
   static DeviceMask configured{0};
   {
     const cudaError_t ec = set_max_dynamic_smem(tensor_ceiling_kernel, static_cast<int>(kCeilSmem), configured);
@@ -197,7 +199,8 @@ cudaError_t launch_tensor_ceiling(int kblocks, uint32_t seed, int random_fill, f
   cfg.numAttrs = 1;
   const uint32_t load_chunks = load_src != nullptr ? static_cast<uint32_t>(load_bytes / kCeilTileBytes) : 0u;
   return cudaLaunchKernelEx(&cfg, tensor_ceiling_kernel, kblocks, seed, random_fill, sink, status,
-                            load_chunks >= 2 ? static_cast<const uint8_t*>(load_src) : nullptr, load_chunks);
+                            load_chunks >= 2 ? static_cast<const uint8_t*>(load_src) : nullptr, load_chunks,
+                            static_cast<uint32_t>(bytes_per_kblock) - kCeilTileBytes);
 }
 
 }  // namespace falqon

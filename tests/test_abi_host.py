@@ -105,11 +105,12 @@ def test_bad_arguments_are_rejected_on_the_host(fq):
     twice = (fq.falqon_layer * 2)(layer, layer)
     assert call(twice, 2, none2, 0.1, i2(1, 1), None, ws2, big2, None) == inv                     # the same layer twice
     # tensor ceiling
-    assert lib.falqon_tensor_ceiling(0, 1, 0, None, None, None, 0, None) == inv
-    assert lib.falqon_tensor_ceiling((1 << 20) + 1, 1, 0, None, None, None, 0, None) == inv
-    assert lib.falqon_tensor_ceiling(8, 1, 3, None, None, None, 0, None) == inv                   # no such fill
-    assert lib.falqon_tensor_ceiling(8, 1, 1, None, None, fake, 16384, None) == inv               # stream buffer too small
-    assert lib.falqon_tensor_ceiling(8, 1, 1, None, None, fake, 40000, None) == inv               # not whole chunks
+    assert lib.falqon_tensor_ceiling(0, 1, 0, None, None, None, 0, 0, None) == inv
+    assert lib.falqon_tensor_ceiling((1 << 20) + 1, 1, 0, None, None, None, 0, 0, None) == inv
+    assert lib.falqon_tensor_ceiling(8, 1, 3, None, None, None, 0, 0, None) == inv                   # no such fill
+    assert lib.falqon_tensor_ceiling(8, 1, 1, None, None, fake, 16384, 0, None) == inv               # stream buffer too small
+    assert lib.falqon_tensor_ceiling(8, 1, 1, None, None, fake, 40000, 0, None) == inv            # not whole chunks
+    assert lib.falqon_tensor_ceiling(8, 1, 1, None, None, fake, 65536, 8192, None) == inv         # fewer bytes per k-block than one tile
 
 
 def test_launch_counts(fq):
