@@ -92,7 +92,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* st
   }
 }
 
-// The same wait executed by a whole converged warp; the verdict is made warp-uniform.
+// The same wait executed by a whole converged warp; the outcome is made warp-uniform.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* status) {
   const bool ok = mbar_wait(bar, parity, status);
   return __all_sync(0xFFFFFFFFu, ok);
