@@ -162,14 +162,16 @@ __device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
 
 // ---- fused per-tensor quantizer: absmax, a grid-wide barrier, then the cast, in ONE kernel, with the tensor held
 // in shared memory across the barrier.  All CTAs are co-resident (one per SM; the host sizes the grid from the
-// occupancy), so a CTA can wait for the others; the wait is bounded.  Each CTA streams its 16 KB chunks (chunk c belongs to CTA c mod grid)
+// occupancy), so a CTA can wait for the others; the wait is bounded.  Each CTA streams its 56 KB chunks (chunk c belongs to CTA c mod grid;
+// every chunk costs a barrier wait and a CTA-wide synchronisation, so few large chunks beat many small ones: 14 x 16 KB
+// was 10 % slower)
 // through a ring of kStagedSlots bulk-copy targets, so up to 224 KB per SM are in flight or resident without
 // costing a register.  After the barrier the chunks still in the ring (the last kStagedSlots of the CTA) are cast
 // straight from shared memory; earlier ones are fetched again, most recent first (what L2 still holds), into the
 // slots as they free up.  Tensors up to 148 x 224 KB are read from memory exactly once.
 constexpr int kStagedThreads = 512;
-constexpr int kChunkBytes = 16384;
-constexpr int kStagedSlots = 14;
+constexpr int kChunkBytes = 57344;
+constexpr int kStagedSlots = 4;
 
 template <int kDt> struct Unit { static constexpr int kElems = kDt == kBF16 ? 8 : 4; };
 
@@ -251,7 +253,7 @@ __device__ __forceinline__ void cast_oa_transposed(const OaCastJob& job, int w, 
 // x mod cols for x < cols + 8192 (a column offset inside one chunk): a compare and a subtract for the wide rows of
 // real layers, a division only for narrow ones.
 __device__ __forceinline__ uint32_t wrap_col(uint32_t x, uint32_t cols) {
-  if (cols >= 8192u) return x >= cols ? x - cols : x;
+  if (cols >= static_cast<uint32_t>(kChunkBytes / 2)) return x >= cols ? x - cols : x;
   return x % cols;
 }
 
@@ -568,7 +570,7 @@ cudaError_t launch_staged_variant(const void* src, int64_t count, uint8_t* dst, 
   int table_floats = 0, slots = kStagedSlots;
   if (kColMul) {
     const int table_chunks = static_cast<int>((static_cast<int64_t>(cols) * 4 + kChunkBytes - 1) / kChunkBytes);
-    if (table_chunks <= kStagedSlots - 8) { table_floats = cols; slots = kStagedSlots - table_chunks; }
+    if (table_chunks <= kStagedSlots - (128 * 1024) / kChunkBytes) { table_floats = cols; slots = kStagedSlots - table_chunks; }
   }
   return launch_pdl(quantize_staged_kernel<kDt, kFmt, kColMul>, dim3(static_cast<unsigned>(grid)), dim3(kStagedThreads), kSmem,
                     stream, 1, src, count, dst, partial, static_cast<GridSync*>(sync), out, status, col_mul, cols, oa_job, slots,
