@@ -145,3 +145,26 @@ def test_batched_adamw_equals_per_layer_calls_and_the_oracle(fq, orc):
         assert np.array_equal(bits32(f32(a[0]["layer"].dbuf)), bits32(dbuf_o))
         assert np.array_equal(bits32(f32(a[0]["ea"])), bits32(ea_o)) and np.array_equal(bits32(f32(a[0]["es"])), bits32(es_o))
     assert fq.last_device_status() == 0
+
+
+def test_ctas_that_walk_several_row_groups(fq, orc):
+    """Eight layers of ten column tiles each and many selected rows: the launch has more (column tile, row group) pairs
+    than resident CTAs, so every CTA walks two or three row groups (prefetch of the next group, ring of row indices,
+    late clearing of the DeltaBuffer rows), with a ragged last group and a ragged last column tile, per-tensor and
+    per-row layers mixed."""
+    specs = [(656 + 16 * i, 1264, 16, 600 + 7 * i, i % 3 == 2, True) for i in range(8)]
+    _check_against_oracle(fq, orc, specs, 2e-2, 77, steps=2)
+
+
+def test_single_layer_call_whose_ctas_walk_several_row_groups(fq, orc):
+    """falqon_proxy_update on one wide layer with every row selected (the set-up meld): 32 column tiles x 64 row groups
+    exceed the resident CTAs, so each CTA of the single-layer merge kernel walks three or four row groups."""
+    m, n, r = 2048, 4096, 16
+    layer, dB = _make(fq, 78, 0, m, n, r, False)
+    wq_o, dbuf_o = u8(layer.wq).copy(), f32(layer.dbuf).copy()
+    idx = fq.proxy_update(layer, dB, 5e-2, m)
+    idx_o, _ = orc.proxy_update(wq_o, dbuf_o, f32(dB), 5e-2, m, m, r)
+    assert np.array_equal(u8(idx), idx_o)
+    assert np.array_equal(u8(layer.wq), wq_o)
+    assert not f32(layer.dbuf).any() and not dbuf_o.any()
+    assert fq.last_device_status() == 0
