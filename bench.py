@@ -568,8 +568,11 @@ def main():
                             if all((n, m) in GEMM_DRAM_BYTES for _, n, m in linears) else None),
                 "traffic_note": "dram read+write bytes per average launch, from the ncu capture of the forward and dX "
                                 "launch of each projection shape (profiles/gemm_fp8_pair_kernel__traffic_by_shape.md); "
-                                "algorithmic operand bytes per average launch: %.1f MB" %
-                                (sum((T * n + (m + r) * n) + (T * m + m * n) for _, n, m in linears) / (2.0 * len(linears)) / 1e6)}
+                                "algorithmic bytes per average launch: %.1f MB of FP8 operands + %.1f MB of bf16 / fp32 "
+                                "outputs (an operand the preceding cast left in L2, or an output still in L2 when the "
+                                "kernel ends, does not show up as DRAM traffic)" %
+                                (sum((T * n + (m + r) * n) + (T * m + m * n) for _, n, m in linears) / (2.0 * len(linears)) / 1e6,
+                                 sum((2 * T * m + 4 * T * r) + 2 * T * n for _, n, m in linears) / (2.0 * len(linears)) / 1e6)}
     t_db = sum(ms for name, ms in records if name == "gemm_db")
 
     # ---- stage breakdown (separate untimed-for-value pass with every stage bracketed)
