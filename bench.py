@@ -366,7 +366,8 @@ def run_stack(args):
     H, F, n_layers = 4096, 11008, args.stack_layers
     peaks = measured_peaks()
     stack = st.Stack(n_layers, H, F, T, r, k, seed=cfg["seed"], device=dev, lr=lr, producer_amax=not args.stack_own_absmax,
-                     batched_proxy=not args.proxy_per_layer)
+                     batched_proxy=not args.proxy_per_layer,
+                     adamw=dict(beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0) if args.stack_adamw else None)
     h0 = synth.normal_bf16(cfg["seed"], 9001, (T, H), 1.0, dev)
     G = synth.normal_bf16(cfg["seed"], 9002, (T, H), 1.0e-2, dev)
     steps, warmup = max(1, min(args.steps, 20)), max(3, min(args.warmup, 5))
@@ -399,7 +400,9 @@ def run_stack(args):
         "config": {"workload": f"configs[2]: {n_layers} chained blocks of the LLaMA-7B projection set, tokens=4096, rank=64, "
                                "top-k=256, q/k/v and gate/up share one quantized input, bf16 chain kernels between the layers",
                    "tokens": T, "rank": r, "topk": k, "matrices": 7 * n_layers, "tflop_per_step": flops / 1e12,
-                   "l2": "working set far larger than L2 (every step touches the whole stack)", "parallelism": "single GPU"},
+                   "l2": "working set far larger than L2 (every step touches the whole stack)", "parallelism": "single GPU",
+                   "optimizer": "AdamW on the DeltaBuffers" if args.stack_adamw else "SGD on the DeltaBuffers",
+                   "proxy_update": "one call per projection" if args.proxy_per_layer else "one batched call per block"},
         "clocks": clocks, "gpu_launches": stack.launches_per_step() * steps,
         "frac_of_fp8_peak": {"of_measured_sustained_x2": tf / (peaks["bf16_sustained"] * FP8_OVER_BF16),
                              "of_nominal_4500": tf / 4500.0},
@@ -431,6 +434,8 @@ def main():
     ap.add_argument("--stack-layers", type=int, default=32)
     ap.add_argument("--stack-own-absmax", action="store_true",
                     help="with --stack: every layer takes the absmax of its input itself (the chain kernels do not hand it over)")
+    ap.add_argument("--stack-adamw", action="store_true",
+                    help="with --stack: AdamW (beta 0.9 / 0.999, eps 1e-8, no weight decay) on every DeltaBuffer instead of plain SGD")
     ap.add_argument("--config3", action="store_true",
                     help="configs[3] instead of configs[1]: the LLaMA-13B projection set, 8192 tokens, per-row-scaled "
                          "heavy-tailed backbone, top-512 (not the headline line)")

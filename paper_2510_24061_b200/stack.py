@@ -95,13 +95,17 @@ class Stack:
     """n_layers blocks with hidden size H and MLP width F, T tokens per step, LoRA rank r, top-k rows per update."""
 
     def __init__(self, n_layers: int, H: int, F: int, T: int, r: int, k: int, seed: int, device, lr: float = 2e-4,
-                 producer_amax: bool = True, batched_proxy: bool = True):
+                 producer_amax: bool = True, batched_proxy: bool = True, adamw: dict | None = None):
         """producer_amax: the chain kernels hand the absmax of their outputs to the layers that consume them, whose
         input casts are then single-pass (False: every layer takes the absmax of its input itself).
         batched_proxy: the seven proxy updates of a block run as one falqon_proxy_update_batched call at the end of
         the block's backward (False: one falqon_proxy_update after every projection's backward; same results, since
-        nothing later in the backward reads an updated backbone)."""
+        nothing later in the backward reads an updated backbone).
+        adamw: None for the plain SGD step with lr, or the hyper-parameters (beta1, beta2, eps, weight_decay; lr is the
+        argument above) of AdamW on every DeltaBuffer -- the optimizer the paper trains with; needs batched_proxy."""
         self.n_layers, self.H, self.F, self.T, self.r, self.k, self.lr = n_layers, H, F, T, r, k, lr
+        self.adamw, self.steps_done = adamw, 0
+        assert adamw is None or batched_proxy
         self.producer_amax = producer_amax
         self.device = torch.device(device)
         self.seed = seed
@@ -152,6 +156,10 @@ class Stack:
             self.batches = [fq.ProxyBatch([self.layers[l][p] for p in PROJ], [self.dB[p] for p in PROJ], [k] * len(PROJ),
                                           wss=[self.ws[p] for p in PROJ], idx_outs=[None] * len(PROJ))
                             for l in range(n_layers)]
+        if adamw is not None:   # first and second moments of every DeltaBuffer, zero before the first step
+            z = lambda p: torch.zeros((self.shapes[p][1], r), dtype=torch.float32, device=dev)
+            self.exp_avg = [[z(p) for p in PROJ] for _ in range(n_layers)]
+            self.exp_avg_sq = [[z(p) for p in PROJ] for _ in range(n_layers)]
         # absmax words of the chain's outputs, one row per block: x1, a, x2, z | ddn, dg, du, dhp, dqkv (cleared every step)
         self.amax = torch.zeros((n_layers, 16), dtype=torch.float32, device=dev)
         self.capture = None   # optional: {(block, proj): dict} filled with references / copies for parity checks
@@ -236,12 +244,17 @@ class Stack:
             combine(self.dh, self.dhp, 1.0, self.dx[1], 1.0)
             dh = self.dh
             if self.batches is not None:
-                self.batches[l].run(self.lr)
+                if self.adamw is None:
+                    self.batches[l].run(self.lr)
+                else:
+                    self.batches[l].run_adamw(self.exp_avg[l], self.exp_avg_sq[l], lr=self.lr, step=self.steps_done + 1,
+                                              **self.adamw)
         return dh
 
     def step(self, h0: torch.Tensor, G: torch.Tensor):
         h = self.forward(h0)
         self.backward(G)
+        self.steps_done += 1
         return h
 
     # ---- bookkeeping for the benchmark line

@@ -170,3 +170,32 @@ def test_stack_7b_shapes_sampled(fq, st, orc):
     last and two other blocks are checked on sampled rows."""
     stack = _run_and_check(fq, st, orc, 32, 4096, 11008, 4096, 64, 256, check_blocks=[0, 11, 22, 31], n_rows=24)
     assert stack.flops_per_step() == pytest.approx(107.41e12, rel=1e-3)
+
+
+def test_small_stack_with_adamw(fq, st, orc):
+    """Two steps of a narrow three-block chain with AdamW on every DeltaBuffer (one batched AdamW update per block): the
+    first projection of every block is followed on the CPU from the captured gradients (oracle AdamW step, then the
+    oracle's selection and merge), bit for bit."""
+    n_layers, H, F, T, r, k = 3, 256, 640, 192, 16, 8
+    hp = dict(beta1=0.9, beta2=0.99, eps=1e-8, weight_decay=0.01)
+    stack = st.Stack(n_layers, H, F, T, r, k, seed=11, device=DEV, lr=3e-3, adamw=hp)
+    h0 = synth.normal_bf16(11, 9001, (T, H), 1.0, DEV)
+    G = synth.normal_bf16(11, 9002, (T, H), 1.0e-2, DEV)
+    follow = {l: dict(wq=u8(stack.layers[l]["q"].wq).copy(), dbuf=f32(stack.layers[l]["q"].dbuf).copy(),
+                      ea=np.zeros((H, r), np.float32), es=np.zeros((H, r), np.float32)) for l in range(n_layers)}
+    for step in (1, 2):
+        stack.capture = {(l, "q"): {} for l in range(n_layers)}
+        h = stack.step(h0, G)
+        torch.cuda.synchronize()
+        assert bool(torch.isfinite(h.float()).all())
+        for l in range(n_layers):
+            o = follow[l]
+            orc.adamw_step(o["dbuf"], f32(stack.capture[(l, "q")]["dB"]), o["ea"], o["es"], 3e-3, hp["beta1"], hp["beta2"],
+                           hp["eps"], hp["weight_decay"], step)
+            orc.proxy_update(o["wq"], o["dbuf"], None, 0.0, k, H, r)
+            layer = stack.layers[l]["q"]
+            assert np.array_equal(u8(layer.wq), o["wq"]), f"block {l} step {step}: backbone"
+            assert np.array_equal(bits32(f32(layer.dbuf)), bits32(o["dbuf"])), f"block {l} step {step}: DeltaBuffer"
+            assert np.array_equal(bits32(f32(stack.exp_avg[l][0])), bits32(o["ea"])), f"block {l} step {step}: exp_avg"
+            assert np.array_equal(bits32(f32(stack.exp_avg_sq[l][0])), bits32(o["es"])), f"block {l} step {step}: exp_avg_sq"
+    assert fq.last_device_status() == 0
