@@ -425,7 +425,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="falqon", choices=["falqon", "reference"])
-    ap.add_argument("--oracle-tokens", type=int, default=256)
+    ap.add_argument("--oracle-tokens", type=int, default=4096,
+                    help="token rows of the q projection the CPU oracle is timed on (4096 = the whole projection, 10-30 s of CPU work)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true",
                     help="configs[4]: sweep rank x tokens x top-k on the 4096->11008 projection; one JSON line per point")
