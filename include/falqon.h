@@ -133,8 +133,16 @@ int falqon_melded_forward(const falqon_layer *L, const void *X, falqon_dtype x_d
                           falqon_dtype y_dt, float *OA, float *amax_oa, float *s_x_out, void *ws,
                           size_t ws_bytes, falqon_stream stream);
 
+/* max |x| over `count` elements (bf16 or fp32) as an fp32 number in *amax_out (device [1]); ws: device scratch of at least
+ * FALQON_QUANTIZE_WS_BYTES.  The first half of Eq. quantize on its own, for callers that hold one shard of a tensor whose
+ * scale is shared (token-sharded data parallelism: the shards' maxima are combined before falqon_melded_forward_amax /
+ * falqon_melded_backward_amax cast each shard with the common scale). */
+int falqon_absmax(const void *src, falqon_dtype src_dt, int64_t count, float *amax_out, void *ws, size_t ws_bytes,
+                  falqon_stream stream);
+
 /* falqon_melded_forward for a caller that already knows amax_x = max |X| (device [1], fp32, exactly the maximum of the
- * absolute values of the tensor as stored): the kernel that produced X took it on the way out.  The cast is then a
+ * absolute values of the tensor as stored -- or of a larger tensor of which X is a shard, so that all shards are cast
+ * with one scale): the kernel that produced X took it on the way out.  The cast is then a
  * single pass -- no absmax reduction, no grid-wide barrier.  Everything else as falqon_melded_forward. */
 int falqon_melded_forward_amax(const falqon_layer *L, const void *X, falqon_dtype x_dt, const float *amax_x, int64_t T,
                                void *Y, falqon_dtype y_dt, float *OA, float *amax_oa, float *s_x_out, void *ws,

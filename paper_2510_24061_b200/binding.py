@@ -20,7 +20,7 @@ BF16, F32 = 0, 1
 PER_TENSOR, PER_ROW = 0, 1
 WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 
-EXPORTS = ["falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
+EXPORTS = ["falqon_absmax", "falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
            "falqon_svd_init_scratch_bytes", "falqon_svd_init", "falqon_tensor_ceiling", "falqon_tensor_ceiling_ctas",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_proxy_update_batched", "falqon_proxy_update_batched_adamw", "falqon_last_device_status", "falqon_launch_count",
@@ -67,6 +67,8 @@ lib.falqon_proxy_update_batched.argtypes = [C.POINTER(falqon_layer), C.c_int32, 
 lib.falqon_proxy_update_batched_adamw.restype = _i
 lib.falqon_proxy_update_batched_adamw.argtypes = [C.POINTER(falqon_layer), C.c_int32, C.POINTER(_p), C.POINTER(_p), C.POINTER(_p),
                                                   C.c_void_p, C.POINTER(_i64), C.POINTER(_p), C.POINTER(_p), C.POINTER(_sz), _p]
+lib.falqon_absmax.restype = _i
+lib.falqon_absmax.argtypes = [_p, _i, _i64, _p, _p, _sz, _p]
 lib.falqon_tensor_ceiling.restype = _i
 lib.falqon_tensor_ceiling.argtypes = [_i64, C.c_uint32, C.c_int32, _p, C.POINTER(C.c_double), _p, _sz, C.c_int32, _p]
 lib.falqon_tensor_ceiling_ctas.restype = _i
@@ -294,6 +296,16 @@ def proxy_update(layer: Layer, dB: torch.Tensor | None, lr: float, k: int, ws: t
     _check("falqon_proxy_update", lib.falqon_proxy_update(C.byref(layer.c), _ptr(dB), lr, k, _ptr(idx_out), _ptr(ws),
                                                           ws.numel(), _stream()))
     return idx_out
+
+
+def absmax(x: torch.Tensor, out: torch.Tensor | None = None, ws: torch.Tensor | None = None) -> torch.Tensor:
+    """falqon_absmax: max |x| of a contiguous bf16 / fp32 tensor as an fp32 device tensor [1]."""
+    assert x.is_contiguous()
+    dev = x.device
+    out = torch.empty(1, dtype=torch.float32, device=dev) if out is None else out
+    ws = torch.empty(8192, dtype=torch.uint8, device=dev) if ws is None else ws
+    _check("falqon_absmax", lib.falqon_absmax(_ptr(x), _dt(x), x.numel(), _ptr(out), _ptr(ws), ws.numel(), _stream()))
+    return out
 
 
 def tensor_ceiling(kblocks: int, seed: int = 1, random_fill: int = 1, sink: torch.Tensor | None = None,

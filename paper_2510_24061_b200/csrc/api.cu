@@ -195,6 +195,15 @@ int falqon_quantize(const void* src, falqon_dtype src_dt, int64_t rows, int64_t 
   return FALQON_OK;
 }
 
+int falqon_absmax(const void* src, falqon_dtype src_dt, int64_t count, float* amax_out, void* ws, size_t ws_bytes,
+                  falqon_stream stream) {
+  if (src == nullptr || amax_out == nullptr || count < 1 || count >= (1ll << 40) || !dtype_ok(src_dt) || !aligned16(src))
+    return FALQON_ERR_INVALID_ARG;
+  if (ws == nullptr || ws_bytes < FALQON_QUANTIZE_WS_BYTES || !aligned16(ws)) return FALQON_ERR_WORKSPACE;
+  FALQON_CUDA(launch_absmax_value(src, src_dt, count, static_cast<uint32_t*>(ws), amax_out, stream));
+  return FALQON_OK;
+}
+
 int falqon_workspace_init(void* ws, size_t ws_bytes, falqon_stream stream) {
   if (ws == nullptr || !aligned16(ws) || ws_bytes < kInitBytes) return FALQON_ERR_WORKSPACE;
   FALQON_CUDA(cudaMemsetAsync(ws, 0, kInitBytes, stream));

@@ -62,6 +62,9 @@ constexpr int kMaxAbsmaxParts = 148 * 8;   // upper bound of the absmax grid = n
 // Pass 1 of per-tensor absmax scaling: one partial max (fp32 bit pattern of |x|) per CTA into partial[0..*nparts).
 cudaError_t launch_absmax(const void* src, int src_dt, int64_t count, float premul, uint32_t* partial, int* nparts,
                           cudaStream_t stream);
+// max |x| of a tensor as an fp32 number in *amax_out (two small launches); partial: kMaxAbsmaxParts words of scratch.
+cudaError_t launch_absmax_value(const void* src, int src_dt, int64_t count, uint32_t* partial, float* amax_out,
+                                cudaStream_t stream);
 // Pass 2: cast with scale = fp8max / max(partial[0..nparts)) when nparts > 0, else with *scale_in.  Writes the
 // scale to scale_out / scale_out2 and the absmax to amax_out when non-null; sets *clear_word = 0 when non-null.
 cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, int fmt, float premul,

@@ -99,6 +99,18 @@ __global__ void __launch_bounds__(kThreads) absmax_kernel(const void* src, int64
   if (threadIdx.x == 0) partial[blockIdx.x] = m;
 }
 
+// ---- the max over the partials of pass 1, as a number of its own (for callers that combine it with the absmax of other
+// shards of the same tensor before the cast)
+__global__ void __launch_bounds__(kThreads) absmax_finalize_kernel(const uint32_t* partial, int nparts, float* amax_out) {
+  __shared__ uint32_t red[32];
+  pdl_trigger();
+  pdl_wait();
+  uint32_t mb = 0;
+  for (int i = threadIdx.x; i < nparts; i += kThreads) mb = max(mb, partial[i]);
+  mb = block_max_u32(mb, red);
+  if (threadIdx.x == 0) *amax_out = __uint_as_float(mb);
+}
+
 // ---- pass 2: cast with one scale for the whole tensor.  nparts > 0: the scale comes from the max of
 // the absmax partials; nparts == 0: *scale_in is used as given.
 struct CastOutputs {
@@ -514,6 +526,15 @@ cudaError_t launch_absmax(const void* src, int src_dt, int64_t count, float prem
   if (src_dt == kBF16)
     return launch_pdl(absmax_kernel<kBF16>, dim3(grid), dim3(kThreads), 0, stream, 1, src, count, premul, use_premul, partial);
   return launch_pdl(absmax_kernel<kF32>, dim3(grid), dim3(kThreads), 0, stream, 1, src, count, premul, use_premul, partial);
+}
+
+cudaError_t launch_absmax_value(const void* src, int src_dt, int64_t count, uint32_t* partial, float* amax_out,
+                                cudaStream_t stream) {
+  int nparts = 0;
+  cudaError_t e = launch_absmax(src, src_dt, count, 1.0f, partial, &nparts, stream);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(absmax_finalize_kernel, dim3(1), dim3(kThreads), 0, stream, 1, static_cast<const uint32_t*>(partial), nparts,
+                    amax_out);
 }
 
 cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, int fmt, float premul,

@@ -104,6 +104,12 @@ def test_bad_arguments_are_rejected_on_the_host(fq):
     assert call(two, 2, none2, 0.1, i2(1, 1), None, p2(fake + 0x300000, None), big2, None) == wsp
     twice = (fq.falqon_layer * 2)(layer, layer)
     assert call(twice, 2, none2, 0.1, i2(1, 1), None, ws2, big2, None) == inv                     # the same layer twice
+    # absmax
+    assert lib.falqon_absmax(None, 0, 64, fake, fake, 8192, None) == inv
+    assert lib.falqon_absmax(fake, 0, 0, fake, fake, 8192, None) == inv
+    assert lib.falqon_absmax(fake, 5, 64, fake, fake, 8192, None) == inv
+    assert lib.falqon_absmax(fake, 0, 64, None, fake, 8192, None) == inv
+    assert lib.falqon_absmax(fake, 0, 64, fake, fake, 64, None) == wsp
     # tensor ceiling
     assert lib.falqon_tensor_ceiling(0, 1, 0, None, None, None, 0, 0, None) == inv
     assert lib.falqon_tensor_ceiling((1 << 20) + 1, 1, 0, None, None, None, 0, 0, None) == inv

@@ -27,7 +27,7 @@ def _worker(rank, world, port, out):
 
 def test_replica_aggregation_two_gloo_ranks():
     world = 2
-    mgr = mp.Manager()
+    mgr = mp.get_context("spawn").Manager()
     out = mgr.dict()
     mp.spawn(_worker, args=(world, 29611, out), nprocs=world, join=True)
     for rank in range(world):
