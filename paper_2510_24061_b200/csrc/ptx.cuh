@@ -112,6 +112,19 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst_smem, const void* src,
                ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
+// The same copy with an L2 eviction hint: the lines it brings in are the first to go, so that a tensor that is read once
+// and then lives in shared memory does not push another kernel's dirty lines out of L2 while it streams in.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void bulk_load_1d_hint(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar,
+                                                  uint64_t policy) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+               ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+}
+
 // ---- 16-byte asynchronous copies global -> shared (through L2 only), tracked per thread in commit groups
 __device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");

@@ -328,6 +328,7 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
     const int64_t rem = bulk_elems - c * kChunkElems;
     return static_cast<int>(rem < kChunkElems ? rem : kChunkElems);
   };
+  const uint64_t evict_first = l2_policy_evict_first();
   auto issue = [&](int i) {   // one thread: fetch the CTA's i-th chunk into slot i mod nslots
     const int s = i % nslots;
     const int64_t c = chunk_of(i);
@@ -335,7 +336,12 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
     const uint32_t bar = smem_u32(&bars[s]);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier reads of the slot come first
     mbar_expect_tx(bar, bytes);
-    bulk_load_1d(smem_u32(stage + s * kChunkBytes), static_cast<const uint8_t*>(src) + c * kChunkBytes, bytes, bar);
+    // a chunk that will still be in the ring when the cast pass starts is read from memory exactly once: it need not
+    // stay in L2 (and should not displace what is there); an earlier chunk will be fetched again and should
+    if (i + nslots >= n_my)
+      bulk_load_1d_hint(smem_u32(stage + s * kChunkBytes), static_cast<const uint8_t*>(src) + c * kChunkBytes, bytes, bar, evict_first);
+    else
+      bulk_load_1d(smem_u32(stage + s * kChunkBytes), static_cast<const uint8_t*>(src) + c * kChunkBytes, bytes, bar);
   };
 
   // ---- pass 1: absmax
