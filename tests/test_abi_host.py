@@ -125,3 +125,17 @@ def test_launch_counts(fq):
     assert fq.launch_count("falqon_proxy_update", k=4) == 2 and fq.launch_count("falqon_proxy_update", k=0) == 1
     assert fq.launch_count("falqon_proxy_update_batched", k=4) == 2 and fq.launch_count("falqon_proxy_update_batched", k=0) == 1
     assert fq.launch_count("nope") == 0
+
+
+def test_headers_are_plain_c(tmp_path):
+    """The ABI headers must compile as C99 (and as C++) on their own: no torch or CUDA types in the signatures."""
+    import shutil
+    import subprocess
+    src = tmp_path / "use_headers.c"
+    src.write_text('#include "falqon.h"\n#include "falqon_chain.h"\n'
+                   "int main(void) { falqon_layer l; falqon_adamw h; (void)l; (void)h; return 0; }\n")
+    inc = os.path.join(ROOT, "include")
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-I", inc, str(src)], check=True)
+    subprocess.run(["g++", "-std=c++11", "-Wall", "-Wextra", "-Werror", "-fsyntax-only", "-x", "c++", "-I", inc, str(src)], check=True)
