@@ -139,3 +139,34 @@ def test_headers_are_plain_c(tmp_path):
         pytest.skip("no C compiler")
     subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-I", inc, str(src)], check=True)
     subprocess.run(["g++", "-std=c++11", "-Wall", "-Wextra", "-Werror", "-fsyntax-only", "-x", "c++", "-I", inc, str(src)], check=True)
+
+
+def test_a_c_program_links_and_calls_the_library(tmp_path, fq):
+    """A program written in C, built with gcc against the header and the shared library, calls the host-side entry
+    points (no device needed): proof that the boundary is a C ABI and not a Python extension."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    src = tmp_path / "client.c"
+    src.write_text(r'''
+#include <stdio.h>
+#include "falqon.h"
+int main(void) {
+  size_t ws = falqon_workspace_bytes(4096, 4096, 64, 4096);
+  size_t off = 0, size = 0;
+  int rc = falqon_workspace_region(4096, 4096, 64, 4096, FALQON_WS_GQ, &off, &size);
+  falqon_layer bad = {250, 256, 16, 0, 0, 0, FALQON_PER_TENSOR, 0};
+  int inv = falqon_proxy_update(&bad, 0, 0.1f, 1, 0, 0, 0, 0);
+  printf("%zu %d %zu %d %d\n", ws, rc, size, inv, falqon_launch_count("falqon_melded_backward", 0, 0, 0, 0, 0));
+  return 0;
+}
+''')
+    pkg = os.path.join(ROOT, "paper_2510_24061_b200")
+    exe = tmp_path / "client"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe),
+                    "-L", pkg, "-l:libfalqon.so", f"-Wl,-rpath,{pkg}"], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
+    assert int(out[0]) == fq.workspace_bytes(4096, 4096, 64, 4096) and int(out[0]) > 4096 * 4096
+    assert int(out[1]) == fq.OK and int(out[2]) == 4096 * 4096
+    assert int(out[3]) == fq.ERR_INVALID_ARG and int(out[4]) == 3
