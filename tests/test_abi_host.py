@@ -170,3 +170,20 @@ int main(void) {
     assert int(out[0]) == fq.workspace_bytes(4096, 4096, 64, 4096) and int(out[0]) > 4096 * 4096
     assert int(out[1]) == fq.OK and int(out[2]) == 4096 * 4096
     assert int(out[3]) == fq.ERR_INVALID_ARG and int(out[4]) == 3
+
+
+def test_the_package_refuses_to_load_without_its_library(tmp_path):
+    """No CPU fallback: a copy of the Python package without libfalqon.so must fail at import, loudly."""
+    import shutil
+    import subprocess
+    import sys
+    pkg = tmp_path / "paper_2510_24061_b200"
+    shutil.copytree(os.path.join(ROOT, "paper_2510_24061_b200"), pkg,
+                    ignore=shutil.ignore_patterns("*.so", "build", "__pycache__", "csrc"))
+    res = subprocess.run([sys.executable, "-c", "import paper_2510_24061_b200.binding"], cwd=tmp_path, capture_output=True,
+                         text=True, env={**os.environ, "PYTHONPATH": str(tmp_path)})
+    assert res.returncode != 0
+    assert "ImportError" in res.stderr and "libfalqon.so is missing" in res.stderr and "no non-CUDA fallback" in res.stderr
+    res = subprocess.run([sys.executable, "-c", "import paper_2510_24061_b200.stack"], cwd=tmp_path, capture_output=True,
+                         text=True, env={**os.environ, "PYTHONPATH": str(tmp_path)})
+    assert res.returncode != 0 and "ImportError" in res.stderr
