@@ -187,3 +187,33 @@ def test_the_package_refuses_to_load_without_its_library(tmp_path):
     res = subprocess.run([sys.executable, "-c", "import paper_2510_24061_b200.stack"], cwd=tmp_path, capture_output=True,
                          text=True, env={**os.environ, "PYTHONPATH": str(tmp_path)})
     assert res.returncode != 0 and "ImportError" in res.stderr
+
+
+def test_the_product_path_never_touches_the_oracle():
+    """The oracle is test infrastructure: nothing in the package may import or execute it, and bench.py may do so only
+    inside the function that times it (the cpu_baseline and reference legs)."""
+    import ast
+    pkg = os.path.join(ROOT, "paper_2510_24061_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for name in files:
+            if name.endswith((".py", ".cu", ".cuh", ".h", ".cpp")):
+                text = open(os.path.join(dirpath, name)).read()
+                if name.endswith(".py"):
+                    for node in ast.walk(ast.parse(text)):
+                        mods = []
+                        if isinstance(node, ast.Import):
+                            mods = [a.name for a in node.names]
+                        elif isinstance(node, ast.ImportFrom):
+                            mods = [node.module or ""]
+                        assert not any(mod.split(".")[0] == "oracle" for mod in mods), f"{name} imports the oracle"
+                else:
+                    assert "oracle/" not in text and "falqon_oracle" not in text, f"{name} refers to the oracle"
+    tree = ast.parse(open(os.path.join(ROOT, "bench.py")).read())
+    importers = set()
+    for fn in [n for n in ast.walk(tree) if isinstance(n, ast.FunctionDef)]:
+        for node in ast.walk(fn):
+            if isinstance(node, ast.ImportFrom) and (node.module or "").split(".")[0] == "oracle":
+                importers.add(fn.name)
+    top_level = [n for n in tree.body if isinstance(n, (ast.Import, ast.ImportFrom))]
+    assert not any(getattr(n, "module", None) == "oracle" or any(a.name.startswith("oracle") for a in n.names) for n in top_level)
+    assert importers == {"time_oracle_sample"}, importers
