@@ -571,6 +571,20 @@ def main():
     records = fq.profile_stop(n_records)
     status = fq.last_device_status()
 
+    # ---- what one proxy update does to a backbone (bookkeeping outside every timed region, first projection):
+    # codes that changed, and codes sitting at the largest finite magnitude (saturation of the requantized rows)
+    L0 = layers[0]
+    before = L0["layer"].wq[: L0["m"]].clone()
+    _, OA0, amax0, _ = fq.melded_forward(L0["layer"], L0["X"], ws=L0["ws"], out=L0["out_f"])
+    _, dB0, _ = fq.melded_backward(L0["layer"], L0["dY"], OA0, amax0, ws=L0["ws"], out=L0["out_b"])
+    fq.proxy_update(L0["layer"], dB0, lr, k, ws=L0["ws"], idx_out=L0["idx"])
+    after = L0["layer"].wq[: L0["m"]]
+    rows = L0["idx"][:k].long()
+    proxy_effect = {"projection": L0["name"], "rows_merged": int(k),
+                    "changed_codes": int((before != after).sum().item()),
+                    "changed_codes_outside_merged_rows": int((before != after).sum().item() - (before[rows] != after[rows]).sum().item()),
+                    "saturated_codes_in_merged_rows": int(((after[rows] & 0x7F) == 0x7E).sum().item())}
+
     # ---- roofline of the dominant kernel: the tcgen05 FP8 GEMM in its two tensor-bound roles
     peaks = measured_peaks()
     per_rec = 3 * len(layers)
@@ -671,6 +685,7 @@ def main():
         "gemm_db_ms_per_step": t_db / args.steps,
         "quantize": {"bound": "hbm", "achieved_gbs": quant_gbs, "peak_gbs": peaks["hbm"], "frac": quant_gbs / peaks["hbm"],
                      "bytes_per_elt": 5, "note": "absmax pass + cast pass of X and dY, algorithmic bytes"},
+        "proxy_update_effect": proxy_effect,
         "device_status": status,
     }
     print(json.dumps(out))
