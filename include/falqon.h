@@ -288,6 +288,12 @@ int falqon_proxy_update_exact(const falqon_layer *L, const float *dB, float lr, 
  * undefined) or FALQON_ERR_CUDA (the synchronize itself failed). */
 int falqon_last_device_status(falqon_stream stream);
 
+/* Self-test of the bounded device-side waits: launches one small CTA that waits on a barrier nobody ever signals.  The
+ * wait gives up after limit_ms (1..1000) milliseconds, records FALQON_ERR_TIMEOUT in the device status word and the
+ * kernel returns; nothing traps, and every later call works as usual.  falqon_last_device_status then returns
+ * FALQON_ERR_TIMEOUT once.  (Every wait inside the library's kernels uses the same helper, with a limit of 2 s.) */
+int falqon_selftest_wait_timeout(uint32_t limit_ms, falqon_stream stream);
+
 /* Measurement aid (no counterpart in the paper): the ceiling of this GPU's FP8 tensor pipe.  One launch in which every
  * SM pair issues kblocks x 4 of the 256 x 256 x 32 E4M3 MMAs that the forward and input-gradient products issue, on
  * operand tiles that stay in shared memory (random_fill 0: zeros; 1: uniformly random codes drawn from `seed`; 2: the

@@ -20,7 +20,7 @@ BF16, F32 = 0, 1
 PER_TENSOR, PER_ROW = 0, 1
 WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 
-EXPORTS = ["falqon_absmax", "falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
+EXPORTS = ["falqon_absmax", "falqon_selftest_wait_timeout", "falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
            "falqon_svd_init_scratch_bytes", "falqon_svd_init", "falqon_tensor_ceiling", "falqon_tensor_ceiling_ctas",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_proxy_update_batched", "falqon_proxy_update_batched_adamw", "falqon_last_device_status", "falqon_launch_count",
@@ -67,6 +67,8 @@ lib.falqon_proxy_update_batched.argtypes = [C.POINTER(falqon_layer), C.c_int32, 
 lib.falqon_proxy_update_batched_adamw.restype = _i
 lib.falqon_proxy_update_batched_adamw.argtypes = [C.POINTER(falqon_layer), C.c_int32, C.POINTER(_p), C.POINTER(_p), C.POINTER(_p),
                                                   C.c_void_p, C.POINTER(_i64), C.POINTER(_p), C.POINTER(_p), C.POINTER(_sz), _p]
+lib.falqon_selftest_wait_timeout.restype = _i
+lib.falqon_selftest_wait_timeout.argtypes = [C.c_uint32, _p]
 lib.falqon_absmax.restype = _i
 lib.falqon_absmax.argtypes = [_p, _i, _i64, _p, _p, _sz, _p]
 lib.falqon_tensor_ceiling.restype = _i

@@ -559,6 +559,14 @@ int falqon_tensor_ceiling(int64_t kblocks, uint32_t seed, int32_t random_fill, f
   return FALQON_OK;
 }
 
+int falqon_selftest_wait_timeout(uint32_t limit_ms, falqon_stream stream) {
+  if (limit_ms < 1 || limit_ms > 1000) return FALQON_ERR_INVALID_ARG;
+  int* status = status_ptr();
+  if (status == nullptr) return FALQON_ERR_CUDA;
+  FALQON_CUDA(launch_wait_timeout_selftest(static_cast<uint64_t>(limit_ms) * 1000000ull, status, stream));
+  return FALQON_OK;
+}
+
 int falqon_last_device_status(falqon_stream stream) {
   if (cudaStreamSynchronize(stream) != cudaSuccess) return FALQON_ERR_CUDA;
   int* p = status_ptr();

@@ -208,4 +208,7 @@ double tensor_ceiling_flops(int kblocks);
 cudaError_t launch_tensor_ceiling(int kblocks, uint32_t seed, int random_fill, float* sink, int* status, const void* load_src,
                                   size_t load_bytes, int bytes_per_kblock, cudaStream_t stream);
 
+// One CTA waits limit_ns on a barrier nobody signals, records the timeout in *status and returns (self-test of the bounded waits).
+cudaError_t launch_wait_timeout_selftest(uint64_t limit_ns, int* status, cudaStream_t stream);
+
 }  // namespace falqon

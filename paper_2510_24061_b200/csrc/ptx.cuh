@@ -77,7 +77,7 @@ __device__ __forceinline__ bool elect_one() {
 // lost signal can never hang the device.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s; a healthy kernel waits microseconds
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+__device__ __forceinline__ bool mbar_wait_for(uint32_t bar, uint32_t parity, int* status, uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (;;) {
@@ -85,11 +85,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* st
     for (int i = 0; i < 128; ++i) {
       if (mbar_try_wait(bar, parity)) return true;
     }
-    if (global_timer_ns() - t0 > kWaitLimitNs) {
+    if (global_timer_ns() - t0 > limit_ns) {
       atomicExch(status, kStatusTimeout);
       return false;
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+  return mbar_wait_for(bar, parity, status, kWaitLimitNs);
 }
 
 // The same wait executed by a whole converged warp; the outcome is made warp-uniform.

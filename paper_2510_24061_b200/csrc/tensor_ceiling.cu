@@ -170,7 +170,24 @@ __global__ void __launch_bounds__(kCeilThreads, 1) tensor_ceiling_kernel(int kbl
   }
 }
 
+// A self-test of the bounded waits, not a measurement: one CTA waits on a barrier that nobody ever arrives on.  The wait
+// gives up after limit_ns, records the timeout in the status word and the kernel returns; the context stays usable.
+__global__ void __launch_bounds__(32) wait_timeout_selftest_kernel(uint64_t limit_ns, int* status) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    mbar_fence_init();
+  }
+  __syncwarp();
+  mbar_wait_for(smem_u32(&bar), 0u, status, limit_ns);
+}
+
 }  // namespace
+
+cudaError_t launch_wait_timeout_selftest(uint64_t limit_ns, int* status, cudaStream_t stream) {
+  wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(limit_ns, status);
+  return cudaGetLastError();
+}
 
 int tensor_ceiling_ctas() { return (sm_count() / 2) * 2; }
 

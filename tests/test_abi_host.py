@@ -104,6 +104,8 @@ def test_bad_arguments_are_rejected_on_the_host(fq):
     assert call(two, 2, none2, 0.1, i2(1, 1), None, p2(fake + 0x300000, None), big2, None) == wsp
     twice = (fq.falqon_layer * 2)(layer, layer)
     assert call(twice, 2, none2, 0.1, i2(1, 1), None, ws2, big2, None) == inv                     # the same layer twice
+    # bounded-wait self-test: the limit must be 1..1000 ms
+    assert lib.falqon_selftest_wait_timeout(0, None) == inv and lib.falqon_selftest_wait_timeout(1001, None) == inv
     # absmax
     assert lib.falqon_absmax(None, 0, 64, fake, fake, 8192, None) == inv
     assert lib.falqon_absmax(fake, 0, 0, fake, fake, 8192, None) == inv
