@@ -37,3 +37,17 @@ def test_activation_outlier_channels():
     assert cols == [0, 128, 256, 384, 512, 640, 768, 896]
     ratio = x[:, cols].std() / x[:, [c + 1 for c in cols]].std()
     assert 14 < ratio < 18
+
+
+def test_projection_shapes_give_the_papers_parameter_counts():
+    """Rank 64 on all seven projections of every block: the DeltaBuffers (B only) of the 7B shapes hold 87.0 M values, A
+    and B together 159.9 M (the paper's table rounds these to 80 M and 160 M), and 250.3 M for the 13B shapes (250 M)."""
+    from paper_2510_24061_b200 import synth
+    r = 64
+    b7 = 32 * sum(m * r for _, n, m in synth.LLAMA_7B_LINEARS)
+    ab7 = 32 * sum((m + n) * r for _, n, m in synth.LLAMA_7B_LINEARS)
+    ab13 = 40 * sum((m + n) * r for _, n, m in synth.LLAMA_13B_LINEARS)
+    assert round(b7 / 1e6, 1) == 87.0 and round(ab7 / 1e6, 1) == 159.9 and round(ab13 / 1e6, 1) == 250.3
+    assert abs(ab7 / 160e6 - 1) < 0.01 and abs(ab13 / 250e6 - 1) < 0.01
+    # backbone bytes of the 7B stack in FP8: 6.48 GB
+    assert round(32 * sum(m * n for _, n, m in synth.LLAMA_7B_LINEARS) / 1e9, 2) == 6.48
