@@ -683,7 +683,7 @@ def main():
         "frac_of_fp8_peak": {"of_measured_sustained_x2": value / world / peak, "of_nominal_4500": value / world / 4500.0},
         "stage_ms_per_step": {k_: round(v, 4) for k_, v in sorted(breakdown.items())},
         "gemm_db_ms_per_step": t_db / args.steps,
-        "quantize": {"bound": "hbm", "achieved_gbs": quant_gbs, "peak_gbs": peaks["hbm"], "frac": quant_gbs / peaks["hbm"],
+        "quantize": {"bound": "hbm", "achieved_gbs": quant_gbs, "peak_gbs": peaks["hbm"], "frac": quant_gbs / peaks["hbm"], "frac_of_nominal_8000": quant_gbs / 8000.0,
                      "bytes_per_elt": 5, "note": "absmax pass + cast pass of X and dY, algorithmic bytes"},
         "proxy_update_effect": proxy_effect,
         "device_status": status,
