@@ -444,6 +444,9 @@ def main():
                     help="measure the FP8 tensor pipe alone (MMA issue on shared-memory operands) for SECONDS per fill; one JSON line")
     ap.add_argument("--no-tensor-ceiling", action="store_true",
                     help="skip the 3 s measurement of the FP8 tensor pipe alone that the default line reports beside the roofline")
+    ap.add_argument("--eager", action="store_true",
+                    help="time the step as one library call after another instead of as replays of one CUDA graph of the "
+                         "step (the library's calls only enqueue kernels, so a step can be captured; replays are about 2 %% faster)")
     ap.add_argument("--proxy-per-layer", action="store_true",
                     help="run one falqon_proxy_update per projection instead of one falqon_proxy_update_batched per step")
     ap.add_argument("--only", default=None, help="profiling aid: restrict the workload to one projection (q,k,v,o,gate,up,down)")
@@ -466,7 +469,8 @@ def main():
                 "l2": "inputs larger than L2 (%.2f GB of inputs and outputs touched per step)" %
                       (sum(2.0 * T * (n + m) * 2 for _, n, m in linears) / 1e9),
                 "parallelism": f"replicas x{world}",
-                "proxy_update": "one call per projection" if args.proxy_per_layer else "one batched call per step"}
+                "proxy_update": "one call per projection" if args.proxy_per_layer else "one batched call per step",
+                "launch": "one library call after another" if args.eager else "replays of one CUDA graph of the step"}
 
     if args.tensor_ceiling > 0:
         if rank == 0:
@@ -526,13 +530,22 @@ def main():
     for _ in range(max(args.warmup, 3)):
         run_step(fq, layers, lr, k, batch)
     barrier()
+    one_step = lambda: run_step(fq, layers, lr, k, batch)
+    if not args.eager:
+        step_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(step_graph):
+            run_step(fq, layers, lr, k, batch)
+        one_step = step_graph.replay
+        for _ in range(3):
+            one_step()
+        barrier()
     sampler = ClockSampler(local_rank)
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     ev0.record()
     for _ in range(args.steps):
-        run_step(fq, layers, lr, k, batch)
+        one_step()
     ev1.record()
     barrier()
     ms_total = max_over_ranks(ev0.elapsed_time(ev1))
