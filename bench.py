@@ -374,12 +374,22 @@ def run_stack(args):
     for _ in range(warmup):
         stack.step(h0, G)
     torch.cuda.synchronize()
+    one_step = lambda: stack.step(h0, G)
+    use_graph = not args.eager and not args.stack_adamw     # AdamW's step count is a call argument: not captured
+    if use_graph:
+        step_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(step_graph):
+            stack.step(h0, G)
+        one_step = step_graph.replay
+        for _ in range(2):
+            one_step()
+        torch.cuda.synchronize()
     sampler = ClockSampler(0)
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(steps):
-        stack.step(h0, G)
+        one_step()
     e1.record()
     torch.cuda.synchronize()
     clocks = sampler.stop()
@@ -402,7 +412,8 @@ def run_stack(args):
                    "tokens": T, "rank": r, "topk": k, "matrices": 7 * n_layers, "tflop_per_step": flops / 1e12,
                    "l2": "working set far larger than L2 (every step touches the whole stack)", "parallelism": "single GPU",
                    "optimizer": "AdamW on the DeltaBuffers" if args.stack_adamw else "SGD on the DeltaBuffers",
-                   "proxy_update": "one call per projection" if args.proxy_per_layer else "one batched call per block"},
+                   "proxy_update": "one call per projection" if args.proxy_per_layer else "one batched call per block",
+                   "launch": "replays of one CUDA graph of the step" if use_graph else "one library call after another"},
         "clocks": clocks, "gpu_launches": stack.launches_per_step() * steps,
         "frac_of_fp8_peak": {"of_measured_sustained_x2": tf / (peaks["bf16_sustained"] * FP8_OVER_BF16),
                              "of_nominal_4500": tf / 4500.0},
