@@ -238,17 +238,39 @@ def run_sweep(args):
     topks = [0, 64, 512, 4096]
     iters = 10
 
-    def timed(fn):
+    def timed(fn, graph=True):
+        """ms per call, calls back to back on one stream: as replays of a CUDA graph of the call (forward and backward:
+        three to five kernels per call, timed without their launch gaps) or, for the proxy update and with --eager, as plain
+        calls (its two kernels overlap from one call to the next under programmatic stream serialization, which separate
+        graph launches do not allow: 24 against 43 us at top-64).  A first batch of calls sizes the run: at least 10 calls
+        and about 20 ms, and the timed batch follows the warm one without a pause -- a call of 35 us timed ten times after
+        an idle gap measures the clock ramp of the GPU, not the call."""
         for _ in range(3):
             fn()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        run = fn
+        if graph and not args.eager:
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
+            run = g.replay
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
         torch.cuda.synchronize()
         e0.record()
         for _ in range(iters):
-            fn()
+            run()
         e1.record()
+        e1.synchronize()
+        est = max(e0.elapsed_time(e1) / iters, 1e-3)
+        n_timed = max(iters, min(2000, int(20.0 / est)))
+        for _ in range(n_timed):          # warm batch, same length, no pause before the timed one
+            run()
+        e1.record()
+        for _ in range(n_timed):
+            run()
+        e2.record()
         torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / iters
+        return e1.elapsed_time(e2) / n_timed
 
     W = synth.backbone(0, 4, m, n, dev)
     for r in ranks:
@@ -278,11 +300,11 @@ def run_sweep(args):
         ws = layer.workspace(1)
         for k in topks:
             idx = torch.empty(max(k, 1), dtype=torch.int32, device=dev)
-            t_p = timed(lambda: fq.proxy_update(layer, dB, 2e-4, k, ws=ws, idx_out=idx if k > 0 else None))
+            t_p = timed(lambda: fq.proxy_update(layer, dB, 2e-4, k, ws=ws, idx_out=idx if k > 0 else None), graph=False)
             t_x = None
             if k > 0:   # the same update with the correctly rounded merge on the tensor cores
                 scratch = torch.empty(int(fq.lib.falqon_exact_merge_scratch_bytes(m, n, r)), dtype=torch.uint8, device=dev)
-                t_x = timed(lambda: fq.proxy_update_exact(layer, dB, 2e-4, k, ws=ws, idx_out=idx, scratch=scratch, want_count=False))
+                t_x = timed(lambda: fq.proxy_update_exact(layer, dB, 2e-4, k, ws=ws, idx_out=idx, scratch=scratch, want_count=False), graph=False)
                 del scratch
             bytes_p = 12.0 * m * r + 4.0 * m + k * (2.0 * n + 8.0 * r) + r * n   # optimizer+score pass, merged rows, A~ once
             fma = float(k) * n * r
