@@ -560,6 +560,8 @@ def main():
 
     batch = None if args.proxy_per_layer else make_proxy_batch(fq, layers, k)
     # ---- device-resident timing: EXACTLY --steps steps between two events, nothing else in the stream
+    sampler = ClockSampler(local_rank)
+    sampler.start()           # before the warm-up: starting it takes long enough for an idle GPU to drop its clocks
     for _ in range(max(args.warmup, 3)):
         run_step(fq, layers, lr, k, batch)
     barrier()
@@ -569,11 +571,8 @@ def main():
         with torch.cuda.graph(step_graph):
             run_step(fq, layers, lr, k, batch)
         one_step = step_graph.replay
-        for _ in range(3):
-            one_step()
-        barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
+    for _ in range(max(args.warmup, 3)):      # the W warm-up steps proper, in the form that is timed
+        one_step()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     ev0.record()
