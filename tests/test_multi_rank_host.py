@@ -41,3 +41,21 @@ def test_single_process_aggregation_is_identity():
     import bench
     ms, tflops = bench.aggregate_over_ranks(4.0, 8.0e12)
     assert ms == 4.0 and abs(tflops - 8.0e12 / 4.0e-3 / 1e12) < 1e-9
+
+
+def test_reference_arm_prints_one_json_line_with_the_agreed_keys():
+    """`bench.py --impl reference` (the CPU oracle timed on a bounded sample) on a tiny sample: one JSON line, same metric
+    and unit as the CUDA arm, the keys the measurement contract names."""
+    import json
+    import subprocess
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "0",
+                          "--oracle-tokens", "32"], capture_output=True, text=True, cwd=ROOT, timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["unit"] == "TFLOP/s" and d["higher_is_better"] is True and d["vs_baseline"] is None
+    assert d["metric"].startswith("melded FP8-LoRA layer fwd+bwd TFLOP/s") and d["value"] > 0 and d["n_gpus"] == 1
+    assert d["config"]["workload"].startswith("configs[1]") and "model" not in d["config"]
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1 and d["cpu_baseline"]["value"] == d["value"]
+    assert d["e2e"] == {"value": d["value"], "unit": d["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
