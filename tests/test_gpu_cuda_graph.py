@@ -66,3 +66,36 @@ def test_a_captured_step_replays_bit_for_bit():
             assert torch.equal(a["out_f"][0], b["out_f"][0]) and torch.equal(a["out_b"][0], b["out_b"][0])
             assert torch.equal(a["out_b"][1].view(torch.int32), b["out_b"][1].view(torch.int32))
     assert fq.last_device_status() == 0
+
+
+def test_the_benchmarks_graph_replay_equals_call_by_call_at_full_size():
+    """configs[1] exactly as bench.py runs it (the seven 7B projections, 4096 tokens, rank 64, top-256, batched proxy
+    update): two replays of the captured step against two steps run call by call on a twin workload, bit for bit."""
+    import os
+    import sys
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import bench
+    from paper_2510_24061_b200 import binding as fq
+    c = synth.config1()
+    T, r, k, lr = c["T"], c["r"], c["k"], c["lr"]
+    sets = []
+    for _ in range(2):
+        layers = bench.build_workload(fq, torch.device(DEV), c["seed"], T, r, k, c["linears"], c["outlier_frac"])
+        sets.append((layers, bench.make_proxy_batch(fq, layers, k)))
+    (Lg, bg), (Le, be) = sets
+    bench.run_step(fq, Lg, lr, k, bg)          # first use of every kernel happens outside the capture
+    bench.run_step(fq, Le, lr, k, be)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        bench.run_step(fq, Lg, lr, k, bg)
+    for step in range(2):
+        graph.replay()
+        bench.run_step(fq, Le, lr, k, be)
+        torch.cuda.synchronize()
+        for a, b in zip(Lg, Le):
+            assert torch.equal(a["layer"].wq, b["layer"].wq), f"{a['name']} step {step}: backbone"
+            assert torch.equal(a["layer"].dbuf.view(torch.int32), b["layer"].dbuf.view(torch.int32)), f"{a['name']}: DeltaBuffer"
+            assert torch.equal(a["out_f"][0], b["out_f"][0]) and torch.equal(a["out_b"][0], b["out_b"][0]), f"{a['name']}: Y / dX"
+            assert torch.equal(a["idx"], b["idx"]), f"{a['name']}: selected rows"
+    assert fq.last_device_status() == 0
