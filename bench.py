@@ -128,13 +128,14 @@ def aggregate_over_ranks(ms_local: float, flops_per_rank: float, dist=None, devi
     return ms, world * flops_per_rank / (ms * 1e-3) / 1e12
 
 
-def build_workload(fq, device, seed, T, r, k, linears, outlier_frac, per_row=False, heavy_tailed=False):
+def build_workload(fq, device, seed, T, r, k, linears, outlier_frac, per_row=False, heavy_tailed=False, flags=0):
     layers = []
     for idx, (name, n, m) in enumerate(linears):
         W = synth.backbone(seed, idx, m, n, device, heavy_tailed=heavy_tailed)
         A = synth.adapter_a(seed, idx, r, n, device)
         B = synth.adapter_b(seed, idx, m, r, device)
         layer = fq.setup_layer(W, A, B, 1.0, per_row=per_row)
+        layer.flags = flags
         del W
         X = synth.activations(seed, idx, T, n, round(outlier_frac * n), device)
         dY = synth.out_grad(seed, idx, 0, T, m, device)
@@ -482,6 +483,9 @@ def main():
                          "step (the library's calls only enqueue kernels, so a step can be captured; replays are about 2 %% faster)")
     ap.add_argument("--proxy-per-layer", action="store_true",
                     help="run one falqon_proxy_update per projection instead of one falqon_proxy_update_batched per step")
+    ap.add_argument("--fused", action="store_true",
+                    help="cast X and dY inside the producers of the tensor-core products (FALQON_LAYER_FUSED_CAST) instead of "
+                         "in cast kernels of their own")
     ap.add_argument("--only", default=None, help="profiling aid: restrict the workload to one projection (q,k,v,o,gate,up,down)")
     args = ap.parse_args()
 
@@ -547,7 +551,8 @@ def main():
     from paper_2510_24061_b200 import binding as fq
 
     layers = build_workload(fq, device, cfg["seed"] + rank, T, r, k, linears, cfg["outlier_frac"],
-                            per_row=cfg.get("per_row", False), heavy_tailed=cfg.get("heavy_tailed", False))
+                            per_row=cfg.get("per_row", False), heavy_tailed=cfg.get("heavy_tailed", False),
+                            flags=fq.LAYER_FUSED_CAST if args.fused else 0)
     torch.cuda.synchronize()
 
     def barrier():
@@ -689,7 +694,8 @@ def main():
     ms_e2e = max_over_ranks(ev0.elapsed_time(ev1)) / e2e_steps
     e2e_value = world * flops_step / (ms_e2e * 1e-3) / 1e12
 
-    launches_per_step = sum(fq.launch_count("falqon_melded_forward") + fq.launch_count("falqon_melded_backward") +
+    suffix = ":fused" if args.fused else ""
+    launches_per_step = sum(fq.launch_count("falqon_melded_forward" + suffix) + fq.launch_count("falqon_melded_backward" + suffix) +
                             (fq.launch_count("falqon_proxy_update", k=k) if batch is None else 0) for L in layers)
     if batch is not None:
         launches_per_step += fq.launch_count("falqon_proxy_update_batched", k=k) * ((len(layers) + 7) // 8)

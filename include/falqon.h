@@ -73,8 +73,22 @@ typedef struct {
                      s_w[i] before its E5M2 cast (the row scales lie on dX's contraction axis) and
                      multiplies row i of dB back; the merge weighs DeltaBuffer row i by
                      s_w[i] / s_w[m].  Scales stay frozen after set-up in both modes.          */
-  int32_t reserved_;
+  int32_t flags;  /* bit set of falqon_layer_flag; 0 = none                              */
 } falqon_layer;
+
+/* Per-layer options (falqon_layer.flags).
+ *  FALQON_LAYER_FUSED_CAST  The casts of X (forward) and dY (backward) run inside the producers of the tensor-core
+ *      products instead of as passes of their own: the product kernels fetch the bf16 tensor tile by tile, scale and
+ *      round it in shared memory, and multiply the codes from there (Alg. 2 lines 5-6 and the cast of Alg. 3's incoming
+ *      gradient, Eq. quantize, fused with Eq. o_split's product).  x~ is then never written to memory; g~ is written once,
+ *      by the input-gradient product, because the adapter-gradient product reads it as a tensor.  The codes, the
+ *      scales and therefore every result are bit for bit those of the un-fused calls.  Only the absmax reduction (one
+ *      read of the tensor) remains as a separate pass, and not even that in the *_amax calls.  Applies where the fused
+ *      kernel can run -- bf16 inputs; forward: (m + r) a multiple of 16; backward: per-tensor s_w and dX requested -- and
+ *      silently falls back to the un-fused path elsewhere.  FALQON_WS_XQ holds no codes after a fused forward.
+ *  FALQON_LAYER_EMIT_XQ     With FALQON_LAYER_FUSED_CAST: the fused forward also writes x~ to FALQON_WS_XQ (one extra
+ *      write of T*n bytes), for layers that share it through falqon_melded_forward_codes. */
+typedef enum { FALQON_LAYER_FUSED_CAST = 1, FALQON_LAYER_EMIT_XQ = 2 } falqon_layer_flag;
 
 /* Names of the regions inside the workspace that hold staged intermediates of the last call
  * (readable by a caller that wants to inspect or reuse them; see falqon_workspace_region). */
@@ -175,6 +189,21 @@ int falqon_melded_backward(const falqon_layer *L, const void *dY, falqon_dtype d
 int falqon_melded_backward_amax(const falqon_layer *L, const void *dY, falqon_dtype dy_dt, const float *amax_dy, int64_t T,
                                 const float *OA, const float *amax_oa, void *dX, falqon_dtype dx_dt, float *dB,
                                 float *s_g_out, void *ws, size_t ws_bytes, falqon_stream stream);
+
+/* Debug hook of the fused casts ("identical FP8 operands"): falqon_melded_forward / _backward for a layer with
+ * FALQON_LAYER_FUSED_CAST, in which the product's tiles of output-column block n_block (256 columns each; forward:
+ * columns of [Y | O_A], backward: columns of dX) also write the codes they staged in shared memory to FALQON_WS_XQ /
+ * FALQON_WS_GQ.  Every column block converts the whole A operand for itself, so running this for each n_block and
+ * comparing the region with falqon_quantize (or the oracle's cast) checks every staged tile.  amax (device [1],
+ * nullable): max |X| / max |dY| if already known.  Returns FALQON_ERR_UNSUPPORTED where the fused kernel does not
+ * apply (see FALQON_LAYER_FUSED_CAST), FALQON_ERR_INVALID_ARG for an n_block outside the product.  In the backward
+ * the adapter gradient is computed from the codes this block wrote. */
+int falqon_melded_forward_dump(const falqon_layer *L, const void *X, falqon_dtype x_dt, const float *amax_x, int64_t T,
+                               void *Y, falqon_dtype y_dt, float *OA, float *amax_oa, float *s_x_out, int32_t n_block,
+                               void *ws, size_t ws_bytes, falqon_stream stream);
+int falqon_melded_backward_dump(const falqon_layer *L, const void *dY, falqon_dtype dy_dt, const float *amax_dy, int64_t T,
+                                const float *OA, const float *amax_oa, void *dX, falqon_dtype dx_dt, float *dB,
+                                float *s_g_out, int32_t n_block, void *ws, size_t ws_bytes, falqon_stream stream);
 
 /* Row-wise proxy update (Alg. 3 lines 4-6; Eq. update):
  *   DeltaBuffer <- fma(-lr, dB, DeltaBuffer)          (plain SGD form; skipped when dB is NULL, so a
@@ -337,7 +366,8 @@ typedef enum {
 int falqon_profile_start(int max_records, unsigned stage_mask);
 int falqon_profile_stop(float *ms_out, int *stage_out, int capacity);
 
-/* Host, pure.  Number of kernels the named call launches for this shape (for launch accounting). */
+/* Host, pure.  Number of kernels the named call launches for this shape (for launch accounting).  The forward and
+ * backward of a layer with FALQON_LAYER_FUSED_CAST are named "falqon_melded_forward:fused" / "falqon_melded_backward:fused". */
 int falqon_launch_count(const char *entry_point, int64_t m, int64_t n, int64_t r, int64_t T, int64_t k);
 
 #ifdef __cplusplus

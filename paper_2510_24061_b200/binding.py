@@ -18,10 +18,12 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, 
 E4M3, E5M2 = 0, 1
 BF16, F32 = 0, 1
 PER_TENSOR, PER_ROW = 0, 1
+LAYER_FUSED_CAST, LAYER_EMIT_XQ = 1, 2
 WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 
 EXPORTS = ["falqon_absmax", "falqon_selftest_wait_timeout", "falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
-           "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
+           "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax",
+           "falqon_melded_forward_dump", "falqon_melded_backward_dump", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
            "falqon_svd_init_scratch_bytes", "falqon_svd_init", "falqon_tensor_ceiling", "falqon_tensor_ceiling_ctas",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_proxy_update_batched", "falqon_proxy_update_batched_adamw", "falqon_last_device_status", "falqon_launch_count",
            "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static", "falqon_workspace_init", "falqon_proxy_update_adamw"]
@@ -37,7 +39,7 @@ lib = C.CDLL(LIB_PATH)
 class falqon_layer(C.Structure):
     _fields_ = [("m", C.c_int64), ("n", C.c_int64), ("r", C.c_int64),
                 ("wq", C.c_void_p), ("s_w", C.c_void_p), ("dbuf", C.c_void_p),
-                ("gran", C.c_int32), ("reserved_", C.c_int32)]
+                ("gran", C.c_int32), ("flags", C.c_int32)]
 
 
 _i64, _sz, _p, _f, _i = C.c_int64, C.c_size_t, C.c_void_p, C.c_float, C.c_int
@@ -55,6 +57,10 @@ lib.falqon_melded_forward_amax.restype = _i
 lib.falqon_melded_forward_amax.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _i, _p, _p, _p, _p, _sz, _p]
 lib.falqon_melded_backward_amax.restype = _i
 lib.falqon_melded_backward_amax.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _p, _p, _i, _p, _p, _p, _sz, _p]
+lib.falqon_melded_forward_dump.restype = _i
+lib.falqon_melded_forward_dump.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _i, _p, _p, _p, C.c_int32, _p, _sz, _p]
+lib.falqon_melded_backward_dump.restype = _i
+lib.falqon_melded_backward_dump.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _p, _p, _i, _p, _p, C.c_int32, _p, _sz, _p]
 lib.falqon_melded_forward_codes.restype = _i
 lib.falqon_melded_forward_codes.argtypes = [C.POINTER(falqon_layer), _p, _p, _i64, _p, _i, _p, _p, _p, _sz, _p]
 lib.falqon_melded_backward.restype = _i
@@ -132,14 +138,23 @@ def _stream():
 class Layer:
     """Owns the device tensors of one melded layer and the host struct that points at them."""
 
-    def __init__(self, wq: torch.Tensor, s_w: torch.Tensor, dbuf: torch.Tensor, r: int):
+    def __init__(self, wq: torch.Tensor, s_w: torch.Tensor, dbuf: torch.Tensor, r: int, flags: int = 0):
         assert wq.dtype == torch.uint8 and wq.is_contiguous() and dbuf.dtype == torch.float32 and dbuf.is_contiguous()
         self.wq, self.s_w, self.dbuf = wq, s_w, dbuf
         self.m, self.n, self.r = wq.shape[0] - r, wq.shape[1], r
         assert s_w.numel() in (1, self.m + 1) and s_w.dtype == torch.float32 and s_w.is_contiguous()
         self.gran = PER_ROW if s_w.numel() == self.m + 1 else PER_TENSOR
-        self.c = falqon_layer(self.m, self.n, self.r, wq.data_ptr(), s_w.data_ptr(), dbuf.data_ptr(), self.gran, 0)
+        self.c = falqon_layer(self.m, self.n, self.r, wq.data_ptr(), s_w.data_ptr(), dbuf.data_ptr(), self.gran, flags)
         self._ws = None
+
+    @property
+    def flags(self) -> int:
+        return int(self.c.flags)
+
+    @flags.setter
+    def flags(self, value: int):
+        """falqon_layer.flags: LAYER_FUSED_CAST moves the casts of X and dY into the products' producers."""
+        self.c.flags = int(value)
 
     def workspace(self, T: int) -> torch.Tensor:
         need = workspace_bytes(self.m, self.n, self.r, T)
@@ -239,6 +254,39 @@ def melded_forward(layer: Layer, X: torch.Tensor, y_dtype=torch.bfloat16, ws: to
                                                               _ptr(OA), _ptr(amax_oa), _ptr(s_x), _ptr(ws), ws.numel(),
                                                               _stream()))
     return Y, OA, amax_oa, s_x
+
+
+def melded_forward_dump(layer: Layer, X: torch.Tensor, n_block: int, y_dtype=torch.float32, ws: torch.Tensor | None = None,
+                        amax_x: torch.Tensor | None = None):
+    """falqon_melded_forward_dump: the fused forward whose column block n_block also writes its staged codes to WS_XQ.
+    Returns (Y, OA, amax_oa, s_x) like melded_forward."""
+    T = X.shape[0]
+    dev = X.device
+    ws = layer.workspace(T) if ws is None else ws
+    Y = torch.empty((T, layer.m), dtype=y_dtype, device=dev)
+    OA = torch.empty((T, layer.r), dtype=torch.float32, device=dev)
+    amax_oa = torch.empty(1, dtype=torch.float32, device=dev)
+    s_x = torch.empty(1, dtype=torch.float32, device=dev)
+    _check("falqon_melded_forward_dump",
+           lib.falqon_melded_forward_dump(C.byref(layer.c), _ptr(X), _dt(X), _ptr(amax_x), T, _ptr(Y), _dt(Y), _ptr(OA),
+                                          _ptr(amax_oa), _ptr(s_x), n_block, _ptr(ws), ws.numel(), _stream()))
+    return Y, OA, amax_oa, s_x
+
+
+def melded_backward_dump(layer: Layer, dY: torch.Tensor, OA: torch.Tensor, amax_oa: torch.Tensor, n_block: int,
+                         dx_dtype=torch.float32, ws: torch.Tensor | None = None, amax_dy: torch.Tensor | None = None):
+    """falqon_melded_backward_dump: the fused backward whose dX column block n_block writes the codes of dY to WS_GQ.
+    Returns (dX, dB, s_g) like melded_backward."""
+    T = dY.shape[0]
+    dev = dY.device
+    ws = layer.workspace(T) if ws is None else ws
+    dX = torch.empty((T, layer.n), dtype=dx_dtype, device=dev)
+    dB = torch.empty((layer.m, layer.r), dtype=torch.float32, device=dev)
+    s_g = torch.empty(1, dtype=torch.float32, device=dev)
+    _check("falqon_melded_backward_dump",
+           lib.falqon_melded_backward_dump(C.byref(layer.c), _ptr(dY), _dt(dY), _ptr(amax_dy), T, _ptr(OA), _ptr(amax_oa),
+                                           _ptr(dX), _dt(dX), _ptr(dB), _ptr(s_g), n_block, _ptr(ws), ws.numel(), _stream()))
+    return dX, dB, s_g
 
 
 def melded_forward_codes(layer: Layer, xq: torch.Tensor, s_x: torch.Tensor, y_dtype=torch.bfloat16,

@@ -73,7 +73,8 @@ inline bool dtype_ok(int dt) { return dt == FALQON_BF16 || dt == FALQON_F32; }
 
 bool layer_ok(const falqon_layer* L) {
   return L != nullptr && shape_ok(L->m, L->n, L->r) && L->wq != nullptr && L->s_w != nullptr && L->dbuf != nullptr &&
-         aligned16(L->wq) && aligned16(L->dbuf) && (L->gran == FALQON_PER_TENSOR || L->gran == FALQON_PER_ROW);
+         aligned16(L->wq) && aligned16(L->dbuf) && (L->gran == FALQON_PER_TENSOR || L->gran == FALQON_PER_ROW) &&
+         (L->flags & ~(FALQON_LAYER_FUSED_CAST | FALQON_LAYER_EMIT_XQ)) == 0;
 }
 
 #define FALQON_CUDA(expr)                                   \
@@ -110,7 +111,8 @@ struct StageTimer {
 
 // S2: [Y | O_A] = x~ W~'^T / (s_W s_x), amax(O_A) from the epilogue (which accumulates into *amax_oa: zero beforehand)
 int forward_product(const falqon_layer* L, const uint8_t* xq, const float* s_x, int64_t T, void* Y, int y_dt, float* OA,
-                    float* amax_oa, uint8_t* base, const WorkspaceLayout& w, int* status, cudaStream_t stream) {
+                    float* amax_oa, uint8_t* base, const WorkspaceLayout& w, int* status, cudaStream_t stream,
+                    const FusedOperand* fused = nullptr) {
   const int64_t m = L->m, n = L->n, r = L->r;
   const bool per_row = L->gran == FALQON_PER_ROW;
   float* col_scale = reinterpret_cast<float*>(base + w.col_scale);
@@ -127,8 +129,17 @@ int forward_product(const falqon_layer* L, const uint8_t* xq, const float* s_x, 
   g.col_scale = per_row ? col_scale : nullptr;
   g.status = status;
   StageTimer timer(FALQON_STAGE_GEMM_FWD, stream);
-  FALQON_CUDA(launch_gemm_fp8(g, stream));
+  if (fused != nullptr) FALQON_CUDA(launch_gemm_fp8_fused(g, *fused, stream));
+  else FALQON_CUDA(launch_gemm_fp8(g, stream));
   return FALQON_OK;
+}
+
+// The product shapes of a layer that the fused kernel takes (see FALQON_LAYER_FUSED_CAST).
+bool fused_forward_ok(const falqon_layer* L, int x_dt) {
+  return (L->flags & FALQON_LAYER_FUSED_CAST) != 0 && x_dt == FALQON_BF16 && (L->m + L->r) % 16 == 0;
+}
+bool fused_backward_ok(const falqon_layer* L, int dy_dt, const void* dX) {
+  return (L->flags & FALQON_LAYER_FUSED_CAST) != 0 && dy_dt == FALQON_BF16 && L->gran == FALQON_PER_TENSOR && dX != nullptr;
 }
 
 }  // namespace
@@ -213,11 +224,17 @@ int falqon_workspace_init(void* ws, size_t ws_bytes, falqon_stream stream) {
 namespace {
 // amax_x (nullable, device [1]): the caller already knows max |X| (the kernel that produced X took it), so the cast is a
 // single pass with no reduction and no grid barrier.
+// dump_block >= 0: the debug hook (fused path required; that column block writes its staged codes to FALQON_WS_XQ).
 int forward_impl(const falqon_layer* L, const void* X, falqon_dtype x_dt, const float* amax_x, int64_t T, void* Y,
-                 falqon_dtype y_dt, float* OA, float* amax_oa, float* s_x_out, void* ws, size_t ws_bytes, falqon_stream stream) {
+                 falqon_dtype y_dt, float* OA, float* amax_oa, float* s_x_out, void* ws, size_t ws_bytes, falqon_stream stream,
+                 int dump_block = -1) {
   if (!layer_ok(L) || X == nullptr || Y == nullptr || OA == nullptr || amax_oa == nullptr || T < 1 || !dtype_ok(x_dt) ||
       !dtype_ok(y_dt) || !aligned16(X) || !aligned16(Y) || !aligned16(OA))
     return FALQON_ERR_INVALID_ARG;
+  if (dump_block >= 0) {
+    if (!fused_forward_ok(L, x_dt)) return FALQON_ERR_UNSUPPORTED;
+    if (dump_block >= (L->m + L->r + 255) / 256) return FALQON_ERR_INVALID_ARG;
+  }
   WorkspaceLayout w;
   if (!make_layout(L->m, L->n, L->r, T, &w)) return FALQON_ERR_INVALID_ARG;
   if (ws == nullptr || !aligned16(ws) || ws_bytes < w.total) return FALQON_ERR_WORKSPACE;
@@ -228,8 +245,20 @@ int forward_impl(const falqon_layer* L, const void* X, falqon_dtype x_dt, const 
   uint8_t* xq = base + w.act8;
   const int64_t n = L->n;
 
-  // S1: x~, s_x = Q_e4m3(X); the cast also clears amax(O_A), which the product's epilogue accumulates
   uint32_t* partial = reinterpret_cast<uint32_t*>(base + w.scales + kPartialsOffset);
+  if (fused_forward_ok(L, x_dt)) {
+    // S1 + S2 in one product: only the scale is prepared here (from an absmax pass over X when it is not known)
+    {
+      StageTimer timer(FALQON_STAGE_QUANT_X, stream);
+      int nparts = 0;
+      if (amax_x == nullptr) FALQON_CUDA(launch_absmax(X, x_dt, T * n, 1.0f, partial, &nparts, stream));
+      FALQON_CUDA(launch_scale_prep(partial, nparts, amax_x, kE4M3, scales + 1, s_x_out, scales + 0, amax_oa, stream));
+    }
+    const bool emit = dump_block >= 0 || (L->flags & FALQON_LAYER_EMIT_XQ) != 0;
+    const FusedOperand f{X, n, scales + 1, emit ? xq : nullptr, n, dump_block >= 0 ? dump_block : 0};
+    return forward_product(L, nullptr, scales + 1, T, Y, y_dt, OA, amax_oa, base, w, status, stream, &f);
+  }
+  // S1: x~, s_x = Q_e4m3(X); the cast also clears amax(O_A), which the product's epilogue accumulates
   {
     StageTimer timer(FALQON_STAGE_QUANT_X, stream);
     if (amax_x != nullptr) {
@@ -256,6 +285,13 @@ int falqon_melded_forward_amax(const falqon_layer* L, const void* X, falqon_dtyp
   return forward_impl(L, X, x_dt, amax_x, T, Y, y_dt, OA, amax_oa, s_x_out, ws, ws_bytes, stream);
 }
 
+int falqon_melded_forward_dump(const falqon_layer* L, const void* X, falqon_dtype x_dt, const float* amax_x, int64_t T, void* Y,
+                               falqon_dtype y_dt, float* OA, float* amax_oa, float* s_x_out, int32_t n_block, void* ws,
+                               size_t ws_bytes, falqon_stream stream) {
+  if (n_block < 0) return FALQON_ERR_INVALID_ARG;
+  return forward_impl(L, X, x_dt, amax_x, T, Y, y_dt, OA, amax_oa, s_x_out, ws, ws_bytes, stream, n_block);
+}
+
 int falqon_melded_forward_codes(const falqon_layer* L, const uint8_t* xq, const float* s_x, int64_t T, void* Y,
                                 falqon_dtype y_dt, float* OA, float* amax_oa, void* ws, size_t ws_bytes, falqon_stream stream) {
   if (!layer_ok(L) || xq == nullptr || s_x == nullptr || Y == nullptr || OA == nullptr || amax_oa == nullptr || T < 1 ||
@@ -274,10 +310,14 @@ namespace {
 // amax_dy (nullable, device [1]; per-tensor layers only): max |dY| is already known, see forward_impl.
 int backward_impl(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, const float* amax_dy, int64_t T, const float* OA,
                   const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, float* s_g_out, void* ws, size_t ws_bytes,
-                  falqon_stream stream) {
+                  falqon_stream stream, int dump_block = -1) {
   if (!layer_ok(L) || dY == nullptr || OA == nullptr || amax_oa == nullptr || dB == nullptr || T < 1 || !dtype_ok(dy_dt) ||
       !dtype_ok(dx_dt) || !aligned16(dY) || !aligned16(OA) || !aligned16(dB) || (dX != nullptr && !aligned16(dX)))
     return FALQON_ERR_INVALID_ARG;
+  if (dump_block >= 0) {
+    if (!fused_backward_ok(L, dy_dt, dX)) return FALQON_ERR_UNSUPPORTED;
+    if (dump_block >= (L->n + 255) / 256) return FALQON_ERR_INVALID_ARG;
+  }
   WorkspaceLayout w;
   if (!make_layout(L->m, L->n, L->r, T, &w)) return FALQON_ERR_INVALID_ARG;
   if (ws == nullptr || !aligned16(ws) || ws_bytes < w.total) return FALQON_ERR_WORKSPACE;
@@ -289,8 +329,40 @@ int backward_impl(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, con
   uint8_t* oaq_t = base + w.oaq_t;
   const int64_t m = L->m, n = L->n, r = L->r;
 
-  // S3: g~, s_g = Q_e5m2(dY)
   uint32_t* partial = reinterpret_cast<uint32_t*>(base + w.scales + kPartialsOffset);
+  if (fused_backward_ok(L, dy_dt, dX)) {
+    // S3 inside S4's producer: the input-gradient product casts dY tile by tile and its first column block also writes
+    // g~, which S5b (run after it here) reads as a tensor
+    {
+      StageTimer timer(FALQON_STAGE_QUANT_DY, stream);
+      int nparts = 0;
+      if (amax_dy == nullptr) FALQON_CUDA(launch_absmax(dY, dy_dt, T * m, 1.0f, partial, &nparts, stream));
+      FALQON_CUDA(launch_scale_prep(partial, nparts, amax_dy, kE5M2, scales + 3, s_g_out, scales + 2, nullptr, stream));
+      const OaCastJob oa_cast{OA, amax_oa, T, static_cast<int>(r), w.t16, oaq_t, scales + 5, scales + 4};
+      FALQON_CUDA(launch_oa_cast(oa_cast, stream));
+    }
+    {
+      GemmProblem g{};
+      g.M = T; g.N = n; g.K = m;
+      g.a = nullptr; g.lda = m; g.a_fmt = kE5M2;
+      g.b = L->wq; g.ldb = n; g.b_mn_major = true; g.b_fmt = kE4M3;
+      g.block_n = 256;
+      g.c0 = dX; g.ldc0 = n; g.c0_dt = dx_dt; g.n_split = n;
+      g.scale_a = scales + 3; g.scale_b = L->s_w;
+      g.status = status;
+      const FusedOperand f{dY, m, scales + 3, gq, m, dump_block >= 0 ? dump_block : 0};
+      StageTimer timer(FALQON_STAGE_GEMM_DX, stream);
+      FALQON_CUDA(launch_gemm_fp8_fused(g, f, stream));
+    }
+    DbFusedProblem d{};
+    d.m = m; d.r = r; d.T = T;
+    d.gq = gq; d.oaq_t = oaq_t; d.ldt = w.t16; d.s_oa = scales + 5;
+    d.s_g = scales + 3; d.row_mul = nullptr; d.dB = dB; d.status = status;
+    StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
+    FALQON_CUDA(launch_db_fused(d, stream));
+    return FALQON_OK;
+  }
+  // S3: g~, s_g = Q_e5m2(dY)
   const bool per_row = L->gran == FALQON_PER_ROW;
   float* inv_sw = reinterpret_cast<float*>(base + w.inv_sw);
   if (per_row)   // the row scales lie on dX's contraction axis: divide them out of dY before its cast
@@ -342,6 +414,13 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
                            const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, float* s_g_out, void* ws,
                            size_t ws_bytes, falqon_stream stream) {
   return backward_impl(L, dY, dy_dt, nullptr, T, OA, amax_oa, dX, dx_dt, dB, s_g_out, ws, ws_bytes, stream);
+}
+
+int falqon_melded_backward_dump(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, const float* amax_dy, int64_t T,
+                                const float* OA, const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, float* s_g_out,
+                                int32_t n_block, void* ws, size_t ws_bytes, falqon_stream stream) {
+  if (n_block < 0) return FALQON_ERR_INVALID_ARG;
+  return backward_impl(L, dY, dy_dt, amax_dy, T, OA, amax_oa, dX, dx_dt, dB, s_g_out, ws, ws_bytes, stream, n_block);
 }
 
 int falqon_melded_backward_amax(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, const float* amax_dy, int64_t T,
@@ -626,6 +705,9 @@ int falqon_launch_count(const char* entry_point, int64_t m, int64_t n, int64_t r
   if (std::strcmp(entry_point, "falqon_quantize") == 0) return 2;           // absmax, cast
   if (std::strcmp(entry_point, "falqon_melded_forward") == 0) return 2;     // fused quantize, GEMM
   if (std::strcmp(entry_point, "falqon_melded_backward") == 0) return 3;    // fused quantize, dX, fused dB
+  // with FALQON_LAYER_FUSED_CAST: absmax, scale, product / absmax, scale, O_A cast, dX product (casts dY, writes g~), dB
+  if (std::strcmp(entry_point, "falqon_melded_forward:fused") == 0) return 3;
+  if (std::strcmp(entry_point, "falqon_melded_backward:fused") == 0) return 5;
   if (std::strcmp(entry_point, "falqon_proxy_update") == 0) return k > 0 ? 2 : 1;  // optimizer+score+top-k, merge+clear
   if (std::strcmp(entry_point, "falqon_proxy_update_batched") == 0) return k > 0 ? 2 : 1;   // per 8 layers
   return 0;

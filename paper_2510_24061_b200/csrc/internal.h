@@ -71,6 +71,10 @@ cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, i
                                    const uint32_t* partial, int nparts, const float* scale_in, uint8_t* dst,
                                    float* scale_out, float* scale_out2, float* amax_out, float* clear_word,
                                    cudaStream_t stream);
+// The scale of a tensor without its cast (one small CTA): fp8max / amax with amax = max(partial[0..nparts)) when nparts > 0,
+// else *amax_in; outputs as launch_cast_per_tensor (all nullable).
+cudaError_t launch_scale_prep(const uint32_t* partial, int nparts, const float* amax_in, int fmt, float* scale_out,
+                              float* scale_out2, float* amax_out, float* clear_word, cudaStream_t stream);
 // A small cast that rides along with a fused quantizer launch (S5a inside S3's kernel): O_A [T][r] fp32 -> E4M3 codes
 // written transposed as [r][ldt] with s_OA = 448 / *amax_oa; *amax_copy = *amax_oa.  oa == nullptr: none.
 struct OaCastJob {
@@ -114,6 +118,22 @@ struct GemmProblem {
   int* status;
 };
 cudaError_t launch_gemm_fp8(const GemmProblem& p, cudaStream_t stream);
+
+// ---- gemm_fp8_fused.cu: the same product on CTA pairs with the cast of the A operand fused into the producer.  A arrives
+// as bf16 [M][lda16]; converter warps scale it by *a_scale (the scale of Eq. quantize, already on the device) and
+// round it to a_fmt straight into the swizzled operand slots, so its codes need never be written to memory.
+// p.a / p.lda are ignored; p.scale_a must be a_scale.  emit_dst (nullable): the tiles of output-column block
+// emit_n_block (256 columns each) also write the codes they staged to emit_dst[M][emit_ld] (emit_ld >= K).
+struct FusedOperand {
+  const void* a16; int64_t lda16;
+  const float* a_scale;
+  uint8_t* emit_dst; int64_t emit_ld; int emit_n_block;
+};
+// Whether the fused kernel takes this problem (CTA-pair tiling: block_n == 256, N a multiple of 16, K a multiple of 16).
+bool gemm_fp8_fused_supported(const GemmProblem& p);
+cudaError_t launch_gemm_fp8_fused(const GemmProblem& p, const FusedOperand& f, cudaStream_t stream);
+bool make_tensor_map_u16(CUtensorMap_st* map, const void* base, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols,
+                         uint32_t box_rows);
 // 2-D uint8 tensor [rows][cols] with row pitch ld bytes; box = box_cols x box_rows, 128-byte swizzle.
 bool make_tensor_map(CUtensorMap_st* map, const uint8_t* base, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols,
                      uint32_t box_rows);

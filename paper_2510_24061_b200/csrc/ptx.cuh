@@ -95,6 +95,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* st
   return mbar_wait_for(bar, parity, status, kWaitLimitNs);
 }
 
+// Makes this thread's earlier writes to shared memory visible to the asynchronous proxy (TMA, tcgen05.mma operands).
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 // The same wait executed by a whole converged warp; the outcome is made warp-uniform.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* status) {
   const bool ok = mbar_wait(bar, parity, status);
@@ -224,6 +227,12 @@ __device__ __forceinline__ float4 ld_shared_cluster_f32x4(uint32_t cluster_addr)
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {  // may target the peer CTA's barrier
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// The same arrival with the default (CTA-scope) release: for a thread whose earlier writes the barrier's waiters never
+// read themselves -- data handed to the tensor core through fence.proxy.async -- so that no cluster-wide memory fence
+// (hundreds of cycles) is paid per arrival.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }

@@ -159,6 +159,31 @@ __global__ void __launch_bounds__(kThreads) cast_kernel(const void* src, int64_t
   }
 }
 
+// ---- the scale of Eq. quantize on its own, for the products that cast their A operand themselves: from the partial
+// maxima of absmax_kernel (nparts > 0) or from an absmax the caller already has (*amax_in), with the same side outputs
+// as the cast kernels.  One CTA.
+__global__ void __launch_bounds__(kThreads) scale_prep_kernel(const uint32_t* partial, int nparts, const float* amax_in, int fmt,
+                                                              CastOutputs out) {
+  __shared__ uint32_t red[32];
+  pdl_trigger();
+  pdl_wait();
+  float amax;
+  if (nparts > 0) {
+    uint32_t mb = 0;
+    for (int i = threadIdx.x; i < nparts; i += kThreads) mb = max(mb, ld_stream(partial + i));
+    amax = __uint_as_float(block_max_u32(mb, red));
+  } else {
+    amax = ld_stream(amax_in);
+  }
+  if (threadIdx.x == 0) {
+    const float s = scale_from_amax(amax, fmt);
+    if (out.scale_out) *out.scale_out = s;
+    if (out.scale_out2) *out.scale_out2 = s;
+    if (out.amax_out) *out.amax_out = amax;
+    if (out.clear_word) *out.clear_word = 0.0f;
+  }
+}
+
 // The grid-wide barrier of the fused quantizer: two counters in the caller's workspace that start at zero and are
 // put back to zero by the last CTA to leave.
 struct GridSync {
@@ -556,6 +581,12 @@ cudaError_t launch_cast_per_tensor(const void* src, int src_dt, int64_t count, i
   if (src_dt == kBF16) { if (fmt == kE4M3) FALQON_CAST(kBF16, kE4M3); else FALQON_CAST(kBF16, kE5M2); }
   else { if (fmt == kE4M3) FALQON_CAST(kF32, kE4M3); else FALQON_CAST(kF32, kE5M2); }
 #undef FALQON_CAST
+}
+
+cudaError_t launch_scale_prep(const uint32_t* partial, int nparts, const float* amax_in, int fmt, float* scale_out,
+                              float* scale_out2, float* amax_out, float* clear_word, cudaStream_t stream) {
+  const CastOutputs out{scale_out, scale_out2, amax_out, clear_word};
+  return launch_pdl(scale_prep_kernel, dim3(1), dim3(kThreads), 0, stream, 1, partial, nparts, amax_in, fmt, out);
 }
 
 // The O_A cast as a kernel of its own (for a backward whose output-gradient absmax is already known, so that no fused

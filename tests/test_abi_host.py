@@ -74,6 +74,16 @@ def test_bad_arguments_are_rejected_on_the_host(fq):
     assert lib.falqon_melded_forward(C.byref(layer), fake, 0, 0, fake, 0, fake, fake, None, fake, big, None) == inv
     assert lib.falqon_melded_forward(C.byref(layer), fake, 3, 16, fake, 0, fake, fake, None, fake, big, None) == inv
     assert lib.falqon_melded_forward(C.byref(layer), fake, 0, 16, fake, 0, fake, fake, None, fake, 1024, None) == wsp
+    bad_flags = fq.falqon_layer(256, 256, 16, fake, fake, fake, 0, 8)     # an undefined flag bit
+    assert lib.falqon_melded_forward(C.byref(bad_flags), fake, 0, 16, fake, 0, fake, fake, None, fake, big, None) == inv
+    fused = fq.falqon_layer(256, 256, 16, fake, fake, fake, 0, fq.LAYER_FUSED_CAST)
+    assert lib.falqon_melded_forward_dump(C.byref(fused), fake, 0, None, 16, fake, 0, fake, fake, None, -1, fake, big, None) == inv
+    assert lib.falqon_melded_forward_dump(C.byref(fused), fake, 0, None, 16, fake, 0, fake, fake, None, 2, fake, big, None) == inv   # 272 columns: blocks 0, 1
+    assert lib.falqon_melded_forward_dump(C.byref(fused), fake, 1, None, 16, fake, 0, fake, fake, None, 0, fake, big, None) == fq.ERR_UNSUPPORTED   # fp32 X
+    assert lib.falqon_melded_forward_dump(C.byref(layer), fake, 0, None, 16, fake, 0, fake, fake, None, 0, fake, big, None) == fq.ERR_UNSUPPORTED   # flag not set
+    assert lib.falqon_melded_backward_dump(C.byref(fused), fake, 0, None, 16, fake, fake, fake, 0, fake, None, 1, fake, big, None) == inv   # 256 columns: block 0 only
+    assert lib.falqon_melded_backward_dump(C.byref(fused), fake, 0, None, 16, fake, fake, None, 0, fake, None, 0, fake, big, None) == fq.ERR_UNSUPPORTED   # no dX
+    assert fq.launch_count("falqon_melded_forward:fused") == 3 and fq.launch_count("falqon_melded_backward:fused") == 5
     bad_gran = fq.falqon_layer(256, 256, 16, fake, fake, fake, 2, 0)
     assert lib.falqon_melded_forward(C.byref(bad_gran), fake, 0, 16, fake, 0, fake, fake, None, fake, big, None) == inv
     odd = fq.falqon_layer(250, 256, 16, fake, fake, fake, 0, 0)
