@@ -38,7 +38,7 @@ FP8_OVER_BF16 = 2.0        # nominal dense FP8 : bf16 tensor throughput on B200 
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one forward and one dX launch of gemm_fp8_pair_kernel, measured with ncu on
-# the three projection shapes of the workload (profiles/gemm_fp8_pair_kernel__traffic_by_shape.md), in bytes:
+# the three projection shapes of the workload, in bytes:
 GEMM_DRAM_BYTES = {   # (n, m): (forward, dX)
     (4096, 4096): (33950976 + 2122240, 33630720 + 351488),
     (4096, 11008): (62336256 + 53340160, 136442624 + 18720512),
@@ -64,55 +64,72 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-             "clocks_event_reasons.sw_power_cap")
+    """Samples SM clock, power and clock-event reasons of one GPU every 10 ms on a host thread (NVML; reading only), each
+    sample stamped with the host clock, so that every timed pass gets the record of its own window."""
+    REASONS = [("hw_slowdown", "nvmlClocksEventReasonHwSlowdown"), ("hw_thermal_slowdown", "nvmlClocksEventReasonHwThermalSlowdown"),
+               ("sw_thermal_slowdown", "nvmlClocksEventReasonSwThermalSlowdown"), ("sw_power_cap", "nvmlClocksEventReasonSwPowerCap")]
 
-    def __init__(self, gpu_index: int):
-        self.gpu_index = gpu_index
-        self.proc = None
-        self.lines = []
+    def __init__(self, cuda_index: int, period_s: float = 0.01):
+        self.cuda_index, self.period = cuda_index, period_s
+        self.samples = []          # (t, sm_mhz, power_w, reason bits)
+        self.sm_max = None
+        self._stop = threading.Event()
         self.thread = None
+        self.error = None
+
+    def _handle(self, nv):
+        try:
+            uuid = str(torch.cuda.get_device_properties(self.cuda_index).uuid)
+            return nv.nvmlDeviceGetHandleByUUID(("GPU-" + uuid) if not uuid.startswith("GPU-") else uuid)
+        except Exception:
+            return nv.nvmlDeviceGetHandleByIndex(self.cuda_index)
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "50"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except Exception:
-            self.proc = None
+            import pynvml as nv
+            nv.nvmlInit()
+            h = self._handle(nv)
+            self.sm_max = float(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
+            masks = [(name, getattr(nv, attr)) for name, attr in self.REASONS]
+        except Exception as exc:      # no NVML: the record says so
+            self.error = f"NVML unavailable: {exc}"
             return
 
         def pump():
-            for line in self.proc.stdout:
-                self.lines.append(line.strip())
+            while not self._stop.is_set():
+                try:
+                    sm = float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                    pw = nv.nvmlDeviceGetPowerUsage(h) / 1000.0
+                    bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))
+                    self.samples.append((time.perf_counter(), sm, pw, tuple(name for name, m in masks if bits & m)))
+                except Exception as exc:
+                    self.error = str(exc)
+                    return
+                time.sleep(self.period)
         self.thread = threading.Thread(target=pump, daemon=True)
         self.thread.start()
 
+    @staticmethod
+    def now():
+        return time.perf_counter()
+
+    def window(self, t0: float, t1: float):
+        """Record of the samples taken between two host times (the caller synchronizes the device at both)."""
+        if self.thread is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": [self.error or "no sampler"]}
+        rows = [r for r in self.samples if t0 <= r[0] <= t1]
+        reasons = sorted({name for r in rows for name in r[3]})
+        return {"sm_mhz": statistics.median(r[1] for r in rows) if rows else None, "sm_max_mhz": self.sm_max,
+                "power_w_max": max((r[2] for r in rows), default=None), "samples": len(rows), "seconds": round(t1 - t0, 4),
+                "reasons": reasons}
+
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, smax, power, reasons = [], [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.lines:
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 7:
-                continue
-            try:
-                sm.append(float(parts[0])); smax.append(float(parts[1])); power.append(float(parts[2]))
-            except ValueError:
-                continue
-            for name, val in zip(names, parts[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+        self._stop.set()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        if self.samples:
+            return self.window(self.samples[0][0], self.samples[-1][0])
+        return self.window(0.0, 0.0)
 
 
 def aggregate_over_ranks(ms_local: float, flops_per_rank: float, dist=None, device=None):
@@ -483,6 +500,8 @@ def main():
                          "step (the library's calls only enqueue kernels, so a step can be captured; replays are about 2 %% faster)")
     ap.add_argument("--proxy-per-layer", action="store_true",
                     help="run one falqon_proxy_update per projection instead of one falqon_proxy_update_batched per step")
+    ap.add_argument("--soak", type=float, default=2.0, metavar="SECONDS",
+                    help="how long the step loop runs right before the timed steps, so that they see the clocks of a long job")
     ap.add_argument("--fused", action="store_true",
                     help="cast X and dY inside the producers of the tensor-core products (FALQON_LAYER_FUSED_CAST) instead of "
                          "in cast kernels of their own")
@@ -564,9 +583,42 @@ def main():
         return aggregate_over_ranks(ms, 0.0, dist, device)[0]
 
     batch = None if args.proxy_per_layer else make_proxy_batch(fq, layers, k)
-    # ---- device-resident timing: EXACTLY --steps steps between two events, nothing else in the stream
     sampler = ClockSampler(local_rank)
-    sampler.start()           # before the warm-up: starting it takes long enough for an idle GPU to drop its clocks
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(run, steps):
+        """EXACTLY `steps` calls of run() between two events, a barrier and a device synchronize on both sides; returns
+        (ms per step as the max over ranks, clock record of that window)."""
+        barrier()
+        t0 = sampler.now()
+        ev0.record()
+        for _ in range(steps):
+            run()
+        ev1.record()
+        barrier()
+        t1 = sampler.now()
+        return max_over_ranks(ev0.elapsed_time(ev1)) / steps, sampler.window(t0, t1)
+
+    def soak(run, seconds):
+        """Runs run() back to back for at least `seconds` (device busy the whole time), so that what is timed next sees
+        the clocks of a long job -- the board's power cap pulls the SM clock down within a second or so -- and not those
+        of a GPU that has just been idle.  Returns the clock record of the soak."""
+        t0 = sampler.now()
+        while True:
+            for _ in range(20):
+                run()
+            ev1.record()
+            ev1.synchronize()
+            if sampler.now() - t0 >= seconds:
+                break
+        return sampler.window(t0, sampler.now())
+
+    def with_cycles(ms, clocks):
+        """time x median SM clock of the pass: passes that ran at different clocks compare in cycles."""
+        mhz = clocks.get("sm_mhz")
+        return None if mhz is None else ms * 1e-3 * mhz * 1e6 / 1e6      # million SM cycles per step
+
     for _ in range(max(args.warmup, 3)):
         run_step(fq, layers, lr, k, batch)
     barrier()
@@ -578,15 +630,20 @@ def main():
         one_step = step_graph.replay
     for _ in range(max(args.warmup, 3)):      # the W warm-up steps proper, in the form that is timed
         one_step()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    # ---- burst: the first steps after an idle second (clocks at their maximum, power average still low)
+    burst_steps = 20
     barrier()
-    ev0.record()
-    for _ in range(args.steps):
-        one_step()
-    ev1.record()
-    barrier()
-    ms_total = max_over_ranks(ev0.elapsed_time(ev1))
-    ms_step = ms_total / args.steps
+    time.sleep(1.0)
+    ms_burst, clocks_burst = timed(one_step, burst_steps)
+
+    # ---- sustained (the headline): the same step loop for SOAK seconds first, then EXACTLY --steps steps
+    t_soak = sampler.now()
+    clocks_soak = soak(one_step, args.soak)
+    ms_step, clocks_timed = timed(one_step, args.steps)
+    clocks = sampler.window(t_soak, sampler.now())       # the soak and the timed steps: one continuous stretch of the same loop
+    clocks["soak_before"] = clocks_soak
+    clocks["timed_steps_only"] = clocks_timed
     value = world * flops_step / (ms_step * 1e-3) / 1e12
 
     # ---- forward and backward alone (quantization included, no proxy update): the quantity the metric's name describes;
@@ -595,31 +652,20 @@ def main():
         for L in layers:
             _, OA, amax_oa, _ = fq.melded_forward(L["layer"], L["X"], ws=L["ws"], out=L["out_f"])
             fq.melded_backward(L["layer"], L["dY"], OA, amax_oa, ws=L["ws"], out=L["out_b"])
-    for _ in range(3):
-        run_fwd_bwd()
-    barrier()
-    ev0.record()
-    for _ in range(args.steps):
-        run_fwd_bwd()
-    ev1.record()
-    barrier()
-    ms_fwd_bwd = max_over_ranks(ev0.elapsed_time(ev1)) / args.steps
+    soak(run_fwd_bwd, min(args.soak, 1.0))
+    ms_fwd_bwd, clocks_fwd_bwd = timed(run_fwd_bwd, args.steps)
 
-    # ---- the same steps again with the tensor-core products bracketed by CUDA events on the launching stream
-    # (an event between two kernels removes their launch overlap, so this pass is a little slower per step)
-    gemm_stages = ["gemm_fwd", "gemm_dx", "gemm_db"]
-    n_records = 3 * len(layers) * args.steps
-    fq.profile_start(n_records, gemm_stages)
-    barrier()
-    ev0.record()
-    for _ in range(args.steps):
-        run_step(fq, layers, lr, k, batch)
-    ev1.record()
-    barrier()
-    ms_step_instrumented = max_over_ranks(ev0.elapsed_time(ev1)) / args.steps
-    clocks = sampler.stop()
+    # ---- the same steps again, call by call, with EVERY stage bracketed by CUDA events on the launching stream (an event
+    # between two kernels removes their launch overlap, so this pass is slower per step): after a soak of its own, so
+    # that the kernel durations it records are those of the sustained regime too
+    eager_step = lambda: run_step(fq, layers, lr, k, batch)
+    soak(eager_step, min(args.soak, 1.0))
+    n_records = 12 * len(layers) * args.steps
+    fq.profile_start(n_records, None)
+    ms_step_instrumented, clocks_instrumented = timed(eager_step, args.steps)
     records = fq.profile_stop(n_records)
     status = fq.last_device_status()
+    sampler.stop()
 
     # ---- what one proxy update does to a backbone (bookkeeping outside every timed region, first projection):
     # codes that changed, and codes sitting at the largest finite magnitude (saturation of the requantized rows)
@@ -635,43 +681,70 @@ def main():
                     "changed_codes_outside_merged_rows": int((before != after).sum().item() - (before[rows] != after[rows]).sum().item()),
                     "saturated_codes_in_merged_rows": int(((after[rows] & 0x7F) == 0x7E).sum().item())}
 
-    # ---- roofline of the dominant kernel: the tcgen05 FP8 GEMM in its two tensor-bound roles
+    # ---- roofline of the dominant kernel: the tcgen05 FP8 GEMM in its two tensor-bound roles.  Its launches were timed
+    # by the library's stage events inside the soaked, instrumented pass above, so the matching peak is the SUSTAINED one.
     peaks = measured_peaks()
-    per_rec = 3 * len(layers)
     t_big = sum(ms for name, ms in records if name in ("gemm_fwd", "gemm_dx"))
     f_big = args.steps * sum(2.0 * T * n * (m + r) + 2.0 * T * m * n for _, n, m in linears)
     launches_big = sum(1 for name, _ in records if name in ("gemm_fwd", "gemm_dx"))
     achieved = f_big / (t_big * 1e-3) / 1e12 if t_big > 0 else 0.0
     peak = peaks["bf16_sustained"] * FP8_OVER_BF16
-    roofline = {"kernel": "gemm_fp8_pair_kernel (forward and input-gradient products)", "bound": "tensor",
+    gemm_name = "gemm_fp8_pair_fused_kernel" if args.fused else "gemm_fp8_pair_kernel"
+    roofline = {"kernel": f"{gemm_name} (forward and input-gradient products)", "bound": "tensor",
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "regime": "sustained: launch durations recorded by CUDA events on the launching stream inside a step loop that "
+                          "had been running for %.1f s; clocks of that pass under instrumented_pass" % min(args.soak, 1.0),
                 "peak_source": f"{peaks['source']} bf16 sustained x{FP8_OVER_BF16:g} (nominal FP8:bf16 ratio)",
-                "frac_of_burst_peak": achieved / (peaks["bf16_burst"] * FP8_OVER_BF16),
                 "frac_of_nominal_4500": achieved / 4500.0,
                 "launches": launches_big, "avg_launch_ms": t_big / max(launches_big, 1),
                 "gflop_per_launch": f_big / max(launches_big, 1) / 1e9,
                 "traffic": (sum(sum(GEMM_DRAM_BYTES[(n, m)]) for _, n, m in linears) / (2.0 * len(linears))
-                            if all((n, m) in GEMM_DRAM_BYTES for _, n, m in linears) else None),
-                "traffic_note": "dram read+write bytes per average launch, from the ncu capture of the forward and dX "
-                                "launch of each projection shape (profiles/gemm_fp8_pair_kernel__traffic_by_shape.md); "
+                            if all((n, m) in GEMM_DRAM_BYTES for _, n, m in linears) and not args.fused else None),
+                "traffic_note": "dram read+write bytes per average launch, from an ncu capture of the forward and the dX "
+                                "launch of each projection shape (un-fused kernel); "
                                 "algorithmic bytes per average launch: %.1f MB of FP8 operands + %.1f MB of bf16 / fp32 "
                                 "outputs (an operand the preceding cast left in L2, or an output still in L2 when the "
                                 "kernel ends, does not show up as DRAM traffic)" %
                                 (sum((T * n + (m + r) * n) + (T * m + m * n) for _, n, m in linears) / (2.0 * len(linears)) / 1e6,
                                  sum((2 * T * m + 4 * T * r) + 2 * T * n for _, n, m in linears) / (2.0 * len(linears)) / 1e6)}
-    t_db = sum(ms for name, ms in records if name == "gemm_db")
 
-    # ---- stage breakdown (separate untimed-for-value pass with every stage bracketed)
-    fq.profile_start(10 * len(layers) * 3, None)
-    for _ in range(3):
-        run_step(fq, layers, lr, k, batch)
-    torch.cuda.synchronize()
+    # ---- stage breakdown of the same pass, and the HBM-bound stages against the measured copy rate
     breakdown = {}
-    for name, ms in fq.profile_stop(10 * len(layers) * 3):
-        breakdown[name] = breakdown.get(name, 0.0) + ms / 3.0
-    hbm_bytes_quant = sum(T * n * 5 + T * m * 5 for _, n, m in linears)   # 2 B absmax read + 2 B cast read + 1 B write
+    for name, ms in records:
+        breakdown[name] = breakdown.get(name, 0.0) + ms / args.steps
+    t_db = breakdown.get("gemm_db", 0.0)
+    L2_BYTES = 126e6
+
+    def cast_bytes(elems, per_elt_small, per_elt_large):
+        return elems * (per_elt_small if 2.0 * elems <= L2_BYTES else per_elt_large)
+    # un-fused: the tensor is read once from DRAM (2 B), its codes written (1 B); a tensor larger than L2 is read a second
+    # time for the cast (5 B).  fused: only the absmax pass reads it (2 B).
+    lo, hi = (2, 2) if args.fused else (3, 5)
+    q_bytes = sum(cast_bytes(T * n, lo, hi) + cast_bytes(T * m, lo, hi) for _, n, m in linears)
+    q_bytes_5 = sum(5.0 * T * (n + m) for _, n, m in linears)
     t_quant = (breakdown.get("quant_x", 0) + breakdown.get("quant_dy", 0)) * 1e-3
-    quant_gbs = hbm_bytes_quant / t_quant / 1e9 if t_quant > 0 else 0.0
+    quant_gbs = q_bytes / t_quant / 1e9 if t_quant > 0 else 0.0
+    quantize = {"bound": "hbm", "achieved_gbs": quant_gbs, "peak_gbs": peaks["hbm"], "frac": quant_gbs / peaks["hbm"],
+                "frac_of_nominal_8000": quant_gbs / 8000.0, "ms_per_step": t_quant * 1e3,
+                "bytes_per_elt": lo, "bytes_per_step": q_bytes,
+                "frac_if_counted_at_5_bytes_per_elt": (q_bytes_5 / t_quant / 1e9 / peaks["hbm"]) if t_quant > 0 and not args.fused else None,
+                "note": ("absmax pass over X and dY (the casts run inside the products)" if args.fused else
+                         "absmax + cast of X and dY in one kernel each: every tensor of this workload fits L2, so it is read from "
+                         "DRAM once (2 B/elt) and its codes written once (1 B/elt); 5 B/elt would apply beyond L2") +
+                        "; the O_A cast rides in the same stage"}
+    db_bytes = sum(T * m + T * r + 4.0 * m * r for _, n, m in linears)
+    db = {"bound": "hbm", "kernel": "db_fused_kernel", "bytes_per_step": db_bytes, "ms_per_step": t_db,
+          "achieved_gbs": db_bytes / (t_db * 1e-3) / 1e9 if t_db > 0 else 0.0, "peak_gbs": peaks["hbm"],
+          "note": "reads g~ (T m bytes, written just before and largely still in L2) and O~_A, writes dB"}
+    db["frac"] = db["achieved_gbs"] / peaks["hbm"]
+    t_proxy = breakdown.get("sgd_score", 0.0) + breakdown.get("merge", 0.0)
+    proxy_bytes = sum(12.0 * m * r + 4.0 * m + k * (2.0 * n + 8.0 * r) + r * n for _, n, m in linears)
+    proxy = {"bound": "hbm for the optimizer pass, fp32 ALU for the merge at this rank", "bytes_per_step": proxy_bytes,
+             "ms_per_step": t_proxy, "achieved_gbs": proxy_bytes / (t_proxy * 1e-3) / 1e9 if t_proxy > 0 else 0.0,
+             "peak_gbs": peaks["hbm"], "merge_fma_per_step": sum(float(k) * n * r for _, n, m in linears),
+             "merge_frac_of_fp32_fma_peak": (sum(float(k) * n * r for _, n, m in linears) / (breakdown.get("merge", 0.0) * 1e-3) /
+                                             (148 * 128 * peaks_clock_ghz() * 1e9)) if breakdown.get("merge", 0.0) > 0 else None}
+    proxy["frac"] = proxy["achieved_gbs"] / peaks["hbm"]
 
     # ---- end to end: inputs in pinned host memory, results read back, every step
     host = []
@@ -722,20 +795,31 @@ def main():
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": ms_step, "ms_per_step_with_gemm_events": ms_step_instrumented,
+        "ms_per_step": ms_step, "mcycles_per_step": with_cycles(ms_step, clocks),
+        "regime": "sustained: %.1f s of the same step loop ran right before the timed steps" % args.soak,
+        "burst": {"ms_per_step": ms_burst, "value": world * flops_step / (ms_burst * 1e-3) / 1e12, "unit": UNIT, "steps": burst_steps,
+                  "mcycles_per_step": with_cycles(ms_burst, clocks_burst), "clocks": clocks_burst,
+                  "note": "the first steps after one idle second: clocks at their maximum, the board not yet at its power cap"},
         "fwd_bwd_only": {"ms_per_step": ms_fwd_bwd, "value": world * flops_step / (ms_fwd_bwd * 1e-3) / 1e12, "unit": UNIT,
-                         "note": "forward + backward of the seven projections with their input casts, without the proxy update"}, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8",
+                         "mcycles_per_step": with_cycles(ms_fwd_bwd, clocks_fwd_bwd), "clocks": clocks_fwd_bwd,
+                         "note": "forward + backward of the seven projections with their input casts, without the proxy update, "
+                                 "call by call after a soak of its own"},
+        "instrumented_pass": {"ms_per_step": ms_step_instrumented, "mcycles_per_step": with_cycles(ms_step_instrumented, clocks_instrumented),
+                              "clocks": clocks_instrumented,
+                              "note": "the step call by call with every stage bracketed by CUDA events (no launch overlap across the "
+                                      "brackets); source of roofline, stage_ms_per_step, quantize, db and proxy_update"},
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8",
         "data": "synthetic", "config": workload, "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e, "steps": e2e_steps,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches_per_step * args.steps,
         "roofline": roofline,
         "cpu_baseline": cpu_baseline,
-        "frac_of_fp8_peak": {"of_measured_sustained_x2": value / world / peak, "of_nominal_4500": value / world / 4500.0},
+        "frac_of_fp8_peak": {"of_measured_sustained_x2": value / world / peak, "of_nominal_4500": value / world / 4500.0,
+                             "burst_of_measured_burst_x2": world * flops_step / (ms_burst * 1e-3) / 1e12 / world / (peaks["bf16_burst"] * FP8_OVER_BF16),
+                             "note": "whole step (casts, dB and proxy update inside the time, only product FLOP counted)"},
         "stage_ms_per_step": {k_: round(v, 4) for k_, v in sorted(breakdown.items())},
-        "gemm_db_ms_per_step": t_db / args.steps,
-        "quantize": {"bound": "hbm", "achieved_gbs": quant_gbs, "peak_gbs": peaks["hbm"], "frac": quant_gbs / peaks["hbm"], "frac_of_nominal_8000": quant_gbs / 8000.0,
-                     "bytes_per_elt": 5, "note": "absmax pass + cast pass of X and dY, algorithmic bytes"},
+        "quantize": quantize, "db": db, "proxy_update": proxy,
         "proxy_update_effect": proxy_effect,
         "device_status": status,
     }

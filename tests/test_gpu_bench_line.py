@@ -37,4 +37,16 @@ def test_default_line_has_the_contract_keys():
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] >= 1 and c["value"] > 0 and "sample" in c
     assert set(("sm_mhz", "sm_max_mhz", "reasons")) <= set(d["clocks"])
+    # both regimes are on the line, each with its own clock record; the headline steps follow a soak of the same loop
+    assert d["clocks"]["samples"] >= 1 and d["clocks"]["soak_before"]["samples"] >= 20 and d["clocks"]["soak_before"]["seconds"] >= 2.0
+    b = d["burst"]
+    assert b["steps"] == 20 and abs(b["value"] - flops / (b["ms_per_step"] * 1e-3) / 1e12) < 1e-6 * b["value"] and "clocks" in b
+    assert b["ms_per_step"] <= d["ms_per_step"] * 1.05          # a cold board is not slower than one at its power cap
+    # the HBM-bound stages: achieved = stated bytes / stated time, fraction of the measured copy rate
+    for key in ("quantize", "db", "proxy_update"):
+        q = d[key]
+        assert abs(q["achieved_gbs"] - q["bytes_per_step"] / (q["ms_per_step"] * 1e-3) / 1e9) < 1e-6 * q["achieved_gbs"]
+        assert abs(q["frac"] - q["achieved_gbs"] / q["peak_gbs"]) < 1e-9 and 0 < q["frac"] < 1.2
+    assert d["quantize"]["bytes_per_elt"] == 3               # every tensor of configs[1] fits L2: one DRAM read, one write
+    assert "sustained" in r["regime"] and "instrumented_pass" in d and d["instrumented_pass"]["clocks"]["samples"] >= 1
     assert d["device_status"] == 0
