@@ -23,6 +23,13 @@
  *    programmatic stream serialization (each may be scheduled while its predecessor in
  *    the stream still runs and waits on the device for it to finish); a caller's own
  *    kernels placed between two calls are ordinary stream work and need nothing special.
+ *    The cast inside falqon_melded_forward / _backward (absmax, grid-wide barrier, cast: one kernel whose CTAs wait
+ *    for one another) is launched COOPERATIVELY: the driver starts it only when its whole grid -- one CTA per SM --
+ *    can be resident, so work of other streams on the same device delays it but cannot make it wait on CTAs that
+ *    never start.  Its barrier counters are balanced even when a wait runs out.  The *_amax calls, the fused casts
+ *    and falqon_quantize contain no such barrier.
+ *  - Devices: per-device look-ups (symbol addresses, occupancy) are cached for the life of the process; do not keep
+ *    using the library on a device after a cudaDeviceReset of it.
  *  - Errors: the return value is a falqon_status.  Bad arguments are detected on the
  *    host before anything is launched (nothing is written).  CUDA launch failures map
  *    to FALQON_ERR_CUDA.  Every device-side wait is bounded; a wait that runs out
@@ -263,7 +270,8 @@ int falqon_proxy_update_batched_adamw(const falqon_layer *layers, int32_t count,
  * cudaMalloc of its own would fail or stall the whole device mid-step.  The scratch (row scores and
  * the selected-row list) is a fixed 128 KB array inside the library image, resident on every GPU that
  * loads the library until the process exits.
- *   - Limit: L->m <= FALQON_STATIC_MAX_ROWS, otherwise FALQON_ERR_UNSUPPORTED and nothing is launched.
+ *   - Limits: L->m <= FALQON_STATIC_MAX_ROWS and a per-tensor scaled layer (FALQON_PER_TENSOR); otherwise
+ *     FALQON_ERR_UNSUPPORTED and nothing is launched.
  *   - The first call on each device looks up the array's device address (that device must be current);
  *     make that first call outside any stream capture.  Nothing is allocated or freed, ever.
  *   - All calls on a device share the array, which keeps the previous call's contents; nothing needs to
@@ -351,7 +359,8 @@ typedef enum {
   FALQON_STAGE_GEMM_DB = 5,   /* adapter-gradient product with the slab sum (S5b) */
   FALQON_STAGE_REDUCE_DB = 6, /* unused: the slab sum runs inside stage 5 */
   FALQON_STAGE_SGD_SCORE = 7, /* optimizer step, row scores and row selection (S6, S7) */
-  FALQON_STAGE_TOPK = 8,      /* row selection when it runs as its own kernel (falqon_proxy_update_static) */
+  FALQON_STAGE_TOPK = 8,      /* unused: the row selection runs inside stage 7 (falqon_proxy_update_static, where it is
+                                 a kernel of its own, is not bracketed by the timing hook) */
   FALQON_STAGE_MERGE = 9      /* merge + requantize + clear    (S8) */
 } falqon_stage;
 

@@ -10,17 +10,18 @@ namespace {
 
 __device__ int g_status_word;  // written by kernels whose bounded waits run out
 
-constexpr int kMaxDevices = 64;
-int* status_ptr() {
-  static int* ptrs[kMaxDevices] = {nullptr};
+int* status_ptr() {   // of the current device; host threads may race here: every racer looks up and stores the same address
+  static std::atomic<int*> ptrs[kMaxDevices];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-  if (ptrs[dev] == nullptr) {
+  int* cached = ptrs[dev].load(std::memory_order_acquire);
+  if (cached == nullptr) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
-    ptrs[dev] = static_cast<int*>(p);
+    cached = static_cast<int*>(p);
+    ptrs[dev].store(cached, std::memory_order_release);
   }
-  return ptrs[dev];
+  return cached;
 }
 
 struct WorkspaceLayout {
@@ -710,6 +711,7 @@ int falqon_launch_count(const char* entry_point, int64_t m, int64_t n, int64_t r
   if (std::strcmp(entry_point, "falqon_melded_backward:fused") == 0) return 5;
   if (std::strcmp(entry_point, "falqon_proxy_update") == 0) return k > 0 ? 2 : 1;  // optimizer+score+top-k, merge+clear
   if (std::strcmp(entry_point, "falqon_proxy_update_batched") == 0) return k > 0 ? 2 : 1;   // per 8 layers
+  if (std::strcmp(entry_point, "falqon_proxy_update_static") == 0) return k > 0 ? 4 : 1;   // optimizer+score, top-k, merge, clear (+ one copy of idx)
   return 0;
 }
 

@@ -15,6 +15,11 @@ constexpr int kBF16 = 0, kF32 = 1;
 
 inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
 
+// Per-device caches (symbol addresses, occupancy figures, configured attributes) are tables of this many entries, indexed
+// by the device ordinal; a device beyond it is refused.  The caches are filled on first use and never invalidated: the
+// library must not be used across a cudaDeviceReset of a device it has already run on.
+constexpr int kMaxDevices = 64;
+
 // The largest dynamic shared-memory size of a kernel is a property of the (kernel, device) pair: set it the first time a
 // launch site is used on a device.  `done` is the launch site's own word, one bit per device.
 using DeviceMask = std::atomic<unsigned long long>;
@@ -32,6 +37,8 @@ cudaError_t set_max_dynamic_smem(K kernel, int bytes, DeviceMask& done) {
 // Launches `kernel` so that it may be scheduled before the previous kernel in the stream has drained
 // (programmatic stream serialization).  The kernel itself must call pdl_wait() before it reads or writes
 // anything another kernel touches.  cluster_x > 1 adds a thread-block-cluster dimension.
+// cluster_x < 0: a COOPERATIVE launch without clusters -- the driver starts the grid only when all of its CTAs can be
+// resident at once, which a kernel whose CTAs wait for one another needs.
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, int cluster_x,
                        Args... args) {
@@ -45,6 +52,11 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[n].val.programmaticStreamSerializationAllowed = 1;
   ++n;
+  if (cluster_x < 0) {
+    attr[n].id = cudaLaunchAttributeCooperative;
+    attr[n].val.cooperative = 1;
+    ++n;
+  }
   if (cluster_x > 1) {
     attr[n].id = cudaLaunchAttributeClusterDimension;
     attr[n].val.clusterDim.x = static_cast<unsigned>(cluster_x);

@@ -34,7 +34,7 @@ constexpr size_t kScratchBytes = 2 * kScoreBytes;   // scores, then selected row
 
 static __device__ __align__(256) unsigned char g_proxy_scratch[kScratchBytes];
 
-constexpr int kMaxDevices = 64;
+using falqon::kMaxDevices;
 std::mutex g_lookup_mutex;
 unsigned char* g_scratch_addr[kMaxDevices] = {nullptr};
 

@@ -404,13 +404,16 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
   // bulk copies have landed, so the rider's loads do not queue behind them
   if (oa_job.oa != nullptr && tid >= kStagedThreads / 2)   // the upper half of the CTA's warps
     cast_oa_transposed(oa_job, (tid >> 5) - kStagedThreads / 64, kStagedThreads / 64);
-  // ---- grid barrier (a CTA that gave up above does not arrive: the others time out and report it)
+  // ---- grid barrier.  Every CTA arrives and (below) departs, whatever happened to it, so that the two counters are
+  // back at zero once the whole grid has run: a wait that ran out is reported through the status word and does not
+  // leave the workspace unusable for the next call.
   if (tid == 0) {
     int ok = failed ? 0 : 1;
+    if (!ok) atomicExch(status, kStatusTimeout);
+    partial[blockIdx.x] = m;
+    __threadfence();
+    atomicAdd(&sync->arrive, 1u);
     if (ok) {
-      partial[blockIdx.x] = m;
-      __threadfence();
-      atomicAdd(&sync->arrive, 1u);
       if (ld_acquire_gpu(&sync->arrive) < gridDim.x) {
         const uint64_t t0 = global_timer_ns();
         for (;;) {
@@ -479,7 +482,7 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
     while (global_timer_ns() - t0 < 200000ull) { }
   }
   __syncthreads();
-  if (tid == 0 && !failed) {
+  if (tid == 0) {
     const unsigned int prev = atomicAdd(&sync->depart, 1u);
     if (prev == gridDim.x - 1) {
       sync->arrive = 0u;
@@ -607,17 +610,20 @@ cudaError_t launch_staged_variant(const void* src, int64_t count, uint8_t* dst, 
     const cudaError_t ec = set_max_dynamic_smem(quantize_staged_kernel<kDt, kFmt, kColMul>, static_cast<int>(kSmem), configured);
     if (ec != cudaSuccess) return ec;
   }
-  static std::atomic<int> blocks_per_sm{0};   // the kernel's grid barrier needs every CTA resident: checked once
-  if (blocks_per_sm.load() == 0) {
-    int b = 0;
-    const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, quantize_staged_kernel<kDt, kFmt, kColMul>,
+  // the kernel's grid barrier needs every CTA resident: the grid is sized from the occupancy of the current device
+  // (looked up once per device) and the launch is cooperative, so the driver holds it until the whole grid fits
+  static std::atomic<int> blocks_per_sm_of[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  int blocks_per_sm = blocks_per_sm_of[dev].load();
+  if (blocks_per_sm == 0) {
+    const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, quantize_staged_kernel<kDt, kFmt, kColMul>,
                                                                         kStagedThreads, kSmem);
     if (e != cudaSuccess) return e;
-    if (b < 1) return cudaErrorLaunchOutOfResources;
-    blocks_per_sm.store(b);
+    if (blocks_per_sm < 1) return cudaErrorLaunchOutOfResources;
+    blocks_per_sm_of[dev].store(blocks_per_sm);
   }
-  int dev = 0, sms = 148;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = sm_count();
   const int64_t chunk_elems = kChunkBytes / (kDt == kBF16 ? 2 : 4);
   int64_t grid = (count / 16 * 16 + chunk_elems - 1) / chunk_elems;
   const int64_t resident = static_cast<int64_t>(blocks_per_sm) * sms;   // all CTAs must be resident together
@@ -631,8 +637,8 @@ cudaError_t launch_staged_variant(const void* src, int64_t count, uint8_t* dst, 
     if (table_chunks <= kStagedSlots - (128 * 1024) / kChunkBytes) { table_floats = cols; slots = kStagedSlots - table_chunks; }
   }
   return launch_pdl(quantize_staged_kernel<kDt, kFmt, kColMul>, dim3(static_cast<unsigned>(grid)), dim3(kStagedThreads), kSmem,
-                    stream, 1, src, count, dst, partial, static_cast<GridSync*>(sync), out, status, col_mul, cols, oa_job, slots,
-                    table_floats);
+                    stream, -1 /* cooperative */, src, count, dst, partial, static_cast<GridSync*>(sync), out, status, col_mul, cols,
+                    oa_job, slots, table_floats);
 }
 
 cudaError_t launch_quantize_fused(const void* src, int src_dt, int64_t count, int fmt, uint8_t* dst, uint32_t* partial,

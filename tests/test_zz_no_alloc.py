@@ -8,6 +8,7 @@ DeltaBuffer and selected indices are all bit-exact stages.
 """
 import ctypes as C
 
+import numpy as np
 import pytest
 import torch
 
@@ -60,4 +61,36 @@ def test_static_variant_matches_workspace_variant_on_two_calls():
     torch.cuda.synchronize()
     assert torch.equal(out.cpu(), torch.arange(m, dtype=torch.int32))
     assert torch.equal(ref.wq, new.wq) and not new.dbuf.any()
+    assert fq.last_device_status() == 0
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("k", [1, 300, 16384])
+def test_static_variant_at_its_row_limit_against_the_oracle(k):
+    """m = FALQON_STATIC_MAX_ROWS: the selection kernel of this path then needs its opted-in 64 KB of shared memory and
+    16 rows per thread.  Narrow rows keep the oracle quick.  Duplicated DeltaBuffer rows give tied scores, which must
+    go to the lower index.  Checked against the CPU oracle and against the workspace entry point, bit for bit."""
+    fq = _fq()
+    from oracle import falqon_oracle as orc
+    dev = "cuda:0"
+    m, n, r, lr = fq.STATIC_MAX_ROWS, 128, 8, 0.25
+    W = synth.backbone(22, 0, m, n, dev)
+    A = synth.adapter_a(22, 0, r, n, dev)
+    ref = fq.setup_layer(W, A, None, 1.0)
+    dB = synth.normal_bf16(22, 70, (m, r), 1.0, dev).float()
+    dB[1::2] = dB[0::2]                       # every odd row repeats the row before it: 8192 pairs of tied scores
+    new = fq.Layer(ref.wq.clone(), ref.s_w.clone(), ref.dbuf.clone(), r)
+    wq_o, dbuf_o = ref.wq.cpu().numpy().copy(), ref.dbuf.cpu().numpy().copy()
+    idx_ref = fq.proxy_update(ref, dB, lr, k)
+    idx_new = fq.proxy_update_static(new, dB, lr, k)
+    idx_o, _ = orc.proxy_update(wq_o, dbuf_o, dB.cpu().numpy(), lr, k, m, r)
+    torch.cuda.synchronize()
+    assert np.array_equal(idx_new.cpu().numpy(), idx_o), "selected rows differ from the oracle"
+    assert np.array_equal(new.wq.cpu().numpy(), wq_o), "merged rows differ from the oracle"
+    assert np.array_equal(new.dbuf.cpu().numpy().view(np.uint32), dbuf_o.view(np.uint32)), "DeltaBuffer differs from the oracle"
+    assert torch.equal(idx_ref, idx_new) and torch.equal(ref.wq, new.wq)
+    assert torch.equal(ref.dbuf.view(torch.int32), new.dbuf.view(torch.int32))
+    if k == 300:   # ties went to the lower index: an odd row is selected only together with its even twin
+        chosen = set(idx_o.tolist())
+        assert all((i - 1) in chosen for i in chosen if i % 2 == 1)
     assert fq.last_device_status() == 0
