@@ -197,6 +197,16 @@ int falqon_melded_backward_amax(const falqon_layer *L, const void *dY, falqon_dt
                                 const float *OA, const float *amax_oa, void *dX, falqon_dtype dx_dt, float *dB,
                                 float *s_g_out, void *ws, size_t ws_bytes, falqon_stream stream);
 
+/* The second half of falqon_melded_backward as a call of its own (the input-gradient product implied by Alg. 3): after a
+ * falqon_melded_backward[_amax] with dX == NULL -- which casts dY and O_A and computes dB -- this call computes
+ *   dX = g~ * W~ / (s_W * s_g)
+ * from the codes g~ and the scale s_g that call left in the workspace (FALQON_WS_GQ, FALQON_WS_SCALES; same T, same
+ * workspace, nothing else run on it in between).  The result is bit for bit the dX of the single call.  For callers
+ * that start exchanging dB while dX is still being computed (token-sharded data parallelism: dB is the one tensor
+ * that has to be summed over the shards, and nothing needs it before the proxy update). */
+int falqon_melded_backward_dx(const falqon_layer *L, int64_t T, void *dX, falqon_dtype dx_dt, void *ws, size_t ws_bytes,
+                              falqon_stream stream);
+
 /* Debug hook of the fused casts ("identical FP8 operands"): falqon_melded_forward / _backward for a layer with
  * FALQON_LAYER_FUSED_CAST, in which the product's tiles of output-column block n_block (256 columns each; forward:
  * columns of [Y | O_A], backward: columns of dX) also write the codes they staged in shared memory to FALQON_WS_XQ /

@@ -23,7 +23,7 @@ WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 
 EXPORTS = ["falqon_absmax", "falqon_selftest_wait_timeout", "falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax",
-           "falqon_melded_forward_dump", "falqon_melded_backward_dump", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
+           "falqon_melded_forward_dump", "falqon_melded_backward_dump", "falqon_melded_backward_dx", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
            "falqon_svd_init_scratch_bytes", "falqon_svd_init", "falqon_tensor_ceiling", "falqon_tensor_ceiling_ctas",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_proxy_update_batched", "falqon_proxy_update_batched_adamw", "falqon_last_device_status", "falqon_launch_count",
            "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static", "falqon_workspace_init", "falqon_proxy_update_adamw"]
@@ -61,6 +61,8 @@ lib.falqon_melded_forward_dump.restype = _i
 lib.falqon_melded_forward_dump.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _i, _p, _p, _p, C.c_int32, _p, _sz, _p]
 lib.falqon_melded_backward_dump.restype = _i
 lib.falqon_melded_backward_dump.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _p, _p, _i, _p, _p, C.c_int32, _p, _sz, _p]
+lib.falqon_melded_backward_dx.restype = _i
+lib.falqon_melded_backward_dx.argtypes = [C.POINTER(falqon_layer), _i64, _p, _i, _p, _sz, _p]
 lib.falqon_melded_forward_codes.restype = _i
 lib.falqon_melded_forward_codes.argtypes = [C.POINTER(falqon_layer), _p, _p, _i64, _p, _i, _p, _p, _p, _sz, _p]
 lib.falqon_melded_backward.restype = _i
@@ -335,6 +337,16 @@ def melded_backward(layer: Layer, dY: torch.Tensor, OA: torch.Tensor, amax_oa: t
                                                                 _ptr(amax_oa), _ptr(dX), dx_dt, _ptr(dB), _ptr(s_g),
                                                                 _ptr(ws), ws.numel(), _stream()))
     return dX, dB, s_g
+
+
+def melded_backward_dx(layer: Layer, T: int, dx_dtype=torch.bfloat16, ws: torch.Tensor | None = None, out: torch.Tensor | None = None):
+    """falqon_melded_backward_dx: dX [T, n] from the gradient codes the preceding melded_backward(need_dx=False) on the same
+    workspace left behind."""
+    ws = layer.workspace(T) if ws is None else ws
+    dX = torch.empty((T, layer.n), dtype=dx_dtype, device=layer.wq.device) if out is None else out
+    _check("falqon_melded_backward_dx", lib.falqon_melded_backward_dx(C.byref(layer.c), T, _ptr(dX), _dt(dX), _ptr(ws), ws.numel(),
+                                                                      _stream()))
+    return dX
 
 
 def proxy_update(layer: Layer, dB: torch.Tensor | None, lr: float, k: int, ws: torch.Tensor | None = None,

@@ -417,6 +417,30 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
   return backward_impl(L, dY, dy_dt, nullptr, T, OA, amax_oa, dX, dx_dt, dB, s_g_out, ws, ws_bytes, stream);
 }
 
+int falqon_melded_backward_dx(const falqon_layer* L, int64_t T, void* dX, falqon_dtype dx_dt, void* ws, size_t ws_bytes,
+                              falqon_stream stream) {
+  if (!layer_ok(L) || dX == nullptr || T < 1 || !dtype_ok(dx_dt) || !aligned16(dX)) return FALQON_ERR_INVALID_ARG;
+  WorkspaceLayout w;
+  if (!make_layout(L->m, L->n, L->r, T, &w)) return FALQON_ERR_INVALID_ARG;
+  if (ws == nullptr || !aligned16(ws) || ws_bytes < w.total) return FALQON_ERR_WORKSPACE;
+  int* status = status_ptr();
+  if (status == nullptr) return FALQON_ERR_CUDA;
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  float* scales = reinterpret_cast<float*>(base + w.scales);
+  // S4 on the codes and the scale that the backward call before it left in the workspace
+  GemmProblem g{};
+  g.M = T; g.N = L->n; g.K = L->m;
+  g.a = base + w.act8; g.lda = L->m; g.a_fmt = kE5M2;
+  g.b = L->wq; g.ldb = L->n; g.b_mn_major = true; g.b_fmt = kE4M3;
+  g.block_n = 256;
+  g.c0 = dX; g.ldc0 = L->n; g.c0_dt = dx_dt; g.n_split = L->n;
+  g.scale_a = scales + 3; g.scale_b = L->gran == FALQON_PER_ROW ? nullptr : L->s_w;
+  g.status = status;
+  StageTimer timer(FALQON_STAGE_GEMM_DX, stream);
+  FALQON_CUDA(launch_gemm_fp8(g, stream));
+  return FALQON_OK;
+}
+
 int falqon_melded_backward_dump(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, const float* amax_dy, int64_t T,
                                 const float* OA, const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, float* s_g_out,
                                 int32_t n_block, void* ws, size_t ws_bytes, falqon_stream stream) {

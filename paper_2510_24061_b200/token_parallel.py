@@ -33,11 +33,42 @@ class DistComm:
         self.dist.all_reduce(t, op=self.dist.ReduceOp.SUM, group=self.group)
 
 
+class SideStream:
+    """Where the exchange of dB runs while the compute stream goes on with the input-gradient product.  On a CUDA device:
+    a second stream and two events (fork: the side stream waits for what the compute stream has enqueued so far; join:
+    the compute stream waits for what the side stream has enqueued).  Without one (CPU tensors, in the tests): both are
+    no-ops and the calls simply run in program order."""
+
+    def __init__(self, device=None):
+        self.cuda = device is not None and torch.device(device).type == "cuda"
+        if self.cuda:
+            self.stream = torch.cuda.Stream(device=device)
+            self.forked, self.joined = torch.cuda.Event(), torch.cuda.Event()
+
+    def fork(self):
+        if self.cuda:
+            self.forked.record(torch.cuda.current_stream())
+            self.stream.wait_event(self.forked)
+
+    def run(self, fn):
+        if self.cuda:
+            with torch.cuda.stream(self.stream):
+                fn()
+        else:
+            fn()
+
+    def join(self):
+        if self.cuda:
+            self.joined.record(self.stream)
+            torch.cuda.current_stream().wait_event(self.joined)
+
+
 class TokenShardedLayer:
     def __init__(self, layer, ops=None, comm=None):
         if ops is None:
             from . import binding as ops      # fails loudly when the CUDA library is missing
         self.layer, self.ops, self.comm = layer, ops, comm
+        self.side = None        # SideStream for the exchange of dB, created on first use
         self.OA = None          # this shard's O_A, saved by forward() for backward()
         self.amax_oa = None     # max |O_A|: of this shard after forward(), of all shards once combined
 
@@ -61,13 +92,23 @@ class TokenShardedLayer:
                                              amax_dy=amax_dy)
         return dX, dB
 
+    def backward_db(self, dY: torch.Tensor, amax_dy: torch.Tensor):
+        """The first half of backward(): the casts and this shard's partial dB.  Leaves the gradient codes behind for
+        backward_dx()."""
+        _, dB, _ = self.ops.melded_backward(self.layer, dY, self.OA, self.amax_oa, need_dx=False, amax_dy=amax_dy)
+        return dB
+
+    def backward_dx(self, T: int, dx_dtype=torch.bfloat16):
+        """The second half: dX of this shard from the codes backward_db() left in the layer's workspace."""
+        return self.ops.melded_backward_dx(self.layer, T, dx_dtype=dx_dtype)
+
     def update(self, dB_total: torch.Tensor, lr: float, k: int):
         """The proxy update with the summed gradient; identical on every rank."""
         return self.ops.proxy_update(self.layer, dB_total, lr, k)
 
     # ---- all phases, with collectives ------------------------------------------------------------------------------
     def step(self, X: torch.Tensor, dY: torch.Tensor, lr: float, k: int, y_dtype=torch.bfloat16, need_dx: bool = True,
-             dx_dtype=torch.bfloat16):
+             dx_dtype=torch.bfloat16, overlap: bool = True):
         comm = self.comm if self.comm is not None else DistComm()
         amax_x = self.input_absmax(X)
         comm.all_reduce_max(amax_x)
@@ -75,7 +116,17 @@ class TokenShardedLayer:
         comm.all_reduce_max(self.amax_oa)
         amax_dy = self.output_grad_absmax(dY)
         comm.all_reduce_max(amax_dy)
-        dX, dB = self.backward(dY, amax_dy, need_dx=need_dx, dx_dtype=dx_dtype)
-        comm.all_reduce_sum(dB)                       # the method's one exchange step: 4 m r bytes per layer
+        if not (overlap and need_dx):
+            dX, dB = self.backward(dY, amax_dy, need_dx=need_dx, dx_dtype=dx_dtype)
+            comm.all_reduce_sum(dB)                   # the method's one exchange step: 4 m r bytes per layer
+            return Y, dX, dB, self.update(dB, lr, k)
+        # the exchange of dB overlaps the input-gradient product: nothing needs dB before the proxy update
+        if self.side is None:
+            self.side = SideStream(dY.device)
+        dB = self.backward_db(dY, amax_dy)
+        self.side.fork()                              # the side stream waits for dB ...
+        self.side.run(lambda: comm.all_reduce_sum(dB))
+        dX = self.backward_dx(dY.shape[0], dx_dtype=dx_dtype)   # ... while the compute stream goes on with dX
+        self.side.join()                              # the update needs the summed dB
         idx = self.update(dB, lr, k)
         return Y, dX, dB, idx

@@ -9,7 +9,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import bits32, f32, layer_inputs, rel_fro, u8
+from helpers import bits32, f32, layer_inputs, product_close, rel_fro, u8
 from paper_2510_24061_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -100,8 +100,8 @@ def _run_layer_stages(fq, orc, seed, m, n, r, T, k, gamma, n_outliers, steps, lr
         wq_now = u8(layer.wq)
         Y_o, OA_o, _ = orc.forward(xq_g, np.float32(f32(s_x)[0]), wq_now, s_w_g, m, r)
         OA_g = f32(OA)
-        assert rel_fro(f32(Y), Y_o) <= GEMM_TOL, f"Y step {step}"
-        assert rel_fro(OA_g, OA_o) <= GEMM_TOL, f"OA step {step}"
+        assert product_close(f32(Y), Y_o, GEMM_TOL), f"Y step {step}"
+        assert product_close(OA_g, OA_o, GEMM_TOL), f"OA step {step}"
         assert bits32(f32(amax_oa))[0] == bits32(np.abs(OA_g).max())
         # ---- backward
         dY = synth.out_grad(seed, 0, step, T, m)
@@ -120,8 +120,8 @@ def _run_layer_stages(fq, orc, seed, m, n, r, T, k, gamma, n_outliers, steps, lr
         assert np.array_equal(oaq_t[:r, :T].T, oaq_o)
         dX_o = orc.dx_gemm(gq_g, s_g_o, wq_now, s_w_g, m)
         dB_o = orc.db_gemm(gq_g, s_g_o, oaq_o, s_oa_o, row_scale=s_w_g[:m] if per_row else None)
-        assert rel_fro(f32(dX), dX_o) <= GEMM_TOL, f"dX step {step}"
-        assert rel_fro(f32(dB), dB_o) <= GEMM_TOL, f"dB step {step}"
+        assert product_close(f32(dX), dX_o, GEMM_TOL), f"dX step {step}"
+        assert product_close(f32(dB), dB_o, GEMM_TOL), f"dB step {step}"
         # ---- proxy update, fed the GPU's own dB
         dbuf_o = f32(layer.dbuf).copy()
         wq_o2 = wq_now.copy()
@@ -325,9 +325,9 @@ def _sampled_projection(fq, orc, matrix, n, m, T, r, k, lr, outlier_frac, per_ro
     fsel = np.sort(rng.choice(m, 48, replace=False))
     merged = torch.cat([Y, OA], dim=1)
     rows_o = orc.forward_gemm(xq_g, s_x_o, wq, s_w, m, r, tsel=tsel)                 # 48 token rows x all features
-    assert rel_fro(f32(merged[torch.from_numpy(tsel).to(DEV)]), rows_o) <= GEMM_TOL
+    assert product_close(f32(merged[torch.from_numpy(tsel).to(DEV)]), rows_o, GEMM_TOL)
     cols_o = orc.forward_gemm(xq_g, s_x_o, wq, s_w, m, r, fsel=fsel)                 # all tokens x 48 features
-    assert rel_fro(f32(Y[:, torch.from_numpy(fsel).to(DEV)]), cols_o) <= GEMM_TOL
+    assert product_close(f32(Y[:, torch.from_numpy(fsel).to(DEV)]), cols_o, GEMM_TOL)
     assert bits32(f32(amax_oa))[0] == bits32(f32(OA.abs().max()))
     dX, dB, s_g = fq.melded_backward(layer, dY, OA, amax_oa, dx_dtype=torch.float32, ws=ws)
     gq_g = u8(fq.ws_view(layer, ws, T, fq.WS_GQ)).reshape(T, m)
@@ -337,12 +337,12 @@ def _sampled_projection(fq, orc, matrix, n, m, T, r, k, lr, outlier_frac, per_ro
         gq_o, s_g_o, _ = orc.quantize(f32(dY), orc.E5M2)
     assert bits32(f32(s_g))[0] == bits32(s_g_o) and np.array_equal(gq_g, gq_o)
     csel = np.sort(rng.choice(n, 48, replace=False))
-    assert rel_fro(f32(dX[torch.from_numpy(tsel).to(DEV)]), orc.dx_gemm(gq_g, s_g_o, wq, s_w, m, tsel=tsel)) <= GEMM_TOL
-    assert rel_fro(f32(dX[:, torch.from_numpy(csel).to(DEV)]), orc.dx_gemm(gq_g, s_g_o, wq, s_w, m, csel=csel)) <= GEMM_TOL
+    assert product_close(f32(dX[torch.from_numpy(tsel).to(DEV)]), orc.dx_gemm(gq_g, s_g_o, wq, s_w, m, tsel=tsel), GEMM_TOL)
+    assert product_close(f32(dX[:, torch.from_numpy(csel).to(DEV)]), orc.dx_gemm(gq_g, s_g_o, wq, s_w, m, csel=csel), GEMM_TOL)
     oaq_o, s_oa_o, _ = orc.quantize(f32(OA), orc.E4M3)
     isel = np.sort(rng.choice(m, 96, replace=False))
     dB_o = orc.db_gemm(gq_g, s_g_o, oaq_o, s_oa_o, isel=isel, row_scale=s_w[:m] if per_row else None)
-    assert rel_fro(f32(dB[torch.from_numpy(isel).to(DEV)]), dB_o) <= GEMM_TOL
+    assert product_close(f32(dB[torch.from_numpy(isel).to(DEV)]), dB_o, GEMM_TOL)
     dbuf_o, wq_o = f32(layer.dbuf).copy(), wq.copy()
     idx = fq.proxy_update(layer, dB, lr, k, ws=ws)
     idx_o, score_o = orc.proxy_update(wq_o, dbuf_o, f32(dB), lr, k, m, r, row_scales=s_w if per_row else None)

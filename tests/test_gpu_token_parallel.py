@@ -7,7 +7,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import bits32, f32, layer_inputs, rel_fro, u8
+from helpers import bits32, f32, layer_inputs, product_close, rel_fro, u8
 from paper_2510_24061_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -50,7 +50,7 @@ def test_two_token_shards_against_the_unsharded_call(m, n, r, T, split, k):
     gq = u8(fq.ws_view(full, ws, T, fq.WS_GQ)).reshape(T, m)
     oaq_o, s_oa_o, _ = orc.quantize(f32(OA_f), orc.E4M3)
     dB_o = orc.db_gemm(gq, np.float32(s_g_f.item()), oaq_o, s_oa_o)
-    assert rel_fro(f32(dB_total), dB_o) <= 2e-5
+    assert product_close(f32(dB_total), dB_o, 2e-5)
     # the update: identical on both sharded replicas, and the oracle's update of the same summed gradient
     wq_o, dbuf_o = u8(reps[0].wq).copy(), f32(reps[0].dbuf).copy()
     idx = [t.update(dB_total, lr, k) for t in ts]
@@ -59,4 +59,42 @@ def test_two_token_shards_against_the_unsharded_call(m, n, r, T, split, k):
     assert torch.equal(reps[0].wq, reps[1].wq) and np.array_equal(u8(reps[0].wq), wq_o)
     assert torch.equal(reps[0].dbuf.view(torch.int32), reps[1].dbuf.view(torch.int32))
     assert np.array_equal(bits32(f32(reps[0].dbuf)), bits32(dbuf_o))
+    assert fq.last_device_status() == 0
+
+
+def test_split_backward_and_overlapped_step_equal_the_single_call():
+    """falqon_melded_backward_dx after a backward without dX gives the dX of the single call bit for bit, and a step whose
+    dB exchange runs on a side stream between the two halves (one rank: the reductions are identities) leaves the same
+    results and the same layer as the step that runs them in order."""
+    from paper_2510_24061_b200 import binding as fq
+    from paper_2510_24061_b200.token_parallel import TokenShardedLayer
+    m, n, r, T, k, lr = 768, 1024, 32, 900, 40, 2e-2
+    W, A, B, X = layer_inputs(32, 0, m, n, r, T, 5, DEV)
+    dY = synth.out_grad(32, 0, 0, T, m, DEV)
+    base = fq.setup_layer(W, A, B, 1.0)
+    ws = base.workspace(T)
+    Y, OA, amax_oa, _ = fq.melded_forward(base, X, y_dtype=torch.float32, ws=ws)
+    dX0, dB0, _ = fq.melded_backward(base, dY, OA, amax_oa, dx_dtype=torch.float32, ws=ws)
+    _, dB1, _ = fq.melded_backward(base, dY, OA, amax_oa, need_dx=False, ws=ws)
+    dX1 = fq.melded_backward_dx(base, T, dx_dtype=torch.float32, ws=ws)
+    assert torch.equal(dX0.view(torch.int32), dX1.view(torch.int32)) and torch.equal(dB0.view(torch.int32), dB1.view(torch.int32))
+
+    class OneRank:
+        def all_reduce_max(self, t):
+            pass
+
+        def all_reduce_sum(self, t):
+            t.mul_(1.0)        # some work on whatever stream is current, in place like a collective
+
+    results = []
+    for overlap in (False, True):
+        rep = fq.Layer(base.wq.clone(), base.s_w.clone(), base.dbuf.clone(), r)
+        ts = TokenShardedLayer(rep, comm=OneRank())
+        out = ts.step(X, dY, lr, k, y_dtype=torch.float32, dx_dtype=torch.float32, overlap=overlap)
+        torch.cuda.synchronize()
+        results.append((out, rep))
+    (a, ra), (b, rb) = results
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+    assert torch.equal(ra.wq, rb.wq) and torch.equal(ra.dbuf.view(torch.int32), rb.dbuf.view(torch.int32))
     assert fq.last_device_status() == 0

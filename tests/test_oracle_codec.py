@@ -182,3 +182,28 @@ def test_quantize_per_row():
     for i in range(5):
         qi, si, ai = orc.quantize(x[i:i + 1], orc.E4M3)
         assert si == s[i] and ai == amax[i] and np.array_equal(qi[0], q[i])
+
+
+def test_f32_to_bf16_rounding_matches_library_cast():
+    """The oracle's fp32 -> bf16 rounding (nearest, ties to even) against PyTorch's CPU cast, an independent
+    implementation: every exact tie between two bf16 neighbours and its two fp32 neighbours for a spread of exponents,
+    hand-worked cases, and random values."""
+    import torch
+    from oracle import falqon_oracle as orc
+    cases = {1.0: 0x3F80, -1.0: 0xBF80, 0.0: 0x0000, 1.00390625: 0x3F80,    # 1 + 2^-8: tie, even mantissa below
+             1.01171875: 0x3F82,                                            # 1 + 3*2^-8: tie, rounds up to the even code
+             1.0078125: 0x3F81, 3.3895313892515355e38: 0x7F7F}              # largest finite bf16
+    for v, code in cases.items():
+        assert orc.f32_to_bf16_bits(v) == code, v
+    rng = np.random.default_rng(3)
+    hi = rng.integers(0x0080, 0x7F00, size=4000, dtype=np.uint32)           # positive normal bf16 patterns
+    vals = []
+    for h in hi:
+        tie = (int(h) << 16) | 0x8000
+        vals += [tie - 1, tie, tie + 1]
+    bits = np.array(vals, dtype=np.uint32)
+    bits = np.concatenate([bits, bits | 0x80000000, rng.integers(0, 0x7F800000, size=20000, dtype=np.uint32)])
+    x = bits.view(np.float32)
+    want = torch.from_numpy(x.copy()).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    got = np.array([orc.f32_to_bf16_bits(v) for v in x], dtype=np.uint16)
+    assert np.array_equal(got, want)

@@ -44,9 +44,17 @@ class OracleOps:
         s_oa = self._scale(amax_oa.item(), 448.0)
         gq, _, _ = o.quantize(dY.float().numpy(), o.E5M2, scale_in=s_g)
         oaq, _, _ = o.quantize(OA.numpy(), o.E4M3, scale_in=s_oa)
-        dX = o.dx_gemm(gq, s_g, layer.wq, layer.s_w, layer.m)
+        self._gq, self._s_g = gq, s_g
+        dX = torch.from_numpy(o.dx_gemm(gq, s_g, layer.wq, layer.s_w, layer.m).astype(np.float32)) if need_dx else None
         dB = o.db_gemm(gq, s_g, oaq, s_oa)
-        return torch.from_numpy(dX.astype(np.float32)), torch.from_numpy(dB.astype(np.float32)), torch.tensor([s_g])
+        return dX, torch.from_numpy(dB.astype(np.float32)), torch.tensor([s_g])
+
+        # (need_dx=False: the first half of the split backward; the codes stay behind for melded_backward_dx)
+
+    def melded_backward_dx(self, layer, T, dx_dtype=torch.float32):
+        dX = self.orc.dx_gemm(self._gq, self._s_g, layer.wq, layer.s_w, layer.m)
+        assert dX.shape[0] == T
+        return torch.from_numpy(dX.astype(np.float32))
 
     def proxy_update(self, layer, dB, lr, k):
         idx, _ = self.orc.proxy_update(layer.wq, layer.dbuf, dB.numpy(), lr, k, layer.m, layer.r)
@@ -107,3 +115,62 @@ def test_two_ranks_reproduce_the_unsharded_step():
     # against the unsharded update: the same rows unless two scores are within the last bit of each other
     assert len(set(a["idx"].tolist()) & set(idx_full.tolist())) >= K - 1
     assert float((a["wq"] != wq_full).mean()) < 2e-2
+
+
+def test_exchange_of_db_is_issued_between_the_two_halves_of_backward():
+    """The order in which TokenShardedLayer.step issues its work when the exchange overlaps the input-gradient product:
+    dB is computed first, its sum is started on the side stream right after a fork, dX is enqueued while it runs, and the
+    update comes only after the join.  A recording communicator and a recording side stream stand in for the real ones;
+    the result equals the un-overlapped order's."""
+    sys.path.insert(0, ROOT)
+    from paper_2510_24061_b200.token_parallel import TokenShardedLayer
+    orc, wq, s_w, dbuf, X, dY = _inputs()
+    log = []
+
+    class Ops(OracleOps):
+        def melded_forward(self, *a, **k):
+            log.append("forward")
+            return super().melded_forward(*a, **k)
+
+        def melded_backward(self, layer, dY, OA, amax_oa, need_dx=True, **k):
+            log.append("backward" if need_dx else "backward_db")
+            return super().melded_backward(layer, dY, OA, amax_oa, need_dx=need_dx, **k)
+
+        def melded_backward_dx(self, *a, **k):
+            log.append("backward_dx")
+            return super().melded_backward_dx(*a, **k)
+
+        def proxy_update(self, *a, **k):
+            log.append("update")
+            return super().proxy_update(*a, **k)
+
+    class Comm:     # a single rank: the reductions are identities
+        def all_reduce_max(self, t):
+            log.append("max")
+
+        def all_reduce_sum(self, t):
+            log.append("sum")
+
+    class Side:
+        def fork(self):
+            log.append("fork")
+
+        def run(self, fn):
+            log.append("side:")
+            fn()
+
+        def join(self):
+            log.append("join")
+
+    results = {}
+    for overlap in (True, False):
+        del log[:]
+        layer = types.SimpleNamespace(wq=wq.copy(), s_w=s_w, dbuf=dbuf.copy(), m=M, n=N, r=R)
+        ts = TokenShardedLayer(layer, ops=Ops(orc), comm=Comm())
+        ts.side = Side()
+        Y, dX, dB, idx = ts.step(X, dY, LR, K, y_dtype=torch.float32, dx_dtype=torch.float32, overlap=overlap)
+        results[overlap] = (Y.numpy(), dX.numpy(), dB.numpy(), idx.numpy(), layer.wq.copy(), list(log))
+    assert results[True][5] == ["max", "forward", "max", "max", "backward_db", "fork", "side:", "sum", "backward_dx", "join", "update"]
+    assert results[False][5] == ["max", "forward", "max", "max", "backward", "sum", "update"]
+    for a, b in zip(results[True][:5], results[False][:5]):
+        assert np.array_equal(a, b)
