@@ -167,6 +167,15 @@ def build_workload(fq, device, seed, T, r, k, linears, outlier_frac, per_row=Fal
     return layers
 
 
+def run_step_fused_update(fq, layers, lr, k, batch):
+    """The step with Alg. 3 line 4 and the row scores inside the adapter-gradient kernel (falqon_melded_backward_update) and
+    one batched selection + merge (falqon_proxy_update_scored_batched)."""
+    for L in layers:
+        _, OA, amax_oa, _ = fq.melded_forward(L["layer"], L["X"], ws=L["ws"], out=L["out_f"])
+        fq.melded_backward_update(L["layer"], L["dY"], OA, amax_oa, lr, ws=L["ws"], out=L["out_b"])
+    batch.run_scored()
+
+
 def run_step(fq, layers, lr, k, batch=None):
     """Forward and backward of every projection, and the proxy update of each: one batched call for the whole set
     (batch: a ProxyBatch over the layers' gradient buffers), or one call per projection when batch is None."""
@@ -500,6 +509,9 @@ def main():
                          "step (the library's calls only enqueue kernels, so a step can be captured; replays are about 2 %% faster)")
     ap.add_argument("--proxy-per-layer", action="store_true",
                     help="run one falqon_proxy_update per projection instead of one falqon_proxy_update_batched per step")
+    ap.add_argument("--fused-update", action="store_true",
+                    help="run the optimizer step and the row scores inside the adapter-gradient kernel "
+                         "(falqon_melded_backward_update + falqon_proxy_update_scored_batched)")
     ap.add_argument("--soak", type=float, default=2.0, metavar="SECONDS",
                     help="how long the step loop runs right before the timed steps, so that they see the clocks of a long job")
     ap.add_argument("--fused", action="store_true",
@@ -619,14 +631,17 @@ def main():
         mhz = clocks.get("sm_mhz")
         return None if mhz is None else ms * 1e-3 * mhz * 1e6 / 1e6      # million SM cycles per step
 
+    step_fn = run_step
+    if args.fused_update:
+        step_fn = lambda fq_, layers_, lr_, k_, batch_: run_step_fused_update(fq_, layers_, lr_, k_, batch_)
     for _ in range(max(args.warmup, 3)):
-        run_step(fq, layers, lr, k, batch)
+        step_fn(fq, layers, lr, k, batch)
     barrier()
-    one_step = lambda: run_step(fq, layers, lr, k, batch)
+    one_step = lambda: step_fn(fq, layers, lr, k, batch)
     if not args.eager:
         step_graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(step_graph):
-            run_step(fq, layers, lr, k, batch)
+            step_fn(fq, layers, lr, k, batch)
         one_step = step_graph.replay
     for _ in range(max(args.warmup, 3)):      # the W warm-up steps proper, in the form that is timed
         one_step()
@@ -658,7 +673,7 @@ def main():
     # ---- the same steps again, call by call, with EVERY stage bracketed by CUDA events on the launching stream (an event
     # between two kernels removes their launch overlap, so this pass is slower per step): after a soak of its own, so
     # that the kernel durations it records are those of the sustained regime too
-    eager_step = lambda: run_step(fq, layers, lr, k, batch)
+    eager_step = lambda: step_fn(fq, layers, lr, k, batch)
     soak(eager_step, min(args.soak, 1.0))
     n_records = 12 * len(layers) * args.steps
     fq.profile_start(n_records, None)

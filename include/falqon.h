@@ -235,6 +235,28 @@ int falqon_melded_backward_dump(const falqon_layer *L, const void *dY, falqon_dt
 int falqon_proxy_update(const falqon_layer *L, const float *dB, float lr, int64_t k, int32_t *idx_out,
                         void *ws, size_t ws_bytes, falqon_stream stream);
 
+/* Alg. 3 lines 3-4 in one call: falqon_melded_backward (or, with amax_dy non-NULL, falqon_melded_backward_amax) followed
+ * by the plain-SGD step on the DeltaBuffer and the row scores,
+ *     DeltaBuffer <- fma(-lr, dB, DeltaBuffer);   score_i = sum_j |DeltaBuffer[i][j]|  (fp32, j ascending),
+ * both computed where dB is produced (the adapter-gradient kernel's slab-sum phase holds whole rows of dB), so the
+ * DeltaBuffer and dB are not read again by a pass of their own.  The scores are left in FALQON_WS_SCORE.  Bit for bit the
+ * DeltaBuffer and scores that falqon_melded_backward + falqon_proxy_update(dB, lr, k = 0) produce.  Mutates L->dbuf.
+ * dB (device [m][r] fp32) is still written.  Follow it with falqon_proxy_update_scored on the same workspace.
+ * (Where the kernel's shared memory has no room for the fused step -- ranks near 256 with few token slabs -- the same
+ * arithmetic runs as a pass of its own, with the same results.) */
+int falqon_melded_backward_update(const falqon_layer *L, const void *dY, falqon_dtype dy_dt, const float *amax_dy, int64_t T,
+                                  const float *OA, const float *amax_oa, void *dX, falqon_dtype dx_dt, float *dB, float lr,
+                                  float *s_g_out, void *ws, size_t ws_bytes, falqon_stream stream);
+
+/* Alg. 3 lines 5-6 (Eq. update) on their own: row selection and merge, as in falqon_proxy_update, from the row scores
+ * that falqon_melded_backward_update left in this workspace (they must be those of the current DeltaBuffer; nothing is
+ * recomputed).  k == 0 is a no-op.  The batched form takes host arrays like falqon_proxy_update_batched and is
+ * bit-identical to the per-layer calls. */
+int falqon_proxy_update_scored(const falqon_layer *L, int64_t k, int32_t *idx_out, void *ws, size_t ws_bytes,
+                               falqon_stream stream);
+int falqon_proxy_update_scored_batched(const falqon_layer *layers, int32_t count, const int64_t *k, int32_t *const *idx_out,
+                                       void *const *ws, const size_t *ws_bytes, falqon_stream stream);
+
 /* falqon_proxy_update for `count` layers in two launches instead of 2 x count (Alg. 3 lines 4-6, Eq. update, for each
  * layer; the paper's layer-wise schedule runs the updates of a block's projections back to back, and one layer's update
  * moves only a few MB, so a single call is bound by launch latency rather than by memory).  All arrays are HOST arrays

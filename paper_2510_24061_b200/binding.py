@@ -23,7 +23,8 @@ WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 
 EXPORTS = ["falqon_absmax", "falqon_selftest_wait_timeout", "falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax",
-           "falqon_melded_forward_dump", "falqon_melded_backward_dump", "falqon_melded_backward_dx", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
+           "falqon_melded_forward_dump", "falqon_melded_backward_dump", "falqon_melded_backward_dx",
+           "falqon_melded_backward_update", "falqon_proxy_update_scored", "falqon_proxy_update_scored_batched", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
            "falqon_svd_init_scratch_bytes", "falqon_svd_init", "falqon_tensor_ceiling", "falqon_tensor_ceiling_ctas",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_proxy_update_batched", "falqon_proxy_update_batched_adamw", "falqon_last_device_status", "falqon_launch_count",
            "falqon_profile_start", "falqon_profile_stop", "falqon_proxy_update_static", "falqon_workspace_init", "falqon_proxy_update_adamw"]
@@ -61,6 +62,13 @@ lib.falqon_melded_forward_dump.restype = _i
 lib.falqon_melded_forward_dump.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _i, _p, _p, _p, C.c_int32, _p, _sz, _p]
 lib.falqon_melded_backward_dump.restype = _i
 lib.falqon_melded_backward_dump.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _p, _p, _i, _p, _p, C.c_int32, _p, _sz, _p]
+lib.falqon_melded_backward_update.restype = _i
+lib.falqon_melded_backward_update.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _p, _p, _i, _p, _f, _p, _p, _sz, _p]
+lib.falqon_proxy_update_scored.restype = _i
+lib.falqon_proxy_update_scored.argtypes = [C.POINTER(falqon_layer), _i64, _p, _p, _sz, _p]
+lib.falqon_proxy_update_scored_batched.restype = _i
+lib.falqon_proxy_update_scored_batched.argtypes = [C.POINTER(falqon_layer), C.c_int32, C.POINTER(_i64), C.POINTER(_p), C.POINTER(_p),
+                                                   C.POINTER(_sz), _p]
 lib.falqon_melded_backward_dx.restype = _i
 lib.falqon_melded_backward_dx.argtypes = [C.POINTER(falqon_layer), _i64, _p, _i, _p, _sz, _p]
 lib.falqon_melded_forward_codes.restype = _i
@@ -339,6 +347,36 @@ def melded_backward(layer: Layer, dY: torch.Tensor, OA: torch.Tensor, amax_oa: t
     return dX, dB, s_g
 
 
+def melded_backward_update(layer: Layer, dY: torch.Tensor, OA: torch.Tensor, amax_oa: torch.Tensor, lr: float, need_dx: bool = True,
+                           dx_dtype=torch.bfloat16, ws: torch.Tensor | None = None, out=None, amax_dy: torch.Tensor | None = None):
+    """falqon_melded_backward_update: the backward with the plain-SGD step on the DeltaBuffer and the row scores fused into
+    the adapter-gradient kernel (the scores stay in the workspace for proxy_update_scored).  Returns (dX or None, dB, s_g)."""
+    T = dY.shape[0]
+    dev = dY.device
+    ws = layer.workspace(T) if ws is None else ws
+    if out is None:
+        dX = torch.empty((T, layer.n), dtype=dx_dtype, device=dev) if need_dx else None
+        dB = torch.empty((layer.m, layer.r), dtype=torch.float32, device=dev)
+        s_g = torch.empty(1, dtype=torch.float32, device=dev)
+    else:
+        dX, dB, s_g = out
+    _check("falqon_melded_backward_update",
+           lib.falqon_melded_backward_update(C.byref(layer.c), _ptr(dY), _dt(dY), _ptr(amax_dy), T, _ptr(OA), _ptr(amax_oa), _ptr(dX),
+                                             _dt(dX) if dX is not None else BF16, _ptr(dB), lr, _ptr(s_g), _ptr(ws), ws.numel(),
+                                             _stream()))
+    return dX, dB, s_g
+
+
+def proxy_update_scored(layer: Layer, k: int, ws: torch.Tensor | None = None, idx_out: torch.Tensor | None = None):
+    """falqon_proxy_update_scored: selection and merge from the scores melded_backward_update left in the workspace."""
+    ws = layer.workspace(1) if ws is None else ws
+    if idx_out is None and 0 < k <= layer.m:
+        idx_out = torch.empty(k, dtype=torch.int32, device=layer.wq.device)
+    _check("falqon_proxy_update_scored", lib.falqon_proxy_update_scored(C.byref(layer.c), k, _ptr(idx_out), _ptr(ws), ws.numel(),
+                                                                        _stream()))
+    return idx_out
+
+
 def melded_backward_dx(layer: Layer, T: int, dx_dtype=torch.bfloat16, ws: torch.Tensor | None = None, out: torch.Tensor | None = None):
     """falqon_melded_backward_dx: dX [T, n] from the gradient codes the preceding melded_backward(need_dx=False) on the same
     workspace left behind."""
@@ -416,6 +454,13 @@ class ProxyBatch:
         _check("falqon_proxy_update_batched_adamw",
                lib.falqon_proxy_update_batched_adamw(self.c_layers, self.count, self.c_dB, c_ea, c_es, C.byref(hp), self.c_k,
                                                      self.c_idx, self.c_ws, self.c_ws_bytes, _stream()))
+        return self.idx_outs
+
+    def run_scored(self):
+        """falqon_proxy_update_scored_batched: selection and merge only, after melded_backward_update on every layer."""
+        _check("falqon_proxy_update_scored_batched",
+               lib.falqon_proxy_update_scored_batched(self.c_layers, self.count, self.c_k, self.c_idx, self.c_ws, self.c_ws_bytes,
+                                                      _stream()))
         return self.idx_outs
 
     def run(self, lr: float):

@@ -309,9 +309,11 @@ int falqon_melded_forward_codes(const falqon_layer* L, const uint8_t* xq, const 
 
 namespace {
 // amax_dy (nullable, device [1]; per-tensor layers only): max |dY| is already known, see forward_impl.
+// sgd_lr (nullable, host): also run Alg. 3 line 4 in its plain-SGD form and the row scores (into the workspace's score region),
+// inside the dB kernel where its shared memory has the room, else as the separate pass.
 int backward_impl(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, const float* amax_dy, int64_t T, const float* OA,
                   const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, float* s_g_out, void* ws, size_t ws_bytes,
-                  falqon_stream stream, int dump_block = -1) {
+                  falqon_stream stream, int dump_block = -1, const float* sgd_lr = nullptr) {
   if (!layer_ok(L) || dY == nullptr || OA == nullptr || amax_oa == nullptr || dB == nullptr || T < 1 || !dtype_ok(dy_dt) ||
       !dtype_ok(dx_dt) || !aligned16(dY) || !aligned16(OA) || !aligned16(dB) || (dX != nullptr && !aligned16(dX)))
     return FALQON_ERR_INVALID_ARG;
@@ -359,8 +361,16 @@ int backward_impl(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, con
     d.m = m; d.r = r; d.T = T;
     d.gq = gq; d.oaq_t = oaq_t; d.ldt = w.t16; d.s_oa = scales + 5;
     d.s_g = scales + 3; d.row_mul = nullptr; d.dB = dB; d.status = status;
-    StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
-    FALQON_CUDA(launch_db_fused(d, stream));
+    const bool fuse_update = sgd_lr != nullptr && db_fused_update_fits(m, r, T);
+    if (fuse_update) { d.dbuf = L->dbuf; d.score = reinterpret_cast<float*>(base + w.score); d.neg_lr = -*sgd_lr; }
+    {
+      StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
+      FALQON_CUDA(launch_db_fused(d, stream));
+    }
+    if (sgd_lr != nullptr && !fuse_update) {
+      StageTimer timer(FALQON_STAGE_SGD_SCORE, stream);
+      FALQON_CUDA(launch_sgd_score(L->dbuf, dB, *sgd_lr, m, r, reinterpret_cast<float*>(base + w.score), stream));
+    }
     return FALQON_OK;
   }
   // S3: g~, s_g = Q_e5m2(dY)
@@ -389,8 +399,16 @@ int backward_impl(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, con
     d.m = m; d.r = r; d.T = T;
     d.gq = gq; d.oaq_t = oaq_t; d.ldt = w.t16; d.s_oa = scales + 5;
     d.s_g = scales + 3; d.row_mul = per_row ? L->s_w : nullptr; d.dB = dB; d.status = status;
-    StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
-    FALQON_CUDA(launch_db_fused(d, stream));
+    const bool fuse_update = sgd_lr != nullptr && db_fused_update_fits(m, r, T);
+    if (fuse_update) { d.dbuf = L->dbuf; d.score = reinterpret_cast<float*>(base + w.score); d.neg_lr = -*sgd_lr; }
+    {
+      StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
+      FALQON_CUDA(launch_db_fused(d, stream));
+    }
+    if (sgd_lr != nullptr && !fuse_update) {
+      StageTimer timer(FALQON_STAGE_SGD_SCORE, stream);
+      FALQON_CUDA(launch_sgd_score(L->dbuf, dB, *sgd_lr, m, r, reinterpret_cast<float*>(base + w.score), stream));
+    }
   }
   // S4: dX = g~ W~ / (s_W s_g)   (contraction over the m output channels; W~ read MN-major)
   if (dX != nullptr) {
@@ -415,6 +433,14 @@ int falqon_melded_backward(const falqon_layer* L, const void* dY, falqon_dtype d
                            const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, float* s_g_out, void* ws,
                            size_t ws_bytes, falqon_stream stream) {
   return backward_impl(L, dY, dy_dt, nullptr, T, OA, amax_oa, dX, dx_dt, dB, s_g_out, ws, ws_bytes, stream);
+}
+
+int falqon_melded_backward_update(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, const float* amax_dy, int64_t T,
+                                  const float* OA, const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, float lr,
+                                  float* s_g_out, void* ws, size_t ws_bytes, falqon_stream stream) {
+  if (!(lr == lr)) return FALQON_ERR_INVALID_ARG;
+  if (amax_dy != nullptr && L != nullptr && L->gran == FALQON_PER_ROW) return FALQON_ERR_UNSUPPORTED;
+  return backward_impl(L, dY, dy_dt, amax_dy, T, OA, amax_oa, dX, dx_dt, dB, s_g_out, ws, ws_bytes, stream, -1, &lr);
 }
 
 int falqon_melded_backward_dx(const falqon_layer* L, int64_t T, void* dX, falqon_dtype dx_dt, void* ws, size_t ws_bytes,
@@ -466,7 +492,7 @@ struct ExactMergeArgs {
 };
 int proxy_update_impl(const falqon_layer* L, const float* dB, float lr, const falqon_adamw* adamw, float* exp_avg,
                       float* exp_avg_sq, int64_t k, int32_t* idx_out, void* ws, size_t ws_bytes, falqon_stream stream,
-                      const ExactMergeArgs* exact = nullptr) {
+                      const ExactMergeArgs* exact = nullptr, bool scored = false) {
   if (!layer_ok(L) || k < 0 || k > L->m || !(lr == lr) || (dB != nullptr && !aligned16(dB)))
     return FALQON_ERR_INVALID_ARG;
   WorkspaceLayout w;
@@ -481,7 +507,9 @@ int proxy_update_impl(const falqon_layer* L, const float* dB, float lr, const fa
   const bool fused_merge = static_cast<size_t>(merge_group_count(k)) <= kMaxMergeGroups;
   {
     StageTimer timer(FALQON_STAGE_SGD_SCORE, stream);   // optimizer step, scores and (k > 0) the selection: one kernel
-    if (adamw != nullptr) {
+    if (scored) {    // the scores of the current DeltaBuffer are in the workspace already: selection only
+      if (k > 0) FALQON_CUDA(launch_topk(score, m, k, sel, idx_out, stream));
+    } else if (adamw != nullptr) {
       FALQON_CUDA(launch_adamw_score_topk(L->dbuf, dB, exp_avg, exp_avg_sq, adamw->lr, adamw->beta1, adamw->beta2, adamw->eps,
                                           adamw->weight_decay, adamw->step, m, r, k, score, sel, idx_out, done_counter, stream));
     } else {
@@ -514,6 +542,11 @@ int falqon_proxy_update(const falqon_layer* L, const float* dB, float lr, int64_
   return proxy_update_impl(L, dB, lr, nullptr, nullptr, nullptr, k, idx_out, ws, ws_bytes, stream);
 }
 
+int falqon_proxy_update_scored(const falqon_layer* L, int64_t k, int32_t* idx_out, void* ws, size_t ws_bytes,
+                               falqon_stream stream) {
+  return proxy_update_impl(L, nullptr, 0.0f, nullptr, nullptr, nullptr, k, idx_out, ws, ws_bytes, stream, nullptr, true);
+}
+
 namespace {
 bool adamw_ok(const falqon_adamw* hp) {
   return hp != nullptr && hp->step >= 1 && hp->lr == hp->lr && hp->beta1 >= 0.0f && hp->beta1 < 1.0f && hp->beta2 >= 0.0f &&
@@ -523,15 +556,15 @@ bool adamw_ok(const falqon_adamw* hp) {
 // hp == null: plain SGD with lr.  hp != null: AdamW on every layer (dB, exp_avg, exp_avg_sq all required).
 int proxy_update_batched_impl(const falqon_layer* layers, int32_t count, const float* const* dB, float lr, const falqon_adamw* hp,
                               float* const* exp_avg, float* const* exp_avg_sq, const int64_t* k, int32_t* const* idx_out,
-                              void* const* ws, const size_t* ws_bytes, falqon_stream stream) {
+                              void* const* ws, const size_t* ws_bytes, falqon_stream stream, bool scored = false) {
   if (count < 0 || !(lr == lr)) return FALQON_ERR_INVALID_ARG;
   if (count == 0) return FALQON_OK;
-  if (layers == nullptr || dB == nullptr || k == nullptr || ws == nullptr || ws_bytes == nullptr) return FALQON_ERR_INVALID_ARG;
+  if (layers == nullptr || (dB == nullptr && !scored) || k == nullptr || ws == nullptr || ws_bytes == nullptr) return FALQON_ERR_INVALID_ARG;
   if (hp != nullptr && (exp_avg == nullptr || exp_avg_sq == nullptr)) return FALQON_ERR_INVALID_ARG;
   bool fused = true;
   for (int32_t i = 0; i < count; ++i) {
     const falqon_layer* L = &layers[i];
-    if (!layer_ok(L) || k[i] < 0 || k[i] > L->m || (dB[i] != nullptr && !aligned16(dB[i]))) return FALQON_ERR_INVALID_ARG;
+    if (!layer_ok(L) || k[i] < 0 || k[i] > L->m || (!scored && dB[i] != nullptr && !aligned16(dB[i]))) return FALQON_ERR_INVALID_ARG;
     if (hp != nullptr && (dB[i] == nullptr || exp_avg[i] == nullptr || exp_avg_sq[i] == nullptr || !aligned16(exp_avg[i]) ||
                           !aligned16(exp_avg_sq[i])))
       return FALQON_ERR_INVALID_ARG;
@@ -544,9 +577,9 @@ int proxy_update_batched_impl(const falqon_layer* layers, int32_t count, const f
   }
   if (!fused) {
     for (int32_t i = 0; i < count; ++i) {
-      const int rc = proxy_update_impl(&layers[i], dB[i], lr, hp, hp != nullptr ? exp_avg[i] : nullptr,
+      const int rc = proxy_update_impl(&layers[i], scored ? nullptr : dB[i], lr, hp, hp != nullptr ? exp_avg[i] : nullptr,
                                        hp != nullptr ? exp_avg_sq[i] : nullptr, k[i], idx_out != nullptr ? idx_out[i] : nullptr,
-                                       ws[i], ws_bytes[i], stream);
+                                       ws[i], ws_bytes[i], stream, nullptr, scored);
       if (rc != FALQON_OK) return rc;
     }
     return FALQON_OK;
@@ -566,7 +599,8 @@ int proxy_update_batched_impl(const falqon_layer* layers, int32_t count, const f
       uint8_t* base = static_cast<uint8_t*>(ws[i]);
       b[c].wq = L->wq;
       b[c].dbuf = L->dbuf;
-      b[c].dB = dB[i];
+      b[c].dB = scored ? nullptr : dB[i];
+      b[c].scored = scored;
       b[c].exp_avg = hp != nullptr ? exp_avg[i] : nullptr;
       b[c].exp_avg_sq = hp != nullptr ? exp_avg_sq[i] : nullptr;
       b[c].row_scales = L->gran == FALQON_PER_ROW ? L->s_w : nullptr;
@@ -595,6 +629,11 @@ int proxy_update_batched_impl(const falqon_layer* layers, int32_t count, const f
 int falqon_proxy_update_batched(const falqon_layer* layers, int32_t count, const float* const* dB, float lr, const int64_t* k,
                                 int32_t* const* idx_out, void* const* ws, const size_t* ws_bytes, falqon_stream stream) {
   return proxy_update_batched_impl(layers, count, dB, lr, nullptr, nullptr, nullptr, k, idx_out, ws, ws_bytes, stream);
+}
+
+int falqon_proxy_update_scored_batched(const falqon_layer* layers, int32_t count, const int64_t* k, int32_t* const* idx_out,
+                                       void* const* ws, const size_t* ws_bytes, falqon_stream stream) {
+  return proxy_update_batched_impl(layers, count, nullptr, 0.0f, nullptr, nullptr, nullptr, k, idx_out, ws, ws_bytes, stream, true);
 }
 
 int falqon_proxy_update_batched_adamw(const falqon_layer* layers, int32_t count, const float* const* dB, float* const* exp_avg,
@@ -735,6 +774,9 @@ int falqon_launch_count(const char* entry_point, int64_t m, int64_t n, int64_t r
   if (std::strcmp(entry_point, "falqon_melded_backward:fused") == 0) return 5;
   if (std::strcmp(entry_point, "falqon_proxy_update") == 0) return k > 0 ? 2 : 1;  // optimizer+score+top-k, merge+clear
   if (std::strcmp(entry_point, "falqon_proxy_update_batched") == 0) return k > 0 ? 2 : 1;   // per 8 layers
+  if (std::strcmp(entry_point, "falqon_melded_backward_update") == 0) return 3;   // as the backward; the update rides in the dB kernel
+  if (std::strcmp(entry_point, "falqon_proxy_update_scored") == 0) return k > 0 ? 2 : 0;
+  if (std::strcmp(entry_point, "falqon_proxy_update_scored_batched") == 0) return k > 0 ? 2 : 0;
   if (std::strcmp(entry_point, "falqon_proxy_update_static") == 0) return k > 0 ? 4 : 1;   // optimizer+score, top-k, merge, clear (+ one copy of idx)
   return 0;
 }

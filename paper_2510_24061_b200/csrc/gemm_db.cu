@@ -33,7 +33,10 @@ struct DbParams {
   const float* s_oa;        // [1]
   const float* s_g;         // [1]
   const float* row_mul;     // nullable [m]
-  float* dB;                // [m][r]
+  float* dB;                // [m][r], nullable when the update below is fused
+  float* dbuf;              // nullable [m][r]: DeltaBuffer <- fma(neg_lr, dB, DeltaBuffer) (Alg. 3 line 4, plain SGD) ...
+  float* score;             // ... and [m]: score_i = sum_j |DeltaBuffer_ij|, fp32, j ascending
+  float neg_lr;
   int* status;
 };
 
@@ -156,18 +159,33 @@ db_fused_kernel(const __grid_constant__ CUtensorMap tmap_g, const __grid_constan
 
   // ------------------------------------------------------------ slab sum across the cluster (every thread passes
   // both cluster barriers, also after a timeout, so that no CTA of the cluster is left waiting)
+  constexpr int kU = 4;   // positions per thread whose loads (all slabs) are issued before the first add
+  const int tidc = static_cast<int>(threadIdx.x) - 64;
+  const int rows_per_cta = (kDbBlock + p.splits - 1) / p.splits;
+  const int r4 = p.r >> 2;
+  const int row_begin = split * rows_per_cta;
+  const int row_end = min(row_begin + rows_per_cta, kDbBlock);
+  // fused optimizer step: the DeltaBuffer values of this thread's first positions are fetched before the cluster barrier,
+  // so their latency overlaps the wait for the other slabs
+  float4 dpre[kU];
+  if (warp >= 2 && p.dbuf != nullptr) {
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const int e = tidc + u * kDbEpilogueWarps * 32;
+      const int row = m_idx * kDbBlock + row_begin + e / r4;
+      dpre[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (e < (row_end - row_begin) * r4 && row < p.m)
+        dpre[u] = ld_stream(reinterpret_cast<const float4*>(p.dbuf + static_cast<long long>(row) * p.r + 4 * (e % r4)));
+    }
+  }
   cluster_arrive();
   cluster_wait();
   if (warp >= 2) {
-    const int tidc = static_cast<int>(threadIdx.x) - 64;
-    const int rows_per_cta = (kDbBlock + p.splits - 1) / p.splits;
-    const int r4 = p.r >> 2;
-    const int row_begin = split * rows_per_cta;
-    const int row_end = min(row_begin + rows_per_cta, kDbBlock);
     const float inv = 1.0f / (ld_stream(p.s_g) * ld_stream(p.s_oa));
     const uint32_t local = smem_base;   // the partial tile starts at the (1 KB aligned) base in every CTA of the cluster
     const int total = (row_end - row_begin) * r4;
-    constexpr int kU = 4;   // positions per thread whose loads (all slabs) are issued before the first add
+    // fused optimizer step: |DeltaBuffer| of this CTA's rows, behind the partial tile, row pitch r + 1 floats
+    float* abs_rows = reinterpret_cast<float*>(smem_gen) + kDbBlock * (p.r + 4);
     for (int e0 = tidc; e0 < total; e0 += kU * kDbEpilogueWarps * 32) {
       float4 y[kU][kDbMaxSplits];
 #pragma unroll
@@ -195,7 +213,28 @@ db_fused_kernel(const __grid_constant__ CUtensorMap tmap_g, const __grid_constan
           const float f = ld_stream(p.row_mul + row);
           acc.x *= f; acc.y *= f; acc.z *= f; acc.w *= f;
         }
-        *reinterpret_cast<float4*>(p.dB + static_cast<long long>(row) * p.r + 4 * c4) = acc;
+        if (p.dB != nullptr) *reinterpret_cast<float4*>(p.dB + static_cast<long long>(row) * p.r + 4 * c4) = acc;
+        if (p.dbuf != nullptr) {   // one fma per element on the value dB holds, exactly as the separate pass would
+          float4* dp = reinterpret_cast<float4*>(p.dbuf + static_cast<long long>(row) * p.r + 4 * c4);
+          float4 d = e0 == tidc ? dpre[u] : ld_stream(dp);
+          d.x = __fmaf_rn(p.neg_lr, acc.x, d.x); d.y = __fmaf_rn(p.neg_lr, acc.y, d.y);
+          d.z = __fmaf_rn(p.neg_lr, acc.z, d.z); d.w = __fmaf_rn(p.neg_lr, acc.w, d.w);
+          *dp = d;
+          float* a = abs_rows + (row_l - row_begin) * (p.r + 1) + 4 * c4;
+          a[0] = fabsf(d.x); a[1] = fabsf(d.y); a[2] = fabsf(d.z); a[3] = fabsf(d.w);
+        }
+      }
+    }
+    if (p.dbuf != nullptr) {
+      asm volatile("bar.sync 1, %0;" ::"n"(kDbEpilogueWarps * 32) : "memory");   // the four epilogue warps only
+      const int row_l = row_begin + tidc;
+      const int row = m_idx * kDbBlock + row_l;
+      if (row_l < row_end && row < p.m) {
+        const float* a = abs_rows + tidc * (p.r + 1);
+        float sc = 0.0f;
+#pragma unroll 8
+        for (int j = 0; j < p.r; ++j) sc = __fadd_rn(sc, a[j]);   // strictly left to right
+        p.score[row] = sc;
       }
     }
   }
@@ -217,6 +256,28 @@ db_fused_kernel(const __grid_constant__ CUtensorMap tmap_g, const __grid_constan
 
 }  // namespace
 
+namespace {
+int db_splits(int64_t m, int64_t T) {
+  const int m_tiles = static_cast<int>((m + kDbBlock - 1) / kDbBlock);
+  const int kblocks = static_cast<int>((T + kDbBlock - 1) / kDbBlock);
+  // slabs per row tile = cluster size: a power of two up to kDbMaxSplits, enough for two CTAs on every SM
+  const int want = (2 * sm_count() + m_tiles - 1) / m_tiles;
+  int splits = 1;
+  while (splits * 2 <= kDbMaxSplits && splits * 2 <= want && splits * 2 <= kblocks) splits *= 2;
+  return splits;
+}
+}  // namespace
+
+// The fused optimizer step parks |DeltaBuffer| of a CTA's rows behind the 128 x (r + 4) partial tile, inside the drained
+// operand ring; it needs that much room.
+bool db_fused_update_fits(int64_t m, int64_t r, int64_t T) {
+  const int splits = db_splits(m, T);
+  const int64_t r16 = round_up(r, 16);
+  const int64_t ring = static_cast<int64_t>(kDbStages) * (kDbATileBytes + r16 * kDbBlock);
+  const int64_t rows_per_cta = (kDbBlock + splits - 1) / splits;
+  return 4 * (kDbBlock * (r + 4) + rows_per_cta * (r + 1)) <= ring;
+}
+
 cudaError_t launch_db_fused(const DbFusedProblem& q, cudaStream_t stream) {
   if (q.m < 1 || q.T < 1 || q.r < 8 || q.r > 256 || q.r % 8) return cudaErrorInvalidValue;
   DbParams p{};
@@ -224,10 +285,7 @@ cudaError_t launch_db_fused(const DbFusedProblem& q, cudaStream_t stream) {
   p.T = q.T;
   p.m_tiles = static_cast<int>((q.m + kDbBlock - 1) / kDbBlock);
   p.kblocks_total = static_cast<int>((q.T + kDbBlock - 1) / kDbBlock);
-  // slabs per row tile = cluster size: a power of two up to 8, enough for two CTAs on every SM
-  const int want = (2 * sm_count() + p.m_tiles - 1) / p.m_tiles;
-  int splits = 1;
-  while (splits * 2 <= kDbMaxSplits && splits * 2 <= want && splits * 2 <= p.kblocks_total) splits *= 2;
+  const int splits = db_splits(q.m, q.T);
   p.splits = splits;
   p.kblocks_per_split = (p.kblocks_total + splits - 1) / splits;
   // instruction descriptor: fp32 accumulate, A = E5M2 MN-major, B = E4M3 K-major, N = r16, M = 128
@@ -238,6 +296,9 @@ cudaError_t launch_db_fused(const DbFusedProblem& q, cudaStream_t stream) {
   p.tmem_cols = cols;
   p.s_oa = q.s_oa;
   p.s_g = q.s_g; p.row_mul = q.row_mul; p.dB = q.dB; p.status = q.status;
+  p.dbuf = q.dbuf; p.score = q.score; p.neg_lr = q.neg_lr;
+  if ((q.dbuf != nullptr) != (q.score != nullptr) || (q.dbuf == nullptr && q.dB == nullptr)) return cudaErrorInvalidValue;
+  if (q.dbuf != nullptr && !db_fused_update_fits(q.m, q.r, q.T)) return cudaErrorInvalidValue;
   CUtensorMap tg, toa;
   if (!make_tensor_map(&tg, q.gq, q.T, q.m, q.m, kDbBlock, kDbBlock)) return cudaErrorInvalidValue;
   if (!make_tensor_map(&toa, q.oaq_t, p.r16, q.T, q.ldt, kDbBlock, static_cast<uint32_t>(p.r16))) return cudaErrorInvalidValue;

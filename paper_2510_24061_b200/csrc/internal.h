@@ -160,10 +160,15 @@ struct DbFusedProblem {
   const float* s_oa;           // [1]
   const float* s_g;            // [1]
   const float* row_mul;        // nullable [m]: dB row i is also multiplied by row_mul[i]
-  float* dB;                   // [m][r]
+  float* dB;                   // [m][r]; nullable when dbuf is given
   int* status;
+  // optional, together: the plain-SGD step of Alg. 3 line 4 and the row scores, in the kernel's slab-sum phase
+  float* dbuf;                 // [m][r]: DeltaBuffer <- fma(neg_lr, dB, DeltaBuffer)
+  float* score;                // [m]: sum_j |DeltaBuffer_ij|, fp32, j ascending
+  float neg_lr;
 };
 cudaError_t launch_db_fused(const DbFusedProblem& p, cudaStream_t stream);
+bool db_fused_update_fits(int64_t m, int64_t r, int64_t T);   // whether the fused step has room in the kernel's shared memory
 
 // ---- merge_exact.cu: the correctly rounded merge of the selected rows on the tensor cores (guard band + exact fallback).
 // scratch: exact_merge_scratch_bytes(m, n, r) bytes, no initialisation needed.  Clears the merged DeltaBuffer rows.
@@ -220,6 +225,7 @@ struct ProxyBatchLayer {
   unsigned int* done_counter;
   unsigned int* group_counters;
   int64_t m, n, r, k;
+  bool scored;                  // the optimizer step and the scores are done already (score holds them): selection only
 };
 // phase 0: optimizer step, scores and selection of every layer; phase 1: the merge of every layer with k > 0.
 // adamw == null: plain SGD with `lr`; else AdamW with these hyper-parameters on every layer (lr is then ignored).

@@ -308,6 +308,7 @@ struct BatchedScoreLayer {
   int32_t* idx_out;
   unsigned int* done_counter;
   int m, r, k, cta_begin;
+  int scored;      // scores are in place already: the layer's single CTA runs the selection only
 };
 struct BatchedScoreArgs {
   BatchedScoreLayer layer[kProxyBatchMax];
@@ -322,6 +323,11 @@ __global__ void __launch_bounds__(kTopkThreads) score_topk_batched_kernel(const 
 #pragma unroll 1
   for (int i = 1; i < args.count; ++i) l = static_cast<int>(blockIdx.x) >= args.layer[i].cta_begin ? i : l;
   const BatchedScoreLayer& a = args.layer[l];
+  if (a.scored) {
+    if (a.k > 0)
+      topk_block(a.score, a.m, a.k, a.sel_idx, a.idx_out, a.m <= kTopkSmemRows ? reinterpret_cast<uint32_t*>(fused_smem_dyn) : nullptr);
+    return;
+  }
   const int n_ctas = (a.m + kFusedScoreRows - 1) / kFusedScoreRows;
   OptimizerArgs opt = args.opt;
   if (a.dB == nullptr) opt.kind = 0;
@@ -789,8 +795,9 @@ cudaError_t launch_proxy_update_batched(const ProxyBatchLayer* layers, int count
     a.done_counter = L.done_counter;
     a.m = static_cast<int>(L.m); a.r = static_cast<int>(L.r); a.k = static_cast<int>(L.k);
     a.cta_begin = score_ctas;
-    score_ctas += static_cast<int>((L.m + kFusedScoreRows - 1) / kFusedScoreRows);
-    size_t smem = sizeof(float) * kFusedScoreRows * (L.r + 1);
+    a.scored = L.scored ? 1 : 0;
+    score_ctas += L.scored ? 1 : static_cast<int>((L.m + kFusedScoreRows - 1) / kFusedScoreRows);
+    size_t smem = L.scored ? 0 : sizeof(float) * kFusedScoreRows * (L.r + 1);
     if (L.m <= kTopkSmemRows && static_cast<size_t>(L.m) * sizeof(uint32_t) > smem) smem = static_cast<size_t>(L.m) * sizeof(uint32_t);
     if (smem > score_smem) score_smem = smem;
   }
