@@ -493,6 +493,31 @@ int orc_adamw_step(float* p, const float* g, float* exp_avg, float* exp_avg_sq, 
   return 0;
 }
 
+// ---- "update A" variant (the paper's ablation with a trainable A: dL/dA = B^T dL/dO x^T).
+// A plain product of two matrices of FP8 codes, both stored with the contraction index innermost, in double:
+//   out[i][j] = sum_k dec_a(a[i][k]) * dec_b(b[j][k]) / (s_a * s_b)
+int orc_codes_gemm(const uint8_t* a, int fmt_a, float s_a, const uint8_t* b, int fmt_b, float s_b, int64_t M, int64_t N,
+                   int64_t K, double* out) {
+  if (M < 0 || N < 0 || K < 0) return -1;
+  const DecodeTable ta(fmt_a), tb(fmt_b);
+  const double d = (double)s_a * (double)s_b;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int64_t i = 0; i < M; ++i) {
+    for (int64_t j = 0; j < N; ++j) {
+      double acc = 0.0;
+      for (int64_t k = 0; k < K; ++k) acc += ta.v[a[i * K + k]] * tb.v[b[j * K + k]];
+      out[i * N + j] = acc / d;
+    }
+  }
+  return 0;
+}
+
+// Plain SGD on an fp32 tensor: p[e] = fma(-lr, g[e], p[e]), one rounding per element.
+int orc_sgd_step(float* p, const float* g, float lr, int64_t count) {
+  for (int64_t e = 0; e < count; ++e) p[e] = std::fmaf(-lr, g[e], p[e]);
+  return 0;
+}
+
 int orc_num_threads(void) {
   int nthreads = 1;
 #ifdef _OPENMP

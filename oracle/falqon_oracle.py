@@ -52,6 +52,10 @@ _lib.orc_quantize_colscaled.restype = _i32
 _lib.orc_quantize_colscaled.argtypes = [_p, _i32, _i64, _i64, _i32, _p, _p, _p, _p]
 _lib.orc_adamw_step.restype = _i32
 _lib.orc_adamw_step.argtypes = [_p, _p, _p, _p, _i64, _f32, _f32, _f32, _f32, _f32, _i64]
+_lib.orc_codes_gemm.restype = _i32
+_lib.orc_codes_gemm.argtypes = [_p, _i32, _f32, _p, _i32, _f32, _i64, _i64, _i64, _p]
+_lib.orc_sgd_step.restype = _i32
+_lib.orc_sgd_step.argtypes = [_p, _p, _f32, _i64]
 _lib.orc_num_threads.restype = _i32
 
 
@@ -319,3 +323,47 @@ def layer_backward(dY, OA, wq, s_w, m: int, r: int):
     dX = dx_gemm(gq, s_g, wq, s_w, m)
     dB = db_gemm(gq, s_g, oaq, s_oa, row_scale=np.asarray(s_w)[:m] if per_row else None)
     return dict(gq=gq, s_g=s_g, oaq=oaq, s_oa=s_oa, dX=dX, dB=dB)
+
+
+# ---- the "update A" variant (the paper's ablation with a trainable A) ----
+
+def codes_gemm(a, fmt_a: int, s_a, b, fmt_b: int, s_b) -> np.ndarray:
+    """out[i, j] = sum_k dec(a[i, k]) dec(b[j, k]) / (s_a s_b) in float64; a uint8 [M, K], b uint8 [N, K]."""
+    a, b = _c(a, np.uint8), _c(b, np.uint8)
+    M, K = a.shape
+    N = b.shape[0]
+    assert b.shape[1] == K
+    out = np.empty((M, N), dtype=np.float64)
+    rc = _lib.orc_codes_gemm(_ptr(a), fmt_a, float(np.float32(s_a)), _ptr(b), fmt_b, float(np.float32(s_b)), M, N, K, _ptr(out))
+    assert rc == 0
+    return out
+
+
+def sgd_step(p, g, lr: float):
+    """In place: p = fma(-lr, g, p) element by element (float32)."""
+    assert p.dtype == np.float32 and p.flags.c_contiguous
+    g = _c(g, np.float32)
+    assert g.size == p.size
+    assert _lib.orc_sgd_step(_ptr(p), _ptr(g), float(np.float32(lr)), p.size) == 0
+
+
+def update_a(gq, s_g, xq, s_x, B, A_master, wq, s_w, gamma: float, lr: float, m: int, r: int):
+    """One step of a trainable A (the paper's appendix ablation: dL/dA = B^T dL/dO x^T), in the same FP8 scheme as the
+    rest of the layer.  gq [T, m] E5M2 codes of dY with scale s_g and xq [T, n] E4M3 codes of X with scale s_x are the
+    operands the backward and the forward already cast.  Steps, in this order:
+      B~, s_B = Q_e4m3(B)                       (per tensor; B fp32 [m, r] is the caller's record of the adapter's B)
+      P = g~ B~ / (s_g s_B)                     ([T, r]: dY B, contraction over the m outputs), rounded to fp32
+      P~, s_P = Q_e4m3(P)                       (per tensor)
+      dA = P~^T x~ / (s_P s_x)                  ([r, n], contraction over the tokens), rounded to fp32
+      A_master = fma(-lr, dA, A_master)         (fp32 master copy of A, [r, n], in place)
+      A~ = Q_e4m3(gamma * A_master; s_W)        (written over rows m.. of wq; Eq. A_integ)
+    Rows of W~ merged earlier keep the products with the A~ of their time.  Returns a dict of the intermediates."""
+    B = _c(B, np.float32)
+    Bq, s_B, _ = quantize(B, E4M3)
+    P = codes_gemm(gq, E5M2, s_g, np.ascontiguousarray(Bq.T), E4M3, s_B).astype(np.float32)
+    Pq, s_P, amax_P = quantize(P, E4M3)
+    dA = codes_gemm(np.ascontiguousarray(Pq.T), E4M3, s_P, np.ascontiguousarray(_c(xq, np.uint8).T), E4M3, s_x).astype(np.float32)
+    sgd_step(A_master, dA, lr)
+    Aq, _, _ = quantize(A_master, E4M3, scale_in=s_w, premul=gamma)
+    wq[m:m + r] = Aq
+    return dict(Bq=Bq, s_B=s_B, P=P, Pq=Pq, s_P=s_P, amax_P=amax_P, dA=dA)
