@@ -352,6 +352,31 @@ int falqon_proxy_update_exact(const falqon_layer *L, const float *dB, float lr, 
                               size_t ws_bytes, void *scratch, size_t scratch_bytes, float *sums_out,
                               uint32_t *fix_count_out, falqon_stream stream);
 
+/* The "update A" variant (the paper's appendix ablation with a trainable A; an extension: the melded scheme freezes A):
+ *     dL/dA = B^T dL/dO x^T
+ * evaluated in the layer's FP8 scheme and applied, after the backward of the same step, in this order:
+ *     B~, s_B = Q_e4m3(B)                    per tensor; B: device [m][r] fp32, the caller's record of the adapter's B
+ *                                            (the melded scheme keeps none: whatever the caller accumulates)
+ *     P = g~ B~ / (s_g s_B)                  [T][r] fp32, g~ and s_g as the backward left them in the workspace
+ *     P~, s_P = Q_e4m3(P)                    per tensor
+ *     dA = P~^T x~ / (s_P s_x)               [r][n] fp32 (kept transposed, [n][r], in the scratch)
+ *     A_master <- fma(-lr, dA, A_master)     device [r][n] fp32, the master copy of A, in place (fold gamma into lr)
+ *     A~ <- Q_e4m3(gamma * A_master; s_W)    over rows m .. m+r-1 of L->wq (Eq. A_integ)
+ * Rows of W~ merged earlier keep the products with the A~ of their time.  Per-tensor scaled layers only.
+ *   xq, s_x   device [T][n] E4M3 codes of the step's X and their scale [1]: a copy the caller kept from the forward
+ *             (FALQON_WS_XQ / entry 1 of FALQON_WS_SCALES; the backward reuses that workspace region for g~)
+ *   ws        the layer's workspace, holding g~ and s_g of falqon_melded_backward for the same T
+ *   scratch   device, falqon_update_a_scratch_bytes(m, n, r, T) bytes, no initialisation needed; afterwards its
+ *             regions (falqon_update_a_region) hold the intermediates: FALQON_UA_SCALARS float [4] = amax(B), s_B,
+ *             amax(P), s_P; FALQON_UA_BQ_T uint8 [r16][m] codes of B transposed; FALQON_UA_P float [T][r];
+ *             FALQON_UA_PQ_T uint8 [r16][T16] codes of P transposed; FALQON_UA_DA_T float [n][r] = dA transposed.
+ * Returns FALQON_OK, _INVALID_ARG, _UNSUPPORTED (per-row layer), _WORKSPACE or _CUDA. */
+typedef enum { FALQON_UA_SCALARS = 0, FALQON_UA_BQ_T = 1, FALQON_UA_P = 2, FALQON_UA_PQ_T = 3, FALQON_UA_DA_T = 4 } falqon_ua_region;
+size_t falqon_update_a_scratch_bytes(int64_t m, int64_t n, int64_t r, int64_t T);
+int falqon_update_a_region(int64_t m, int64_t n, int64_t r, int64_t T, falqon_ua_region which, size_t *offset, size_t *bytes);
+int falqon_update_a(const falqon_layer *L, const uint8_t *xq, const float *s_x, const float *B, float *A_master, float gamma,
+                    float lr, int64_t T, void *ws, size_t ws_bytes, void *scratch, size_t scratch_bytes, falqon_stream stream);
+
 /* Synchronizes `stream`, then returns and clears the device status word of the current device:
  * FALQON_OK, FALQON_ERR_TIMEOUT (a bounded device-side wait ran out; results of that call are
  * undefined) or FALQON_ERR_CUDA (the synchronize itself failed). */

@@ -24,6 +24,7 @@ WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 EXPORTS = ["falqon_absmax", "falqon_selftest_wait_timeout", "falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax",
            "falqon_melded_forward_dump", "falqon_melded_backward_dump", "falqon_melded_backward_dx",
+           "falqon_update_a", "falqon_update_a_scratch_bytes", "falqon_update_a_region",
            "falqon_melded_backward_update", "falqon_proxy_update_scored", "falqon_proxy_update_scored_batched", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
            "falqon_svd_init_scratch_bytes", "falqon_svd_init", "falqon_tensor_ceiling", "falqon_tensor_ceiling_ctas",
            "falqon_melded_backward", "falqon_proxy_update", "falqon_proxy_update_batched", "falqon_proxy_update_batched_adamw", "falqon_last_device_status", "falqon_launch_count",
@@ -62,6 +63,12 @@ lib.falqon_melded_forward_dump.restype = _i
 lib.falqon_melded_forward_dump.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _i, _p, _p, _p, C.c_int32, _p, _sz, _p]
 lib.falqon_melded_backward_dump.restype = _i
 lib.falqon_melded_backward_dump.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _p, _p, _i, _p, _p, C.c_int32, _p, _sz, _p]
+lib.falqon_update_a_scratch_bytes.restype = _sz
+lib.falqon_update_a_scratch_bytes.argtypes = [_i64, _i64, _i64, _i64]
+lib.falqon_update_a_region.restype = _i
+lib.falqon_update_a_region.argtypes = [_i64, _i64, _i64, _i64, _i, C.POINTER(_sz), C.POINTER(_sz)]
+lib.falqon_update_a.restype = _i
+lib.falqon_update_a.argtypes = [C.POINTER(falqon_layer), _p, _p, _p, _p, _f, _f, _i64, _p, _sz, _p, _sz, _p]
 lib.falqon_melded_backward_update.restype = _i
 lib.falqon_melded_backward_update.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _p, _p, _i, _p, _f, _p, _p, _sz, _p]
 lib.falqon_proxy_update_scored.restype = _i
@@ -345,6 +352,31 @@ def melded_backward(layer: Layer, dY: torch.Tensor, OA: torch.Tensor, amax_oa: t
                                                                 _ptr(amax_oa), _ptr(dX), dx_dt, _ptr(dB), _ptr(s_g),
                                                                 _ptr(ws), ws.numel(), _stream()))
     return dX, dB, s_g
+
+
+UA_SCALARS, UA_BQ_T, UA_P, UA_PQ_T, UA_DA_T = range(5)
+
+
+def update_a(layer: Layer, xq: torch.Tensor, s_x: torch.Tensor, B: torch.Tensor, A_master: torch.Tensor, gamma: float, lr: float,
+             T: int, ws: torch.Tensor | None = None, scratch: torch.Tensor | None = None) -> torch.Tensor:
+    """falqon_update_a: one SGD step of a trainable A after the backward of the same step (in place on A_master fp32 [r, n]
+    and on the A~ rows of layer.wq).  xq uint8 [T, n], s_x fp32 [1]: the forward's codes of X, kept by the caller; B fp32
+    [m, r].  Returns the scratch tensor; ua_view gives its regions."""
+    assert xq.dtype == torch.uint8 and xq.is_contiguous() and B.dtype == torch.float32 and B.is_contiguous()
+    assert A_master.dtype == torch.float32 and A_master.is_contiguous() and A_master.shape == (layer.r, layer.n)
+    ws = layer.workspace(T) if ws is None else ws
+    if scratch is None:
+        scratch = torch.empty(int(lib.falqon_update_a_scratch_bytes(layer.m, layer.n, layer.r, T)), dtype=torch.uint8,
+                              device=layer.wq.device)
+    _check("falqon_update_a", lib.falqon_update_a(C.byref(layer.c), _ptr(xq), _ptr(s_x), _ptr(B), _ptr(A_master), gamma, lr, T,
+                                                  _ptr(ws), ws.numel(), _ptr(scratch), scratch.numel(), _stream()))
+    return scratch
+
+
+def ua_view(layer: Layer, scratch: torch.Tensor, T: int, which: int) -> torch.Tensor:
+    off, size = _sz(), _sz()
+    _check("falqon_update_a_region", lib.falqon_update_a_region(layer.m, layer.n, layer.r, T, which, C.byref(off), C.byref(size)))
+    return scratch[off.value:off.value + size.value]
 
 
 def melded_backward_update(layer: Layer, dY: torch.Tensor, OA: torch.Tensor, amax_oa: torch.Tensor, lr: float, need_dx: bool = True,

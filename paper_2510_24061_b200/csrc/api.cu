@@ -24,6 +24,10 @@ int* status_ptr() {   // of the current device; host threads may race here: ever
   return cached;
 }
 
+}  // namespace
+int* device_status_ptr() { return status_ptr(); }
+namespace {
+
 struct WorkspaceLayout {
   size_t scales, act8, oaq_t, score, sel_idx, inv_sw, col_scale, total;
   size_t act8_bytes, oaq_t_bytes, score_bytes, sel_idx_bytes, inv_sw_bytes, col_scale_bytes;

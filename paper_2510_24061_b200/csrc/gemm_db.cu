@@ -289,7 +289,7 @@ cudaError_t launch_db_fused(const DbFusedProblem& q, cudaStream_t stream) {
   p.splits = splits;
   p.kblocks_per_split = (p.kblocks_total + splits - 1) / splits;
   // instruction descriptor: fp32 accumulate, A = E5M2 MN-major, B = E4M3 K-major, N = r16, M = 128
-  p.idesc = (1u << 4) | (static_cast<uint32_t>(kE5M2) << 7) | (static_cast<uint32_t>(kE4M3) << 10) | (1u << 15) |
+  p.idesc = (1u << 4) | (static_cast<uint32_t>(q.g_is_e4m3 ? kE4M3 : kE5M2) << 7) | (static_cast<uint32_t>(kE4M3) << 10) | (1u << 15) |
             (static_cast<uint32_t>(p.r16 >> 3) << 17) | (static_cast<uint32_t>(kDbBlock >> 4) << 24);
   uint32_t cols = 32;
   while (cols < static_cast<uint32_t>(p.r16)) cols <<= 1;

@@ -69,6 +69,9 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// ---- api.cu: the device status word of the current device (bounded waits that run out report there), or nullptr
+int* device_status_ptr();
+
 // ---- quantize.cu
 constexpr int kMaxAbsmaxParts = 148 * 8;   // upper bound of the absmax grid = number of partial maxima
 // Pass 1 of per-tensor absmax scaling: one partial max (fp32 bit pattern of |x|) per CTA into partial[0..*nparts).
@@ -163,12 +166,16 @@ struct DbFusedProblem {
   float* dB;                   // [m][r]; nullable when dbuf is given
   int* status;
   // optional, together: the plain-SGD step of Alg. 3 line 4 and the row scores, in the kernel's slab-sum phase
+  bool g_is_e4m3;              // the [T][m] operand holds E4M3 codes (the update-A product reads x~ here) instead of E5M2
   float* dbuf;                 // [m][r]: DeltaBuffer <- fma(neg_lr, dB, DeltaBuffer)
   float* score;                // [m]: sum_j |DeltaBuffer_ij|, fp32, j ascending
   float neg_lr;
 };
 cudaError_t launch_db_fused(const DbFusedProblem& p, cudaStream_t stream);
 bool db_fused_update_fits(int64_t m, int64_t r, int64_t T);   // whether the fused step has room in the kernel's shared memory
+
+// ---- update_a.cu: p[j][c] = fma(-lr, g_t[c][j], p[j][c]) for p [rows][cols] and the transposed gradient g_t [cols][rows]
+cudaError_t launch_sgd_step_transposed(float* p, const float* g_t, float lr, int64_t rows, int64_t cols, cudaStream_t stream);
 
 // ---- merge_exact.cu: the correctly rounded merge of the selected rows on the tensor cores (guard band + exact fallback).
 // scratch: exact_merge_scratch_bytes(m, n, r) bytes, no initialisation needed.  Clears the merged DeltaBuffer rows.
