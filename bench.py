@@ -436,20 +436,51 @@ def run_stack(args):
     sampler = ClockSampler(0)
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        one_step()
-    e1.record()
-    torch.cuda.synchronize()
-    clocks = sampler.stop()
-    ms = e0.elapsed_time(e1) / steps
+
+    def soak(run, seconds):     # the same loop for `seconds` right before a timed region: the clocks of a long job
+        t0 = sampler.now()
+        while sampler.now() - t0 < seconds:
+            run()
+            e1.record()
+            e1.synchronize()
+        return sampler.window(t0, sampler.now())
+
+    def timed(run, n):
+        torch.cuda.synchronize()
+        t0 = sampler.now()
+        e0.record()
+        for _ in range(n):
+            run()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n, sampler.window(t0, sampler.now())
+
+    t_soak = sampler.now()
+    clocks_soak = soak(one_step, args.soak)
+    ms, clocks_timed = timed(one_step, steps)
+    clocks = sampler.window(t_soak, sampler.now())
+    clocks["soak_before"] = clocks_soak
+    clocks["timed_steps_only"] = clocks_timed
     # forward alone and backward (+ updates) alone, same protocol
-    e0.record()
-    for _ in range(steps):
-        stack.forward(h0)
-    e1.record()
-    torch.cuda.synchronize()
-    ms_f = e0.elapsed_time(e1) / steps
+    ms_f, _ = timed(lambda: stack.forward(h0), steps)
+    # where the step goes: the same step call by call with the library's stages bracketed by events (the brackets cost the
+    # launch overlap, so this pass is slower); what the brackets do not cover is the chain between the layers
+    eager = lambda: stack.step(h0, G)
+    soak(eager, min(args.soak, 1.0))
+    n_rec = 12 * 7 * n_layers * 2
+    fq.profile_start(n_rec, None)
+    ms_inst, clocks_inst = timed(eager, 2)
+    recs = fq.profile_stop(n_rec)
+    fam = {"products": 0.0, "casts": 0.0, "adapter_gradient": 0.0, "proxy_update": 0.0}
+    names = {"gemm_fwd": "products", "gemm_dx": "products", "quant_x": "casts", "quant_dy": "casts", "quant_oa": "casts",
+             "gemm_db": "adapter_gradient", "reduce_db": "adapter_gradient", "sgd_score": "proxy_update", "topk": "proxy_update",
+             "merge": "proxy_update"}
+    for name, t in recs:
+        fam[names[name]] += t / 2.0
+    fam["chain_kernels_and_gaps"] = max(ms_inst - sum(fam.values()), 0.0)
+    shares = {k_: {"ms_per_step": round(v, 3), "share": round(v / ms_inst, 4)} for k_, v in fam.items()}
+    f_products = stack.flops_per_step()
+    products_tf = f_products / (fam["products"] * 1e-3) / 1e12 if fam["products"] > 0 else 0.0
     flops = stack.flops_per_step()
     tf = flops / (ms * 1e-3) / 1e12
     print(json.dumps({
@@ -464,8 +495,16 @@ def run_stack(args):
                    "proxy_update": "one call per projection" if args.proxy_per_layer else "one batched call per block",
                    "launch": "replays of one CUDA graph of the step" if use_graph else "one library call after another"},
         "clocks": clocks, "gpu_launches": stack.launches_per_step() * steps,
+        "regime": "sustained: %.1f s of the same step loop ran right before the timed steps" % args.soak,
         "frac_of_fp8_peak": {"of_measured_sustained_x2": tf / (peaks["bf16_sustained"] * FP8_OVER_BF16),
-                             "of_nominal_4500": tf / 4500.0},
+                             "of_nominal_4500": tf / 4500.0,
+                             "target": "north_star: >= 0.60 of dense FP8 peak on this stack -- not met"},
+        "where_the_step_goes": {"pass_ms_per_step": ms_inst, "clocks": clocks_inst, "families": shares,
+                                "products_alone_tflops": products_tf,
+                                "products_alone_frac_of_measured_sustained_x2": products_tf / (peaks["bf16_sustained"] * FP8_OVER_BF16),
+                                "products_alone_frac_of_nominal_4500": products_tf / 4500.0,
+                                "note": "call-by-call pass with the library's stages bracketed by CUDA events (slower than the "
+                                        "graph replay above: no launch overlap across brackets); chain = what no bracket covers"},
         "memory": {"layers_bytes": stack.bytes_resident(), "allocated_bytes": torch.cuda.memory_allocated(dev),
                    "peak_allocated_bytes": torch.cuda.max_memory_allocated(dev)},
         "device_status": fq.last_device_status()}))
