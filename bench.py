@@ -778,13 +778,15 @@ def main():
     q_bytes_5 = sum(5.0 * T * (n + m) for _, n, m in linears)
     t_quant = (breakdown.get("quant_x", 0) + breakdown.get("quant_dy", 0)) * 1e-3
     quant_gbs = q_bytes / t_quant / 1e9 if t_quant > 0 else 0.0
+    n_beyond_l2 = sum((2.0 * T * n > L2_BYTES) + (2.0 * T * m > L2_BYTES) for _, n, m in linears)
     quantize = {"bound": "hbm", "achieved_gbs": quant_gbs, "peak_gbs": peaks["hbm"], "frac": quant_gbs / peaks["hbm"],
                 "frac_of_nominal_8000": quant_gbs / 8000.0, "ms_per_step": t_quant * 1e3,
-                "bytes_per_elt": lo, "bytes_per_step": q_bytes,
+                "bytes_per_elt": lo if n_beyond_l2 == 0 else f"{lo} for {2 * len(linears) - n_beyond_l2} tensors that fit L2, {hi} for {n_beyond_l2} beyond it",
+                "bytes_per_step": q_bytes,
                 "frac_if_counted_at_5_bytes_per_elt": (q_bytes_5 / t_quant / 1e9 / peaks["hbm"]) if t_quant > 0 and not args.fused else None,
                 "note": ("absmax pass over X and dY (the casts run inside the products)" if args.fused else
-                         "absmax + cast of X and dY in one kernel each: every tensor of this workload fits L2, so it is read from "
-                         "DRAM once (2 B/elt) and its codes written once (1 B/elt); 5 B/elt would apply beyond L2") +
+                         "absmax + cast of X and dY in one kernel each: a tensor that fits L2 is read from DRAM once (2 B/elt) and its "
+                         "codes written once (1 B/elt); beyond L2 (126 MB of bf16) the cast pass reads it again: 5 B/elt") +
                         "; the O_A cast rides in the same stage"}
     db_bytes = sum(T * m + T * r + 4.0 * m * r for _, n, m in linears)
     db = {"bound": "hbm", "kernel": "db_fused_kernel", "bytes_per_step": db_bytes, "ms_per_step": t_db,
