@@ -377,6 +377,23 @@ int falqon_update_a_region(int64_t m, int64_t n, int64_t r, int64_t T, falqon_ua
 int falqon_update_a(const falqon_layer *L, const uint8_t *xq, const float *s_x, const float *B, float *A_master, float gamma,
                     float lr, int64_t T, void *ws, size_t ws_bytes, void *scratch, size_t scratch_bytes, falqon_stream stream);
 
+/* falqon_proxy_update_exact for `count` layers: the optimizer steps, scores and selections in one launch and the correctly
+ * rounded merges of all layers in three (row preparation, tensor-core sums with the guard-band rounding, exact
+ * recomputation of the flagged elements).  Host arrays as in falqon_proxy_update_batched, plus one scratch per layer
+ * (falqon_exact_merge_scratch_bytes; two layers must not share one).  Bit-identical to the per-layer
+ * falqon_proxy_update_exact calls.
+ *   a_prepared  0: the bf16 copy of each layer's A~ rows and its column maxima are rebuilt in this call (two more
+ *               launches per layer).  Non-zero: falqon_exact_merge_prepare was run on every layer's scratch and the A~
+ *               rows have not changed since (the proxy update never changes them; falqon_update_a does).
+ * When to prefer it over the fp32 chain of falqon_proxy_update_batched is a matter of definition first (the two round
+ * differently: the chain after every fma, this once) and of size second: the chain costs k n r fp32 fmas, this a
+ * tensor-core product plus fixed launches. */
+int falqon_exact_merge_prepare(const falqon_layer *L, void *scratch, size_t scratch_bytes, falqon_stream stream);
+int falqon_proxy_update_batched_exact(const falqon_layer *layers, int32_t count, const float *const *dB, float lr,
+                                      const int64_t *k, int32_t *const *idx_out, void *const *ws, const size_t *ws_bytes,
+                                      void *const *scratch, const size_t *scratch_bytes, int32_t a_prepared,
+                                      falqon_stream stream);
+
 /* Synchronizes `stream`, then returns and clears the device status word of the current device:
  * FALQON_OK, FALQON_ERR_TIMEOUT (a bounded device-side wait ran out; results of that call are
  * undefined) or FALQON_ERR_CUDA (the synchronize itself failed). */

@@ -24,6 +24,7 @@ WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 EXPORTS = ["falqon_absmax", "falqon_selftest_wait_timeout", "falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax",
            "falqon_melded_forward_dump", "falqon_melded_backward_dump", "falqon_melded_backward_dx",
+           "falqon_exact_merge_prepare", "falqon_proxy_update_batched_exact",
            "falqon_update_a", "falqon_update_a_scratch_bytes", "falqon_update_a_region",
            "falqon_melded_backward_update", "falqon_proxy_update_scored", "falqon_proxy_update_scored_batched", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
            "falqon_svd_init_scratch_bytes", "falqon_svd_init", "falqon_tensor_ceiling", "falqon_tensor_ceiling_ctas",
@@ -63,6 +64,11 @@ lib.falqon_melded_forward_dump.restype = _i
 lib.falqon_melded_forward_dump.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _i, _p, _p, _p, C.c_int32, _p, _sz, _p]
 lib.falqon_melded_backward_dump.restype = _i
 lib.falqon_melded_backward_dump.argtypes = [C.POINTER(falqon_layer), _p, _i, _p, _i64, _p, _p, _p, _i, _p, _p, C.c_int32, _p, _sz, _p]
+lib.falqon_exact_merge_prepare.restype = _i
+lib.falqon_exact_merge_prepare.argtypes = [C.POINTER(falqon_layer), _p, _sz, _p]
+lib.falqon_proxy_update_batched_exact.restype = _i
+lib.falqon_proxy_update_batched_exact.argtypes = [C.POINTER(falqon_layer), C.c_int32, C.POINTER(_p), _f, C.POINTER(_i64), C.POINTER(_p),
+                                                  C.POINTER(_p), C.POINTER(_sz), C.POINTER(_p), C.POINTER(_sz), C.c_int32, _p]
 lib.falqon_update_a_scratch_bytes.restype = _sz
 lib.falqon_update_a_scratch_bytes.argtypes = [_i64, _i64, _i64, _i64]
 lib.falqon_update_a_region.restype = _i
@@ -486,6 +492,25 @@ class ProxyBatch:
         _check("falqon_proxy_update_batched_adamw",
                lib.falqon_proxy_update_batched_adamw(self.c_layers, self.count, self.c_dB, c_ea, c_es, C.byref(hp), self.c_k,
                                                      self.c_idx, self.c_ws, self.c_ws_bytes, _stream()))
+        return self.idx_outs
+
+    def prepare_exact(self):
+        """Scratch for the correctly rounded merge of every layer, with the bf16 copy of its A~ rows prepared once
+        (falqon_exact_merge_prepare).  Call again after anything changed the A~ rows."""
+        self.scratch = [torch.empty(int(lib.falqon_exact_merge_scratch_bytes(L.m, L.n, L.r)), dtype=torch.uint8, device=L.wq.device)
+                        for L in self.layers]
+        n = max(self.count, 1)
+        self.c_scratch = (_p * n)(*[_ptr(t) for t in self.scratch])
+        self.c_scratch_bytes = (_sz * n)(*[t.numel() for t in self.scratch])
+        for L, sc in zip(self.layers, self.scratch):
+            _check("falqon_exact_merge_prepare", lib.falqon_exact_merge_prepare(C.byref(L.c), _ptr(sc), sc.numel(), _stream()))
+
+    def run_exact(self, lr: float, prepared: bool = True):
+        """falqon_proxy_update_batched_exact (prepare_exact must have been called once)."""
+        _check("falqon_proxy_update_batched_exact",
+               lib.falqon_proxy_update_batched_exact(self.c_layers, self.count, self.c_dB, lr, self.c_k, self.c_idx, self.c_ws,
+                                                     self.c_ws_bytes, self.c_scratch, self.c_scratch_bytes, 1 if prepared else 0,
+                                                     _stream()))
         return self.idx_outs
 
     def run_scored(self):

@@ -673,6 +673,70 @@ int falqon_proxy_update_exact(const falqon_layer* L, const float* dB, float lr, 
   return proxy_update_impl(L, dB, lr, nullptr, nullptr, nullptr, k, idx_out, ws, ws_bytes, stream, &exact);
 }
 
+int falqon_exact_merge_prepare(const falqon_layer* L, void* scratch, size_t scratch_bytes, falqon_stream stream) {
+  if (!layer_ok(L)) return FALQON_ERR_INVALID_ARG;
+  if (scratch == nullptr || !aligned16(scratch) || scratch_bytes < exact_merge_scratch_bytes(L->m, L->n, L->r))
+    return FALQON_ERR_WORKSPACE;
+  FALQON_CUDA(launch_exact_merge_prepare(L->wq, L->m, L->n, L->r, scratch, stream));
+  return FALQON_OK;
+}
+
+int falqon_proxy_update_batched_exact(const falqon_layer* layers, int32_t count, const float* const* dB, float lr, const int64_t* k,
+                                      int32_t* const* idx_out, void* const* ws, const size_t* ws_bytes, void* const* scratch,
+                                      const size_t* scratch_bytes, int32_t a_prepared, falqon_stream stream) {
+  if (count < 0 || !(lr == lr)) return FALQON_ERR_INVALID_ARG;
+  if (count == 0) return FALQON_OK;
+  if (layers == nullptr || dB == nullptr || k == nullptr || ws == nullptr || ws_bytes == nullptr || scratch == nullptr ||
+      scratch_bytes == nullptr)
+    return FALQON_ERR_INVALID_ARG;
+  for (int32_t i = 0; i < count; ++i) {
+    const falqon_layer* L = &layers[i];
+    if (!layer_ok(L) || k[i] < 0 || k[i] > L->m || (dB[i] != nullptr && !aligned16(dB[i]))) return FALQON_ERR_INVALID_ARG;
+    WorkspaceLayout w;
+    if (!make_layout(L->m, L->n, L->r, 1, &w)) return FALQON_ERR_INVALID_ARG;
+    if (ws[i] == nullptr || !aligned16(ws[i]) || ws_bytes[i] < w.total) return FALQON_ERR_WORKSPACE;
+    if (scratch[i] == nullptr || !aligned16(scratch[i]) || scratch_bytes[i] < exact_merge_scratch_bytes(L->m, L->n, L->r))
+      return FALQON_ERR_WORKSPACE;
+    for (int32_t j = 0; j < i; ++j)
+      if (ws[j] == ws[i] || scratch[j] == scratch[i] || layers[j].wq == L->wq || layers[j].dbuf == L->dbuf) return FALQON_ERR_INVALID_ARG;
+  }
+  int* status = status_ptr();
+  if (status == nullptr) return FALQON_ERR_CUDA;
+  for (int32_t first = 0; first < count; first += kProxyBatchMax) {
+    const int chunk = count - first < kProxyBatchMax ? count - first : kProxyBatchMax;
+    ProxyBatchLayer b[kProxyBatchMax];
+    ExactMergeLayer x[kProxyBatchMax];
+    bool any_merge = false;
+    for (int c = 0; c < chunk; ++c) {
+      const int32_t i = first + c;
+      const falqon_layer* L = &layers[i];
+      WorkspaceLayout w;
+      make_layout(L->m, L->n, L->r, 1, &w);
+      uint8_t* base = static_cast<uint8_t*>(ws[i]);
+      b[c] = ProxyBatchLayer{};
+      b[c].wq = L->wq; b[c].dbuf = L->dbuf; b[c].dB = dB[i];
+      b[c].row_scales = L->gran == FALQON_PER_ROW ? L->s_w : nullptr;
+      b[c].score = reinterpret_cast<float*>(base + w.score);
+      b[c].sel_idx = reinterpret_cast<int32_t*>(base + w.sel_idx);
+      b[c].idx_out = idx_out != nullptr ? idx_out[i] : nullptr;
+      b[c].done_counter = reinterpret_cast<unsigned int*>(base + w.scales + kDoneOffset);
+      b[c].group_counters = reinterpret_cast<unsigned int*>(base + w.scales + kGroupCountersOffset);
+      b[c].m = L->m; b[c].n = L->n; b[c].r = L->r; b[c].k = k[i];
+      x[c] = ExactMergeLayer{L->wq, L->dbuf, b[c].sel_idx, b[c].row_scales, scratch[i], nullptr, nullptr, L->m, L->n, L->r, k[i]};
+      any_merge = any_merge || k[i] > 0;
+    }
+    {
+      StageTimer timer(FALQON_STAGE_SGD_SCORE, stream);
+      FALQON_CUDA(launch_proxy_update_batched(b, chunk, lr, nullptr, 0, stream));
+    }
+    if (any_merge) {
+      StageTimer timer(FALQON_STAGE_MERGE, stream);
+      FALQON_CUDA(launch_merge_exact_batched(x, chunk, a_prepared != 0, status, stream));
+    }
+  }
+  return FALQON_OK;
+}
+
 size_t falqon_svd_init_scratch_bytes(int64_t m, int64_t n, int64_t l) {
   if (m < 16 || n < 16 || m % 16 || n % 16 || l < 2 || l % 2 || l > 160) return 0;
   return svd_init_scratch_bytes(m, n, l);

@@ -186,6 +186,21 @@ cudaError_t launch_merge_exact(uint8_t* wq, float* dbuf, const int32_t* sel_idx,
                                const float* row_scales, void* scratch, float* sums_out, unsigned int* fix_count_out, int* status,
                                cudaStream_t stream);
 
+// The same for several layers per launch (three launches for the whole set, plus two per layer when the bf16 copy of A~ has
+// not been prepared beforehand).  Layers with k == 0 are skipped.
+struct ExactMergeLayer {
+  uint8_t* wq;
+  float* dbuf;
+  const int32_t* sel_idx;
+  const float* row_scales;       // nullable
+  void* scratch;                 // exact_merge_scratch_bytes(m, n, r)
+  float* sums_out;               // nullable
+  unsigned int* fix_count_out;   // nullable
+  int64_t m, n, r, k;
+};
+cudaError_t launch_exact_merge_prepare(const uint8_t* wq, int64_t m, int64_t n, int64_t r, void* scratch, cudaStream_t stream);
+cudaError_t launch_merge_exact_batched(const ExactMergeLayer* layers, int count, bool a_prepared, int* status, cudaStream_t stream);
+
 // ---- svd_init.cu: A^ = sqrt(S_r) V_r^T of Delta W = W - dec(W~) / s_W by randomized subspace iteration (set-up code).
 // omega: [n][l] fp32 Gaussian test matrix drawn by the caller, l even, r <= l <= 160; scratch: svd_init_scratch_bytes.
 size_t svd_init_scratch_bytes(int64_t m, int64_t n, int64_t l);

@@ -80,13 +80,39 @@ __global__ void __launch_bounds__(256) exact_amax_a_kernel(const uint16_t* a_t, 
 // ---- step 0b: the selected DeltaBuffer rows -> d' (fp32 copy for the exact fallback), three exact bf16 limbs
 // (the A operand, [k][3 r_pad]), sum_j |d'_j| for the guard band; the DeltaBuffer rows are cleared here.
 // One warp per selected row, eight rows per CTA.
-__global__ void __launch_bounds__(256) exact_prep_rows_kernel(float* dbuf, const int32_t* sel_idx, int k, int r, int r_pad,
-                                                              const float* row_scales, int64_t m, uint16_t* limbs,
-                                                              float* dprime, float* sprime) {
+// Several layers per launch: the CTAs of all layers are laid end to end (cta_begin), as in the batched score kernel.
+constexpr int kXBatchMax = kProxyBatchMax;
+struct PrepRowsLayer {
+  float* dbuf;
+  const int32_t* sel_idx;
+  const float* row_scales;
+  uint16_t* limbs;
+  float* dprime;
+  float* sprime;
+  long long m;
+  int k, r, r_pad, cta_begin;
+};
+struct PrepRowsBatch {
+  PrepRowsLayer layer[kXBatchMax];
+  int count;
+};
+__global__ void __launch_bounds__(256) exact_prep_rows_kernel(const __grid_constant__ PrepRowsBatch args) {
   pdl_trigger();
   pdl_wait();
+  int l = 0;
+#pragma unroll 1
+  for (int i = 1; i < args.count; ++i) l = static_cast<int>(blockIdx.x) >= args.layer[i].cta_begin ? i : l;
+  const PrepRowsLayer& a = args.layer[l];
+  float* dbuf = a.dbuf;
+  const int32_t* sel_idx = a.sel_idx;
+  const float* row_scales = a.row_scales;
+  uint16_t* limbs = a.limbs;
+  float* dprime = a.dprime;
+  float* sprime = a.sprime;
+  const long long m = a.m;
+  const int k = a.k, r = a.r, r_pad = a.r_pad;
   const int lane = threadIdx.x & 31;
-  const int q = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int q = (static_cast<int>(blockIdx.x) - a.cta_begin) * 8 + (threadIdx.x >> 5);
   if (q >= k) return;
   const int row = ld_stream(sel_idx + q);
   float coef = 1.0f;
@@ -140,21 +166,37 @@ struct XParams {
   uint32_t* flags;          // [k][words_per_row]
   int words_per_row;
   float* sums_out;          // nullable [k][n]: the accumulated sums, for diagnostics
+};
+// The layers of one launch: per layer its two tensor maps and parameters; the tiles of all layers are laid end to end
+// (tile_begin), every layer with the same tile width, so the shared-memory stages and barriers serve them all.
+struct XBatch {
+  CUtensorMap ta[kXBatchMax];
+  CUtensorMap tb[kXBatchMax];
+  XParams p[kXBatchMax];
+  int tile_begin[kXBatchMax + 1];
+  int count, block_n;
+  uint32_t tmem_cols;
   int* status;
 };
+__device__ __forceinline__ int xbatch_layer(const XBatch& b, int tile) {
+  int l = 0;
+#pragma unroll 1
+  for (int i = 1; i < b.count; ++i) l = tile >= b.tile_begin[i] ? i : l;
+  return l;
+}
 
 // ---- steps 1-3: S = limbs x a_t^T on the tensor cores (K-major bf16 operands, fp32 accumulators in TMEM), then the
 // guard-band rounding in the epilogue (the heavy part: two CTAs per SM give it sixteen warps).  Persistent CTAs walk
 // 128 x block_n tiles (block_n <= 128); the B operand's k
 // coordinate wraps every r_pad elements (the three limb blocks of A meet the same A~ block).
 __global__ void __launch_bounds__(kXThreads, 2)
-merge_exact_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const XParams p) {
+merge_exact_kernel(const __grid_constant__ XBatch args) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t smem_base = (raw_addr + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - raw_addr);
 
-  const uint32_t b_tile = static_cast<uint32_t>(p.block_n) * kXBlockKBytes;
+  const uint32_t b_tile = static_cast<uint32_t>(args.block_n) * kXBlockKBytes;
   const uint32_t stage_bytes = kXATile + b_tile;
   constexpr int S = kXStages;
   const uint32_t bars = smem_base + S * stage_bytes;
@@ -170,14 +212,16 @@ merge_exact_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
   constexpr uint32_t kEpiWarps = 8;
 
   if (threadIdx.x == 0) {
-    prefetch_tensor_map(&tmap_a);
-    prefetch_tensor_map(&tmap_b);
+    for (int i = 0; i < args.count; ++i) {
+      prefetch_tensor_map(&args.ta[i]);
+      prefetch_tensor_map(&args.tb[i]);
+    }
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tmem_full_bar(a), 1); mbar_init(tmem_empty_bar(a), kEpiWarps); }
     mbar_fence_init();
   }
   if (warp == 1) {
-    tmem_alloc(smem_base + slot_off, p.tmem_cols);
+    tmem_alloc(smem_base + slot_off, args.tmem_cols);
     tmem_relinquish();
   }
   pdl_trigger();
@@ -187,23 +231,27 @@ merge_exact_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();
 
-  const int total_tiles = p.m_tiles * p.n_tiles;
-  const uint32_t acc_cols = static_cast<uint32_t>(p.block_n);
+  const int total_tiles = args.tile_begin[args.count];
+  const uint32_t acc_cols = static_cast<uint32_t>(args.block_n);
+  int* const status = args.status;
   bool aborted = false;
 
   if (warp == 0) {
     int stage = 0;
     uint32_t phase = 0;
-    for (int tile = blockIdx.x; tile < total_tiles && !aborted; tile += gridDim.x) {
+    for (int gtile = blockIdx.x; gtile < total_tiles && !aborted; gtile += gridDim.x) {
+      const int l = xbatch_layer(args, gtile);
+      const XParams& p = args.p[l];
+      const int tile = gtile - args.tile_begin[l];
       const int n_idx = tile / p.m_tiles, m_idx = tile - n_idx * p.m_tiles;
       for (int kb = 0; kb < p.kblocks_total; ++kb) {
-        if (!mbar_wait_warp(empty_bar(stage), phase ^ 1u, p.status)) { aborted = true; break; }
+        if (!mbar_wait_warp(empty_bar(stage), phase ^ 1u, status)) { aborted = true; break; }
         if (elect_one()) {
           const uint32_t fb = full_bar(stage);
           mbar_expect_tx(fb, stage_bytes);
           const uint32_t a_dst = smem_base + stage * stage_bytes;
-          tma_load_2d(a_dst, &tmap_a, fb, kb * kXBlockKBytes, m_idx * kXBlockM);
-          tma_load_2d(a_dst + kXATile, &tmap_b, fb, (kb % p.kblocks_wrap) * kXBlockKBytes, n_idx * p.block_n);
+          tma_load_2d(a_dst, &args.ta[l], fb, kb * kXBlockKBytes, m_idx * kXBlockM);
+          tma_load_2d(a_dst + kXATile, &args.tb[l], fb, (kb % p.kblocks_wrap) * kXBlockKBytes, n_idx * p.block_n);
         }
         __syncwarp();
         if (++stage == S) { stage = 0; phase ^= 1u; }
@@ -215,12 +263,13 @@ merge_exact_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
     const uint64_t a_desc0 = make_smem_desc(smem_base, 16, 1024);
     const uint64_t b_desc0 = make_smem_desc(smem_base + kXATile, 16, 1024);
     constexpr uint32_t kStep = kXUmmaKBytes >> 4;
-    for (int tile = blockIdx.x; tile < total_tiles && !aborted; tile += gridDim.x) {
-      if (!mbar_wait_warp(tmem_empty_bar(acc), acc_phase ^ 1u, p.status)) { aborted = true; break; }
+    for (int gtile = blockIdx.x; gtile < total_tiles && !aborted; gtile += gridDim.x) {
+      const XParams& p = args.p[xbatch_layer(args, gtile)];
+      if (!mbar_wait_warp(tmem_empty_bar(acc), acc_phase ^ 1u, status)) { aborted = true; break; }
       tc_fence_after_sync();
       const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * acc_cols;
       for (int kb = 0; kb < p.kblocks_total; ++kb) {
-        if (!mbar_wait_warp(full_bar(stage), phase, p.status)) { aborted = true; break; }
+        if (!mbar_wait_warp(full_bar(stage), phase, status)) { aborted = true; break; }
         tc_fence_after_sync();
         const uint32_t stage_off = (static_cast<uint32_t>(stage) * stage_bytes) >> 4;
         if (elect_one()) {
@@ -245,9 +294,12 @@ merge_exact_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
     const int col_half = (warp - 2) >> 2;
     int acc = 0;
     uint32_t acc_phase = 0;
-    for (int tile = blockIdx.x; tile < total_tiles && !aborted; tile += gridDim.x) {
+    for (int gtile = blockIdx.x; gtile < total_tiles && !aborted; gtile += gridDim.x) {
+      const int l = xbatch_layer(args, gtile);
+      const XParams& p = args.p[l];
+      const int tile = gtile - args.tile_begin[l];
       const int n_idx = tile / p.m_tiles, m_idx = tile - n_idx * p.m_tiles;
-      if (!mbar_wait(tmem_full_bar(acc), acc_phase, p.status)) { aborted = true; break; }
+      if (!mbar_wait(tmem_full_bar(acc), acc_phase, status)) { aborted = true; break; }
       tc_fence_after_sync();
       const int q = m_idx * kXBlockM + quad * 32 + lane;
       const bool row_ok = q < p.k;
@@ -325,7 +377,7 @@ merge_exact_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
   __syncthreads();
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, p.tmem_cols);
+    tmem_dealloc(tmem_base, args.tmem_cols);
   }
 }
 
@@ -415,15 +467,40 @@ __device__ __noinline__ uint32_t exact_element_warp(uint32_t w_code, const float
 }
 
 // A warp scans 32 flag words at a time (one per lane); for every set bit all its lanes recompute that element.
-__global__ void __launch_bounds__(256) exact_fix_kernel(uint8_t* wq, const uint8_t* aq, const int32_t* sel_idx,
-                                                        const float* dprime, const uint32_t* flags, int64_t total_words, int64_t n,
-                                                        int r, int r_pad, int words_per_row, unsigned int* fix_count) {
+struct FixLayer {
+  uint8_t* wq;
+  const uint8_t* aq;
+  const int32_t* sel_idx;
+  const float* dprime;
+  const uint32_t* flags;
+  unsigned int* fix_count;     // nullable
+  long long total_words, n;
+  int r, r_pad, words_per_row, cta_begin, ctas;
+};
+struct FixBatch {
+  FixLayer layer[kXBatchMax];
+  int count;
+};
+__global__ void __launch_bounds__(256) exact_fix_kernel(const __grid_constant__ FixBatch args) {
   pdl_trigger();
   pdl_wait();
+  int l = 0;
+#pragma unroll 1
+  for (int i = 1; i < args.count; ++i) l = static_cast<int>(blockIdx.x) >= args.layer[i].cta_begin ? i : l;
+  const FixLayer& a = args.layer[l];
+  uint8_t* wq = a.wq;
+  const uint8_t* aq = a.aq;
+  const int32_t* sel_idx = a.sel_idx;
+  const float* dprime = a.dprime;
+  const uint32_t* flags = a.flags;
+  unsigned int* fix_count = a.fix_count;
+  const int64_t total_words = a.total_words, n = a.n;
+  const int r = a.r, r_pad = a.r_pad, words_per_row = a.words_per_row;
+  const int cta = static_cast<int>(blockIdx.x) - a.cta_begin;
   const int lane = threadIdx.x & 31;
   unsigned int fixed = 0;
-  const int64_t warps = static_cast<int64_t>(gridDim.x) * 8;
-  for (int64_t base = (blockIdx.x * 8ll + (threadIdx.x >> 5)) * 32; base < total_words; base += warps * 32) {
+  const int64_t warps = static_cast<int64_t>(a.ctas) * 8;
+  for (int64_t base = (cta * 8ll + (threadIdx.x >> 5)) * 32; base < total_words; base += warps * 32) {
     const int64_t wi = base + lane;
     const uint32_t mine = wi < total_words ? ld_stream(flags + wi) : 0u;
     uint32_t pending = __ballot_sync(0xFFFFFFFFu, mine != 0);
@@ -462,58 +539,129 @@ size_t exact_merge_scratch_bytes(int64_t m, int64_t n, int64_t r) {
   return b;
 }
 
-cudaError_t launch_merge_exact(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n, int64_t r,
-                               const float* row_scales, void* scratch, float* sums_out, unsigned int* fix_count_out, int* status,
-                               cudaStream_t stream) {
-  if (k < 1 || k > m || r < 8 || r > 256 || n % 16) return cudaErrorInvalidValue;
-  const int64_t r_pad = round_up(r, 64);
+namespace {
+struct ExactScratch {
+  uint16_t* a_t; float* amax_c; uint16_t* limbs; float* dprime; float* sprime; uint32_t* flags; unsigned int* counter;
+};
+ExactScratch carve_scratch(void* scratch, int64_t m, int64_t n, int64_t r_pad) {
   uint8_t* base = static_cast<uint8_t*>(scratch);
   size_t off = 0;
-  uint16_t* a_t = reinterpret_cast<uint16_t*>(base + off); off += round_up(n * r_pad * 2, 1024);
-  float* amax_c = reinterpret_cast<float*>(base + off); off += round_up(round_up(n, 32) * 4, 1024);
-  uint16_t* limbs = reinterpret_cast<uint16_t*>(base + off); off += round_up(m * 3 * r_pad * 2, 1024);
-  float* dprime = reinterpret_cast<float*>(base + off); off += round_up(m * r_pad * 4, 1024);
-  float* sprime = reinterpret_cast<float*>(base + off); off += round_up(m * 4, 1024);
-  uint32_t* flags = reinterpret_cast<uint32_t*>(base + off); off += round_up(m * ((n + 31) / 32) * 4, 1024);
-  unsigned int* counter = reinterpret_cast<unsigned int*>(base + off);
+  ExactScratch x;
+  x.a_t = reinterpret_cast<uint16_t*>(base + off); off += round_up(n * r_pad * 2, 1024);
+  x.amax_c = reinterpret_cast<float*>(base + off); off += round_up(round_up(n, 32) * 4, 1024);
+  x.limbs = reinterpret_cast<uint16_t*>(base + off); off += round_up(m * 3 * r_pad * 2, 1024);
+  x.dprime = reinterpret_cast<float*>(base + off); off += round_up(m * r_pad * 4, 1024);
+  x.sprime = reinterpret_cast<float*>(base + off); off += round_up(m * 4, 1024);
+  x.flags = reinterpret_cast<uint32_t*>(base + off); off += round_up(m * ((n + 31) / 32) * 4, 1024);
+  x.counter = reinterpret_cast<unsigned int*>(base + off);
+  return x;
+}
+}  // namespace
+
+// Step 0a on its own: the bf16 copy of A~ (transposed) and its column maxima depend only on the A~ rows of the backbone,
+// which the proxy update never changes, so a caller may prepare them once per layer.
+cudaError_t launch_exact_merge_prepare(const uint8_t* wq, int64_t m, int64_t n, int64_t r, void* scratch, cudaStream_t stream) {
+  const int64_t r_pad = round_up(r, 64);
+  const ExactScratch x = carve_scratch(scratch, m, n, r_pad);
   const uint8_t* aq = wq + m * n;
-
   cudaError_t e = launch_pdl(exact_prep_a_kernel, dim3(static_cast<unsigned>((n + 255) / 256), static_cast<unsigned>(r_pad / 2)),
-                             dim3(256), 0, stream, 1, aq, n, static_cast<int>(r), static_cast<int>(r_pad), a_t);
+                             dim3(256), 0, stream, 1, aq, n, static_cast<int>(r), static_cast<int>(r_pad), x.a_t);
   if (e != cudaSuccess) return e;
-  e = launch_pdl(exact_amax_a_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, stream, 1,
-                 static_cast<const uint16_t*>(a_t), n, static_cast<int>(r_pad), amax_c);
-  if (e != cudaSuccess) return e;
-  e = launch_pdl(exact_prep_rows_kernel, dim3(static_cast<unsigned>((k + 7) / 8)), dim3(256), 0, stream, 1, dbuf, sel_idx,
-                 static_cast<int>(k), static_cast<int>(r), static_cast<int>(r_pad), row_scales, m, limbs, dprime, sprime);
+  return launch_pdl(exact_amax_a_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, stream, 1,
+                    static_cast<const uint16_t*>(x.a_t), n, static_cast<int>(r_pad), x.amax_c);
+}
+
+// Steps 0b-4 for up to kProxyBatchMax layers in three launches (row preparation, tensor-core sums with the guard-band
+// rounding, exact recomputation of the flagged elements).  a_prepared: step 0a was run on every layer's scratch
+// (launch_exact_merge_prepare) and the A~ rows have not changed since; otherwise it runs here, two launches per layer.
+cudaError_t launch_merge_exact_batched(const ExactMergeLayer* layers, int count, bool a_prepared, int* status, cudaStream_t stream) {
+  if (count < 1 || count > kXBatchMax) return cudaErrorInvalidValue;
+  PrepRowsBatch pb{};
+  XBatch xb{};
+  FixBatch fb{};
+  ExactScratch xs[kXBatchMax];
+  int64_t r_pad[kXBatchMax];
+  int active = 0, prep_ctas = 0;
+  for (int i = 0; i < count; ++i) {
+    const ExactMergeLayer& L = layers[i];
+    if (L.k == 0) continue;
+    if (L.k < 1 || L.k > L.m || L.r < 8 || L.r > 256 || L.n % 16) return cudaErrorInvalidValue;
+    r_pad[active] = round_up(L.r, 64);
+    xs[active] = carve_scratch(L.scratch, L.m, L.n, r_pad[active]);
+    if (!a_prepared) {
+      const cudaError_t e = launch_exact_merge_prepare(L.wq, L.m, L.n, L.r, L.scratch, stream);
+      if (e != cudaSuccess) return e;
+    }
+    PrepRowsLayer& a = pb.layer[active];
+    a.dbuf = L.dbuf; a.sel_idx = L.sel_idx; a.row_scales = L.row_scales; a.limbs = xs[active].limbs; a.dprime = xs[active].dprime;
+    a.sprime = xs[active].sprime; a.m = L.m; a.k = static_cast<int>(L.k); a.r = static_cast<int>(L.r);
+    a.r_pad = static_cast<int>(r_pad[active]); a.cta_begin = prep_ctas;
+    prep_ctas += static_cast<int>((L.k + 7) / 8);
+    ++active;
+  }
+  if (active == 0) return cudaSuccess;
+  pb.count = active;
+  cudaError_t e = launch_pdl(exact_prep_rows_kernel, dim3(static_cast<unsigned>(prep_ctas)), dim3(256), 0, stream, 1, pb);
   if (e != cudaSuccess) return e;
 
-  XParams p{};
-  p.k = static_cast<int>(k); p.n = static_cast<int>(n); p.r_pad = static_cast<int>(r_pad);
-  p.m_tiles = static_cast<int>((k + kXBlockM - 1) / kXBlockM);
-  int block_n = 128;   // narrower tiles when there would be too few of them for two CTAs per SM
-  while (block_n > 32 && static_cast<int64_t>(p.m_tiles) * ((n + block_n - 1) / block_n) < 2 * sm_count()) block_n >>= 1;
-  p.block_n = block_n;
-  p.n_tiles = static_cast<int>((n + block_n - 1) / block_n);
-  p.kblocks_wrap = static_cast<int>(r_pad * 2 / kXBlockKBytes);
-  p.kblocks_total = 3 * p.kblocks_wrap;
-  // instruction descriptor: fp32 accumulate, A and B bf16 K-major, N = block_n, M = 128
-  p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(block_n >> 3) << 17) |
-            (static_cast<uint32_t>(kXBlockM >> 4) << 24);
-  p.tmem_cols = static_cast<uint32_t>(2 * block_n);
-  // accumulation error: 3 r_pad exact products summed in fp32 in an unknown order, each partial sum bounded by
-  // T = |w| + sum|d'| max|a|: (N - 1) 2^-24 T for round-to-nearest adds; taken with a factor 2 (2^-23 per add) for adds
-  // that truncate, plus the final add of w.  Measured on B200: the sums use 0.2-0.7 % of this band.
-  p.kappa = 1.02f * static_cast<float>(3 * r_pad + 8) * 1.1920928955078125e-07f;   // 2^-23
-  p.wq = wq; p.sel_idx = sel_idx; p.sprime = sprime; p.amax_c = amax_c; p.flags = flags;
-  p.words_per_row = static_cast<int>((n + 31) / 32);
-  p.sums_out = sums_out; p.status = status;
-  CUtensorMap ta, tb;
-  if (!make_tensor_map(&ta, reinterpret_cast<const uint8_t*>(limbs), k, 3 * r_pad * 2, 3 * r_pad * 2, kXBlockKBytes, kXBlockM))
-    return cudaErrorInvalidValue;
-  if (!make_tensor_map(&tb, reinterpret_cast<const uint8_t*>(a_t), n, r_pad * 2, r_pad * 2, kXBlockKBytes,
-                       static_cast<uint32_t>(block_n)))
-    return cudaErrorInvalidValue;
+  // one tile width for the whole launch: narrower tiles when there would be too few of them for two CTAs per SM
+  int block_n = 128;
+  auto tiles_at = [&](int bn) {
+    int64_t t = 0;
+    for (int i = 0; i < count; ++i)
+      if (layers[i].k > 0) t += ((layers[i].k + kXBlockM - 1) / kXBlockM) * ((layers[i].n + bn - 1) / bn);
+    return t;
+  };
+  while (block_n > 32 && tiles_at(block_n) < 2 * sm_count()) block_n >>= 1;
+  xb.count = active; xb.block_n = block_n; xb.tmem_cols = static_cast<uint32_t>(2 * block_n); xb.status = status;
+  int tiles = 0, fix_ctas = 0, a = 0;
+  for (int i = 0; i < count; ++i) {
+    const ExactMergeLayer& L = layers[i];
+    if (L.k == 0) continue;
+    XParams& p = xb.p[a];
+    p.k = static_cast<int>(L.k); p.n = static_cast<int>(L.n); p.r_pad = static_cast<int>(r_pad[a]);
+    p.m_tiles = static_cast<int>((L.k + kXBlockM - 1) / kXBlockM);
+    p.block_n = block_n;
+    p.n_tiles = static_cast<int>((L.n + block_n - 1) / block_n);
+    p.kblocks_wrap = static_cast<int>(r_pad[a] * 2 / kXBlockKBytes);
+    p.kblocks_total = 3 * p.kblocks_wrap;
+    // instruction descriptor: fp32 accumulate, A and B bf16 K-major, N = block_n, M = 128
+    p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(block_n >> 3) << 17) |
+              (static_cast<uint32_t>(kXBlockM >> 4) << 24);
+    p.tmem_cols = xb.tmem_cols;
+    // accumulation error: 3 r_pad exact products summed in fp32 in an unknown order, each partial sum bounded by
+    // T = |w| + sum|d'| max|a|: (N - 1) 2^-24 T for round-to-nearest adds; taken with a factor 2 (2^-23 per add) for adds
+    // that truncate, plus the final add of w.  Measured on B200: the sums use 0.2-0.7 % of this band.
+    p.kappa = 1.02f * static_cast<float>(3 * r_pad[a] + 8) * 1.1920928955078125e-07f;   // 2^-23
+    p.wq = L.wq; p.sel_idx = L.sel_idx; p.sprime = xs[a].sprime; p.amax_c = xs[a].amax_c; p.flags = xs[a].flags;
+    p.words_per_row = static_cast<int>((L.n + 31) / 32);
+    p.sums_out = L.sums_out;
+    if (!make_tensor_map(&xb.ta[a], reinterpret_cast<const uint8_t*>(xs[a].limbs), L.k, 3 * r_pad[a] * 2, 3 * r_pad[a] * 2,
+                         kXBlockKBytes, kXBlockM))
+      return cudaErrorInvalidValue;
+    if (!make_tensor_map(&xb.tb[a], reinterpret_cast<const uint8_t*>(xs[a].a_t), L.n, r_pad[a] * 2, r_pad[a] * 2, kXBlockKBytes,
+                         static_cast<uint32_t>(block_n)))
+      return cudaErrorInvalidValue;
+    xb.tile_begin[a] = tiles;
+    tiles += p.m_tiles * p.n_tiles;
+    FixLayer& f = fb.layer[a];
+    f.wq = L.wq; f.aq = L.wq + L.m * L.n; f.sel_idx = L.sel_idx; f.dprime = xs[a].dprime; f.flags = xs[a].flags;
+    f.fix_count = L.fix_count_out != nullptr ? xs[a].counter : nullptr;
+    f.total_words = L.k * p.words_per_row; f.n = L.n; f.r = static_cast<int>(L.r); f.r_pad = static_cast<int>(r_pad[a]);
+    f.words_per_row = p.words_per_row; f.cta_begin = fix_ctas;
+    int64_t fg = (f.total_words + 255) / 256;
+    const int64_t cap = static_cast<int64_t>(sm_count()) * 8 / active;
+    if (fg > cap) fg = cap > 0 ? cap : 1;
+    f.ctas = static_cast<int>(fg);
+    fix_ctas += f.ctas;
+    if (L.fix_count_out != nullptr) {
+      e = cudaMemsetAsync(xs[a].counter, 0, sizeof(unsigned int), stream);
+      if (e != cudaSuccess) return e;
+    }
+    ++a;
+  }
+  xb.tile_begin[active] = tiles;
+  fb.count = active;
   const size_t smem = static_cast<size_t>(kXStages) * (kXATile + static_cast<size_t>(block_n) * kXBlockKBytes) + 256 + 1024;
   static DeviceMask configured{0};
   {
@@ -521,24 +669,29 @@ cudaError_t launch_merge_exact(uint8_t* wq, float* dbuf, const int32_t* sel_idx,
     if (ec != cudaSuccess) return ec;
   }
   int grid = 2 * sm_count();
-  const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
-  if (tiles < grid) grid = static_cast<int>(tiles);
-  e = launch_pdl(merge_exact_kernel, dim3(static_cast<unsigned>(grid)), dim3(kXThreads), smem, stream, 1, ta, tb, p);
+  if (tiles < grid) grid = tiles;
+  e = launch_pdl(merge_exact_kernel, dim3(static_cast<unsigned>(grid)), dim3(kXThreads), smem, stream, 1, xb);
   if (e != cudaSuccess) return e;
-  if (fix_count_out != nullptr) {
-    e = cudaMemsetAsync(counter, 0, sizeof(unsigned int), stream);
-    if (e != cudaSuccess) return e;
+  e = launch_pdl(exact_fix_kernel, dim3(static_cast<unsigned>(fix_ctas)), dim3(256), 0, stream, 1, fb);
+  if (e != cudaSuccess) return e;
+  a = 0;
+  for (int i = 0; i < count; ++i) {
+    if (layers[i].k == 0) continue;
+    if (layers[i].fix_count_out != nullptr) {
+      e = cudaMemcpyAsync(layers[i].fix_count_out, xs[a].counter, sizeof(unsigned int), cudaMemcpyDeviceToDevice, stream);
+      if (e != cudaSuccess) return e;
+    }
+    ++a;
   }
-  const int64_t words = k * p.words_per_row;
-  int64_t fgrid = (words + 255) / 256;
-  if (fgrid > static_cast<int64_t>(sm_count()) * 8) fgrid = static_cast<int64_t>(sm_count()) * 8;
-  e = launch_pdl(exact_fix_kernel, dim3(static_cast<unsigned>(fgrid)), dim3(256), 0, stream, 1, wq, aq, sel_idx, dprime, flags,
-                 words, n, static_cast<int>(r), static_cast<int>(r_pad), p.words_per_row,
-                 fix_count_out != nullptr ? counter : nullptr);
-  if (e != cudaSuccess) return e;
-  if (fix_count_out != nullptr)
-    e = cudaMemcpyAsync(fix_count_out, counter, sizeof(unsigned int), cudaMemcpyDeviceToDevice, stream);
-  return e;
+  return cudaSuccess;
+}
+
+cudaError_t launch_merge_exact(uint8_t* wq, float* dbuf, const int32_t* sel_idx, int64_t k, int64_t m, int64_t n, int64_t r,
+                               const float* row_scales, void* scratch, float* sums_out, unsigned int* fix_count_out, int* status,
+                               cudaStream_t stream) {
+  if (k < 1 || k > m || r < 8 || r > 256 || n % 16) return cudaErrorInvalidValue;
+  const ExactMergeLayer one{wq, dbuf, sel_idx, row_scales, scratch, sums_out, fix_count_out, m, n, r, k};
+  return launch_merge_exact_batched(&one, 1, false, status, stream);
 }
 
 }  // namespace falqon

@@ -117,3 +117,45 @@ def test_ties_tiny_terms_and_saturation_take_the_exact_path(fq, orc):
 def test_exact_merge_full_size(fq, orc, name, n, m, r, k):
     fixed, total = _run(fq, orc, 63, m, n, r, k, 2e-4, dbuf_scale=1e-3, want_sums=False)
     assert fixed <= 0.02 * total, f"{fixed} of {total} elements took the exact path"
+
+
+@pytest.mark.parametrize("prepared", [True, False])
+def test_batched_exact_equals_per_layer_calls_and_the_oracle(fq, orc, prepared):
+    """falqon_proxy_update_batched_exact: layers of different shapes, ranks, granularities and k (one with k = 0, one with
+    adversarially large DeltaBuffer entries so that many elements take the exact path) in one call, twice in a row (the
+    second call reuses the prepared copy of A~): bit-identical to the per-layer falqon_proxy_update_exact calls and to the
+    oracle's exact merge."""
+    specs = [(512, 384, 16, 40, False, 0.05), (272, 528, 64, 0, False, 0.05), (1024, 256, 128, 300, True, 0.05),
+             (384, 640, 8, 384, False, 5.0)]
+    lr = 0.05
+    per, bat, dBs, ks, oracle_state = [], [], [], [], []
+    for i, (m, n, r, k, per_row, scale) in enumerate(specs):
+        W, A, _, _ = layer_inputs(61, i, m, n, r, 16, 0)
+        if per_row:
+            W = synth.backbone(61, i, m, n, heavy_tailed=True)
+        a = fq.setup_layer(W.to(DEV), A.to(DEV), None, 1.0, per_row=per_row)
+        a.dbuf.copy_(synth.normal_bf16(61, 50 + i, (m, r), scale).float().to(DEV) * 1.0009765625)
+        b = fq.Layer(a.wq.clone(), a.s_w.clone(), a.dbuf.clone(), r)
+        per.append(a); bat.append(b); ks.append(k)
+        oracle_state.append((u8(a.wq).copy(), f32(a.dbuf).copy(), f32(a.s_w) if per_row else None))
+    batch = None
+    for call in range(2):
+        dBs = [(synth.normal_bf16(61, 70 + 10 * call + i, (L.m, L.r), 1.0).float() * 0.337).to(DEV) for i, L in enumerate(per)]
+        idx_per = [fq.proxy_update_exact(L, dB, lr, k, want_count=False)[0] for L, dB, k in zip(per, dBs, ks)]
+        if batch is None:
+            batch = fq.ProxyBatch(bat, dBs, ks)
+            batch.prepare_exact()
+        else:
+            batch = fq.ProxyBatch(bat, dBs, ks)
+            batch.scratch, batch.c_scratch, batch.c_scratch_bytes = keep
+        keep = (batch.scratch, batch.c_scratch, batch.c_scratch_bytes)
+        idx_bat = batch.run_exact(lr, prepared=prepared)
+        torch.cuda.synchronize()
+        for i, (La, Lb, ia, ib) in enumerate(zip(per, bat, idx_per, idx_bat)):
+            assert (ia is None and ib is None) or torch.equal(ia, ib), f"layer {i} call {call}: selected rows"
+            assert torch.equal(La.wq, Lb.wq), f"layer {i} call {call}: {int((La.wq != Lb.wq).sum())} codes differ"
+            assert torch.equal(La.dbuf.view(torch.int32), Lb.dbuf.view(torch.int32))
+            wq_o, dbuf_o, rs = oracle_state[i]
+            orc.proxy_update_exact(wq_o, dbuf_o, f32(dBs[i]), lr, ks[i], La.m, La.r, row_scales=rs)
+            assert np.array_equal(u8(Lb.wq), wq_o) and np.array_equal(bits32(f32(Lb.dbuf)), bits32(dbuf_o))
+    assert fq.last_device_status() == 0
