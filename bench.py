@@ -684,7 +684,7 @@ def main():
     def with_cycles(ms, clocks):
         """time x median SM clock of the pass: passes that ran at different clocks compare in cycles."""
         mhz = clocks.get("sm_mhz")
-        return None if mhz is None else ms * 1e-3 * mhz * 1e6 / 1e6      # million SM cycles per step
+        return None if mhz is None else ms * mhz * 1e-3      # ms x MHz = thousand cycles; / 1000 = million SM cycles per step
 
     step_fn = run_step
     if args.fused_update:
