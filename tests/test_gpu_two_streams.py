@@ -1,0 +1,42 @@
+"""Two layers driven from two streams at once.  The cast inside falqon_melded_forward / _backward is one kernel whose CTAs
+wait for one another at a grid-wide barrier; it is launched cooperatively, so the driver starts each such kernel only when
+its whole grid can be resident, whatever the other stream has running.  The results must be those of the same calls made
+one after another, and no bounded wait may run out."""
+import pytest
+import torch
+
+from helpers import layer_inputs
+from paper_2510_24061_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def test_forward_and_backward_of_two_layers_on_two_streams():
+    from paper_2510_24061_b200 import binding as fq
+    shapes = [(1024, 2048, 32, 2048), (2048, 1024, 64, 1536)]
+    layers, inputs, ref = [], [], []
+    for i, (m, n, r, T) in enumerate(shapes):
+        W, A, B, X = layer_inputs(71, i, m, n, r, T, 4, DEV)
+        dY = synth.out_grad(71, i, 0, T, m, DEV)
+        L = fq.setup_layer(W, A, B, 1.0)
+        ws = L.workspace(T)
+        layers.append((L, ws))
+        inputs.append((X, dY))
+        Y, OA, amax_oa, _ = fq.melded_forward(L, X, y_dtype=torch.float32, ws=ws)
+        dX, dB, _ = fq.melded_backward(L, dY, OA, amax_oa, dx_dtype=torch.float32, ws=ws)
+        ref.append((Y.clone(), OA.clone(), dX.clone(), dB.clone()))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [None, None]
+    for rep in range(8):                       # interleave the enqueues so that the two streams really overlap
+        for i, ((L, ws), (X, dY)) in enumerate(zip(layers, inputs)):
+            with torch.cuda.stream(streams[i]):
+                Y, OA, amax_oa, _ = fq.melded_forward(L, X, y_dtype=torch.float32, ws=ws)
+                dX, dB, _ = fq.melded_backward(L, dY, OA, amax_oa, dx_dtype=torch.float32, ws=ws)
+                outs[i] = (Y, OA, dX, dB)
+    torch.cuda.synchronize()
+    for got, want in zip(outs, ref):
+        for a, b in zip(got, want):
+            assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+    assert fq.last_device_status() == 0
