@@ -428,7 +428,7 @@ def run_stack(args):
     H, F, n_layers = 4096, 11008, args.stack_layers
     peaks = measured_peaks()
     stack = st.Stack(n_layers, H, F, T, r, k, seed=cfg["seed"], device=dev, lr=lr, producer_amax=not args.stack_own_absmax,
-                     batched_proxy=not args.proxy_per_layer,
+                     batched_proxy=not args.proxy_per_layer, fuse_chain=not args.stack_unfused_chain,
                      adamw=dict(beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0) if args.stack_adamw else None)
     h0 = synth.normal_bf16(cfg["seed"], 9001, (T, H), 1.0, dev)
     G = synth.normal_bf16(cfg["seed"], 9002, (T, H), 1.0e-2, dev)
@@ -547,6 +547,8 @@ def main():
     ap.add_argument("--stack-layers", type=int, default=32)
     ap.add_argument("--stack-own-absmax", action="store_true",
                     help="with --stack: every layer takes the absmax of its input itself (the chain kernels do not hand it over)")
+    ap.add_argument("--stack-unfused-chain", action="store_true",
+                    help="with --stack: residual sums and the normalisations (or their gradients) that follow them as separate kernels")
     ap.add_argument("--stack-adamw", action="store_true",
                     help="with --stack: AdamW (beta 0.9 / 0.999, eps 1e-8, no weight decay) on every DeltaBuffer instead of plain SGD")
     ap.add_argument("--config3", action="store_true",

@@ -39,6 +39,17 @@ int falqon_chain_rmsnorm(void *y, float *inv_rms, const void *x, int64_t rows, i
 int falqon_chain_rmsnorm_grad(void *dx, const void *dy, const void *x, const float *inv_rms, int64_t rows,
                               int64_t cols, falqon_stream stream);
 
+/* falqon_chain_combine (two inputs) followed by falqon_chain_rmsnorm of its result, in one pass: sum_out = bf16(sa*a + sb*b)
+ * is stored, y = rmsnorm(sum_out) with inv_rms kept.  Bit for bit the two calls; saves writing the sum and reading it back. */
+int falqon_chain_combine_rmsnorm(void *sum_out, void *y, float *inv_rms, const void *a, float sa, const void *b, float sb,
+                                 int64_t rows, int64_t cols, float eps, float *amax_out, falqon_stream stream);
+
+/* Three calls in one pass: dy = bf16(dy_a + dy_b (+ dy_c, nullable));  g = falqon_chain_rmsnorm_grad(dy, x, inv_rms);
+ * out = bf16(s_res * res + g).  Bit for bit the three calls.  out may alias dy_a, dy_b, dy_c or res. */
+int falqon_chain_rmsnorm_grad_combine(void *out, const void *dy_a, const void *dy_b, const void *dy_c, const void *x,
+                                      const float *inv_rms, const void *res, float s_res, int64_t rows, int64_t cols,
+                                      float *amax_out, falqon_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

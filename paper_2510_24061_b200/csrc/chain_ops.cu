@@ -215,6 +215,113 @@ __global__ void __launch_bounds__(kNormThreads) rmsnorm_grad_kernel(uint4* dx, c
   }
 }
 
+// sum = bf16(sa * a + sb * b), stored, and the RMS normalisation of that stored (rounded) sum, in one pass over the row:
+// the results are bit for bit those of combine_kernel followed by rmsnorm_kernel, without writing the sum and reading it back.
+__global__ void __launch_bounds__(kNormThreads) combine_rmsnorm_kernel(uint4* sum_out, uint4* y, float* inv_rms, const uint4* a,
+                                                                       float sa, const uint4* b, float sb, int vec_per_row,
+                                                                       float inv_cols, float eps, float* amax) {
+  __shared__ float red[4];
+  pdl_trigger();
+  pdl_wait();
+  const int64_t base = static_cast<int64_t>(blockIdx.x) * vec_per_row;
+  uint4 raw[kNormMaxVec];
+  float ss = 0.0f;
+#pragma unroll
+  for (int i = 0; i < kNormMaxVec; ++i) {
+    const int v = threadIdx.x + i * kNormThreads;
+    if (v < vec_per_row) {
+      float fa[8], fb[8], acc[8];
+      unpack8(ld_stream(a + base + v), fa);
+      unpack8(ld_stream(b + base + v), fb);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = __fmaf_rn(sb, fb[e], __fmul_rn(sa, fa[e]));
+      raw[i] = pack8(acc);
+      sum_out[base + v] = raw[i];
+      float f[8];
+      unpack8(raw[i], f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) ss = __fmaf_rn(f[e], f[e], ss);
+    }
+  }
+  const float inv = rsqrtf(block_sum_128(ss, red) * inv_cols + eps);
+  if (threadIdx.x == 0) inv_rms[blockIdx.x] = inv;
+  uint32_t mx = 0;
+#pragma unroll
+  for (int i = 0; i < kNormMaxVec; ++i) {
+    const int v = threadIdx.x + i * kNormThreads;
+    if (v < vec_per_row) {
+      float f[8];
+      unpack8(raw[i], f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) f[e] *= inv;
+      const uint4 o = pack8(f);
+      y[base + v] = o;
+      mx = max_abs_bf16(o, mx);
+    }
+  }
+  if (amax != nullptr) publish_amax(mx, amax);
+}
+
+// out = bf16(s_res * res + g) with g = rmsnorm_grad(dy, x, inv_rms) and dy = bf16(dy_a + dy_b (+ dy_c)), in one pass over
+// the row: bit for bit combine_kernel, rmsnorm_grad_kernel, combine_kernel in a row (the two intermediates are rounded to
+// bf16 in registers exactly as they would be in memory).
+__global__ void __launch_bounds__(kNormThreads) rmsnorm_grad_combine_kernel(uint4* out, const uint4* dy_a, const uint4* dy_b,
+                                                                            const uint4* dy_c, const uint4* x,
+                                                                            const float* inv_rms, const uint4* res, float s_res,
+                                                                            int vec_per_row, float inv_cols, float* amax) {
+  __shared__ float red[4];
+  pdl_trigger();
+  pdl_wait();
+  const int64_t base = static_cast<int64_t>(blockIdx.x) * vec_per_row;
+  const float inv = ld_stream(inv_rms + blockIdx.x);
+  uint4 rx[kNormMaxVec], rdy[kNormMaxVec];
+  float dot = 0.0f;
+#pragma unroll
+  for (int i = 0; i < kNormMaxVec; ++i) {
+    const int v = threadIdx.x + i * kNormThreads;
+    if (v < vec_per_row) {
+      float fa[8], fb[8], acc[8];
+      rx[i] = ld_stream(x + base + v);
+      unpack8(ld_stream(dy_a + base + v), fa);
+      unpack8(ld_stream(dy_b + base + v), fb);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = __fmaf_rn(1.0f, fb[e], __fmul_rn(1.0f, fa[e]));
+      if (dy_c != nullptr) {
+        unpack8(ld_stream(dy_c + base + v), fb);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = __fmaf_rn(1.0f, fb[e], acc[e]);
+      }
+      rdy[i] = pack8(acc);
+      float fx[8], fd[8];
+      unpack8(rx[i], fx);
+      unpack8(rdy[i], fd);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) dot = __fmaf_rn(fd[e], fx[e] * inv, dot);
+    }
+  }
+  const float mean = block_sum_128(dot, red) * inv_cols;
+  uint32_t mx = 0;
+#pragma unroll
+  for (int i = 0; i < kNormMaxVec; ++i) {
+    const int v = threadIdx.x + i * kNormThreads;
+    if (v < vec_per_row) {
+      float fx[8], fd[8], o[8], fr[8], g[8];
+      unpack8(rx[i], fx);
+      unpack8(rdy[i], fd);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) o[e] = inv * (fd[e] - fx[e] * inv * mean);
+      unpack8(pack8(o), g);                       // the gradient as the separate kernel would have stored it
+      unpack8(ld_stream(res + base + v), fr);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) o[e] = __fmaf_rn(1.0f, g[e], __fmul_rn(s_res, fr[e]));
+      const uint4 q = pack8(o);
+      out[base + v] = q;
+      mx = max_abs_bf16(q, mx);
+    }
+  }
+  if (amax != nullptr) publish_amax(mx, amax);
+}
+
 inline bool ok16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 inline unsigned chain_grid(int64_t nvec) {
   int64_t blocks = (nvec + kChainThreads - 1) / kChainThreads;
@@ -282,6 +389,34 @@ int falqon_chain_rmsnorm_grad(void* dx, const void* dy, const void* x, const flo
   cudaError_t e = launch_pdl(rmsnorm_grad_kernel, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
                              static_cast<cudaStream_t>(stream), 1, static_cast<uint4*>(dx), static_cast<const uint4*>(dy),
                              static_cast<const uint4*>(x), inv_rms, static_cast<int>(cols / 8), 1.0f / static_cast<float>(cols));
+  return e == cudaSuccess ? FALQON_OK : FALQON_ERR_CUDA;
+}
+
+int falqon_chain_combine_rmsnorm(void* sum_out, void* y, float* inv_rms, const void* a, float sa, const void* b, float sb,
+                                 int64_t rows, int64_t cols, float eps, float* amax_out, falqon_stream stream) {
+  if (sum_out == nullptr || y == nullptr || inv_rms == nullptr || a == nullptr || b == nullptr || rows < 1 || rows > (1ll << 30) ||
+      cols < 8 || cols % 8 || cols > kNormThreads * kNormMaxVec * 8 || !ok16(sum_out) || !ok16(y) || !ok16(a) || !ok16(b) ||
+      !(eps >= 0.0f))
+    return FALQON_ERR_INVALID_ARG;
+  cudaError_t e = launch_pdl(combine_rmsnorm_kernel, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
+                             static_cast<cudaStream_t>(stream), 1, static_cast<uint4*>(sum_out), static_cast<uint4*>(y), inv_rms,
+                             static_cast<const uint4*>(a), sa, static_cast<const uint4*>(b), sb, static_cast<int>(cols / 8),
+                             1.0f / static_cast<float>(cols), eps, amax_out);
+  return e == cudaSuccess ? FALQON_OK : FALQON_ERR_CUDA;
+}
+
+int falqon_chain_rmsnorm_grad_combine(void* out, const void* dy_a, const void* dy_b, const void* dy_c, const void* x,
+                                      const float* inv_rms, const void* res, float s_res, int64_t rows, int64_t cols,
+                                      float* amax_out, falqon_stream stream) {
+  if (out == nullptr || dy_a == nullptr || dy_b == nullptr || x == nullptr || inv_rms == nullptr || res == nullptr || rows < 1 ||
+      rows > (1ll << 30) || cols < 8 || cols % 8 || cols > kNormThreads * kNormMaxVec * 8 || !ok16(out) || !ok16(dy_a) ||
+      !ok16(dy_b) || !ok16(dy_c) || !ok16(x) || !ok16(res))
+    return FALQON_ERR_INVALID_ARG;
+  cudaError_t e = launch_pdl(rmsnorm_grad_combine_kernel, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
+                             static_cast<cudaStream_t>(stream), 1, static_cast<uint4*>(out), static_cast<const uint4*>(dy_a),
+                             static_cast<const uint4*>(dy_b), static_cast<const uint4*>(dy_c), static_cast<const uint4*>(x), inv_rms,
+                             static_cast<const uint4*>(res), s_res, static_cast<int>(cols / 8), 1.0f / static_cast<float>(cols),
+                             amax_out);
   return e == cudaSuccess ? FALQON_OK : FALQON_ERR_CUDA;
 }
 

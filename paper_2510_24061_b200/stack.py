@@ -37,8 +37,12 @@ lib.falqon_chain_rmsnorm.restype = C.c_int
 lib.falqon_chain_rmsnorm.argtypes = [_p, _p, _p, _i64, _i64, _f, _p, _p]
 lib.falqon_chain_rmsnorm_grad.restype = C.c_int
 lib.falqon_chain_rmsnorm_grad.argtypes = [_p, _p, _p, _p, _i64, _i64, _p]
+lib.falqon_chain_combine_rmsnorm.restype = C.c_int
+lib.falqon_chain_combine_rmsnorm.argtypes = [_p, _p, _p, _p, _f, _p, _f, _i64, _i64, _f, _p, _p]
+lib.falqon_chain_rmsnorm_grad_combine.restype = C.c_int
+lib.falqon_chain_rmsnorm_grad_combine.argtypes = [_p, _p, _p, _p, _p, _p, _p, _f, _i64, _i64, _p, _p]
 CHAIN_EXPORTS = ["falqon_chain_combine", "falqon_chain_silu_mul", "falqon_chain_silu_mul_grad", "falqon_chain_rmsnorm",
-                 "falqon_chain_rmsnorm_grad"]
+                 "falqon_chain_rmsnorm_grad", "falqon_chain_combine_rmsnorm", "falqon_chain_rmsnorm_grad_combine"]
 NORM_EPS = 1e-6
 
 PROJ = ["q", "k", "v", "o", "gate", "up", "down"]
@@ -91,11 +95,35 @@ def rmsnorm_grad(dx, dy, x, inv_rms):
     return dx
 
 
+def combine_rmsnorm(sum_out, y, inv_rms, a, sa, b, sb, amax=None):
+    """sum_out = bf16(sa*a + sb*b) and y = rmsnorm(sum_out) in one pass (bit for bit combine followed by rmsnorm)."""
+    for t in (sum_out, y, a, b):
+        assert t.dtype == torch.bfloat16 and t.dim() == 2 and t.is_contiguous() and t.shape == a.shape
+    assert inv_rms.dtype == torch.float32 and inv_rms.numel() == a.shape[0]
+    fq._check("falqon_chain_combine_rmsnorm",
+              lib.falqon_chain_combine_rmsnorm(_ptr(sum_out), _ptr(y), _ptr(inv_rms), _ptr(a), sa, _ptr(b), sb, a.shape[0], a.shape[1],
+                                               NORM_EPS, _ptr(amax), fq._stream()))
+    return y
+
+
+def rmsnorm_grad_combine(out, dys, x, inv_rms, res, s_res, amax=None):
+    """out = bf16(s_res*res + rmsnorm_grad(bf16(sum of the two or three dys), x, inv_rms)) in one pass (bit for bit the three
+    separate kernels)."""
+    assert len(dys) in (2, 3)
+    for t in (out, x, res, *dys):
+        assert t.dtype == torch.bfloat16 and t.is_contiguous() and t.shape == x.shape
+    fq._check("falqon_chain_rmsnorm_grad_combine",
+              lib.falqon_chain_rmsnorm_grad_combine(_ptr(out), _ptr(dys[0]), _ptr(dys[1]), _ptr(dys[2]) if len(dys) == 3 else None,
+                                                    _ptr(x), _ptr(inv_rms), _ptr(res), s_res, x.shape[0], x.shape[1], _ptr(amax),
+                                                    fq._stream()))
+    return out
+
+
 class Stack:
     """n_layers blocks with hidden size H and MLP width F, T tokens per step, LoRA rank r, top-k rows per update."""
 
     def __init__(self, n_layers: int, H: int, F: int, T: int, r: int, k: int, seed: int, device, lr: float = 2e-4,
-                 producer_amax: bool = True, batched_proxy: bool = True, adamw: dict | None = None):
+                 producer_amax: bool = True, batched_proxy: bool = True, adamw: dict | None = None, fuse_chain: bool = True):
         """producer_amax: the chain kernels hand the absmax of their outputs to the layers that consume them, whose
         input casts are then single-pass (False: every layer takes the absmax of its input itself).
         batched_proxy: the seven proxy updates of a block run as one falqon_proxy_update_batched call at the end of
@@ -107,6 +135,7 @@ class Stack:
         self.adamw, self.steps_done = adamw, 0
         assert adamw is None or batched_proxy
         self.producer_amax = producer_amax
+        self.fuse_chain = fuse_chain        # residual sums fused with the normalisation (or its gradient) that follows them
         self.device = torch.device(device)
         self.seed = seed
         self.shapes = {"q": (H, H), "k": (H, H), "v": (H, H), "o": (H, H), "gate": (H, F), "up": (H, F), "down": (F, H)}  # n -> m
@@ -204,20 +233,27 @@ class Stack:
             if l == 0:
                 sv["h"].copy_(h0)
             h, hp = sv["h"], sv["hp"]
-            rmsnorm(self.x1, sv["inv1"], h, amax=self._am(l, 0))
+            if l == 0 or not self.fuse_chain:      # (fused: the block before has already normalised its output into x1)
+                rmsnorm(self.x1, sv["inv1"], h, amax=self._am(l, 0))
             self._fwd(l, "q", self.x1, self.q, self._am(l, 0))
             self._fwd_shared(l, "k", "q", self.x1, self.kk)
             self._fwd_shared(l, "v", "q", self.x1, self.v)
             combine(self.a, self.q, INV_SQRT3, self.kk, INV_SQRT3, self.v, INV_SQRT3, amax=self._am(l, 1))
             self._fwd(l, "o", self.a, self.o, self._am(l, 1))
-            combine(hp, h, 1.0, self.o, 1.0)
-            rmsnorm(self.x2, sv["inv2"], hp, amax=self._am(l, 2))
+            if self.fuse_chain:
+                combine_rmsnorm(hp, self.x2, sv["inv2"], h, 1.0, self.o, 1.0, amax=self._am(l, 2))
+            else:
+                combine(hp, h, 1.0, self.o, 1.0)
+                rmsnorm(self.x2, sv["inv2"], hp, amax=self._am(l, 2))
             self._fwd(l, "gate", self.x2, sv["g"], self._am(l, 2))
             self._fwd_shared(l, "up", "gate", self.x2, sv["u"])
             silu_mul(self.z, sv["g"], sv["u"], amax=self._am(l, 3))
             self._fwd(l, "down", self.z, self.dn, self._am(l, 3))
             out = self.saved[l + 1]["h"] if l + 1 < self.n_layers else self.h_out   # the next block's saved input
-            combine(out, hp, INV_SQRT2, self.dn, INV_SQRT2)
+            if self.fuse_chain and l + 1 < self.n_layers:   # ... and, in the same pass, its first normalisation
+                combine_rmsnorm(out, self.x1, self.saved[l + 1]["inv1"], hp, INV_SQRT2, self.dn, INV_SQRT2, amax=self._am(l + 1, 0))
+            else:
+                combine(out, hp, INV_SQRT2, self.dn, INV_SQRT2)
         return self.h_out
 
     def backward(self, G: torch.Tensor):
@@ -231,17 +267,23 @@ class Stack:
             silu_mul_grad(self.dg, self.du, sv["g"], sv["u"], self.dz, self._am(l, 5), self._am(l, 6))
             self._bwd(l, "gate", self.dg, self.dx[0], self._am(l, 5))
             self._bwd(l, "up", self.du, self.dx[1], self._am(l, 6))
-            combine(self.dx[0], self.dx[0], 1.0, self.dx[1], 1.0)               # d x2
-            rmsnorm_grad(self.dx[1], self.dx[0], sv["hp"], sv["inv2"])
-            combine(self.dhp, dh, INV_SQRT2, self.dx[1], 1.0, amax=self._am(l, 7))   # dh' = dh/sqrt(2) + norm'(d x2)
+            if self.fuse_chain:                                                 # dh' = dh/sqrt(2) + norm'(d x2), d x2 = the two dX
+                rmsnorm_grad_combine(self.dhp, [self.dx[0], self.dx[1]], sv["hp"], sv["inv2"], dh, INV_SQRT2, amax=self._am(l, 7))
+            else:
+                combine(self.dx[0], self.dx[0], 1.0, self.dx[1], 1.0)               # d x2
+                rmsnorm_grad(self.dx[1], self.dx[0], sv["hp"], sv["inv2"])
+                combine(self.dhp, dh, INV_SQRT2, self.dx[1], 1.0, amax=self._am(l, 7))   # dh' = dh/sqrt(2) + norm'(d x2)
             self._bwd(l, "o", self.dhp, self.da, self._am(l, 7))
             combine(self.dqkv, self.da, INV_SQRT3, amax=self._am(l, 8))         # dq = dk = dv = da / sqrt(3)
             self._bwd(l, "q", self.dqkv, self.dx[0], self._am(l, 8))
             self._bwd(l, "k", self.dqkv, self.dx[1], self._am(l, 8))
             self._bwd(l, "v", self.dqkv, self.dx[2], self._am(l, 8))
-            combine(self.dx[0], self.dx[0], 1.0, self.dx[1], 1.0, self.dx[2], 1.0)   # d x1
-            rmsnorm_grad(self.dx[1], self.dx[0], sv["h"], sv["inv1"])
-            combine(self.dh, self.dhp, 1.0, self.dx[1], 1.0)
+            if self.fuse_chain:                                                 # dh = dh' + norm'(d x1), d x1 = the three dX
+                rmsnorm_grad_combine(self.dh, [self.dx[0], self.dx[1], self.dx[2]], sv["h"], sv["inv1"], self.dhp, 1.0)
+            else:
+                combine(self.dx[0], self.dx[0], 1.0, self.dx[1], 1.0, self.dx[2], 1.0)   # d x1
+                rmsnorm_grad(self.dx[1], self.dx[0], sv["h"], sv["inv1"])
+                combine(self.dh, self.dhp, 1.0, self.dx[1], 1.0)
             dh = self.dh
             if self.batches is not None:
                 if self.adamw is None:
@@ -273,7 +315,10 @@ class Stack:
         if self.batches is not None:
             per_block += fq.launch_count("falqon_proxy_update_batched", k=self.k)
         per_block += 6 + 9   # chain kernels: forward 6 (2 norms, mix, 2 residuals, gate), backward 9
-        return per_block * self.n_layers
+        total = per_block * self.n_layers
+        if self.fuse_chain:  # per block 2 residual + norm pairs in one launch each (the last block keeps its plain residual, the
+            total -= self.n_layers * (2 + 4) - 1   # first its plain norm) and 2 x (sum, norm gradient, residual) in one each
+        return total
 
     def bytes_resident(self) -> int:
         tot = 0

@@ -99,6 +99,55 @@ def test_chain_rmsnorm_and_its_gradient(st):
     assert torch.allclose(dx.cpu().double(), xa.grad, rtol=2e-2, atol=1e-3)
 
 
+def test_fused_chain_kernels_equal_the_separate_ones_bit_for_bit(st):
+    """combine + rmsnorm in one pass, and sum + rmsnorm gradient + residual in one pass, against the kernels they replace
+    (which the tests above check against the formulas): identical bits, identical absmax hand-over."""
+    torch.manual_seed(3)
+    rows, cols = 53, 8 * 77
+    mk = lambda scale=1.0: (torch.randn(rows, cols) * scale).to(torch.bfloat16).to(DEV)
+    a, b, c, x, res = mk(2.0), mk(0.5), mk(), mk(3.0), mk()
+    s1, y1, s2, y2 = (torch.empty_like(a) for _ in range(4))
+    inv1, inv2 = (torch.empty(rows, dtype=torch.float32, device=DEV) for _ in range(2))
+    am1, am2 = (torch.zeros(1, dtype=torch.float32, device=DEV) for _ in range(2))
+    st.combine(s1, a, st.INV_SQRT2, b, st.INV_SQRT2)
+    st.rmsnorm(y1, inv1, s1, amax=am1)
+    st.combine_rmsnorm(s2, y2, inv2, a, st.INV_SQRT2, b, st.INV_SQRT2, amax=am2)
+    assert torch.equal(s1.view(torch.int16), s2.view(torch.int16)) and torch.equal(y1.view(torch.int16), y2.view(torch.int16))
+    assert torch.equal(inv1.view(torch.int32), inv2.view(torch.int32)) and float(am1) == float(am2)
+    for dys in ([a, b], [a, b, c]):
+        t, g, o1, o2 = (torch.empty_like(a) for _ in range(4))
+        am1.zero_(); am2.zero_()
+        st.combine(t, dys[0], 1.0, dys[1], 1.0, dys[2] if len(dys) == 3 else None, 1.0)
+        st.rmsnorm_grad(g, t, x, inv1)
+        st.combine(o1, res, st.INV_SQRT2, g, 1.0, amax=am1)
+        st.rmsnorm_grad_combine(o2, dys, x, inv1, res, st.INV_SQRT2, amax=am2)
+        assert torch.equal(o1.view(torch.int16), o2.view(torch.int16)) and float(am1) == float(am2)
+        # in place on the residual, as the stack does not, and on a gradient operand, as it may
+        o3 = dys[0].clone()
+        st.rmsnorm_grad_combine(o3, [o3, *dys[1:]], x, inv1, res, st.INV_SQRT2)
+        assert torch.equal(o1.view(torch.int16), o3.view(torch.int16))
+
+
+def test_stack_with_fused_chain_equals_the_unfused_stack(fq, st):
+    """Three narrow blocks, one step each way: outputs, input gradient, every backbone and DeltaBuffer identical."""
+    H, F, T, r, k = 256, 512, 300, 16, 24
+    dev = torch.device(DEV)
+    h0 = synth.normal_bf16(5, 9001, (T, H), 1.0, dev)
+    G = synth.normal_bf16(5, 9002, (T, H), 1.0e-2, dev)
+    outs = []
+    for fuse in (False, True):
+        stack = st.Stack(3, H, F, T, r, k, seed=5, device=dev, lr=2e-2, fuse_chain=fuse)
+        h = stack.forward(h0).clone()
+        dh = stack.backward(G).clone()
+        torch.cuda.synchronize()
+        outs.append((h, dh, [(L.wq.clone(), L.dbuf.clone()) for blk in stack.layers for L in (blk.values() if isinstance(blk, dict) else blk)]))
+    (h_a, dh_a, la), (h_b, dh_b, lb) = outs
+    assert torch.equal(h_a.view(torch.int16), h_b.view(torch.int16)) and torch.equal(dh_a.view(torch.int16), dh_b.view(torch.int16))
+    for (wa, da), (wb, db) in zip(la, lb):
+        assert torch.equal(wa, wb) and torch.equal(da.view(torch.int32), db.view(torch.int32))
+    assert fq.last_device_status() == 0
+
+
 def _close_bf16(gpu: torch.Tensor, ref_f32: np.ndarray, what: str):
     """A bf16 tensor-core output against the oracle's fp32 result: every element within one bf16 step of the
     oracle's value (plus a floor of 2e-5 of the tensor's rms for elements that cancel to almost nothing), and
