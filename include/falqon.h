@@ -197,6 +197,17 @@ int falqon_melded_backward_amax(const falqon_layer *L, const void *dY, falqon_dt
                                 const float *OA, const float *amax_oa, void *dX, falqon_dtype dx_dt, float *dB,
                                 float *s_g_out, void *ws, size_t ws_bytes, falqon_stream stream);
 
+/* falqon_melded_backward for an output gradient that is already quantized: several layers that receive the same gradient
+ * (the q, k and v projections of a block whose outputs are summed) share one g~, as falqon_melded_forward_codes shares x~.
+ *   gq   device [T][m] E5M2 codes, e.g. the FALQON_WS_GQ region of the workspace of the layer whose
+ *        falqon_melded_backward cast the same dY
+ *   s_g  device [1], the scale they were cast with (entry 3 of that workspace's FALQON_WS_SCALES)
+ * O_A is still cast here (it is the layer's own).  Per-tensor scaled layers only (FALQON_ERR_UNSUPPORTED otherwise: a
+ * per-row layer's codes are those of dY divided by its own row scales).  This call's workspace holds no g~ afterwards. */
+int falqon_melded_backward_codes(const falqon_layer *L, const uint8_t *gq, const float *s_g, int64_t T, const float *OA,
+                                 const float *amax_oa, void *dX, falqon_dtype dx_dt, float *dB, void *ws, size_t ws_bytes,
+                                 falqon_stream stream);
+
 /* The second half of falqon_melded_backward as a call of its own (the input-gradient product implied by Alg. 3): after a
  * falqon_melded_backward[_amax] with dX == NULL -- which casts dY and O_A and computes dB -- this call computes
  *   dX = g~ * W~ / (s_W * s_g)

@@ -23,7 +23,7 @@ WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 
 EXPORTS = ["falqon_absmax", "falqon_selftest_wait_timeout", "falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
            "falqon_melded_forward_codes", "falqon_melded_forward_amax", "falqon_melded_backward_amax",
-           "falqon_melded_forward_dump", "falqon_melded_backward_dump", "falqon_melded_backward_dx",
+           "falqon_melded_forward_dump", "falqon_melded_backward_dump", "falqon_melded_backward_dx", "falqon_melded_backward_codes",
            "falqon_exact_merge_prepare", "falqon_proxy_update_batched_exact",
            "falqon_update_a", "falqon_update_a_scratch_bytes", "falqon_update_a_region",
            "falqon_melded_backward_update", "falqon_proxy_update_scored", "falqon_proxy_update_scored_batched", "falqon_exact_merge_scratch_bytes", "falqon_proxy_update_exact",
@@ -82,6 +82,8 @@ lib.falqon_proxy_update_scored.argtypes = [C.POINTER(falqon_layer), _i64, _p, _p
 lib.falqon_proxy_update_scored_batched.restype = _i
 lib.falqon_proxy_update_scored_batched.argtypes = [C.POINTER(falqon_layer), C.c_int32, C.POINTER(_i64), C.POINTER(_p), C.POINTER(_p),
                                                    C.POINTER(_sz), _p]
+lib.falqon_melded_backward_codes.restype = _i
+lib.falqon_melded_backward_codes.argtypes = [C.POINTER(falqon_layer), _p, _p, _i64, _p, _p, _p, _i, _p, _p, _sz, _p]
 lib.falqon_melded_backward_dx.restype = _i
 lib.falqon_melded_backward_dx.argtypes = [C.POINTER(falqon_layer), _i64, _p, _i, _p, _sz, _p]
 lib.falqon_melded_forward_codes.restype = _i
@@ -413,6 +415,25 @@ def proxy_update_scored(layer: Layer, k: int, ws: torch.Tensor | None = None, id
     _check("falqon_proxy_update_scored", lib.falqon_proxy_update_scored(C.byref(layer.c), k, _ptr(idx_out), _ptr(ws), ws.numel(),
                                                                         _stream()))
     return idx_out
+
+
+def melded_backward_codes(layer: Layer, gq: torch.Tensor, s_g: torch.Tensor, OA: torch.Tensor, amax_oa: torch.Tensor,
+                          need_dx: bool = True, dx_dtype=torch.bfloat16, ws: torch.Tensor | None = None, out=None):
+    """falqon_melded_backward_codes: the backward on gradient codes another layer already cast (gq uint8 [T, m], s_g fp32 [1]).
+    Returns (dX or None, dB)."""
+    assert gq.dim() == 2 and gq.is_contiguous() and gq.shape[1] == layer.m and gq.dtype == torch.uint8
+    T = gq.shape[0]
+    dev = gq.device
+    ws = layer.workspace(T) if ws is None else ws
+    if out is None:
+        dX = torch.empty((T, layer.n), dtype=dx_dtype, device=dev) if need_dx else None
+        dB = torch.empty((layer.m, layer.r), dtype=torch.float32, device=dev)
+    else:
+        dX, dB = out
+    _check("falqon_melded_backward_codes",
+           lib.falqon_melded_backward_codes(C.byref(layer.c), _ptr(gq), _ptr(s_g), T, _ptr(OA), _ptr(amax_oa), _ptr(dX),
+                                            _dt(dX) if dX is not None else BF16, _ptr(dB), _ptr(ws), ws.numel(), _stream()))
+    return dX, dB
 
 
 def melded_backward_dx(layer: Layer, T: int, dx_dtype=torch.bfloat16, ws: torch.Tensor | None = None, out: torch.Tensor | None = None):

@@ -447,6 +447,49 @@ int falqon_melded_backward_update(const falqon_layer* L, const void* dY, falqon_
   return backward_impl(L, dY, dy_dt, amax_dy, T, OA, amax_oa, dX, dx_dt, dB, s_g_out, ws, ws_bytes, stream, -1, &lr);
 }
 
+int falqon_melded_backward_codes(const falqon_layer* L, const uint8_t* gq, const float* s_g, int64_t T, const float* OA,
+                                 const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, void* ws, size_t ws_bytes,
+                                 falqon_stream stream) {
+  if (!layer_ok(L) || gq == nullptr || s_g == nullptr || OA == nullptr || amax_oa == nullptr || dB == nullptr || T < 1 ||
+      !dtype_ok(dx_dt) || !aligned16(gq) || !aligned16(OA) || !aligned16(dB) || (dX != nullptr && !aligned16(dX)))
+    return FALQON_ERR_INVALID_ARG;
+  if (L->gran == FALQON_PER_ROW) return FALQON_ERR_UNSUPPORTED;   // there the codes are those of dY / s_w[column]: the layer's own
+  WorkspaceLayout w;
+  if (!make_layout(L->m, L->n, L->r, T, &w)) return FALQON_ERR_INVALID_ARG;
+  if (ws == nullptr || !aligned16(ws) || ws_bytes < w.total) return FALQON_ERR_WORKSPACE;
+  int* status = status_ptr();
+  if (status == nullptr) return FALQON_ERR_CUDA;
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  float* scales = reinterpret_cast<float*>(base + w.scales);
+  uint8_t* oaq_t = base + w.oaq_t;
+  const int64_t m = L->m, n = L->n, r = L->r;
+  {
+    StageTimer timer(FALQON_STAGE_QUANT_DY, stream);   // only S5a is left of this stage
+    const OaCastJob oa_cast{OA, amax_oa, T, static_cast<int>(r), w.t16, oaq_t, scales + 5, scales + 4};
+    FALQON_CUDA(launch_oa_cast(oa_cast, stream));
+  }
+  {
+    DbFusedProblem d{};
+    d.m = m; d.r = r; d.T = T;
+    d.gq = gq; d.oaq_t = oaq_t; d.ldt = w.t16; d.s_oa = scales + 5; d.s_g = s_g; d.dB = dB; d.status = status;
+    StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
+    FALQON_CUDA(launch_db_fused(d, stream));
+  }
+  if (dX != nullptr) {
+    GemmProblem g{};
+    g.M = T; g.N = n; g.K = m;
+    g.a = gq; g.lda = m; g.a_fmt = kE5M2;
+    g.b = L->wq; g.ldb = n; g.b_mn_major = true; g.b_fmt = kE4M3;
+    g.block_n = 256;
+    g.c0 = dX; g.ldc0 = n; g.c0_dt = dx_dt; g.n_split = n;
+    g.scale_a = s_g; g.scale_b = L->s_w;
+    g.status = status;
+    StageTimer timer(FALQON_STAGE_GEMM_DX, stream);
+    FALQON_CUDA(launch_gemm_fp8(g, stream));
+  }
+  return FALQON_OK;
+}
+
 int falqon_melded_backward_dx(const falqon_layer* L, int64_t T, void* dX, falqon_dtype dx_dt, void* ws, size_t ws_bytes,
                               falqon_stream stream) {
   if (!layer_ok(L) || dX == nullptr || T < 1 || !dtype_ok(dx_dt) || !aligned16(dX)) return FALQON_ERR_INVALID_ARG;

@@ -221,6 +221,21 @@ class Stack:
             fq.proxy_update(self.layers[l][name], self.dB[name], self.lr, self.k, ws=self.ws[name],
                             idx_out=self.idx if self.k > 0 else None)
 
+    def _bwd_shared(self, l, name, owner, dY, dX):
+        """The backward of a projection whose output gradient is the one `owner` has just cast (q, k and v all receive
+        da / sqrt(3)): it multiplies the owner's codes instead of casting dY again."""
+        m = self.shapes[name][1]
+        lo = self.layers[l][owner]
+        gq = fq.ws_view(lo, self.ws[owner], self.T, fq.WS_GQ)[: self.T * m].view(self.T, m)
+        s_g = fq.ws_view(lo, self.ws[owner], self.T, fq.WS_SCALES).view(torch.float32)[3:4]
+        sv = self.saved[l]
+        fq.melded_backward_codes(self.layers[l][name], gq, s_g, sv["oa"][name], sv["amax"][name], ws=self.ws[name],
+                                 out=(dX, self.dB[name]))
+        self._cap(l, name, dY=dY, dX=dX, dB=self.dB[name], OA=sv["oa"][name])
+        if self.batches is None:
+            fq.proxy_update(self.layers[l][name], self.dB[name], self.lr, self.k, ws=self.ws[name],
+                            idx_out=self.idx if self.k > 0 else None)
+
     def _cap(self, l, name, **tensors):
         if self.capture is not None and (l, name) in self.capture:
             self.capture[(l, name)].update({k2: v.clone() for k2, v in tensors.items()})
@@ -276,8 +291,8 @@ class Stack:
             self._bwd(l, "o", self.dhp, self.da, self._am(l, 7))
             combine(self.dqkv, self.da, INV_SQRT3, amax=self._am(l, 8))         # dq = dk = dv = da / sqrt(3)
             self._bwd(l, "q", self.dqkv, self.dx[0], self._am(l, 8))
-            self._bwd(l, "k", self.dqkv, self.dx[1], self._am(l, 8))
-            self._bwd(l, "v", self.dqkv, self.dx[2], self._am(l, 8))
+            self._bwd_shared(l, "k", "q", self.dqkv, self.dx[1])       # the same gradient: q's codes serve all three
+            self._bwd_shared(l, "v", "q", self.dqkv, self.dx[2])
             if self.fuse_chain:                                                 # dh = dh' + norm'(d x1), d x1 = the three dX
                 rmsnorm_grad_combine(self.dh, [self.dx[0], self.dx[1], self.dx[2]], sv["h"], sv["inv1"], self.dhp, 1.0)
             else:
@@ -309,7 +324,10 @@ class Stack:
         for name in PROJ:
             shared = name in ("k", "v", "up")
             per_block += (1 if shared else fq.launch_count("falqon_melded_forward"))   # codes: the product alone
-            per_block += fq.launch_count("falqon_melded_backward") + (1 if self.producer_amax else 0)   # + the O_A cast
+            if name in ("k", "v"):
+                per_block += 3                                  # on q's gradient codes: O_A cast, dB, dX
+            else:
+                per_block += fq.launch_count("falqon_melded_backward") + (1 if self.producer_amax else 0)   # + the O_A cast
             if self.batches is None:
                 per_block += fq.launch_count("falqon_proxy_update", k=self.k)
         if self.batches is not None:

@@ -395,3 +395,33 @@ def test_adamw_proxy_update_bit_exact(fq, orc):
         assert np.array_equal(bits32(f32(layer.dbuf)), bits32(dbuf_o)), step
         assert np.array_equal(u8(layer.wq), wq_o), step
     assert fq.last_device_status() == 0
+
+
+def test_backward_on_shared_gradient_codes(fq, orc):
+    """falqon_melded_backward_codes: a second layer of the same output width multiplies the gradient codes the first one
+    cast -- bit for bit what its own falqon_melded_backward gives; per-row layers are refused."""
+    m, n1, n2, r, T = 768, 512, 1024, 32, 700
+    W1, A1, B1, X1 = layer_inputs(81, 0, m, n1, r, T, 3, DEV)
+    W2, A2, B2, X2 = layer_inputs(81, 1, m, n2, r, T, 3, DEV)
+    dY = synth.out_grad(81, 0, 0, T, m, DEV)
+    L1, L2 = fq.setup_layer(W1, A1, B1, 1.0), fq.setup_layer(W2, A2, B2, 1.0)
+    ws1, ws2 = L1.workspace(T), L2.workspace(T)
+    _, OA1, am1, _ = fq.melded_forward(L1, X1, ws=ws1)
+    _, OA2, am2, _ = fq.melded_forward(L2, X2, ws=ws2)
+    dX_ref, dB_ref, _ = fq.melded_backward(L2, dY, OA2, am2, dx_dtype=torch.float32, ws=ws2)
+    dX_ref, dB_ref = dX_ref.clone(), dB_ref.clone()
+    fq.ws_view(L2, ws2, T, fq.WS_GQ).fill_(0)          # L2's own codes are gone: the shared call must not need them
+    fq.melded_backward(L1, dY, OA1, am1, ws=ws1)
+    gq = fq.ws_view(L1, ws1, T, fq.WS_GQ)[: T * m].view(T, m)
+    s_g = fq.ws_view(L1, ws1, T, fq.WS_SCALES).view(torch.float32)[3:4]
+    dX, dB = fq.melded_backward_codes(L2, gq, s_g, OA2, am2, dx_dtype=torch.float32, ws=ws2)
+    assert torch.equal(dX.view(torch.int32), dX_ref.view(torch.int32)) and torch.equal(dB.view(torch.int32), dB_ref.view(torch.int32))
+    _, dB_only = fq.melded_backward_codes(L2, gq, s_g, OA2, am2, need_dx=False, ws=ws2)
+    assert torch.equal(dB_only.view(torch.int32), dB_ref.view(torch.int32))
+    gq_o, s_g_o, _ = orc.quantize(f32(dY), orc.E5M2)
+    assert np.array_equal(u8(gq), gq_o) and bits32(f32(s_g))[0] == bits32(s_g_o)
+    Lr = fq.setup_layer(W2, A2, B2, 1.0, per_row=True)
+    with pytest.raises(fq.FalqonError) as e:
+        fq.melded_backward_codes(Lr, gq, s_g, OA2, am2, ws=Lr.workspace(T))
+    assert e.value.status == fq.ERR_UNSUPPORTED
+    assert fq.last_device_status() == 0
