@@ -169,3 +169,38 @@ def test_fused_forward_emits_shared_codes(fq, orc):
     Y2, OA2, amax2 = fq.melded_forward_codes(plain, xq, sx1, y_dtype=torch.float32, ws=ws)
     assert torch.equal(Y1, Y2) and torch.equal(OA1, OA2) and torch.equal(amax1, amax2)
     assert fq.last_device_status() == 0
+
+
+@pytest.mark.parametrize("amax", [448.0, 448.0 / 3.7, 57344.0, 1.0e-3])
+def test_fused_converters_on_every_bf16_value(fq, orc, amax):
+    """The converters' cast (packed multiply, cvt.rn.satfinite, in-place swizzled store) on ALL finite bf16 inputs: a
+    [512][128] activation tensor that holds every bit pattern once, cast with a given absmax (scale 1, an odd scale, a tiny
+    one that underflows most values, a huge one that saturates many), dumped and compared with the oracle's cast; the same
+    values as an output gradient through the input-gradient product's E5M2 converters."""
+    bits = torch.arange(1 << 16, dtype=torch.int32).to(torch.int16).view(torch.bfloat16).reshape(512, 128)
+    X = torch.where(torch.isfinite(bits.float()), bits, torch.zeros_like(bits)).to(DEV)
+    T, n, m, r = 512, 128, 240, 16
+    W, A, B, _ = layer_inputs(14, 0, m, n, r, 16, 0, DEV)
+    layer = fq.setup_layer(W, A, B, 1.0)
+    layer.flags = fq.LAYER_FUSED_CAST
+    ws = layer.workspace(T)
+    am = torch.tensor([amax], dtype=torch.float32, device=DEV)
+    s = np.float32(448.0) / np.float32(amax)
+    fq.ws_view(layer, ws, T, fq.WS_XQ).fill_(0xAA)
+    _, _, _, s_x = fq.melded_forward_dump(layer, X, 0, ws=ws, amax_x=am)
+    assert bits32(f32(s_x))[0] == bits32(s)
+    want, _, _ = orc.quantize(f32(X), orc.E4M3, scale_in=s)
+    assert np.array_equal(u8(fq.ws_view(layer, ws, T, fq.WS_XQ)).reshape(T, n), want)
+    # E5M2: the same patterns as dY of a layer with m = 128 outputs
+    m2, n2 = 128, 256
+    W2, A2, B2, X2 = layer_inputs(14, 1, m2, n2, r, T, 2, DEV)
+    back = fq.setup_layer(W2, A2, B2, 1.0)
+    back.flags = fq.LAYER_FUSED_CAST
+    ws2 = back.workspace(T)
+    _, OA, amax_oa, _ = fq.melded_forward(back, X2, ws=ws2)
+    s5 = np.float32(57344.0) / np.float32(amax)
+    fq.ws_view(back, ws2, T, fq.WS_GQ).fill_(0xAA)
+    fq.melded_backward_dump(back, X, OA, amax_oa, 0, ws=ws2, amax_dy=am)
+    want5, _, _ = orc.quantize(f32(X), orc.E5M2, scale_in=s5)
+    assert np.array_equal(u8(fq.ws_view(back, ws2, T, fq.WS_GQ)).reshape(T, m2), want5)
+    assert fq.last_device_status() == 0
