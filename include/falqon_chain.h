@@ -50,6 +50,47 @@ int falqon_chain_rmsnorm_grad_combine(void *out, const void *dy_a, const void *d
                                       const float *inv_rms, const void *res, float s_res, int64_t rows, int64_t cols,
                                       float *amax_out, falqon_stream stream);
 
+/* ---- Quantizing forms: the chain operation AND the per-tensor cast of its result (Eq. quantize: s = fp8max / absmax,
+ * saturating round to nearest even) in one launch, so that the tensor a melded layer consumes never takes a separate
+ * quantize pass: the codes go straight to falqon_melded_forward_codes / falqon_melded_backward_codes.  Bit for bit:
+ * codes and *scale_out are those of falqon_quantize applied to the bf16 tensor the plain call would have stored.
+ *   codes      device [count] bytes, 16-byte aligned (count = rows * cols for the row-wise calls)
+ *   scale_out  device [1] fp32
+ *   fmt        FALQON_E4M3 (a forward input) or FALQON_E5M2 (an output gradient)
+ *   out16      device [count] bf16, 16-byte aligned.  keep16 != 0: receives the bf16 result as the plain call stores it.
+ *              keep16 == 0: working space -- the part of the tensor that does not fit in the SMs' shared memory between
+ *              the two phases of the kernel passes through it; its contents afterwards are unspecified.
+ *   scratch    FALQON_CHAIN_SCRATCH_BYTES device bytes, 16-byte aligned, zero before the first call and left zero by every
+ *              call; calls that may run at the same time need scratch of their own.
+ * The kernel holds a grid-wide barrier (the absmax of the whole tensor precedes the first code), so the launch is
+ * cooperative with one CTA per SM; the barrier's wait is bounded and a wait that runs out is reported by
+ * falqon_last_device_status (the codes are then incomplete). */
+#define FALQON_CHAIN_SCRATCH_BYTES 4096
+
+int falqon_chain_combine_quantize(void *codes, float *scale_out, int fmt, void *out16, int keep16, const void *a, float sa,
+                                  const void *b, float sb, const void *c, float sc, const void *d, float sd, int64_t count,
+                                  void *scratch, falqon_stream stream);
+
+int falqon_chain_silu_mul_quantize(void *codes, float *scale_out, int fmt, void *out16, int keep16, const void *g, const void *u,
+                                   int64_t count, void *scratch, falqon_stream stream);
+
+/* Two results, each with its own codes, scale and bf16 buffer (index 0 of the scratch's partial maxima serves dg, 1 du). */
+int falqon_chain_silu_mul_grad_quantize(void *codes_dg, void *codes_du, float *scale_dg, float *scale_du, int fmt, void *dg16,
+                                        void *du16, int keep16, const void *g, const void *u, const void *dz, int64_t count,
+                                        void *scratch, falqon_stream stream);
+
+/* y = rmsnorm(x) with x = a (b == NULL and sum_out == NULL; sa, sb ignored) or x = bf16(sa*a + sb*b), which is stored to
+ * sum_out (falqon_chain_combine_rmsnorm).  inv_rms as in falqon_chain_rmsnorm; y16 plays the part of out16. */
+int falqon_chain_rmsnorm_quantize(void *codes, float *scale_out, int fmt, void *y16, int keep16, float *inv_rms, void *sum_out,
+                                  const void *a, float sa, const void *b, float sb, int64_t rows, int64_t cols, float eps,
+                                  void *scratch, falqon_stream stream);
+
+/* falqon_chain_rmsnorm_grad_combine whose result is stored to out (always: the chain needs it again) and cast. */
+int falqon_chain_rmsnorm_grad_combine_quantize(void *codes, float *scale_out, int fmt, void *out, const void *dy_a,
+                                               const void *dy_b, const void *dy_c, const void *x, const float *inv_rms,
+                                               const void *res, float s_res, int64_t rows, int64_t cols, void *scratch,
+                                               falqon_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -9,8 +9,8 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfalqon.so")
-SOURCES = ["api.cu", "quantize.cu", "gemm_fp8.cu", "gemm_fp8_fused.cu", "gemm_db.cu", "update_a.cu", "proxy_update.cu", "proxy_update_static.cu", "chain_ops.cu", "merge_exact.cu", "svd_init.cu", "tensor_ceiling.cu"]
-HEADERS = ["internal.h", "ptx.cuh", "gemm_common.cuh", "convert_tile.cuh", os.path.join("..", "..", "include", "falqon.h"),
+SOURCES = ["api.cu", "quantize.cu", "gemm_fp8.cu", "gemm_fp8_fused.cu", "gemm_db.cu", "update_a.cu", "proxy_update.cu", "proxy_update_static.cu", "chain_ops.cu", "chain_quant.cu", "merge_exact.cu", "svd_init.cu", "tensor_ceiling.cu"]
+HEADERS = ["internal.h", "ptx.cuh", "gemm_common.cuh", "convert_tile.cuh", "chain_math.cuh", "grid_sync.cuh", os.path.join("..", "..", "include", "falqon.h"),
            os.path.join("..", "..", "include", "falqon_chain.h")]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v", "-Xptxas", "-dlcm=cg"]

@@ -1,6 +1,7 @@
 // Element-wise bf16 kernels of the stand-in decoder chain (see include/falqon_chain.h): harness code for the
 // 32-layer stack benchmark, HBM-bound, 16-byte loads and stores, eight elements per thread and iteration.
 #include "../../include/falqon_chain.h"
+#include "chain_math.cuh"
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -9,30 +10,6 @@ namespace {
 
 constexpr int kChainThreads = 256;
 
-__device__ __forceinline__ void unpack8(const uint4& q, float (&x)[8]) {
-  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    x[2 * i] = __uint_as_float(w[i] << 16);
-    x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-  }
-}
-__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-  uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
-__device__ __forceinline__ uint4 pack8(const float (&x)[8]) {
-  return make_uint4(pack2(x[0], x[1]), pack2(x[2], x[3]), pack2(x[4], x[5]), pack2(x[6], x[7]));
-}
-
-// Largest |bf16| bit pattern (15 bits) among the two halves of each word.
-__device__ __forceinline__ uint32_t max_abs_bf16(const uint4& q, uint32_t m) {
-  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) m = max(m, max(w[i] & 0x7FFFu, (w[i] >> 16) & 0x7FFFu));
-  return m;
-}
 // Raises *amax (the fp32 bit pattern of a non-negative value) to the CTA's largest |bf16| with one atomic per CTA.
 __device__ __forceinline__ void publish_amax(uint32_t m, float* amax) {
   __shared__ uint32_t s_max;
@@ -50,34 +27,16 @@ __global__ void __launch_bounds__(kChainThreads) combine_kernel(uint4* out, cons
   pdl_trigger();
   pdl_wait();
   uint32_t mx = 0;
+  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
   for (int64_t v = blockIdx.x * (int64_t)kChainThreads + threadIdx.x; v < nvec; v += (int64_t)gridDim.x * kChainThreads) {
-    float x[8], y[8], acc[8];
-    unpack8(ld_stream(a + v), x);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) acc[i] = __fmul_rn(sa, x[i]);
-    if (b != nullptr) {
-      unpack8(ld_stream(b + v), y);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) acc[i] = __fmaf_rn(sb, y[i], acc[i]);
-    }
-    if (c != nullptr) {
-      unpack8(ld_stream(c + v), y);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) acc[i] = __fmaf_rn(sc, y[i], acc[i]);
-    }
-    if (d != nullptr) {
-      unpack8(ld_stream(d + v), y);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) acc[i] = __fmaf_rn(sd, y[i], acc[i]);
-    }
-    const uint4 o = pack8(acc);
+    const uint4 o = combine8(ld_stream(a + v), sa, b != nullptr ? ld_stream(b + v) : zero, sb, b != nullptr,
+                             c != nullptr ? ld_stream(c + v) : zero, sc, c != nullptr, d != nullptr ? ld_stream(d + v) : zero, sd,
+                             d != nullptr);
     out[v] = o;
     mx = max_abs_bf16(o, mx);
   }
   if (amax != nullptr) publish_amax(mx, amax);
 }
-
-__device__ __forceinline__ float sigmoidf(float x) { return 1.0f / (1.0f + expf(-x)); }
 
 __global__ void __launch_bounds__(kChainThreads) silu_mul_kernel(uint4* z, const uint4* g, const uint4* u, int64_t nvec,
                                                                  float* amax) {
@@ -85,12 +44,7 @@ __global__ void __launch_bounds__(kChainThreads) silu_mul_kernel(uint4* z, const
   pdl_wait();
   uint32_t mx = 0;
   for (int64_t v = blockIdx.x * (int64_t)kChainThreads + threadIdx.x; v < nvec; v += (int64_t)gridDim.x * kChainThreads) {
-    float x[8], y[8], o[8];
-    unpack8(ld_stream(g + v), x);
-    unpack8(ld_stream(u + v), y);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) o[i] = x[i] * sigmoidf(x[i]) * y[i];
-    const uint4 q = pack8(o);
+    const uint4 q = silu_mul8(ld_stream(g + v), ld_stream(u + v));
     z[v] = q;
     mx = max_abs_bf16(q, mx);
   }
@@ -104,17 +58,8 @@ __global__ void __launch_bounds__(kChainThreads) silu_mul_grad_kernel(uint4* dg,
   pdl_wait();
   uint32_t mg = 0, mu = 0;
   for (int64_t v = blockIdx.x * (int64_t)kChainThreads + threadIdx.x; v < nvec; v += (int64_t)gridDim.x * kChainThreads) {
-    float x[8], y[8], t[8], og[8], ou[8];
-    unpack8(ld_stream(g + v), x);
-    unpack8(ld_stream(u + v), y);
-    unpack8(ld_stream(dz + v), t);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float s = sigmoidf(x[i]);
-      ou[i] = t[i] * x[i] * s;
-      og[i] = t[i] * y[i] * s * (1.0f + x[i] * (1.0f - s));
-    }
-    const uint4 qg = pack8(og), qu = pack8(ou);
+    uint4 qg, qu;
+    silu_mul_grad8(ld_stream(g + v), ld_stream(u + v), ld_stream(dz + v), qg, qu);
     dg[v] = qg;
     du[v] = qu;
     mg = max_abs_bf16(qg, mg);
@@ -124,57 +69,21 @@ __global__ void __launch_bounds__(kChainThreads) silu_mul_grad_kernel(uint4* dg,
   if (amax_du != nullptr) publish_amax(mu, amax_du);
 }
 
-// One CTA of 128 threads per row; a thread keeps its elements (up to 16 vectors of 8) in registers between the
-// reduction and the scaling.
-constexpr int kNormThreads = 128;
-constexpr int kNormMaxVec = 16;   // cols <= 128 * 16 * 8 = 16384
-
-__device__ __forceinline__ float block_sum_128(float v, float* red /* [4] */) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
-  __syncthreads();
-  const float total = (red[0] + red[1]) + (red[2] + red[3]);
-  __syncthreads();
-  return total;
-}
-
+// The row-wise kernels: one CTA of 128 threads per row (the row arithmetic is in chain_math.cuh).
 __global__ void __launch_bounds__(kNormThreads) rmsnorm_kernel(uint4* y, float* inv_rms, const uint4* x, int vec_per_row,
                                                                float inv_cols, float eps, float* amax) {
   __shared__ float red[4];
   pdl_trigger();
   pdl_wait();
-  const uint4* xr = x + static_cast<int64_t>(blockIdx.x) * vec_per_row;
-  uint4* yr = y + static_cast<int64_t>(blockIdx.x) * vec_per_row;
-  uint4 raw[kNormMaxVec];
-  float ss = 0.0f;
-#pragma unroll
-  for (int i = 0; i < kNormMaxVec; ++i) {
-    const int v = threadIdx.x + i * kNormThreads;
-    if (v < vec_per_row) {
-      raw[i] = ld_stream(xr + v);
-      float f[8];
-      unpack8(raw[i], f);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) ss = __fmaf_rn(f[e], f[e], ss);
-    }
-  }
-  const float inv = rsqrtf(block_sum_128(ss, red) * inv_cols + eps);
-  if (threadIdx.x == 0) inv_rms[blockIdx.x] = inv;
+  const int64_t base = static_cast<int64_t>(blockIdx.x) * vec_per_row;
+  const RowGroup grp{static_cast<int>(threadIdx.x), 0, red};
   uint32_t mx = 0;
-#pragma unroll
-  for (int i = 0; i < kNormMaxVec; ++i) {
-    const int v = threadIdx.x + i * kNormThreads;
-    if (v < vec_per_row) {
-      float f[8];
-      unpack8(raw[i], f);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) f[e] *= inv;
-      const uint4 o = pack8(f);
-      yr[v] = o;
-      mx = max_abs_bf16(o, mx);
-    }
-  }
+  const float inv = rmsnorm_row<kNormMaxVec, false>(x + base, 0.0f, nullptr, 0.0f, vec_per_row, inv_cols, eps, grp, [](int, const uint4&) {},
+                                       [&](int v, const uint4& o) {
+                                         y[base + v] = o;
+                                         mx = max_abs_bf16(o, mx);
+                                       });
+  if (threadIdx.x == 0) inv_rms[blockIdx.x] = inv;
   if (amax != nullptr) publish_amax(mx, amax);
 }
 
@@ -184,35 +93,9 @@ __global__ void __launch_bounds__(kNormThreads) rmsnorm_grad_kernel(uint4* dx, c
   pdl_trigger();
   pdl_wait();
   const int64_t base = static_cast<int64_t>(blockIdx.x) * vec_per_row;
-  const float inv = ld_stream(inv_rms + blockIdx.x);
-  uint4 rx[kNormMaxVec], rdy[kNormMaxVec];
-  float dot = 0.0f;
-#pragma unroll
-  for (int i = 0; i < kNormMaxVec; ++i) {
-    const int v = threadIdx.x + i * kNormThreads;
-    if (v < vec_per_row) {
-      rx[i] = ld_stream(x + base + v);
-      rdy[i] = ld_stream(dy + base + v);
-      float fx[8], fd[8];
-      unpack8(rx[i], fx);
-      unpack8(rdy[i], fd);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) dot = __fmaf_rn(fd[e], fx[e] * inv, dot);
-    }
-  }
-  const float mean = block_sum_128(dot, red) * inv_cols;
-#pragma unroll
-  for (int i = 0; i < kNormMaxVec; ++i) {
-    const int v = threadIdx.x + i * kNormThreads;
-    if (v < vec_per_row) {
-      float fx[8], fd[8], o[8];
-      unpack8(rx[i], fx);
-      unpack8(rdy[i], fd);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) o[e] = inv * (fd[e] - fx[e] * inv * mean);
-      dx[base + v] = pack8(o);
-    }
-  }
+  const RowGroup grp{static_cast<int>(threadIdx.x), 0, red};
+  rmsnorm_grad_row<kNormMaxVec, false>(dy + base, nullptr, nullptr, x + base, ld_stream(inv_rms + blockIdx.x), nullptr, 0.0f, vec_per_row,
+                          inv_cols, grp, [&](int v, const uint4& o) { dx[base + v] = o; });
 }
 
 // sum = bf16(sa * a + sb * b), stored, and the RMS normalisation of that stored (rounded) sum, in one pass over the row:
@@ -224,41 +107,15 @@ __global__ void __launch_bounds__(kNormThreads) combine_rmsnorm_kernel(uint4* su
   pdl_trigger();
   pdl_wait();
   const int64_t base = static_cast<int64_t>(blockIdx.x) * vec_per_row;
-  uint4 raw[kNormMaxVec];
-  float ss = 0.0f;
-#pragma unroll
-  for (int i = 0; i < kNormMaxVec; ++i) {
-    const int v = threadIdx.x + i * kNormThreads;
-    if (v < vec_per_row) {
-      float fa[8], fb[8], acc[8];
-      unpack8(ld_stream(a + base + v), fa);
-      unpack8(ld_stream(b + base + v), fb);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) acc[e] = __fmaf_rn(sb, fb[e], __fmul_rn(sa, fa[e]));
-      raw[i] = pack8(acc);
-      sum_out[base + v] = raw[i];
-      float f[8];
-      unpack8(raw[i], f);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) ss = __fmaf_rn(f[e], f[e], ss);
-    }
-  }
-  const float inv = rsqrtf(block_sum_128(ss, red) * inv_cols + eps);
-  if (threadIdx.x == 0) inv_rms[blockIdx.x] = inv;
+  const RowGroup grp{static_cast<int>(threadIdx.x), 0, red};
   uint32_t mx = 0;
-#pragma unroll
-  for (int i = 0; i < kNormMaxVec; ++i) {
-    const int v = threadIdx.x + i * kNormThreads;
-    if (v < vec_per_row) {
-      float f[8];
-      unpack8(raw[i], f);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) f[e] *= inv;
-      const uint4 o = pack8(f);
-      y[base + v] = o;
-      mx = max_abs_bf16(o, mx);
-    }
-  }
+  const float inv = rmsnorm_row<kNormMaxVec, true>(a + base, sa, b + base, sb, vec_per_row, inv_cols, eps, grp,
+                                      [&](int v, const uint4& s) { sum_out[base + v] = s; },
+                                      [&](int v, const uint4& o) {
+                                        y[base + v] = o;
+                                        mx = max_abs_bf16(o, mx);
+                                      });
+  if (threadIdx.x == 0) inv_rms[blockIdx.x] = inv;
   if (amax != nullptr) publish_amax(mx, amax);
 }
 
@@ -273,52 +130,14 @@ __global__ void __launch_bounds__(kNormThreads) rmsnorm_grad_combine_kernel(uint
   pdl_trigger();
   pdl_wait();
   const int64_t base = static_cast<int64_t>(blockIdx.x) * vec_per_row;
-  const float inv = ld_stream(inv_rms + blockIdx.x);
-  uint4 rx[kNormMaxVec], rdy[kNormMaxVec];
-  float dot = 0.0f;
-#pragma unroll
-  for (int i = 0; i < kNormMaxVec; ++i) {
-    const int v = threadIdx.x + i * kNormThreads;
-    if (v < vec_per_row) {
-      float fa[8], fb[8], acc[8];
-      rx[i] = ld_stream(x + base + v);
-      unpack8(ld_stream(dy_a + base + v), fa);
-      unpack8(ld_stream(dy_b + base + v), fb);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) acc[e] = __fmaf_rn(1.0f, fb[e], __fmul_rn(1.0f, fa[e]));
-      if (dy_c != nullptr) {
-        unpack8(ld_stream(dy_c + base + v), fb);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e] = __fmaf_rn(1.0f, fb[e], acc[e]);
-      }
-      rdy[i] = pack8(acc);
-      float fx[8], fd[8];
-      unpack8(rx[i], fx);
-      unpack8(rdy[i], fd);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) dot = __fmaf_rn(fd[e], fx[e] * inv, dot);
-    }
-  }
-  const float mean = block_sum_128(dot, red) * inv_cols;
+  const RowGroup grp{static_cast<int>(threadIdx.x), 0, red};
   uint32_t mx = 0;
-#pragma unroll
-  for (int i = 0; i < kNormMaxVec; ++i) {
-    const int v = threadIdx.x + i * kNormThreads;
-    if (v < vec_per_row) {
-      float fx[8], fd[8], o[8], fr[8], g[8];
-      unpack8(rx[i], fx);
-      unpack8(rdy[i], fd);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) o[e] = inv * (fd[e] - fx[e] * inv * mean);
-      unpack8(pack8(o), g);                       // the gradient as the separate kernel would have stored it
-      unpack8(ld_stream(res + base + v), fr);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) o[e] = __fmaf_rn(1.0f, g[e], __fmul_rn(s_res, fr[e]));
-      const uint4 q = pack8(o);
-      out[base + v] = q;
-      mx = max_abs_bf16(q, mx);
-    }
-  }
+  rmsnorm_grad_row<kNormMaxVec, true>(dy_a + base, dy_b + base, dy_c != nullptr ? dy_c + base : nullptr, x + base,
+                         ld_stream(inv_rms + blockIdx.x), res + base, s_res, vec_per_row, inv_cols, grp,
+                         [&](int v, const uint4& q) {
+                           out[base + v] = q;
+                           mx = max_abs_bf16(q, mx);
+                         });
   if (amax != nullptr) publish_amax(mx, amax);
 }
 

@@ -2,6 +2,7 @@
 // round-to-nearest-even cast to E4M3 / E5M2.  HBM-bound: 128-bit loads and stores, warp-shuffle
 // reductions, one partial maximum per CTA on the bit pattern of |x| (max is order-free, so the result
 // is bit-exact whatever the schedule; nothing has to be cleared between calls).
+#include "grid_sync.cuh"
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -182,19 +183,6 @@ __global__ void __launch_bounds__(kThreads) scale_prep_kernel(const uint32_t* pa
     if (out.amax_out) *out.amax_out = amax;
     if (out.clear_word) *out.clear_word = 0.0f;
   }
-}
-
-// The grid-wide barrier of the fused quantizer: two counters in the caller's workspace that start at zero and are
-// put back to zero by the last CTA to leave.
-struct GridSync {
-  unsigned int arrive;
-  unsigned int depart;
-};
-
-__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
-  unsigned int v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
 }
 
 // ---- fused per-tensor quantizer: absmax, a grid-wide barrier, then the cast, in ONE kernel, with the tensor held

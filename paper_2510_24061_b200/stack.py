@@ -41,8 +41,22 @@ lib.falqon_chain_combine_rmsnorm.restype = C.c_int
 lib.falqon_chain_combine_rmsnorm.argtypes = [_p, _p, _p, _p, _f, _p, _f, _i64, _i64, _f, _p, _p]
 lib.falqon_chain_rmsnorm_grad_combine.restype = C.c_int
 lib.falqon_chain_rmsnorm_grad_combine.argtypes = [_p, _p, _p, _p, _p, _p, _p, _f, _i64, _i64, _p, _p]
+_fp, _int = C.c_void_p, C.c_int
+lib.falqon_chain_combine_quantize.restype = C.c_int
+lib.falqon_chain_combine_quantize.argtypes = [_p, _fp, _int, _p, _int, _p, _f, _p, _f, _p, _f, _p, _f, _i64, _p, _p]
+lib.falqon_chain_silu_mul_quantize.restype = C.c_int
+lib.falqon_chain_silu_mul_quantize.argtypes = [_p, _fp, _int, _p, _int, _p, _p, _i64, _p, _p]
+lib.falqon_chain_silu_mul_grad_quantize.restype = C.c_int
+lib.falqon_chain_silu_mul_grad_quantize.argtypes = [_p, _p, _fp, _fp, _int, _p, _p, _int, _p, _p, _p, _i64, _p, _p]
+lib.falqon_chain_rmsnorm_quantize.restype = C.c_int
+lib.falqon_chain_rmsnorm_quantize.argtypes = [_p, _fp, _int, _p, _int, _p, _p, _p, _f, _p, _f, _i64, _i64, _f, _p, _p]
+lib.falqon_chain_rmsnorm_grad_combine_quantize.restype = C.c_int
+lib.falqon_chain_rmsnorm_grad_combine_quantize.argtypes = [_p, _fp, _int, _p, _p, _p, _p, _p, _p, _p, _f, _i64, _i64, _p, _p]
 CHAIN_EXPORTS = ["falqon_chain_combine", "falqon_chain_silu_mul", "falqon_chain_silu_mul_grad", "falqon_chain_rmsnorm",
-                 "falqon_chain_rmsnorm_grad", "falqon_chain_combine_rmsnorm", "falqon_chain_rmsnorm_grad_combine"]
+                 "falqon_chain_rmsnorm_grad", "falqon_chain_combine_rmsnorm", "falqon_chain_rmsnorm_grad_combine",
+                 "falqon_chain_combine_quantize", "falqon_chain_silu_mul_quantize", "falqon_chain_silu_mul_grad_quantize",
+                 "falqon_chain_rmsnorm_quantize", "falqon_chain_rmsnorm_grad_combine_quantize"]
+CHAIN_SCRATCH_BYTES = 4096
 NORM_EPS = 1e-6
 
 PROJ = ["q", "k", "v", "o", "gate", "up", "down"]
@@ -117,6 +131,73 @@ def rmsnorm_grad_combine(out, dys, x, inv_rms, res, s_res, amax=None):
                                                     _ptr(x), _ptr(inv_rms), _ptr(res), s_res, x.shape[0], x.shape[1], _ptr(amax),
                                                     fq._stream()))
     return out
+
+
+def chain_scratch(device):
+    """The zeroed scratch of the quantizing chain calls (one per stream that runs them)."""
+    return torch.zeros(CHAIN_SCRATCH_BYTES, dtype=torch.uint8, device=device)
+
+
+def _q_args(codes, scale, out16, count):
+    assert codes.dtype == torch.uint8 and codes.is_contiguous() and codes.numel() >= count
+    assert scale.dtype == torch.float32 and scale.numel() == 1
+    assert out16.dtype == torch.bfloat16 and out16.is_contiguous() and out16.numel() == count
+
+
+def combine_quantize(codes, scale, fmt, out16, keep16, scratch, a, sa=1.0, b=None, sb=1.0, c=None, sc=1.0, d=None, sd=1.0):
+    """combine(...) and the per-tensor cast of its result in one launch: codes (uint8) and scale (fp32 [1]) as quantize gives
+    them for the bf16 result; out16 receives that result only if keep16 (otherwise it is working space)."""
+    _q_args(codes, scale, out16, a.numel())
+    for t in (a, b, c, d):
+        assert t is None or (t.dtype == torch.bfloat16 and t.is_contiguous() and t.numel() == a.numel())
+    fq._check("falqon_chain_combine_quantize",
+              lib.falqon_chain_combine_quantize(_ptr(codes), _ptr(scale), fmt, _ptr(out16), int(keep16), _ptr(a), sa, _ptr(b), sb,
+                                                _ptr(c), sc, _ptr(d), sd, a.numel(), _ptr(scratch), fq._stream()))
+
+
+def silu_mul_quantize(codes, scale, fmt, out16, keep16, scratch, g, u):
+    _q_args(codes, scale, out16, g.numel())
+    for t in (g, u):
+        assert t.dtype == torch.bfloat16 and t.is_contiguous() and t.numel() == g.numel()
+    fq._check("falqon_chain_silu_mul_quantize",
+              lib.falqon_chain_silu_mul_quantize(_ptr(codes), _ptr(scale), fmt, _ptr(out16), int(keep16), _ptr(g), _ptr(u), g.numel(),
+                                                 _ptr(scratch), fq._stream()))
+
+
+def silu_mul_grad_quantize(codes_dg, codes_du, scale_dg, scale_du, fmt, dg16, du16, keep16, scratch, g, u, dz):
+    _q_args(codes_dg, scale_dg, dg16, g.numel())
+    _q_args(codes_du, scale_du, du16, g.numel())
+    for t in (g, u, dz):
+        assert t.dtype == torch.bfloat16 and t.is_contiguous() and t.numel() == g.numel()
+    fq._check("falqon_chain_silu_mul_grad_quantize",
+              lib.falqon_chain_silu_mul_grad_quantize(_ptr(codes_dg), _ptr(codes_du), _ptr(scale_dg), _ptr(scale_du), fmt, _ptr(dg16),
+                                                      _ptr(du16), int(keep16), _ptr(g), _ptr(u), _ptr(dz), g.numel(), _ptr(scratch),
+                                                      fq._stream()))
+
+
+def rmsnorm_quantize(codes, scale, fmt, y16, keep16, scratch, inv_rms, a, sum_out=None, sa=1.0, b=None, sb=1.0):
+    """rmsnorm(a), or combine_rmsnorm(sum_out, ., a, sa, b, sb) when b and sum_out are given, with the cast of the result."""
+    _q_args(codes, scale, y16, a.numel())
+    assert a.dtype == torch.bfloat16 and a.dim() == 2 and a.is_contiguous()
+    assert inv_rms.dtype == torch.float32 and inv_rms.numel() == a.shape[0]
+    for t in (b, sum_out):
+        assert t is None or (t.dtype == torch.bfloat16 and t.is_contiguous() and t.shape == a.shape)
+    fq._check("falqon_chain_rmsnorm_quantize",
+              lib.falqon_chain_rmsnorm_quantize(_ptr(codes), _ptr(scale), fmt, _ptr(y16), int(keep16), _ptr(inv_rms), _ptr(sum_out),
+                                                _ptr(a), sa, _ptr(b), sb, a.shape[0], a.shape[1], NORM_EPS, _ptr(scratch),
+                                                fq._stream()))
+
+
+def rmsnorm_grad_combine_quantize(codes, scale, fmt, out, scratch, dys, x, inv_rms, res, s_res):
+    """rmsnorm_grad_combine(out, ...) with the cast of out in the same launch."""
+    assert len(dys) in (2, 3)
+    _q_args(codes, scale, out, x.numel())
+    for t in (x, res, *dys):
+        assert t.dtype == torch.bfloat16 and t.is_contiguous() and t.shape == x.shape
+    fq._check("falqon_chain_rmsnorm_grad_combine_quantize",
+              lib.falqon_chain_rmsnorm_grad_combine_quantize(_ptr(codes), _ptr(scale), fmt, _ptr(out), _ptr(dys[0]), _ptr(dys[1]),
+                                                             _ptr(dys[2]) if len(dys) == 3 else None, _ptr(x), _ptr(inv_rms),
+                                                             _ptr(res), s_res, x.shape[0], x.shape[1], _ptr(scratch), fq._stream()))
 
 
 class Stack:
