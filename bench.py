@@ -429,6 +429,7 @@ def run_stack(args):
     peaks = measured_peaks()
     stack = st.Stack(n_layers, H, F, T, r, k, seed=cfg["seed"], device=dev, lr=lr, producer_amax=not args.stack_own_absmax,
                      batched_proxy=not args.proxy_per_layer, fuse_chain=not args.stack_unfused_chain,
+                     fuse_cast=not (args.stack_separate_casts or args.stack_own_absmax or args.stack_unfused_chain),
                      adamw=dict(beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0) if args.stack_adamw else None)
     h0 = synth.normal_bf16(cfg["seed"], 9001, (T, H), 1.0, dev)
     G = synth.normal_bf16(cfg["seed"], 9002, (T, H), 1.0e-2, dev)
@@ -506,6 +507,8 @@ def run_stack(args):
                    "l2": "working set far larger than L2 (every step touches the whole stack)", "parallelism": "single GPU",
                    "optimizer": "AdamW on the DeltaBuffers" if args.stack_adamw else "SGD on the DeltaBuffers",
                    "proxy_update": "one call per projection" if args.proxy_per_layer else "one batched call per block",
+                   "casts": ("inside the chain kernels that produce the tensors (two phases around a grid barrier)"
+                             if stack.fuse_cast else "single-pass kernels of their own (the producing kernel hands over the absmax)"),
                    "launch": "replays of one CUDA graph of the step" if use_graph else "one library call after another"},
         "clocks": clocks, "gpu_launches": stack.launches_per_step() * steps,
         "regime": "sustained: %.1f s of the same step loop ran right before the timed steps" % args.soak,
@@ -549,6 +552,9 @@ def main():
                     help="with --stack: every layer takes the absmax of its input itself (the chain kernels do not hand it over)")
     ap.add_argument("--stack-unfused-chain", action="store_true",
                     help="with --stack: residual sums and the normalisations (or their gradients) that follow them as separate kernels")
+    ap.add_argument("--stack-separate-casts", action="store_true",
+                    help="with --stack: every cast is a kernel of its own (default: the casts run inside the chain kernels that "
+                         "produce the tensors, all but those of the gated MLP's two gradients)")
     ap.add_argument("--stack-adamw", action="store_true",
                     help="with --stack: AdamW (beta 0.9 / 0.999, eps 1e-8, no weight decay) on every DeltaBuffer instead of plain SGD")
     ap.add_argument("--config3", action="store_true",

@@ -69,7 +69,9 @@ __global__ void __launch_bounds__(kChainThreads) silu_mul_grad_kernel(uint4* dg,
   if (amax_du != nullptr) publish_amax(mu, amax_du);
 }
 
-// The row-wise kernels: one CTA of 128 threads per row (the row arithmetic is in chain_math.cuh).
+// The row-wise kernels: one CTA of 128 threads per row (the row arithmetic is in chain_math.cuh).  kMaxVec: vectors a thread
+// holds; rows of up to 4096 values take the 4-vector form (a third of the registers, twice the resident warps).
+template <int kMaxVec>
 __global__ void __launch_bounds__(kNormThreads) rmsnorm_kernel(uint4* y, float* inv_rms, const uint4* x, int vec_per_row,
                                                                float inv_cols, float eps, float* amax) {
   __shared__ float red[4];
@@ -78,7 +80,7 @@ __global__ void __launch_bounds__(kNormThreads) rmsnorm_kernel(uint4* y, float* 
   const int64_t base = static_cast<int64_t>(blockIdx.x) * vec_per_row;
   const RowGroup grp{static_cast<int>(threadIdx.x), 0, red};
   uint32_t mx = 0;
-  const float inv = rmsnorm_row<kNormMaxVec, false>(x + base, 0.0f, nullptr, 0.0f, vec_per_row, inv_cols, eps, grp, [](int, const uint4&) {},
+  const float inv = rmsnorm_row<kMaxVec, false>(x + base, 0.0f, nullptr, 0.0f, vec_per_row, inv_cols, eps, grp, [](int, const uint4&) {},
                                        [&](int v, const uint4& o) {
                                          y[base + v] = o;
                                          mx = max_abs_bf16(o, mx);
@@ -87,6 +89,7 @@ __global__ void __launch_bounds__(kNormThreads) rmsnorm_kernel(uint4* y, float* 
   if (amax != nullptr) publish_amax(mx, amax);
 }
 
+template <int kMaxVec>
 __global__ void __launch_bounds__(kNormThreads) rmsnorm_grad_kernel(uint4* dx, const uint4* dy, const uint4* x,
                                                                     const float* inv_rms, int vec_per_row, float inv_cols) {
   __shared__ float red[4];
@@ -94,12 +97,13 @@ __global__ void __launch_bounds__(kNormThreads) rmsnorm_grad_kernel(uint4* dx, c
   pdl_wait();
   const int64_t base = static_cast<int64_t>(blockIdx.x) * vec_per_row;
   const RowGroup grp{static_cast<int>(threadIdx.x), 0, red};
-  rmsnorm_grad_row<kNormMaxVec, false>(dy + base, nullptr, nullptr, x + base, ld_stream(inv_rms + blockIdx.x), nullptr, 0.0f, vec_per_row,
+  rmsnorm_grad_row<kMaxVec, false>(dy + base, nullptr, nullptr, x + base, ld_stream(inv_rms + blockIdx.x), nullptr, 0.0f, vec_per_row,
                           inv_cols, grp, [&](int v, const uint4& o) { dx[base + v] = o; });
 }
 
 // sum = bf16(sa * a + sb * b), stored, and the RMS normalisation of that stored (rounded) sum, in one pass over the row:
 // the results are bit for bit those of combine_kernel followed by rmsnorm_kernel, without writing the sum and reading it back.
+template <int kMaxVec>
 __global__ void __launch_bounds__(kNormThreads) combine_rmsnorm_kernel(uint4* sum_out, uint4* y, float* inv_rms, const uint4* a,
                                                                        float sa, const uint4* b, float sb, int vec_per_row,
                                                                        float inv_cols, float eps, float* amax) {
@@ -109,7 +113,7 @@ __global__ void __launch_bounds__(kNormThreads) combine_rmsnorm_kernel(uint4* su
   const int64_t base = static_cast<int64_t>(blockIdx.x) * vec_per_row;
   const RowGroup grp{static_cast<int>(threadIdx.x), 0, red};
   uint32_t mx = 0;
-  const float inv = rmsnorm_row<kNormMaxVec, true>(a + base, sa, b + base, sb, vec_per_row, inv_cols, eps, grp,
+  const float inv = rmsnorm_row<kMaxVec, true>(a + base, sa, b + base, sb, vec_per_row, inv_cols, eps, grp,
                                       [&](int v, const uint4& s) { sum_out[base + v] = s; },
                                       [&](int v, const uint4& o) {
                                         y[base + v] = o;
@@ -122,6 +126,7 @@ __global__ void __launch_bounds__(kNormThreads) combine_rmsnorm_kernel(uint4* su
 // out = bf16(s_res * res + g) with g = rmsnorm_grad(dy, x, inv_rms) and dy = bf16(dy_a + dy_b (+ dy_c)), in one pass over
 // the row: bit for bit combine_kernel, rmsnorm_grad_kernel, combine_kernel in a row (the two intermediates are rounded to
 // bf16 in registers exactly as they would be in memory).
+template <int kMaxVec>
 __global__ void __launch_bounds__(kNormThreads) rmsnorm_grad_combine_kernel(uint4* out, const uint4* dy_a, const uint4* dy_b,
                                                                             const uint4* dy_c, const uint4* x,
                                                                             const float* inv_rms, const uint4* res, float s_res,
@@ -132,7 +137,7 @@ __global__ void __launch_bounds__(kNormThreads) rmsnorm_grad_combine_kernel(uint
   const int64_t base = static_cast<int64_t>(blockIdx.x) * vec_per_row;
   const RowGroup grp{static_cast<int>(threadIdx.x), 0, red};
   uint32_t mx = 0;
-  rmsnorm_grad_row<kNormMaxVec, true>(dy_a + base, dy_b + base, dy_c != nullptr ? dy_c + base : nullptr, x + base,
+  rmsnorm_grad_row<kMaxVec, true>(dy_a + base, dy_b + base, dy_c != nullptr ? dy_c + base : nullptr, x + base,
                          ld_stream(inv_rms + blockIdx.x), res + base, s_res, vec_per_row, inv_cols, grp,
                          [&](int v, const uint4& q) {
                            out[base + v] = q;
@@ -194,7 +199,11 @@ int falqon_chain_rmsnorm(void* y, float* inv_rms, const void* x, int64_t rows, i
   if (y == nullptr || inv_rms == nullptr || x == nullptr || rows < 1 || rows > (1ll << 30) || cols < 8 || cols % 8 ||
       cols > kNormThreads * kNormMaxVec * 8 || !ok16(y) || !ok16(x) || !(eps >= 0.0f))
     return FALQON_ERR_INVALID_ARG;
-  cudaError_t e = launch_pdl(rmsnorm_kernel, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
+  const bool narrow = cols <= 4 * kNormThreads * 8;
+  cudaError_t e = narrow ? launch_pdl(rmsnorm_kernel<4>, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
+                             static_cast<cudaStream_t>(stream), 1, static_cast<uint4*>(y), inv_rms, static_cast<const uint4*>(x),
+                             static_cast<int>(cols / 8), 1.0f / static_cast<float>(cols), eps, amax_out)
+                         : launch_pdl(rmsnorm_kernel<kNormMaxVec>, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
                              static_cast<cudaStream_t>(stream), 1, static_cast<uint4*>(y), inv_rms, static_cast<const uint4*>(x),
                              static_cast<int>(cols / 8), 1.0f / static_cast<float>(cols), eps, amax_out);
   return e == cudaSuccess ? FALQON_OK : FALQON_ERR_CUDA;
@@ -205,7 +214,11 @@ int falqon_chain_rmsnorm_grad(void* dx, const void* dy, const void* x, const flo
   if (dx == nullptr || dy == nullptr || x == nullptr || inv_rms == nullptr || rows < 1 || rows > (1ll << 30) || cols < 8 ||
       cols % 8 || cols > kNormThreads * kNormMaxVec * 8 || !ok16(dx) || !ok16(dy) || !ok16(x))
     return FALQON_ERR_INVALID_ARG;
-  cudaError_t e = launch_pdl(rmsnorm_grad_kernel, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
+  const bool narrow = cols <= 4 * kNormThreads * 8;
+  cudaError_t e = narrow ? launch_pdl(rmsnorm_grad_kernel<4>, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
+                             static_cast<cudaStream_t>(stream), 1, static_cast<uint4*>(dx), static_cast<const uint4*>(dy),
+                             static_cast<const uint4*>(x), inv_rms, static_cast<int>(cols / 8), 1.0f / static_cast<float>(cols))
+                         : launch_pdl(rmsnorm_grad_kernel<kNormMaxVec>, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
                              static_cast<cudaStream_t>(stream), 1, static_cast<uint4*>(dx), static_cast<const uint4*>(dy),
                              static_cast<const uint4*>(x), inv_rms, static_cast<int>(cols / 8), 1.0f / static_cast<float>(cols));
   return e == cudaSuccess ? FALQON_OK : FALQON_ERR_CUDA;
@@ -217,7 +230,12 @@ int falqon_chain_combine_rmsnorm(void* sum_out, void* y, float* inv_rms, const v
       cols < 8 || cols % 8 || cols > kNormThreads * kNormMaxVec * 8 || !ok16(sum_out) || !ok16(y) || !ok16(a) || !ok16(b) ||
       !(eps >= 0.0f))
     return FALQON_ERR_INVALID_ARG;
-  cudaError_t e = launch_pdl(combine_rmsnorm_kernel, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
+  const bool narrow = cols <= 4 * kNormThreads * 8;
+  cudaError_t e = narrow ? launch_pdl(combine_rmsnorm_kernel<4>, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
+                             static_cast<cudaStream_t>(stream), 1, static_cast<uint4*>(sum_out), static_cast<uint4*>(y), inv_rms,
+                             static_cast<const uint4*>(a), sa, static_cast<const uint4*>(b), sb, static_cast<int>(cols / 8),
+                             1.0f / static_cast<float>(cols), eps, amax_out)
+                         : launch_pdl(combine_rmsnorm_kernel<kNormMaxVec>, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
                              static_cast<cudaStream_t>(stream), 1, static_cast<uint4*>(sum_out), static_cast<uint4*>(y), inv_rms,
                              static_cast<const uint4*>(a), sa, static_cast<const uint4*>(b), sb, static_cast<int>(cols / 8),
                              1.0f / static_cast<float>(cols), eps, amax_out);
@@ -231,7 +249,13 @@ int falqon_chain_rmsnorm_grad_combine(void* out, const void* dy_a, const void* d
       rows > (1ll << 30) || cols < 8 || cols % 8 || cols > kNormThreads * kNormMaxVec * 8 || !ok16(out) || !ok16(dy_a) ||
       !ok16(dy_b) || !ok16(dy_c) || !ok16(x) || !ok16(res))
     return FALQON_ERR_INVALID_ARG;
-  cudaError_t e = launch_pdl(rmsnorm_grad_combine_kernel, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
+  const bool narrow = cols <= 4 * kNormThreads * 8;
+  cudaError_t e = narrow ? launch_pdl(rmsnorm_grad_combine_kernel<4>, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
+                             static_cast<cudaStream_t>(stream), 1, static_cast<uint4*>(out), static_cast<const uint4*>(dy_a),
+                             static_cast<const uint4*>(dy_b), static_cast<const uint4*>(dy_c), static_cast<const uint4*>(x), inv_rms,
+                             static_cast<const uint4*>(res), s_res, static_cast<int>(cols / 8), 1.0f / static_cast<float>(cols),
+                             amax_out)
+                         : launch_pdl(rmsnorm_grad_combine_kernel<kNormMaxVec>, dim3(static_cast<unsigned>(rows)), dim3(kNormThreads), 0,
                              static_cast<cudaStream_t>(stream), 1, static_cast<uint4*>(out), static_cast<const uint4*>(dy_a),
                              static_cast<const uint4*>(dy_b), static_cast<const uint4*>(dy_c), static_cast<const uint4*>(x), inv_rms,
                              static_cast<const uint4*>(res), s_res, static_cast<int>(cols / 8), 1.0f / static_cast<float>(cols),

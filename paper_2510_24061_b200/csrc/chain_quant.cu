@@ -20,7 +20,9 @@
 namespace falqon {
 namespace {
 
-constexpr int kCqThreads = 512;
+constexpr int kCqThreads = 512;      // row-wise producers on wide rows: four groups of 128 threads (the registers hold the row)
+constexpr int kCqWideThreads = 1024;  // element-wise producers and rows of up to 4096 values: more warps hide the arithmetic
+                                      // behind the loads
 constexpr int kCqStageBytes = 224 * 1024;
 constexpr int kCqStageVecs = kCqStageBytes / 16;   // 14336 vectors of eight bf16 = 28 rows of 4096
 constexpr int kCqMaxGrid = 256;                    // partial maxima per output in the scratch
@@ -41,12 +43,13 @@ struct CqTail {
   int keep16;
 };
 
+template <int kThreads>
 __device__ __forceinline__ uint32_t cta_max_u32(uint32_t v, uint32_t* red /* >= 32 words */) {
   v = __reduce_max_sync(0xFFFFFFFFu, v);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (lane == 0) red[warp] = v;
   __syncthreads();
-  uint32_t w = threadIdx.x < kCqThreads / 32 ? red[threadIdx.x] : 0u;
+  uint32_t w = threadIdx.x < kThreads / 32 ? red[threadIdx.x] : 0u;
   if (warp == 0) w = __reduce_max_sync(0xFFFFFFFFu, w);
   if (threadIdx.x == 0) red[0] = w;
   __syncthreads();
@@ -66,6 +69,7 @@ __device__ __forceinline__ void share_of(int64_t units, int64_t& first, int64_t&
 
 // ---- producers.  produce(put) computes the CTA's share; put(which, li, o) takes vector li (local index) of output `which`.
 struct CombineOp {
+  static constexpr int kThreads = kCqWideThreads;
   static constexpr int kOutputs = 1;
   const uint4 *a, *b, *c, *d;
   float sa, sb, sc, sd;
@@ -73,13 +77,13 @@ struct CombineOp {
   __device__ __forceinline__ void range(int64_t& first, int64_t& n) const { share_of(nvec, first, n); }
   template <class Put>
   __device__ __forceinline__ void produce(int64_t first, int64_t n, float (*)[4], Put put) const {
-    constexpr int kU = 4;
+    constexpr int kU = 2;
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-    for (int64_t li0 = threadIdx.x; li0 < n; li0 += kCqThreads * kU) {
+    for (int64_t li0 = threadIdx.x; li0 < n; li0 += kThreads * kU) {
       uint4 ra[kU], rb[kU], rc[kU], rd[kU];
 #pragma unroll
       for (int u = 0; u < kU; ++u) {
-        const int64_t li = li0 + u * kCqThreads;
+        const int64_t li = li0 + u * kThreads;
         ra[u] = rb[u] = rc[u] = rd[u] = zero;
         if (li < n) {
           ra[u] = ld_stream(a + first + li);
@@ -90,7 +94,7 @@ struct CombineOp {
       }
 #pragma unroll
       for (int u = 0; u < kU; ++u) {
-        const int64_t li = li0 + u * kCqThreads;
+        const int64_t li = li0 + u * kThreads;
         if (li < n) put(0, li, combine8(ra[u], sa, rb[u], sb, b != nullptr, rc[u], sc, c != nullptr, rd[u], sd, d != nullptr));
       }
     }
@@ -98,26 +102,30 @@ struct CombineOp {
 };
 
 struct SiluMulOp {
+  static constexpr int kThreads = kCqWideThreads;
   static constexpr int kOutputs = 1;
   const uint4 *g, *u;
   int64_t nvec;
   __device__ __forceinline__ void range(int64_t& first, int64_t& n) const { share_of(nvec, first, n); }
   template <class Put>
   __device__ __forceinline__ void produce(int64_t first, int64_t n, float (*)[4], Put put) const {
-    constexpr int kU = 4;
-    for (int64_t li0 = threadIdx.x; li0 < n; li0 += kCqThreads * kU) {
+    constexpr int kU = 2;
+    // the inputs are read once here: marked evict-first, they do not push the part of the result that waits in L2 for
+    // phase 2 out to memory
+    const uint64_t once = l2_policy_evict_first();
+    for (int64_t li0 = threadIdx.x; li0 < n; li0 += kThreads * kU) {
       uint4 rg[kU], ru[kU];
 #pragma unroll
       for (int k = 0; k < kU; ++k) {
-        const int64_t li = li0 + k * kCqThreads;
+        const int64_t li = li0 + k * kThreads;
         if (li < n) {
-          rg[k] = ld_stream(g + first + li);
-          ru[k] = ld_stream(u + first + li);
+          rg[k] = ld_global_hint(g + first + li, once);
+          ru[k] = ld_global_hint(u + first + li, once);
         }
       }
 #pragma unroll
       for (int k = 0; k < kU; ++k) {
-        const int64_t li = li0 + k * kCqThreads;
+        const int64_t li = li0 + k * kThreads;
         if (li < n) put(0, li, silu_mul8(rg[k], ru[k]));
       }
     }
@@ -125,6 +133,7 @@ struct SiluMulOp {
 };
 
 struct SiluMulGradOp {
+  static constexpr int kThreads = kCqWideThreads;
   static constexpr int kOutputs = 2;   // 0: dg, 1: du
   const uint4 *g, *u, *dz;
   int64_t nvec;
@@ -132,11 +141,11 @@ struct SiluMulGradOp {
   template <class Put>
   __device__ __forceinline__ void produce(int64_t first, int64_t n, float (*)[4], Put put) const {
     constexpr int kU = 2;
-    for (int64_t li0 = threadIdx.x; li0 < n; li0 += kCqThreads * kU) {
+    for (int64_t li0 = threadIdx.x; li0 < n; li0 += kThreads * kU) {
       uint4 rg[kU], ru[kU], rz[kU];
 #pragma unroll
       for (int k = 0; k < kU; ++k) {
-        const int64_t li = li0 + k * kCqThreads;
+        const int64_t li = li0 + k * kThreads;
         if (li < n) {
           rg[k] = ld_stream(g + first + li);
           ru[k] = ld_stream(u + first + li);
@@ -145,7 +154,7 @@ struct SiluMulGradOp {
       }
 #pragma unroll
       for (int k = 0; k < kU; ++k) {
-        const int64_t li = li0 + k * kCqThreads;
+        const int64_t li = li0 + k * kThreads;
         if (li < n) {
           uint4 qg, qu;
           silu_mul_grad8(rg[k], ru[k], rz[k], qg, qu);
@@ -160,6 +169,7 @@ struct SiluMulGradOp {
 // Row-wise producers: the CTA owns whole rows; its four groups of 128 threads take them in turn.
 template <bool kCombine, int kMaxVec>
 struct RmsnormOp {
+  static constexpr int kThreads = kMaxVec <= 4 ? kCqWideThreads : kCqThreads;
   static constexpr int kOutputs = 1;
   const uint4 *a, *b;
   float sa, sb;
@@ -178,7 +188,7 @@ struct RmsnormOp {
     const int grp = threadIdx.x >> 7;
     const RowGroup g{static_cast<int>(threadIdx.x & 127), 1 + grp, gred[grp]};
     const int nrows = static_cast<int>(n / vec_per_row);
-    for (int lr = grp; lr < nrows; lr += kCqThreads / kNormThreads) {
+    for (int lr = grp; lr < nrows; lr += kThreads / kNormThreads) {
       const int64_t base = first + static_cast<int64_t>(lr) * vec_per_row;
       const int64_t lbase = static_cast<int64_t>(lr) * vec_per_row;
       const float inv = rmsnorm_row<kMaxVec, kCombine>(a + base, sa, kCombine ? b + base : nullptr, sb, vec_per_row, inv_cols, eps, g,
@@ -191,6 +201,7 @@ struct RmsnormOp {
 
 template <int kMaxVec>
 struct RmsnormGradCombineOp {
+  static constexpr int kThreads = kMaxVec <= 4 ? kCqWideThreads : kCqThreads;
   static constexpr int kOutputs = 1;
   const uint4 *dy_a, *dy_b, *dy_c, *x, *res;
   const float* inv_rms;
@@ -208,7 +219,7 @@ struct RmsnormGradCombineOp {
     const int grp = threadIdx.x >> 7;
     const RowGroup g{static_cast<int>(threadIdx.x & 127), 1 + grp, gred[grp]};
     const int nrows = static_cast<int>(n / vec_per_row);
-    for (int lr = grp; lr < nrows; lr += kCqThreads / kNormThreads) {
+    for (int lr = grp; lr < nrows; lr += kThreads / kNormThreads) {
       const int64_t base = first + static_cast<int64_t>(lr) * vec_per_row;
       const int64_t lbase = static_cast<int64_t>(lr) * vec_per_row;
       rmsnorm_grad_row<kMaxVec, true>(dy_a + base, dy_b + base, dy_c != nullptr ? dy_c + base : nullptr, x + base,
@@ -231,13 +242,14 @@ __device__ __forceinline__ uint2 cast_vec(const uint4& q, float sc) {
 }
 
 template <class Op, int kFmt>
-__global__ void __launch_bounds__(kCqThreads, 1) chain_quant_kernel(const Op op, const CqTail<Op::kOutputs> tail) {
+__global__ void __launch_bounds__(Op::kThreads, 1) chain_quant_kernel(const Op op, const CqTail<Op::kOutputs> tail) {
   constexpr int kOut = Op::kOutputs;
+  constexpr int kThreads = Op::kThreads;
   constexpr int kCap = kCqStageVecs / kOut;   // vectors of each output that stay in shared memory
   extern __shared__ __align__(128) uint8_t cq_smem[];
   uint4* stage = reinterpret_cast<uint4*>(cq_smem);
   __shared__ uint32_t red[32];
-  __shared__ float gred[kCqThreads / kNormThreads][4];
+  __shared__ float gred[kCqWideThreads / kNormThreads][4];
   __shared__ int s_ok;
   pdl_trigger();
   pdl_wait();
@@ -257,7 +269,7 @@ __global__ void __launch_bounds__(kCqThreads, 1) chain_quant_kernel(const Op op,
   });
 #pragma unroll
   for (int w = 0; w < kOut; ++w) {
-    const uint32_t m = cta_max_u32(mx[w], red);
+    const uint32_t m = cta_max_u32<kThreads>(mx[w], red);
     if (tid == 0) tail.scratch->partial[w][blockIdx.x] = m << 16;
   }
   // ---- grid barrier (the CTA-wide barriers above ordered every thread's stores before thread 0's arrival)
@@ -268,38 +280,39 @@ __global__ void __launch_bounds__(kCqThreads, 1) chain_quant_kernel(const Op op,
 #pragma unroll
     for (int w = 0; w < kOut; ++w) {
       uint32_t mb = 0;
-      for (int i = tid; i < static_cast<int>(gridDim.x); i += kCqThreads) mb = max(mb, __ldcg(&tail.scratch->partial[w][i]));
-      const float amax = __uint_as_float(cta_max_u32(mb, red));
+      for (int i = tid; i < static_cast<int>(gridDim.x); i += kThreads) mb = max(mb, __ldcg(&tail.scratch->partial[w][i]));
+      const float amax = __uint_as_float(cta_max_u32<kThreads>(mb, red));
       const float sc = scale_from_amax(amax, kFmt);
       if (blockIdx.x == 0 && tid == 0) *tail.scale_out[w] = sc;
       uint2* dst = reinterpret_cast<uint2*>(tail.codes[w]) + first;
       const uint4* kept = stage + w * kCap;
       const uint4* spilled = tail.out16[w] + first;
+      const uint64_t once = l2_policy_evict_first();   // the passed-through part is dead once it has been read back
       const int64_t n_kept = n < kCap ? n : kCap;
       constexpr int kU = 4;
-      for (int64_t li0 = tid; li0 < n_kept; li0 += kCqThreads * kU) {
+      for (int64_t li0 = tid; li0 < n_kept; li0 += kThreads * kU) {
         uint4 q[kU];
 #pragma unroll
         for (int u = 0; u < kU; ++u) {
-          const int64_t li = li0 + u * kCqThreads;
+          const int64_t li = li0 + u * kThreads;
           if (li < n_kept) q[u] = kept[li];
         }
 #pragma unroll
         for (int u = 0; u < kU; ++u) {
-          const int64_t li = li0 + u * kCqThreads;
+          const int64_t li = li0 + u * kThreads;
           if (li < n_kept) dst[li] = cast_vec<kFmt>(q[u], sc);
         }
       }
-      for (int64_t li0 = kCap + tid; li0 < n; li0 += kCqThreads * kU) {
+      for (int64_t li0 = kCap + tid; li0 < n; li0 += kThreads * kU) {
         uint4 q[kU];
 #pragma unroll
         for (int u = 0; u < kU; ++u) {
-          const int64_t li = li0 + u * kCqThreads;
-          if (li < n) q[u] = __ldcg(spilled + li);
+          const int64_t li = li0 + u * kThreads;
+          if (li < n) q[u] = ld_global_hint(spilled + li, once);
         }
 #pragma unroll
         for (int u = 0; u < kU; ++u) {
-          const int64_t li = li0 + u * kCqThreads;
+          const int64_t li = li0 + u * kThreads;
           if (li < n) dst[li] = cast_vec<kFmt>(q[u], sc);
         }
       }
@@ -321,7 +334,7 @@ cudaError_t launch_variant(const Op& op, const CqTail<Op::kOutputs>& tail, int64
   if (grid > kCqMaxGrid) grid = kCqMaxGrid;
   if (grid > units) grid = units;
   if (grid < 1) grid = 1;
-  return launch_pdl(chain_quant_kernel<Op, kFmt>, dim3(static_cast<unsigned>(grid)), dim3(kCqThreads), kCqStageBytes, stream,
+  return launch_pdl(chain_quant_kernel<Op, kFmt>, dim3(static_cast<unsigned>(grid)), dim3(Op::kThreads), kCqStageBytes, stream,
                     -1 /* cooperative */, op, tail);
 }
 
@@ -359,7 +372,7 @@ int falqon_chain_combine_quantize(void* codes, float* scale_out, int fmt, void* 
                      static_cast<const uint4*>(d), sa, sb, sc, sd, count / 8};
   CqTail<1> tail{{static_cast<uint8_t*>(codes)}, {static_cast<uint4*>(out16)}, {scale_out}, static_cast<CqScratch*>(scratch), nullptr,
                  keep16};
-  return launch_op(op, tail, fmt, (count / 8 + kCqThreads - 1) / kCqThreads, stream);
+  return launch_op(op, tail, fmt, (count / 8 + kCqWideThreads - 1) / kCqWideThreads, stream);
 }
 
 int falqon_chain_silu_mul_quantize(void* codes, float* scale_out, int fmt, void* out16, int keep16, const void* g, const void* u,
@@ -369,7 +382,7 @@ int falqon_chain_silu_mul_quantize(void* codes, float* scale_out, int fmt, void*
   const SiluMulOp op{static_cast<const uint4*>(g), static_cast<const uint4*>(u), count / 8};
   CqTail<1> tail{{static_cast<uint8_t*>(codes)}, {static_cast<uint4*>(out16)}, {scale_out}, static_cast<CqScratch*>(scratch), nullptr,
                  keep16};
-  return launch_op(op, tail, fmt, (count / 8 + kCqThreads - 1) / kCqThreads, stream);
+  return launch_op(op, tail, fmt, (count / 8 + kCqWideThreads - 1) / kCqWideThreads, stream);
 }
 
 int falqon_chain_silu_mul_grad_quantize(void* codes_dg, void* codes_du, float* scale_dg, float* scale_du, int fmt, void* dg16,
@@ -385,7 +398,7 @@ int falqon_chain_silu_mul_grad_quantize(void* codes_dg, void* codes_du, float* s
                  static_cast<CqScratch*>(scratch),
                  nullptr,
                  keep16};
-  return launch_op(op, tail, fmt, (count / 8 + kCqThreads - 1) / kCqThreads, stream);
+  return launch_op(op, tail, fmt, (count / 8 + kCqWideThreads - 1) / kCqWideThreads, stream);
 }
 
 int falqon_chain_rmsnorm_quantize(void* codes, float* scale_out, int fmt, void* y16, int keep16, float* inv_rms, void* sum_out,

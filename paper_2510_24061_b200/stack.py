@@ -204,12 +204,16 @@ class Stack:
     """n_layers blocks with hidden size H and MLP width F, T tokens per step, LoRA rank r, top-k rows per update."""
 
     def __init__(self, n_layers: int, H: int, F: int, T: int, r: int, k: int, seed: int, device, lr: float = 2e-4,
-                 producer_amax: bool = True, batched_proxy: bool = True, adamw: dict | None = None, fuse_chain: bool = True):
+                 producer_amax: bool = True, batched_proxy: bool = True, adamw: dict | None = None, fuse_chain: bool = True,
+                 fuse_cast: bool | None = None):
         """producer_amax: the chain kernels hand the absmax of their outputs to the layers that consume them, whose
         input casts are then single-pass (False: every layer takes the absmax of its input itself).
         batched_proxy: the seven proxy updates of a block run as one falqon_proxy_update_batched call at the end of
         the block's backward (False: one falqon_proxy_update after every projection's backward; same results, since
         nothing later in the backward reads an updated backbone).
+        fuse_cast: every tensor a layer consumes (x1, a, x2, z and the output gradients) leaves the chain kernel that
+        produces it as FP8 codes (the *_quantize calls above): no separate cast kernel runs, the layers take codes
+        (falqon_melded_forward_codes / falqon_melded_backward_codes).  Same codes, so the same results bit for bit.
         adamw: None for the plain SGD step with lr, or the hyper-parameters (beta1, beta2, eps, weight_decay; lr is the
         argument above) of AdamW on every DeltaBuffer -- the optimizer the paper trains with; needs batched_proxy."""
         self.n_layers, self.H, self.F, self.T, self.r, self.k, self.lr = n_layers, H, F, T, r, k, lr
@@ -217,6 +221,10 @@ class Stack:
         assert adamw is None or batched_proxy
         self.producer_amax = producer_amax
         self.fuse_chain = fuse_chain        # residual sums fused with the normalisation (or its gradient) that follows them
+        if fuse_cast is None:               # the default wherever it applies
+            fuse_cast = fuse_chain and producer_amax
+        self.fuse_cast = fuse_cast
+        assert not fuse_cast or (fuse_chain and producer_amax)
         self.device = torch.device(device)
         self.seed = seed
         self.shapes = {"q": (H, H), "k": (H, H), "v": (H, H), "o": (H, H), "gate": (H, F), "up": (H, F), "down": (F, H)}  # n -> m
@@ -273,6 +281,11 @@ class Stack:
         # absmax words of the chain's outputs, one row per block: x1, a, x2, z | ddn, dg, du, dhp, dqkv (cleared every step)
         self.amax = torch.zeros((n_layers, 16), dtype=torch.float32, device=dev)
         self.capture = None   # optional: {(block, proj): dict} filled with references / copies for parity checks
+        if fuse_cast:         # codes and scales of the chain's outputs (reused by every block) and the kernels' scratch
+            u8e = lambda cols: torch.empty((T, cols), dtype=torch.uint8, device=dev)
+            self.cq_H, self.cq_F, self.gq_H = u8e(H), u8e(F), u8e(H)
+            self.cscale = torch.zeros(16, dtype=torch.float32, device=dev)
+            self.cscratch = chain_scratch(dev)
 
     # ---- one linear: forward on X (quantizing it) or on another projection's codes
     def _am(self, l, slot):
@@ -317,11 +330,92 @@ class Stack:
             fq.proxy_update(self.layers[l][name], self.dB[name], self.lr, self.k, ws=self.ws[name],
                             idx_out=self.idx if self.k > 0 else None)
 
+    def _sc(self, slot):
+        return self.cscale[slot:slot + 1]
+
+    def _fwd_codes(self, l, name, X16, xq, slot, Y):
+        sv = self.saved[l]
+        fq.melded_forward_codes(self.layers[l][name], xq, self._sc(slot), ws=self.ws[name], out=(Y, sv["oa"][name], sv["amax"][name]))
+        self._cap(l, name, X=X16, Y=Y)
+
+    def _bwd_codes(self, l, name, dY16, gq, slot, dX):
+        sv = self.saved[l]
+        fq.melded_backward_codes(self.layers[l][name], gq, self._sc(slot), sv["oa"][name], sv["amax"][name], ws=self.ws[name],
+                                 out=(dX, self.dB[name]))
+        self._cap(l, name, dY=dY16, dX=dX, dB=self.dB[name], OA=sv["oa"][name])
+        if self.batches is None:
+            fq.proxy_update(self.layers[l][name], self.dB[name], self.lr, self.k, ws=self.ws[name],
+                            idx_out=self.idx if self.k > 0 else None)
+
+    def _forward_fused_cast(self, h0):
+        keep = self.capture is not None      # the bf16 tensors are only needed by the parity checks
+        E4 = fq.E4M3
+        for l in range(self.n_layers):
+            sv = self.saved[l]
+            if l == 0:
+                sv["h"].copy_(h0)
+                rmsnorm_quantize(self.cq_H, self._sc(0), E4, self.x1, keep, self.cscratch, sv["inv1"], sv["h"])
+            h, hp = sv["h"], sv["hp"]
+            self._fwd_codes(l, "q", self.x1, self.cq_H, 0, self.q)
+            self._fwd_codes(l, "k", self.x1, self.cq_H, 0, self.kk)
+            self._fwd_codes(l, "v", self.x1, self.cq_H, 0, self.v)
+            combine_quantize(self.cq_H, self._sc(1), E4, self.a, keep, self.cscratch, self.q, INV_SQRT3, self.kk, INV_SQRT3,
+                             self.v, INV_SQRT3)
+            self._fwd_codes(l, "o", self.a, self.cq_H, 1, self.o)
+            rmsnorm_quantize(self.cq_H, self._sc(2), E4, self.x2, keep, self.cscratch, sv["inv2"], h, sum_out=hp, sa=1.0, b=self.o,
+                             sb=1.0)
+            self._fwd_codes(l, "gate", self.x2, self.cq_H, 2, sv["g"])
+            self._fwd_codes(l, "up", self.x2, self.cq_H, 2, sv["u"])
+            silu_mul_quantize(self.cq_F, self._sc(3), E4, self.z, keep, self.cscratch, sv["g"], sv["u"])
+            self._fwd_codes(l, "down", self.z, self.cq_F, 3, self.dn)
+            if l + 1 < self.n_layers:
+                nx = self.saved[l + 1]
+                rmsnorm_quantize(self.cq_H, self._sc(0), E4, self.x1, keep, self.cscratch, nx["inv1"], hp, sum_out=nx["h"],
+                                 sa=INV_SQRT2, b=self.dn, sb=INV_SQRT2)
+            else:
+                combine(self.h_out, hp, INV_SQRT2, self.dn, INV_SQRT2)
+        return self.h_out
+
+    def _backward_fused_cast(self, G):
+        self.amax.zero_()
+        keep = self.capture is not None
+        E5 = fq.E5M2
+        dh = G
+        for l in reversed(range(self.n_layers)):
+            sv = self.saved[l]
+            combine_quantize(self.gq_H, self._sc(4), E5, self.ddn, keep, self.cscratch, dh, INV_SQRT2)
+            self._bwd_codes(l, "down", self.ddn, self.gq_H, 4, self.dz)
+            # dg and du (two [T][F] tensors at once) would mostly pass through memory between the two phases of a
+            # quantizing kernel, which then loses to the plain kernel and two single-pass casts: these two stay separate
+            silu_mul_grad(self.dg, self.du, sv["g"], sv["u"], self.dz, self.amax[l, 5:6], self.amax[l, 6:7])
+            self._bwd(l, "gate", self.dg, self.dx[0], self.amax[l, 5:6])
+            self._bwd(l, "up", self.du, self.dx[1], self.amax[l, 6:7])
+            rmsnorm_grad_combine_quantize(self.gq_H, self._sc(7), E5, self.dhp, self.cscratch, [self.dx[0], self.dx[1]], sv["hp"],
+                                          sv["inv2"], dh, INV_SQRT2)
+            self._bwd_codes(l, "o", self.dhp, self.gq_H, 7, self.da)
+            combine_quantize(self.gq_H, self._sc(8), E5, self.dqkv, keep, self.cscratch, self.da, INV_SQRT3)
+            self._bwd_codes(l, "q", self.dqkv, self.gq_H, 8, self.dx[0])
+            self._bwd_codes(l, "k", self.dqkv, self.gq_H, 8, self.dx[1])
+            self._bwd_codes(l, "v", self.dqkv, self.gq_H, 8, self.dx[2])
+            rmsnorm_grad_combine(self.dh, [self.dx[0], self.dx[1], self.dx[2]], sv["h"], sv["inv1"], self.dhp, 1.0)
+            dh = self.dh
+            self._run_batch(l)
+        return dh
+
+    def _run_batch(self, l):
+        if self.batches is not None:
+            if self.adamw is None:
+                self.batches[l].run(self.lr)
+            else:
+                self.batches[l].run_adamw(self.exp_avg[l], self.exp_avg_sq[l], lr=self.lr, step=self.steps_done + 1, **self.adamw)
+
     def _cap(self, l, name, **tensors):
         if self.capture is not None and (l, name) in self.capture:
             self.capture[(l, name)].update({k2: v.clone() for k2, v in tensors.items()})
 
     def forward(self, h0: torch.Tensor) -> torch.Tensor:
+        if self.fuse_cast:
+            return self._forward_fused_cast(h0)
         if self.producer_amax:
             self.amax.zero_()
         for l in range(self.n_layers):
@@ -355,6 +449,8 @@ class Stack:
     def backward(self, G: torch.Tensor):
         """G = d loss / d h_last.  Each block's backward is followed at once by the proxy updates of its layers
         (one batched call, or inside _bwd), as in the paper's layer-wise training loop."""
+        if self.fuse_cast:
+            return self._backward_fused_cast(G)
         dh = G
         for l in reversed(range(self.n_layers)):
             sv = self.saved[l]
@@ -381,12 +477,7 @@ class Stack:
                 rmsnorm_grad(self.dx[1], self.dx[0], sv["h"], sv["inv1"])
                 combine(self.dh, self.dhp, 1.0, self.dx[1], 1.0)
             dh = self.dh
-            if self.batches is not None:
-                if self.adamw is None:
-                    self.batches[l].run(self.lr)
-                else:
-                    self.batches[l].run_adamw(self.exp_avg[l], self.exp_avg_sq[l], lr=self.lr, step=self.steps_done + 1,
-                                              **self.adamw)
+            self._run_batch(l)
         return dh
 
     def step(self, h0: torch.Tensor, G: torch.Tensor):
@@ -401,6 +492,16 @@ class Stack:
         return float(self.n_layers * sum(2 * T * (n * (m + r) + m * n + m * r) for n, m in self.shapes.values()))
 
     def launches_per_step(self) -> int:
+        if self.fuse_cast:
+            # per block: 7 forward products; 7 x (O_A cast, dB, dX) + the two single-pass casts of dg and du; 4 + 5 chain
+            # kernels; the proxy update(s); plus the first block's normalisation (the last block's plain residual sum stands
+            # in for a quantizing one)
+            per_block = 7 + 7 * 3 + 2 + 4 + 5
+            if self.batches is None:
+                per_block += 7 * fq.launch_count("falqon_proxy_update", k=self.k)
+            else:
+                per_block += fq.launch_count("falqon_proxy_update_batched", k=self.k)
+            return per_block * self.n_layers + 1
         per_block = 0
         for name in PROJ:
             shared = name in ("k", "v", "up")

@@ -136,7 +136,7 @@ def test_stack_with_fused_chain_equals_the_unfused_stack(fq, st):
     G = synth.normal_bf16(5, 9002, (T, H), 1.0e-2, dev)
     outs = []
     for fuse in (False, True):
-        stack = st.Stack(3, H, F, T, r, k, seed=5, device=dev, lr=2e-2, fuse_chain=fuse)
+        stack = st.Stack(3, H, F, T, r, k, seed=5, device=dev, lr=2e-2, fuse_chain=fuse, fuse_cast=False)
         h = stack.forward(h0).clone()
         dh = stack.backward(G).clone()
         torch.cuda.synchronize()
@@ -188,9 +188,10 @@ def _check_projection(fq, orc, cap, layer, name, T, r, k, lr, n_rows):
     assert np.array_equal(bits32(f32(layer.dbuf)), bits32(dbuf_o)), f"{name} DeltaBuffer"
 
 
-def _run_and_check(fq, st, orc, n_layers, H, F, T, r, k, check_blocks, n_rows, producer_amax=True):
+def _run_and_check(fq, st, orc, n_layers, H, F, T, r, k, check_blocks, n_rows, producer_amax=True, fuse_cast=False):
     stack = st.Stack(n_layers, H, F, T, r, k, seed=7, device=DEV, lr=2e-2, producer_amax=producer_amax,
-                     batched_proxy=producer_amax)   # the second variant also keeps the per-projection proxy updates
+                     batched_proxy=producer_amax,   # the second variant also keeps the per-projection proxy updates
+                     fuse_cast=fuse_cast)
     h0 = synth.normal_bf16(7, 9001, (T, H), 1.0, DEV)
     G = synth.normal_bf16(7, 9002, (T, H), 1.0e-2, DEV)
     stack.capture = {(l, p): {} for l in check_blocks for p in st.PROJ}
@@ -214,11 +215,41 @@ def test_small_stack_every_projection(fq, st, orc, producer_amax):
     _run_and_check(fq, st, orc, 3, 256, 640, 192, 16, 8, check_blocks=[0, 1, 2], n_rows=192, producer_amax=producer_amax)
 
 
+def test_small_stack_with_the_casts_inside_the_chain_kernels(fq, st, orc):
+    """The same chain with every layer input and output gradient leaving its producing kernel as FP8 codes: every
+    projection against the oracle (the captured bf16 tensors are the ones the codes were made from), and the whole step
+    bit for bit the step of the stack with separate casts."""
+    _run_and_check(fq, st, orc, 3, 256, 640, 192, 16, 8, check_blocks=[0, 1, 2], n_rows=192, fuse_cast=True)
+    H, F, T, r, k = 256, 512, 300, 16, 24
+    dev = torch.device(DEV)
+    h0 = synth.normal_bf16(5, 9001, (T, H), 1.0, dev)
+    G = synth.normal_bf16(5, 9002, (T, H), 1.0e-2, dev)
+    outs = []
+    for fuse in (False, True):
+        stack = st.Stack(3, H, F, T, r, k, seed=5, device=dev, lr=2e-2, fuse_cast=fuse)
+        for _ in range(2):        # two steps: the second runs on updated backbones and reuses the kernels' scratch
+            h = stack.step(h0, G).clone()
+        dh = stack.dh.clone()
+        torch.cuda.synchronize()
+        outs.append((h, dh, [(L.wq.clone(), L.dbuf.clone()) for blk in stack.layers for L in blk.values()]))
+    (h_a, dh_a, la), (h_b, dh_b, lb) = outs
+    assert torch.equal(h_a.view(torch.int16), h_b.view(torch.int16)) and torch.equal(dh_a.view(torch.int16), dh_b.view(torch.int16))
+    for (wa, da), (wb, db) in zip(la, lb):
+        assert torch.equal(wa, wb) and torch.equal(da.view(torch.int32), db.view(torch.int32))
+    assert fq.last_device_status() == 0
+
+
 def test_stack_7b_shapes_sampled(fq, st, orc):
     """The 7B shapes (hidden 4096, MLP 11008, 4096 tokens, rank 64, top-256), 32 blocks in one step: the first, the
     last and two other blocks are checked on sampled rows."""
     stack = _run_and_check(fq, st, orc, 32, 4096, 11008, 4096, 64, 256, check_blocks=[0, 11, 22, 31], n_rows=24)
     assert stack.flops_per_step() == pytest.approx(107.41e12, rel=1e-3)
+
+
+def test_stack_7b_shapes_sampled_with_the_casts_inside_the_chain_kernels(fq, st, orc):
+    """The same at full size with the quantizing chain kernels (x1, a, x2 stay in shared memory across the grid barrier; z,
+    dg and du mostly pass through memory)."""
+    _run_and_check(fq, st, orc, 32, 4096, 11008, 4096, 64, 256, check_blocks=[0, 17, 31], n_rows=24, fuse_cast=True)
 
 
 def test_small_stack_with_adamw(fq, st, orc):
