@@ -585,7 +585,7 @@ cudaError_t launch_scale_prep(const uint32_t* partial, int nparts, const float* 
 __global__ void __launch_bounds__(256) oa_cast_kernel(OaCastJob job) {
   pdl_trigger();
   pdl_wait();
-  cast_oa_transposed(job, threadIdx.x >> 5, 8);
+  cast_oa_transposed(job, threadIdx.x >> 5, blockDim.x >> 5);
 }
 
 template <int kDt, int kFmt, bool kColMul>
@@ -650,10 +650,13 @@ cudaError_t launch_quantize_fused(const void* src, int src_dt, int64_t count, in
 }
 
 cudaError_t launch_oa_cast(const OaCastJob& job, cudaStream_t stream) {
+  // one warp converts a tile of 32 tokens; the tensor is small (T x r fp32), so the kernel is as long as its slowest warp:
+  // few warps per CTA spread the tiles over the whole chip (4096 tokens: 128 tiles on 128 SMs instead of 16)
   const long long tiles = (job.T + 31) / 32;
-  long long grid = (tiles + 7) / 8;
+  const int warps = tiles >= 148 * 8 * 4 ? 8 : tiles >= 148 * 4 ? 2 : 1;
+  long long grid = (tiles + warps - 1) / warps;
   if (grid > 148 * 8) grid = 148 * 8;
-  return launch_pdl(oa_cast_kernel, dim3(static_cast<unsigned>(grid)), dim3(256), 0, stream, 1, job);
+  return launch_pdl(oa_cast_kernel, dim3(static_cast<unsigned>(grid)), dim3(32 * warps), 0, stream, 1, job);
 }
 
 cudaError_t launch_scale_table(int mode, const float* s_w, int64_t m, int64_t r, const float* s_x, float* out, int64_t padded,
