@@ -60,6 +60,7 @@ int falqon_chain_rmsnorm_grad_combine(void *out, const void *dy_a, const void *d
  *   out16      device [count] bf16, 16-byte aligned.  keep16 != 0: receives the bf16 result as the plain call stores it.
  *              keep16 == 0: working space -- the part of the tensor that does not fit in the SMs' shared memory between
  *              the two phases of the kernel passes through it; its contents afterwards are unspecified.
+ *              It may be one of the inputs (every position is read before it is written).
  *   scratch    FALQON_CHAIN_SCRATCH_BYTES device bytes, 16-byte aligned, zero before the first call and left zero by every
  *              call; calls that may run at the same time need scratch of their own.
  * The kernel holds a grid-wide barrier (the absmax of the whole tensor precedes the first code), so the launch is
