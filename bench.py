@@ -726,6 +726,17 @@ def main():
     clocks["soak_before"] = clocks_soak
     clocks["timed_steps_only"] = clocks_timed
     value = world * flops_step / (ms_step * 1e-3) / 1e12
+    # ---- the spread of single steps, right after the timed region (same regime): an event after every step
+    n_spread = max(args.steps, 20)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_spread + 1)]
+    marks[0].record()
+    for i in range(n_spread):
+        one_step()
+        marks[i + 1].record()
+    torch.cuda.synchronize()
+    singles = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(n_spread))
+    per_step = {"n": n_spread, "median_ms": singles[n_spread // 2], "min_ms": singles[0], "max_ms": singles[-1],
+                "note": "this rank's steps one by one, an event after each, right after the timed region"}
 
     # ---- forward and backward alone (quantization included, no proxy update): the quantity the metric's name describes;
     # `value` above is the whole hot path, proxy update included
@@ -878,7 +889,7 @@ def main():
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": ms_step, "mcycles_per_step": with_cycles(ms_step, clocks),
+        "ms_per_step": ms_step, "mcycles_per_step": with_cycles(ms_step, clocks), "per_step": per_step,
         "regime": "sustained: %.1f s of the same step loop ran right before the timed steps" % args.soak,
         "burst": {"ms_per_step": ms_burst, "value": world * flops_step / (ms_burst * 1e-3) / 1e12, "unit": UNIT, "steps": burst_steps,
                   "mcycles_per_step": with_cycles(ms_burst, clocks_burst), "clocks": clocks_burst,

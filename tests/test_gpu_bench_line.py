@@ -49,4 +49,6 @@ def test_default_line_has_the_contract_keys():
         assert abs(q["frac"] - q["achieved_gbs"] / q["peak_gbs"]) < 1e-9 and 0 < q["frac"] < 1.2
     assert d["quantize"]["bytes_per_elt"] == 3               # every tensor of configs[1] fits L2: one DRAM read, one write
     assert "sustained" in r["regime"] and "instrumented_pass" in d and d["instrumented_pass"]["clocks"]["samples"] >= 1
+    ps = d["per_step"]            # single steps right after the timed region: the same regime, so the same time
+    assert ps["n"] >= 20 and ps["min_ms"] <= ps["median_ms"] <= ps["max_ms"] and abs(ps["median_ms"] - d["ms_per_step"]) < 0.1 * d["ms_per_step"]
     assert d["device_status"] == 0
