@@ -301,13 +301,43 @@ __device__ __forceinline__ void cast_unit(const uint4& q, int64_t e, int col, co
   }
 }
 
+// The column-scaled cast of one 16-byte unit of bf16 values with packed multiplies: fl(fl(x * c) * s), each half of
+// a mul.rn.f32x2 being an ordinary rounded product.  f: the unit's eight column factors in shared memory (16-byte aligned).
+template <int kFmt>
+__device__ __forceinline__ uint2 cast_unit_colmul_packed(const uint4& q, const float* f, uint64_t s2) {
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+  const ulonglong2 c01 = *reinterpret_cast<const ulonglong2*>(f);
+  const ulonglong2 c23 = *reinterpret_cast<const ulonglong2*>(f + 4);
+  const uint64_t c[4] = {c01.x, c01.y, c23.x, c23.y};
+  float x[8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint64_t v = pack_f32x2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xFFFF0000u));
+    asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(v) : "l"(c[i]));
+    asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(v) : "l"(s2));
+    unpack_f32x2(v, x[2 * i], x[2 * i + 1]);
+  }
+  uint2 o;
+  o.x = cvt_fp8x4<kFmt>(x[0], x[1], x[2], x[3]);
+  o.y = cvt_fp8x4<kFmt>(x[4], x[5], x[6], x[7]);
+  return o;
+}
+
 template <int kDt, int kFmt, bool kColMul>
 __global__ void __launch_bounds__(kStagedThreads, 1)
 quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* partial, GridSync* sync, CastOutputs out,
-                       int* status, const float* col_mul, int cols, OaCastJob oa_job, int slots, int table_floats) {
+                       int* status, const float* col_mul, int cols, OaCastJob oa_job, int slots, int table_floats,
+                       int rows_per_chunk) {
   constexpr int kEsize = kDt == kBF16 ? 2 : 4;
   constexpr int kUnit = Unit<kDt>::kElems;
-  constexpr int64_t kChunkElems = kChunkBytes / kEsize;
+  // Row-aligned mode of the column-scaled form (rows_per_chunk > 0; bf16 input, the factors in shared memory): a chunk is
+  // a whole number of rows, so unit u of EVERY chunk belongs to columns 8 (u mod cols/8) ..., and a thread, which always
+  // takes the units tid, tid + 512, ..., always sees the same columns.  The absmax pass then needs no multiply at all:
+  // fl(|x| c) is monotone in |x| for c > 0, so max_t |fl(x[t][i] c_i)| = fl(max_t |x[t][i]| c_i) -- the thread keeps the
+  // largest |bf16| pattern per column position (packed 16-bit maxima) and applies the factors once, after the last chunk.
+  const bool row_mode = kColMul && kDt == kBF16 && rows_per_chunk > 0;
+  const int64_t kChunkElems = row_mode ? static_cast<int64_t>(rows_per_chunk) * cols : kChunkBytes / kEsize;
+  constexpr int kRowUnits = kChunkBytes / 16 / kStagedThreads;   // units per thread and chunk in row-aligned mode (7)
   // dynamic shared memory: [table_floats column factors, padded to whole chunks][slots x 16 KB ring]
   extern __shared__ __align__(128) uint8_t staged_smem[];
   // (only the column-scaled form has a table; without one the ring is the whole array and its size a constant)
@@ -332,7 +362,8 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
     __syncthreads();
   }
 
-  const int64_t bulk_elems = (count / 16) * 16;      // the rest (fewer than 16 elements) goes element by element
+  // (row-aligned mode: count is a whole number of rows of a multiple of 8 values, every chunk a multiple of 16 bytes)
+  const int64_t bulk_elems = row_mode ? count : (count / 16) * 16;   // the rest (fewer than 16 elements) goes element by element
   const int64_t n_chunks = (bulk_elems + kChunkElems - 1) / kChunkElems;
   const int grid = static_cast<int>(gridDim.x);
   const int n_my = blockIdx.x < n_chunks ? static_cast<int>((n_chunks - blockIdx.x + grid - 1) / grid) : 0;
@@ -352,9 +383,9 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
     // a chunk that will still be in the ring when the cast pass starts is read from memory exactly once: it need not
     // stay in L2 (and should not displace what is there); an earlier chunk will be fetched again and should
     if (i + nslots >= n_my)
-      bulk_load_1d_hint(smem_u32(stage + s * kChunkBytes), static_cast<const uint8_t*>(src) + c * kChunkBytes, bytes, bar, evict_first);
+      bulk_load_1d_hint(smem_u32(stage + s * kChunkBytes), static_cast<const uint8_t*>(src) + c * kChunkElems * kEsize, bytes, bar, evict_first);
     else
-      bulk_load_1d(smem_u32(stage + s * kChunkBytes), static_cast<const uint8_t*>(src) + c * kChunkBytes, bytes, bar);
+      bulk_load_1d(smem_u32(stage + s * kChunkBytes), static_cast<const uint8_t*>(src) + c * kChunkElems * kEsize, bytes, bar);
   };
 
   // ---- pass 1: absmax
@@ -363,22 +394,63 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
   uint32_t phase_bits = 0;   // bit s: parity of the next completion of slot s
   uint32_t m = 0;
   bool failed = false;
+  // row-aligned mode: the first column of each of this thread's units (the same in every chunk), and the running
+  // maxima of |bf16| per column position, two to a word
+  int my_col[kRowUnits];
+  uint32_t colmax[kRowUnits][4];
+  if (row_mode) {
+    const int upr = cols / kUnit;
+#pragma unroll
+    for (int j = 0; j < kRowUnits; ++j) {
+      my_col[j] = ((tid + j * kStagedThreads) % upr) * kUnit;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) colmax[j][w] = 0u;
+    }
+  }
   // (the slot index is stepped along with i: an integer division per chunk costs as much as a third of the chunk's work)
   for (int i = 0, s = 0; i < n_my; ++i, s = s + 1 == nslots ? 0 : s + 1) {
     const bool ok = mbar_wait(smem_u32(&bars[s]), (phase_bits >> s) & 1u, status);
     phase_bits ^= 1u << s;
     const int64_t e0 = chunk_of(i) * kChunkElems;
-    const uint32_t col0 = kColMul ? static_cast<uint32_t>(e0 % cols) : 0u;   // one 64-bit modulo per chunk, 32-bit ones per unit
     const int units = chunk_elems(chunk_of(i)) / kUnit;
     const uint4* sp = reinterpret_cast<const uint4*>(stage + s * kChunkBytes);
-    for (int u = tid; u < units; u += kStagedThreads) {
-      float x[kUnit];
-      unit_values<kDt, kColMul>(sp[u], col_mul, table, kColMul ? static_cast<int>(wrap_col(col0 + static_cast<uint32_t>(u) * kUnit, static_cast<uint32_t>(cols))) : 0, x);
+    if (row_mode) {
 #pragma unroll
-      for (int e = 0; e < kUnit; ++e) m = max(m, abs_bits(x[e]));
+      for (int j = 0; j < kRowUnits; ++j) {
+        const int u = tid + j * kStagedThreads;
+        if (u < units) {
+          const uint4 q = sp[u];
+          const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            asm("max.u16x2 %0, %0, %1;" : "+r"(colmax[j][k]) : "r"(w[k] & 0x7FFF7FFFu));
+        }
+      }
+    } else {
+      const uint32_t col0 = kColMul ? static_cast<uint32_t>(e0 % cols) : 0u;   // one 64-bit modulo per chunk, 32-bit ones per unit
+      for (int u = tid; u < units; u += kStagedThreads) {
+        float x[kUnit];
+        unit_values<kDt, kColMul>(sp[u], col_mul, table, kColMul ? static_cast<int>(wrap_col(col0 + static_cast<uint32_t>(u) * kUnit, static_cast<uint32_t>(cols))) : 0, x);
+#pragma unroll
+        for (int e = 0; e < kUnit; ++e) m = max(m, abs_bits(x[e]));
+      }
     }
     if (!__syncthreads_and(ok)) { failed = true; break; }   // block-uniform; also: the slot is free again
     if (tid == 0 && i + nslots < n_my) issue(i + nslots);
+  }
+  if (row_mode) {   // the factors, once per column position this thread has seen
+#pragma unroll
+    for (int j = 0; j < kRowUnits; ++j) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const uint32_t pair = colmax[j][k];
+        if (pair != 0u) {
+          const float* f = table + my_col[j] + 2 * k;
+          m = max(m, abs_bits(__fmul_rn(__uint_as_float(pair << 16), f[0])));
+          m = max(m, abs_bits(__fmul_rn(__uint_as_float(pair & 0xFFFF0000u), f[1])));
+        }
+      }
+    }
   }
   if (blockIdx.x == 0) {   // ragged tail
     for (int64_t e = bulk_elems + tid; e < count; e += kStagedThreads) {
@@ -434,13 +506,22 @@ quantize_staged_kernel(const void* src, int64_t count, uint8_t* dst, uint32_t* p
         phase_bits ^= 1u << s;
       }
       const int64_t e0 = chunk_of(i) * kChunkElems;
-      const uint32_t col0 = kColMul ? static_cast<uint32_t>(e0 % cols) : 0u;
+      const uint32_t col0 = kColMul && !row_mode ? static_cast<uint32_t>(e0 % cols) : 0u;
       const uint32_t ucols = kColMul ? static_cast<uint32_t>(cols) : 1u;
       const int units = chunk_elems(chunk_of(i)) / kUnit;
       const uint4* sp = reinterpret_cast<const uint4*>(stage + s * kChunkBytes);
+      if (row_mode) {   // the thread's columns are known; two packed multiplies per pair of values
+        const uint64_t s2 = pack_f32x2(sc, sc);
+#pragma unroll
+        for (int j = 0; j < kRowUnits; ++j) {
+          const int u = tid + j * kStagedThreads;
+          if (u < units)
+            *reinterpret_cast<uint2*>(dst + e0 + static_cast<int64_t>(u) * kUnit) = cast_unit_colmul_packed<kFmt>(sp[u], table + my_col[j], s2);
+        }
+      }
       // two units per thread and iteration (a full chunk is exactly one iteration): both shared-memory loads are
       // issued before either conversion chain starts
-      for (int u = tid; u < units; u += 2 * kStagedThreads) {
+      for (int u = tid; !row_mode && u < units; u += 2 * kStagedThreads) {
         const int u1 = u + kStagedThreads;
         const bool has1 = u1 < units;
         const uint4 q0 = sp[u];
@@ -612,21 +693,24 @@ cudaError_t launch_staged_variant(const void* src, int64_t count, uint8_t* dst, 
     blocks_per_sm_of[dev].store(blocks_per_sm);
   }
   const int sms = sm_count();
-  const int64_t chunk_elems = kChunkBytes / (kDt == kBF16 ? 2 : 4);
-  int64_t grid = (count / 16 * 16 + chunk_elems - 1) / chunk_elems;
+  // per-row mode: the column factors live in shared memory too when they fit beside at least 128 KB of ring slots
+  int table_floats = 0, slots = kStagedSlots, rows_per_chunk = 0;
+  if (kColMul) {
+    const int table_chunks = static_cast<int>((static_cast<int64_t>(cols) * 4 + kChunkBytes - 1) / kChunkBytes);
+    if (table_chunks <= kStagedSlots - (128 * 1024) / kChunkBytes) { table_floats = cols; slots = kStagedSlots - table_chunks; }
+    // ... and the chunks are whole rows (the kernel's row-aligned mode) when a row of bf16 fits a chunk
+    if (kDt == kBF16 && table_floats > 0 && cols % 8 == 0 && count % cols == 0 && static_cast<int64_t>(cols) * 2 <= kChunkBytes)
+      rows_per_chunk = static_cast<int>(kChunkBytes / (static_cast<int64_t>(cols) * 2));
+  }
+  const int64_t chunk_elems = rows_per_chunk > 0 ? static_cast<int64_t>(rows_per_chunk) * cols : kChunkBytes / (kDt == kBF16 ? 2 : 4);
+  int64_t grid = ((rows_per_chunk > 0 ? count : count / 16 * 16) + chunk_elems - 1) / chunk_elems;
   const int64_t resident = static_cast<int64_t>(blocks_per_sm) * sms;   // all CTAs must be resident together
   if (grid > resident) grid = resident;
   if (grid > kMaxAbsmaxParts) grid = kMaxAbsmaxParts;
   if (grid < 1) grid = 1;
-  // per-row mode: the column factors live in shared memory too when they fit beside at least eight ring slots
-  int table_floats = 0, slots = kStagedSlots;
-  if (kColMul) {
-    const int table_chunks = static_cast<int>((static_cast<int64_t>(cols) * 4 + kChunkBytes - 1) / kChunkBytes);
-    if (table_chunks <= kStagedSlots - (128 * 1024) / kChunkBytes) { table_floats = cols; slots = kStagedSlots - table_chunks; }
-  }
   return launch_pdl(quantize_staged_kernel<kDt, kFmt, kColMul>, dim3(static_cast<unsigned>(grid)), dim3(kStagedThreads), kSmem,
                     stream, -1 /* cooperative */, src, count, dst, partial, static_cast<GridSync*>(sync), out, status, col_mul, cols,
-                    oa_job, slots, table_floats);
+                    oa_job, slots, table_floats, rows_per_chunk);
 }
 
 cudaError_t launch_quantize_fused(const void* src, int src_dt, int64_t count, int fmt, uint8_t* dst, uint32_t* partial,
