@@ -425,3 +425,29 @@ def test_backward_on_shared_gradient_codes(fq, orc):
         fq.melded_backward_codes(Lr, gq, s_g, OA2, am2, ws=Lr.workspace(T))
     assert e.value.status == fq.ERR_UNSUPPORTED
     assert fq.last_device_status() == 0
+
+
+@pytest.mark.parametrize("m,T", [(16, 40), (1040, 333), (1040, 20011), (14336, 131), (16384, 37), (28688, 19)])
+def test_column_scaled_cast_of_bf16_gradients_in_every_chunk_geometry(fq, orc, m, T):
+    """The output-gradient cast of a per-row-scaled layer (dY[:, i] / s_w[i], then Eq. quantize in E5M2) on bf16 input:
+    rows that fit a staging chunk many times, exactly twice, once (the row-aligned mode: chunks are whole rows, the absmax
+    pass takes column maxima first and multiplies once), and rows longer than a chunk (linear chunks, a multiply per
+    element); a ragged last chunk; a tensor larger than the chip's shared memory (chunks fetched twice).  Codes and scale
+    bit for bit against the oracle."""
+    n, r = 64, 16
+    W = synth.backbone(41, 0, m, n, DEV, heavy_tailed=True)
+    A = synth.adapter_a(41, 0, r, n, DEV)
+    B = synth.adapter_b(41, 0, m, r, DEV)
+    X = synth.activations(41, 0, T, n, 2, DEV)
+    layer = fq.setup_layer(W, A, B, 1.0, per_row=True)
+    ws = layer.workspace(T)
+    _, OA, amax_oa, _ = fq.melded_forward(layer, X, y_dtype=torch.float32, ws=ws)
+    dY = synth.out_grad(41, 0, 0, T, m, DEV)
+    dY[T // 2, m - 3] = 0.75          # the absmax sits where only the column factor decides
+    assert dY.dtype == torch.bfloat16
+    fq.ws_view(layer, ws, T, fq.WS_GQ).fill_(0x55)
+    _, _, s_g = fq.melded_backward(layer, dY, OA, amax_oa, dx_dtype=torch.float32, ws=ws)
+    gq_o, s_g_o, _ = orc.quantize_colscaled(f32(dY), orc.E5M2, f32(layer.s_w)[:m])
+    assert bits32(f32(s_g))[0] == bits32(s_g_o)
+    assert np.array_equal(u8(fq.ws_view(layer, ws, T, fq.WS_GQ))[: T * m].reshape(T, m), gq_o)
+    assert fq.last_device_status() == 0
