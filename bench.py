@@ -430,6 +430,7 @@ def run_stack(args):
     stack = st.Stack(n_layers, H, F, T, r, k, seed=cfg["seed"], device=dev, lr=lr, producer_amax=not args.stack_own_absmax,
                      batched_proxy=not args.proxy_per_layer, fuse_chain=not args.stack_unfused_chain,
                      fuse_cast=not (args.stack_separate_casts or args.stack_own_absmax or args.stack_unfused_chain),
+                     layer_flags=fq.LAYER_DB_OWN_KERNEL if args.own_db else 0,
                      adamw=dict(beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0) if args.stack_adamw else None)
     h0 = synth.normal_bf16(cfg["seed"], 9001, (T, H), 1.0, dev)
     G = synth.normal_bf16(cfg["seed"], 9002, (T, H), 1.0e-2, dev)
@@ -555,6 +556,9 @@ def main():
     ap.add_argument("--stack-separate-casts", action="store_true",
                     help="with --stack: every cast is a kernel of its own (default: the casts run inside the chain kernels that "
                          "produce the tensors, all but those of the gated MLP's two gradients)")
+    ap.add_argument("--own-db", action="store_true",
+                    help="the adapter gradient as a kernel of its own (FALQON_LAYER_DB_OWN_KERNEL) instead of riding on the "
+                         "input-gradient product's launch")
     ap.add_argument("--stack-adamw", action="store_true",
                     help="with --stack: AdamW (beta 0.9 / 0.999, eps 1e-8, no weight decay) on every DeltaBuffer instead of plain SGD")
     ap.add_argument("--config3", action="store_true",
@@ -646,7 +650,7 @@ def main():
 
     layers = build_workload(fq, device, cfg["seed"] + rank, T, r, k, linears, cfg["outlier_frac"],
                             per_row=cfg.get("per_row", False), heavy_tailed=cfg.get("heavy_tailed", False),
-                            flags=fq.LAYER_FUSED_CAST if args.fused else 0)
+                            flags=(fq.LAYER_FUSED_CAST if args.fused else 0) | (fq.LAYER_DB_OWN_KERNEL if args.own_db else 0))
     torch.cuda.synchronize()
 
     def barrier():
@@ -777,7 +781,8 @@ def main():
     # by the library's stage events inside the soaked, instrumented pass above, so the matching peak is the SUSTAINED one.
     peaks = measured_peaks()
     t_big = sum(ms for name, ms in records if name in ("gemm_fwd", "gemm_dx"))
-    f_big = args.steps * sum(2.0 * T * n * (m + r) + 2.0 * T * m * n for _, n, m in linears)
+    db_rides = not any(name == "gemm_db" for name, _ in records)      # the adapter gradient ran inside the dX launches
+    f_big = args.steps * sum(2.0 * T * n * (m + r) + 2.0 * T * m * n + (2.0 * T * m * r if db_rides else 0.0) for _, n, m in linears)
     launches_big = sum(1 for name, _ in records if name in ("gemm_fwd", "gemm_dx"))
     achieved = f_big / (t_big * 1e-3) / 1e12 if t_big > 0 else 0.0
     peak = peaks["bf16_sustained"] * FP8_OVER_BF16
@@ -831,6 +836,12 @@ def main():
           "achieved_gbs": db_bytes / (t_db * 1e-3) / 1e9 if t_db > 0 else 0.0, "peak_gbs": peaks["hbm"],
           "note": "reads g~ (T m bytes, written just before and largely still in L2) and O~_A, writes dB"}
     db["frac"] = db["achieved_gbs"] / peaks["hbm"]
+    if db_rides:
+        db = {"bound": "hbm", "kernel": "gemm_fp8_pair_kernel (rider of the input-gradient product)", "bytes_per_step": db_bytes,
+              "ms_per_step": None, "achieved_gbs": None, "peak_gbs": peaks["hbm"], "frac": None,
+              "note": "dB is computed inside the launch of the input-gradient product, on the SM pairs its last wave of tiles leaves "
+                      "idle: it has no launch and no duration of its own (its flops are counted in that kernel's roofline entry); "
+                      "--own-db runs and times it as a kernel of its own"}
     t_proxy = breakdown.get("sgd_score", 0.0) + breakdown.get("merge", 0.0)
     proxy_bytes = sum(12.0 * m * r + 4.0 * m + k * (2.0 * n + 8.0 * r) + r * n for _, n, m in linears)
     proxy = {"bound": "hbm for the optimizer pass, fp32 ALU for the merge at this rank", "bytes_per_step": proxy_bytes,
@@ -862,7 +873,8 @@ def main():
     e2e_value = world * flops_step / (ms_e2e * 1e-3) / 1e12
 
     suffix = ":fused" if args.fused else ""
-    launches_per_step = sum(fq.launch_count("falqon_melded_forward" + suffix) + fq.launch_count("falqon_melded_backward" + suffix) +
+    bsuffix = suffix if args.fused else (":own_db" if (cfg.get("per_row", False) or args.own_db) else "")
+    launches_per_step = sum(fq.launch_count("falqon_melded_forward" + suffix) + fq.launch_count("falqon_melded_backward" + bsuffix) +
                             (fq.launch_count("falqon_proxy_update", k=k) if batch is None else 0) for L in layers)
     if batch is not None:
         launches_per_step += fq.launch_count("falqon_proxy_update_batched", k=k) * ((len(layers) + 7) // 8)

@@ -94,8 +94,13 @@ typedef struct {
  *      kernel can run -- bf16 inputs; forward: (m + r) a multiple of 16; backward: per-tensor s_w and dX requested -- and
  *      silently falls back to the un-fused path elsewhere.  FALQON_WS_XQ holds no codes after a fused forward.
  *  FALQON_LAYER_EMIT_XQ     With FALQON_LAYER_FUSED_CAST: the fused forward also writes x~ to FALQON_WS_XQ (one extra
- *      write of T*n bytes), for layers that share it through falqon_melded_forward_codes. */
-typedef enum { FALQON_LAYER_FUSED_CAST = 1, FALQON_LAYER_EMIT_XQ = 2 } falqon_layer_flag;
+ *      write of T*n bytes), for layers that share it through falqon_melded_forward_codes.
+ *  FALQON_LAYER_DB_OWN_KERNEL  By default the adapter gradient (Eq. lora_backward_modified) of a per-tensor-scaled layer
+ *      whose dX is requested is computed inside the launch of the input-gradient product, on the SM pairs that the product's
+ *      last wave of tiles leaves idle: one accumulation over all tokens per element, in token order.  With this flag (and
+ *      always for per-row-scaled layers, for calls without dX and for falqon_melded_backward_update) dB is a kernel of its own
+ *      that sums four token slabs in slab order.  Both are deterministic; they differ in the last bits of dB. */
+typedef enum { FALQON_LAYER_FUSED_CAST = 1, FALQON_LAYER_EMIT_XQ = 2, FALQON_LAYER_DB_OWN_KERNEL = 4 } falqon_layer_flag;
 
 /* Names of the regions inside the workspace that hold staged intermediates of the last call
  * (readable by a caller that wants to inspect or reuse them; see falqon_workspace_region). */
@@ -461,7 +466,8 @@ int falqon_profile_start(int max_records, unsigned stage_mask);
 int falqon_profile_stop(float *ms_out, int *stage_out, int capacity);
 
 /* Host, pure.  Number of kernels the named call launches for this shape (for launch accounting).  The forward and
- * backward of a layer with FALQON_LAYER_FUSED_CAST are named "falqon_melded_forward:fused" / "falqon_melded_backward:fused". */
+ * backward of a layer with FALQON_LAYER_FUSED_CAST are named "falqon_melded_forward:fused" / "falqon_melded_backward:fused",
+ * a backward whose dB is a kernel of its own (see FALQON_LAYER_DB_OWN_KERNEL) "falqon_melded_backward:own_db". */
 int falqon_launch_count(const char *entry_point, int64_t m, int64_t n, int64_t r, int64_t T, int64_t k);
 
 #ifdef __cplusplus

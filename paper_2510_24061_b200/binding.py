@@ -18,7 +18,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, 
 E4M3, E5M2 = 0, 1
 BF16, F32 = 0, 1
 PER_TENSOR, PER_ROW = 0, 1
-LAYER_FUSED_CAST, LAYER_EMIT_XQ = 1, 2
+LAYER_FUSED_CAST, LAYER_EMIT_XQ, LAYER_DB_OWN_KERNEL = 1, 2, 4
 WS_XQ, WS_GQ, WS_OAQ_T, WS_SCALES, WS_SCORE = range(5)
 
 EXPORTS = ["falqon_absmax", "falqon_selftest_wait_timeout", "falqon_workspace_bytes", "falqon_workspace_region", "falqon_quantize", "falqon_melded_forward",
@@ -178,7 +178,8 @@ class Layer:
 
     @flags.setter
     def flags(self, value: int):
-        """falqon_layer.flags: LAYER_FUSED_CAST moves the casts of X and dY into the products' producers."""
+        """falqon_layer.flags: LAYER_FUSED_CAST moves the casts of X and dY into the products' producers; LAYER_DB_OWN_KERNEL
+        keeps the adapter gradient out of the input-gradient product's launch."""
         self.c.flags = int(value)
 
     def workspace(self, T: int) -> torch.Tensor:

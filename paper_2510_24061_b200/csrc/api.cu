@@ -79,7 +79,7 @@ inline bool dtype_ok(int dt) { return dt == FALQON_BF16 || dt == FALQON_F32; }
 bool layer_ok(const falqon_layer* L) {
   return L != nullptr && shape_ok(L->m, L->n, L->r) && L->wq != nullptr && L->s_w != nullptr && L->dbuf != nullptr &&
          aligned16(L->wq) && aligned16(L->dbuf) && (L->gran == FALQON_PER_TENSOR || L->gran == FALQON_PER_ROW) &&
-         (L->flags & ~(FALQON_LAYER_FUSED_CAST | FALQON_LAYER_EMIT_XQ)) == 0;
+         (L->flags & ~(FALQON_LAYER_FUSED_CAST | FALQON_LAYER_EMIT_XQ | FALQON_LAYER_DB_OWN_KERNEL)) == 0;
 }
 
 #define FALQON_CUDA(expr)                                   \
@@ -315,6 +315,24 @@ namespace {
 // amax_dy (nullable, device [1]; per-tensor layers only): max |dY| is already known, see forward_impl.
 // sgd_lr (nullable, host): also run Alg. 3 line 4 in its plain-SGD form and the row scores (into the workspace's score region),
 // inside the dB kernel where its shared memory has the room, else as the separate pass.
+// S5b and S4 of one backward: dB (d) and, when dX is wanted, the input-gradient product (g).  Where the product runs on
+// CTA pairs and d is the plain adapter gradient, dB rides on the product's launch (the pairs its last wave leaves idle);
+// otherwise -- no dX, a per-row-scaled layer, the optimizer step fused into the dB kernel, FALQON_LAYER_DB_OWN_KERNEL -- dB
+// is a kernel of its own, launched first (g~ was written a moment ago and is still in L2).
+int launch_db_and_dx(const falqon_layer* L, DbFusedProblem& d, GemmProblem* g, cudaStream_t stream) {
+  const bool ride = g != nullptr && (L->flags & FALQON_LAYER_DB_OWN_KERNEL) == 0 && gemm_db_rider_supported(*g, d);
+  if (!ride) {
+    StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
+    FALQON_CUDA(launch_db_fused(d, stream));
+  }
+  if (g != nullptr) {
+    g->db_rider = ride ? &d : nullptr;
+    StageTimer timer(FALQON_STAGE_GEMM_DX, stream);
+    FALQON_CUDA(launch_gemm_fp8(*g, stream));
+  }
+  return FALQON_OK;
+}
+
 int backward_impl(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, const float* amax_dy, int64_t T, const float* OA,
                   const float* amax_oa, void* dX, falqon_dtype dx_dt, float* dB, float* s_g_out, void* ws, size_t ws_bytes,
                   falqon_stream stream, int dump_block = -1, const float* sgd_lr = nullptr) {
@@ -396,8 +414,8 @@ int backward_impl(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, con
                                         stream));
     }
   }
-  // S5b: dB = g~^T O~_A / (s_g s_OA) over token slabs, slab sum in slab order across a thread-block cluster.  It runs
-  // before S4 (neither needs the other): g~ was written a moment ago and is still in L2.
+  // S5b: dB = g~^T O~_A / (s_g s_OA), and S4 (neither needs the other): dB rides on S4's launch where it can, and is a
+  // kernel of its own (token slabs, slab sum in slab order across a thread-block cluster) before S4 where it cannot.
   {
     DbFusedProblem d{};
     d.m = m; d.r = r; d.T = T;
@@ -405,17 +423,7 @@ int backward_impl(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, con
     d.s_g = scales + 3; d.row_mul = per_row ? L->s_w : nullptr; d.dB = dB; d.status = status;
     const bool fuse_update = sgd_lr != nullptr && db_fused_update_fits(m, r, T);
     if (fuse_update) { d.dbuf = L->dbuf; d.score = reinterpret_cast<float*>(base + w.score); d.neg_lr = -*sgd_lr; }
-    {
-      StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
-      FALQON_CUDA(launch_db_fused(d, stream));
-    }
-    if (sgd_lr != nullptr && !fuse_update) {
-      StageTimer timer(FALQON_STAGE_SGD_SCORE, stream);
-      FALQON_CUDA(launch_sgd_score(L->dbuf, dB, *sgd_lr, m, r, reinterpret_cast<float*>(base + w.score), stream));
-    }
-  }
-  // S4: dX = g~ W~ / (s_W s_g)   (contraction over the m output channels; W~ read MN-major)
-  if (dX != nullptr) {
+    // S4: dX = g~ W~ / (s_W s_g)   (contraction over the m output channels; W~ read MN-major)
     GemmProblem g{};
     g.M = T; g.N = n; g.K = m;
     g.a = gq; g.lda = m; g.a_fmt = kE5M2;
@@ -426,8 +434,25 @@ int backward_impl(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, con
     g.scale_a = scales + 3; g.scale_b = per_row ? nullptr : L->s_w;
     g.col_scale = nullptr;
     g.status = status;
-    StageTimer timer(FALQON_STAGE_GEMM_DX, stream);
-    FALQON_CUDA(launch_gemm_fp8(g, stream));
+    // with a separate optimizer pass the pass must follow dB: it keeps dB in a kernel of its own, before the product
+    const bool own_db = sgd_lr != nullptr && !fuse_update;
+    if (own_db) {
+      {
+        StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
+        FALQON_CUDA(launch_db_fused(d, stream));
+      }
+      {
+        StageTimer timer(FALQON_STAGE_SGD_SCORE, stream);
+        FALQON_CUDA(launch_sgd_score(L->dbuf, dB, *sgd_lr, m, r, reinterpret_cast<float*>(base + w.score), stream));
+      }
+      if (dX != nullptr) {
+        StageTimer timer(FALQON_STAGE_GEMM_DX, stream);
+        FALQON_CUDA(launch_gemm_fp8(g, stream));
+      }
+    } else {
+      const int rc = launch_db_and_dx(L, d, dX != nullptr ? &g : nullptr, stream);
+      if (rc != FALQON_OK) return rc;
+    }
   }
   return FALQON_OK;
 }
@@ -468,26 +493,18 @@ int falqon_melded_backward_codes(const falqon_layer* L, const uint8_t* gq, const
     const OaCastJob oa_cast{OA, amax_oa, T, static_cast<int>(r), w.t16, oaq_t, scales + 5, scales + 4};
     FALQON_CUDA(launch_oa_cast(oa_cast, stream));
   }
-  {
-    DbFusedProblem d{};
-    d.m = m; d.r = r; d.T = T;
-    d.gq = gq; d.oaq_t = oaq_t; d.ldt = w.t16; d.s_oa = scales + 5; d.s_g = s_g; d.dB = dB; d.status = status;
-    StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
-    FALQON_CUDA(launch_db_fused(d, stream));
-  }
-  if (dX != nullptr) {
-    GemmProblem g{};
-    g.M = T; g.N = n; g.K = m;
-    g.a = gq; g.lda = m; g.a_fmt = kE5M2;
-    g.b = L->wq; g.ldb = n; g.b_mn_major = true; g.b_fmt = kE4M3;
-    g.block_n = 256;
-    g.c0 = dX; g.ldc0 = n; g.c0_dt = dx_dt; g.n_split = n;
-    g.scale_a = s_g; g.scale_b = L->s_w;
-    g.status = status;
-    StageTimer timer(FALQON_STAGE_GEMM_DX, stream);
-    FALQON_CUDA(launch_gemm_fp8(g, stream));
-  }
-  return FALQON_OK;
+  DbFusedProblem d{};
+  d.m = m; d.r = r; d.T = T;
+  d.gq = gq; d.oaq_t = oaq_t; d.ldt = w.t16; d.s_oa = scales + 5; d.s_g = s_g; d.dB = dB; d.status = status;
+  GemmProblem g{};
+  g.M = T; g.N = n; g.K = m;
+  g.a = gq; g.lda = m; g.a_fmt = kE5M2;
+  g.b = L->wq; g.ldb = n; g.b_mn_major = true; g.b_fmt = kE4M3;
+  g.block_n = 256;
+  g.c0 = dX; g.ldc0 = n; g.c0_dt = dx_dt; g.n_split = n;
+  g.scale_a = s_g; g.scale_b = L->s_w;
+  g.status = status;
+  return launch_db_and_dx(L, d, dX != nullptr ? &g : nullptr, stream);
 }
 
 int falqon_melded_backward_dx(const falqon_layer* L, int64_t T, void* dX, falqon_dtype dx_dt, void* ws, size_t ws_bytes,
@@ -879,7 +896,10 @@ int falqon_launch_count(const char* entry_point, int64_t m, int64_t n, int64_t r
   if (entry_point == nullptr) return 0;
   if (std::strcmp(entry_point, "falqon_quantize") == 0) return 2;           // absmax, cast
   if (std::strcmp(entry_point, "falqon_melded_forward") == 0) return 2;     // fused quantize, GEMM
-  if (std::strcmp(entry_point, "falqon_melded_backward") == 0) return 3;    // fused quantize, dX, fused dB
+  // fused quantize (the O_A cast rides on it), dX product (dB rides on it); dB as a kernel of its own where it cannot ride:
+  // per-row-scaled layers, no dX requested, FALQON_LAYER_DB_OWN_KERNEL
+  if (std::strcmp(entry_point, "falqon_melded_backward") == 0) return 2;
+  if (std::strcmp(entry_point, "falqon_melded_backward:own_db") == 0) return 3;
   // with FALQON_LAYER_FUSED_CAST: absmax, scale, product / absmax, scale, O_A cast, dX product (casts dY, writes g~), dB
   if (std::strcmp(entry_point, "falqon_melded_forward:fused") == 0) return 3;
   if (std::strcmp(entry_point, "falqon_melded_backward:fused") == 0) return 5;

@@ -197,10 +197,19 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 // A is K-major; B is K-major or MN-major.  The last N tile is issued with a narrower instruction N.
 constexpr uint32_t kPairStageBytes = kATileBytes + 128 * kBlockKBytes;   // 32 KB per CTA per stage
 
-template <bool kBMn>
+//
+// kRider (the input-gradient product only): the adapter gradient dB = g~^T O~_A / (s_g s_OA) rides on the same launch.
+// Its A operand is the product's own A tensor g~ [T][m], read through the same tensor map with the coordinates swapped
+// (a box of 128 tokens x 128 bytes of m is an MN-major A tile whose M runs over m and whose K runs over the tokens);
+// its B operand is O~_A^T [r16][T], K-major.  One pair tile covers 256 rows of dB and ALL tokens, so no partial
+// sums exist and the order of the accumulation is fixed.  The tiles of dB are appended to the tile list from the
+// far end of the pairs: the last wave of 256 x 256 tiles leaves the highest-numbered pairs idle, and that is where
+// the few microseconds of dB work go -- the launch of a separate kernel (TMEM allocation, two cluster barriers,
+// about 12 us for 2 us of traffic) disappears from the step.  pd: the parameter block of that second problem.
+template <bool kBMn, bool kRider>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                     const GemmParams p) {
+                     const __grid_constant__ CUtensorMap tmap_c, const GemmParams p, const GemmParams pd) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t smem_base = (raw_addr + 1023u) & ~1023u;
@@ -223,6 +232,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   if (threadIdx.x == 0) {
     prefetch_tensor_map(&tmap_a);
     prefetch_tensor_map(&tmap_b);
+    if (kRider) prefetch_tensor_map(&tmap_c);
     for (int s = 0; s < S; ++s) {
       mbar_init(full_bar(s), 1);      // the leader's arrive.expect_tx; bytes from both CTAs
       mbar_init(empty_bar(s), 1);     // one multicast commit
@@ -250,6 +260,11 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   const int pair = blockIdx.x >> 1;
   const int total_tiles = p.m_tiles * p.n_tiles;   // m_tiles counts 256-row pair tiles here
   bool aborted = false;
+  // rider: the pairs without a tile in the product's last wave (the highest-numbered ones) share the tiles of dB among
+  // themselves, round robin from the far end; the others take none
+  const int last_wave = total_tiles % num_pairs;
+  const int rider_step = last_wave == 0 ? num_pairs : num_pairs - last_wave;             // number of such pairs
+  const int rider_first = (num_pairs - 1 - pair) < rider_step ? (num_pairs - 1 - pair) : 0x7FFFFFF0;   // this pair's first dB tile
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (warp 0 of each CTA; one lane issues)
@@ -275,6 +290,25 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         }
         __syncwarp();
         if (++stage == S) { stage = 0; phase ^= 1u; }
+      }
+    }
+    if (kRider) {   // the tiles of dB, from the far end of the pairs
+      const int half_rows = pd.block_n >> 1;                                  // this CTA's rows of O~_A^T (block_n = r16)
+      const uint32_t rider_bytes = kATileBytes + static_cast<uint32_t>(half_rows) * kBlockKBytes;
+      for (int j = rider_first; j < pd.m_tiles && !aborted; j += rider_step) {
+        const int mcol0 = j * 256 + static_cast<int>(rank) * kBlockM;        // first of this CTA's 128 rows of dB
+        for (int kb = 0; kb < pd.kblocks_total; ++kb) {
+          if (!mbar_wait_warp(empty_bar(stage), phase ^ 1u, p.status)) { aborted = true; break; }
+          if (elect_one()) {
+            if (leader) mbar_expect_tx(full_bar(stage), 2 * rider_bytes);
+            const uint32_t fb = map_to_cta(full_bar(stage), 0);
+            const uint32_t a_dst = smem_base + static_cast<uint32_t>(stage) * kPairStageBytes;
+            tma_load_2d_pair(a_dst, &tmap_a, fb, mcol0, kb * kBlockKBytes);                               // 128 tokens x 128 B of m
+            tma_load_2d_pair(a_dst + kATileBytes, &tmap_c, fb, kb * kBlockKBytes, static_cast<int>(rank) * half_rows);
+          }
+          __syncwarp();
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
       }
     }
     // tail: wait until the MMAs have released every stage, so no completion signal can arrive at a CTA
@@ -324,6 +358,36 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
+      if (kRider) {
+        const uint64_t ra_desc0 = make_smem_desc(smem_base, kATileBytes, 1024);          // MN-major: one 128 x 128 chunk
+        const uint64_t rb_desc0 = make_smem_desc(smem_base + kATileBytes, 16, 1024);     // K-major
+        constexpr uint32_t kRaStep = (kUmmaK * 128) >> 4;   // 32 tokens further down the tile
+        constexpr uint32_t kRbStep = kUmmaK >> 4;
+        for (int j = rider_first; j < pd.m_tiles && !aborted; j += rider_step) {
+          if (!mbar_wait_warp(tmem_empty_bar(acc), acc_phase ^ 1u, p.status)) { aborted = true; break; }
+          tc_fence_after_sync();
+          const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * kAccCols;
+          for (int kb = 0; kb < pd.kblocks_total; ++kb) {
+            if (!mbar_wait_warp(full_bar(stage), phase, p.status)) { aborted = true; break; }
+            tc_fence_after_sync();
+            const uint32_t stage_off = (static_cast<uint32_t>(stage) * kPairStageBytes) >> 4;
+            if (elect_one()) {
+#pragma unroll
+              for (int k = 0; k < kBlockKBytes / kUmmaK; ++k)
+                umma_f8_pair(d_tmem, ra_desc0 + stage_off + k * kRaStep, rb_desc0 + stage_off + k * kRbStep, pd.idesc,
+                             (kb > 0 || k > 0) ? 1u : 0u);
+              umma_commit_pair(empty_bar(stage), 3);
+            }
+            __syncwarp();
+            if (++stage == S) { stage = 0; phase ^= 1u; }
+          }
+          if (aborted) break;
+          if (elect_one()) umma_commit_pair(tmem_full_bar(acc), 3);
+          __syncwarp();
+          acc ^= 1;
+          if (acc == 0) acc_phase ^= 1u;
+        }
+      }
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..9 of each CTA)
@@ -350,6 +414,22 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       if (lane == 0) mbar_arrive_cluster(map_to_cta(tmem_empty_bar(acc), 0));
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
+    }
+    if (kRider) {
+      const float inv_db = 1.0f / (ld_stream(pd.scale_a) * ld_stream(pd.scale_b));
+      uint32_t unused = 0;
+      for (int j = rider_first; j < pd.m_tiles && !aborted; j += rider_step) {
+        if (!mbar_wait(tmem_full_bar(acc), acc_phase, p.status)) { aborted = true; break; }
+        tc_fence_after_sync();
+        const int row = j * 256 + static_cast<int>(rank) * kBlockM + quad * 32 + lane;      // row of dB
+        const uint32_t t_row = tmem_base + static_cast<uint32_t>(acc) * kAccCols + (static_cast<uint32_t>(quad * 32) << 16);
+        epilogue_tile(pd, t_row, row, row < pd.M, 0, col_half ? 128 : 0, col_half ? 256 : 128, inv_db, unused, stage_out);
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(map_to_cta(tmem_empty_bar(acc), 0));
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
     }
     if (p.amax1_bits != nullptr) {
       amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
@@ -448,16 +528,16 @@ cudaError_t launch_variant(const CUtensorMap& ta, const CUtensorMap& tb, const G
                     tb, gp);
 }
 
-template <bool kBMn>
-cudaError_t launch_pair_variant(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& gp, int grid, size_t smem,
-                                cudaStream_t stream) {
+template <bool kBMn, bool kRider>
+cudaError_t launch_pair_variant(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const GemmParams& gp,
+                                const GemmParams& gd, int grid, size_t smem, cudaStream_t stream) {
   static DeviceMask configured{0};
   {
-    const cudaError_t ec = set_max_dynamic_smem(gemm_fp8_pair_kernel<kBMn>, static_cast<int>(kSmemBudget), configured);
+    const cudaError_t ec = set_max_dynamic_smem(gemm_fp8_pair_kernel<kBMn, kRider>, static_cast<int>(kSmemBudget), configured);
     if (ec != cudaSuccess) return ec;
   }
-  return launch_pdl(gemm_fp8_pair_kernel<kBMn>, dim3(static_cast<unsigned>(grid)), dim3(kGemmThreads), smem, stream, 2, ta, tb,
-                    gp);
+  return launch_pdl(gemm_fp8_pair_kernel<kBMn, kRider>, dim3(static_cast<unsigned>(grid)), dim3(kGemmThreads), smem, stream, 2,
+                    ta, tb, tc, gp, gd);
 }
 
 bool pair_kernel_disabled() {
@@ -496,14 +576,46 @@ cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
   if (total_tiles < pairs) pairs = total_tiles;
   const int grid = static_cast<int>(pairs * 2);
   const size_t smem = static_cast<size_t>(stages) * kPairStageBytes + kBarrierBytes + kStagingBytes + 1024;
-  if (q.b_mn_major) return launch_pair_variant<true>(ta, tb, gp, grid, smem, stream);
-  return launch_pair_variant<false>(ta, tb, gp, grid, smem, stream);
+  if (q.db_rider != nullptr) {
+    // the adapter gradient as a second problem of the same launch: dB[m][r] = A^T (this product's A, g~ [T][m]) x O~_A^T
+    const DbFusedProblem& d = *q.db_rider;
+    if (!gemm_db_rider_supported(q, d)) return cudaErrorInvalidValue;
+    const int r16 = static_cast<int>(round_up(d.r, 16));
+    GemmParams gd{};
+    gd.M = static_cast<int>(d.m); gd.N = static_cast<int>(d.r); gd.K = static_cast<int>(d.T);
+    gd.block_n = r16;
+    gd.m_tiles = static_cast<int>((d.m + 255) / 256);
+    gd.n_tiles = 1;
+    gd.kblocks_total = static_cast<int>((d.T + kBlockKBytes - 1) / kBlockKBytes);
+    gd.num_stages = stages;
+    // fp32 accumulate, A = the product's own A format read MN-major, B = E4M3 K-major, N = r16, M = 256
+    gd.idesc = (1u << 4) | (static_cast<uint32_t>(q.a_fmt) << 7) | (static_cast<uint32_t>(kE4M3) << 10) | (1u << 15) |
+               (static_cast<uint32_t>(r16 >> 3) << 17) | (static_cast<uint32_t>(256 >> 4) << 24);
+    gd.c0 = d.dB; gd.ldc0 = d.r; gd.c0_dt = kF32; gd.n_split = static_cast<int>(d.r);
+    gd.scale_a = d.s_g; gd.scale_b = d.s_oa;
+    gd.status = q.status;
+    CUtensorMap tc;
+    if (!make_tensor_map(&tc, d.oaq_t, r16, d.T, d.ldt, kBlockKBytes, static_cast<uint32_t>(r16 / 2))) return cudaErrorInvalidValue;
+    return launch_pair_variant<true, true>(ta, tb, tc, gp, gd, grid, smem, stream);
+  }
+  if (q.b_mn_major) return launch_pair_variant<true, false>(ta, tb, ta, gp, gp, grid, smem, stream);
+  return launch_pair_variant<false, false>(ta, tb, ta, gp, gp, grid, smem, stream);
 }
 
 }  // namespace
 
+bool gemm_db_rider_supported(const GemmProblem& q, const DbFusedProblem& d) {
+  // the product must run on CTA pairs with an MN-major B (the input-gradient product), its A must be the rider's g~
+  // ([T][m], the rider's rows on the product's contraction axis), and the rider must be the plain form of dB
+  return q.block_n == 256 && q.N % 16 == 0 && !pair_kernel_disabled() && q.b_mn_major && q.a != nullptr && q.a == d.gq &&
+         q.M == d.T && q.K == d.m && q.lda == d.m && d.m % 16 == 0 && d.r >= 8 && d.r <= 256 && d.r % 8 == 0 && d.dB != nullptr &&
+         d.row_mul == nullptr && d.dbuf == nullptr && d.score == nullptr && d.oaq_t != nullptr && d.s_g != nullptr &&
+         d.s_oa != nullptr && (q.a_fmt == kE5M2) == !d.g_is_e4m3;
+}
+
 cudaError_t launch_gemm_fp8(const GemmProblem& q, cudaStream_t stream) {
   if (q.M <= 0 || q.N <= 0 || q.K <= 0) return cudaErrorInvalidValue;
+  if (q.db_rider != nullptr && !gemm_db_rider_supported(q, *q.db_rider)) return cudaErrorInvalidValue;
   if (q.block_n < 16 || q.block_n > 256 || q.block_n % 16) return cudaErrorInvalidValue;
   if (q.b_mn_major && q.block_n % 128) return cudaErrorInvalidValue;
   // the tensor-bound roles (K-major A, full-width tiles, no token slabs) run on CTA pairs

@@ -119,6 +119,7 @@ cudaError_t launch_quantize_per_row(const void* src, int src_dt, int64_t rows, i
                                     cudaStream_t stream);
 
 // ---- gemm_fp8.cu
+struct DbFusedProblem;
 struct GemmProblem {
   // D[M][N] = A[M][K] * B[N][K]^T with fp32 accumulation on tcgen05
   int64_t M, N, K;
@@ -131,8 +132,14 @@ struct GemmProblem {
   const float* scale_a; const float* scale_b;  // device scalars; output *= 1/(sa*sb); scale_b null: 1/sa; both null: none
   const float* col_scale;                      // nullable: per-column factors (N rounded up to 32 entries) instead
   int* status;
+  // nullable: the adapter gradient of the same layer, computed by the same launch on the CTA pairs that the last wave of
+  // this product's tiles leaves idle (see gemm_db_rider_supported)
+  const DbFusedProblem* db_rider;
 };
 cudaError_t launch_gemm_fp8(const GemmProblem& p, cudaStream_t stream);
+// Whether launch_gemm_fp8 can carry d as p.db_rider: p is an input-gradient product on CTA pairs whose A operand is d's
+// g~, and d is the plain adapter gradient (no row factors, no fused optimizer step).
+bool gemm_db_rider_supported(const GemmProblem& p, const DbFusedProblem& d);
 
 // ---- gemm_fp8_fused.cu: the same product on CTA pairs with the cast of the A operand fused into the producer.  A arrives
 // as bf16 [M][lda16]; converter warps scale it by *a_scale (the scale of Eq. quantize, already on the device) and

@@ -205,7 +205,7 @@ class Stack:
 
     def __init__(self, n_layers: int, H: int, F: int, T: int, r: int, k: int, seed: int, device, lr: float = 2e-4,
                  producer_amax: bool = True, batched_proxy: bool = True, adamw: dict | None = None, fuse_chain: bool = True,
-                 fuse_cast: bool | None = None):
+                 fuse_cast: bool | None = None, layer_flags: int = 0):
         """producer_amax: the chain kernels hand the absmax of their outputs to the layers that consume them, whose
         input casts are then single-pass (False: every layer takes the absmax of its input itself).
         batched_proxy: the seven proxy updates of a block run as one falqon_proxy_update_batched call at the end of
@@ -214,6 +214,7 @@ class Stack:
         fuse_cast: every tensor a layer consumes (x1, a, x2, z and the output gradients) leaves the chain kernel that
         produces it as FP8 codes (the *_quantize calls above): no separate cast kernel runs, the layers take codes
         (falqon_melded_forward_codes / falqon_melded_backward_codes).  Same codes, so the same results bit for bit.
+        layer_flags: falqon_layer.flags of every layer (binding.LAYER_*).
         adamw: None for the plain SGD step with lr, or the hyper-parameters (beta1, beta2, eps, weight_decay; lr is the
         argument above) of AdamW on every DeltaBuffer -- the optimizer the paper trains with; needs batched_proxy."""
         self.n_layers, self.H, self.F, self.T, self.r, self.k, self.lr = n_layers, H, F, T, r, k, lr
@@ -224,6 +225,7 @@ class Stack:
         if fuse_cast is None:               # the default wherever it applies
             fuse_cast = fuse_chain and producer_amax
         self.fuse_cast = fuse_cast
+        self.own_db = (layer_flags & fq.LAYER_DB_OWN_KERNEL) != 0
         assert not fuse_cast or (fuse_chain and producer_amax)
         self.device = torch.device(device)
         self.seed = seed
@@ -238,6 +240,7 @@ class Stack:
                 A = synth.adapter_a(seed, mat, r, n, self.device)
                 B = synth.adapter_b(seed, mat, m, r, self.device)
                 block[name] = fq.setup_layer(W, A, B, 1.0)
+                block[name].flags = layer_flags
                 del W, A, B
             self.layers.append(block)
         dev, bf = self.device, torch.bfloat16
@@ -493,10 +496,10 @@ class Stack:
 
     def launches_per_step(self) -> int:
         if self.fuse_cast:
-            # per block: 7 forward products; 7 x (O_A cast, dB, dX) + the two single-pass casts of dg and du; 4 + 5 chain
-            # kernels; the proxy update(s); plus the first block's normalisation (the last block's plain residual sum stands
-            # in for a quantizing one)
-            per_block = 7 + 7 * 3 + 2 + 4 + 5
+            # per block: 7 forward products; 7 x (O_A cast, dX product with dB riding on it) + the two single-pass casts of
+            # dg and du; 4 + 5 chain kernels; the proxy update(s); plus the first block's normalisation (the last block's
+            # plain residual sum stands in for a quantizing one)
+            per_block = 7 + 7 * (3 if self.own_db else 2) + 2 + 4 + 5
             if self.batches is None:
                 per_block += 7 * fq.launch_count("falqon_proxy_update", k=self.k)
             else:
@@ -507,9 +510,9 @@ class Stack:
             shared = name in ("k", "v", "up")
             per_block += (1 if shared else fq.launch_count("falqon_melded_forward"))   # codes: the product alone
             if name in ("k", "v"):
-                per_block += 3                                  # on q's gradient codes: O_A cast, dB, dX
+                per_block += 3 if self.own_db else 2            # on q's gradient codes: O_A cast, dX (dB rides on it)
             else:
-                per_block += fq.launch_count("falqon_melded_backward") + (1 if self.producer_amax else 0)   # + the O_A cast
+                per_block += fq.launch_count("falqon_melded_backward" + (":own_db" if self.own_db else "")) + (1 if self.producer_amax else 0)   # + the O_A cast
             if self.batches is None:
                 per_block += fq.launch_count("falqon_proxy_update", k=self.k)
         if self.batches is not None:

@@ -133,7 +133,8 @@ def test_bad_arguments_are_rejected_on_the_host(fq):
 
 def test_launch_counts(fq):
     assert fq.launch_count("falqon_melded_forward") == 2
-    assert fq.launch_count("falqon_melded_backward") == 3      # quantize, dX, fused dB
+    assert fq.launch_count("falqon_melded_backward") == 2      # quantize (O_A cast riding), dX (dB riding)
+    assert fq.launch_count("falqon_melded_backward:own_db") == 3
     assert fq.launch_count("falqon_proxy_update", k=4) == 2 and fq.launch_count("falqon_proxy_update", k=0) == 1
     assert fq.launch_count("falqon_proxy_update_batched", k=4) == 2 and fq.launch_count("falqon_proxy_update_batched", k=0) == 1
     assert fq.launch_count("nope") == 0
@@ -181,7 +182,7 @@ int main(void) {
     out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
     assert int(out[0]) == fq.workspace_bytes(4096, 4096, 64, 4096) and int(out[0]) > 4096 * 4096
     assert int(out[1]) == fq.OK and int(out[2]) == 4096 * 4096
-    assert int(out[3]) == fq.ERR_INVALID_ARG and int(out[4]) == 3
+    assert int(out[3]) == fq.ERR_INVALID_ARG and int(out[4]) == 2
 
 
 def test_the_package_refuses_to_load_without_its_library(tmp_path):

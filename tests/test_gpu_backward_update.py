@@ -32,6 +32,7 @@ def test_backward_update_and_scored_proxy_update(m, n, r, T, k, per_row, lr):
         W = synth.backbone(41, 1, m, n, DEV, heavy_tailed=True)
     dY = synth.out_grad(41, 1, 0, T, m, DEV)
     ref = fq.setup_layer(W, A, B, 1.0, per_row=per_row)
+    ref.flags = fq.LAYER_DB_OWN_KERNEL      # the fused step lives in the adapter-gradient kernel: the reference uses that kernel too
     ref.dbuf.copy_(synth.normal_bf16(41, 90, (m, r), 1e-3, DEV).float())      # something for the step to accumulate onto
     new = _twin(fq, ref)
     ws_r, ws_n = ref.workspace(T), new.workspace(T)

@@ -50,6 +50,7 @@ def test_fused_forward_and_backward_match_unfused_and_oracle_codes(fq, orc, m, n
     W, A, B, X = layer_inputs(11, 2, m, n, r, T, outl, DEV)
     dY = synth.out_grad(11, 2, 0, T, m, DEV)
     plain = fq.setup_layer(W, A, B, 1.0)
+    plain.flags = fq.LAYER_DB_OWN_KERNEL    # the fused backward runs dB as a kernel of its own: the reference does the same
     fused = _twin(fq, plain, fq.LAYER_FUSED_CAST)
     ws = plain.workspace(T)
 

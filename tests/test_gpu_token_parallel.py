@@ -72,6 +72,7 @@ def test_split_backward_and_overlapped_step_equal_the_single_call():
     W, A, B, X = layer_inputs(32, 0, m, n, r, T, 5, DEV)
     dY = synth.out_grad(32, 0, 0, T, m, DEV)
     base = fq.setup_layer(W, A, B, 1.0)
+    base.flags = fq.LAYER_DB_OWN_KERNEL     # the split backward computes dB by itself: the single call shall use the same kernel
     ws = base.workspace(T)
     Y, OA, amax_oa, _ = fq.melded_forward(base, X, y_dtype=torch.float32, ws=ws)
     dX0, dB0, _ = fq.melded_backward(base, dY, OA, amax_oa, dx_dtype=torch.float32, ws=ws)
@@ -88,7 +89,7 @@ def test_split_backward_and_overlapped_step_equal_the_single_call():
 
     results = []
     for overlap in (False, True):
-        rep = fq.Layer(base.wq.clone(), base.s_w.clone(), base.dbuf.clone(), r)
+        rep = fq.Layer(base.wq.clone(), base.s_w.clone(), base.dbuf.clone(), r, flags=fq.LAYER_DB_OWN_KERNEL)
         ts = TokenShardedLayer(rep, comm=OneRank())
         out = ts.step(X, dY, lr, k, y_dtype=torch.float32, dx_dtype=torch.float32, overlap=overlap)
         torch.cuda.synchronize()
