@@ -873,8 +873,10 @@ def main():
     e2e_value = world * flops_step / (ms_e2e * 1e-3) / 1e12
 
     suffix = ":fused" if args.fused else ""
-    bsuffix = suffix if args.fused else (":own_db" if (cfg.get("per_row", False) or args.own_db) else "")
+    bsuffix = suffix if args.fused else (":own_db" if args.own_db else "")
+    table_launches = 2 if cfg.get("per_row", False) else 0      # per-row-scaled layers: one small table of scale factors per call
     launches_per_step = sum(fq.launch_count("falqon_melded_forward" + suffix) + fq.launch_count("falqon_melded_backward" + bsuffix) +
+                            table_launches +
                             (fq.launch_count("falqon_proxy_update", k=k) if batch is None else 0) for L in layers)
     if batch is not None:
         launches_per_step += fq.launch_count("falqon_proxy_update_batched", k=k) * ((len(layers) + 7) // 8)

@@ -95,11 +95,11 @@ typedef struct {
  *      silently falls back to the un-fused path elsewhere.  FALQON_WS_XQ holds no codes after a fused forward.
  *  FALQON_LAYER_EMIT_XQ     With FALQON_LAYER_FUSED_CAST: the fused forward also writes x~ to FALQON_WS_XQ (one extra
  *      write of T*n bytes), for layers that share it through falqon_melded_forward_codes.
- *  FALQON_LAYER_DB_OWN_KERNEL  By default the adapter gradient (Eq. lora_backward_modified) of a per-tensor-scaled layer
- *      whose dX is requested is computed inside the launch of the input-gradient product, on the SM pairs that the product's
- *      last wave of tiles leaves idle: one accumulation over all tokens per element, in token order.  With this flag (and
- *      always for per-row-scaled layers, for calls without dX and for falqon_melded_backward_update) dB is a kernel of its own
- *      that sums four token slabs in slab order.  Both are deterministic; they differ in the last bits of dB. */
+ *  FALQON_LAYER_DB_OWN_KERNEL  By default the adapter gradient (Eq. lora_backward_modified) of a call whose dX is
+ *      requested is computed inside the launch of the input-gradient product, on the SM pairs that the product's last wave
+ *      of tiles leaves idle: one accumulation over all tokens per element, in token order.  With this flag (and always for
+ *      calls without dX and for falqon_melded_backward_update) dB is a kernel of its own that sums four token slabs in slab
+ *      order.  Both are deterministic; they differ in the last bits of dB. */
 typedef enum { FALQON_LAYER_FUSED_CAST = 1, FALQON_LAYER_EMIT_XQ = 2, FALQON_LAYER_DB_OWN_KERNEL = 4 } falqon_layer_flag;
 
 /* Names of the regions inside the workspace that hold staged intermediates of the last call

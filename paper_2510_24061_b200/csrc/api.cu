@@ -317,8 +317,8 @@ namespace {
 // inside the dB kernel where its shared memory has the room, else as the separate pass.
 // S5b and S4 of one backward: dB (d) and, when dX is wanted, the input-gradient product (g).  Where the product runs on
 // CTA pairs and d is the plain adapter gradient, dB rides on the product's launch (the pairs its last wave leaves idle);
-// otherwise -- no dX, a per-row-scaled layer, the optimizer step fused into the dB kernel, FALQON_LAYER_DB_OWN_KERNEL -- dB
-// is a kernel of its own, launched first (g~ was written a moment ago and is still in L2).
+// otherwise -- no dX, the optimizer step fused into the dB kernel, FALQON_LAYER_DB_OWN_KERNEL -- dB is a kernel of its own,
+// launched first (g~ was written a moment ago and is still in L2).
 int launch_db_and_dx(const falqon_layer* L, DbFusedProblem& d, GemmProblem* g, cudaStream_t stream) {
   const bool ride = g != nullptr && (L->flags & FALQON_LAYER_DB_OWN_KERNEL) == 0 && gemm_db_rider_supported(*g, d);
   if (!ride) {
@@ -897,7 +897,7 @@ int falqon_launch_count(const char* entry_point, int64_t m, int64_t n, int64_t r
   if (std::strcmp(entry_point, "falqon_quantize") == 0) return 2;           // absmax, cast
   if (std::strcmp(entry_point, "falqon_melded_forward") == 0) return 2;     // fused quantize, GEMM
   // fused quantize (the O_A cast rides on it), dX product (dB rides on it); dB as a kernel of its own where it cannot ride:
-  // per-row-scaled layers, no dX requested, FALQON_LAYER_DB_OWN_KERNEL
+  // no dX requested, FALQON_LAYER_DB_OWN_KERNEL
   if (std::strcmp(entry_point, "falqon_melded_backward") == 0) return 2;
   if (std::strcmp(entry_point, "falqon_melded_backward:own_db") == 0) return 3;
   // with FALQON_LAYER_FUSED_CAST: absmax, scale, product / absmax, scale, O_A cast, dX product (casts dY, writes g~), dB

@@ -37,6 +37,7 @@ struct GemmParams {
   float* c1; long long ldc1; uint32_t* amax1_bits;
   const float* scale_a; const float* scale_b;
   const float* col_scale;
+  const float* row_scale;   // nullable, used by the adapter-gradient rider only: output row i is also multiplied by row_scale[i]
   int* status;
 };
 

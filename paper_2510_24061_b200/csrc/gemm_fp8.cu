@@ -423,7 +423,9 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         tc_fence_after_sync();
         const int row = j * 256 + static_cast<int>(rank) * kBlockM + quad * 32 + lane;      // row of dB
         const uint32_t t_row = tmem_base + static_cast<uint32_t>(acc) * kAccCols + (static_cast<uint32_t>(quad * 32) << 16);
-        epilogue_tile(pd, t_row, row, row < pd.M, 0, col_half ? 128 : 0, col_half ? 256 : 128, inv_db, unused, stage_out);
+        // (per-row-scaled backbone: row i of dB is multiplied back by s_w[i], one rounded product of the two factors)
+        const float inv_row = pd.row_scale != nullptr && row < pd.M ? __fmul_rn(inv_db, ld_stream(pd.row_scale + row)) : inv_db;
+        epilogue_tile(pd, t_row, row, row < pd.M, 0, col_half ? 128 : 0, col_half ? 256 : 128, inv_row, unused, stage_out);
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(map_to_cta(tmem_empty_bar(acc), 0));
@@ -592,7 +594,7 @@ cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
     gd.idesc = (1u << 4) | (static_cast<uint32_t>(q.a_fmt) << 7) | (static_cast<uint32_t>(kE4M3) << 10) | (1u << 15) |
                (static_cast<uint32_t>(r16 >> 3) << 17) | (static_cast<uint32_t>(256 >> 4) << 24);
     gd.c0 = d.dB; gd.ldc0 = d.r; gd.c0_dt = kF32; gd.n_split = static_cast<int>(d.r);
-    gd.scale_a = d.s_g; gd.scale_b = d.s_oa;
+    gd.scale_a = d.s_g; gd.scale_b = d.s_oa; gd.row_scale = d.row_mul;
     gd.status = q.status;
     CUtensorMap tc;
     if (!make_tensor_map(&tc, d.oaq_t, r16, d.T, d.ldt, kBlockKBytes, static_cast<uint32_t>(r16 / 2))) return cudaErrorInvalidValue;
@@ -606,10 +608,10 @@ cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
 
 bool gemm_db_rider_supported(const GemmProblem& q, const DbFusedProblem& d) {
   // the product must run on CTA pairs with an MN-major B (the input-gradient product), its A must be the rider's g~
-  // ([T][m], the rider's rows on the product's contraction axis), and the rider must be the plain form of dB
+  // ([T][m], the rider's rows on the product's contraction axis), and the rider must be dB without the fused optimizer step
   return q.block_n == 256 && q.N % 16 == 0 && !pair_kernel_disabled() && q.b_mn_major && q.a != nullptr && q.a == d.gq &&
          q.M == d.T && q.K == d.m && q.lda == d.m && d.m % 16 == 0 && d.r >= 8 && d.r <= 256 && d.r % 8 == 0 && d.dB != nullptr &&
-         d.row_mul == nullptr && d.dbuf == nullptr && d.score == nullptr && d.oaq_t != nullptr && d.s_g != nullptr &&
+         d.dbuf == nullptr && d.score == nullptr && d.oaq_t != nullptr && d.s_g != nullptr &&
          d.s_oa != nullptr && (q.a_fmt == kE5M2) == !d.g_is_e4m3;
 }
 
