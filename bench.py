@@ -760,6 +760,19 @@ def main():
     fq.profile_start(n_records, None)
     ms_step_instrumented, clocks_instrumented = timed(eager_step, args.steps)
     records = fq.profile_stop(n_records)
+    # ---- for reference: the adapter gradient as a kernel of its own (the default runs it inside the dX launch, where it
+    # has no duration of its own): the same instrumented steps with FALQON_LAYER_DB_OWN_KERNEL on every layer
+    own_db_records = []
+    if not args.own_db and not args.fused:
+        for L in layers:
+            L["layer"].flags |= fq.LAYER_DB_OWN_KERNEL
+        for _ in range(3):
+            eager_step()
+        fq.profile_start(n_records, None)
+        timed(eager_step, args.steps)
+        own_db_records = fq.profile_stop(n_records)
+        for L in layers:
+            L["layer"].flags &= ~fq.LAYER_DB_OWN_KERNEL
     status = fq.last_device_status()
     sampler.stop()
 
@@ -837,8 +850,13 @@ def main():
           "note": "reads g~ (T m bytes, written just before and largely still in L2) and O~_A, writes dB"}
     db["frac"] = db["achieved_gbs"] / peaks["hbm"]
     if db_rides:
+        t_own = sum(ms for name, ms in own_db_records if name == "gemm_db") / args.steps
+        t_dx_own = sum(ms for name, ms in own_db_records if name == "gemm_dx") / args.steps
+        own = {"kernel": "db_fused_kernel", "ms_per_step": t_own, "achieved_gbs": db_bytes / (t_own * 1e-3) / 1e9 if t_own > 0 else None,
+               "frac": db_bytes / (t_own * 1e-3) / 1e9 / peaks["hbm"] if t_own > 0 else None,
+               "gemm_dx_ms_per_step_without_rider": t_dx_own, "gemm_dx_ms_per_step_with_rider": breakdown.get("gemm_dx", 0.0)}
         db = {"bound": "hbm", "kernel": "gemm_fp8_pair_kernel (rider of the input-gradient product)", "bytes_per_step": db_bytes,
-              "ms_per_step": None, "achieved_gbs": None, "peak_gbs": peaks["hbm"], "frac": None,
+              "ms_per_step": None, "achieved_gbs": None, "peak_gbs": peaks["hbm"], "frac": None, "as_a_kernel_of_its_own": own,
               "note": "dB is computed inside the launch of the input-gradient product, on the SM pairs its last wave of tiles leaves "
                       "idle: it has no launch and no duration of its own (its flops are counted in that kernel's roofline entry); "
                       "--own-db runs and times it as a kernel of its own"}

@@ -43,7 +43,9 @@ def test_default_line_has_the_contract_keys():
     assert b["steps"] == 20 and abs(b["value"] - flops / (b["ms_per_step"] * 1e-3) / 1e12) < 1e-6 * b["value"] and "clocks" in b
     assert b["ms_per_step"] <= d["ms_per_step"] * 1.05          # a cold board is not slower than one at its power cap
     # the HBM-bound stages: achieved = stated bytes / stated time, fraction of the measured copy rate
-    assert d["db"]["frac"] is None and "rider" in d["db"]["kernel"]      # no launch of its own on the default path
+    assert d["db"]["frac"] is None and "rider" in d["db"]["kernel"]      # no launch of its own on the default path ...
+    own = d["db"]["as_a_kernel_of_its_own"]                              # ... and, for reference, timed as one
+    assert 0 < own["frac"] < 1.2 and own["ms_per_step"] > 0 and own["gemm_dx_ms_per_step_with_rider"] > 0
     for key in ("quantize", "proxy_update"):
         q = d[key]
         assert abs(q["achieved_gbs"] - q["bytes_per_step"] / (q["ms_per_step"] * 1e-3) / 1e9) < 1e-6 * q["achieved_gbs"]
