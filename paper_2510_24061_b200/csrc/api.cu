@@ -316,17 +316,26 @@ namespace {
 // sgd_lr (nullable, host): also run Alg. 3 line 4 in its plain-SGD form and the row scores (into the workspace's score region),
 // inside the dB kernel where its shared memory has the room, else as the separate pass.
 // S5b and S4 of one backward: dB (d) and, when dX is wanted, the input-gradient product (g).  Where the product runs on
-// CTA pairs and d is the plain adapter gradient, dB rides on the product's launch (the pairs its last wave leaves idle);
-// otherwise -- no dX, the optimizer step fused into the dB kernel, FALQON_LAYER_DB_OWN_KERNEL -- dB is a kernel of its own,
-// launched first (g~ was written a moment ago and is still in L2).
-int launch_db_and_dx(const falqon_layer* L, DbFusedProblem& d, GemmProblem* g, cudaStream_t stream) {
+// CTA pairs and d is the adapter gradient without the fused optimizer step, dB rides on the product's launch (the pairs its
+// last wave leaves idle); otherwise -- no dX, the optimizer step fused into the dB kernel, FALQON_LAYER_DB_OWN_KERNEL -- dB is
+// a kernel of its own, launched first (g~ was written a moment ago and is still in L2).
+// oa_todo (nullable): the cast of O_A (S5a) has not run yet (no output-gradient quantizer launch carried it): it rides on
+// the product's launch too where dB does, and is a small kernel of its own otherwise.  sync: 8 bytes, zero between launches.
+int launch_db_and_dx(const falqon_layer* L, DbFusedProblem& d, GemmProblem* g, const OaCastJob* oa_todo, void* sync,
+                     cudaStream_t stream) {
   const bool ride = g != nullptr && (L->flags & FALQON_LAYER_DB_OWN_KERNEL) == 0 && gemm_db_rider_supported(*g, d);
+  if (oa_todo != nullptr && !ride) {
+    StageTimer timer(FALQON_STAGE_QUANT_DY, stream);   // only S5a is left of this stage
+    FALQON_CUDA(launch_oa_cast(*oa_todo, stream));
+  }
   if (!ride) {
     StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
     FALQON_CUDA(launch_db_fused(d, stream));
   }
   if (g != nullptr) {
     g->db_rider = ride ? &d : nullptr;
+    g->oa_rider = ride ? oa_todo : nullptr;
+    g->oa_sync = sync;
     StageTimer timer(FALQON_STAGE_GEMM_DX, stream);
     FALQON_CUDA(launch_gemm_fp8(*g, stream));
   }
@@ -400,16 +409,17 @@ int backward_impl(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, con
   float* inv_sw = reinterpret_cast<float*>(base + w.inv_sw);
   if (per_row)   // the row scales lie on dX's contraction axis: divide them out of dY before its cast
     FALQON_CUDA(launch_scale_table(0, L->s_w, m, r, nullptr, inv_sw, w.inv_sw_len, stream));
+  // S5a rides along: O~_A = Q_e4m3(O_A) with s_OA from the forward's amax, written transposed for the dB product
+  const OaCastJob oa_cast{OA, amax_oa, T, static_cast<int>(r), w.t16, oaq_t, scales + 5, scales + 4};
+  const OaCastJob* oa_todo = amax_dy != nullptr ? &oa_cast : nullptr;   // not carried by the quantizer launch below
+  void* sync_words = base + w.scales + kSyncOffset;
   {
     StageTimer timer(FALQON_STAGE_QUANT_DY, stream);
-    // S5a rides along: O~_A = Q_e4m3(O_A) with s_OA from the forward's amax, written transposed for the dB product
-    const OaCastJob oa_cast{OA, amax_oa, T, static_cast<int>(r), w.t16, oaq_t, scales + 5, scales + 4};
-    if (amax_dy != nullptr) {   // single-pass cast; the O_A cast has no fused launch to ride on and runs by itself
+    if (amax_dy != nullptr) {   // single-pass cast: no grid barrier for the O_A cast to ride on; it goes with dB / dX below
       FALQON_CUDA(launch_cast_per_tensor(dY, dy_dt, T * m, kE5M2, 1.0f, reinterpret_cast<const uint32_t*>(amax_dy), 1, nullptr, gq,
                                          scales + 3, s_g_out, scales + 2, nullptr, stream));
-      FALQON_CUDA(launch_oa_cast(oa_cast, stream));
     } else {
-      FALQON_CUDA(launch_quantize_fused(dY, dy_dt, T * m, kE5M2, gq, partial, base + w.scales + kSyncOffset, scales + 3, s_g_out,
+      FALQON_CUDA(launch_quantize_fused(dY, dy_dt, T * m, kE5M2, gq, partial, sync_words, scales + 3, s_g_out,
                                         scales + 2, nullptr, status, per_row ? inv_sw : nullptr, static_cast<int>(m), &oa_cast,
                                         stream));
     }
@@ -437,6 +447,10 @@ int backward_impl(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, con
     // with a separate optimizer pass the pass must follow dB: it keeps dB in a kernel of its own, before the product
     const bool own_db = sgd_lr != nullptr && !fuse_update;
     if (own_db) {
+      if (oa_todo != nullptr) {
+        StageTimer timer(FALQON_STAGE_QUANT_DY, stream);
+        FALQON_CUDA(launch_oa_cast(*oa_todo, stream));
+      }
       {
         StageTimer timer(FALQON_STAGE_GEMM_DB, stream);
         FALQON_CUDA(launch_db_fused(d, stream));
@@ -450,7 +464,7 @@ int backward_impl(const falqon_layer* L, const void* dY, falqon_dtype dy_dt, con
         FALQON_CUDA(launch_gemm_fp8(g, stream));
       }
     } else {
-      const int rc = launch_db_and_dx(L, d, dX != nullptr ? &g : nullptr, stream);
+      const int rc = launch_db_and_dx(L, d, dX != nullptr ? &g : nullptr, oa_todo, sync_words, stream);
       if (rc != FALQON_OK) return rc;
     }
   }
@@ -488,11 +502,7 @@ int falqon_melded_backward_codes(const falqon_layer* L, const uint8_t* gq, const
   float* scales = reinterpret_cast<float*>(base + w.scales);
   uint8_t* oaq_t = base + w.oaq_t;
   const int64_t m = L->m, n = L->n, r = L->r;
-  {
-    StageTimer timer(FALQON_STAGE_QUANT_DY, stream);   // only S5a is left of this stage
-    const OaCastJob oa_cast{OA, amax_oa, T, static_cast<int>(r), w.t16, oaq_t, scales + 5, scales + 4};
-    FALQON_CUDA(launch_oa_cast(oa_cast, stream));
-  }
+  const OaCastJob oa_cast{OA, amax_oa, T, static_cast<int>(r), w.t16, oaq_t, scales + 5, scales + 4};   // S5a: still to do
   DbFusedProblem d{};
   d.m = m; d.r = r; d.T = T;
   d.gq = gq; d.oaq_t = oaq_t; d.ldt = w.t16; d.s_oa = scales + 5; d.s_g = s_g; d.dB = dB; d.status = status;
@@ -504,7 +514,7 @@ int falqon_melded_backward_codes(const falqon_layer* L, const uint8_t* gq, const
   g.c0 = dX; g.ldc0 = n; g.c0_dt = dx_dt; g.n_split = n;
   g.scale_a = s_g; g.scale_b = L->s_w;
   g.status = status;
-  return launch_db_and_dx(L, d, dX != nullptr ? &g : nullptr, stream);
+  return launch_db_and_dx(L, d, dX != nullptr ? &g : nullptr, &oa_cast, base + w.scales + kSyncOffset, stream);
 }
 
 int falqon_melded_backward_dx(const falqon_layer* L, int64_t T, void* dX, falqon_dtype dx_dt, void* ws, size_t ws_bytes,

@@ -17,7 +17,9 @@
 #include <cstdlib>
 
 #include "gemm_common.cuh"
+#include "grid_sync.cuh"
 #include "internal.h"
+#include "oa_cast.cuh"
 #include "ptx.cuh"
 
 namespace falqon {
@@ -206,10 +208,15 @@ constexpr uint32_t kPairStageBytes = kATileBytes + 128 * kBlockKBytes;   // 32 K
 // far end of the pairs: the last wave of 256 x 256 tiles leaves the highest-numbered pairs idle, and that is where
 // the few microseconds of dB work go -- the launch of a separate kernel (TMEM allocation, two cluster barriers,
 // about 12 us for 2 us of traffic) disappears from the step.  pd: the parameter block of that second problem.
+// oa_job (oa != nullptr): the cast of O_A that dB's B operand needs has not run yet; the epilogue warps of every CTA do it
+// first thing (they have nothing to drain until the first tile is complete), each CTA then counts itself in at oa_sync
+// (two words that are zero between launches), and the producers of the pairs that carry dB tiles wait for the whole
+// grid's count before their first copy of O~_A^T -- tens of microseconds later, so the (bounded) wait never spins.
 template <bool kBMn, bool kRider>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                     const __grid_constant__ CUtensorMap tmap_c, const GemmParams p, const GemmParams pd) {
+                     const __grid_constant__ CUtensorMap tmap_c, const GemmParams p, const GemmParams pd, const OaCastJob oa_job,
+                     GridSync* oa_sync) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t smem_base = (raw_addr + 1023u) & ~1023u;
@@ -291,6 +298,16 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         __syncwarp();
         if (++stage == S) { stage = 0; phase ^= 1u; }
       }
+    }
+    if (kRider && oa_job.oa != nullptr && rider_first < pd.m_tiles && !aborted) {
+      // O~_A^T must be complete, written by every CTA of the grid (all resident: one persistent CTA per SM)
+      const uint64_t t0 = global_timer_ns();
+      while (ld_acquire_gpu(&oa_sync->arrive) < gridDim.x) {
+        __nanosleep(100);
+        if (global_timer_ns() - t0 > kWaitLimitNs) { aborted = true; atomicExch(p.status, kStatusTimeout); break; }
+      }
+      aborted = __any_sync(0xFFFFFFFFu, aborted);
+      fence_proxy_async_global();   // the codes were stored by ordinary stores; the bulk tensor copies below read them
     }
     if (kRider) {   // the tiles of dB, from the far end of the pairs
       const int half_rows = pd.block_n >> 1;                                  // this CTA's rows of O~_A^T (block_n = r16)
@@ -393,6 +410,16 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     // ------------------------------------------------------------ epilogue (warps 2..9 of each CTA)
     const int quad = warp & 3;
     const int col_half = (warp - 2) >> 2;
+    if (kRider && oa_job.oa != nullptr) {   // S5a, while the first tile is on its way
+      cast_oa_transposed(oa_job, warp - 2, static_cast<int>(kEpilogueWarps));
+      __threadfence();
+      fence_proxy_async_global();
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");   // the eight epilogue warps of this CTA
+      if (warp == 2 && lane == 0) {
+        __threadfence();
+        atomicAdd(&oa_sync->arrive, 1u);
+      }
+    }
     uint8_t* stage_out = smem_gen + static_cast<uint32_t>(S) * kPairStageBytes + kBarrierBytes + (warp - 2) * kStageOutBytes;
     const bool rescale = p.scale_a != nullptr;
     const float inv = rescale ? 1.0f / (p.scale_b != nullptr ? ld_stream(p.scale_a) * ld_stream(p.scale_b) : ld_stream(p.scale_a)) : 1.0f;
@@ -416,7 +443,9 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       if (acc == 0) acc_phase ^= 1u;
     }
     if (kRider) {
-      const float inv_db = 1.0f / (ld_stream(pd.scale_a) * ld_stream(pd.scale_b));
+      // (with the cast riding in this launch, s_OA is taken from the absmax it was made from, not from the word another CTA wrote)
+      const float s_oa = oa_job.oa != nullptr ? scale_from_amax(ld_stream(oa_job.amax_oa), kE4M3) : ld_stream(pd.scale_b);
+      const float inv_db = 1.0f / (ld_stream(pd.scale_a) * s_oa);
       uint32_t unused = 0;
       for (int j = rider_first; j < pd.m_tiles && !aborted; j += rider_step) {
         if (!mbar_wait(tmem_full_bar(acc), acc_phase, p.status)) { aborted = true; break; }
@@ -452,6 +481,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     tc_fence_after_sync();
     tmem_dealloc_pair(tmem_base, kTmemCols);
   }
+  if (kRider && oa_job.oa != nullptr && threadIdx.x == 0) grid_depart(oa_sync);   // the last CTA puts the two words back to zero
 }
 
 // ------------------------------------------------------------------ host side
@@ -532,14 +562,15 @@ cudaError_t launch_variant(const CUtensorMap& ta, const CUtensorMap& tb, const G
 
 template <bool kBMn, bool kRider>
 cudaError_t launch_pair_variant(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const GemmParams& gp,
-                                const GemmParams& gd, int grid, size_t smem, cudaStream_t stream) {
+                                const GemmParams& gd, const OaCastJob& oa_job, void* oa_sync, int grid, size_t smem,
+                                cudaStream_t stream) {
   static DeviceMask configured{0};
   {
     const cudaError_t ec = set_max_dynamic_smem(gemm_fp8_pair_kernel<kBMn, kRider>, static_cast<int>(kSmemBudget), configured);
     if (ec != cudaSuccess) return ec;
   }
   return launch_pdl(gemm_fp8_pair_kernel<kBMn, kRider>, dim3(static_cast<unsigned>(grid)), dim3(kGemmThreads), smem, stream, 2,
-                    ta, tb, tc, gp, gd);
+                    ta, tb, tc, gp, gd, oa_job, static_cast<GridSync*>(oa_sync));
 }
 
 bool pair_kernel_disabled() {
@@ -598,10 +629,15 @@ cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
     gd.status = q.status;
     CUtensorMap tc;
     if (!make_tensor_map(&tc, d.oaq_t, r16, d.T, d.ldt, kBlockKBytes, static_cast<uint32_t>(r16 / 2))) return cudaErrorInvalidValue;
-    return launch_pair_variant<true, true>(ta, tb, tc, gp, gd, grid, smem, stream);
+    OaCastJob oa_job{};
+    if (q.oa_rider != nullptr) {
+      if (q.oa_sync == nullptr) return cudaErrorInvalidValue;
+      oa_job = *q.oa_rider;
+    }
+    return launch_pair_variant<true, true>(ta, tb, tc, gp, gd, oa_job, q.oa_sync, grid, smem, stream);
   }
-  if (q.b_mn_major) return launch_pair_variant<true, false>(ta, tb, ta, gp, gp, grid, smem, stream);
-  return launch_pair_variant<false, false>(ta, tb, ta, gp, gp, grid, smem, stream);
+  if (q.b_mn_major) return launch_pair_variant<true, false>(ta, tb, ta, gp, gp, OaCastJob{}, nullptr, grid, smem, stream);
+  return launch_pair_variant<false, false>(ta, tb, ta, gp, gp, OaCastJob{}, nullptr, grid, smem, stream);
 }
 
 }  // namespace
@@ -618,6 +654,7 @@ bool gemm_db_rider_supported(const GemmProblem& q, const DbFusedProblem& d) {
 cudaError_t launch_gemm_fp8(const GemmProblem& q, cudaStream_t stream) {
   if (q.M <= 0 || q.N <= 0 || q.K <= 0) return cudaErrorInvalidValue;
   if (q.db_rider != nullptr && !gemm_db_rider_supported(q, *q.db_rider)) return cudaErrorInvalidValue;
+  if (q.oa_rider != nullptr && q.db_rider == nullptr) return cudaErrorInvalidValue;
   if (q.block_n < 16 || q.block_n > 256 || q.block_n % 16) return cudaErrorInvalidValue;
   if (q.b_mn_major && q.block_n % 128) return cudaErrorInvalidValue;
   // the tensor-bound roles (K-major A, full-width tiles, no token slabs) run on CTA pairs

@@ -135,6 +135,10 @@ struct GemmProblem {
   // nullable: the adapter gradient of the same layer, computed by the same launch on the CTA pairs that the last wave of
   // this product's tiles leaves idle (see gemm_db_rider_supported)
   const DbFusedProblem* db_rider;
+  // nullable, with db_rider only: the cast of O_A that the rider's B operand needs, done by the same launch too (its
+  // epilogue warps, before the first tile is complete); oa_sync: 8 bytes of device memory that are zero between launches
+  const OaCastJob* oa_rider;
+  void* oa_sync;
 };
 cudaError_t launch_gemm_fp8(const GemmProblem& p, cudaStream_t stream);
 // Whether launch_gemm_fp8 can carry d as p.db_rider: p is an input-gradient product on CTA pairs whose A operand is d's

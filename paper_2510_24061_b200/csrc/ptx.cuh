@@ -97,6 +97,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* st
 
 // Makes this thread's earlier writes to shared memory visible to the asynchronous proxy (TMA, tcgen05.mma operands).
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// The same for global memory: between ordinary stores to a tensor and bulk tensor copies (TMA) that read it in the same kernel.
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 
 // The same wait executed by a whole converged warp; the outcome is made warp-uniform.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* status) {

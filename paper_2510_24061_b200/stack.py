@@ -496,10 +496,10 @@ class Stack:
 
     def launches_per_step(self) -> int:
         if self.fuse_cast:
-            # per block: 7 forward products; 7 x (O_A cast, dX product with dB riding on it) + the two single-pass casts of
-            # dg and du; 4 + 5 chain kernels; the proxy update(s); plus the first block's normalisation (the last block's
-            # plain residual sum stands in for a quantizing one)
-            per_block = 7 + 7 * (3 if self.own_db else 2) + 2 + 4 + 5
+            # per block: 7 forward products; 7 dX products with the O_A cast and dB riding on them (each a kernel of its own
+            # with own_db: + 2 per layer) + the two single-pass casts of dg and du; 4 + 5 chain kernels; the proxy update(s);
+            # plus the first block's normalisation (the last block's plain residual sum stands in for a quantizing one)
+            per_block = 7 + 7 * (3 if self.own_db else 1) + 2 + 4 + 5
             if self.batches is None:
                 per_block += 7 * fq.launch_count("falqon_proxy_update", k=self.k)
             else:
@@ -510,9 +510,9 @@ class Stack:
             shared = name in ("k", "v", "up")
             per_block += (1 if shared else fq.launch_count("falqon_melded_forward"))   # codes: the product alone
             if name in ("k", "v"):
-                per_block += 3 if self.own_db else 2            # on q's gradient codes: O_A cast, dX (dB rides on it)
-            else:
-                per_block += fq.launch_count("falqon_melded_backward" + (":own_db" if self.own_db else "")) + (1 if self.producer_amax else 0)   # + the O_A cast
+                per_block += 3 if self.own_db else 1            # on q's gradient codes: dX, with the O_A cast and dB riding on it
+            else:                                               # cast, dX (with own_db: + dB, + the O_A cast after a single-pass cast)
+                per_block += fq.launch_count("falqon_melded_backward" + (":own_db" if self.own_db else "")) + (1 if self.producer_amax and self.own_db else 0)
             if self.batches is None:
                 per_block += fq.launch_count("falqon_proxy_update", k=self.k)
         if self.batches is not None:

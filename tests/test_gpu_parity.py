@@ -422,6 +422,9 @@ def test_backward_on_shared_gradient_codes(fq, orc):
     s_g = fq.ws_view(L1, ws1, T, fq.WS_SCALES).view(torch.float32)[3:4]
     dX, dB = fq.melded_backward_codes(L2, gq, s_g, OA2, am2, dx_dtype=torch.float32, ws=ws2)
     assert torch.equal(dX.view(torch.int32), dX_ref.view(torch.int32)) and torch.equal(dB.view(torch.int32), dB_ref.view(torch.int32))
+    # (here the O_A cast ran inside the product's launch, synchronised through two control words of the workspace: they
+    # are back at zero, and O~_A^T is what the output-gradient quantizer's rider wrote in the reference call)
+    assert int(ws2[256:264].view(torch.int32).abs().sum()) == 0
     # (without dX, dB is a kernel of its own that sums token slabs: the same numbers in another order of the fp32 sums)
     _, dB_only = fq.melded_backward_codes(L2, gq, s_g, OA2, am2, need_dx=False, ws=ws2)
     assert float((dB_only - dB_ref).abs().max()) <= 2e-6 * float(dB_ref.abs().max())
