@@ -461,3 +461,49 @@ def test_column_scaled_cast_of_bf16_gradients_in_every_chunk_geometry(fq, orc, m
     assert bits32(f32(s_g))[0] == bits32(s_g_o)
     assert np.array_equal(u8(fq.ws_view(layer, ws, T, fq.WS_GQ))[: T * m].reshape(T, m), gq_o)
     assert fq.last_device_status() == 0
+
+
+@pytest.mark.parametrize("m,n,r,T", [
+    (16, 16, 8, 16),            # the smallest layer: one pair, one tile of dB with 16 valid rows, 8 of 16 instruction columns
+    (400, 272, 24, 333),        # two dB tiles, the second partial; r16 = 32 > r; fewer product tiles than SM pairs
+    (4112, 64, 256, 130),       # 17 dB tiles of the widest rank behind ONE product tile: every pair takes some
+    (28688, 128, 8, 1000),      # 113 dB tiles, more than there are pairs: round robin over all of them
+    (1024, 4096, 64, 2049),     # tokens one past a k-block; the product has a partial last wave (8 x 16 tiles)
+])
+@pytest.mark.parametrize("per_row", [False, True])
+def test_adapter_gradient_riding_on_the_input_gradient_product(fq, orc, m, n, r, T, per_row):
+    """dB computed inside the launch of the input-gradient product (the default) against the oracle on the GPU's own
+    codes, against dB from the kernel of its own (same numbers in another summation order), and dX unchanged by the rider;
+    once after the fused quantizer (which carries the O_A cast) and once with a known absmax (the O_A cast rides in the
+    product's launch too).  Shapes at the corners of the rider's tiling."""
+    W = synth.backbone(51, 0, m, n, DEV, heavy_tailed=per_row)
+    A, B = synth.adapter_a(51, 0, r, n, DEV), synth.adapter_b(51, 0, m, r, DEV)
+    X = synth.activations(51, 0, T, n, 1, DEV)
+    dY = synth.out_grad(51, 0, 0, T, m, DEV)
+    ride = fq.setup_layer(W, A, B, 1.0, per_row=per_row)
+    own = fq.Layer(ride.wq, ride.s_w, ride.dbuf, r, flags=fq.LAYER_DB_OWN_KERNEL)
+    ws = ride.workspace(T)
+    _, OA, amax_oa, _ = fq.melded_forward(ride, X, ws=ws)
+    dX0, dB0, s_g0 = fq.melded_backward(own, dY, OA, amax_oa, dx_dtype=torch.float32, ws=ws)
+    dX0, dB0 = dX0.clone(), dB0.clone()
+    oaq0 = fq.ws_view(ride, ws, T, fq.WS_OAQ_T).clone()
+    fq.ws_view(ride, ws, T, fq.WS_OAQ_T).fill_(0x7F)           # NaN codes: whoever multiplies stale O~_A shows it
+    dX1, dB1, s_g1 = fq.melded_backward(ride, dY, OA, amax_oa, dx_dtype=torch.float32, ws=ws)
+    assert torch.equal(dX0.view(torch.int32), dX1.view(torch.int32)) and torch.equal(s_g0, s_g1)
+    scale = float(dB0.abs().max())
+    assert float((dB1 - dB0).abs().max()) <= 4e-6 * scale
+    s_w = f32(ride.s_w)
+    gq = u8(fq.ws_view(ride, ws, T, fq.WS_GQ))[: T * m].reshape(T, m)
+    oaq_o, s_oa_o, _ = orc.quantize(f32(OA), orc.E4M3)
+    dB_o = orc.db_gemm(gq, np.float32(f32(s_g1)[0]), oaq_o, s_oa_o, row_scale=s_w[:m] if per_row else None)
+    assert product_close(f32(dB1), dB_o, GEMM_TOL)
+    if not per_row:     # known absmax of dY: a single-pass cast, and the O_A cast inside the product's launch
+        amax_dy = dY.float().abs().max().reshape(1)
+        fq.ws_view(ride, ws, T, fq.WS_OAQ_T).fill_(0x7F)
+        dX2, dB2, s_g2 = fq.melded_backward(ride, dY, OA, amax_oa, dx_dtype=torch.float32, ws=ws, amax_dy=amax_dy)
+        assert torch.equal(dX2.view(torch.int32), dX0.view(torch.int32)) and torch.equal(dB2.view(torch.int32), dB1.view(torch.int32))
+        got = fq.ws_view(ride, ws, T, fq.WS_OAQ_T)
+        t16 = got.numel() // ((r + 15) // 16 * 16)
+        assert torch.equal(got.view(-1, t16)[:r, :T], oaq0.view(-1, t16)[:r, :T])      # the codes the quantizer's rider wrote
+        assert int(ws[256:264].view(torch.int32).abs().sum()) == 0
+    assert fq.last_device_status() == 0
