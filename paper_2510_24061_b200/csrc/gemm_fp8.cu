@@ -267,11 +267,19 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   const int pair = blockIdx.x >> 1;
   const int total_tiles = p.m_tiles * p.n_tiles;   // m_tiles counts 256-row pair tiles here
   bool aborted = false;
-  // rider: the pairs without a tile in the product's last wave (the highest-numbered ones) share the tiles of dB among
-  // themselves, round robin from the far end; the others take none
+  // rider: which tiles of dB this pair computes after its own tiles of the product.  The pairs without a tile in the
+  // product's last wave (the highest-numbered ones) take up to pd.n_tiles each, round robin from the far end -- that many
+  // fit into the time the others spend on their last tile (the host's estimate) -- and what is left goes round robin to
+  // all pairs, lowest-numbered first.  The same list in all three roles.
   const int last_wave = total_tiles % num_pairs;
-  const int rider_step = last_wave == 0 ? num_pairs : num_pairs - last_wave;             // number of such pairs
-  const int rider_first = (num_pairs - 1 - pair) < rider_step ? (num_pairs - 1 - pair) : 0x7FFFFFF0;   // this pair's first dB tile
+  const int idle_pairs = last_wave == 0 ? num_pairs : num_pairs - last_wave;
+  const int idle_rank = num_pairs - 1 - pair;
+  const int rider_block1 = kRider ? min(pd.m_tiles, idle_pairs * pd.n_tiles) : 0;
+  const int rider_n1 = (kRider && idle_rank < idle_pairs && idle_rank < rider_block1) ? (rider_block1 - idle_rank + idle_pairs - 1) / idle_pairs : 0;
+  const int rider_rest = kRider ? pd.m_tiles - rider_block1 : 0;
+  const int rider_n2 = pair < rider_rest ? (rider_rest - pair + num_pairs - 1) / num_pairs : 0;
+  const int rider_count = rider_n1 + rider_n2;
+  auto rider_tile = [&](int i) { return i < rider_n1 ? idle_rank + i * idle_pairs : rider_block1 + pair + (i - rider_n1) * num_pairs; };
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (warp 0 of each CTA; one lane issues)
@@ -299,7 +307,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         if (++stage == S) { stage = 0; phase ^= 1u; }
       }
     }
-    if (kRider && oa_job.oa != nullptr && rider_first < pd.m_tiles && !aborted) {
+    if (kRider && oa_job.oa != nullptr && rider_count > 0 && !aborted) {
       // O~_A^T must be complete, written by every CTA of the grid (all resident: one persistent CTA per SM)
       const uint64_t t0 = global_timer_ns();
       while (ld_acquire_gpu(&oa_sync->arrive) < gridDim.x) {
@@ -312,7 +320,8 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     if (kRider) {   // the tiles of dB, from the far end of the pairs
       const int half_rows = pd.block_n >> 1;                                  // this CTA's rows of O~_A^T (block_n = r16)
       const uint32_t rider_bytes = kATileBytes + static_cast<uint32_t>(half_rows) * kBlockKBytes;
-      for (int j = rider_first; j < pd.m_tiles && !aborted; j += rider_step) {
+      for (int ri = 0; ri < rider_count && !aborted; ++ri) {
+        const int j = rider_tile(ri);
         const int mcol0 = j * 256 + static_cast<int>(rank) * kBlockM;        // first of this CTA's 128 rows of dB
         for (int kb = 0; kb < pd.kblocks_total; ++kb) {
           if (!mbar_wait_warp(empty_bar(stage), phase ^ 1u, p.status)) { aborted = true; break; }
@@ -380,7 +389,8 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         const uint64_t rb_desc0 = make_smem_desc(smem_base + kATileBytes, 16, 1024);     // K-major
         constexpr uint32_t kRaStep = (kUmmaK * 128) >> 4;   // 32 tokens further down the tile
         constexpr uint32_t kRbStep = kUmmaK >> 4;
-        for (int j = rider_first; j < pd.m_tiles && !aborted; j += rider_step) {
+        for (int ri = 0; ri < rider_count && !aborted; ++ri) {
+        const int j = rider_tile(ri);
           if (!mbar_wait_warp(tmem_empty_bar(acc), acc_phase ^ 1u, p.status)) { aborted = true; break; }
           tc_fence_after_sync();
           const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc) * kAccCols;
@@ -447,7 +457,8 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       const float s_oa = oa_job.oa != nullptr ? scale_from_amax(ld_stream(oa_job.amax_oa), kE4M3) : ld_stream(pd.scale_b);
       const float inv_db = 1.0f / (ld_stream(pd.scale_a) * s_oa);
       uint32_t unused = 0;
-      for (int j = rider_first; j < pd.m_tiles && !aborted; j += rider_step) {
+      for (int ri = 0; ri < rider_count && !aborted; ++ri) {
+        const int j = rider_tile(ri);
         if (!mbar_wait(tmem_full_bar(acc), acc_phase, p.status)) { aborted = true; break; }
         tc_fence_after_sync();
         const int row = j * 256 + static_cast<int>(rank) * kBlockM + quad * 32 + lane;      // row of dB
@@ -618,8 +629,19 @@ cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
     gd.M = static_cast<int>(d.m); gd.N = static_cast<int>(d.r); gd.K = static_cast<int>(d.T);
     gd.block_n = r16;
     gd.m_tiles = static_cast<int>((d.m + 255) / 256);
-    gd.n_tiles = 1;
     gd.kblocks_total = static_cast<int>((d.T + kBlockKBytes - 1) / kBlockKBytes);
+    {
+      // n_tiles carries the quota of the pairs that idle in the product's last wave: how many tiles of dB (bound by the
+      // copies: about 0.17 us per k-block) fit into one tile of the product (bound by the MMAs: about 0.47 us per k-block;
+      // both measured), at least one, and no more than an even share of the tiles
+      const long long last_wave = total_tiles % pairs;
+      const long long idle = last_wave == 0 ? pairs : pairs - last_wave;
+      long long cap = static_cast<long long>(2.75 * gp.kblocks_total / gd.kblocks_total);
+      const long long share = (gd.m_tiles + idle - 1) / idle;
+      if (cap > share) cap = share;
+      if (cap < 1) cap = 1;
+      gd.n_tiles = static_cast<int>(cap);
+    }
     gd.num_stages = stages;
     // fp32 accumulate, A = the product's own A format read MN-major, B = E4M3 K-major, N = r16, M = 256
     gd.idesc = (1u << 4) | (static_cast<uint32_t>(q.a_fmt) << 7) | (static_cast<uint32_t>(kE4M3) << 10) | (1u << 15) |
