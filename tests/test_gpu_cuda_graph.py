@@ -99,3 +99,42 @@ def test_the_benchmarks_graph_replay_equals_call_by_call_at_full_size():
             assert torch.equal(a["out_f"][0], b["out_f"][0]) and torch.equal(a["out_b"][0], b["out_b"][0]), f"{a['name']}: Y / dX"
             assert torch.equal(a["idx"], b["idx"]), f"{a['name']}: selected rows"
     assert fq.last_device_status() == 0
+
+
+def test_a_captured_stack_step_replays_bit_for_bit():
+    """The same for the chained stack in its default form: chain kernels that cast their own results (cooperative launches
+    with a grid barrier), products that carry the adapter gradient and the O_A cast, one batched proxy update per block --
+    two steps as replays of one captured graph against two steps run call by call on a twin stack."""
+    from paper_2510_24061_b200 import binding as fq
+    from paper_2510_24061_b200 import stack as st
+    H, F, T, r, k = 256, 512, 300, 16, 24
+    h0 = synth.normal_bf16(5, 9001, (T, H), 1.0, DEV)
+    G = synth.normal_bf16(5, 9002, (T, H), 1.0e-2, DEV)
+    eager = st.Stack(2, H, F, T, r, k, seed=5, device=DEV, lr=2e-2)
+    graphed = st.Stack(2, H, F, T, r, k, seed=5, device=DEV, lr=2e-2)
+    assert eager.fuse_cast and graphed.fuse_cast
+    state = [(L.wq.clone(), L.dbuf.clone()) for blk in graphed.layers for L in blk.values()]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):          # warm-up (kernel attributes are set on first use) ...
+        graphed.step(h0, G)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    for L, (wq, dbuf) in zip([L for blk in graphed.layers for L in blk.values()], state):   # ... and its effect undone
+        L.wq.copy_(wq)
+        L.dbuf.copy_(dbuf)
+    graphed.steps_done = 0
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        graphed.step(h0, G)
+    for _ in range(2):
+        g.replay()
+        eager.step(h0, G)
+    torch.cuda.synchronize()
+    assert torch.equal(graphed.h_out.view(torch.int16), eager.h_out.view(torch.int16))
+    assert torch.equal(graphed.dh.view(torch.int16), eager.dh.view(torch.int16))
+    for bg, be in zip(graphed.layers, eager.layers):
+        for name in bg:
+            assert torch.equal(bg[name].wq, be[name].wq), name
+            assert torch.equal(bg[name].dbuf.view(torch.int32), be[name].dbuf.view(torch.int32)), name
+    assert fq.last_device_status() == 0
