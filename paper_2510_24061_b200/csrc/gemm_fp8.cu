@@ -10,7 +10,8 @@
 // The accumulator is double buffered (2 x 256 TMEM columns), so the epilogue of tile i overlaps the
 // main loop of tile i+1.  A is K-major (rows along K); B may be K-major or MN-major (rows along N): the
 // melded forward reads both K-major, the input gradient reads W~ MN-major (no transposed copy of the
-// backbone exists).  (The adapter gradient, which reads the output gradient MN-major, has its own kernel.)
+// backbone exists).  The adapter gradient, which reads the output gradient MN-major, rides on the CTA-pair form of the
+// input-gradient product (see gemm_fp8_pair_kernel) or runs as a kernel of its own (gemm_db.cu).
 // Every mbarrier wait is bounded; on a timeout the CTA records it, drains and frees its TMEM.
 #include <cuda.h>
 
