@@ -98,8 +98,8 @@ typedef struct {
  *  FALQON_LAYER_DB_OWN_KERNEL  By default the adapter gradient (Eq. lora_backward_modified) of a call whose dX is
  *      requested is computed inside the launch of the input-gradient product, on the SM pairs that the product's last wave
  *      of tiles leaves idle: one accumulation over all tokens per element, in token order.  With this flag (and always for
- *      calls without dX and for falqon_melded_backward_update) dB is a kernel of its own that sums four token slabs in slab
- *      order.  Both are deterministic; they differ in the last bits of dB. */
+ *      calls without dX, and for falqon_melded_backward_update at ranks above 128) dB is a kernel of its own that sums four
+ *      token slabs in slab order.  Both are deterministic; they differ in the last bits of dB. */
 typedef enum { FALQON_LAYER_FUSED_CAST = 1, FALQON_LAYER_EMIT_XQ = 2, FALQON_LAYER_DB_OWN_KERNEL = 4 } falqon_layer_flag;
 
 /* Names of the regions inside the workspace that hold staged intermediates of the last call
@@ -254,8 +254,9 @@ int falqon_proxy_update(const falqon_layer *L, const float *dB, float lr, int64_
 /* Alg. 3 lines 3-4 in one call: falqon_melded_backward (or, with amax_dy non-NULL, falqon_melded_backward_amax) followed
  * by the plain-SGD step on the DeltaBuffer and the row scores,
  *     DeltaBuffer <- fma(-lr, dB, DeltaBuffer);   score_i = sum_j |DeltaBuffer[i][j]|  (fp32, j ascending),
- * both computed where dB is produced (the adapter-gradient kernel's slab-sum phase holds whole rows of dB), so the
- * DeltaBuffer and dB are not read again by a pass of their own.  The scores are left in FALQON_WS_SCORE.  Bit for bit the
+ * both computed where dB is produced -- in the epilogue of the dB tiles that ride on the input-gradient product's launch
+ * (ranks up to 128, dX requested), else in the adapter-gradient kernel's slab-sum phase: either holds whole rows of dB --
+ * so the DeltaBuffer and dB are not read again by a pass of their own.  The scores are left in FALQON_WS_SCORE.  Bit for bit the
  * DeltaBuffer and scores that falqon_melded_backward + falqon_proxy_update(dB, lr, k = 0) produce.  Mutates L->dbuf.
  * dB (device [m][r] fp32) is still written.  Follow it with falqon_proxy_update_scored on the same workspace.
  * (Where the kernel's shared memory has no room for the fused step -- ranks near 256 with few token slabs -- the same

@@ -316,9 +316,9 @@ namespace {
 // sgd_lr (nullable, host): also run Alg. 3 line 4 in its plain-SGD form and the row scores (into the workspace's score region),
 // inside the dB kernel where its shared memory has the room, else as the separate pass.
 // S5b and S4 of one backward: dB (d) and, when dX is wanted, the input-gradient product (g).  Where the product runs on
-// CTA pairs and d is the adapter gradient without the fused optimizer step, dB rides on the product's launch (the pairs its
-// last wave leaves idle); otherwise -- no dX, the optimizer step fused into the dB kernel, FALQON_LAYER_DB_OWN_KERNEL -- dB is
-// a kernel of its own, launched first (g~ was written a moment ago and is still in L2).
+// CTA pairs, dB rides on the product's launch (the pairs its last wave leaves idle), with the optimizer step and the row
+// scores if d asks for them; otherwise -- no dX, a fused optimizer step at a rank above 128, FALQON_LAYER_DB_OWN_KERNEL -- dB
+// is a kernel of its own, launched first (g~ was written a moment ago and is still in L2).
 // oa_todo (nullable): the cast of O_A (S5a) has not run yet (no output-gradient quantizer launch carried it): it rides on
 // the product's launch too where dB does, and is a small kernel of its own otherwise.  sync: 8 bytes, zero between launches.
 int launch_db_and_dx(const falqon_layer* L, DbFusedProblem& d, GemmProblem* g, const OaCastJob* oa_todo, void* sync,
@@ -915,7 +915,9 @@ int falqon_launch_count(const char* entry_point, int64_t m, int64_t n, int64_t r
   if (std::strcmp(entry_point, "falqon_melded_backward:fused") == 0) return 5;
   if (std::strcmp(entry_point, "falqon_proxy_update") == 0) return k > 0 ? 2 : 1;  // optimizer+score+top-k, merge+clear
   if (std::strcmp(entry_point, "falqon_proxy_update_batched") == 0) return k > 0 ? 2 : 1;   // per 8 layers
-  if (std::strcmp(entry_point, "falqon_melded_backward_update") == 0) return 3;   // as the backward; the update rides in the dB kernel
+  // as the backward: the optimizer step and the scores ride with dB (inside the dX launch, or in the dB kernel)
+  if (std::strcmp(entry_point, "falqon_melded_backward_update") == 0) return 2;
+  if (std::strcmp(entry_point, "falqon_melded_backward_update:own_db") == 0) return 3;
   if (std::strcmp(entry_point, "falqon_proxy_update_scored") == 0) return k > 0 ? 2 : 0;
   if (std::strcmp(entry_point, "falqon_proxy_update_scored_batched") == 0) return k > 0 ? 2 : 0;
   if (std::strcmp(entry_point, "falqon_proxy_update_static") == 0) return k > 0 ? 4 : 1;   // optimizer+score, top-k, merge, clear (+ one copy of idx)

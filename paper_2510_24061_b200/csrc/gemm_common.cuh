@@ -38,6 +38,9 @@ struct GemmParams {
   const float* scale_a; const float* scale_b;
   const float* col_scale;
   const float* row_scale;   // nullable, used by the adapter-gradient rider only: output row i is also multiplied by row_scale[i]
+  // nullable (together), the rider only: DeltaBuffer <- fma(neg_lr, dB, DeltaBuffer) on the rows it has just computed (Alg. 3
+  // line 4, plain SGD), and score[i] = sum_j |DeltaBuffer[i][j]| in fp32, j ascending
+  float* dbuf; float* score; float neg_lr;
   int* status;
 };
 

@@ -466,7 +466,44 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         const uint32_t t_row = tmem_base + static_cast<uint32_t>(acc) * kAccCols + (static_cast<uint32_t>(quad * 32) << 16);
         // (per-row-scaled backbone: row i of dB is multiplied back by s_w[i], one rounded product of the two factors)
         const float inv_row = pd.row_scale != nullptr && row < pd.M ? __fmul_rn(inv_db, ld_stream(pd.row_scale + row)) : inv_db;
-        epilogue_tile(pd, t_row, row, row < pd.M, 0, col_half ? 128 : 0, col_half ? 256 : 128, inv_row, unused, stage_out);
+        if (pd.dbuf == nullptr) {
+          epilogue_tile(pd, t_row, row, row < pd.M, 0, col_half ? 128 : 0, col_half ? 256 : 128, inv_row, unused, stage_out);
+        } else if (col_half == 0) {
+          // with the optimizer step (r <= 128: this warp's lanes hold whole rows): dB as above, then one fma per element on
+          // the value dB holds, and the row's score accumulated strictly left to right -- what the stand-alone kernels do
+          const bool ok = row < pd.M;
+          float sc = 0.0f;
+          for (int c0 = 0; c0 < pd.N; c0 += 32) {
+            uint32_t v[32];
+            __syncwarp();
+            tmem_ld_32x32b_x32(t_row + static_cast<uint32_t>(c0), v);
+            tmem_ld_wait();
+            if (ok) {
+              const long long off = static_cast<long long>(row) * pd.ldc0 + c0;
+              float4* drow = reinterpret_cast<float4*>(pd.dbuf + off);
+              float4* grow = pd.c0 != nullptr ? reinterpret_cast<float4*>(static_cast<float*>(pd.c0) + off) : nullptr;
+              float4 d[8];
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                if (c0 + 4 * q < pd.N) d[q] = ld_stream(drow + q);
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                if (c0 + 4 * q < pd.N) {      // r is a multiple of 8: a group of four is all inside or all outside
+                  const float4 g = make_float4(__fmul_rn(__uint_as_float(v[4 * q]), inv_row), __fmul_rn(__uint_as_float(v[4 * q + 1]), inv_row),
+                                               __fmul_rn(__uint_as_float(v[4 * q + 2]), inv_row), __fmul_rn(__uint_as_float(v[4 * q + 3]), inv_row));
+                  if (grow != nullptr) grow[q] = g;
+                  float4 e = d[q];
+                  e.x = __fmaf_rn(pd.neg_lr, g.x, e.x); e.y = __fmaf_rn(pd.neg_lr, g.y, e.y);
+                  e.z = __fmaf_rn(pd.neg_lr, g.z, e.z); e.w = __fmaf_rn(pd.neg_lr, g.w, e.w);
+                  drow[q] = e;
+                  sc = __fadd_rn(sc, fabsf(e.x)); sc = __fadd_rn(sc, fabsf(e.y));
+                  sc = __fadd_rn(sc, fabsf(e.z)); sc = __fadd_rn(sc, fabsf(e.w));
+                }
+              }
+            }
+          }
+          if (ok) pd.score[row] = sc;
+        }
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(map_to_cta(tmem_empty_bar(acc), 0));
@@ -649,6 +686,7 @@ cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
                (static_cast<uint32_t>(r16 >> 3) << 17) | (static_cast<uint32_t>(256 >> 4) << 24);
     gd.c0 = d.dB; gd.ldc0 = d.r; gd.c0_dt = kF32; gd.n_split = static_cast<int>(d.r);
     gd.scale_a = d.s_g; gd.scale_b = d.s_oa; gd.row_scale = d.row_mul;
+    gd.dbuf = d.dbuf; gd.score = d.score; gd.neg_lr = d.neg_lr;
     gd.status = q.status;
     CUtensorMap tc;
     if (!make_tensor_map(&tc, d.oaq_t, r16, d.T, d.ldt, kBlockKBytes, static_cast<uint32_t>(r16 / 2))) return cudaErrorInvalidValue;
@@ -667,10 +705,12 @@ cudaError_t launch_gemm_fp8_pair(const GemmProblem& q, cudaStream_t stream) {
 
 bool gemm_db_rider_supported(const GemmProblem& q, const DbFusedProblem& d) {
   // the product must run on CTA pairs with an MN-major B (the input-gradient product), its A must be the rider's g~
-  // ([T][m], the rider's rows on the product's contraction axis), and the rider must be dB without the fused optimizer step
+  // ([T][m], the rider's rows on the product's contraction axis); with the optimizer step fused, a warp must hold whole rows
+  // of dB (r <= 128)
   return q.block_n == 256 && q.N % 16 == 0 && !pair_kernel_disabled() && q.b_mn_major && q.a != nullptr && q.a == d.gq &&
-         q.M == d.T && q.K == d.m && q.lda == d.m && d.m % 16 == 0 && d.r >= 8 && d.r <= 256 && d.r % 8 == 0 && d.dB != nullptr &&
-         d.dbuf == nullptr && d.score == nullptr && d.oaq_t != nullptr && d.s_g != nullptr &&
+         q.M == d.T && q.K == d.m && q.lda == d.m && d.m % 16 == 0 && d.r >= 8 && d.r <= 256 && d.r % 8 == 0 &&
+         ((d.dbuf == nullptr && d.score == nullptr && d.dB != nullptr) || (d.dbuf != nullptr && d.score != nullptr && d.r <= 128)) &&
+         d.oaq_t != nullptr && d.s_g != nullptr &&
          d.s_oa != nullptr && (q.a_fmt == kE5M2) == !d.g_is_e4m3;
 }
 

@@ -142,7 +142,7 @@ struct GemmProblem {
 };
 cudaError_t launch_gemm_fp8(const GemmProblem& p, cudaStream_t stream);
 // Whether launch_gemm_fp8 can carry d as p.db_rider: p is an input-gradient product on CTA pairs whose A operand is d's
-// g~, and d is the adapter gradient without the fused optimizer step.
+// g~ (and, with the optimizer step fused into d, r <= 128).
 bool gemm_db_rider_supported(const GemmProblem& p, const DbFusedProblem& d);
 
 // ---- gemm_fp8_fused.cu: the same product on CTA pairs with the cast of the A operand fused into the producer.  A arrives

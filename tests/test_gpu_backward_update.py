@@ -14,7 +14,7 @@ DEV = "cuda:0"
 
 
 def _twin(fq, layer):
-    return fq.Layer(layer.wq.clone(), layer.s_w.clone(), layer.dbuf.clone(), layer.r)
+    return fq.Layer(layer.wq.clone(), layer.s_w.clone(), layer.dbuf.clone(), layer.r, flags=layer.flags)
 
 
 @pytest.mark.parametrize("m,n,r,T,k,per_row,lr", [
@@ -24,7 +24,8 @@ def _twin(fq, layer):
     (528, 384, 256, 130, 40, False, 2e-2),       # rank 256 with two token blocks: no room in shared memory, separate pass
     (384, 512, 32, 700, 25, True, 2e-2),         # per-row-scaled backbone: dB rows are multiplied back by s_w[i] first
 ])
-def test_backward_update_and_scored_proxy_update(m, n, r, T, k, per_row, lr):
+@pytest.mark.parametrize("own_kernel", [False, True])
+def test_backward_update_and_scored_proxy_update(m, n, r, T, k, per_row, lr, own_kernel):
     from paper_2510_24061_b200 import binding as fq
     from oracle import falqon_oracle as orc
     W, A, B, X = layer_inputs(41, 1, m, n, r, T, 3, DEV)
@@ -32,7 +33,10 @@ def test_backward_update_and_scored_proxy_update(m, n, r, T, k, per_row, lr):
         W = synth.backbone(41, 1, m, n, DEV, heavy_tailed=True)
     dY = synth.out_grad(41, 1, 0, T, m, DEV)
     ref = fq.setup_layer(W, A, B, 1.0, per_row=per_row)
-    ref.flags = fq.LAYER_DB_OWN_KERNEL      # the fused step lives in the adapter-gradient kernel: the reference uses that kernel too
+    # the step and the scores ride with dB inside the dX launch, or (own_kernel, and always at ranks above 128) live in the
+    # adapter-gradient kernel: the reference computes dB the same way, so that the two sequences see the same bits
+    if own_kernel or r > 128:
+        ref.flags = fq.LAYER_DB_OWN_KERNEL
     ref.dbuf.copy_(synth.normal_bf16(41, 90, (m, r), 1e-3, DEV).float())      # something for the step to accumulate onto
     new = _twin(fq, ref)
     ws_r, ws_n = ref.workspace(T), new.workspace(T)
